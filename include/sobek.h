@@ -1,0 +1,183 @@
+/*
+ * sobek.h -- C ABI of the streaming edge-conditioned tensor-product convolution
+ * (fully connected `uvw` multiplicity mixing) for NVIDIA B200 (sm_100a).
+ *
+ * The operator (Eq. standard_tpconv_background with W = phi A, Eq. edge_weight_shape;
+ * the radial projection A is called R here):
+ *
+ *     y_i = sum_{j in N(i)} sum_pi sum_{u,w} ( sum_q phi_ij[q] R[q,pi,u,w] ) *
+ *                 sum_{m_in,m_sh} c^pi[m_in,m_sh,m_out] x_j[pi,u,m_in] Y_ij[pi,m_sh]
+ *
+ * evaluated in the receiver-factorised streaming order (Eqs. angular_path_contraction,
+ * receiver_state, receiver_mixing): each edge's CG coupling is scaled by phi_ij and
+ * folded into a bounded per-receiver state Z_i, and Z_i is contracted with R.  No
+ * array with |E| x N_w or |E| x C_out elements is ever formed, in any order of
+ * differentiation.
+ *
+ * Conventions
+ *   - All array arguments of the sobek_conv_* / sobek_graph_prepare calls are DEVICE
+ *     pointers owned by the caller and must stay valid until the work queued on
+ *     `stream` (a cudaStream_t passed as void*; NULL = default stream) has finished.
+ *     Plan handles and descriptor arrays are HOST memory.
+ *   - fp32 data, row-major.  Node features x[N,C_x], y/gy/ggy[N,C_y] use the `ir_mul`
+ *     layout (Section "Generated deterministic runtime and execution contracts"):
+ *     irrep blocks in descriptor order; inside a block the index is m*mult + u with
+ *     m = 0..2l (standing for -l..l).  Y, gY, vY, hY are [E,(l_max+1)^2], l-major.
+ *     phi, gphi, vphi, hphi are [E,K].  R, gR, vR, hR are [K,N_w] with column
+ *     w_off(pi) + u*C_out(pi) + w; paths pi are numbered in nested order (input
+ *     irrep, SH order, output irrep).
+ *   - Real spherical-harmonic basis with sine-type components at m < 0 (l = 1 is
+ *     (y,z,x)); c^pi = sqrt(2 l_out+1) x (unit-norm real 3j tensor whose first nonzero
+ *     entry in lexicographic (m_in,m_sh,m_out) order is positive).
+ *   - Graph: receiver-sorted CSR.  Edge e in [row_ptr[i], row_ptr[i+1]) runs from
+ *     sender col[e] to receiver i; the order inside a row is the caller's and is kept.
+ *     Empty rows, self loops and duplicate edges are legal.
+ *   - Every entry point returns 0 on success or a negative sobek_status.  Nothing
+ *     throws.  The sobek_conv_* calls never allocate device memory and never
+ *     synchronise: they only enqueue kernels on `stream`.  Results are bitwise
+ *     reproducible from run to run (fixed reduction order, no floating-point atomics).
+ *   - Outputs are overwritten, never accumulated into.  A NULL output pointer means
+ *     "not wanted"; a NULL direction pointer in sobek_conv_dbwd means zero.
+ */
+#ifndef SOBEK_H_
+#define SOBEK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SOBEK_OK = 0,
+    SOBEK_ERR_INVALID_ARG = -1,    /* null pointer, negative size, bad descriptor            */
+    SOBEK_ERR_UNSUPPORTED = -2,    /* l above the supported maximum, no valid path, ...     */
+    SOBEK_ERR_WORKSPACE = -3,      /* workspace missing, misaligned or too small            */
+    SOBEK_ERR_GRAPH = -4,          /* row_ptr not monotone / col out of range               */
+    SOBEK_ERR_NEED_TRANSPOSE = -5, /* gx / hx wanted but src_ptr / src_perm are NULL        */
+    SOBEK_ERR_CUDA = -6,           /* a CUDA runtime call or a launch failed                */
+    SOBEK_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait gave up                    */
+} sobek_status;
+
+/* One irrep block of a feature vector: `mul` copies of order l with parity +1 (e) / -1 (o). */
+typedef struct {
+    int32_t mul;
+    int32_t l;
+    int32_t parity;
+} sobek_irrep;
+
+typedef struct sobek_plan sobek_plan; /* opaque; host-owned; immutable after creation */
+
+enum { SOBEK_MAX_L = 4 };
+
+/*
+ * sobek_plan_create -- the static contract of one layer (Section "Generated
+ * deterministic runtime and execution contracts"): enumerates the paths allowed by the
+ * selection rules (Eq. cg_selection_rules) for spherical harmonics 1 x l, parity (-1)^l,
+ * l = 0..l_max, computes the real Clebsch-Gordan tensors and uploads the sparse tables to
+ * the current CUDA device (the only device allocation the library ever makes; it is
+ * released by sobek_plan_destroy).  `in`/`out` are host arrays.  K >= 1 is the width of
+ * the radial embedding.  `flags` must be 0.
+ * Errors: INVALID_ARG (null, mul < 1, parity not +-1, K < 1), UNSUPPORTED (l or l_max >
+ * SOBEK_MAX_L, or no valid path), CUDA.
+ */
+int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
+                      int l_max, int K, uint32_t flags, sobek_plan** plan);
+void sobek_plan_destroy(sobek_plan* plan);
+
+typedef struct {
+    int32_t C_x;     /* flattened input width  (Eq. flattened_feature_dimension) */
+    int32_t C_y;     /* flattened output width                                   */
+    int32_t dim_sh;  /* (l_max+1)^2                                              */
+    int32_t K;
+    int32_t n_paths;
+    int32_t l_max;
+    int64_t N_w;     /* Eq. num_weights                                          */
+    int64_t state_floats_fwd; /* K*F : floats of receiver state Z per node       */
+    int64_t state_floats_bwd; /* K*F': floats of sender state V per node         */
+} sobek_info;
+
+typedef struct {
+    int32_t i_in, l_sh, i_out;   /* input irrep index, SH order, output irrep index */
+    int32_t l_in, l_out;
+    int32_t c_in, c_out;         /* coupled multiplicities: n_pi = c_in*c_out       */
+    int32_t in_off, sh_off, out_off; /* offsets inside an x row, a Y row, a y row   */
+    int64_t w_off;               /* first column of this path in R                  */
+} sobek_path_info;
+
+int sobek_plan_info(const sobek_plan* plan, sobek_info* info);
+int sobek_plan_path(const sobek_plan* plan, int path, sobek_path_info* info);
+/* Dense c^pi[m_in][m_sh][m_out] (host, (2l_in+1)(2l_sh+1)(2l_out+1) doubles) as the library
+ * computed it (Eq. angular_path_contraction); for inspection and tests. */
+int sobek_plan_cg(const sobek_plan* plan, int path, double* dense);
+
+/*
+ * Graph in receiver-sorted CSR form plus its sender-sorted view ("cached stable CSR
+ * views", Section "Generated deterministic runtime and execution contracts").
+ */
+typedef struct {
+    int64_t N, E;
+    const int64_t* row_ptr;  /* [N+1] row_ptr[0] = 0, row_ptr[N] = E, non-decreasing        */
+    const int32_t* col;      /* [E]   sender of each edge                                   */
+    const int64_t* src_ptr;  /* [N+1] sender-sorted view; may be NULL if gx/hx not wanted   */
+    const int32_t* src_perm; /* [E]   edge ids grouped by sender, increasing inside a group */
+} sobek_graph;
+
+/*
+ * sobek_graph_prepare -- validates (row_ptr, col) and builds the stable sender-sorted view
+ * used by the source-owned traversal of the backward passes (Section "Receiver-factorized
+ * backward").  Integer work; the result is unique, so it can be compared bit for bit.
+ * `ws` needs sobek_graph_prepare_bytes(N, E) bytes, 256-byte aligned.  This call
+ * synchronises `stream` and returns SOBEK_ERR_GRAPH if validation failed.
+ */
+size_t sobek_graph_prepare_bytes(int64_t N, int64_t E);
+int sobek_graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* col,
+                        int64_t* src_ptr, int32_t* src_perm, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/*
+ * Workspace needed by one call of the given order (0 = fwd, 1 = bwd, 2 = dbwd).  It holds
+ * re-laid-out copies of R, the bounded receiver/sender state of one node chunk and a
+ * status word.  It depends on the plan and on min(N, chunk size) only -- never on E.
+ * The pointer passed as `ws` must be 256-byte aligned.
+ */
+size_t sobek_workspace_bytes(const sobek_plan* plan, int64_t N, int64_t E, int order);
+
+/* Forward: y (Eqs. receiver_state, receiver_mixing, receiver_matrix_product). */
+int sobek_conv_fwd(const sobek_plan* plan, const sobek_graph* g,
+                   const float* x, const float* Y, const float* phi, const float* R,
+                   float* y, void* ws, size_t ws_bytes, void* stream);
+
+/* First backward: adjoints of (x, Y, phi, R) for the output adjoint gy
+ * (Eqs. streamed_radial_adjoints, streamed_operand_adjoints, receiver_adjoint). */
+int sobek_conv_bwd(const sobek_plan* plan, const sobek_graph* g,
+                   const float* x, const float* Y, const float* phi, const float* R,
+                   const float* gy,
+                   float* gx, float* gY, float* gphi, float* gR,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* Double backward (Eqs. streamed_directional_terms .. streamed_operand_second_adjoints,
+ * receiver_double_adjoint) with the direction on gy equal to zero: for the backward map
+ * b(x,Y,phi,R; gy) = (gx,gY,gphi,gR) and cotangents v = (vx,vY,vphi,vR) it returns
+ * ggy = d<v,b>/d gy and h_theta = d<v,b>/d theta for theta in (x,Y,phi,R). */
+int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
+                    const float* x, const float* Y, const float* phi, const float* R,
+                    const float* gy,
+                    const float* vx, const float* vY, const float* vphi, const float* vR,
+                    float* ggy, float* hx, float* hY, float* hphi, float* hR,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, then returns the status word the kernels of earlier calls wrote
+ * into `ws` (0, or SOBEK_ERR_DEVICE_TIMEOUT / SOBEK_ERR_GRAPH ...). */
+int sobek_last_device_status(void* ws, void* stream);
+
+const char* sobek_status_string(int status);
+
+/* Number of kernels this library has launched in this process (for benchmarks). */
+int64_t sobek_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOBEK_H_ */

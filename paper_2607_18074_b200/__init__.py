@@ -1,0 +1,210 @@
+"""Thin Python binding of libsobek (argument marshalling only).
+
+Every step of the convolution runs in the library's CUDA kernels; torch is used for device
+memory and streams.  There is no fallback: if the shared library is missing or a call
+fails, an exception is raised.
+
+Names mirror the C ABI (include/sobek.h): `Plan` <-> sobek_plan_*, `graph_prepare`,
+`workspace_bytes`, `conv_fwd`, `conv_bwd`, `conv_dbwd`, `last_device_status`.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsobek.so")
+
+EXPORTS = [
+    "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
+    "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_workspace_bytes", "sobek_conv_fwd",
+    "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
+    "sobek_launch_count",
+]
+
+
+class SobekError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+class Irrep(Structure):
+    _fields_ = [("mul", c_int32), ("l", c_int32), ("parity", c_int32)]
+
+
+class Info(Structure):
+    _fields_ = [("C_x", c_int32), ("C_y", c_int32), ("dim_sh", c_int32), ("K", c_int32),
+                ("n_paths", c_int32), ("l_max", c_int32), ("N_w", c_int64),
+                ("state_floats_fwd", c_int64), ("state_floats_bwd", c_int64)]
+
+
+class PathInfo(Structure):
+    _fields_ = [("i_in", c_int32), ("l_sh", c_int32), ("i_out", c_int32), ("l_in", c_int32),
+                ("l_out", c_int32), ("c_in", c_int32), ("c_out", c_int32), ("in_off", c_int32),
+                ("sh_off", c_int32), ("out_off", c_int32), ("w_off", c_int64)]
+
+
+class Graph(Structure):
+    _fields_ = [("N", c_int64), ("E", c_int64), ("row_ptr", c_void_p), ("col", c_void_p),
+                ("src_ptr", c_void_p), ("src_perm", c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_2607_18074_b200.build` (needs nvcc)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.sobek_plan_create.argtypes = [POINTER(Irrep), c_int, POINTER(Irrep), c_int, c_int, c_int,
+                                        c_uint32, POINTER(c_void_p)]
+        L.sobek_plan_destroy.argtypes = [c_void_p]
+        L.sobek_plan_destroy.restype = None
+        L.sobek_plan_info.argtypes = [c_void_p, POINTER(Info)]
+        L.sobek_plan_path.argtypes = [c_void_p, c_int, POINTER(PathInfo)]
+        L.sobek_plan_cg.argtypes = [c_void_p, c_int, POINTER(c_double)]
+        L.sobek_graph_prepare_bytes.argtypes = [c_int64, c_int64]
+        L.sobek_graph_prepare_bytes.restype = c_size_t
+        L.sobek_graph_prepare.argtypes = [c_int64, c_int64] + [c_void_p] * 5 + [c_size_t, c_void_p]
+        L.sobek_workspace_bytes.argtypes = [c_void_p, c_int64, c_int64, c_int]
+        L.sobek_workspace_bytes.restype = c_size_t
+        L.sobek_conv_fwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6 + [c_size_t, c_void_p]
+        L.sobek_conv_bwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 10 + [c_size_t, c_void_p]
+        L.sobek_conv_dbwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 15 + [c_size_t, c_void_p]
+        L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
+        L.sobek_status_string.argtypes = [c_int]
+        L.sobek_status_string.restype = c_char_p
+        L.sobek_launch_count.restype = c_int64
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().sobek_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().sobek_launch_count())
+
+
+def _check(code, where):
+    if code != 0:
+        raise SobekError(code, where)
+
+
+def _irreps(seq):
+    arr = (Irrep * len(seq))()
+    for k, (mul, l, p) in enumerate(seq):
+        arr[k] = Irrep(mul, l, p)
+    return arr
+
+
+class Plan:
+    """sobek_plan: irreps are sequences of (mul, l, parity) with parity +1 / -1."""
+
+    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0):
+        self._h = c_void_p()
+        a, b = _irreps(irreps_in), _irreps(irreps_out)
+        _check(lib().sobek_plan_create(a, len(irreps_in), b, len(irreps_out), l_max, K, flags,
+                                       byref(self._h)), "sobek_plan_create")
+        self.info = Info()
+        _check(lib().sobek_plan_info(self._h, byref(self.info)), "sobek_plan_info")
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h and _lib is not None:
+            _lib.sobek_plan_destroy(h)
+            self._h = None
+
+    @property
+    def handle(self):
+        return self._h
+
+    def path(self, k: int) -> PathInfo:
+        pi = PathInfo()
+        _check(lib().sobek_plan_path(self._h, k, byref(pi)), "sobek_plan_path")
+        return pi
+
+    def cg(self, k: int):
+        import numpy as np
+        pi = self.path(k)
+        shape = (2 * pi.l_in + 1, 2 * pi.l_sh + 1, 2 * pi.l_out + 1)
+        out = np.zeros(shape, dtype=np.float64)
+        _check(lib().sobek_plan_cg(self._h, k, out.ctypes.data_as(POINTER(c_double))), "sobek_plan_cg")
+        return out
+
+    def col_std(self):
+        """1/sqrt(fan_in) per column of R (fan_in = K * sum of input multiplicities over the
+        paths into the column's output block): the scale used for synthetic weights."""
+        import numpy as np
+        paths = [self.path(k) for k in range(self.info.n_paths)]
+        fan = {}
+        for p in paths:
+            fan[p.i_out] = fan.get(p.i_out, 0) + p.c_in
+        std = np.zeros(self.info.N_w)
+        for p in paths:
+            std[p.w_off:p.w_off + p.c_in * p.c_out] = (self.info.K * fan[p.i_out]) ** -0.5
+        return std
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def graph_prepare_bytes(N: int, E: int) -> int:
+    return int(lib().sobek_graph_prepare_bytes(N, E))
+
+
+def graph_prepare(row_ptr, col):
+    """Validates the receiver-sorted CSR (int64 row_ptr[N+1], int32 col[E], CUDA tensors) and
+    returns the sender-sorted view (src_ptr int64[N+1], src_perm int32[E])."""
+    import torch
+    N, E = row_ptr.numel() - 1, col.numel()
+    src_ptr = torch.empty(N + 1, dtype=torch.int64, device=row_ptr.device)
+    src_perm = torch.empty(E, dtype=torch.int32, device=row_ptr.device)
+    nbytes = graph_prepare_bytes(N, E)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=row_ptr.device)
+    _check(lib().sobek_graph_prepare(N, E, _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm),
+                                     _ptr(ws), nbytes, _stream()), "sobek_graph_prepare")
+    return src_ptr, src_perm
+
+
+def make_graph(row_ptr, col, src_ptr=None, src_perm=None) -> Graph:
+    return Graph(row_ptr.numel() - 1, col.numel(), _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm))
+
+
+def workspace_bytes(plan: Plan, N: int, E: int, order: int) -> int:
+    return int(lib().sobek_workspace_bytes(plan.handle, N, E, order))
+
+
+def conv_fwd(plan, graph, x, Y, phi, R, y, ws):
+    _check(lib().sobek_conv_fwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(y),
+                                _ptr(ws), ws.numel() * ws.element_size(), _stream()), "sobek_conv_fwd")
+
+
+def conv_bwd(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws):
+    _check(lib().sobek_conv_bwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(gy),
+                                _ptr(gx), _ptr(gY), _ptr(gphi), _ptr(gR), _ptr(ws),
+                                ws.numel() * ws.element_size(), _stream()), "sobek_conv_bwd")
+
+
+def conv_dbwd(plan, graph, x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi, hR, ws):
+    _check(lib().sobek_conv_dbwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(gy),
+                                 _ptr(vx), _ptr(vY), _ptr(vphi), _ptr(vR), _ptr(ggy), _ptr(hx), _ptr(hY),
+                                 _ptr(hphi), _ptr(hR), _ptr(ws), ws.numel() * ws.element_size(),
+                                 _stream()), "sobek_conv_dbwd")
+
+
+def last_device_status(ws) -> int:
+    return int(lib().sobek_last_device_status(_ptr(ws), _stream()))

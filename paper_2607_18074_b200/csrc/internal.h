@@ -1,0 +1,149 @@
+// Internal declarations shared by the translation units of libsobek (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+
+#include "sobek.h"
+
+namespace sobek {
+
+// ---------------------------------------------------------------------------------------
+// Device-side description of one traversal direction.
+//
+// FORWARD direction:    destination groups = output irrep blocks, sources = input blocks of x.
+// TRANSPOSED direction: destination groups = input irrep blocks (for gx), sources = output
+//                       blocks of gy.  It is the same operator on the reversed graph with
+//                       c'[m_out,m_sh,m_in] = c[m_in,m_sh,m_out] and R'[q,pi,w,u] = R[q,pi,u,w].
+//
+// For one edge and one path the angular contraction (Eq. angular_path_contraction) is split
+// as  C[u,o] = sum_s xs[u,s] * M[s,o],  M[s,o] = sum_b coef * Y[b]: M depends on the edge and
+// the path only, not on the multiplicity index, and is produced from the sparse table below.
+// ---------------------------------------------------------------------------------------
+struct DPath {
+    int32_t src_off;   // offset of the source block inside a source feature row
+    int32_t c_src;     // source multiplicity
+    int32_t d_src;     // 2 l_src + 1
+    int32_t sh_off;    // offset of the SH block inside a Y row
+    int32_t d_sh;      // 2 l_sh + 1
+    int32_t d_dst;     // 2 l_dst + 1
+    int32_t c_dst;     // destination multiplicity
+    int32_t koff;      // offset in the group's contraction axis; k = koff + u*K + q
+    int32_t m_off;     // offset of M[s][o] inside the group's per-edge M area
+    int32_t tabM;      // index into tab_ptr: entry (s*d_dst+o) -> terms (b, coef)
+    int32_t tabY;      // index into tab_ptr: b -> terms (s*d_dst+o, coef)   (adjoint wrt Y)
+    int32_t pad;
+    int64_t rp_off;    // offset (floats) of the owning group's slab in the packed R
+    int64_t w_off;     // first column of the path in R[K, N_w]
+    int32_t c_in, c_out;  // multiplicities in the ORIGINAL orientation (column = u*c_out + w)
+};
+
+struct DGroup {
+    int32_t dst_off;   // offset of the block inside a destination feature row
+    int32_t c_dst;     // destination multiplicity (GEMM columns)
+    int32_t d_dst;     // 2l+1 (rows per node)
+    int32_t D;         // contraction width = K * sum c_src over the group's paths
+    int32_t path_begin, path_end;
+    int32_t m_entries; // sum over paths of d_src*d_dst
+    int32_t wt_begin, wt_end;   // range in the warp-task list
+    int32_t pad;
+    int64_t z_off;     // offset (floats per node) of this group's state rows: sum_{g'<g} d*D
+    int64_t rp_off;    // offset (floats) of this group's slab in the packed R: sum_{g'<g} D*c_dst
+};
+
+struct WTask {         // one warp's share of a group: 32 consecutive multiplicities of one path
+    int32_t path;
+    int32_t u0;
+};
+
+struct Direction {
+    // host copies
+    std::vector<DPath> paths;
+    std::vector<DGroup> groups;
+    std::vector<WTask> wtasks;
+    int64_t state_floats = 0;   // per node: sum_g d*D
+    int32_t max_m_entries = 0;
+    int32_t C_src = 0, C_dst = 0;
+    // device copies
+    DPath* d_paths = nullptr;
+    DGroup* d_groups = nullptr;
+    WTask* d_wtasks = nullptr;
+};
+
+struct HPath {
+    sobek_path_info info;
+    std::vector<double> cg;   // dense [d_in][d_sh][d_out]
+};
+
+}  // namespace sobek
+
+struct sobek_plan {
+    std::vector<sobek_irrep> in, out;
+    int l_max = 0, K = 0;
+    int C_x = 0, C_y = 0, dim_sh = 0;
+    int64_t N_w = 0;
+    std::vector<sobek::HPath> paths;
+    sobek::Direction fwd, tr;
+    // sparse tables (shared by both directions)
+    std::vector<int32_t> tab_ptr;
+    std::vector<int32_t> tab_idx;
+    std::vector<float> tab_coef;
+    int32_t* d_tab_ptr = nullptr;
+    int32_t* d_tab_idx = nullptr;
+    float* d_tab_coef = nullptr;
+    int device = -1;
+};
+
+namespace sobek {
+
+// bytes reserved at the start of every workspace for the device status word
+constexpr size_t kHeaderBytes = 256;
+// budget for the bounded node-state buffer (floats of Z / V held at once)
+constexpr size_t kStateBudgetBytes = size_t(96) << 20;
+
+int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);
+
+void count_launch(int n = 1);
+
+// --- kernels.cu ---------------------------------------------------------------------
+struct EdgeView {          // how a traversal walks the graph
+    const int64_t* ptr;    // [N+1] segment pointers of the owning node
+    const int32_t* perm;   // NULL: position == edge id; else edge id = perm[position]
+    const int32_t* col;    // sender of each edge (edge-id indexed)
+    const int64_t* row_ptr;// receiver CSR (to recover the receiver of an edge id)
+    int64_t N, E;
+    int transposed;        // 0: source node = col[e];  1: source node = receiver(e)
+};
+
+cudaError_t launch_pack_R(const sobek_plan* p, const Direction& dir, int transposed, const float* R,
+                          float* Rp, cudaStream_t s);
+cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
+                            cudaStream_t s);
+cudaError_t launch_state(const sobek_plan* p, const Direction& dir, const EdgeView& ev,
+                         int64_t node0, int64_t n_nodes, const float* src, const float* Y,
+                         const float* phi, float* Z, int accumulate, cudaStream_t s);
+// y_g = Z_g * Rp_g  for every group (C written through the node/component row map)
+cudaError_t launch_mix(const sobek_plan* p, const Direction& dir, int64_t node0, int64_t n_nodes,
+                       const float* Z, const float* Rp, float* dst, int accumulate, cudaStream_t s);
+// Zbar_g = gy_g * Rp_g^T
+cudaError_t launch_state_adjoint(const sobek_plan* p, const Direction& dir, int64_t node0,
+                                 int64_t n_nodes, const float* gdst, const float* Rp, float* Zbar,
+                                 cudaStream_t s);
+// gRp_g (+)= Z_g^T * gy_g
+cudaError_t launch_weight_grad(const sobek_plan* p, const Direction& dir, int64_t node0,
+                               int64_t n_nodes, const float* Z, const float* gdst, float* gRp,
+                               int accumulate, cudaStream_t s);
+// receiver-owned edge pass: gphi_e = <Zbar, C_e>, gY_e = CG^T_Y(x, phi_e Zbar)
+cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev,
+                             int64_t node0, int64_t n_nodes, const float* src, const float* Y,
+                             const float* phi, const float* Zbar, float* gphi, float* gY,
+                             int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
+                             cudaStream_t s);
+cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
+
+// --- graph.cu -----------------------------------------------------------------------
+size_t graph_prepare_bytes(int64_t N, int64_t E);
+int graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* col, int64_t* src_ptr,
+                  int32_t* src_perm, void* ws, size_t ws_bytes, cudaStream_t s);
+
+}  // namespace sobek

@@ -1,0 +1,221 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 oracle on the same
+seeded inputs.  Element by element on small cases that still span several node chunks and
+ragged multiplicities; on sampled receivers at the benchmark's full sizes."""
+import numpy as np
+import pytest
+
+from oracle import conv as oconv
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import BWD_TOL, FWD_TOL, Case, rel_err  # noqa: E402
+
+P = synth.parse_irreps
+
+
+def small_cases():
+    c = {}
+    c["cfg1"] = synth.config("cfg1")
+    c["cfg2_N200"] = synth.scaled(synth.config("cfg2"), 200)
+    c["cfg3_N120"] = synth.scaled(synth.config("cfg3"), 120)
+    c["cfg4_N150"] = synth.scaled(synth.config("cfg4"), 150)
+    c["cfg5_N60"] = synth.scaled(synth.config("cfg5"), 60)
+    # ragged multiplicities, odd K, mixed parities (odd-sum paths), a block with no path
+    c["ragged"] = synth.Workload("ragged", P("5x0e+3x1o+2x1e+33x2e"), P("7x0e+1x0o+35x1o+2x2e+3x3o+2x4e"),
+                                 3, 3, 40, 4.0, 1.9, "gaussian", seed=3)
+    c["K20"] = synth.Workload("K20", P("6x0e+4x1o"), P("6x0e+4x1o+2x2e"), 2, 20, 50, 4.0, 1.8, "bessel", seed=4)
+    return c
+
+
+CASES = small_cases()
+
+
+@pytest.fixture(scope="module")
+def cases():
+    return {}
+
+
+def get(cases, name):
+    if name not in cases:
+        cases[name] = Case(CASES[name])
+    return cases[name]
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_forward(cases, name):
+    c = get(cases, name)
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_backward(cases, name):
+    c = get(cases, name)
+    for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_double_backward(cases, name):
+    c = get(cases, name)
+    for got, ref, nm in zip(c.dbwd(), c.o_dbwd(), ("ggy", "hx", "hY", "hphi", "hR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+
+
+@pytest.mark.parametrize("dirs", [(1, 0, 0, 0), (0, 1, 0, 0), (0, 0, 1, 0), (0, 0, 0, 1), (0, 0, 0, 0), (1, 0, 1, 0)])
+def test_double_backward_null_directions(cases, dirs):
+    c = get(cases, "cfg1")
+    dirs = tuple(bool(v) for v in dirs)
+    for got, ref, nm in zip(c.dbwd(dirs=dirs), c.o_dbwd(dirs=dirs), ("ggy", "hx", "hY", "hphi", "hR")):
+        if np.abs(ref).max() == 0:
+            assert np.all(got == 0), nm
+        else:
+            assert rel_err(got, ref) <= BWD_TOL, nm
+
+
+def test_partial_outputs(cases):
+    """NULL outputs are skipped and do not change the others."""
+    import torch
+    c = get(cases, "cfg1")
+    sb, i = c.sb, c.plan.info
+    full = c.bwd()
+    gphi = torch.full((c.E, i.K), float("nan"), device="cuda:0")
+    sb.conv_bwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, None, None, gphi, None, c.ws(1))
+    assert np.array_equal(gphi.cpu().numpy(), full[2])
+    gx = torch.full((c.N, i.C_x), float("nan"), device="cuda:0")
+    sb.conv_bwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, gx, None, None, None, c.ws(1))
+    assert np.array_equal(gx.cpu().numpy(), full[0])
+
+
+def test_bitwise_reproducible(cases):
+    c = get(cases, "cfg2_N200")
+    assert np.array_equal(c.fwd(), c.fwd())
+    for a, b in zip(c.bwd(), c.bwd()):
+        assert np.array_equal(a, b)
+    for a, b in zip(c.dbwd(), c.dbwd()):
+        assert np.array_equal(a, b)
+
+
+def test_graph_prepare_bit_exact(cases):
+    for name in ("cfg1", "cfg2_N200", "ragged"):
+        c = get(cases, name)
+        sp, perm = oconv.sender_view(c.d.row_ptr, c.d.col)
+        assert np.array_equal(c.src_ptr.cpu().numpy(), sp)
+        assert np.array_equal(c.src_perm.cpu().numpy(), perm)
+
+
+def test_graph_prepare_large_and_hub():
+    """A hub sender with thousands of out-edges and many empty rows."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    rng = np.random.default_rng(0)
+    N, E = 5000, 60000
+    recv = np.sort(rng.integers(0, N // 2, E))          # upper half of the nodes receives nothing
+    col = rng.integers(0, N, E).astype(np.int32)
+    col[rng.random(E) < 0.2] = 17                         # hub
+    row_ptr = np.concatenate([[0], np.cumsum(np.bincount(recv, minlength=N))]).astype(np.int64)
+    sp, perm = sb.graph_prepare(torch.from_numpy(row_ptr).cuda(), torch.from_numpy(col).cuda())
+    assert np.array_equal(perm.cpu().numpy(), np.argsort(col, kind="stable").astype(np.int32))
+    assert np.array_equal(sp.cpu().numpy(), np.concatenate([[0], np.cumsum(np.bincount(col, minlength=N))]))
+
+
+def test_graph_prepare_rejects_bad_graphs():
+    import torch
+    import paper_2607_18074_b200 as sb
+    rp = torch.tensor([0, 2, 1, 3], dtype=torch.int64, device="cuda:0")       # not monotone
+    col = torch.tensor([0, 1, 2], dtype=torch.int32, device="cuda:0")
+    with pytest.raises(sb.SobekError) as ei:
+        sb.graph_prepare(rp, col)
+    assert ei.value.code == -4
+    rp = torch.tensor([0, 1, 2, 3], dtype=torch.int64, device="cuda:0")
+    col = torch.tensor([0, 7, 2], dtype=torch.int32, device="cuda:0")         # sender out of range
+    with pytest.raises(sb.SobekError) as ei:
+        sb.graph_prepare(rp, col)
+    assert ei.value.code == -4
+
+
+def test_degenerate_graphs():
+    """No edges at all; empty receivers, self loops and duplicate edges."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    ii, io = P("3x0e+2x1o"), P("2x0e+3x1o+1x2e")
+    o = oconv.Oracle(ii, io, 2, 4)
+    plan = sb.Plan(ii, io, 2, 4)
+    rng = np.random.default_rng(0)
+    for row_ptr, col in [(np.zeros(6, dtype=np.int64), np.zeros(0, dtype=np.int32)),
+                         (np.array([0, 0, 3, 3, 4, 4], dtype=np.int64), np.array([1, 2, 2, 0], dtype=np.int32))]:
+        N, E = 5, col.shape[0]
+        f = lambda *s: rng.standard_normal(s).astype(np.float32)
+        x, Y, phi, R, gy = f(N, o.C_x), f(E, 9), f(E, 4), f(4, o.N_w), f(N, o.C_y)
+        t = lambda a: torch.from_numpy(a).cuda()
+        rp_d, col_d = t(row_ptr), t(col)
+        sp, perm = sb.graph_prepare(rp_d, col_d)
+        g = sb.make_graph(rp_d, col_d, sp, perm)
+        ws = torch.empty(sb.workspace_bytes(plan, N, E, 1), dtype=torch.uint8, device="cuda:0")
+        y = torch.full((N, o.C_y), float("nan"), device="cuda:0")
+        sb.conv_fwd(plan, g, t(x), t(Y), t(phi), t(R), y, ws)
+        ref = o.fwd(row_ptr, col, x, Y, phi, R)
+        assert np.abs(y.cpu().numpy() - ref).max() <= FWD_TOL * max(np.abs(ref).max(), 1.0)
+        outs = [torch.full(s, float("nan"), device="cuda:0") for s in ((N, o.C_x), (E, 9), (E, 4), (4, o.N_w))]
+        sb.conv_bwd(plan, g, t(x), t(Y), t(phi), t(R), t(gy), *outs, ws)
+        for got, r in zip(outs, o.bwd(row_ptr, col, x, Y, phi, R, gy)):
+            assert np.abs(got.cpu().numpy() - r).max() <= BWD_TOL * max(np.abs(r).max(), 1.0)
+
+
+def test_errors_on_device_calls(cases):
+    import ctypes
+    import torch
+    c = get(cases, "cfg1")
+    sb = c.sb
+    y = torch.empty(c.N, c.plan.info.C_y, device="cuda:0")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(sb.SobekError) as ei:
+        sb.conv_fwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, y, small)
+    assert ei.value.code == -3
+    g = sb.make_graph(c.row_ptr, c.col)          # no sender view
+    gx = torch.empty(c.N, c.plan.info.C_x, device="cuda:0")
+    with pytest.raises(sb.SobekError) as ei:
+        sb.conv_bwd(c.plan, g, c.x, c.Y, c.phi, c.R, c.gy, gx, None, None, None, c.ws(1))
+    assert ei.value.code == -5
+
+
+# ---------------------------------------------------------------------------------------
+# benchmark-sized workloads, in the configuration bench.py times: sampled receivers
+# ---------------------------------------------------------------------------------------
+FULL = {
+    "cfg2": (synth.config("cfg2"), 48, (0, 1, 2)),
+    "cfg3": (synth.config("cfg3"), 6, (0, 1, 2)),
+    "cfg4_1e5": (synth.config("cfg4", edges=1e5), 8, (0, 1)),
+    "cfg4_1e6": (synth.config("cfg4", edges=1e6), 8, (0, 1)),
+    "cfg5": (synth.config("cfg5"), 3, (0, 1, 2)),
+}
+
+
+@pytest.mark.parametrize("name", list(FULL))
+def test_full_size_sampled(name):
+    w, n_sample, orders = FULL[name]
+    c = Case(w)
+    rng = np.random.default_rng(123)
+    # spread the sample over the node range so that several chunks are hit
+    act = np.sort(rng.choice(c.N, size=n_sample, replace=False))
+    act[0], act[-1] = 0, c.N - 1
+    act = np.unique(act)
+    ed = c.edges_into(act)
+    y = c.fwd()
+    assert np.isfinite(y).all()
+    assert rel_err(y[act], c.o_fwd(act)[act]) <= FWD_TOL
+    gym = c.masked_gy(act)
+    if 1 in orders:
+        got = c.bwd(gy=gym)
+        ref = c.o_bwd(act)
+        assert rel_err(got[0], ref[0]) <= BWD_TOL          # gx: every sender
+        assert rel_err(got[3], ref[3]) <= BWD_TOL          # gR
+        assert rel_err(got[1][ed], ref[1][ed]) <= BWD_TOL and rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL
+        mask = np.ones(c.E, dtype=bool); mask[ed] = False
+        assert np.all(got[1][mask] == 0) and np.all(got[2][mask] == 0)
+    if 2 in orders:
+        got = c.dbwd(gy=gym)
+        ref = c.o_dbwd(act)
+        assert rel_err(got[0][act], ref[0][act]) <= BWD_TOL
+        assert rel_err(got[1], ref[1]) <= BWD_TOL and rel_err(got[4], ref[4]) <= BWD_TOL
+        assert rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL and rel_err(got[3][ed], ref[3][ed]) <= BWD_TOL

@@ -1,0 +1,107 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares,
+its host-side plan logic (path enumeration, Clebsch-Gordan tensors from the library's own
+numerical route) agrees with the oracle's closed-form route, and argument errors are
+reported as status codes.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2607_18074_b200 as sb
+from oracle import tables
+from workloads import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2607_18074_b200 import build
+    build.build()
+
+
+def test_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "sobek.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(sobek_[a-z_0-9]+)\s*\(", hdr))
+    assert declared == set(sb.EXPORTS)
+    L = ctypes.CDLL(sb.LIB_PATH)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_status_strings():
+    assert sb.status_string(0) == "ok"
+    for c in range(-7, 0):
+        assert sb.status_string(c) not in ("ok", "unknown status")
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_plan_paths_and_cg_match_oracle(name):
+    w = synth.config(name)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    paths, n_w = tables.enumerate_paths(w.irreps_in, w.irreps_out, w.l_max)
+    assert plan.info.N_w == n_w and plan.info.n_paths == len(paths)
+    assert plan.info.C_x == synth.irreps_dim(w.irreps_in) and plan.info.C_y == synth.irreps_dim(w.irreps_out)
+    for k, p in enumerate(paths):
+        q = plan.path(k)
+        assert (q.i_in, q.l_sh, q.i_out, q.l_in, q.l_out, q.c_in, q.c_out, q.in_off, q.sh_off, q.out_off,
+                q.w_off) == (p.i_in, p.l_sh, p.i_out, p.l_in, p.l_out, p.c_in, p.c_out, p.in_off, p.sh_off,
+                             p.out_off, p.w_off)
+        assert np.abs(plan.cg(k) - p.cg).max() < 1e-9
+    assert np.allclose(plan.col_std(), tables.weight_col_std(w.irreps_in, w.irreps_out, w.l_max, w.K))
+
+
+def test_cg_all_triples_including_odd_sums():
+    ir_in = [(1, l, p) for l in range(5) for p in (1, -1)]
+    plan = sb.Plan(ir_in, ir_in, 4, 1)
+    paths, _ = tables.enumerate_paths(ir_in, ir_in, 4)
+    assert plan.info.n_paths == len(paths)
+    seen = set()
+    for k, p in enumerate(paths):
+        seen.add((p.l_in, p.l_sh, p.l_out))
+        assert np.abs(plan.cg(k) - p.cg).max() < 1e-9
+    assert len(seen) == sum(1 for a in range(5) for b in range(5) for c in range(abs(a - b), min(a + b, 4) + 1))
+
+
+def test_state_widths():
+    w = synth.config("cfg4")
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    assert plan.info.state_floats_fwd == 35840          # K*F
+    w = synth.config("cfg3")
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    assert plan.info.state_floats_fwd == 40960 and plan.info.state_floats_bwd == 8 * 2816
+
+
+def test_workspace_does_not_grow_with_edges():
+    w = synth.config("cfg4")
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    for order in (0, 1, 2):
+        a = sb.workspace_bytes(plan, 3125, 10**5, order)
+        assert a > 0
+        # same node count, any edge count
+        assert sb.workspace_bytes(plan, 3125, 10**9, order) == a
+        # more nodes: bounded by the state budget, identical from some size on
+        assert sb.workspace_bytes(plan, 10**6, 10**8, order) == sb.workspace_bytes(plan, 3 * 10**6, 10**8, order)
+        assert sb.workspace_bytes(plan, 10**6, 10**8, order) < 400 * 2**20
+
+
+def test_argument_errors_are_status_codes():
+    L = sb.lib()
+    h = ctypes.c_void_p()
+    ok = sb._irreps([(2, 0, 1)])
+    assert L.sobek_plan_create(None, 1, ok, 1, 0, 4, 0, ctypes.byref(h)) == -1
+    assert L.sobek_plan_create(ok, 1, ok, 1, 0, 0, 0, ctypes.byref(h)) == -1            # K < 1
+    assert L.sobek_plan_create(ok, 1, ok, 1, 5, 4, 0, ctypes.byref(h)) == -2            # l_max too high
+    assert L.sobek_plan_create(sb._irreps([(2, 0, 3)]), 1, ok, 1, 0, 4, 0, ctypes.byref(h)) == -1   # parity
+    assert L.sobek_plan_create(sb._irreps([(2, 7, 1)]), 1, ok, 1, 0, 4, 0, ctypes.byref(h)) == -2   # l too high
+    # no valid path: 0e x (0e) -> 0o
+    assert L.sobek_plan_create(ok, 1, sb._irreps([(2, 0, -1)]), 1, 0, 4, 0, ctypes.byref(h)) == -2
+    plan = sb.Plan([(2, 0, 1)], [(2, 0, 1)], 0, 4)
+    g = sb.Graph(4, 0, None, None, None, None)
+    assert L.sobek_conv_fwd(None, ctypes.byref(g), None, None, None, None, None, None, 0, None) == -1
+    assert L.sobek_plan_path(plan.handle, 99, ctypes.byref(sb.PathInfo())) == -1
+    assert sb.workspace_bytes(plan, 4, 0, 7) == 0
+    assert L.sobek_last_device_status(None, None) == -1
