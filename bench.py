@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the streaming tensor-product convolution on B200.
+
+One step = one pass of the whole hot path over one synthetic workload: forward, first
+backward (all four adjoints) and double backward (all five outputs), each called through
+the C ABI.  `value` is edges per second of a whole step with inputs resident in HBM;
+`orders` gives edges/s of each differentiation order on its own; `e2e` is the same step
+with host buffers (pinned host -> device copies of every floating-point input and
+device -> host copies of every output inside the timed region).
+
+Prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import synth  # noqa: E402
+
+METRIC = "edges/s (one step = fwd + bwd + double-bwd)"
+FP32_FMA_LANES = 148 * 128            # SMs x FP32 lanes
+L2_FLUSH_BYTES = 512 << 20
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "sm_max_mhz": d.get("sm_max_mhz", 1965.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+def work_model(plan):
+    """Algorithmic multiply-adds per edge / per node of each order, from the path table."""
+    K = plan.info.K
+    KF = KFt = CG = CGt = Gf = Gt = 0
+    for k in range(plan.info.n_paths):
+        p = plan.path(k)
+        di, do = 2 * p.l_in + 1, 2 * p.l_out + 1
+        nnz = int((np.abs(plan.cg(k)) > 0).sum())
+        KF += K * p.c_in * do
+        KFt += K * p.c_out * di
+        CG += p.c_in * nnz
+        CGt += p.c_out * nnz
+        Gf += K * p.c_in * p.c_out * do
+        Gt += K * p.c_in * p.c_out * di
+    edge = {"fwd": KF + CG, "bwd": 3 * KF + KFt + 3 * CG + CGt, "dbwd": 8 * KF + 3 * KFt + 5 * CG + 2 * CGt}
+    node = {"fwd": Gf, "bwd": 2 * Gf + Gt, "dbwd": 5 * Gf + 2 * Gt}
+    # split of the edge work between the two edge-stream kernel classes
+    cls = {"edge_stream_state": (KF + CG) + (KF + CG + KFt + CGt) + (3 * KF + 2 * CG + 3 * KFt + 2 * CGt),
+           "edge_pass": (2 * KF + 2 * CG) + (5 * KF + 3 * CG)}
+    return edge, node, cls
+
+
+class ClockSampler:
+    def __init__(self, device_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={device_index}", f"--query-gpu={q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.strip()]
+        os.unlink(self.f.name)
+        sm, names = [], ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                out["sm_max_mhz"] = float(r[1])
+                for nm, v in zip(names, r[3:7]):
+                    if v.strip().lower().startswith("active"):
+                        reasons.add(nm)
+            except (ValueError, IndexError):
+                pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+def oracle_sample_rate(w, d, oracle, target_s=15.0):
+    """Times the fp64 oracle (fwd + bwd + dbwd) on a contiguous receiver sample and returns
+    (edges/s, edges in the sample, seconds, per-order seconds)."""
+    def run(act):
+        t = {}
+        t0 = time.perf_counter()
+        oracle.fwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, act=act)
+        t["fwd"] = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.bwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, act=act)
+        t["bwd"] = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.dbwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, d.vx, d.vY, d.vphi, d.vR, act=act)
+        t["dbwd"] = time.perf_counter() - t0
+        return t
+
+    from oracle import conv as oconv
+    cores = oconv.threads()
+    n0 = min(d.N, max(2 * cores, 16))
+    t = run(np.arange(n0))
+    tot = sum(t.values())
+    n1 = int(min(d.N, max(n0, n0 * target_s / max(tot, 1e-6))))
+    if n1 > 2 * n0:
+        t = run(np.arange(n1))
+        n0 = n1
+        tot = sum(t.values())
+    edges = int(d.row_ptr[n0] - d.row_ptr[0])
+    return edges / tot, edges, tot, t, n0, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import conv as oconv
+    w = synth.config(args.workload)
+    oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    d = synth.make_inputs(w, oracle.col_std())
+    cores = oconv.threads()
+    # one step = fwd+bwd+dbwd on a bounded contiguous receiver sample
+    n = min(d.N, max(cores, 8))
+    act = np.arange(n)
+    edges = int(d.row_ptr[n] - d.row_ptr[0])
+
+    def step():
+        oracle.fwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, act=act)
+        oracle.bwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, act=act)
+        oracle.dbwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, d.vx, d.vY, d.vphi, d.vR, act=act)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = edges / dt
+    sample = f"{n} contiguous receivers ({edges} edges) of {w.name} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "edges/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "N": d.N, "E": d.E, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "edges/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "edges/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2607_18074_b200 as sb
+    sb.lib()   # fails loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+
+    w = synth.config(args.workload)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    # replicas only: every rank runs the same workload on its own GPU (different seed per rank)
+    w.seed = rank
+    d = synth.make_inputs(w, plan.col_std())
+    i = plan.info
+    N, E = d.N, d.E
+
+    host = {k: torch.from_numpy(np.ascontiguousarray(getattr(d, k))).pin_memory()
+            for k in ("x", "Y", "phi", "R", "gy", "vx", "vY", "vphi", "vR")}
+    torch.cuda.reset_peak_memory_stats(dev)
+    base_alloc = torch.cuda.memory_allocated(dev)
+    t = {k: v.to(dev) for k, v in host.items()}
+    rp = torch.from_numpy(d.row_ptr.astype(np.int64)).to(dev)
+    col = torch.from_numpy(d.col.astype(np.int32)).to(dev)
+    sp, perm = sb.graph_prepare(rp, col)
+    g = sb.make_graph(rp, col, sp, perm)
+    in_bytes = torch.cuda.memory_allocated(dev) - base_alloc
+    new = lambda *s: torch.empty(*s, dtype=torch.float32, device=dev)
+    out = {"y": new(N, i.C_y), "gx": new(N, i.C_x), "gY": new(E, i.dim_sh), "gphi": new(E, i.K),
+           "gR": new(i.K, i.N_w), "ggy": new(N, i.C_y), "hx": new(N, i.C_x), "hY": new(E, i.dim_sh),
+           "hphi": new(E, i.K), "hR": new(i.K, i.N_w)}
+    out_bytes = sum(v.numel() * 4 for v in out.values())
+    ws_bytes = sb.workspace_bytes(plan, N, E, 2)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
+
+    def fwd():
+        sb.conv_fwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], out["y"], ws)
+
+    def bwd():
+        sb.conv_bwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], t["gy"], out["gx"], out["gY"], out["gphi"],
+                    out["gR"], ws)
+
+    def dbwd():
+        sb.conv_dbwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], t["gy"], t["vx"], t["vY"], t["vphi"], t["vR"],
+                     out["ggy"], out["hx"], out["hY"], out["hphi"], out["hR"], ws)
+
+    orders = [("fwd", fwd), ("bwd", bwd), ("dbwd", dbwd)]
+
+    def timed_step():
+        """One step; returns per-order device milliseconds.  L2 is flushed (a buffer larger than
+        L2 is overwritten) before every order, outside the event brackets."""
+        evs = []
+        for _, fn in orders:
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        timed_step()
+    assert sb.last_device_status(ws) == 0
+    peak_bytes = torch.cuda.max_memory_allocated(dev) - base_alloc
+
+    # ---- timed region: exactly K steps -------------------------------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    l0 = sb.launch_count()
+    per = []
+    wall0 = time.perf_counter()
+    for _ in range(args.steps):
+        per.append(timed_step())
+    barrier()
+    wall = time.perf_counter() - wall0
+    launches = sb.launch_count() - l0
+    per = np.array(per)                                  # [steps, 3] device ms
+    step_ms = float(per.sum(axis=1).mean())
+    order_ms = per.mean(axis=0)
+
+    # ---- per-kernel-class device time over K more steps (events around every launch)
+    sb.timing_enable(True)
+    for _ in range(args.steps):
+        for _, fn in orders:
+            flush.fill_(1)
+            fn()
+    torch.cuda.synchronize(dev)
+    sb.timing_enable(False)
+    classes = sb.timing_collect()
+    clocks = sampler.stop() if sampler else None
+
+    # ---- end to end: host buffers in, host buffers out ---------------------------------
+    def e2e_step():
+        for k, v in host.items():
+            t[k].copy_(v, non_blocking=True)
+        fwd(); bwd(); dbwd()
+        for k, v in out.items():
+            host_out[k].copy_(v, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize(dev)
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        flush.fill_(1)
+        e2e_step()
+    b.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b) / args.steps
+    h2d = sum(v.numel() * 4 for v in host.values())
+    d2h = out_bytes
+
+    # ---- max over ranks ------------------------------------------------------------------
+    if dist is not None:
+        v = torch.tensor([step_ms, e2e_ms] + list(order_ms), device=dev, dtype=torch.float64)
+        dist.all_reduce(v, op=dist.ReduceOp.MAX)
+        step_ms, e2e_ms = float(v[0]), float(v[1])
+        order_ms = v[2:].cpu().numpy()
+        es = torch.tensor([E], device=dev, dtype=torch.float64)
+        dist.all_reduce(es, op=dist.ReduceOp.SUM)
+        E_total = float(es[0])
+    else:
+        E_total = float(E)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    edge_w, node_w, cls_w = work_model(plan)
+    # dominant kernel class and its roofline
+    tot_cls = sum(v[0] for v in classes.values()) or 1.0
+    dom = max(classes, key=lambda k: classes[k][0])
+    dom_ms, dom_launches = classes[dom]
+    steps_timed = args.steps
+    if dom == "node_gemm":
+        fmas = (node_w["fwd"] + node_w["bwd"] + node_w["dbwd"]) * N * steps_timed
+    else:
+        fmas = cls_w.get(dom, 0) * E * steps_timed
+    alu_peak = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
+    achieved = 2.0 * fmas / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
+    roofline = {"kernel": dom, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                "frac": achieved / alu_peak, "traffic": None,
+                "peak_source": f"derived: 148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz "
+                               f"(HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_tflops']} TFLOP/s {peaks['source']})",
+                "avg_launch_ms": dom_ms / max(dom_launches, 1), "launches": int(dom_launches),
+                "share_of_kernel_time": dom_ms / tot_cls,
+                "classes": {k: {"ms_per_step": v[0] / steps_timed, "launches_per_step": v[1] / steps_timed}
+                            for k, v in classes.items()}}
+
+    res = {
+        "metric": METRIC, "value": E_total / (step_ms * 1e-3), "unit": "edges/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "N": N, "E": E, "K": i.K, "N_w": int(i.N_w), "C_x": i.C_x, "C_y": i.C_y,
+                   "l_max": i.l_max, "replicas": world, "l2": f"flushed before every order ({L2_FLUSH_BYTES >> 20} MiB write)"},
+        "orders": {nm: {"edges_per_s": E_total / (ms * 1e-3), "ms": float(ms),
+                        "edge_fma_per_edge": edge_w[nm], "node_fma_per_node": node_w[nm]}
+                   for (nm, _), ms in zip(orders, order_ms)},
+        "e2e": {"value": E_total / (e2e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "wall_s_timed_region": wall,
+        "peak_bytes": {"total": int(peak_bytes), "inputs_and_graph": int(in_bytes), "outputs": int(out_bytes),
+                       "workspace": int(ws_bytes), "l2_flush_buffer": L2_FLUSH_BYTES},
+        "roofline": roofline,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import conv as oconv
+        oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
+        rate, edges, secs, tt, nrecv, cores = oracle_sample_rate(w, d, oracle)
+        res["cpu_baseline"] = {"value": rate, "unit": "edges/s", "cores": cores, "kind": "oracle",
+                               "sample": f"first {nrecv} receivers ({edges} edges) of {w.name}, fwd+bwd+dbwd, {secs:.1f} s",
+                               "seconds": {k: round(v, 3) for k, v in tt.items()}}
+    print(json.dumps(res))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

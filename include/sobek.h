@@ -177,6 +177,17 @@ const char* sobek_status_string(int status);
 /* Number of kernels this library has launched in this process (for benchmarks). */
 int64_t sobek_launch_count(void);
 
+/*
+ * Instrumentation for benchmarks (the paper has no counterpart).  While enabled, every kernel
+ * launch is bracketed by two CUDA events on its stream.  sobek_timing_collect waits for them,
+ * returns per kernel class the summed device time in milliseconds and the number of launches
+ * (arrays of sobek_timing_classes() entries), and forgets them.  Host-side only; not thread-safe.
+ */
+int sobek_timing_enable(int on);
+int sobek_timing_classes(void);
+const char* sobek_timing_class_name(int cls);
+int sobek_timing_collect(double* total_ms, int64_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,7 +20,8 @@ EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
     "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_workspace_bytes", "sobek_conv_fwd",
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
-    "sobek_launch_count",
+    "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
+    "sobek_timing_collect",
 ]
 
 
@@ -81,6 +82,10 @@ def lib():
         L.sobek_status_string.argtypes = [c_int]
         L.sobek_status_string.restype = c_char_p
         L.sobek_launch_count.restype = c_int64
+        L.sobek_timing_enable.argtypes = [c_int]
+        L.sobek_timing_class_name.argtypes = [c_int]
+        L.sobek_timing_class_name.restype = c_char_p
+        L.sobek_timing_collect.argtypes = [POINTER(c_double), POINTER(c_int64)]
         _lib = L
     return _lib
 
@@ -91,6 +96,18 @@ def status_string(code: int) -> str:
 
 def launch_count() -> int:
     return int(lib().sobek_launch_count())
+
+
+def timing_enable(on: bool):
+    lib().sobek_timing_enable(1 if on else 0)
+
+
+def timing_collect():
+    """{kernel class: (total device ms, launches)} since timing was enabled / last collected."""
+    n = lib().sobek_timing_classes()
+    ms, cnt = (c_double * n)(), (c_int64 * n)()
+    _check(lib().sobek_timing_collect(ms, cnt), "sobek_timing_collect")
+    return {lib().sobek_timing_class_name(k).decode(): (ms[k], cnt[k]) for k in range(n)}
 
 
 def _check(code, where):

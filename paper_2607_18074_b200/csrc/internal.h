@@ -105,6 +105,19 @@ int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);
 
 void count_launch(int n = 1);
 
+enum KernelClass { K_PACK = 0, K_STATE, K_GEMM, K_EDGE, K_FILL, K_NCLASS };
+// Brackets one launch with CUDA events when timing is enabled (sobek_timing_enable).
+class KernelTimer {
+public:
+    KernelTimer(int cls, cudaStream_t s);
+    ~KernelTimer();
+private:
+    int cls_;
+    cudaStream_t s_;
+    bool on_;
+    cudaEvent_t a_{}, b_{};
+};
+
 // --- kernels.cu ---------------------------------------------------------------------
 struct EdgeView {          // how a traversal walks the graph
     const int64_t* ptr;    // [N+1] segment pointers of the owning node

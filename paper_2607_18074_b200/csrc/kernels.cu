@@ -14,6 +14,8 @@
 #include <stdio.h>
 
 #include <atomic>
+#include <type_traits>
+#include <vector>
 
 #include "internal.h"
 
@@ -22,9 +24,57 @@ namespace sobek {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Optional per-kernel-class timing (off by default): every launch is bracketed by two CUDA
+// events on the launching stream; sobek_timing_collect sums the elapsed times per class.
+static bool g_timing = false;
+struct TimedLaunch { cudaEvent_t a, b; int cls; };
+static std::vector<TimedLaunch> g_timed;
+static const char* kClassNames[K_NCLASS] = {"pack_R", "edge_stream_state", "node_gemm", "edge_pass", "fill"};
+
+KernelTimer::KernelTimer(int cls, cudaStream_t s) : cls_(cls), s_(s), on_(g_timing) {
+    if (!on_) return;
+    if (cudaEventCreate(&a_) != cudaSuccess || cudaEventCreate(&b_) != cudaSuccess) { on_ = false; return; }
+    cudaEventRecord(a_, s_);
+}
+KernelTimer::~KernelTimer() {
+    if (!on_) return;
+    cudaEventRecord(b_, s_);
+    g_timed.push_back(TimedLaunch{a_, b_, cls_});
+}
+
 }  // namespace sobek
 
 extern "C" int64_t sobek_launch_count(void) { return sobek::g_launches.load(); }
+
+extern "C" int sobek_timing_enable(int on) {
+    sobek::g_timing = on != 0;
+    return SOBEK_OK;
+}
+
+extern "C" int sobek_timing_classes(void) { return sobek::K_NCLASS; }
+
+extern "C" const char* sobek_timing_class_name(int cls) {
+    return (cls >= 0 && cls < sobek::K_NCLASS) ? sobek::kClassNames[cls] : "";
+}
+
+extern "C" int sobek_timing_collect(double* total_ms, int64_t* launches) {
+    if (!total_ms || !launches) return SOBEK_ERR_INVALID_ARG;
+    for (int c = 0; c < sobek::K_NCLASS; ++c) { total_ms[c] = 0.0; launches[c] = 0; }
+    int rc = SOBEK_OK;
+    for (auto& t : sobek::g_timed) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(t.b) != cudaSuccess || cudaEventElapsedTime(&ms, t.a, t.b) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = SOBEK_ERR_CUDA;
+        }
+        total_ms[t.cls] += ms;
+        launches[t.cls] += 1;
+        cudaEventDestroy(t.a);
+        cudaEventDestroy(t.b);
+    }
+    sobek::g_timed.clear();
+    return rc;
+}
 
 namespace sobek {
 namespace {
@@ -476,6 +526,7 @@ cudaError_t dispatch_d(int d, F&& f) {
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    KernelTimer kt(K_FILL, s);
     k_fill_zero<<<blocks, 256, 0, s>>>(p, n);
     count_launch();
     return cudaGetLastError();
@@ -484,6 +535,7 @@ cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s) {
 cudaError_t launch_pack_R(const sobek_plan* p, const Direction& dir, int transposed, const float* R,
                           float* Rp, cudaStream_t s) {
     dim3 grid(32, (unsigned)dir.paths.size());
+    KernelTimer kt(K_PACK, s);
     k_pack_R<false><<<grid, 256, 0, s>>>(dir.d_paths, transposed, p->K, p->N_w, R, Rp);
     count_launch();
     return cudaGetLastError();
@@ -492,6 +544,7 @@ cudaError_t launch_pack_R(const sobek_plan* p, const Direction& dir, int transpo
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s) {
     dim3 grid(32, (unsigned)dir.paths.size());
+    KernelTimer kt(K_PACK, s);
     k_pack_R<true><<<grid, 256, 0, s>>>(dir.d_paths, 0, p->K, p->N_w, Rp, R);
     count_launch();
     return cudaGetLastError();
@@ -515,10 +568,8 @@ cudaError_t launch_state(const sobek_plan* p, const Direction& dir, const EdgeVi
         const int KC = k16 ? 16 : 8;
         size_t sh = sizeof(float) * ((size_t)ST_EB * a.m_stride + (size_t)ST_EB * a.dsh + (size_t)ST_EB * KC) +
                     sizeof(int64_t) * ST_EB + 16;
-        // keep the int64 array 8-byte aligned: pad the float part to an even count
-        if (((size_t)ST_EB * a.m_stride + (size_t)ST_EB * a.dsh + (size_t)ST_EB * KC) & 1) {
-            // EB is even, so the count is always even; nothing to do
-        }
+        // (EB is even, so the float part has an even count and the int64 array stays aligned)
+        KernelTimer kt(K_STATE, s);
         cudaError_t e = dispatch_d(G.d_dst, [&](auto dtag) -> cudaError_t {
             constexpr int D = decltype(dtag)::value;
             if (k16) {
@@ -541,6 +592,7 @@ cudaError_t launch_state(const sobek_plan* p, const Direction& dir, const EdgeVi
 static cudaError_t run_gemm(const GemmArgs& g, cudaStream_t s) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     dim3 grid((unsigned)((g.N + GN - 1) / GN), (unsigned)((g.M + GM - 1) / GM));
+    KernelTimer kt(K_GEMM, s);
     k_gemm<<<grid, 256, 0, s>>>(g);
     count_launch();
     return cudaGetLastError();
@@ -638,6 +690,7 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
         a.warp_floats = wf + 64;   // + 32 int64
         const size_t sh = (size_t)a.warp_floats * EP_WARPS * sizeof(float);
         dim3 grid((unsigned)((n_nodes + EP_WARPS - 1) / EP_WARPS));
+        KernelTimer kt(K_EDGE, s);
         cudaError_t e = dispatch_d(G.d_dst, [&](auto dtag) -> cudaError_t {
             constexpr int D = decltype(dtag)::value;
             if (k16) {
