@@ -168,6 +168,29 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
                     float* ggy, float* hx, float* hY, float* hphi, float* hR,
                     void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * sobek_conv_fwd_static -- the forward convolution with NO workspace argument and no
+ * allocation of any kind (the paper has no counterpart; it exists for hosts of this library
+ * that cannot allocate device memory when they run the operator: code running inside another
+ * framework's fixed memory plan, real-time loops, processes whose device memory was handed out
+ * completely at start-up).  Same inputs, output and results as sobek_conv_fwd.  The scratch that
+ * sobek_conv_fwd takes from the caller lives in a fixed array inside the library image:
+ * sobek_static_scratch_bytes() bytes (32 MiB) on every GPU that loads the library, held until the
+ * process exits.  The call makes no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - Limit: 256 + 4*K*N_w (rounded up to 256) + 4*K*F bytes must fit in the array, K*F being
+ *     sobek_info.state_floats_fwd (the state of a single node); otherwise SOBEK_ERR_WORKSPACE is
+ *     returned and nothing is launched.  Larger graphs only mean more node chunks.
+ *   - The first call on a device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - Every call on a device shares the one array, and the array keeps the previous call's
+ *     contents: the call clears what must start at zero itself, but two calls whose kernels
+ *     overlap on the GPU (different streams) race.  Serialise them.
+ */
+size_t sobek_static_scratch_bytes(void);
+int sobek_conv_fwd_static(const sobek_plan* plan, const sobek_graph* g,
+                          const float* x, const float* Y, const float* phi, const float* R,
+                          float* y, void* stream);
+
 /* Synchronises `stream`, then returns the status word the kernels of earlier calls wrote
  * into `ws` (0, or SOBEK_ERR_DEVICE_TIMEOUT / SOBEK_ERR_GRAPH ...). */
 int sobek_last_device_status(void* ws, void* stream);

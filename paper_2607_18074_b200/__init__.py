@@ -21,7 +21,7 @@ EXPORTS = [
     "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_workspace_bytes", "sobek_conv_fwd",
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
-    "sobek_timing_collect",
+    "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static",
 ]
 
 
@@ -79,6 +79,8 @@ def lib():
         L.sobek_conv_bwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 10 + [c_size_t, c_void_p]
         L.sobek_conv_dbwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 15 + [c_size_t, c_void_p]
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
+        L.sobek_static_scratch_bytes.restype = c_size_t
+        L.sobek_conv_fwd_static.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6
         L.sobek_status_string.argtypes = [c_int]
         L.sobek_status_string.restype = c_char_p
         L.sobek_launch_count.restype = c_int64
@@ -208,6 +210,18 @@ def workspace_bytes(plan: Plan, N: int, E: int, order: int) -> int:
 def conv_fwd(plan, graph, x, Y, phi, R, y, ws):
     _check(lib().sobek_conv_fwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(y),
                                 _ptr(ws), ws.numel() * ws.element_size(), _stream()), "sobek_conv_fwd")
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().sobek_static_scratch_bytes())
+
+
+def conv_fwd_static(plan, graph, x, Y, phi, R, y):
+    """Forward convolution without a workspace: for callers that cannot allocate device memory
+    when they run the operator.  Scratch lives in a fixed 32 MiB array inside the library (see
+    sobek_conv_fwd_static in include/sobek.h for the size limit and the sharing rules)."""
+    _check(lib().sobek_conv_fwd_static(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R),
+                                       _ptr(y), _stream()), "sobek_conv_fwd_static")
 
 
 def conv_bwd(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws):
