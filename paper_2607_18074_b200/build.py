@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsobek.so")
-SOURCES = ["plan.cu", "graph.cu", "kernels.cu", "api.cu", "static_scratch.cu"]
+SOURCES = ["plan.cu", "graph.cu", "kernels.cu", "gemm_tc.cu", "api.cu", "static_scratch.cu"]
 
 
 def nvcc_cmd(verbose_ptxas: bool = False):

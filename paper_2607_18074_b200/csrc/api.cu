@@ -1,6 +1,8 @@
 // C-ABI entry points: argument checks, workspace carving and the launch schedules of
 // forward, backward and double backward.  Everything here only enqueues work on the
 // caller's stream.
+#include <stdlib.h>
+
 #include <algorithm>
 
 #include "internal.h"
@@ -13,12 +15,16 @@ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Workspace {
     int* status;
-    float* Rp;     // R   packed for the receiver direction
-    float* Rt;     // R   packed for the sender direction
-    float* gRp;    // packed accumulator of the R adjoint
-    float* vRp;    // vR  packed, receiver direction
-    float* vRt;    // vR  packed, sender direction
-    float* state;  // bounded node state (Z / Zbar / V) of one chunk
+    // bf16 (hi, lo) copies of R as tensor-core operands
+    uint16_t *fNKh, *fNKl;    // receiver direction, [w][k]   (y = Z Rp)
+    uint16_t *fKNh, *fKNl;    // receiver direction, [k][w]   (Zbar = gy Rp^T)
+    uint16_t *tNKh, *tNKl;    // sender direction,   [u][k']  (gx = V Rt)
+    uint16_t *vfNKh, *vfNKl, *vfKNh, *vfKNl, *vtNKh, *vtNKl;   // the same for vR
+    float* gRp;               // fp32 accumulator of the R adjoint, packed [k][w] per group
+    float *Rp, *Rt, *vRp, *vRt;   // DEBUG: fp32 packs for the SIMT GEMM
+    float* state;             // fp32 node state of one chunk (Z / Zbar / V)
+    uint16_t *zbh, *zbl;      // bf16 split of the node state of one chunk
+    uint16_t *gbh, *gbl;      // bf16 split of the chunk's output-adjoint rows
     int64_t chunk;
     size_t bytes;
 };
@@ -26,23 +32,34 @@ struct Workspace {
 Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     Workspace w{};
     char* c = (char*)ws;
-    const size_t rbytes = align256((size_t)p->K * (size_t)p->N_w * 4);
     size_t off = kHeaderBytes;
+    auto take = [&](size_t bytes) { char* r = c + off; off += align256(bytes); return r; };
     w.status = (int*)c;
-    w.Rp = (float*)(c + off); off += rbytes;
+    w.fNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.fNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
     if (order >= 1) {
-        w.Rt = (float*)(c + off); off += rbytes;
-        w.gRp = (float*)(c + off); off += rbytes;
+        w.fKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.fKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
+        w.tNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.tNKl = (uint16_t*)take(p->tr.nk_elems * 2);
+        w.gRp = (float*)take((size_t)p->K * (size_t)p->N_w * 4);
     }
     if (order >= 2) {
-        w.vRp = (float*)(c + off); off += rbytes;
-        w.vRt = (float*)(c + off); off += rbytes;
+        w.vfNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.vfNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
+        w.vfKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.vfKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
+        w.vtNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.vtNKl = (uint16_t*)take(p->tr.nk_elems * 2);
+    }
+    {
+        const size_t rb = (size_t)p->K * (size_t)p->N_w * 4;
+        w.Rp = (float*)take(rb); w.Rt = (float*)take(rb); w.vRp = (float*)take(rb); w.vRt = (float*)take(rb);
     }
     w.chunk = chunk_nodes(p, N, order);
-    int64_t per = p->fwd.state_floats;
-    if (order >= 1) per = std::max(per, p->tr.state_floats);
-    w.state = (float*)(c + off);
-    off += align256((size_t)w.chunk * (size_t)per * 4);
+    int64_t sf = p->fwd.state_floats, zb = p->fwd.zb_elems;
+    if (order >= 1) { sf = std::max(sf, p->tr.state_floats); zb = std::max(zb, p->tr.zb_elems); }
+    w.state = (float*)take((size_t)w.chunk * (size_t)sf * 4);
+    w.zbh = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
+    w.zbl = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
+    if (order >= 1) {
+        w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
+        w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
+    }
     w.bytes = off;
     return w;
 }
@@ -75,10 +92,85 @@ EdgeView sender_view(const sobek_graph* g) {
     return EdgeView{g->src_ptr, g->src_perm, g->col, g->row_ptr, g->N, g->E, 1};
 }
 
+int tc_mask() {
+    static int m = -1;
+    if (m < 0) { const char* e = getenv("SOBEK_TC_MASK"); m = e ? atoi(e) : 7; }
+    return m;
+}
+
 bool has_uncovered(const Direction& d) {
     for (const DGroup& G : d.groups)
         if (G.path_end == G.path_begin) return true;
     return false;
+}
+
+
+// fp32 node state -> bf16 (hi, lo), group by group
+cudaError_t split_state(const Direction& dir, int64_t nn, const float* Z, uint16_t* zh, uint16_t* zl, cudaStream_t s) {
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        cudaError_t e = launch_split(Z + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, dir.nk_ld[gi],
+                                     zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// rows (node, o) of the chunk's output adjoint -> bf16 (hi, lo), group by group
+cudaError_t split_adjoint(const Direction& dir, int64_t n0, int64_t nn, const float* gdst, uint16_t* gh, uint16_t* gl,
+                          cudaStream_t s) {
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        cudaError_t e = launch_split(gdst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst, nn * G.d_dst,
+                                     G.c_dst, dir.kn_ld[gi], gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// dst_g (+)= Z_g * Rp_g        (Eq. receiver_matrix_product)
+cudaError_t mix_tc(const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh, const uint16_t* zl,
+                   const uint16_t* nkh, const uint16_t* nkl, float* dst, int accumulate, int* status, cudaStream_t s) {
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
+                                       nkh + dir.nk_off[gi], nkl + dir.nk_off[gi], dir.nk_ld[gi],
+                                       dst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst,
+                                       nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// Zbar_g = gy_g * Rp_g^T       (Eq. receiver_adjoint)
+cudaError_t state_adjoint_tc(const Direction& dir, int64_t nn, const uint16_t* gh, const uint16_t* gl,
+                             const uint16_t* knh, const uint16_t* knl, float* Zbar, int* status, cudaStream_t s) {
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        cudaError_t e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                                       knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi],
+                                       Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint)
+cudaError_t weight_grad_tc(const Direction& dir, int64_t nn, const uint16_t* zh, const uint16_t* zl,
+                           const uint16_t* gh, const uint16_t* gl, float* gRp, int* status, cudaStream_t s) {
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
+                                       gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                                       gRp + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 1, 1, status, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -112,12 +204,19 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
     if (g->N == 0) return SOBEK_OK;
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
-    CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
+    const bool tc = tc_mask() & 1;
+    if (tc) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+    else CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
     const EdgeView rv = receiver_view(g);
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
         CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, 0, s));
-        CK(launch_mix(p, p->fwd, n0, nn, w.state, w.Rp, y, 0, s));
+        if (tc) {
+            CK(split_state(p->fwd, nn, w.state, w.zbh, w.zbl, s));
+            CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
+        } else {
+            CK(launch_mix(p, p->fwd, n0, nn, w.state, w.Rp, y, 0, s));
+        }
     }
     return SOBEK_OK;
 }
@@ -138,18 +237,27 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
         if (gR) CK(launch_fill_zero(gR, KN, s));
         return SOBEK_OK;
     }
+    const int tcm = tc_mask();
     CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
+    if (tcm & 2) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
     if (gR) CK(launch_fill_zero(w.gRp, KN, s));
     const EdgeView rv = receiver_view(g);
     if (gR || gphi || gY) {
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
+            if (tcm & 6) CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             if (gR) {
                 CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, 0, s));
-                CK(launch_weight_grad(p, p->fwd, n0, nn, w.state, gy, w.gRp, 1, s));
+                if (tcm & 4) {
+                    CK(split_state(p->fwd, nn, w.state, w.zbh, w.zbl, s));
+                    CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
+                } else {
+                    CK(launch_weight_grad(p, p->fwd, n0, nn, w.state, gy, w.gRp, 1, s));
+                }
             }
             if (gphi || gY) {
-                CK(launch_state_adjoint(p, p->fwd, n0, nn, gy, w.Rp, w.state, s));
+                if (tcm & 2) CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.state, w.status, s));
+                else CK(launch_state_adjoint(p, p->fwd, n0, nn, gy, w.Rp, w.state, s));
                 CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, gphi, gY, gphi ? 1 : 0,
                                     gY ? 1 : 0, s));
             }
@@ -158,12 +266,18 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
     if (gx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(gx, g->N * (int64_t)p->C_x, s));
-        CK(launch_pack_R(p, p->tr, 1, R, w.Rt, s));
+        if (tcm & 1) CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
+        else CK(launch_pack_R(p, p->tr, 1, R, w.Rt, s));
         const EdgeView sv = sender_view(g);
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             CK(launch_state(p, p->tr, sv, n0, nn, gy, Y, phi, w.state, 0, s));
-            CK(launch_mix(p, p->tr, n0, nn, w.state, w.Rt, gx, 0, s));
+            if (tcm & 1) {
+                CK(split_state(p->tr, nn, w.state, w.zbh, w.zbl, s));
+                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
+            } else {
+                CK(launch_mix(p, p->tr, n0, nn, w.state, w.Rt, gx, 0, s));
+            }
         }
     }
     return SOBEK_OK;

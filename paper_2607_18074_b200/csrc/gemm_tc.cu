@@ -1,0 +1,384 @@
+// Node-side contractions on the 5th-generation tensor cores (tcgen05, accumulators in TMEM,
+// operands staged by TMA).
+//
+// fp32 parity on bf16 tensor cores: every fp32 operand a is split as a = a_hi + a_lo with
+// a_hi = bf16(a), a_lo = bf16(a - a_hi), and a product is evaluated in three passes
+//     a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo        (fp32 accumulation in TMEM)
+// which leaves a relative error of about 2^-16 per product (the dropped a_lo*b_lo term and the
+// second-order remainders), well inside the 1e-4 / 5e-4 max-norm tolerances.
+//
+// Kernel k_gemm_tc computes  C[M,N] (+)= A[M,Kd] * B[N,Kd]^T  for row-major ("K-major") bf16
+// operands (hi and lo parts), used for
+//     y   = Z  * Rp          (Eq. receiver_matrix_product;  A = Z,  B = Rp^T  [w][k])
+//     Zbar = gy * Rp^T       (Eq. receiver_adjoint;         A = gy, B = Rp    [k][w])
+// and, with MN-major operand descriptors (TRANSPOSED_AB), for the weight adjoint
+//     gRp = Z^T * gy         (Eq. receiver_adjoint;  A^T = Z [r][k],  B^T = gy [r][w]).
+//
+// CTA = 192 threads: warp 0 issues TMA loads, warp 1 allocates TMEM and issues tcgen05.mma,
+// warps 2..5 drain the accumulator (tcgen05.ld) and write C.  Every mbarrier wait is bounded:
+// if it gives up it records SOBEK_ERR_DEVICE_TIMEOUT in the status word and carries on, so the
+// kernel always reaches its TMEM release and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdio.h>
+
+#include "internal.h"
+
+namespace sobek {
+namespace {
+
+// ------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  A healthy wait ends after a handful of polls; the limit only exists so that a
+// broken pipeline cannot spin for ever.  On give-up the status word is set and the caller goes on.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try(bar, parity)) return;
+        if (it > 4096) __nanosleep(256);
+    }
+    atomicExch(status, (int)SOBEK_ERR_DEVICE_TIMEOUT);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// shared-memory operand descriptor (sm_100 format): start address and offsets in 16-byte units,
+// descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;   // version
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+constexpr int BM = 128;     // rows of C per CTA (UMMA M)
+constexpr int BK = 64;      // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int TC_THREADS = 192;
+
+struct TcArgs {
+    float* C;
+    int64_t c_outer, c_inner;   // C(m,n) = C[(m/c_d)*c_outer + (m%c_d)*c_inner + n]
+    int32_t c_d;
+    int32_t accumulate;
+    int64_t M, N, Kd;
+    int32_t BN;                 // tile width (multiple of 16, <= 256)
+    int32_t stages;
+    int32_t tmem_cols;          // power of two >= max(32, BN)
+    int32_t mn_major;           // 0: A[M,Kd], B[N,Kd] row-major;  1: A^T[Kd,M], B^T[Kd,N] row-major
+    int* status;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
+          const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const TcArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the 128-byte swizzle atoms
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t a_bytes = BM * BK * 2;             // 16 KiB
+    const uint32_t b_bytes = (uint32_t)g.BN * BK * 2;
+    const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;
+    uint64_t* bars = (uint64_t*)(smem + (size_t)g.stages * stage_bytes);
+    // bars[0..S) full, bars[S..2S) empty, bars[2S] accumulator ready; then the TMEM base word
+    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * g.stages + 1);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = smem_u32(bars);
+    const int S = g.stages;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * g.BN;
+    const int num_kb = (int)((g.Kd + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(bar0 + 8 * s, 1); mbar_init(bar0 + 8 * (S + s), 1); }
+        mbar_init(bar0 + 8 * 2 * S, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                const uint32_t ph = (kb / S) & 1;
+                mbar_wait(bar0 + 8 * (S + s), ph ^ 1, g.status);        // slot free
+                const uint32_t full = bar0 + 8 * s;
+                mbar_expect_tx(full, stage_bytes);
+                const uint32_t sa = sbase + s * stage_bytes;
+                if (!g.mn_major) {
+                    tma_load_2d(sa, &tmAh, kb * BK, m0, full);
+                    tma_load_2d(sa + a_bytes, &tmAl, kb * BK, m0, full);
+                    tma_load_2d(sa + 2 * a_bytes, &tmBh, kb * BK, n0, full);
+                    tma_load_2d(sa + 2 * a_bytes + b_bytes, &tmBl, kb * BK, n0, full);
+                } else {
+                    // operands stored [Kd rows][M or N contiguous]: boxes of 64 MN-elements x 64 k-rows
+                    for (int j = 0; j < BM / 64; ++j) {
+                        tma_load_2d(sa + j * (64 * BK * 2), &tmAh, m0 + 64 * j, kb * BK, full);
+                        tma_load_2d(sa + a_bytes + j * (64 * BK * 2), &tmAl, m0 + 64 * j, kb * BK, full);
+                    }
+                    for (int j = 0; j < g.BN / 64; ++j) {
+                        tma_load_2d(sa + 2 * a_bytes + j * (64 * BK * 2), &tmBh, n0 + 64 * j, kb * BK, full);
+                        tma_load_2d(sa + 2 * a_bytes + b_bytes + j * (64 * BK * 2), &tmBl, n0 + 64 * j, kb * BK, full);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // instruction descriptor: D = F32, A = B = BF16, M = 128, N = BN
+            uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            if (g.mn_major) idesc |= (1u << 15) | (1u << 16);
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % S;
+                const uint32_t ph = (kb / S) & 1;
+                mbar_wait(bar0 + 8 * s, ph, g.status);                  // operands landed
+                tc_fence_after();
+                const uint32_t sa = sbase + s * stage_bytes;
+                const uint32_t ah = sa, al = sa + a_bytes, bh = sa + 2 * a_bytes, bl = bh + b_bytes;
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k) {
+                    uint64_t dAh, dAl, dBh, dBl;
+                    if (!g.mn_major) {
+                        // K-major: rows of 128 B, 8-row groups 1024 B apart; 16 k-elements = 32 B
+                        dAh = make_desc(ah + 32 * k, 16, 1024); dAl = make_desc(al + 32 * k, 16, 1024);
+                        dBh = make_desc(bh + 32 * k, 16, 1024); dBl = make_desc(bl + 32 * k, 16, 1024);
+                    } else {
+                        // MN-major: 64 MN-elements per 128-B row, 8 k-rows per 1024-B group (stride),
+                        // next 64 MN-elements one box further (leading); 16 k = two groups
+                        dAh = make_desc(ah + 2048 * k, 64 * BK * 2, 1024); dAl = make_desc(al + 2048 * k, 64 * BK * 2, 1024);
+                        dBh = make_desc(bh + 2048 * k, 64 * BK * 2, 1024); dBl = make_desc(bl + 2048 * k, 64 * BK * 2, 1024);
+                    }
+                    const uint32_t first = (kb > 0 || k > 0) ? 1u : 0u;
+                    tc_mma_bf16(tmem_base, dAh, dBh, idesc, first);
+                    tc_mma_bf16(tmem_base, dAl, dBh, idesc, 1u);
+                    tc_mma_bf16(tmem_base, dAh, dBl, idesc, 1u);
+                }
+                tc_commit(bar0 + 8 * (S + s));                           // frees the slot when the MMAs retire
+            }
+            tc_commit(bar0 + 8 * 2 * S);                                 // accumulator complete
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+        const int q = warp & 3;
+        mbar_wait(bar0 + 8 * 2 * S, 0, g.status);
+        tc_fence_after();
+        const int64_t m = (int64_t)m0 + q * 32 + lane;
+        float* crow = nullptr;
+        if (m < g.M) crow = g.C + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+        for (int c0 = 0; c0 < g.BN; c0 += 16) {
+            float v[16];
+            tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);   // warp-collective
+            if (crow) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int64_t n = (int64_t)n0 + c0 + j;
+                    if (n < g.N) crow[n] = g.accumulate ? crow[n] + v[j] : v[j];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// fp32 -> (bf16 hi, bf16 lo) with mapped source rows: dst[r*ld + c] for r < rows, c < cols
+// ------------------------------------------------------------------------------------
+__global__ void k_split(const float* __restrict__ src, int64_t s_outer, int64_t s_inner, int s_d,
+                        int64_t rows, int cols, int64_t ld, __nv_bfloat16* __restrict__ hi,
+                        __nv_bfloat16* __restrict__ lo) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols;
+        const int c = (int)(i - r * cols);
+        const float v = src[(r / s_d) * s_outer + (r % s_d) * s_inner + c];
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[r * ld + c] = h;
+        lo[r * ld + c] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// R[K, N_w] -> bf16 hi/lo GEMM operands of one direction, per group g:
+//   layout KN (n_major = 0): [k][c_dst] rows of length ldn_g      (B operand of Zbar = gy Rp^T)
+//   layout NK (n_major = 1): [c_dst][k] rows of length ldk_g      (B operand of y = Z Rp)
+__global__ void k_pack_R_bf16(const DPath* __restrict__ paths, const int64_t* __restrict__ grp_off,
+                              const int32_t* __restrict__ grp_ld, const int32_t* __restrict__ path_group,
+                              int transposed, int n_major, int K, int64_t N_w, const float* __restrict__ R,
+                              __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    const DPath P = paths[blockIdx.y];
+    const int gi = path_group[blockIdx.y];
+    const int64_t base = grp_off[gi];
+    const int64_t ld = grp_ld[gi];
+    const int64_t total = (int64_t)K * P.c_src * P.c_dst;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(i % P.c_dst);
+        const int64_t r = i / P.c_dst;
+        const int q = (int)(r % K);
+        const int us = (int)(r / K);
+        const int u = transposed ? n : us, w = transposed ? us : n;
+        const float v = R[(int64_t)q * N_w + P.w_off + (int64_t)u * P.c_out + w];
+        const int64_t k = (int64_t)P.koff + (int64_t)us * K + q;
+        const int64_t o = n_major ? base + (int64_t)n * ld + k : base + k * ld + n;
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[o] = h;
+        lo[o] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// ------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeFn)p;
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows][inner] with row pitch ld elements; box = box_inner x box_rows; 128-B swizzle
+bool make_map(CUtensorMap* tm, const void* ptr, int64_t inner, int64_t rows, int64_t ld, int box_inner, int box_rows) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows};
+    cuuint32_t es[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int64_t round8(int64_t v) { return (v + 7) & ~int64_t(7); }
+
+cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int s_d, int64_t rows, int cols,
+                         int64_t ld, void* hi, void* lo, cudaStream_t s) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    const int64_t total = rows * cols;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
+    KernelTimer kt(K_PACK, s);
+    k_split<<<blocks, 256, 0, s>>>(src, s_outer, s_inner, s_d, rows, cols, ld, (__nv_bfloat16*)hi, (__nv_bfloat16*)lo);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int transposed, int n_major,
+                               const float* R, void* hi, void* lo, cudaStream_t s) {
+    dim3 grid(32, (unsigned)dir.paths.size());
+    KernelTimer kt(K_PACK, s);
+    k_pack_R_bf16<<<grid, 256, 0, s>>>(dir.d_paths, n_major ? dir.d_nk_off : dir.d_kn_off,
+                                       n_major ? dir.d_nk_ld : dir.d_kn_ld, dir.d_path_group, transposed, n_major,
+                                       p->K, p->N_w, R, (__nv_bfloat16*)hi, (__nv_bfloat16*)lo);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// C[M,N] (+)= A * B^T on tensor cores.  mn_major = 0: A[M][lda], B[N][ldb] (rows contiguous in k).
+// mn_major = 1: A^T[Kd][lda] (contiguous in m), B^T[Kd][ldb] (contiguous in n).
+cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
+                           int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
+                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s) {
+    if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
+    TcArgs g{};
+    g.C = C; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate;
+    g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
+    int BN;
+    if (mn_major) BN = N <= 64 ? 64 : (N <= 128 ? 128 : 256);     // whole 64-wide boxes
+    else BN = (int)std::min<int64_t>(256, (N + 15) / 16 * 16);
+    g.BN = BN;
+    const size_t stage = 2 * (size_t)BM * BK * 2 + 2 * (size_t)BN * BK * 2;
+    int stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
+    g.stages = std::max(stages, 2);
+    int cols = 32;
+    while (cols < BN) cols <<= 1;
+    g.tmem_cols = cols;
+    CUtensorMap tAh, tAl, tBh, tBl;
+    bool ok;
+    if (!mn_major) {
+        ok = make_map(&tAh, Ahi, Kd, M, lda, BK, BM) && make_map(&tAl, Alo, Kd, M, lda, BK, BM) &&
+             make_map(&tBh, Bhi, Kd, N, ldb, BK, BN) && make_map(&tBl, Blo, Kd, N, ldb, BK, BN);
+    } else {
+        ok = make_map(&tAh, Ahi, M, Kd, lda, 64, BK) && make_map(&tAl, Alo, M, Kd, lda, 64, BK) &&
+             make_map(&tBh, Bhi, N, Kd, ldb, 64, BK) && make_map(&tBl, Blo, N, Kd, ldb, 64, BK);
+    }
+    if (!ok) return cudaErrorInvalidValue;
+    const size_t sh = (size_t)g.stages * stage + 1024 + 8 * (2 * g.stages + 1) + 16;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN));
+    KernelTimer kt(K_GEMM, s);
+    k_gemm_tc<<<grid, TC_THREADS, sh, s>>>(tAh, tAl, tBh, tBl, g);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace sobek

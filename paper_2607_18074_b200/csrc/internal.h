@@ -64,10 +64,20 @@ struct Direction {
     int64_t state_floats = 0;   // per node: sum_g d*D
     int32_t max_m_entries = 0;
     int32_t C_src = 0, C_dst = 0;
+    // bf16 operand layouts (element offsets / leading dimensions per group; groups without paths get 0)
+    //   KN: [k][c_dst], ld = round8(c_dst)   NK: [c_dst][k], ld = round8(D)
+    std::vector<int64_t> kn_off, nk_off;
+    std::vector<int32_t> kn_ld, nk_ld, path_group;
+    int64_t kn_elems = 0, nk_elems = 0;
+    std::vector<int64_t> zb_off;      // per node, elements: sum_{g'<g} d * round8(D)     (bf16 state rows)
+    std::vector<int64_t> gb_off;      // per node, elements: sum_{g'<g} d * round8(c_dst) (bf16 adjoint rows)
+    int64_t zb_elems = 0, gb_elems = 0;
     // device copies
     DPath* d_paths = nullptr;
     DGroup* d_groups = nullptr;
     WTask* d_wtasks = nullptr;
+    int64_t *d_kn_off = nullptr, *d_nk_off = nullptr;
+    int32_t *d_kn_ld = nullptr, *d_nk_ld = nullptr, *d_path_group = nullptr;
 };
 
 struct HPath {
@@ -153,6 +163,16 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
                              int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
                              cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
+
+// --- gemm_tc.cu ---------------------------------------------------------------------
+int64_t round8(int64_t v);
+cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int s_d, int64_t rows, int cols,
+                         int64_t ld, void* hi, void* lo, cudaStream_t s);
+cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int transposed, int n_major,
+                               const float* R, void* hi, void* lo, cudaStream_t s);
+cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
+                           int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
+                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s);
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);

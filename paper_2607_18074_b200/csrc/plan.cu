@@ -345,14 +345,31 @@ void build_direction(sobek_plan* p, int transposed, Direction& dir) {
         dir.groups.push_back(G);   // groups without paths are kept (their block is zero-filled)
     }
     dir.state_floats = z_off;
+    // bf16 operand layouts
+    auto r8 = [](int64_t v) { return (v + 7) & ~int64_t(7); };
+    dir.path_group.assign(dir.paths.size(), 0);
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        dir.kn_off.push_back(dir.kn_elems); dir.nk_off.push_back(dir.nk_elems);
+        dir.kn_ld.push_back((int32_t)r8(G.c_dst)); dir.nk_ld.push_back((int32_t)r8(G.D));
+        dir.zb_off.push_back(dir.zb_elems); dir.gb_off.push_back(dir.gb_elems);
+        if (G.path_end == G.path_begin) continue;
+        dir.kn_elems += int64_t(G.D) * r8(G.c_dst);
+        dir.nk_elems += int64_t(G.c_dst) * r8(G.D);
+        dir.zb_elems += int64_t(G.d_dst) * r8(G.D);
+        dir.gb_elems += int64_t(G.d_dst) * r8(G.c_dst);
+        for (int k = G.path_begin; k < G.path_end; ++k) dir.path_group[k] = (int32_t)gi;
+    }
 }
 
 }  // namespace
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order) {
-    int64_t per = p->fwd.state_floats;
-    if (order >= 1) per = std::max(per, p->tr.state_floats);
-    per = std::max<int64_t>(per, 1) * 4;
+    // per node: fp32 state + its bf16 (hi, lo) split + (orders >= 1) the split output-adjoint rows
+    int64_t sf = p->fwd.state_floats, zb = p->fwd.zb_elems;
+    if (order >= 1) { sf = std::max(sf, p->tr.state_floats); zb = std::max(zb, p->tr.zb_elems); }
+    int64_t per = 4 * sf + 4 * zb + (order >= 1 ? 4 * p->fwd.gb_elems : 0);
+    per = std::max<int64_t>(per, 1);
     int64_t n = (int64_t)(kStateBudgetBytes / (size_t)per);
     n = std::max<int64_t>(n, 1);
     return std::min<int64_t>(std::max<int64_t>(N, 1), n);
@@ -440,6 +457,11 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         if (e == cudaSuccess) e = upload(d->paths, &d->d_paths);
         if (e == cudaSuccess) e = upload(d->groups, &d->d_groups);
         if (e == cudaSuccess) e = upload(d->wtasks, &d->d_wtasks);
+        if (e == cudaSuccess) e = upload(d->kn_off, &d->d_kn_off);
+        if (e == cudaSuccess) e = upload(d->nk_off, &d->d_nk_off);
+        if (e == cudaSuccess) e = upload(d->kn_ld, &d->d_kn_ld);
+        if (e == cudaSuccess) e = upload(d->nk_ld, &d->d_nk_ld);
+        if (e == cudaSuccess) e = upload(d->path_group, &d->d_path_group);
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -453,7 +475,10 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
 extern "C" void sobek_plan_destroy(sobek_plan* p) {
     if (!p) return;
     cudaFree(p->d_tab_ptr); cudaFree(p->d_tab_idx); cudaFree(p->d_tab_coef);
-    for (Direction* d : {&p->fwd, &p->tr}) { cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks); }
+    for (Direction* d : {&p->fwd, &p->tr}) {
+        cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);
+        cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);
+    }
     (void)cudaGetLastError();
     delete p;
 }
