@@ -177,7 +177,7 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
  * sobek_conv_fwd takes from the caller lives in a fixed array inside the library image:
  * sobek_static_scratch_bytes() bytes (32 MiB) on every GPU that loads the library, held until the
  * process exits.  The call makes no cudaMalloc / cudaFree and calls no allocating routine.
- *   - Limit: 256 + 4*K*N_w (rounded up to 256) + 4*K*F bytes must fit in the array, K*F being
+ *   - Limit: about 4*K*N_w + 4*K*F bytes (plus padding) must fit in the array, K*F being
  *     sobek_info.state_floats_fwd (the state of a single node); otherwise SOBEK_ERR_WORKSPACE is
  *     returned and nothing is launched.  Larger graphs only mean more node chunks.
  *   - The first call on a device looks up the array's device address (with that device

@@ -1,40 +1,51 @@
-"""Builds libsobek.so (sm_100a) in-tree with nvcc."""
+"""Builds libsobek.so (sm_100a) in-tree with nvcc: one object per source, compiled in parallel."""
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libsobek.so")
-SOURCES = ["plan.cu", "graph.cu", "kernels.cu", "gemm_tc.cu", "api.cu", "static_scratch.cu"]
+SOURCES = ["plan.cu", "graph.cu", "kernels.cu", "edge_stream.cu", "edge_stream_k8.cu", "edge_stream_k8d.cu",
+           "edge_stream_k16.cu", "edge_stream_k16d.cu", "gemm_tc.cu", "api.cu", "static_scratch.cu"]
+FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
+         "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 
-def nvcc_cmd(verbose_ptxas: bool = False):
-    cmd = ["nvcc", "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB]
-    if verbose_ptxas:
-        cmd += ["-Xptxas", "-v"]
-    return cmd + [os.path.join(CSRC, s) for s in SOURCES]
+def _headers():
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))] + \
+           [os.path.join(ROOT, "include", "sobek.h")]
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "sobek.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+def _compile(src: str, force: bool, verbose_ptxas: bool) -> str:
+    obj = os.path.join(OBJ, src.replace(".cu", ".o"))
+    path = os.path.join(CSRC, src)
+    deps = [path] + _headers()
+    if not force and os.path.exists(obj) and all(os.path.getmtime(d) <= os.path.getmtime(obj) for d in deps):
+        return obj
+    cmd = ["nvcc"] + FLAGS + (["-Xptxas", "-v"] if verbose_ptxas else []) + ["-c", path, "-o", obj]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    if verbose_ptxas or r.returncode != 0:
+        sys.stderr.write(r.stdout + r.stderr)
+    if r.returncode != 0:
+        raise RuntimeError(f"nvcc failed on {src}")
+    return obj
 
 
 def build(force: bool = False, verbose_ptxas: bool = False) -> str:
-    if force or stale():
-        subprocess.check_call(nvcc_cmd(verbose_ptxas))
+    os.makedirs(OBJ, exist_ok=True)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        objs = list(ex.map(lambda s: _compile(s, force, verbose_ptxas), SOURCES))
+    if force or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
+        subprocess.check_call(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + objs)
     return LIB
 
 
 if __name__ == "__main__":
-    build(force=True, verbose_ptxas="-v" in sys.argv)
+    build(force="-f" in sys.argv, verbose_ptxas="-v" in sys.argv)
     print(LIB)

@@ -1,8 +1,6 @@
 // C-ABI entry points: argument checks, workspace carving and the launch schedules of
 // forward, backward and double backward.  Everything here only enqueues work on the
 // caller's stream.
-#include <stdlib.h>
-
 #include <algorithm>
 
 #include "internal.h"
@@ -21,10 +19,9 @@ struct Workspace {
     uint16_t *tNKh, *tNKl;    // sender direction,   [u][k']  (gx = V Rt)
     uint16_t *vfNKh, *vfNKl, *vfKNh, *vfKNl, *vtNKh, *vtNKl;   // the same for vR
     float* gRp;               // fp32 accumulator of the R adjoint, packed [k][w] per group
-    float *Rp, *Rt, *vRp, *vRt;   // DEBUG: fp32 packs for the SIMT GEMM
-    float* state;             // fp32 node state of one chunk (Z / Zbar / V)
-    uint16_t *zbh, *zbl;      // bf16 split of the node state of one chunk
-    uint16_t *gbh, *gbl;      // bf16 split of the chunk's output-adjoint rows
+    float* zbar;              // fp32 adjoint state Zbar of one chunk (input of the edge pass)
+    uint16_t *zbh, *zbl;      // bf16 (hi, lo) node state Z / dZ / V of one chunk
+    uint16_t *gbh, *gbl;      // bf16 (hi, lo) rows of the chunk's output adjoint
     int64_t chunk;
     size_t bytes;
 };
@@ -46,17 +43,13 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         w.vfKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.vfKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
         w.vtNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.vtNKl = (uint16_t*)take(p->tr.nk_elems * 2);
     }
-    {
-        const size_t rb = (size_t)p->K * (size_t)p->N_w * 4;
-        w.Rp = (float*)take(rb); w.Rt = (float*)take(rb); w.vRp = (float*)take(rb); w.vRt = (float*)take(rb);
-    }
     w.chunk = chunk_nodes(p, N, order);
-    int64_t sf = p->fwd.state_floats, zb = p->fwd.zb_elems;
-    if (order >= 1) { sf = std::max(sf, p->tr.state_floats); zb = std::max(zb, p->tr.zb_elems); }
-    w.state = (float*)take((size_t)w.chunk * (size_t)sf * 4);
+    int64_t zb = p->fwd.zb_elems;
+    if (order >= 1) zb = std::max(zb, p->tr.zb_elems);
     w.zbh = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
     w.zbl = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
     if (order >= 1) {
+        w.zbar = (float*)take((size_t)w.chunk * (size_t)p->fwd.state_floats * 4);
         w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
         w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
     }
@@ -92,30 +85,12 @@ EdgeView sender_view(const sobek_graph* g) {
     return EdgeView{g->src_ptr, g->src_perm, g->col, g->row_ptr, g->N, g->E, 1};
 }
 
-int tc_mask() {
-    static int m = -1;
-    if (m < 0) { const char* e = getenv("SOBEK_TC_MASK"); m = e ? atoi(e) : 7; }
-    return m;
-}
-
 bool has_uncovered(const Direction& d) {
     for (const DGroup& G : d.groups)
         if (G.path_end == G.path_begin) return true;
     return false;
 }
 
-
-// fp32 node state -> bf16 (hi, lo), group by group
-cudaError_t split_state(const Direction& dir, int64_t nn, const float* Z, uint16_t* zh, uint16_t* zl, cudaStream_t s) {
-    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        const DGroup& G = dir.groups[gi];
-        if (G.path_end == G.path_begin) continue;
-        cudaError_t e = launch_split(Z + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, dir.nk_ld[gi],
-                                     zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], s);
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
-}
 
 // rows (node, o) of the chunk's output adjoint -> bf16 (hi, lo), group by group
 cudaError_t split_adjoint(const Direction& dir, int64_t n0, int64_t nn, const float* gdst, uint16_t* gh, uint16_t* gl,
@@ -204,19 +179,12 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
     if (g->N == 0) return SOBEK_OK;
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
-    const bool tc = tc_mask() & 1;
-    if (tc) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
-    else CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
+    CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     const EdgeView rv = receiver_view(g);
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
-        CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, 0, s));
-        if (tc) {
-            CK(split_state(p->fwd, nn, w.state, w.zbh, w.zbl, s));
-            CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
-        } else {
-            CK(launch_mix(p, p->fwd, n0, nn, w.state, w.Rp, y, 0, s));
-        }
+        CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+        CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
     }
     return SOBEK_OK;
 }
@@ -237,47 +205,33 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
         if (gR) CK(launch_fill_zero(gR, KN, s));
         return SOBEK_OK;
     }
-    const int tcm = tc_mask();
-    CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
-    if (tcm & 2) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
-    if (gR) CK(launch_fill_zero(w.gRp, KN, s));
     const EdgeView rv = receiver_view(g);
     if (gR || gphi || gY) {
+        if (gphi || gY) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
+        if (gR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            if (tcm & 6) CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
-            if (gR) {
-                CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, 0, s));
-                if (tcm & 4) {
-                    CK(split_state(p->fwd, nn, w.state, w.zbh, w.zbl, s));
-                    CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
-                } else {
-                    CK(launch_weight_grad(p, p->fwd, n0, nn, w.state, gy, w.gRp, 1, s));
-                }
+            CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
             }
             if (gphi || gY) {
-                if (tcm & 2) CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.state, w.status, s));
-                else CK(launch_state_adjoint(p, p->fwd, n0, nn, gy, w.Rp, w.state, s));
-                CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, gphi, gY, gphi ? 1 : 0,
+                CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, gphi, gY, gphi ? 1 : 0,
                                     gY ? 1 : 0, s));
             }
         }
+        if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
     }
-    if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
     if (gx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(gx, g->N * (int64_t)p->C_x, s));
-        if (tcm & 1) CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
-        else CK(launch_pack_R(p, p->tr, 1, R, w.Rt, s));
+        CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
         const EdgeView sv = sender_view(g);
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            CK(launch_state(p, p->tr, sv, n0, nn, gy, Y, phi, w.state, 0, s));
-            if (tcm & 1) {
-                CK(split_state(p->tr, nn, w.state, w.zbh, w.zbl, s));
-                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
-            } else {
-                CK(launch_mix(p, p->tr, n0, nn, w.state, w.Rt, gx, 0, s));
-            }
+            CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+            CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
         }
     }
     return SOBEK_OK;
@@ -309,83 +263,79 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
         if ((rc = zero_out(hR, KN))) return rc;
         return SOBEK_OK;
     }
-    if (!(any_edge_dir || vR)) {
-        if ((rc = zero_out(ggy, g->N * (int64_t)p->C_y))) return rc;
-    }
+    if (!(any_edge_dir || vR)) { if ((rc = zero_out(ggy, g->N * (int64_t)p->C_y))) return rc; }
     if (!any_edge_dir) { if ((rc = zero_out(hR, KN))) return rc; }
     if (!(vx || vY || vR)) { if ((rc = zero_out(hphi, g->E * (int64_t)p->K))) return rc; }
     if (!(vx || vphi || vR)) { if ((rc = zero_out(hY, g->E * (int64_t)p->dim_sh))) return rc; }
     if (!(vY || vphi || vR)) { if ((rc = zero_out(hx, g->N * (int64_t)p->C_x))) return rc; }
 
-    CK(launch_pack_R(p, p->fwd, 0, R, w.Rp, s));
-    if (vR) CK(launch_pack_R(p, p->fwd, 0, vR, w.vRp, s));
-    if (hR) CK(launch_fill_zero(w.gRp, KN, s));
     const EdgeView rv = receiver_view(g);
-    if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
-
     if (ggy || hR || hphi || hY) {
+        if (ggy && any_edge_dir) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+        if (ggy && vR) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
+        if ((hphi || hY) && any_edge_dir) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
+        if ((hphi || hY) && vR) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl, s));
+        if (hR) CK(launch_fill_zero(w.gRp, KN, s));
+        if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint, d(gy) = 0)
+            if (hR || hphi || hY) CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint with d(gy) = 0)
             int ggy_written = 0;
             if (ggy && vR) {
-                CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, 0, s));
-                CK(launch_mix(p, p->fwd, n0, nn, w.state, w.vRp, ggy, 0, s));
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
                 ggy_written = 1;
             }
             if ((ggy || hR) && any_edge_dir) {
-                int acc = 0;   // dZ = Z(vx,Y,phi) + Z(x,vY,phi) + Z(x,Y,vphi)
-                if (vx) { CK(launch_state(p, p->fwd, rv, n0, nn, vx, Y, phi, w.state, acc, s)); acc = 1; }
-                if (vY) { CK(launch_state(p, p->fwd, rv, n0, nn, x, vY, phi, w.state, acc, s)); acc = 1; }
-                if (vphi) { CK(launch_state(p, p->fwd, rv, n0, nn, x, Y, vphi, w.state, acc, s)); acc = 1; }
-                if (ggy) CK(launch_mix(p, p->fwd, n0, nn, w.state, w.Rp, ggy, ggy_written, s));
-                if (hR) CK(launch_weight_grad(p, p->fwd, n0, nn, w.state, gy, w.gRp, 1, s));
+                // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
+                if (ggy) CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
+                if (hR) CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
             }
             if (hphi || hY) {
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate
                 if (any_edge_dir) {
-                    CK(launch_state_adjoint(p, p->fwd, n0, nn, gy, w.Rp, w.state, s));
+                    CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
                     if (vx) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, vx, Y, phi, w.state, hphi, hY,
+                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, vx, Y, phi, w.zbar, hphi, hY,
                                             hphi ? pm : 0, hY ? ym : 0, s));
                         pm = ym = 2;
                     }
                     if (vY && hphi) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vY, phi, w.state, hphi, hY, pm, 0, s));
+                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vY, phi, w.zbar, hphi, hY, pm, 0, s));
                         pm = 2;
                     }
                     if (vphi && hY) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, vphi, w.state, hphi, hY, 0, ym, s));
+                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, vphi, w.zbar, hphi, hY, 0, ym, s));
                         ym = 2;
                     }
                 }
                 if (vR) {
-                    CK(launch_state_adjoint(p, p->fwd, n0, nn, gy, w.vRp, w.state, s));
-                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.state, hphi, hY, hphi ? pm : 0,
+                    CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
+                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, hphi, hY, hphi ? pm : 0,
                                         hY ? ym : 0, s));
                 }
             }
         }
+        if (hR) CK(launch_unpack_R(p, p->fwd, w.gRp, hR, s));
     }
-    if (hR) CK(launch_unpack_R(p, p->fwd, w.gRp, hR, s));
     if (hx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(hx, g->N * (int64_t)p->C_x, s));
-        CK(launch_pack_R(p, p->tr, 1, R, w.Rt, s));
-        if (vR) CK(launch_pack_R(p, p->tr, 1, vR, w.vRt, s));
+        if (vY || vphi) CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
+        if (vR) CK(launch_pack_R_bf16(p, p->tr, 1, 1, vR, w.vtNKh, w.vtNKl, s));
         const EdgeView sv = sender_view(g);
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             int wrote = 0;
-            if (vY || vphi) {
-                int acc = 0;
-                if (vY) { CK(launch_state(p, p->tr, sv, n0, nn, gy, vY, phi, w.state, acc, s)); acc = 1; }
-                if (vphi) { CK(launch_state(p, p->tr, sv, n0, nn, gy, Y, vphi, w.state, acc, s)); acc = 1; }
-                CK(launch_mix(p, p->tr, n0, nn, w.state, w.Rt, hx, 0, s));
+            if (vY || vphi) {   // dV = V(gy; vY, phi) + V(gy; Y, vphi) in one pass
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
+                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, hx, 0, w.status, s));
                 wrote = 1;
             }
             if (vR) {
-                CK(launch_state(p, p->tr, sv, n0, nn, gy, Y, phi, w.state, 0, s));
-                CK(launch_mix(p, p->tr, n0, nn, w.state, w.vRt, hx, wrote, s));
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, hx, wrote, w.status, s));
             }
         }
     }

@@ -56,6 +56,16 @@ struct WTask {         // one warp's share of a group: 32 consecutive multiplici
     int32_t u0;
 };
 
+struct STask {         // one warp's task of the edge stream
+    int32_t path;
+    int32_t u0;        // first multiplicity of the block (32*ub wide)
+    int32_t o0, oc;    // chunk of output components [o0, o0+oc)
+    int32_t ub;        // multiplicities per lane
+    int32_t cls;       // 3*index(OC in {1,3,4,5}) + index(UB in {1,2,4})
+    int32_t group;
+    int32_t pad;
+};
+
 struct Direction {
     // host copies
     std::vector<DPath> paths;
@@ -72,6 +82,12 @@ struct Direction {
     std::vector<int64_t> zb_off;      // per node, elements: sum_{g'<g} d * round8(D)     (bf16 state rows)
     std::vector<int64_t> gb_off;      // per node, elements: sum_{g'<g} d * round8(c_dst) (bf16 adjoint rows)
     int64_t zb_elems = 0, gb_elems = 0;
+    std::vector<STask> stasks;        // sorted by kernel class
+    struct SClass { int cls, begin, count; };
+    std::vector<SClass> sclasses;
+    int32_t ms_max = 4;               // row pitch (floats) of the per-edge M stage
+    STask* d_stasks = nullptr;
+    int64_t* d_zb_off = nullptr;
     // device copies
     DPath* d_paths = nullptr;
     DGroup* d_groups = nullptr;
@@ -138,24 +154,8 @@ struct EdgeView {          // how a traversal walks the graph
     int transposed;        // 0: source node = col[e];  1: source node = receiver(e)
 };
 
-cudaError_t launch_pack_R(const sobek_plan* p, const Direction& dir, int transposed, const float* R,
-                          float* Rp, cudaStream_t s);
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s);
-cudaError_t launch_state(const sobek_plan* p, const Direction& dir, const EdgeView& ev,
-                         int64_t node0, int64_t n_nodes, const float* src, const float* Y,
-                         const float* phi, float* Z, int accumulate, cudaStream_t s);
-// y_g = Z_g * Rp_g  for every group (C written through the node/component row map)
-cudaError_t launch_mix(const sobek_plan* p, const Direction& dir, int64_t node0, int64_t n_nodes,
-                       const float* Z, const float* Rp, float* dst, int accumulate, cudaStream_t s);
-// Zbar_g = gy_g * Rp_g^T
-cudaError_t launch_state_adjoint(const sobek_plan* p, const Direction& dir, int64_t node0,
-                                 int64_t n_nodes, const float* gdst, const float* Rp, float* Zbar,
-                                 cudaStream_t s);
-// gRp_g (+)= Z_g^T * gy_g
-cudaError_t launch_weight_grad(const sobek_plan* p, const Direction& dir, int64_t node0,
-                               int64_t n_nodes, const float* Z, const float* gdst, float* gRp,
-                               int accumulate, cudaStream_t s);
 // receiver-owned edge pass: gphi_e = <Zbar, C_e>, gY_e = CG^T_Y(x, phi_e Zbar)
 cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev,
                              int64_t node0, int64_t n_nodes, const float* src, const float* Y,
@@ -163,6 +163,26 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
                              int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
                              cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
+
+// --- edge_stream.cu ---------------------------------------------------------------
+void build_stream_tasks(const sobek_plan* p, Direction& dir);
+cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
+                          int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
+                          const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s);
+
+#define SOBEK_STREAM_DECL(name)                                                                              \
+    cudaError_t name(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,           \
+                     int64_t n_nodes, const float* src, const float* Y, const float* phi, void* zh, void* zl, \
+                     int cls, int t_begin, int t_count, cudaStream_t s)
+#define SOBEK_STREAM_DECL_DUAL(name)                                                                         \
+    cudaError_t name(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,           \
+                     int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,  \
+                     const float* phi, const float* vphi, void* zh, void* zl, int cls, int t_begin,           \
+                     int t_count, cudaStream_t s)
+SOBEK_STREAM_DECL(stream_launch_k8);
+SOBEK_STREAM_DECL(stream_launch_k16);
+SOBEK_STREAM_DECL_DUAL(stream_launch_k8_dual);
+SOBEK_STREAM_DECL_DUAL(stream_launch_k16_dual);
 
 // --- gemm_tc.cu ---------------------------------------------------------------------
 int64_t round8(int64_t v);

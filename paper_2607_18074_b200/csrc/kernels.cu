@@ -1,16 +1,10 @@
 // Device kernels of the streaming convolution (sm_100a).
 //
-//   k_pack_R / k_unpack_R : re-layout of the radial projection R[K, N_w] into per-group
-//                           GEMM operands  Rp_g[(pi,u,q), w]  (and back, for gR)
-//   k_state               : edge stream.  For one destination node and one group it folds
-//                           every incident edge into the bounded state
-//                           Z[pi,u,q,o] = sum_e phi_e[q] * C_e[pi,u,o]     (Eq. receiver_state)
-//                           with C_e the angular contraction (Eq. angular_path_contraction).
-//                           The same kernel serves the sender-owned transposed traversal.
-//   k_gemm                : node-side contractions  y = Z Rp,  Zbar = gy Rp^T,  gRp += Z^T gy
-//                           (Eqs. receiver_matrix_product, receiver_adjoint)
+//   k_pack_R<UNPACK>      : the accumulated R adjoint, kept per group as gRp_g[(pi,u,q), w],
+//                           back into the layout of R[K, N_w]
 //   k_edge_pass           : receiver-owned edge derivatives gphi_e, gY_e
 //                           (Section "Receiver-factorized backward")
+// (the edge stream lives in edge_stream*.cu, the node-side contractions in gemm_tc.cu)
 #include <stdio.h>
 
 #include <atomic>
@@ -120,219 +114,6 @@ __global__ void k_pack_R(const DPath* __restrict__ paths, int transposed, int K,
         const int64_t ri = (int64_t)q * N_w + P.w_off + (int64_t)u * P.c_out + w;
         const int64_t pi = P.rp_off + ((int64_t)P.koff + (int64_t)us * K + q) * P.c_dst + n;
         if (UNPACK) dst[ri] = src[pi]; else dst[pi] = src[ri];
-    }
-}
-
-// ------------------------------------------------------------------------------------
-// Edge stream.
-// grid = (n_nodes, ceil(wtasks_of_group / WARPS)), block = WARPS*32 threads.
-// Each warp owns one (path, 32 multiplicities) task: lane <-> multiplicity u.  The CTA walks
-// the node's edge segment in batches of EB edges; per batch it stages the edge operands
-// (source node, Y row, phi row) in shared memory, expands M[s][o] = sum_b c Y_b for the
-// paths it needs, and every lane then accumulates, for its u,
-//     C[o]      = sum_s xs[s] * M[s][o]
-//     acc[o][q] += phi[q] * C[o]
-// No atomics: each Z element has one owning thread, edges are taken in segment order.
-// ------------------------------------------------------------------------------------
-constexpr int ST_WARPS = 8;
-constexpr int ST_EB = 16;
-
-struct StateArgs {
-    const DPath* paths;
-    const WTask* wtasks;
-    const int32_t* tab_ptr;
-    const int32_t* tab_idx;
-    const float* tab_coef;
-    DGroup G;
-    EdgeView ev;
-    int64_t node0, n_nodes;
-    const float* src;
-    const float* Y;
-    const float* phi;
-    float* Z;       // chunk buffer; group region at n_nodes*G.z_off, row stride G.D
-    int K, dsh, C_src, accumulate, m_stride;
-};
-
-template <int D_DST, int KC>
-__global__ void __launch_bounds__(ST_WARPS * 32) k_state(const StateArgs a) {
-    extern __shared__ float smem[];
-    float* sM = smem;                                  // [EB][m_stride]
-    float* sY = sM + ST_EB * a.m_stride;               // [EB][dsh]
-    float* sPhi = sY + ST_EB * a.dsh;                  // [EB][KC]
-    int64_t* sSrc = (int64_t*)(sPhi + ST_EB * KC);     // [EB] (8-byte aligned: sizes are even)
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int wt0 = a.G.wt_begin + blockIdx.y * ST_WARPS;
-    const int wt1 = min(wt0 + ST_WARPS, a.G.wt_end);
-    const bool has_task = wt0 + warp < wt1;
-    const int pb = a.wtasks[wt0].path, pe = a.wtasks[wt1 - 1].path + 1;   // paths this CTA needs
-    WTask wt = has_task ? a.wtasks[wt0 + warp] : WTask{pb, 0};
-    const DPath P = a.paths[wt.path];
-    const int u = wt.u0 + lane;
-    const bool active = has_task && u < P.c_src;
-
-    const int64_t node = a.node0 + blockIdx.x;
-    const int64_t seg0 = a.ev.ptr[node], seg1 = a.ev.ptr[node + 1];
-
-    for (int q0 = 0; q0 < a.K; q0 += KC) {
-        float acc[D_DST][KC];
-#pragma unroll
-        for (int o = 0; o < D_DST; ++o)
-#pragma unroll
-            for (int q = 0; q < KC; ++q) acc[o][q] = 0.f;
-
-        for (int64_t b0 = seg0; b0 < seg1; b0 += ST_EB) {
-            const int nb = (int)min((int64_t)ST_EB, seg1 - b0);
-            __syncthreads();
-            // ---- stage edge operands
-            for (int i = threadIdx.x; i < nb; i += blockDim.x) {
-                const int64_t pos = b0 + i;
-                const int64_t e = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
-                sSrc[i] = a.ev.transposed ? owner_of_edge(a.ev.row_ptr, a.ev.N, e) : (int64_t)a.ev.col[e];
-            }
-            for (int i = threadIdx.x; i < nb * a.dsh; i += blockDim.x) {
-                const int el = i / a.dsh, b = i - el * a.dsh;
-                const int64_t pos = b0 + el;
-                const int64_t e = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
-                sY[el * a.dsh + b] = a.Y[e * a.dsh + b];
-            }
-            for (int i = threadIdx.x; i < nb * KC; i += blockDim.x) {
-                const int el = i / KC, q = i - el * KC;
-                const int64_t pos = b0 + el;
-                const int64_t e = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
-                sPhi[el * KC + q] = (q0 + q < a.K) ? a.phi[e * a.K + q0 + q] : 0.f;
-            }
-            __syncthreads();
-            // ---- expand M for the needed paths
-            for (int pp = pb; pp < pe; ++pp) {
-                const DPath Q = a.paths[pp];
-                const int ne = Q.d_src * D_DST;
-                for (int i = threadIdx.x; i < nb * ne; i += blockDim.x) {
-                    const int el = i / ne, t = i - el * ne;
-                    const int t0 = a.tab_ptr[Q.tabM + t], t1 = a.tab_ptr[Q.tabM + t + 1];
-                    float s = 0.f;
-                    for (int k = t0; k < t1; ++k)
-                        s = fmaf(a.tab_coef[k], sY[el * a.dsh + Q.sh_off + a.tab_idx[k]], s);
-                    sM[el * a.m_stride + Q.m_off + t] = s;
-                }
-            }
-            __syncthreads();
-            // ---- accumulate
-            if (active) {
-                for (int el = 0; el < nb; ++el) {
-                    const float* xr = a.src + sSrc[el] * a.C_src + P.src_off + u;
-                    const float* Me = sM + el * a.m_stride + P.m_off;
-                    float C[D_DST];
-#pragma unroll
-                    for (int o = 0; o < D_DST; ++o) C[o] = 0.f;
-                    for (int s = 0; s < P.d_src; ++s) {
-                        const float xs = __ldg(xr + s * P.c_src);
-#pragma unroll
-                        for (int o = 0; o < D_DST; ++o) C[o] = fmaf(xs, Me[s * D_DST + o], C[o]);
-                    }
-                    const float* ph = sPhi + el * KC;
-#pragma unroll
-                    for (int q = 0; q < KC; ++q) {
-                        const float pq = ph[q];
-#pragma unroll
-                        for (int o = 0; o < D_DST; ++o) acc[o][q] = fmaf(pq, C[o], acc[o][q]);
-                    }
-                }
-            }
-        }
-        if (active) {
-            float* Zg = a.Z + a.n_nodes * a.G.z_off;
-#pragma unroll
-            for (int o = 0; o < D_DST; ++o) {
-                float* zr = Zg + ((int64_t)blockIdx.x * D_DST + o) * a.G.D + P.koff + (int64_t)u * a.K + q0;
-#pragma unroll
-                for (int q = 0; q < KC; ++q)
-                    if (q0 + q < a.K) zr[q] = a.accumulate ? zr[q] + acc[o][q] : acc[o][q];
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------
-// Generic fp32 GEMM with mapped addressing (rows/cols may be (node, component) pairs):
-//   C(m,n) (+)= sum_k A(m,k) B(k,n)
-//   addr(X; i, j) = base + (i / d)*outer + (i % d)*inner + j*cs     for the "row-like" index i
-// ------------------------------------------------------------------------------------
-struct Map2 {
-    int64_t outer, inner;   // row-like index i -> (i/d)*outer + (i%d)*inner
-    int64_t cs;             // stride of the other index
-    int32_t d;
-    int32_t fast_second;    // 1 if the second index is the contiguous one
-};
-__device__ __forceinline__ int64_t map_addr(const Map2& m, int64_t i, int64_t j) {
-    return (i / m.d) * m.outer + (i % m.d) * m.inner + j * m.cs;
-}
-
-struct GemmArgs {
-    const float* A; const float* B; float* C;
-    Map2 a;   // A: row-like index = m, second = k      (if a_rowlike_is_k: row-like = k, second = m)
-    Map2 b;   // B: row-like index = k, second = n      (if b_rowlike_is_n: row-like = n, second = k)
-    Map2 c;   // C: row-like index = m, second = n
-    int a_rowlike_is_k, b_rowlike_is_n;
-    int64_t M, N, Kd;
-    int accumulate;
-};
-
-constexpr int GM = 64, GN = 64, GK = 16;
-
-__global__ void __launch_bounds__(256) k_gemm(const GemmArgs g) {
-    __shared__ float As[GK][GM + 4];
-    __shared__ float Bs[GK][GN + 4];
-    const int tid = threadIdx.x;
-    const int64_t m0 = (int64_t)blockIdx.y * GM, n0 = (int64_t)blockIdx.x * GN;
-    const int tx = tid & 15, ty = tid >> 4;   // 16 x 16 threads, 4x4 outputs each
-    float acc[4][4] = {};
-    // which index runs fastest over consecutive threads when loading
-    const bool a_kfast = g.a_rowlike_is_k ? !g.a.fast_second : g.a.fast_second;
-    const bool b_nfast = g.b_rowlike_is_n ? !g.b.fast_second : g.b.fast_second;
-    for (int64_t k0 = 0; k0 < g.Kd; k0 += GK) {
-        for (int i = tid; i < GM * GK; i += 256) {
-            int m, k;
-            if (a_kfast) { k = i % GK; m = i / GK; } else { m = i % GM; k = i / GM; }
-            float v = 0.f;
-            if (m0 + m < g.M && k0 + k < g.Kd)
-                v = g.A[g.a_rowlike_is_k ? map_addr(g.a, k0 + k, m0 + m) : map_addr(g.a, m0 + m, k0 + k)];
-            As[k][m] = v;
-        }
-        for (int i = tid; i < GN * GK; i += 256) {
-            int n, k;
-            if (b_nfast) { n = i % GN; k = i / GN; } else { k = i % GK; n = i / GK; }
-            float v = 0.f;
-            if (n0 + n < g.N && k0 + k < g.Kd)
-                v = g.B[g.b_rowlike_is_n ? map_addr(g.b, n0 + n, k0 + k) : map_addr(g.b, k0 + k, n0 + n)];
-            Bs[k][n] = v;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < GK; ++k) {
-            float av[4], bv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) av[i] = As[k][ty * 4 + i];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) bv[j] = Bs[k][tx * 4 + j];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int64_t m = m0 + ty * 4 + i;
-        if (m >= g.M) continue;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int64_t n = n0 + tx * 4 + j;
-            if (n >= g.N) continue;
-            float* c = g.C + map_addr(g.c, m, n);
-            *c = g.accumulate ? *c + acc[i][j] : acc[i][j];
-        }
     }
 }
 
@@ -532,15 +313,6 @@ cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_pack_R(const sobek_plan* p, const Direction& dir, int transposed, const float* R,
-                          float* Rp, cudaStream_t s) {
-    dim3 grid(32, (unsigned)dir.paths.size());
-    KernelTimer kt(K_PACK, s);
-    k_pack_R<false><<<grid, 256, 0, s>>>(dir.d_paths, transposed, p->K, p->N_w, R, Rp);
-    count_launch();
-    return cudaGetLastError();
-}
-
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s) {
     dim3 grid(32, (unsigned)dir.paths.size());
@@ -548,115 +320,6 @@ cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const flo
     k_pack_R<true><<<grid, 256, 0, s>>>(dir.d_paths, 0, p->K, p->N_w, Rp, R);
     count_launch();
     return cudaGetLastError();
-}
-
-cudaError_t launch_state(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
-                         int64_t n_nodes, const float* src, const float* Y, const float* phi, float* Z,
-                         int accumulate, cudaStream_t s) {
-    for (const DGroup& G : dir.groups) {
-        if (G.path_end == G.path_begin) continue;
-        StateArgs a;
-        a.paths = dir.d_paths; a.wtasks = dir.d_wtasks;
-        a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
-        a.G = G; a.ev = ev; a.node0 = node0; a.n_nodes = n_nodes;
-        a.src = src; a.Y = Y; a.phi = phi; a.Z = Z;
-        a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.accumulate = accumulate;
-        a.m_stride = G.m_entries;
-        const int nwt = G.wt_end - G.wt_begin;
-        dim3 grid((unsigned)n_nodes, (unsigned)((nwt + ST_WARPS - 1) / ST_WARPS));
-        const bool k16 = (p->K > 8) && (G.d_dst <= 5);
-        const int KC = k16 ? 16 : 8;
-        size_t sh = sizeof(float) * ((size_t)ST_EB * a.m_stride + (size_t)ST_EB * a.dsh + (size_t)ST_EB * KC) +
-                    sizeof(int64_t) * ST_EB + 16;
-        // (EB is even, so the float part has an even count and the int64 array stays aligned)
-        KernelTimer kt(K_STATE, s);
-        cudaError_t e = dispatch_d(G.d_dst, [&](auto dtag) -> cudaError_t {
-            constexpr int D = decltype(dtag)::value;
-            if (k16) {
-                auto kern = k_state<D, 16>;
-                if (sh > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
-                kern<<<grid, ST_WARPS * 32, sh, s>>>(a);
-            } else {
-                auto kern = k_state<D, 8>;
-                if (sh > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
-                kern<<<grid, ST_WARPS * 32, sh, s>>>(a);
-            }
-            return cudaGetLastError();
-        });
-        count_launch();
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
-}
-
-static cudaError_t run_gemm(const GemmArgs& g, cudaStream_t s) {
-    if (g.M <= 0 || g.N <= 0) return cudaSuccess;
-    dim3 grid((unsigned)((g.N + GN - 1) / GN), (unsigned)((g.M + GM - 1) / GM));
-    KernelTimer kt(K_GEMM, s);
-    k_gemm<<<grid, 256, 0, s>>>(g);
-    count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t launch_mix(const sobek_plan* p, const Direction& dir, int64_t node0, int64_t n_nodes,
-                       const float* Z, const float* Rp, float* dst, int accumulate, cudaStream_t s) {
-    (void)p;
-    for (const DGroup& G : dir.groups) {
-        if (G.path_end == G.path_begin) continue;
-        GemmArgs g{};
-        g.A = Z + n_nodes * G.z_off;
-        g.a = Map2{(int64_t)G.D, 0, 1, 1, 1};                 // A(m,k) = Zg[m*D + k]
-        g.B = Rp + G.rp_off;
-        g.b = Map2{(int64_t)G.c_dst, 0, 1, 1, 1};             // B(k,n) = Rp[k*c + n]
-        g.C = dst + node0 * dir.C_dst + G.dst_off;
-        g.c = Map2{(int64_t)dir.C_dst, (int64_t)G.c_dst, 1, G.d_dst, 1};   // (node, o) rows
-        g.M = n_nodes * G.d_dst; g.N = G.c_dst; g.Kd = G.D; g.accumulate = accumulate;
-        cudaError_t e = run_gemm(g, s);
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
-}
-
-cudaError_t launch_state_adjoint(const sobek_plan* p, const Direction& dir, int64_t node0,
-                                 int64_t n_nodes, const float* gdst, const float* Rp, float* Zbar,
-                                 cudaStream_t s) {
-    (void)p;
-    for (const DGroup& G : dir.groups) {
-        if (G.path_end == G.path_begin) continue;
-        GemmArgs g{};
-        g.A = gdst + node0 * dir.C_dst + G.dst_off;           // A(m,k): (node,o) rows, k = w
-        g.a = Map2{(int64_t)dir.C_dst, (int64_t)G.c_dst, 1, G.d_dst, 1};
-        g.B = Rp + G.rp_off;                                  // B(k,n) = Rp[n*c + k]
-        g.b = Map2{(int64_t)G.c_dst, 0, 1, 1, 1};
-        g.b_rowlike_is_n = 1;
-        g.C = Zbar + n_nodes * G.z_off;
-        g.c = Map2{(int64_t)G.D, 0, 1, 1, 1};
-        g.M = n_nodes * G.d_dst; g.N = G.D; g.Kd = G.c_dst; g.accumulate = 0;
-        cudaError_t e = run_gemm(g, s);
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
-}
-
-cudaError_t launch_weight_grad(const sobek_plan* p, const Direction& dir, int64_t node0,
-                               int64_t n_nodes, const float* Z, const float* gdst, float* gRp,
-                               int accumulate, cudaStream_t s) {
-    (void)p;
-    for (const DGroup& G : dir.groups) {
-        if (G.path_end == G.path_begin) continue;
-        GemmArgs g{};
-        g.A = Z + n_nodes * G.z_off;                          // A(m,k) = Zg[k*D + m]
-        g.a = Map2{(int64_t)G.D, 0, 1, 1, 1};
-        g.a_rowlike_is_k = 1;
-        g.B = gdst + node0 * dir.C_dst + G.dst_off;           // B(k,n): k = (node,o) rows
-        g.b = Map2{(int64_t)dir.C_dst, (int64_t)G.c_dst, 1, G.d_dst, 1};
-        g.C = gRp + G.rp_off;
-        g.c = Map2{(int64_t)G.c_dst, 0, 1, 1, 1};
-        g.M = G.D; g.N = G.c_dst; g.Kd = n_nodes * G.d_dst; g.accumulate = accumulate;
-        cudaError_t e = run_gemm(g, s);
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
 }
 
 cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev,

@@ -365,10 +365,11 @@ void build_direction(sobek_plan* p, int transposed, Direction& dir) {
 }  // namespace
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order) {
-    // per node: fp32 state + its bf16 (hi, lo) split + (orders >= 1) the split output-adjoint rows
-    int64_t sf = p->fwd.state_floats, zb = p->fwd.zb_elems;
-    if (order >= 1) { sf = std::max(sf, p->tr.state_floats); zb = std::max(zb, p->tr.zb_elems); }
-    int64_t per = 4 * sf + 4 * zb + (order >= 1 ? 4 * p->fwd.gb_elems : 0);
+    // bytes per node held at once: the bf16 (hi, lo) state and, for orders >= 1, the fp32 adjoint
+    // state and the bf16 (hi, lo) rows of the output adjoint
+    int64_t zb = p->fwd.zb_elems;
+    if (order >= 1) zb = std::max(zb, p->tr.zb_elems);
+    int64_t per = 4 * zb + (order >= 1 ? 4 * p->fwd.state_floats + 4 * p->fwd.gb_elems : 0);
     per = std::max<int64_t>(per, 1);
     int64_t n = (int64_t)(kStateBudgetBytes / (size_t)per);
     n = std::max<int64_t>(n, 1);
@@ -441,6 +442,8 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     }
     build_direction(p, 0, p->fwd);
     build_direction(p, 1, p->tr);
+    build_stream_tasks(p, p->fwd);
+    build_stream_tasks(p, p->tr);
     cudaError_t e = cudaGetDevice(&p->device);
     if (e != cudaSuccess) {
         // No CUDA device: the plan stays usable for inspection (info, paths, CG tensors);
@@ -462,6 +465,8 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         if (e == cudaSuccess) e = upload(d->kn_ld, &d->d_kn_ld);
         if (e == cudaSuccess) e = upload(d->nk_ld, &d->d_nk_ld);
         if (e == cudaSuccess) e = upload(d->path_group, &d->d_path_group);
+        if (e == cudaSuccess) e = upload(d->stasks, &d->d_stasks);
+        if (e == cudaSuccess) e = upload(d->zb_off, &d->d_zb_off);
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -478,6 +483,7 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
     for (Direction* d : {&p->fwd, &p->tr}) {
         cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);
         cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);
+        cudaFree(d->d_stasks); cudaFree(d->d_zb_off);
     }
     (void)cudaGetLastError();
     delete p;

@@ -51,14 +51,16 @@ extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, 
         g_scratch_addr[dev] = (unsigned char*)ptr;
     }
     unsigned char* base = g_scratch_addr[dev];
-    // layout: [status 256 B][R re-laid out][receiver state of one node chunk]
-    const size_t rbytes = align256((size_t)p->K * (size_t)p->N_w * 4);
-    const size_t per_node = (size_t)std::max<int64_t>(p->fwd.state_floats, 1) * 4;
-    if (kHeaderBytes + rbytes + per_node > kStaticScratchBytes) return SOBEK_ERR_WORKSPACE;
-    const int64_t chunk = std::min<int64_t>(std::max<int64_t>(g->N, 1),
-                                            (int64_t)((kStaticScratchBytes - kHeaderBytes - rbytes) / per_node));
-    float* Rp = (float*)(base + kHeaderBytes);
-    float* state = (float*)(base + kHeaderBytes + rbytes);
+    // layout: [status 256 B][R as bf16 hi, lo][receiver state of one node chunk as bf16 hi, lo]
+    const size_t rbytes = align256((size_t)p->fwd.nk_elems * 2);
+    const size_t per_node = (size_t)std::max<int64_t>(p->fwd.zb_elems, 1) * 2;   // one of (hi, lo)
+    if (kHeaderBytes + 2 * rbytes + 2 * (per_node + 256) > kStaticScratchBytes) return SOBEK_ERR_WORKSPACE;
+    const int64_t chunk = std::min<int64_t>(
+        std::max<int64_t>(g->N, 1), (int64_t)((kStaticScratchBytes - kHeaderBytes - 2 * rbytes - 512) / (2 * per_node)));
+    unsigned char* nkh = base + kHeaderBytes;
+    unsigned char* nkl = nkh + rbytes;
+    unsigned char* zh = nkl + rbytes;
+    unsigned char* zl = zh + align256((size_t)chunk * per_node);
     cudaStream_t s = (cudaStream_t)stream;
 #define CKS(expr)                                            \
     do {                                                     \
@@ -74,13 +76,23 @@ extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, 
     for (const DGroup& G : p->fwd.groups) uncovered = uncovered || (G.path_end == G.path_begin);
     if (g->E == 0 || uncovered) CKS(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
-    CKS(launch_pack_R(p, p->fwd, 0, R, Rp, s));
+    CKS(launch_pack_R_bf16(p, p->fwd, 0, 1, R, nkh, nkl, s));
     const EdgeView rv{g->row_ptr, nullptr, g->col, g->row_ptr, g->N, g->E, 0};
+    const Direction& dir = p->fwd;
     for (int64_t n0 = 0; n0 < g->N; n0 += chunk) {
         const int64_t nn = std::min(chunk, g->N - n0);
-        // every element of the chunk's state is overwritten before it is read
-        CKS(launch_state(p, p->fwd, rv, n0, nn, x, Y, phi, state, 0, s));
-        CKS(launch_mix(p, p->fwd, n0, nn, state, Rp, y, 0, s));
+        // every element of the chunk's state that the contraction reads is overwritten first
+        CKS(launch_stream(p, dir, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, zh, zl, s));
+        for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+            const DGroup& G = dir.groups[gi];
+            if (G.path_end == G.path_begin) continue;
+            const uint16_t* ah = (const uint16_t*)zh + nn * dir.zb_off[gi];
+            const uint16_t* al = (const uint16_t*)zl + nn * dir.zb_off[gi];
+            CKS(launch_gemm_tc(ah, al, dir.nk_ld[gi], (const uint16_t*)nkh + dir.nk_off[gi],
+                               (const uint16_t*)nkl + dir.nk_off[gi], dir.nk_ld[gi],
+                               y + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst, nn * G.d_dst, G.c_dst,
+                               G.D, 0, 0, (int*)base, s));
+        }
     }
 #undef CKS
     return SOBEK_OK;
