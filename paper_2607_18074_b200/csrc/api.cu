@@ -93,22 +93,27 @@ bool has_uncovered(const Direction& d) {
 
 
 // rows (node, o) of the chunk's output adjoint -> bf16 (hi, lo), group by group
-cudaError_t split_adjoint(const Direction& dir, int64_t n0, int64_t nn, const float* gdst, uint16_t* gh, uint16_t* gl,
-                          cudaStream_t s) {
+cudaError_t split_adjoint(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const float* gdst,
+                          uint16_t* gh, uint16_t* gl, cudaStream_t s0) {
+    Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
         cudaError_t e = launch_split(gdst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst, nn * G.d_dst,
                                      G.c_dst, dir.kn_ld[gi], gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], s);
         if (e != cudaSuccess) return e;
     }
-    return cudaSuccess;
+    return fork.join();
 }
 
 // dst_g (+)= Z_g * Rp_g        (Eq. receiver_matrix_product)
-cudaError_t mix_tc(const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh, const uint16_t* zl,
-                   const uint16_t* nkh, const uint16_t* nkl, float* dst, int accumulate, int* status, cudaStream_t s) {
+cudaError_t mix_tc(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh,
+                   const uint16_t* zl, const uint16_t* nkh, const uint16_t* nkl, float* dst, int accumulate,
+                   int* status, cudaStream_t s0) {
+    Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
         cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
@@ -117,13 +122,16 @@ cudaError_t mix_tc(const Direction& dir, int64_t n0, int64_t nn, const uint16_t*
                                        nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s);
         if (e != cudaSuccess) return e;
     }
-    return cudaSuccess;
+    return fork.join();
 }
 
 // Zbar_g = gy_g * Rp_g^T       (Eq. receiver_adjoint)
-cudaError_t state_adjoint_tc(const Direction& dir, int64_t nn, const uint16_t* gh, const uint16_t* gl,
-                             const uint16_t* knh, const uint16_t* knl, float* Zbar, int* status, cudaStream_t s) {
+cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t nn, const uint16_t* gh,
+                             const uint16_t* gl, const uint16_t* knh, const uint16_t* knl, float* Zbar, int* status,
+                             cudaStream_t s0) {
+    Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
         cudaError_t e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
@@ -131,13 +139,16 @@ cudaError_t state_adjoint_tc(const Direction& dir, int64_t nn, const uint16_t* g
                                        Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s);
         if (e != cudaSuccess) return e;
     }
-    return cudaSuccess;
+    return fork.join();
 }
 
 // gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint)
-cudaError_t weight_grad_tc(const Direction& dir, int64_t nn, const uint16_t* zh, const uint16_t* zl,
-                           const uint16_t* gh, const uint16_t* gl, float* gRp, int* status, cudaStream_t s) {
+cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn, const uint16_t* zh,
+                           const uint16_t* zl, const uint16_t* gh, const uint16_t* gl, float* gRp, int* status,
+                           cudaStream_t s0) {
+    Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
         cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
@@ -145,7 +156,7 @@ cudaError_t weight_grad_tc(const Direction& dir, int64_t nn, const uint16_t* zh,
                                        gRp + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 1, 1, status, s);
         if (e != cudaSuccess) return e;
     }
-    return cudaSuccess;
+    return fork.join();
 }
 
 }  // namespace
@@ -184,7 +195,7 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
         CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-        CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
+        CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
     }
     return SOBEK_OK;
 }
@@ -211,13 +222,13 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
         if (gR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-                CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
+                CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
             }
             if (gphi || gY) {
-                CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
                 CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, gphi, gY, gphi ? 1 : 0,
                                     gY ? 1 : 0, s));
             }
@@ -231,7 +242,7 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-            CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
+            CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
         }
     }
     return SOBEK_OK;
@@ -279,24 +290,24 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
         if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            if (hR || hphi || hY) CK(split_adjoint(p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            if (hR || hphi || hY) CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint with d(gy) = 0)
             int ggy_written = 0;
             if (ggy && vR) {
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-                CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
+                CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
                 ggy_written = 1;
             }
             if ((ggy || hR) && any_edge_dir) {
                 // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
-                if (ggy) CK(mix_tc(p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
-                if (hR) CK(weight_grad_tc(p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
+                if (ggy) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
+                if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
             }
             if (hphi || hY) {
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate
                 if (any_edge_dir) {
-                    CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
                     if (vx) {
                         CK(launch_edge_pass(p, p->fwd, rv, n0, nn, vx, Y, phi, w.zbar, hphi, hY,
                                             hphi ? pm : 0, hY ? ym : 0, s));
@@ -312,7 +323,7 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
                     }
                 }
                 if (vR) {
-                    CK(state_adjoint_tc(p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
+                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
                     CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, hphi, hY, hphi ? pm : 0,
                                         hY ? ym : 0, s));
                 }
@@ -330,12 +341,12 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             int wrote = 0;
             if (vY || vphi) {   // dV = V(gy; vY, phi) + V(gy; Y, vphi) in one pass
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
-                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, hx, 0, w.status, s));
+                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, hx, 0, w.status, s));
                 wrote = 1;
             }
             if (vR) {
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-                CK(mix_tc(p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, hx, wrote, w.status, s));
+                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, hx, wrote, w.status, s));
             }
         }
     }

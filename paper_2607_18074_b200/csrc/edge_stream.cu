@@ -60,7 +60,10 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
                           const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s) {
     if (n_nodes <= 0 || dir.stasks.empty()) return cudaSuccess;
     const int KC = p->K <= 8 ? 8 : 16;
+    Fork fork(p, s);   // the kernel classes touch disjoint parts of the state: run them concurrently
+    const cudaStream_t main = s;
     for (const auto& c : dir.sclasses) {
+        s = fork.pick();
         KernelTimer kt(K_STATE, s);
         cudaError_t e;
         if (KC == 8) e = dual ? stream_launch_k8_dual(p, dir, ev, node0, n_nodes, src, vsrc, Y, vY, phi, vphi, zh, zl, c.cls, c.begin, c.count, s)
@@ -70,7 +73,8 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
         count_launch();
         if (e != cudaSuccess) return e;
     }
-    return cudaSuccess;
+    (void)main;
+    return fork.join();
 }
 
 }  // namespace sobek

@@ -172,41 +172,42 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
                         }
             }
             __syncwarp();
-            // ---- fold the batch's edges, sender rows prefetched one edge ahead
-            float xn[DS][UB], vxn[DS][UB];
-            {
-                const float* xr = a.src + (int64_t)sSrc[0] * a.C_src + P.src_off + u;
+            // ---- fold the batch's edges.  The sender rows of PB edges are requested together so
+            //      that PB gathers are in flight per warp, then the PB edges are folded one by one.
+            constexpr int PB = (40 / (DS * UB * (DUAL ? 2 : 1))) >= 8 ? 8 : ((40 / (DS * UB * (DUAL ? 2 : 1))) >= 4 ? 4 :
+                               ((40 / (DS * UB * (DUAL ? 2 : 1))) >= 2 ? 2 : 1));
+            for (int el0 = 0; el0 < nb; el0 += PB) {
+                float xb[PB][DS][UB], vxb[PB][DS][UB];
 #pragma unroll
-                for (int s = 0; s < DS; ++s)
-                    if (s < P.d_src) load_x<UB>(xr + s * P.c_src, vec_ok, u, P.c_src, xn[s]);
-                if (has_vx) {
-                    const float* vr = a.vsrc + (int64_t)sSrc[0] * a.C_src + P.src_off + u;
+                for (int pe = 0; pe < PB; ++pe) {
+                    const int el = min(el0 + pe, nb - 1);
+                    const float* xr = a.src + (int64_t)sSrc[el] * a.C_src + P.src_off + u;
 #pragma unroll
-                    for (int s = 0; s < DS; ++s)
-                        if (s < P.d_src) load_x<UB>(vr + s * P.c_src, vec_ok, u, P.c_src, vxn[s]);
-                }
-            }
-            for (int el = 0; el < nb; ++el) {
-                float xs[DS][UB], vxs[DS][UB];
+                    for (int s = 0; s < DS; ++s) {
+                        if (s < P.d_src) load_x<UB>(xr + s * P.c_src, vec_ok, u, P.c_src, xb[pe][s]);
+                        else {
 #pragma unroll
-                for (int s = 0; s < DS; ++s)
-#pragma unroll
-                    for (int i = 0; i < UB; ++i) {
-                        xs[s][i] = (s < P.d_src) ? xn[s][i] : 0.f;
-                        if (DUAL) vxs[s][i] = (has_vx && s < P.d_src) ? vxn[s][i] : 0.f;
+                            for (int i = 0; i < UB; ++i) xb[pe][s][i] = 0.f;
+                        }
                     }
-                if (el + 1 < nb) {
-                    const float* xr = a.src + (int64_t)sSrc[el + 1] * a.C_src + P.src_off + u;
+                    if (DUAL) {
+                        const float* vr = a.vsrc + (int64_t)sSrc[el] * a.C_src + P.src_off + u;
 #pragma unroll
-                    for (int s = 0; s < DS; ++s)
-                        if (s < P.d_src) load_x<UB>(xr + s * P.c_src, vec_ok, u, P.c_src, xn[s]);
-                    if (has_vx) {
-                        const float* vr = a.vsrc + (int64_t)sSrc[el + 1] * a.C_src + P.src_off + u;
+                        for (int s = 0; s < DS; ++s) {
+                            if (has_vx && s < P.d_src) load_x<UB>(vr + s * P.c_src, vec_ok, u, P.c_src, vxb[pe][s]);
+                            else {
 #pragma unroll
-                        for (int s = 0; s < DS; ++s)
-                            if (s < P.d_src) load_x<UB>(vr + s * P.c_src, vec_ok, u, P.c_src, vxn[s]);
+                                for (int i = 0; i < UB; ++i) vxb[pe][s][i] = 0.f;
+                            }
+                        }
                     }
                 }
+#pragma unroll
+                for (int pe = 0; pe < PB; ++pe) {
+                const int el = el0 + pe;
+                if (el < nb) {
+                const float (&xs)[DS][UB] = xb[pe];
+                const float (&vxs)[DS][UB] = vxb[pe];
                 const float4* Me = reinterpret_cast<const float4*>(sM + el * MS);
                 const float4* dMe = reinterpret_cast<const float4*>(sdM + el * MS);
                 float C[UB][OC], dC[UB][OC];
@@ -261,6 +262,8 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
                                 for (int o = 0; o < OC; ++o)
                                     acc[i][o][4 * q4 + j] = fmaf(vq[j], C[i][o], acc[i][o][4 * q4 + j]);
                     }
+                }
+                }
                 }
             }
         }

@@ -118,6 +118,13 @@ struct sobek_plan {
     int32_t* d_tab_idx = nullptr;
     float* d_tab_coef = nullptr;
     int device = -1;
+    // side streams used to run independent kernels of one call concurrently (joined back into the
+    // caller's stream before the call returns control of ordering)
+    static constexpr int kSide = 4;
+    cudaStream_t side[kSide] = {};
+    cudaEvent_t ev_fork = nullptr;
+    cudaEvent_t ev_join[kSide] = {};
+    int n_side = 0;
 };
 
 namespace sobek {
@@ -125,11 +132,26 @@ namespace sobek {
 // bytes reserved at the start of every workspace for the device status word
 constexpr size_t kHeaderBytes = 256;
 // budget for the bounded node-state buffer (floats of Z / V held at once)
-constexpr size_t kStateBudgetBytes = size_t(96) << 20;
+constexpr size_t kStateBudgetBytes = size_t(256) << 20;
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);
 
 void count_launch(int n = 1);
+
+// Fork/join of the caller's stream into the plan's side streams: kernels launched on pick() run
+// concurrently with each other and are all ordered after what was queued on `main` before the
+// fork and before what is queued on `main` after join().
+class Fork {
+public:
+    Fork(const sobek_plan* p, cudaStream_t main);
+    cudaStream_t pick();
+    cudaError_t join();
+private:
+    const sobek_plan* p_;
+    cudaStream_t main_;
+    int used_ = 0;
+    bool on_ = false;
+};
 
 enum KernelClass { K_PACK = 0, K_STATE, K_GEMM, K_EDGE, K_FILL, K_NCLASS };
 // Brackets one launch with CUDA events when timing is enabled (sobek_timing_enable).

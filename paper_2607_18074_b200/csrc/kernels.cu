@@ -35,6 +35,31 @@ KernelTimer::~KernelTimer() {
     g_timed.push_back(TimedLaunch{a_, b_, cls_});
 }
 
+Fork::Fork(const sobek_plan* p, cudaStream_t main) : p_(p), main_(main) {
+    if (p->n_side <= 0) return;
+    if (cudaEventRecord(p->ev_fork, main) != cudaSuccess) { (void)cudaGetLastError(); return; }
+    on_ = true;
+}
+cudaStream_t Fork::pick() {
+    if (!on_) return main_;
+    const int i = used_ % p_->n_side;
+    if (used_ < p_->n_side) cudaStreamWaitEvent(p_->side[i], p_->ev_fork, 0);
+    ++used_;
+    return p_->side[i];
+}
+cudaError_t Fork::join() {
+    if (!on_) return cudaSuccess;
+    const int n = used_ < p_->n_side ? used_ : p_->n_side;
+    for (int i = 0; i < n; ++i) {
+        cudaError_t e = cudaEventRecord(p_->ev_join[i], p_->side[i]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(main_, p_->ev_join[i], 0);
+        if (e != cudaSuccess) return e;
+    }
+    used_ = 0;
+    on_ = false;
+    return cudaSuccess;
+}
+
 }  // namespace sobek
 
 extern "C" int64_t sobek_launch_count(void) { return sobek::g_launches.load(); }

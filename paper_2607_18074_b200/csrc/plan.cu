@@ -473,12 +473,27 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         sobek_plan_destroy(p);
         return SOBEK_ERR_CUDA;
     }
+    // side streams (optional: without them everything runs on the caller's stream)
+    if (cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) == cudaSuccess) {
+        for (int i = 0; i < sobek_plan::kSide; ++i) {
+            if (cudaStreamCreateWithFlags(&p->side[i], cudaStreamNonBlocking) != cudaSuccess ||
+                cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming) != cudaSuccess)
+                break;
+            p->n_side = i + 1;
+        }
+    }
+    (void)cudaGetLastError();
     *plan = p;
     return SOBEK_OK;
 }
 
 extern "C" void sobek_plan_destroy(sobek_plan* p) {
     if (!p) return;
+    for (int i = 0; i < sobek_plan::kSide; ++i) {
+        if (p->side[i]) cudaStreamDestroy(p->side[i]);
+        if (p->ev_join[i]) cudaEventDestroy(p->ev_join[i]);
+    }
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     cudaFree(p->d_tab_ptr); cudaFree(p->d_tab_idx); cudaFree(p->d_tab_coef);
     for (Direction* d : {&p->fwd, &p->tr}) {
         cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);
