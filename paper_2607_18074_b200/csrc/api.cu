@@ -18,6 +18,8 @@ struct Workspace {
     uint16_t *fKNh, *fKNl;    // receiver direction, [k][w]   (Zbar = gy Rp^T)
     uint16_t *tNKh, *tNKl;    // sender direction,   [u][k']  (gx = V Rt)
     uint16_t *vfNKh, *vfNKl, *vfKNh, *vfKNl, *vtNKh, *vtNKl;   // the same for vR
+    uint16_t *fFKh, *fFKl, *tFKh, *tFKl, *vfFKh, *vfFKl, *vtFKh, *vtFKl;   // stage-ordered copies (fused kernels)
+    bool fused_f, fused_t;    // fused kernels usable for the receiver / sender direction
     float* gRp;               // fp32 accumulator of the R adjoint, packed [k][w] per group
     float* zbar;              // fp32 adjoint state Zbar of one chunk (input of the edge pass)
     uint16_t *zbh, *zbl;      // bf16 (hi, lo) node state Z / dZ / V of one chunk
@@ -32,6 +34,17 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     size_t off = kHeaderBytes;
     auto take = [&](size_t bytes) { char* r = c + off; off += align256(bytes); return r; };
     w.status = (int*)c;
+    w.fused_f = fused_supported(p, p->fwd);
+    w.fused_t = fused_supported(p, p->tr);
+    if (w.fused_f) { w.fFKh = (uint16_t*)take(p->fwd.fk_elems * 2); w.fFKl = (uint16_t*)take(p->fwd.fk_elems * 2); }
+    if (w.fused_f && order >= 2) { w.vfFKh = (uint16_t*)take(p->fwd.fk_elems * 2); w.vfFKl = (uint16_t*)take(p->fwd.fk_elems * 2); }
+    if (w.fused_t && order >= 1) { w.tFKh = (uint16_t*)take(p->tr.fk_elems * 2); w.tFKl = (uint16_t*)take(p->tr.fk_elems * 2); }
+    if (w.fused_t && order >= 2) { w.vtFKh = (uint16_t*)take(p->tr.fk_elems * 2); w.vtFKl = (uint16_t*)take(p->tr.fk_elems * 2); }
+    if (order == 0 && w.fused_f) {   // the forward needs nothing else: the state stays on chip
+        w.chunk = 0;
+        w.bytes = off;
+        return w;
+    }
     w.fNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.fNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
     if (order >= 1) {
         w.fKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.fKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
@@ -190,8 +203,13 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
     if (g->N == 0) return SOBEK_OK;
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
-    CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     const EdgeView rv = receiver_view(g);
+    if (w.fused_f) {
+        CK(launch_pack_R_fused(p, p->fwd, 0, R, w.fFKh, w.fFKl, s));
+        CK(launch_fused(p, p->fwd, rv, x, nullptr, Y, nullptr, phi, nullptr, 0, w.fFKh, w.fFKl, y, 0, w.status, s));
+        return SOBEK_OK;
+    }
+    CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
         CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
@@ -237,12 +255,17 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     }
     if (gx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(gx, g->N * (int64_t)p->C_x, s));
-        CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
         const EdgeView sv = sender_view(g);
-        for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
-            const int64_t nn = std::min(w.chunk, g->N - n0);
-            CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-            CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
+        if (w.fused_t) {
+            CK(launch_pack_R_fused(p, p->tr, 1, R, w.tFKh, w.tFKl, s));
+            CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.tFKh, w.tFKl, gx, 0, w.status, s));
+        } else {
+            CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
+            for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
+                const int64_t nn = std::min(w.chunk, g->N - n0);
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
+            }
         }
     }
     return SOBEK_OK;
@@ -282,26 +305,41 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
 
     const EdgeView rv = receiver_view(g);
     if (ggy || hR || hphi || hY) {
-        if (ggy && any_edge_dir) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
-        if (ggy && vR) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
+        if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
+        // ggy = Z vR + dZ R.  The fused kernels produce it without leaving the SM; when hR is wanted too the
+        // directional state dZ is materialised chunk by chunk (it also feeds hR = dZ^T gy).
+        const bool fuse_ggy = ggy && w.fused_f;
+        const bool fuse_dz = fuse_ggy && !hR;
+        int ggy_done = 0;
+        if (fuse_ggy && vR) {
+            CK(launch_pack_R_fused(p, p->fwd, 0, vR, w.vfFKh, w.vfFKl, s));
+            CK(launch_fused(p, p->fwd, rv, x, nullptr, Y, nullptr, phi, nullptr, 0, w.vfFKh, w.vfFKl, ggy, 0, w.status, s));
+            ggy_done = 1;
+        }
+        if (fuse_dz && any_edge_dir) {
+            CK(launch_pack_R_fused(p, p->fwd, 0, R, w.fFKh, w.fFKl, s));
+            CK(launch_fused(p, p->fwd, rv, x, vx, Y, vY, phi, vphi, 1, w.fFKh, w.fFKl, ggy, ggy_done, w.status, s));
+            ggy_done = 1;
+        }
+        if (ggy && any_edge_dir && !fuse_dz) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+        if (ggy && vR && !fuse_ggy) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
         if ((hphi || hY) && any_edge_dir) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
         if ((hphi || hY) && vR) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl, s));
         if (hR) CK(launch_fill_zero(w.gRp, KN, s));
-        if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             if (hR || hphi || hY) CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint with d(gy) = 0)
-            int ggy_written = 0;
-            if (ggy && vR) {
+            int ggy_written = ggy_done;
+            if (ggy && vR && !fuse_ggy) {
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
                 CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
                 ggy_written = 1;
             }
-            if ((ggy || hR) && any_edge_dir) {
+            if (((ggy && !fuse_dz) || hR) && any_edge_dir) {
                 // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
-                if (ggy) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
+                if (ggy && !fuse_dz) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
                 if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
             }
             if (hphi || hY) {
@@ -333,9 +371,22 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
     }
     if (hx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(hx, g->N * (int64_t)p->C_x, s));
+        const EdgeView sv = sender_view(g);
+        if (w.fused_t) {
+            int wrote = 0;
+            if (vY || vphi) {   // dV = V(gy; vY, phi) + V(gy; Y, vphi) in one pass
+                CK(launch_pack_R_fused(p, p->tr, 1, R, w.tFKh, w.tFKl, s));
+                CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, vY, phi, vphi, 1, w.tFKh, w.tFKl, hx, 0, w.status, s));
+                wrote = 1;
+            }
+            if (vR) {
+                CK(launch_pack_R_fused(p, p->tr, 1, vR, w.vtFKh, w.vtFKl, s));
+                CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.vtFKh, w.vtFKl, hx, wrote, w.status, s));
+            }
+            return SOBEK_OK;
+        }
         if (vY || vphi) CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
         if (vR) CK(launch_pack_R_bf16(p, p->tr, 1, 1, vR, w.vtNKh, w.vtNKl, s));
-        const EdgeView sv = sender_view(g);
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             int wrote = 0;

@@ -1,0 +1,11 @@
+// Instantiation of the fused kernels for 16 radial components per stage.
+#include "fused_impl.cuh"
+
+namespace sobek {
+
+cudaError_t fused_launch_k16(int D, const CUtensorMap& th, const CUtensorMap& tl, const void* args, int grid, size_t sh,
+                     cudaStream_t s) {
+    return launch_fused_d<16, false>(D, th, tl, *(const FusedArgs*)args, grid, sh, s);
+}
+
+}  // namespace sobek

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libsobek (not installed).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <vector>
@@ -66,6 +67,13 @@ struct STask {         // one warp's task of the edge stream
     int32_t pad;
 };
 
+struct FStage {        // one 256-column stage of the fused kernel's contraction axis
+    int32_t path;
+    int32_t u0;        // first multiplicity of the block (256/KP wide)
+    int32_t q0;        // first radial component (0 unless K > 16)
+    int32_t group;
+};
+
 struct Direction {
     // host copies
     std::vector<DPath> paths;
@@ -88,6 +96,14 @@ struct Direction {
     int32_t ms_max = 4;               // row pitch (floats) of the per-edge M stage
     STask* d_stasks = nullptr;
     int64_t* d_zb_off = nullptr;
+    // fused kernels: stage list, per-group ranges and the stage-ordered bf16 copy of R
+    std::vector<FStage> fstages;
+    std::vector<int32_t> fs_begin, fs_count;
+    std::vector<int64_t> fk_off;
+    int64_t fk_elems = 0;
+    FStage* d_fstages = nullptr;
+    int32_t *d_fs_begin = nullptr, *d_fs_count = nullptr;
+    int64_t* d_fk_off = nullptr;
     // device copies
     DPath* d_paths = nullptr;
     DGroup* d_groups = nullptr;
@@ -153,7 +169,7 @@ private:
     bool on_ = false;
 };
 
-enum KernelClass { K_PACK = 0, K_STATE, K_GEMM, K_EDGE, K_FILL, K_NCLASS };
+enum KernelClass { K_PACK = 0, K_STATE, K_GEMM, K_EDGE, K_FILL, K_FUSED, K_NCLASS };
 // Brackets one launch with CUDA events when timing is enabled (sobek_timing_enable).
 class KernelTimer {
 public:
@@ -205,6 +221,53 @@ SOBEK_STREAM_DECL(stream_launch_k8);
 SOBEK_STREAM_DECL(stream_launch_k16);
 SOBEK_STREAM_DECL_DUAL(stream_launch_k8_dual);
 SOBEK_STREAM_DECL_DUAL(stream_launch_k16_dual);
+
+// --- fused.cu -------------------------------------------------------------------------
+struct FusedArgs {   // arguments of the fused kernels (fused_impl.cuh)
+    const DPath* paths;
+    const FStage* stages;
+    const int32_t* tab_ptr;
+    const int32_t* tab_idx;
+    const float* tab_coef;
+    DGroup G;
+    int32_t fs_begin, fs_count;
+    EdgeView ev;
+    int64_t N;
+    const float* src;
+    const float* vsrc;
+    const float* Y;
+    const float* vY;
+    const float* phi;
+    const float* vphi;
+    float* dst;
+    int32_t C_src, C_dst, accumulate;
+    int32_t K, dsh;
+    int32_t NT;          // nodes per tile = 128 / D
+    int32_t BN;          // padded destination multiplicity (multiple of 16)
+    int32_t tmem_cols;
+    int32_t nb_slots;    // B ring slots
+    int32_t EB;          // edges staged per batch (<= 16, <= multiplicities per stage)
+    int32_t MS;          // row pitch of the M stage
+    int32_t sub_floats;  // shared floats of one node's staging area (one per node handled by a warp)
+    int* status;
+};
+
+constexpr size_t A_BYTES_HOST = 4 * 128 * 128;   // one of (hi, lo) of the 128 x 256 bf16 A tile
+void build_fused_stages(const sobek_plan* p, Direction& dir);
+bool fused_supported(const sobek_plan* p, const Direction& dir);
+cudaError_t launch_pack_R_fused(const sobek_plan* p, const Direction& dir, int transposed, const float* R, void* hi,
+                                void* lo, cudaStream_t s);
+cudaError_t launch_fused(const sobek_plan* p, const Direction& dir, const EdgeView& ev, const float* src,
+                         const float* vsrc, const float* Y, const float* vY, const float* phi, const float* vphi,
+                         int dual, const void* fkh, const void* fkl, float* dst, int accumulate, int* status,
+                         cudaStream_t s0);
+#define SOBEK_FUSED_DECL(name)                                                                              \
+    cudaError_t name(int D, const CUtensorMap& th, const CUtensorMap& tl, const void* args, int grid, size_t sh, \
+                     cudaStream_t s)
+SOBEK_FUSED_DECL(fused_launch_k8);
+SOBEK_FUSED_DECL(fused_launch_k8_dual);
+SOBEK_FUSED_DECL(fused_launch_k16);
+SOBEK_FUSED_DECL(fused_launch_k16_dual);
 
 // --- gemm_tc.cu ---------------------------------------------------------------------
 int64_t round8(int64_t v);

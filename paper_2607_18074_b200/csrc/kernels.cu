@@ -22,7 +22,7 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 static bool g_timing = false;
 struct TimedLaunch { cudaEvent_t a, b; int cls; };
 static std::vector<TimedLaunch> g_timed;
-static const char* kClassNames[K_NCLASS] = {"pack_R", "edge_stream_state", "node_gemm", "edge_pass", "fill"};
+static const char* kClassNames[K_NCLASS] = {"pack_R", "edge_stream_state", "node_gemm", "edge_pass", "fill", "fused_stream_gemm"};
 
 KernelTimer::KernelTimer(int cls, cudaStream_t s) : cls_(cls), s_(s), on_(g_timing) {
     if (!on_) return;
