@@ -247,8 +247,8 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
             }
             if (gphi || gY) {
                 CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
-                CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, gphi, gY, gphi ? 1 : 0,
-                                    gY ? 1 : 0, s));
+                CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
+                                    gphi ? 1 : 0, gY ? 1 : 0, s));
             }
         }
         if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
@@ -345,25 +345,16 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             if (hphi || hY) {
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate
                 if (any_edge_dir) {
+                    // the three direction terms that share Zbar = gy R^T, in one pass
                     CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
-                    if (vx) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, vx, Y, phi, w.zbar, hphi, hY,
-                                            hphi ? pm : 0, hY ? ym : 0, s));
-                        pm = ym = 2;
-                    }
-                    if (vY && hphi) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vY, phi, w.zbar, hphi, hY, pm, 0, s));
-                        pm = 2;
-                    }
-                    if (vphi && hY) {
-                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, vphi, w.zbar, hphi, hY, 0, ym, s));
-                        ym = 2;
-                    }
+                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbar, hphi, hY,
+                                        hphi ? pm : 0, hY ? ym : 0, s));
+                    pm = ym = 2;
                 }
-                if (vR) {
+                if (vR) {   // the term through dZbar = gy vR^T
                     CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
-                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, Y, phi, w.zbar, hphi, hY, hphi ? pm : 0,
-                                        hY ? ym : 0, s));
+                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, hphi, hY,
+                                        hphi ? pm : 0, hY ? ym : 0, s));
                 }
             }
         }

@@ -2,49 +2,50 @@
 // instantiated in edge_stream_k*.cu).
 #include <algorithm>
 
+#include "edge_stream_args.h"
 #include "internal.h"
 
 namespace sobek {
 
-// Task list of one direction, sorted by kernel class.  Output components are cut into chunks of at
-// most 5, and the multiplicity block per lane (UB) is the largest of {4,2,1} that keeps OC*KC*UB
-// accumulators within the register budget and does not exceed what the path's multiplicity can use.
+// Source-major task list of one direction, sorted by kernel class (= padded d_src).  For every source
+// irrep block and every block of 32 multiplicities, the output components (path, o) of all paths that
+// read this block are packed into tasks of at most CAP components, split evenly.
 void build_stream_tasks(const sobek_plan* p, Direction& dir) {
     const int KC = p->K <= 8 ? 8 : 16;
+    const int CAP = KC == 8 ? 12 : 6;
     dir.stasks.clear();
+    dir.scomps.clear();
     dir.sclasses.clear();
-    dir.ms_max = 4;
-    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        const DGroup& G = dir.groups[gi];
-        for (int k = G.path_begin; k < G.path_end; ++k) {
-            const DPath& P = dir.paths[k];
-            int chunks[2][2];
-            int nch = 0;
-            const int D = G.d_dst;
-            if (D <= 5) { chunks[0][0] = 0; chunks[0][1] = D; nch = 1; }
-            else if (D == 7) { chunks[0][0] = 0; chunks[0][1] = 4; chunks[1][0] = 4; chunks[1][1] = 3; nch = 2; }
-            else { chunks[0][0] = 0; chunks[0][1] = 5; chunks[1][0] = 5; chunks[1][1] = 4; nch = 2; }
-            for (int c = 0; c < nch; ++c) {
-                const int oc = chunks[c][1];
-                const int ub_budget = 96 / (oc * KC);
-                int ub = ub_budget >= 4 ? 4 : (ub_budget >= 2 ? 2 : 1);
-                const int need = P.c_src <= 32 ? 1 : (P.c_src <= 64 ? 2 : 4);
-                ub = std::min(ub, need);
-                const int oci = oc == 1 ? 0 : (oc == 3 ? 1 : (oc == 4 ? 2 : 3));
-                const int ubi = ub == 1 ? 0 : (ub == 2 ? 1 : 2);
-                const int dsi = P.d_src <= 3 ? 0 : (P.d_src <= 5 ? 1 : 2);
-                for (int u0 = 0; u0 < P.c_src; u0 += 32 * ub) {
-                    STask t{};
-                    t.path = k; t.u0 = u0; t.o0 = chunks[c][0]; t.oc = oc; t.ub = ub;
-                    t.cls = (3 * oci + ubi) * 3 + dsi; t.group = (int)gi;
-                    dir.stasks.push_back(t);
-                }
-                int ms = P.d_src * oc;
-                ms = (ms + 3) & ~3;
-                if ((ms & 31) == 0) ms += 4;
-                dir.ms_max = std::max(dir.ms_max, ms);
+    // distinct source blocks, in order of appearance
+    std::vector<int> src_offs;
+    for (const DPath& P : dir.paths)
+        if (std::find(src_offs.begin(), src_offs.end(), P.src_off) == src_offs.end()) src_offs.push_back(P.src_off);
+    for (int so : src_offs) {
+        std::vector<SComp> all;
+        int c_src = 0, d_src = 0;
+        for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+            const DGroup& G = dir.groups[gi];
+            for (int k = G.path_begin; k < G.path_end; ++k) {
+                const DPath& P = dir.paths[k];
+                if (P.src_off != so) continue;
+                c_src = P.c_src; d_src = P.d_src;
+                for (int o = 0; o < G.d_dst; ++o)
+                    all.push_back(SComp{P.tabM + o, G.d_dst, P.sh_off, (int)gi, o, P.koff, G.d_dst, 0});
             }
         }
+        if (all.empty()) continue;
+        const int ntask = ((int)all.size() + CAP - 1) / CAP;
+        const int per = ((int)all.size() + ntask - 1) / ntask;
+        const int cls = d_src <= 3 ? 0 : (d_src <= 5 ? 1 : 2);
+        for (int u0 = 0; u0 < c_src; u0 += 32)
+            for (int t = 0; t < ntask; ++t) {
+                const int c0 = t * per, c1 = std::min((int)all.size(), c0 + per);
+                STask T{};
+                T.src_off = so; T.c_src = c_src; T.d_src = d_src; T.u0 = u0;
+                T.ncomp = c1 - c0; T.comp_begin = (int)dir.scomps.size(); T.cls = cls;
+                dir.scomps.insert(dir.scomps.end(), all.begin() + c0, all.begin() + c1);
+                dir.stasks.push_back(T);
+            }
     }
     std::stable_sort(dir.stasks.begin(), dir.stasks.end(), [](const STask& x, const STask& y) { return x.cls < y.cls; });
     for (size_t i = 0; i < dir.stasks.size();) {
@@ -60,20 +61,24 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
                           const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s) {
     if (n_nodes <= 0 || dir.stasks.empty()) return cudaSuccess;
     const int KC = p->K <= 8 ? 8 : 16;
+    StreamArgsHost a{};
+    a.tasks = dir.d_stasks; a.comps = dir.d_scomps;
+    a.zb_off = dir.d_zb_off; a.zb_ld = dir.d_nk_ld;
+    a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
+    a.ev = ev; a.node0 = node0; a.n_nodes = n_nodes;
+    a.src = src; a.vsrc = vsrc; a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
+    a.zh = zh; a.zl = zl;
+    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.warp_floats = 0;
     Fork fork(p, s);   // the kernel classes touch disjoint parts of the state: run them concurrently
-    const cudaStream_t main = s;
     for (const auto& c : dir.sclasses) {
-        s = fork.pick();
-        KernelTimer kt(K_STATE, s);
+        cudaStream_t cs = fork.pick();
+        KernelTimer kt(K_STATE, cs);
         cudaError_t e;
-        if (KC == 8) e = dual ? stream_launch_k8_dual(p, dir, ev, node0, n_nodes, src, vsrc, Y, vY, phi, vphi, zh, zl, c.cls, c.begin, c.count, s)
-                              : stream_launch_k8(p, dir, ev, node0, n_nodes, src, Y, phi, zh, zl, c.cls, c.begin, c.count, s);
-        else e = dual ? stream_launch_k16_dual(p, dir, ev, node0, n_nodes, src, vsrc, Y, vY, phi, vphi, zh, zl, c.cls, c.begin, c.count, s)
-                      : stream_launch_k16(p, dir, ev, node0, n_nodes, src, Y, phi, zh, zl, c.cls, c.begin, c.count, s);
+        if (KC == 8) e = dual ? stream_launch_k8_dual(&a, c.cls, c.begin, c.count, cs) : stream_launch_k8(&a, c.cls, c.begin, c.count, cs);
+        else e = dual ? stream_launch_k16_dual(&a, c.cls, c.begin, c.count, cs) : stream_launch_k16(&a, c.cls, c.begin, c.count, cs);
         count_launch();
         if (e != cudaSuccess) return e;
     }
-    (void)main;
     return fork.join();
 }
 

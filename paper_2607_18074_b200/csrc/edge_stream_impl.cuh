@@ -1,24 +1,24 @@
-// Edge-stream kernels (sm_100a): the per-edge work of the convolution.
+// Edge-stream kernel (sm_100a): the per-edge work of the convolution, SOURCE-MAJOR.
 //
-// k_stream<KC, DUAL> folds the edges of every node of a chunk into the bounded node state
-//     Z[pi,u,q,o] = sum_e phi_e[q] * C_e[pi,u,o],   C_e[pi,u,o] = sum_s xs_e[u,s] * M_e[s,o]
-// (Eqs. angular_path_contraction, receiver_state) and writes it as the split-bf16 (hi, lo)
-// A operand of the tensor-core contraction with R.  M_e[s,o] = sum_b c[s,b,o] * Y_e[b] depends on
-// the edge and the path only; it is expanded from the sparse table once per (edge, task).
-// With DUAL it produces the directional state of the double backward in one pass,
-//     dZ = sum_e ( vphi_e (x) C(x,Y) + phi_e (x) [ C(vx,Y) + C(x,vY) ] )
-// (Eq. receiver_double_adjoint: dS).  The same kernel runs the sender-owned transposed traversal
-// (source rows = output adjoints of the receivers, edges through the sender view).
+// k_stream<CAP, KC, DS, DUAL> folds the edges of every node of a chunk into the bounded node state
+//     Z[pi,u,q,o] = sum_e phi_e[q] * C_e[pi,u,o],   C_e[pi,u,o] = sum_s xs_e[u,s] * M_e[pi][s,o]
+// (Eqs. angular_path_contraction, receiver_state) and writes it as the split-bf16 (hi, lo) A operand of
+// the tensor-core contraction with R.  M_e[pi][s,o] = sum_b c[s,b,o] * Y_e[b] depends on the edge and
+// the path only and is expanded from the sparse table once per (edge, task).
 //
-// Work decomposition: one WARP per (node, task); a task is (path, block of 32*UB multiplicities,
-// chunk of OC output components).  Lanes own multiplicities, so the sum over a node's edges needs
-// no cross-lane reduction and no atomics, and sender rows are read with coalesced (vector) loads.
-// Each lane keeps acc[UB][OC][KC] in registers; per edge the operands that are uniform across lanes
-// (M_e, phi_e) come from the warp's private shared-memory stage as 128-bit broadcast loads.
-// Warps never synchronise with each other.
+// A task is (source irrep block, 32 multiplicities, up to CAP output components taken from ALL paths
+// that read this source block).  The gathered sender row xs_e[u, 0..d_src) is therefore loaded once per
+// edge and reused by every path that consumes it, and each lane keeps acc[CAP][KC] in registers.
+// One WARP per (node, task); lanes own multiplicities, so the sum over a node's edges needs no
+// cross-lane reduction and no atomics; the operands that are uniform across lanes (M_e, phi_e) come from
+// the warp's private shared-memory stage as 128-bit broadcast loads.  Warps never synchronise with
+// each other.  With DUAL the kernel produces the directional state of the double backward in one pass,
+//     dZ = sum_e ( vphi_e (x) C(x,Y) + phi_e (x) [ C(vx,Y) + C(x,vY) ] )       (Eq. receiver_double_adjoint).
+// The same kernel runs the sender-owned transposed traversal.
 #pragma once
 #include <cuda_bf16.h>
 
+#include "edge_stream_args.h"
 #include "internal.h"
 
 namespace sobek {
@@ -33,103 +33,47 @@ __device__ __forceinline__ int64_t owner_of(const int64_t* __restrict__ row_ptr,
     return lo;
 }
 
-struct StreamArgs {
-    const DPath* paths;
-    const STask* tasks;
-    const DGroup* groups;
-    const int64_t* zb_off;     // per group: bf16 state offset per node (elements)
-    const int32_t* zb_ld;      // per group: row pitch of the bf16 state (elements)
-    const int32_t* tab_ptr;
-    const int32_t* tab_idx;
-    const float* tab_coef;
-    EdgeView ev;
-    int64_t node0, n_nodes;
-    int32_t n_tasks;
-    const float* src;
-    const float* vsrc;         // DUAL only; may be NULL
-    const float* Y;
-    const float* vY;           // DUAL only; may be NULL
-    const float* phi;
-    const float* vphi;         // DUAL only; may be NULL
-    __nv_bfloat16* zh;
-    __nv_bfloat16* zl;
-    int32_t K, dsh, C_src;
-    int32_t warp_floats;       // shared floats per warp
-    int32_t ms_max;            // row pitch of the M stage
-};
+constexpr int S_EB = 16;       // edges staged per batch
 
-template <int UB>
-__device__ __forceinline__ void load_x(const float* __restrict__ p, bool vec_ok, int u, int c_src, float (&v)[UB]) {
-    if (UB == 4 && vec_ok) {
-        if (u < c_src) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(p));
-            v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3 % UB] = t.w;
-        } else {
-#pragma unroll
-            for (int i = 0; i < UB; ++i) v[i] = 0.f;
-        }
-    } else if (UB == 2 && vec_ok) {
-        if (u < c_src) {
-            const float2 t = __ldg(reinterpret_cast<const float2*>(p));
-            v[0] = t.x; v[1 % UB] = t.y;
-        } else {
-#pragma unroll
-            for (int i = 0; i < UB; ++i) v[i] = 0.f;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < UB; ++i) v[i] = (u + i < c_src) ? __ldg(p + i) : 0.f;
-    }
-}
-
-template <int OC, int KC, int UB, int DS, bool DUAL>
+template <int CAP, int KC, int DS, bool DUAL>
 __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, const int64_t nl, float* sm,
                                          const int lane) {
-    const DPath P = a.paths[T.path];
-    const int D = P.d_dst;
-    const int MS = a.ms_max;
+    constexpr int DSP = DS <= 3 ? 4 : (DS <= 5 ? 8 : 12);   // padded d_src: M rows as float4s
+    constexpr int MS = CAP * DSP;                           // floats of M per edge
     const int YS = a.dsh + 1;
-    // warp-private stage
-    float* sM = sm;                               // [32][MS]
-    float* sPhi = sM + 32 * MS;                   // [32][KC]
-    float* sY = sPhi + 32 * KC;                   // [32][YS]
-    int32_t* sSrc = (int32_t*)(sY + 32 * YS);     // [32] source node
-    int32_t* sE = sSrc + 32;                      // [32] edge id
-    float* sdM = (float*)(sE + 32);               // DUAL: [32][MS]
-    float* sVphi = sdM + 32 * MS;                 // DUAL: [32][KC]
-    float* sVY = sVphi + 32 * KC;                 // DUAL: [32][YS]
+    float* sM = sm;                                // [EB][MS]
+    float* sPhi = sM + S_EB * MS;                  // [EB][KC]
+    float* sY = sPhi + S_EB * KC;                  // [EB][YS]
+    int32_t* sSrc = (int32_t*)(sY + S_EB * YS);    // [EB] source node
+    int32_t* sE = sSrc + S_EB;                     // [EB] edge id
+    float* sdM = (float*)(sE + S_EB);              // DUAL: [EB][MS]
+    float* sVphi = sdM + S_EB * MS;                // DUAL: [EB][KC]
+    float* sVY = sVphi + S_EB * KC;                // DUAL: [EB][YS]
 
     const int64_t node = a.node0 + nl;
     const int64_t seg0 = a.ev.ptr[node], seg1 = a.ev.ptr[node + 1];
-    const int u = T.u0 + lane * UB;
-    const bool vec_ok = (UB == 1) || (((P.src_off | P.c_src | a.C_src) & (UB - 1)) == 0);
+    const int u = T.u0 + lane;
+    const bool act = u < T.c_src;
     const bool has_vx = DUAL && a.vsrc != nullptr, has_vY = DUAL && a.vY != nullptr,
                has_vphi = DUAL && a.vphi != nullptr;
-    const int oc = T.oc;   // <= OC
+    const SComp* comps = a.comps + T.comp_begin;
+    const int ncomp = T.ncomp;
 
     for (int q0 = 0; q0 < a.K; q0 += KC) {
-        float acc[UB][OC][KC];
+        float acc[CAP][KC];
 #pragma unroll
-        for (int i = 0; i < UB; ++i)
+        for (int c = 0; c < CAP; ++c)
 #pragma unroll
-            for (int o = 0; o < OC; ++o)
-#pragma unroll
-                for (int q = 0; q < KC; ++q) acc[i][o][q] = 0.f;
+            for (int q = 0; q < KC; ++q) acc[c][q] = 0.f;
 
-        for (int64_t b0 = seg0; b0 < seg1; b0 += 32) {
-            const int nb = (int)min((int64_t)32, seg1 - b0);
+        for (int64_t b0 = seg0; b0 < seg1; b0 += S_EB) {
+            const int nb = (int)min((int64_t)S_EB, seg1 - b0);
             __syncwarp();
-            // ---- stage the batch: lane <-> edge for ids, then flat copies of the Y and phi rows
-            {
-                int32_t e = 0, sn = 0;
-                if (lane < nb) {
-                    const int64_t pos = b0 + lane;
-                    const int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
-                    e = (int32_t)eid;
-                    sn = a.ev.transposed ? (int32_t)owner_of(a.ev.row_ptr, a.ev.N, eid) : a.ev.col[eid];
-                }
-                sE[lane] = e;
-                sSrc[lane] = sn;
+            if (lane < nb) {
+                const int64_t pos = b0 + lane;
+                const int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
+                sE[lane] = (int32_t)eid;
+                sSrc[lane] = a.ev.transposed ? (int32_t)owner_of(a.ev.row_ptr, a.ev.N, eid) : a.ev.col[eid];
             }
             __syncwarp();
             for (int i = lane; i < nb * a.dsh; i += 32) {
@@ -146,160 +90,134 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
                 if (has_vphi) sVphi[i] = in ? a.vphi[g] : 0.f;
             }
             __syncwarp();
-            // ---- expand M (and dM) for this lane's edge, own output components only
-            if (lane < nb) {
-                const float* y = sY + lane * YS + P.sh_off;
-                const float* vy = sVY + lane * YS + P.sh_off;
-                for (int s = 0; s < P.d_src; ++s)
-                    for (int o = 0; o < oc; ++o) {
-                        const int t = P.tabM + s * D + T.o0 + o;
-                        const int t0 = __ldg(a.tab_ptr + t), t1 = __ldg(a.tab_ptr + t + 1);
-                        float m = 0.f, dm = 0.f;
-                        for (int k = t0; k < t1; ++k) {
-                            const float c = __ldg(a.tab_coef + k);
-                            const int b = __ldg(a.tab_idx + k);
-                            m = fmaf(c, y[b], m);
-                            if (has_vY) dm = fmaf(c, vy[b], dm);
+            // ---- expand M (and dM): lane <-> (edge = lane % 16, components of parity lane / 16)
+            {
+                const int el = lane & 15;
+                if (el < nb) {
+                    const float* y = sY + el * YS;
+                    const float* vy = sVY + el * YS;
+                    for (int c = lane >> 4; c < ncomp; c += 2) {
+                        const SComp cp = comps[c];
+                        for (int s = 0; s < DSP; ++s) {     // padded rows are written as zeros
+                            const int t = cp.tab0 + s * cp.tstride;
+                            int t0 = 0, t1 = 0;
+                            if (s < T.d_src) { t0 = __ldg(a.tab_ptr + t); t1 = __ldg(a.tab_ptr + t + 1); }
+                            float m = 0.f, dm = 0.f;
+                            for (int k = t0; k < t1; ++k) {
+                                const float cf = __ldg(a.tab_coef + k);
+                                const int b = cp.sh_off + __ldg(a.tab_idx + k);
+                                m = fmaf(cf, y[b], m);
+                                if (has_vY) dm = fmaf(cf, vy[b], dm);
+                            }
+                            sM[el * MS + c * DSP + s] = m;
+                            if (has_vY) sdM[el * MS + c * DSP + s] = dm;
                         }
-                        sM[lane * MS + s * OC + o] = m;
-                        if (has_vY) sdM[lane * MS + s * OC + o] = dm;
                     }
-                if (oc < OC)
-                    for (int s = 0; s < P.d_src; ++s)
-                        for (int o = oc; o < OC; ++o) {
-                            sM[lane * MS + s * OC + o] = 0.f;
-                            if (has_vY) sdM[lane * MS + s * OC + o] = 0.f;
-                        }
+                }
             }
             __syncwarp();
-            // ---- fold the batch's edges.  The sender rows of PB edges are requested together so
-            //      that PB gathers are in flight per warp, then the PB edges are folded one by one.
-            constexpr int PB = (40 / (DS * UB * (DUAL ? 2 : 1))) >= 8 ? 8 : ((40 / (DS * UB * (DUAL ? 2 : 1))) >= 4 ? 4 :
-                               ((40 / (DS * UB * (DUAL ? 2 : 1))) >= 2 ? 2 : 1));
+            // ---- fold the batch's edges; the sender rows of PB edges are requested together
+            constexpr int PB = (24 / (DS * (DUAL ? 2 : 1))) >= 8 ? 8 : ((24 / (DS * (DUAL ? 2 : 1))) >= 4 ? 4 :
+                               ((24 / (DS * (DUAL ? 2 : 1))) >= 2 ? 2 : 1));
             for (int el0 = 0; el0 < nb; el0 += PB) {
-                float xb[PB][DS][UB], vxb[PB][DS][UB];
+                float xb[PB][DS], vxb[PB][DS];
 #pragma unroll
                 for (int pe = 0; pe < PB; ++pe) {
                     const int el = min(el0 + pe, nb - 1);
-                    const float* xr = a.src + (int64_t)sSrc[el] * a.C_src + P.src_off + u;
+                    const float* xr = a.src + (int64_t)sSrc[el] * a.C_src + T.src_off + u;
 #pragma unroll
-                    for (int s = 0; s < DS; ++s) {
-                        if (s < P.d_src) load_x<UB>(xr + s * P.c_src, vec_ok, u, P.c_src, xb[pe][s]);
-                        else {
-#pragma unroll
-                            for (int i = 0; i < UB; ++i) xb[pe][s][i] = 0.f;
-                        }
-                    }
+                    for (int s = 0; s < DS; ++s) xb[pe][s] = (act && s < T.d_src) ? __ldg(xr + s * T.c_src) : 0.f;
                     if (DUAL) {
-                        const float* vr = a.vsrc + (int64_t)sSrc[el] * a.C_src + P.src_off + u;
+                        const float* vr = a.vsrc + (int64_t)sSrc[el] * a.C_src + T.src_off + u;
 #pragma unroll
-                        for (int s = 0; s < DS; ++s) {
-                            if (has_vx && s < P.d_src) load_x<UB>(vr + s * P.c_src, vec_ok, u, P.c_src, vxb[pe][s]);
-                            else {
-#pragma unroll
-                                for (int i = 0; i < UB; ++i) vxb[pe][s][i] = 0.f;
-                            }
-                        }
+                        for (int s = 0; s < DS; ++s) vxb[pe][s] = (has_vx && act && s < T.d_src) ? __ldg(vr + s * T.c_src) : 0.f;
                     }
                 }
 #pragma unroll
                 for (int pe = 0; pe < PB; ++pe) {
-                const int el = el0 + pe;
-                if (el < nb) {
-                const float (&xs)[DS][UB] = xb[pe];
-                const float (&vxs)[DS][UB] = vxb[pe];
-                const float4* Me = reinterpret_cast<const float4*>(sM + el * MS);
-                const float4* dMe = reinterpret_cast<const float4*>(sdM + el * MS);
-                float C[UB][OC], dC[UB][OC];
+                    const int el = el0 + pe;
+                    if (el < nb) {
+                        const float4* Me = reinterpret_cast<const float4*>(sM + el * MS);
+                        const float4* dMe = reinterpret_cast<const float4*>(sdM + el * MS);
+                        const float4* ph4 = reinterpret_cast<const float4*>(sPhi + el * KC);
+                        const float4* vph4 = reinterpret_cast<const float4*>(sVphi + el * KC);
+                        float ph[KC], vph[KC];
 #pragma unroll
-                for (int i = 0; i < UB; ++i)
-#pragma unroll
-                    for (int o = 0; o < OC; ++o) { C[i][o] = 0.f; dC[i][o] = 0.f; }
-                float4 mv = make_float4(0.f, 0.f, 0.f, 0.f), dmv = mv;
-#pragma unroll
-                for (int s = 0; s < DS; ++s) {
-                    if (s < P.d_src) {
-#pragma unroll
-                        for (int o = 0; o < OC; ++o) {
-                            const int t = s * OC + o;     // static after unrolling
-                            if ((t & 3) == 0) { mv = Me[t >> 2]; if (has_vY) dmv = dMe[t >> 2]; }
-                            const float m = (t & 3) == 0 ? mv.x : ((t & 3) == 1 ? mv.y : ((t & 3) == 2 ? mv.z : mv.w));
-#pragma unroll
-                            for (int i = 0; i < UB; ++i) C[i][o] = fmaf(xs[s][i], m, C[i][o]);
-                            if (has_vx) {
-#pragma unroll
-                                for (int i = 0; i < UB; ++i) dC[i][o] = fmaf(vxs[s][i], m, dC[i][o]);
+                        for (int q4 = 0; q4 < KC / 4; ++q4) {
+                            const float4 t = ph4[q4];
+                            ph[4 * q4] = t.x; ph[4 * q4 + 1] = t.y; ph[4 * q4 + 2] = t.z; ph[4 * q4 + 3] = t.w;
+                            if (has_vphi) {
+                                const float4 v = vph4[q4];
+                                vph[4 * q4] = v.x; vph[4 * q4 + 1] = v.y; vph[4 * q4 + 2] = v.z; vph[4 * q4 + 3] = v.w;
                             }
-                            if (has_vY) {
-                                const float dm = (t & 3) == 0 ? dmv.x : ((t & 3) == 1 ? dmv.y : ((t & 3) == 2 ? dmv.z : dmv.w));
+                        }
 #pragma unroll
-                                for (int i = 0; i < UB; ++i) dC[i][o] = fmaf(xs[s][i], dm, dC[i][o]);
+                        for (int c = 0; c < CAP; ++c) {
+                            if (c < ncomp) {
+                                float C = 0.f, dC = 0.f;
+#pragma unroll
+                                for (int s4 = 0; s4 < DSP / 4; ++s4) {
+                                    const float4 m = Me[c * (DSP / 4) + s4];
+                                    const float mm[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j)
+                                        if (4 * s4 + j < DS) {
+                                            C = fmaf(xb[pe][4 * s4 + j], mm[j], C);
+                                            if (has_vx) dC = fmaf(vxb[pe][4 * s4 + j], mm[j], dC);
+                                        }
+                                    if (has_vY) {
+                                        const float4 d = dMe[c * (DSP / 4) + s4];
+                                        const float dd[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j)
+                                            if (4 * s4 + j < DS) dC = fmaf(xb[pe][4 * s4 + j], dd[j], dC);
+                                    }
+                                }
+                                const float Cm = DUAL ? dC : C;
+#pragma unroll
+                                for (int q = 0; q < KC; ++q) acc[c][q] = fmaf(ph[q], Cm, acc[c][q]);
+                                if (has_vphi) {
+#pragma unroll
+                                    for (int q = 0; q < KC; ++q) acc[c][q] = fmaf(vph[q], C, acc[c][q]);
+                                }
                             }
                         }
                     }
-                }
-                const float4* ph4 = reinterpret_cast<const float4*>(sPhi + el * KC);
-                const float4* vph4 = reinterpret_cast<const float4*>(sVphi + el * KC);
-#pragma unroll
-                for (int q4 = 0; q4 < KC / 4; ++q4) {
-                    const float4 pv = ph4[q4];
-                    const float pq[4] = {pv.x, pv.y, pv.z, pv.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-#pragma unroll
-                        for (int i = 0; i < UB; ++i)
-#pragma unroll
-                            for (int o = 0; o < OC; ++o)
-                                acc[i][o][4 * q4 + j] = fmaf(pq[j], DUAL ? dC[i][o] : C[i][o], acc[i][o][4 * q4 + j]);
-                    if (has_vphi) {
-                        const float4 vv = vph4[q4];
-                        const float vq[4] = {vv.x, vv.y, vv.z, vv.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-#pragma unroll
-                            for (int i = 0; i < UB; ++i)
-#pragma unroll
-                                for (int o = 0; o < OC; ++o)
-                                    acc[i][o][4 * q4 + j] = fmaf(vq[j], C[i][o], acc[i][o][4 * q4 + j]);
-                    }
-                }
-                }
                 }
             }
         }
         // ---- write the state slice as bf16 (hi, lo)
-        const int gi = T.group;
-        const int64_t ld = a.zb_ld[gi];
-        const int64_t gbase = a.n_nodes * a.zb_off[gi];
+        if (act) {
 #pragma unroll
-        for (int i = 0; i < UB; ++i) {
-            if (u + i >= P.c_src) continue;
+            for (int c = 0; c < CAP; ++c) {
+                if (c < ncomp) {
+                    const SComp cp = comps[c];
+                    const int64_t ld = a.zb_ld[cp.group];
+                    const int64_t off = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * ld + cp.koff +
+                                        (int64_t)u * a.K + q0;
+                    if ((a.K & 7) == 0) {
 #pragma unroll
-            for (int o = 0; o < OC; ++o) {
-                if (o >= oc) continue;
-                const int64_t off = gbase + (nl * D + T.o0 + o) * ld + P.koff + (int64_t)(u + i) * a.K + q0;
-                if ((a.K & 7) == 0) {
+                        for (int q = 0; q < KC; q += 8) {
+                            if (q0 + q >= a.K) break;
+                            __align__(16) __nv_bfloat16 h[8], l[8];
 #pragma unroll
-                    for (int q = 0; q < KC; q += 8) {
-                        if (q0 + q >= a.K) break;
-                        __align__(16) __nv_bfloat16 h[8], l[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float v = acc[i][o][q + j];
-                            h[j] = __float2bfloat16_rn(v);
-                            l[j] = __float2bfloat16_rn(v - __bfloat162float(h[j]));
+                            for (int j = 0; j < 8; ++j) {
+                                const float v = acc[c][q + j];
+                                h[j] = __float2bfloat16_rn(v);
+                                l[j] = __float2bfloat16_rn(v - __bfloat162float(h[j]));
+                            }
+                            *reinterpret_cast<uint4*>((__nv_bfloat16*)a.zh + off + q) = *reinterpret_cast<const uint4*>(h);
+                            *reinterpret_cast<uint4*>((__nv_bfloat16*)a.zl + off + q) = *reinterpret_cast<const uint4*>(l);
                         }
-                        *reinterpret_cast<uint4*>(a.zh + off + q) = *reinterpret_cast<const uint4*>(h);
-                        *reinterpret_cast<uint4*>(a.zl + off + q) = *reinterpret_cast<const uint4*>(l);
-                    }
-                } else {
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < KC; ++q) {
-                        if (q0 + q < a.K) {
-                            const float v = acc[i][o][q];
-                            const __nv_bfloat16 h = __float2bfloat16_rn(v);
-                            a.zh[off + q] = h;
-                            a.zl[off + q] = __float2bfloat16_rn(v - __bfloat162float(h));
+                        for (int q = 0; q < KC; ++q) {
+                            if (q0 + q < a.K) {
+                                const float v = acc[c][q];
+                                const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                                ((__nv_bfloat16*)a.zh)[off + q] = h;
+                                ((__nv_bfloat16*)a.zl)[off + q] = __float2bfloat16_rn(v - __bfloat162float(h));
+                            }
                         }
                     }
                 }
@@ -310,13 +228,8 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
 
 constexpr int SW = 8;   // warps per CTA
 
-constexpr int min_blocks(int OC, int KC, int UB, int DS, bool DUAL) {
-    const int est = UB * OC * KC + 2 * DS * UB * (DUAL ? 2 : 1) + 2 * UB * OC + 40;
-    return est <= 80 ? 3 : (est <= 124 ? 2 : 1);
-}
-
-template <int OC, int KC, int UB, int DS, bool DUAL>
-__global__ void __launch_bounds__(SW * 32, min_blocks(OC, KC, UB, DS, DUAL))
+template <int CAP, int KC, int DS, bool DUAL>
+__global__ void __launch_bounds__(SW * 32, (CAP * KC <= 64 && !DUAL) ? 2 : 1)
 k_stream(const StreamArgs a, const int t_begin, const int t_count) {
     extern __shared__ float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -325,49 +238,37 @@ k_stream(const StreamArgs a, const int t_begin, const int t_count) {
     for (int64_t item = (int64_t)blockIdx.x * SW + warp; item < total; item += (int64_t)gridDim.x * SW) {
         const int64_t nl = item / t_count;
         const STask T = a.tasks[t_begin + (int)(item - nl * t_count)];
-        run_task<OC, KC, UB, DS, DUAL>(a, T, nl, sm, lane);
+        run_task<CAP, KC, DS, DUAL>(a, T, nl, sm, lane);
     }
 }
 
-template <int OC, int KC, int UB, int DS, bool DUAL>
-cudaError_t launch_one(const StreamArgs& a, int t_begin, int t_count, size_t sh, cudaStream_t s) {
-    auto kern = k_stream<OC, KC, UB, DS, DUAL>;
+template <int CAP, int KC, int DS, bool DUAL>
+cudaError_t launch_one(StreamArgs a, int t_begin, int t_count, cudaStream_t s) {
+    constexpr int DSP = DS <= 3 ? 4 : (DS <= 5 ? 8 : 12);
+    int wf = S_EB * CAP * DSP + S_EB * KC + S_EB * (a.dsh + 1) + 2 * S_EB;
+    if (DUAL) wf += S_EB * CAP * DSP + S_EB * KC + S_EB * (a.dsh + 1);
+    wf = (wf + 3) & ~3;
+    a.warp_floats = wf;
+    const size_t sh = (size_t)wf * SW * sizeof(float);
+    auto kern = k_stream<CAP, KC, DS, DUAL>;
     if (sh > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
         if (e != cudaSuccess) return e;
     }
     const int64_t total = a.n_nodes * t_count;
-    const int per_sm = min_blocks(OC, KC, UB, DS, DUAL);
-    const int grid = (int)std::min<int64_t>((total + SW - 1) / SW, (int64_t)148 * per_sm * 2);
+    const int grid = (int)std::min<int64_t>((total + SW - 1) / SW, (int64_t)148 * 8);
     kern<<<grid, SW * 32, sh, s>>>(a, t_begin, t_count);
     return cudaGetLastError();
 }
 
-template <int OC, int KC, int UB, bool DUAL>
-cudaError_t launch_ds(int ds, const StreamArgs& a, int t_begin, int t_count, size_t sh, cudaStream_t s) {
-    switch (ds) {
-        case 3: return launch_one<OC, KC, UB, 3, DUAL>(a, t_begin, t_count, sh, s);
-        case 5: return launch_one<OC, KC, UB, 5, DUAL>(a, t_begin, t_count, sh, s);
-        default: return launch_one<OC, KC, UB, 9, DUAL>(a, t_begin, t_count, sh, s);
-    }
-}
-
-// class key = (index(OC in {1,3,4,5}) * 3 + index(UB in {1,2,4})) * 3 + index(DS in {3,5,9})
+// class = index(DS in {3,5,9})
 template <int KC, bool DUAL>
-cudaError_t launch_class(int cls, const StreamArgs& a, int t_begin, int t_count, size_t sh, cudaStream_t s) {
-    const int ds = (cls % 3 == 0) ? 3 : (cls % 3 == 1 ? 5 : 9);
-    switch (cls / 3) {
-        case 0: return launch_ds<1, KC, 1, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 1: return launch_ds<1, KC, 2, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 2: return launch_ds<1, KC, 4, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 3: return launch_ds<3, KC, 1, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 4: return launch_ds<3, KC, 2, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 5: return launch_ds<3, KC, (KC == 8 ? 4 : 1), DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 6: return launch_ds<4, KC, 1, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 7: return launch_ds<4, KC, (KC == 8 ? 2 : 1), DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 9: return launch_ds<5, KC, 1, DUAL>(ds, a, t_begin, t_count, sh, s);
-        case 10: return launch_ds<5, KC, (KC == 8 ? 2 : 1), DUAL>(ds, a, t_begin, t_count, sh, s);
-        default: return cudaErrorInvalidValue;
+cudaError_t launch_class(int cls, const StreamArgs& a, int t_begin, int t_count, cudaStream_t s) {
+    constexpr int CAP = KC == 8 ? 12 : 6;
+    switch (cls) {
+        case 0: return launch_one<CAP, KC, 3, DUAL>(a, t_begin, t_count, s);
+        case 1: return launch_one<CAP, KC, 5, DUAL>(a, t_begin, t_count, s);
+        default: return launch_one<CAP, KC, 9, DUAL>(a, t_begin, t_count, s);
     }
 }
 

@@ -57,13 +57,25 @@ struct WTask {         // one warp's share of a group: 32 consecutive multiplici
     int32_t u0;
 };
 
-struct STask {         // one warp's task of the edge stream
-    int32_t path;
-    int32_t u0;        // first multiplicity of the block (32*ub wide)
-    int32_t o0, oc;    // chunk of output components [o0, o0+oc)
-    int32_t ub;        // multiplicities per lane
-    int32_t cls;       // 3*index(OC in {1,3,4,5}) + index(UB in {1,2,4})
-    int32_t group;
+struct SComp {         // one output component handled by an edge-stream task
+    int32_t tab0;      // tab_ptr index of the (s = 0, o) entry of the path's M table
+    int32_t tstride;   // distance between consecutive s in that table (= d_dst of the path)
+    int32_t sh_off;    // offset of the path's SH block inside a Y row
+    int32_t group;     // destination group
+    int32_t o;         // component inside the destination irrep
+    int32_t koff;      // offset of the path in the group's contraction axis
+    int32_t d_dst;     // 2l+1 of the destination group
+    int32_t pad;
+};
+
+struct STask {         // one warp's task of the edge stream (source-major)
+    int32_t src_off;   // offset of the source block inside a source feature row
+    int32_t c_src;     // source multiplicity
+    int32_t d_src;     // 2l+1 of the source
+    int32_t u0;        // first of the 32 multiplicities of the task
+    int32_t ncomp;     // output components of the task
+    int32_t comp_begin;
+    int32_t cls;       // kernel class: padded d_src (0: <=3, 1: <=5, 2: <=9)
     int32_t pad;
 };
 
@@ -91,10 +103,11 @@ struct Direction {
     std::vector<int64_t> gb_off;      // per node, elements: sum_{g'<g} d * round8(c_dst) (bf16 adjoint rows)
     int64_t zb_elems = 0, gb_elems = 0;
     std::vector<STask> stasks;        // sorted by kernel class
+    std::vector<SComp> scomps;
     struct SClass { int cls, begin, count; };
     std::vector<SClass> sclasses;
-    int32_t ms_max = 4;               // row pitch (floats) of the per-edge M stage
     STask* d_stasks = nullptr;
+    SComp* d_scomps = nullptr;
     int64_t* d_zb_off = nullptr;
     // fused kernels: stage list, per-group ranges and the stage-ordered bf16 copy of R
     std::vector<FStage> fstages;
@@ -194,11 +207,12 @@ struct EdgeView {          // how a traversal walks the graph
 
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s);
-// receiver-owned edge pass: gphi_e = <Zbar, C_e>, gY_e = CG^T_Y(x, phi_e Zbar)
-cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev,
-                             int64_t node0, int64_t n_nodes, const float* src, const float* Y,
-                             const float* phi, const float* Zbar, float* gphi, float* gY,
-                             int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
+// receiver-owned edge pass: gphi_e = <Zbar, C_e>, gY_e = CG^T_Y(x, phi_e Zbar); with `dual` the
+// second-order terms that share Zbar: <Zbar, C(vx,Y)+C(x,vY)> and CG^T_Y(vx, phi Zbar) + CG^T_Y(x, vphi Zbar)
+cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
+                             int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
+                             const float* phi, const float* vphi, int dual, const float* Zbar, float* gphi,
+                             float* gY, int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
                              cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
 
@@ -208,19 +222,10 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
                           int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
                           const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s);
 
-#define SOBEK_STREAM_DECL(name)                                                                              \
-    cudaError_t name(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,           \
-                     int64_t n_nodes, const float* src, const float* Y, const float* phi, void* zh, void* zl, \
-                     int cls, int t_begin, int t_count, cudaStream_t s)
-#define SOBEK_STREAM_DECL_DUAL(name)                                                                         \
-    cudaError_t name(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,           \
-                     int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,  \
-                     const float* phi, const float* vphi, void* zh, void* zl, int cls, int t_begin,           \
-                     int t_count, cudaStream_t s)
-SOBEK_STREAM_DECL(stream_launch_k8);
-SOBEK_STREAM_DECL(stream_launch_k16);
-SOBEK_STREAM_DECL_DUAL(stream_launch_k8_dual);
-SOBEK_STREAM_DECL_DUAL(stream_launch_k16_dual);
+cudaError_t stream_launch_k8(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);
+cudaError_t stream_launch_k16(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);
+cudaError_t stream_launch_k8_dual(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);
+cudaError_t stream_launch_k16_dual(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);
 
 // --- fused.cu -------------------------------------------------------------------------
 struct FusedArgs {   // arguments of the fused kernels (fused_impl.cuh)
