@@ -12,7 +12,7 @@ namespace sobek {
 // read this block are packed into tasks of at most CAP components, split evenly.
 void build_stream_tasks(const sobek_plan* p, Direction& dir) {
     const int KC = p->K <= 8 ? 8 : 16;
-    const int CAP = KC == 8 ? 12 : 6;
+    const int CAP = KC == 8 ? 4 : 3;
     dir.stasks.clear();
     dir.scomps.clear();
     dir.sclasses.clear();

@@ -229,7 +229,7 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
 constexpr int SW = 8;   // warps per CTA
 
 template <int CAP, int KC, int DS, bool DUAL>
-__global__ void __launch_bounds__(SW * 32, (CAP * KC <= 64 && !DUAL) ? 2 : 1)
+__global__ void __launch_bounds__(SW * 32, (DUAL ? 2 : 3) - (KC == 16 ? 1 : 0))
 k_stream(const StreamArgs a, const int t_begin, const int t_count) {
     extern __shared__ float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -264,7 +264,7 @@ cudaError_t launch_one(StreamArgs a, int t_begin, int t_count, cudaStream_t s) {
 // class = index(DS in {3,5,9})
 template <int KC, bool DUAL>
 cudaError_t launch_class(int cls, const StreamArgs& a, int t_begin, int t_count, cudaStream_t s) {
-    constexpr int CAP = KC == 8 ? 12 : 6;
+    constexpr int CAP = KC == 8 ? 4 : 3;
     switch (cls) {
         case 0: return launch_one<CAP, KC, 3, DUAL>(a, t_begin, t_count, s);
         case 1: return launch_one<CAP, KC, 5, DUAL>(a, t_begin, t_count, s);

@@ -66,7 +66,7 @@ __global__ void k_pack_R_fused(const DPath* __restrict__ paths, const FStage* __
 }  // namespace
 
 bool fused_supported(const sobek_plan* p, const Direction& dir) {
-    (void)p;
+    if (!p->use_fused) return false;
     for (const DGroup& G : dir.groups)
         if (G.path_end > G.path_begin && G.c_dst > 256) return false;
     return !dir.fstages.empty();

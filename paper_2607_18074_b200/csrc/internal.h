@@ -147,6 +147,7 @@ struct sobek_plan {
     int32_t* d_tab_idx = nullptr;
     float* d_tab_coef = nullptr;
     int device = -1;
+    bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
     static constexpr int kSide = 4;

@@ -11,6 +11,7 @@
 // is applied.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -440,6 +441,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         const double nrm = sqrt(2.0 * p->paths[k].info.l_out + 1.0);
         for (double& v : p->paths[k].cg) v *= nrm;
     }
+    if (const char* e = getenv("SOBEK_FUSED")) p->use_fused = atoi(e) != 0;
     build_direction(p, 0, p->fwd);
     build_direction(p, 1, p->tr);
     build_stream_tasks(p, p->fwd);
