@@ -108,6 +108,12 @@ struct Direction {
     std::vector<SClass> sclasses;
     STask* d_stasks = nullptr;
     SComp* d_scomps = nullptr;
+    // receiver-owned edge pass: source-major tasks over all multiplicities
+    std::vector<STask> etasks;
+    std::vector<SComp> ecomps;
+    std::vector<SClass> eclasses;
+    STask* d_etasks = nullptr;
+    SComp* d_ecomps = nullptr;
     int64_t* d_zb_off = nullptr;
     // fused kernels: stage list, per-group ranges and the stage-ordered bf16 copy of R
     std::vector<FStage> fstages;
@@ -208,6 +214,7 @@ struct EdgeView {          // how a traversal walks the graph
 
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s);
+void build_edge_tasks(const sobek_plan* p, Direction& dir);
 // receiver-owned edge pass: gphi_e = <Zbar, C_e>, gY_e = CG^T_Y(x, phi_e Zbar); with `dual` the
 // second-order terms that share Zbar: <Zbar, C(vx,Y)+C(x,vY)> and CG^T_Y(vx, phi Zbar) + CG^T_Y(x, vphi Zbar)
 cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,

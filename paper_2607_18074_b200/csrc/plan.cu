@@ -446,6 +446,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     build_direction(p, 1, p->tr);
     build_stream_tasks(p, p->fwd);
     build_stream_tasks(p, p->tr);
+    build_edge_tasks(p, p->fwd);
     build_fused_stages(p, p->fwd);
     build_fused_stages(p, p->tr);
     cudaError_t e = cudaGetDevice(&p->device);
@@ -471,6 +472,8 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         if (e == cudaSuccess) e = upload(d->path_group, &d->d_path_group);
         if (e == cudaSuccess) e = upload(d->stasks, &d->d_stasks);
         if (e == cudaSuccess) e = upload(d->scomps, &d->d_scomps);
+        if (e == cudaSuccess) e = upload(d->etasks, &d->d_etasks);
+        if (e == cudaSuccess) e = upload(d->ecomps, &d->d_ecomps);
         if (e == cudaSuccess) e = upload(d->zb_off, &d->d_zb_off);
         if (e == cudaSuccess) e = upload(d->fstages, &d->d_fstages);
         if (e == cudaSuccess) e = upload(d->fs_begin, &d->d_fs_begin);
@@ -507,7 +510,7 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
     for (Direction* d : {&p->fwd, &p->tr}) {
         cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);
         cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);
-        cudaFree(d->d_stasks); cudaFree(d->d_scomps); cudaFree(d->d_zb_off);
+        cudaFree(d->d_stasks); cudaFree(d->d_scomps); cudaFree(d->d_etasks); cudaFree(d->d_ecomps); cudaFree(d->d_zb_off);
         cudaFree(d->d_fstages); cudaFree(d->d_fs_begin); cudaFree(d->d_fs_count); cudaFree(d->d_fk_off);
     }
     (void)cudaGetLastError();
