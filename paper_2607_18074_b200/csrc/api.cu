@@ -21,6 +21,8 @@ struct Workspace {
     uint16_t *fFKh, *fFKl, *tFKh, *tFKl, *vfFKh, *vfFKl, *vtFKh, *vtFKl;   // stage-ordered copies (fused kernels)
     bool fused_f, fused_t;    // fused kernels usable for the receiver / sender direction
     float* gRp;               // fp32 accumulator of the R adjoint, packed [k][w] per group
+    float* part;              // split-K partial results of the weight-adjoint GEMM
+    int splits;
     float* zbar;              // fp32 adjoint state Zbar of one chunk (input of the edge pass)
     uint16_t *zbh, *zbl;      // bf16 (hi, lo) node state Z / dZ / V of one chunk
     uint16_t *gbh, *gbl;      // bf16 (hi, lo) rows of the chunk's output adjoint
@@ -50,6 +52,8 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         w.fKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.fKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
         w.tNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.tNKl = (uint16_t*)take(p->tr.nk_elems * 2);
         w.gRp = (float*)take((size_t)p->K * (size_t)p->N_w * 4);
+        w.splits = (int)std::max<size_t>(1, std::min<size_t>(kMaxSplits, kPartBudgetBytes / ((size_t)p->K * (size_t)p->N_w * 4)));
+        w.part = (float*)take((size_t)w.splits * (size_t)p->K * (size_t)p->N_w * 4);
     }
     if (order >= 2) {
         w.vfNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.vfNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
@@ -155,18 +159,25 @@ cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t 
     return fork.join();
 }
 
-// gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint)
+// gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint).  The contraction runs over every (node, component)
+// row of the chunk; it is cut into `splits` pieces that run concurrently and are summed in a fixed order.
 cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn, const uint16_t* zh,
-                           const uint16_t* zl, const uint16_t* gh, const uint16_t* gl, float* gRp, int* status,
-                           cudaStream_t s0) {
+                           const uint16_t* zl, const uint16_t* gh, const uint16_t* gl, float* gRp, float* part,
+                           int splits, int* status, cudaStream_t s0) {
+    const int64_t KN = (int64_t)p->K * p->N_w;
     Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
+        cudaStream_t s = fork.pick();
+        const int64_t kblocks = (nn * G.d_dst + 63) / 64;
+        const int sp = (int)std::max<int64_t>(1, std::min<int64_t>(splits, kblocks));
         cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
                                        gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
-                                       gRp + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 1, 1, status, s);
+                                       part + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 0, 1, status, s,
+                                       sp, KN);
+        if (e != cudaSuccess) return e;
+        e = launch_reduce_parts(gRp + G.rp_off, part + G.rp_off, (int64_t)G.D * G.c_dst, KN, sp, s);
         if (e != cudaSuccess) return e;
     }
     return fork.join();
@@ -243,7 +254,7 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
             CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
-                CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
+                CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
             }
             if (gphi || gY) {
                 CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
@@ -340,7 +351,7 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
                 // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
                 if (ggy && !fuse_dz) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
-                if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.status, s));
+                if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
             }
             if (hphi || hY) {
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate

@@ -43,6 +43,8 @@ struct TcArgs {
     int32_t stages;
     int32_t tmem_cols;          // power of two >= max(32, BN)
     int32_t mn_major;           // 0: A[M,Kd], B[N,Kd] row-major;  1: A^T[Kd,M], B^T[Kd,N] row-major
+    int32_t splits;             // gridDim.z: the contraction range is cut into this many pieces,
+    int64_t split_stride;       //   piece z writes its partial result to C + z*split_stride
     int* status;
 };
 
@@ -63,7 +65,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
     const int S = g.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * BM, n0 = blockIdx.y * g.BN;
-    const int num_kb = (int)((g.Kd + BK - 1) / BK);
+    const int num_kb_all = (int)((g.Kd + BK - 1) / BK);
+    const int kb_per = (num_kb_all + g.splits - 1) / g.splits;
+    const int kb_first = blockIdx.z * kb_per;
+    const int num_kb = max(0, min(kb_per, num_kb_all - kb_first));   // k-blocks of this piece
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(bar0 + 8 * s, 1); mbar_init(bar0 + 8 * (S + s), 1); }
@@ -90,19 +95,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
                 mbar_expect_tx(full, stage_bytes);
                 const uint32_t sa = sbase + s * stage_bytes;
                 if (!g.mn_major) {
-                    tma_load_2d(sa, &tmAh, kb * BK, m0, full);
-                    tma_load_2d(sa + a_bytes, &tmAl, kb * BK, m0, full);
-                    tma_load_2d(sa + 2 * a_bytes, &tmBh, kb * BK, n0, full);
-                    tma_load_2d(sa + 2 * a_bytes + b_bytes, &tmBl, kb * BK, n0, full);
+                    tma_load_2d(sa, &tmAh, (kb_first + kb) * BK, m0, full);
+                    tma_load_2d(sa + a_bytes, &tmAl, (kb_first + kb) * BK, m0, full);
+                    tma_load_2d(sa + 2 * a_bytes, &tmBh, (kb_first + kb) * BK, n0, full);
+                    tma_load_2d(sa + 2 * a_bytes + b_bytes, &tmBl, (kb_first + kb) * BK, n0, full);
                 } else {
                     // operands stored [Kd rows][M or N contiguous]: boxes of 64 MN-elements x 64 k-rows
                     for (int j = 0; j < BM / 64; ++j) {
-                        tma_load_2d(sa + j * (64 * BK * 2), &tmAh, m0 + 64 * j, kb * BK, full);
-                        tma_load_2d(sa + a_bytes + j * (64 * BK * 2), &tmAl, m0 + 64 * j, kb * BK, full);
+                        tma_load_2d(sa + j * (64 * BK * 2), &tmAh, m0 + 64 * j, (kb_first + kb) * BK, full);
+                        tma_load_2d(sa + a_bytes + j * (64 * BK * 2), &tmAl, m0 + 64 * j, (kb_first + kb) * BK, full);
                     }
                     for (int j = 0; j < g.BN / 64; ++j) {
-                        tma_load_2d(sa + 2 * a_bytes + j * (64 * BK * 2), &tmBh, n0 + 64 * j, kb * BK, full);
-                        tma_load_2d(sa + 2 * a_bytes + b_bytes + j * (64 * BK * 2), &tmBl, n0 + 64 * j, kb * BK, full);
+                        tma_load_2d(sa + 2 * a_bytes + j * (64 * BK * 2), &tmBh, n0 + 64 * j, (kb_first + kb) * BK, full);
+                        tma_load_2d(sa + 2 * a_bytes + b_bytes + j * (64 * BK * 2), &tmBl, n0 + 64 * j, (kb_first + kb) * BK, full);
                     }
                 }
             }
@@ -146,17 +151,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
         const int q = warp & 3;
         mbar_wait(bar0 + 8 * 2 * S, 0, g.status);
         tc_fence_after();
-        const int64_t m = (int64_t)m0 + q * 32 + lane;
-        float* crow = nullptr;
-        if (m < g.M) crow = g.C + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+        // The pipeline buffers are idle now: each warp parks its 32 x BN block there (row pitch BN+1, so
+        // that both the row-wise writes and the column-wise reads are bank-conflict free) and then writes
+        // C row by row with the lanes along the columns (coalesced).
+        float* park = reinterpret_cast<float*>(smem) + (size_t)q * 32 * (g.BN + 1);
         for (int c0 = 0; c0 < g.BN; c0 += 16) {
             float v[16];
             tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);   // warp-collective
-            if (crow) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int64_t n = (int64_t)n0 + c0 + j;
-                    if (n < g.N) crow[n] = g.accumulate ? crow[n] + v[j] : v[j];
+            for (int j = 0; j < 16; ++j) park[lane * (g.BN + 1) + c0 + j] = v[j];
+        }
+        __syncwarp();
+        for (int r = 0; r < 32; ++r) {
+            const int64_t m = (int64_t)m0 + q * 32 + r;
+            if (m >= g.M) break;
+            float* crow = g.C + blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+            for (int c = lane; c < g.BN; c += 32) {
+                const int64_t n = (int64_t)n0 + c;
+                if (n < g.N) {
+                    const float v = num_kb > 0 ? park[r * (g.BN + 1) + c] : 0.f;
+                    crow[n] = g.accumulate ? crow[n] + v : v;
                 }
             }
         }
@@ -217,6 +231,27 @@ __global__ void k_pack_R_bf16(const DPath* __restrict__ paths, const int64_t* __
 
 int64_t round8(int64_t v) { return (v + 7) & ~int64_t(7); }
 
+namespace {
+// dst[i] += part[0][i] + part[1][i] + ... in this fixed order (deterministic split-K reduction)
+__global__ void k_reduce_parts(float* __restrict__ dst, const float* __restrict__ part, int64_t n, int64_t stride,
+                               int splits) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        float s = dst[i];
+        for (int z = 0; z < splits; ++z) s += part[z * stride + i];
+        dst[i] = s;
+    }
+}
+}  // namespace
+
+cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s) {
+    if (n <= 0 || splits <= 0) return cudaSuccess;
+    const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    KernelTimer kt(K_GEMM, s);
+    k_reduce_parts<<<blocks, 256, 0, s>>>(dst, part, n, stride, splits);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int s_d, int64_t rows, int cols,
                          int64_t ld, void* hi, void* lo, cudaStream_t s) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
@@ -243,11 +278,13 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 // mn_major = 1: A^T[Kd][lda] (contiguous in m), B^T[Kd][ldb] (contiguous in n).
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
-                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s) {
+                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
+                           int64_t split_stride) {
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
     TcArgs g{};
     g.C = C; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate;
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
+    g.splits = std::max(1, std::min<int>(splits, (int)((Kd + BK - 1) / BK))); g.split_stride = split_stride;
     int BN;
     if (mn_major) BN = N <= 64 ? 64 : (N <= 128 ? 128 : 256);     // whole 64-wide boxes
     else BN = (int)std::min<int64_t>(256, (N + 15) / 16 * 16);
@@ -275,7 +312,7 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN));
+    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN), (unsigned)g.splits);
     KernelTimer kt(K_GEMM, s);
     k_gemm_tc<<<grid, TC_THREADS, sh, s>>>(tAh, tAl, tBh, tBl, g);
     count_launch();

@@ -290,7 +290,11 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
                                const float* R, void* hi, void* lo, cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
-                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s);
+                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
+                           int64_t split_stride = 0);
+cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
+constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
+constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);
