@@ -267,14 +267,17 @@ k_edge_pass(const EdgeArgs a, const int t_begin, const int t_count) {
     float* sVphi = sVY + a.dsh * 32;        // DUAL: [Kp][32]
     const bool has_vY = DUAL && a.vY != nullptr, has_vphi = DUAL && a.vphi != nullptr;
 
-    for (int64_t nl = (int64_t)blockIdx.x * EW + warp; nl < a.n_nodes; nl += (int64_t)gridDim.x * EW) {
+    // One CTA per receiver; its warps share the receiver's tasks (warp w takes tasks w, w+nw, ...), each
+    // accumulating partial gphi / gY of the same 32 edges in its own stage; the partials are then summed
+    // across warps in a fixed order by the owner thread of each output element.
+    const int nw = blockDim.x >> 5;
+    for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
         const int64_t node = a.node0 + nl;
         const int64_t seg0 = a.ev.ptr[node], seg1 = a.ev.ptr[node + 1];
         for (int64_t b0 = seg0; b0 < seg1; b0 += 32) {
             const int64_t e = b0 + lane;
             const bool valid = e < seg1;
             const int64_t sn = (int64_t)a.ev.col[valid ? e : seg0];
-            __syncwarp();
             for (int b = 0; b < a.dsh; ++b) {
                 sY[b * 32 + lane] = valid ? a.Y[e * a.dsh + b] : 0.f;
                 if (has_vY) sVY[b * 32 + lane] = valid ? a.vY[e * a.dsh + b] : 0.f;
@@ -285,21 +288,30 @@ k_edge_pass(const EdgeArgs a, const int t_begin, const int t_count) {
                 if (has_vphi) sVphi[q * 32 + lane] = (valid && q < a.K) ? a.vphi[e * a.K + q] : 0.f;
                 sGphi[q * 32 + lane] = 0.f;
             }
-            for (int t = 0; t < t_count; ++t)
+            __syncwarp();
+            for (int t = warp; t < t_count; t += nw)
                 run_task<CAP, KC, DS, DUAL>(a, a.tasks[t_begin + t], nl, sn, sY, sVY, sGY, sZ0, sZ1, sPhi, sVphi,
                                             sGphi, lane);
+            __syncthreads();
+            // fixed-order sum over the warps' partials; thread (warp, lane) owns the outputs of edge b0+lane
+            // with index == warp (mod nw)
             if (valid) {
                 if (a.phi_mode)
-                    for (int q = 0; q < a.K; ++q) {
+                    for (int q = warp; q < a.K; q += nw) {
+                        float v = 0.f;
+                        for (int w = 0; w < nw; ++w) v += smem[(size_t)w * a.warp_floats + (2 * a.dsh + Kp + q) * 32 + lane];
                         float* p = a.gphi + e * a.K + q;
-                        *p = (a.phi_mode == 2 ? *p : 0.f) + sGphi[q * 32 + lane];
+                        *p = (a.phi_mode == 2 ? *p : 0.f) + v;
                     }
                 if (a.Y_mode)
-                    for (int b = 0; b < a.dsh; ++b) {
+                    for (int b = warp; b < a.dsh; b += nw) {
+                        float v = 0.f;
+                        for (int w = 0; w < nw; ++w) v += smem[(size_t)w * a.warp_floats + (a.dsh + b) * 32 + lane];
                         float* p = a.gY + e * a.dsh + b;
-                        *p = (a.Y_mode == 2 ? *p : 0.f) + sGY[b * 32 + lane];
+                        *p = (a.Y_mode == 2 ? *p : 0.f) + v;
                     }
             }
+            __syncthreads();
         }
     }
 }
@@ -309,14 +321,15 @@ cudaError_t launch_one(EdgeArgs a, int t_begin, int t_count, cudaStream_t s) {
     const int Kp = (a.K + KC - 1) / KC * KC;
     a.zslab = CAP * XB * KC;
     a.warp_floats = 2 * a.dsh * 32 + 2 * Kp * 32 + 2 * a.zslab + (DUAL ? a.dsh * 32 + Kp * 32 : 0);
-    const size_t sh = (size_t)a.warp_floats * EW * sizeof(float);
+    const int nw = std::max(1, std::min(EW, t_count));
+    const size_t sh = (size_t)a.warp_floats * nw * sizeof(float);
     auto kern = k_edge_pass<CAP, KC, DS, DUAL>;
     if (sh > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
         if (e != cudaSuccess) return e;
     }
-    const int grid = (int)std::min<int64_t>((a.n_nodes + EW - 1) / EW, 148 * 8);
-    kern<<<grid, EW * 32, sh, s>>>(a, t_begin, t_count);
+    const int grid = (int)std::min<int64_t>(a.n_nodes, 148 * 32);
+    kern<<<grid, nw * 32, sh, s>>>(a, t_begin, t_count);
     return cudaGetLastError();
 }
 
