@@ -33,6 +33,11 @@ METRIC = "edges/s (one step = fwd + bwd + double-bwd)"
 FP32_FMA_LANES = 148 * 128            # SMs x FP32 lanes
 L2_FLUSH_BYTES = 512 << 20
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the edge-stream kernel,
+# from the ncu capture summarised in profiles/ncu_edge_stream_cfg2.md (average of the two kernel
+# classes of one pass).  Only known for the workload that was captured.
+NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 31.0e6, ("cfg2", "edge_pass"): 91.6e6}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -63,7 +68,8 @@ def work_model(plan):
     node = {"fwd": Gf, "bwd": 2 * Gf + Gt, "dbwd": 5 * Gf + 2 * Gt}
     # split of the edge work between the two edge-stream kernel classes
     cls = {"edge_stream_state": (KF + CG) + (KF + CG + KFt + CGt) + (3 * KF + 2 * CG + 3 * KFt + 2 * CGt),
-           "edge_pass": (2 * KF + 2 * CG) + (5 * KF + 3 * CG)}
+           "edge_pass": (2 * KF + 2 * CG) + (5 * KF + 3 * CG),
+           "fused_stream_gemm": 0}
     return edge, node, cls
 
 
@@ -150,7 +156,7 @@ def run_reference(args):
     d = synth.make_inputs(w, oracle.col_std())
     cores = oconv.threads()
     # one step = fwd+bwd+dbwd on a bounded contiguous receiver sample
-    n = min(d.N, max(cores, 8))
+    n = min(d.N, max(8 * cores, 64))
     act = np.arange(n)
     edges = int(d.row_ptr[n] - d.row_ptr[0])
 
@@ -342,13 +348,13 @@ def main():
     dom_ms, dom_launches = classes[dom]
     steps_timed = args.steps
     if dom == "node_gemm":
-        fmas = (node_w["fwd"] + node_w["bwd"] + node_w["dbwd"]) * N * steps_timed
+        fmas = 3 * (node_w["fwd"] + node_w["bwd"] + node_w["dbwd"]) * N * steps_timed   # three bf16 passes
     else:
         fmas = cls_w.get(dom, 0) * E * steps_timed
     alu_peak = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
     achieved = 2.0 * fmas / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
     roofline = {"kernel": dom, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                "frac": achieved / alu_peak, "traffic": None,
+                "frac": achieved / alu_peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
                 "peak_source": f"derived: 148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz "
                                f"(HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_tflops']} TFLOP/s {peaks['source']})",
                 "avg_launch_ms": dom_ms / max(dom_launches, 1), "launches": int(dom_launches),

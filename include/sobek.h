@@ -34,7 +34,10 @@
  *     Empty rows, self loops and duplicate edges are legal.
  *   - Every entry point returns 0 on success or a negative sobek_status.  Nothing
  *     throws.  The sobek_conv_* calls never allocate device memory and never
- *     synchronise: they only enqueue kernels on `stream`.  Results are bitwise
+ *     synchronise: they only enqueue work on `stream` and on side streams owned by the
+ *     plan that are forked from and joined back into `stream` with events (so the call
+ *     is ordered like a single kernel on `stream`).  Two calls using the same plan must
+ *     not be issued concurrently from different host threads.  Results are bitwise
  *     reproducible from run to run (fixed reduction order, no floating-point atomics).
  *   - Outputs are overwritten, never accumulated into.  A NULL output pointer means
  *     "not wanted"; a NULL direction pointer in sobek_conv_dbwd means zero.
@@ -204,7 +207,9 @@ int64_t sobek_launch_count(void);
  * Instrumentation for benchmarks (the paper has no counterpart).  While enabled, every kernel
  * launch is bracketed by two CUDA events on its stream.  sobek_timing_collect waits for them,
  * returns per kernel class the summed device time in milliseconds and the number of launches
- * (arrays of sobek_timing_classes() entries), and forgets them.  Host-side only; not thread-safe.
+ * (arrays of sobek_timing_classes() entries), and forgets them.  While enabled, kernels that normally run
+ * concurrently on the library's internal side streams are serialised on the caller's stream, so that the
+ * brackets do not overlap.  Host-side only; not thread-safe.
  */
 int sobek_timing_enable(int on);
 int sobek_timing_classes(void);

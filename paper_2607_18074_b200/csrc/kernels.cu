@@ -36,7 +36,9 @@ KernelTimer::~KernelTimer() {
 }
 
 Fork::Fork(const sobek_plan* p, cudaStream_t main) : p_(p), main_(main) {
-    if (p->n_side <= 0) return;
+    // while per-kernel timing is on, everything stays on the caller's stream so that the event
+    // brackets of different kernels do not overlap
+    if (p->n_side <= 0 || g_timing) return;
     if (cudaEventRecord(p->ev_fork, main) != cudaSuccess) { (void)cudaGetLastError(); return; }
     on_ = true;
 }
