@@ -81,7 +81,10 @@ enum { SOBEK_MAX_L = 4 };
  * l = 0..l_max, computes the real Clebsch-Gordan tensors and uploads the sparse tables to
  * the current CUDA device (the only device allocation the library ever makes; it is
  * released by sobek_plan_destroy).  `in`/`out` are host arrays.  K >= 1 is the width of
- * the radial embedding.  `flags` must be 0.
+ * the radial embedding.  `flags` must be 0.  If the environment variable SOBEK_FUSED is set to a
+ * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
+ * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise
+ * by the stream -> bounded state -> GEMM schedule, which is the faster one at present.
  * Errors: INVALID_ARG (null, mul < 1, parity not +-1, K < 1), UNSUPPORTED (l or l_max >
  * SOBEK_MAX_L, or no valid path), CUDA.
  */

@@ -219,3 +219,29 @@ def test_full_size_sampled(name):
         assert rel_err(got[0][act], ref[0][act]) <= BWD_TOL
         assert rel_err(got[1], ref[1]) <= BWD_TOL and rel_err(got[4], ref[4]) <= BWD_TOL
         assert rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL and rel_err(got[3][ed], ref[3][ed]) <= BWD_TOL
+
+
+# ---------------------------------------------------------------------------------------
+# the fused schedule (edge stream feeding the tensor core without leaving the SM)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["cfg2_N200", "cfg4_N150", "cfg5_N60", "ragged", "K20"])
+def test_fused_schedule(name, monkeypatch):
+    """The plan-level schedule switch selects the fused stream+contraction kernels for y, gx, ggy
+    and hx; results must match the oracle to the same tolerances."""
+    monkeypatch.setenv("SOBEK_FUSED", "1")
+    c = Case(CASES[name])
+    monkeypatch.delenv("SOBEK_FUSED")
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+    for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+    # hR not requested: ggy then comes from the fused directional kernel as well
+    import torch
+    i = c.plan.info
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    ggy, hx = new(c.N, i.C_y), new(c.N, i.C_x)
+    c.sb.conv_dbwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, c.vx, c.vY, c.vphi, c.vR, ggy, hx, None, None,
+                   None, c.ws(2))
+    ref = c.o_dbwd()
+    assert rel_err(ggy.cpu().numpy(), ref[0]) <= BWD_TOL and rel_err(hx.cpu().numpy(), ref[1]) <= BWD_TOL
+    for got, r, nm in zip(c.dbwd(), ref, ("ggy", "hx", "hY", "hphi", "hR")):
+        assert rel_err(got, r) <= BWD_TOL, nm
