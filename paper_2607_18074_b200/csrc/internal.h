@@ -169,6 +169,7 @@ namespace sobek {
 constexpr size_t kHeaderBytes = 256;
 // budget for the bounded node-state buffer (floats of Z / V held at once)
 constexpr size_t kStateBudgetBytes = size_t(256) << 20;
+constexpr int64_t kMinChunkNodes = 512;
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);
 

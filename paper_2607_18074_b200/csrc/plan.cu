@@ -372,8 +372,10 @@ int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order) {
     if (order >= 1) zb = std::max(zb, p->tr.zb_elems);
     int64_t per = 4 * zb + (order >= 1 ? 4 * p->fwd.state_floats + 4 * p->fwd.gb_elems : 0);
     per = std::max<int64_t>(per, 1);
+    // the budget bounds the chunk, but a chunk never has fewer than kMinChunkNodes nodes: below that the
+    // node-side kernels cannot fill the machine
     int64_t n = (int64_t)(kStateBudgetBytes / (size_t)per);
-    n = std::max<int64_t>(n, 1);
+    n = std::max<int64_t>(n, kMinChunkNodes);
     return std::min<int64_t>(std::max<int64_t>(N, 1), n);
 }
 

@@ -86,6 +86,10 @@ def test_workspace_does_not_grow_with_edges():
         # more nodes: bounded by the state budget, identical from some size on
         assert sb.workspace_bytes(plan, 10**6, 10**8, order) == sb.workspace_bytes(plan, 3 * 10**6, 10**8, order)
         assert sb.workspace_bytes(plan, 10**6, 10**8, order) < 400 * 2**20
+    # the widest benchmark contract: bounded by 512 nodes of state, whatever the graph size
+    w = synth.config("cfg5")
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    assert sb.workspace_bytes(plan, 50000, 2 * 10**6, 2) == sb.workspace_bytes(plan, 10**7, 4 * 10**8, 2) < 1400 * 2**20
 
 
 def test_argument_errors_are_status_codes():
