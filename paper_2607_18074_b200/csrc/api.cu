@@ -26,6 +26,8 @@ struct Workspace {
     float* zbar;              // fp32 adjoint state Zbar of one chunk (input of the edge pass)
     uint16_t *zbh, *zbl;      // bf16 (hi, lo) node state Z / dZ / V of one chunk
     uint16_t *gbh, *gbl;      // bf16 (hi, lo) rows of the chunk's output adjoint
+    // bf16 (hi, lo) copies of x, gy and vx, [N][C] each: the gathered operand of the tensor-core stream
+    uint16_t *xsh, *xsl, *gsh, *gsl, *vsh, *vsl;
     int64_t chunk;
     size_t bytes;
 };
@@ -70,8 +72,19 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
         w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
     }
+    if (p->use_tc_stream) {
+        const size_t nx = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 2, ny = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 2;
+        if (p->fwd.tc[0].ok || (order >= 2 && p->fwd.tc[1].ok)) { w.xsh = (uint16_t*)take(nx); w.xsl = (uint16_t*)take(nx); }
+        if (order >= 1 && (p->tr.tc[0].ok || (order >= 2 && p->tr.tc[1].ok))) { w.gsh = (uint16_t*)take(ny); w.gsl = (uint16_t*)take(ny); }
+        if (order >= 2 && p->fwd.tc[1].ok) { w.vsh = (uint16_t*)take(nx); w.vsl = (uint16_t*)take(nx); }
+    }
     w.bytes = off;
     return w;
+}
+
+// whole feature matrix [N][C] -> bf16 (hi, lo)
+cudaError_t split_features(const float* src, int64_t N, int C, uint16_t* h, uint16_t* l, cudaStream_t s) {
+    return launch_split(src, C, 0, 1, N, C, C, h, l, s);
 }
 
 int check_common(const sobek_plan* p, const sobek_graph* g, void* ws, size_t ws_bytes, int order) {
@@ -221,9 +234,11 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
         return SOBEK_OK;
     }
     CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+    SplitSrc xs{};
+    if (w.xsh) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
-        CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+        CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
         CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
     }
     return SOBEK_OK;
@@ -246,6 +261,9 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
         return SOBEK_OK;
     }
     const EdgeView rv = receiver_view(g);
+    SplitSrc xs{}, gs{};
+    if (w.xsh && gR) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
+    if (w.gsh && gx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (gR || gphi || gY) {
         if (gphi || gY) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
         if (gR) CK(launch_fill_zero(w.gRp, KN, s));
@@ -253,7 +271,7 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
             const int64_t nn = std::min(w.chunk, g->N - n0);
             CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
-                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
                 CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
             }
             if (gphi || gY) {
@@ -274,7 +292,7 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
             CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
             for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
                 const int64_t nn = std::min(w.chunk, g->N - n0);
-                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
                 CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
             }
         }
@@ -315,6 +333,12 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
     if (!(vY || vphi || vR)) { if ((rc = zero_out(hx, g->N * (int64_t)p->C_x))) return rc; }
 
     const EdgeView rv = receiver_view(g);
+    SplitSrc xs{}, gs{};
+    if (w.xsh && (ggy || hR)) {
+        CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl;
+        if (vx && w.vsh) { CK(split_features(vx, g->N, p->C_x, w.vsh, w.vsl, s)); xs.vh = w.vsh; xs.vl = w.vsl; }
+    }
+    if (w.gsh && hx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (ggy || hR || hphi || hY) {
         if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
         // ggy = Z vR + dZ R.  The fused kernels produce it without leaving the SM; when hR is wanted too the
@@ -343,13 +367,13 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint with d(gy) = 0)
             int ggy_written = ggy_done;
             if (ggy && vR && !fuse_ggy) {
-                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
                 CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
                 ggy_written = 1;
             }
             if (((ggy && !fuse_dz) || hR) && any_edge_dir) {
                 // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
-                CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, xs, Y, vY, phi, vphi, 1, w.zbh, w.zbl, w.status, s));
                 if (ggy && !fuse_dz) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
                 if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
             }
@@ -393,12 +417,12 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             const int64_t nn = std::min(w.chunk, g->N - n0);
             int wrote = 0;
             if (vY || vphi) {   // dV = V(gy; vY, phi) + V(gy; Y, vphi) in one pass
-                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, vY, phi, vphi, 1, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, vY, phi, vphi, 1, w.zbh, w.zbl, w.status, s));
                 CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, hx, 0, w.status, s));
                 wrote = 1;
             }
             if (vR) {
-                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, s));
+                CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
                 CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, hx, wrote, w.status, s));
             }
         }

@@ -54,42 +54,42 @@ struct EdgeArgs {
 __device__ __forceinline__ void cp_async4(float* dst, const float* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
+__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+
 // Stage the Zbar rows of the task's components for multiplicities [u0, u0+XB) and K-chunk [q0, q0+KC):
-// sZ[(c*XB + uu)*KC + q]
+// sZ[(c*KC + q)*XB + uu]   (the contraction index of the state is k = koff + q*c_src + u, so the XB
+// multiplicities of one (component, q) are 16 contiguous bytes)
 template <int CAP, int KC>
 __device__ __forceinline__ void stage_zbar(const EdgeArgs& a, const STask& T, const SComp* comps, const int64_t nl,
                                            int u0, int q0, float* sZ, int lane) {
-    const bool vec = (a.K & 3) == 0;       // then every row pitch and offset is a multiple of 4 floats
+    const bool vec = (T.c_src & 3) == 0;       // then every row pitch and offset is a multiple of 4 floats
     if (vec) {
-        constexpr int per_c = XB * KC / 4;  // 16-byte pieces per component
-        for (int i = lane; i < T.ncomp * per_c; i += 32) {
-            const int c = i / per_c, r = i - c * per_c;
-            const int uu = r / (KC / 4), q = (r - uu * (KC / 4)) * 4;
+        for (int i = lane; i < T.ncomp * KC; i += 32) {
+            const int c = i / KC, q = i - c * KC;
             const SComp cp = comps[c];
             const DGroup G = a.groups[cp.group];
-            float* dst = sZ + (c * XB + uu) * KC + q;
-            if (u0 + uu < T.c_src && q0 + q < a.K)
+            float* dst = sZ + i * XB;
+            if (u0 + XB <= T.c_src && q0 + q < a.K)
                 cp_async16(dst, a.Zbar + a.n_nodes * G.z_off + (nl * G.d_dst + cp.o) * (int64_t)G.D + cp.koff +
-                                    (int64_t)(u0 + uu) * a.K + q0 + q);
+                                    (int64_t)(q0 + q) * T.c_src + u0);
             else
                 *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
         }
     } else {
-        for (int i = lane; i < T.ncomp * XB * KC; i += 32) {
-            const int c = i / (XB * KC), r = i - c * (XB * KC);
-            const int uu = r / KC, q = r - uu * KC;
+        for (int i = lane; i < T.ncomp * KC * XB; i += 32) {
+            const int uu = i % XB, cq = i / XB;
+            const int c = cq / KC, q = cq - c * KC;
             const SComp cp = comps[c];
             const DGroup G = a.groups[cp.group];
             float* dst = sZ + i;
             if (u0 + uu < T.c_src && q0 + q < a.K)
                 cp_async4(dst, a.Zbar + a.n_nodes * G.z_off + (nl * G.d_dst + cp.o) * (int64_t)G.D + cp.koff +
-                                   (int64_t)(u0 + uu) * a.K + q0 + q);
+                                   (int64_t)(q0 + q) * T.c_src + u0 + uu);
             else
                 *dst = 0.f;
         }
@@ -183,43 +183,40 @@ __device__ __forceinline__ void run_task(const EdgeArgs& a, const STask T, const
 #pragma unroll
             for (int c = 0; c < CAP; ++c) {
                 if (c < ncomp) {
+                    float Co[XB], Cb[XB], Cbv[XB];
 #pragma unroll
                     for (int uu = 0; uu < XB; ++uu) {
-                        float Co = 0.f;
+                        float v = 0.f;
 #pragma unroll
                         for (int s = 0; s < DS; ++s) {
-                            if (!DUAL) Co = fmaf(xs[s][uu], m[c][s], Co);
+                            if (!DUAL) v = fmaf(xs[s][uu], m[c][s], v);
                             else {
-                                if (has_vx) Co = fmaf(vxs[s][uu], m[c][s], Co);
-                                if (has_vY) Co = fmaf(xs[s][uu], dm[c][s], Co);
+                                if (has_vx) v = fmaf(vxs[s][uu], m[c][s], v);
+                                if (has_vY) v = fmaf(xs[s][uu], dm[c][s], v);
                             }
                         }
-                        const float4* z4 = reinterpret_cast<const float4*>(sZ + (c * XB + uu) * KC);
-                        float Cb = 0.f, Cbv = 0.f;
+                        Co[uu] = v; Cb[uu] = 0.f; Cbv[uu] = 0.f;
+                    }
+                    const float4* z4 = reinterpret_cast<const float4*>(sZ + c * KC * XB);
 #pragma unroll
-                        for (int q4 = 0; q4 < KC / 4; ++q4) {
-                            const float4 z = z4[q4];
-                            gp[4 * q4] = fmaf(z.x, Co, gp[4 * q4]);
-                            gp[4 * q4 + 1] = fmaf(z.y, Co, gp[4 * q4 + 1]);
-                            gp[4 * q4 + 2] = fmaf(z.z, Co, gp[4 * q4 + 2]);
-                            gp[4 * q4 + 3] = fmaf(z.w, Co, gp[4 * q4 + 3]);
-                            Cb = fmaf(ph[4 * q4], z.x, Cb);
-                            Cb = fmaf(ph[4 * q4 + 1], z.y, Cb);
-                            Cb = fmaf(ph[4 * q4 + 2], z.z, Cb);
-                            Cb = fmaf(ph[4 * q4 + 3], z.w, Cb);
-                            if (has_vphi) {
-                                Cbv = fmaf(vph[4 * q4], z.x, Cbv);
-                                Cbv = fmaf(vph[4 * q4 + 1], z.y, Cbv);
-                                Cbv = fmaf(vph[4 * q4 + 2], z.z, Cbv);
-                                Cbv = fmaf(vph[4 * q4 + 3], z.w, Cbv);
-                            }
+                    for (int q = 0; q < KC; ++q) {
+                        const float4 z = z4[q];       // the XB multiplicities of (component c, q)
+                        const float zz[XB] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                        for (int uu = 0; uu < XB; ++uu) {
+                            gp[q] = fmaf(zz[uu], Co[uu], gp[q]);
+                            Cb[uu] = fmaf(ph[q], zz[uu], Cb[uu]);
+                            if (has_vphi) Cbv[uu] = fmaf(vph[q], zz[uu], Cbv[uu]);
                         }
+                    }
+#pragma unroll
+                    for (int uu = 0; uu < XB; ++uu) {
 #pragma unroll
                         for (int s = 0; s < DS; ++s) {
-                            if (!DUAL) G[c][s] = fmaf(xs[s][uu], Cb, G[c][s]);
+                            if (!DUAL) G[c][s] = fmaf(xs[s][uu], Cb[uu], G[c][s]);
                             else {
-                                if (has_vx) G[c][s] = fmaf(vxs[s][uu], Cb, G[c][s]);
-                                if (has_vphi) G[c][s] = fmaf(xs[s][uu], Cbv, G[c][s]);
+                                if (has_vx) G[c][s] = fmaf(vxs[s][uu], Cb[uu], G[c][s]);
+                                if (has_vphi) G[c][s] = fmaf(xs[s][uu], Cbv[uu], G[c][s]);
                             }
                         }
                     }

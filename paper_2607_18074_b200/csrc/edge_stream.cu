@@ -57,9 +57,13 @@ void build_stream_tasks(const sobek_plan* p, Direction& dir) {
 }
 
 cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
-                          int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
-                          const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s) {
+                          int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,
+                          const float* vY, const float* phi, const float* vphi, int dual, void* zh, void* zl,
+                          int* status, cudaStream_t s) {
     if (n_nodes <= 0 || dir.stasks.empty()) return cudaSuccess;
+    // tensor-core stream when the profile allows it and the caller made the bf16 copies of the sources
+    if (p->use_tc_stream && dir.tc[dual ? 1 : 0].ok && status && ss.h && ss.l && (!vsrc || (ss.vh && ss.vl)))
+        return launch_stream_tc(p, dir, ev, node0, n_nodes, ss, Y, vY, phi, vphi, dual, zh, zl, status, s);
     const int KC = p->K <= 8 ? 8 : 16;
     StreamArgsHost a{};
     a.tasks = dir.d_stasks; a.comps = dir.d_scomps;

@@ -186,38 +186,22 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
                 }
             }
         }
-        // ---- write the state slice as bf16 (hi, lo)
+        // ---- write the state slice as bf16 (hi, lo); contraction index k = koff + q*c_src + u
         if (act) {
 #pragma unroll
             for (int c = 0; c < CAP; ++c) {
                 if (c < ncomp) {
                     const SComp cp = comps[c];
                     const int64_t ld = a.zb_ld[cp.group];
-                    const int64_t off = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * ld + cp.koff +
-                                        (int64_t)u * a.K + q0;
-                    if ((a.K & 7) == 0) {
+                    const int64_t off = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * ld + cp.koff + u;
 #pragma unroll
-                        for (int q = 0; q < KC; q += 8) {
-                            if (q0 + q >= a.K) break;
-                            __align__(16) __nv_bfloat16 h[8], l[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float v = acc[c][q + j];
-                                h[j] = __float2bfloat16_rn(v);
-                                l[j] = __float2bfloat16_rn(v - __bfloat162float(h[j]));
-                            }
-                            *reinterpret_cast<uint4*>((__nv_bfloat16*)a.zh + off + q) = *reinterpret_cast<const uint4*>(h);
-                            *reinterpret_cast<uint4*>((__nv_bfloat16*)a.zl + off + q) = *reinterpret_cast<const uint4*>(l);
-                        }
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < KC; ++q) {
-                            if (q0 + q < a.K) {
-                                const float v = acc[c][q];
-                                const __nv_bfloat16 h = __float2bfloat16_rn(v);
-                                ((__nv_bfloat16*)a.zh)[off + q] = h;
-                                ((__nv_bfloat16*)a.zl)[off + q] = __float2bfloat16_rn(v - __bfloat162float(h));
-                            }
+                    for (int q = 0; q < KC; ++q) {
+                        if (q0 + q < a.K) {
+                            const float v = acc[c][q];
+                            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                            const int64_t o = off + (int64_t)(q0 + q) * T.c_src;
+                            ((__nv_bfloat16*)a.zh)[o] = h;
+                            ((__nv_bfloat16*)a.zl)[o] = __float2bfloat16_rn(v - __bfloat162float(h));
                         }
                     }
                 }

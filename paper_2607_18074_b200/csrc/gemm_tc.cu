@@ -219,7 +219,7 @@ __global__ void k_pack_R_bf16(const DPath* __restrict__ paths, const int64_t* __
         const int us = (int)(r / K);
         const int u = transposed ? n : us, w = transposed ? us : n;
         const float v = R[(int64_t)q * N_w + P.w_off + (int64_t)u * P.c_out + w];
-        const int64_t k = (int64_t)P.koff + (int64_t)us * K + q;
+        const int64_t k = (int64_t)P.koff + (int64_t)q * P.c_src + us;
         const int64_t o = n_major ? base + (int64_t)n * ld + k : base + k * ld + n;
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         hi[o] = h;

@@ -29,7 +29,7 @@ struct DPath {
     int32_t d_sh;      // 2 l_sh + 1
     int32_t d_dst;     // 2 l_dst + 1
     int32_t c_dst;     // destination multiplicity
-    int32_t koff;      // offset in the group's contraction axis; k = koff + u*K + q
+    int32_t koff;      // offset in the group's contraction axis; k = koff + q*c_src + u
     int32_t m_off;     // offset of M[s][o] inside the group's per-edge M area
     int32_t tabM;      // index into tab_ptr: entry (s*d_dst+o) -> terms (b, coef)
     int32_t tabY;      // index into tab_ptr: b -> terms (s*d_dst+o, coef)   (adjoint wrt Y)
@@ -79,6 +79,56 @@ struct STask {         // one warp's task of the edge stream (source-major)
     int32_t pad;
 };
 
+// --- tensor-core edge stream (stream_tc.cu) ------------------------------------------------
+// Per receiver and source irrep block the fold over its edges is the dense contraction
+//     Z[(comp,q), u] = sum_{(e,s)} ( phi_e[q] * M_e[s,comp] ) * x_{src(e)}[s,u]
+// A "unit" is one accumulator tile of it: up to 128 rows (comp,q) of one source block.  A "set" is
+// the group of units one CTA pass holds at once (bounded by shared memory and TMEM columns).
+struct TEnt {          // one (unit, component, s) entry of a set: a row block of one A slab
+    int32_t tab;       // tab_ptr index of the entry's sparse terms (b, coef)
+    int32_t sh_off;    // offset of the path's SH block inside a Y row
+    int32_t a_off;     // byte offset of row (component*KP) of slab s inside one A copy
+    int32_t pad;
+};
+struct TUnit {
+    int32_t blk;           // index into the block list
+    int32_t comp_begin;    // first component (index into the TC component list)
+    int32_t ncomp;
+    int32_t a_off;         // byte offset of the unit's slab 0 inside one A copy
+    int32_t slab_stride;   // bytes between consecutive s slabs of the unit
+    int32_t tmem_col;      // first accumulator column
+    int32_t pad[2];
+};
+struct TBlk {
+    int32_t src_off, c_src, d_src;
+    int32_t ncols;         // accumulator columns = c_src rounded up to 16
+    int32_t b_off;         // byte offset of the block's slab 0 inside one B copy
+    int32_t slab_bytes;    // bytes of one (s, 16 edges) slab = 2048 * ceil(c_src / 64)
+    int32_t pad[2];
+};
+struct TSet {
+    int32_t unit_begin, nunit, blk_begin, nblk, ent_begin, nent;
+    int32_t b_items;       // float4 pieces of sender rows gathered per 16-edge batch
+    int32_t pad;
+};
+struct TcSets {
+    bool ok = false;       // the tensor-core stream supports this direction
+    std::vector<TSet> sets;
+    std::vector<TUnit> units;
+    std::vector<TBlk> blks;
+    std::vector<TEnt> ents;
+    std::vector<SComp> comps;
+    TSet* d_sets = nullptr;
+    TUnit* d_units = nullptr;
+    TBlk* d_blks = nullptr;
+    TEnt* d_ents = nullptr;
+    SComp* d_comps = nullptr;
+    int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
+    int32_t max_ent = 0, tmem_cols = 32;
+    int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
+    int32_t smem_bytes = 0, ctas_per_sm = 1;
+};
+
 struct FStage {        // one 256-column stage of the fused kernel's contraction axis
     int32_t path;
     int32_t u0;        // first multiplicity of the block (256/KP wide)
@@ -108,6 +158,7 @@ struct Direction {
     std::vector<SClass> sclasses;
     STask* d_stasks = nullptr;
     SComp* d_scomps = nullptr;
+    TcSets tc[2];                     // tensor-core stream: [0] plain, [1] dual
     // receiver-owned edge pass: source-major tasks over all multiplicities
     std::vector<STask> etasks;
     std::vector<SComp> ecomps;
@@ -153,6 +204,7 @@ struct sobek_plan {
     int32_t* d_tab_idx = nullptr;
     float* d_tab_coef = nullptr;
     int device = -1;
+    bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -211,6 +263,7 @@ struct EdgeView {          // how a traversal walks the graph
     const int64_t* row_ptr;// receiver CSR (to recover the receiver of an edge id)
     int64_t N, E;
     int transposed;        // 0: source node = col[e];  1: source node = receiver(e)
+    const int32_t* recv;   // transposed only, optional: receiver of the edge at each position (else searched)
 };
 
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
@@ -227,9 +280,23 @@ cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
 
 // --- edge_stream.cu ---------------------------------------------------------------
 void build_stream_tasks(const sobek_plan* p, Direction& dir);
+// bf16 (hi, lo) copies of the source features of a traversal, [N][C_src] each (made once per call);
+// all NULL when the caller has none (the FP32-pipe stream is used then)
+struct SplitSrc {
+    const void* h = nullptr;
+    const void* l = nullptr;
+    const void* vh = nullptr;   // the same for the source direction of the dual stream (NULL without it)
+    const void* vl = nullptr;
+};
 cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
-                          int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
-                          const float* phi, const float* vphi, int dual, void* zh, void* zl, cudaStream_t s);
+                          int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,
+                          const float* vY, const float* phi, const float* vphi, int dual, void* zh, void* zl,
+                          int* status, cudaStream_t s);
+// --- stream_tc.cu ---------------------------------------------------------------------
+void build_tc_sets(const sobek_plan* p, Direction& dir);
+cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
+                             int64_t n_nodes, const SplitSrc& ss, const float* Y, const float* vY, const float* phi,
+                             const float* vphi, int dual, void* zh, void* zl, int* status, cudaStream_t s);
 
 cudaError_t stream_launch_k8(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);
 cudaError_t stream_launch_k16(const void* args, int cls, int t_begin, int t_count, cudaStream_t s);

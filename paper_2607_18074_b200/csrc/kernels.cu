@@ -121,8 +121,8 @@ __global__ void k_fill_zero(float* __restrict__ p, int64_t n) {
 
 // ------------------------------------------------------------------------------------
 // R re-layout.  One blockIdx.y per path; element (us, q, n) of the path's slab:
-//   forward    : us = u (input mult.), n = w      Rp[rp_off + (koff + u*K + q)*c_out + w]
-//   transposed : us = w (output mult.), n = u     Rt[rp_off + (koff + w*K + q)*c_in  + u]
+//   forward    : us = u (input mult.), n = w      Rp[rp_off + (koff + q*c_in  + u)*c_out + w]
+//   transposed : us = w (output mult.), n = u     Rt[rp_off + (koff + q*c_out + w)*c_in  + u]
 // both read/write R[q*N_w + w_off + u*c_out + w].
 // ------------------------------------------------------------------------------------
 template <bool UNPACK>
@@ -138,7 +138,7 @@ __global__ void k_pack_R(const DPath* __restrict__ paths, int transposed, int K,
         const int us = (int)(r / K);
         const int u = transposed ? n : us, w = transposed ? us : n;
         const int64_t ri = (int64_t)q * N_w + P.w_off + (int64_t)u * P.c_out + w;
-        const int64_t pi = P.rp_off + ((int64_t)P.koff + (int64_t)us * K + q) * P.c_dst + n;
+        const int64_t pi = P.rp_off + ((int64_t)P.koff + (int64_t)q * P.c_src + us) * P.c_dst + n;
         if (UNPACK) dst[ri] = src[pi]; else dst[pi] = src[ri];
     }
 }

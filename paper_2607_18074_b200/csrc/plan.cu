@@ -448,6 +448,9 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     build_direction(p, 1, p->tr);
     build_stream_tasks(p, p->fwd);
     build_stream_tasks(p, p->tr);
+    if (const char* e = getenv("SOBEK_TC_STREAM")) p->use_tc_stream = atoi(e) != 0;
+    build_tc_sets(p, p->fwd);
+    build_tc_sets(p, p->tr);
     build_edge_tasks(p, p->fwd);
     build_fused_stages(p, p->fwd);
     build_fused_stages(p, p->tr);
@@ -481,6 +484,14 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         if (e == cudaSuccess) e = upload(d->fs_begin, &d->d_fs_begin);
         if (e == cudaSuccess) e = upload(d->fs_count, &d->d_fs_count);
         if (e == cudaSuccess) e = upload(d->fk_off, &d->d_fk_off);
+        for (TcSets& t : d->tc) {
+            if (!t.ok) continue;
+            if (e == cudaSuccess) e = upload(t.sets, &t.d_sets);
+            if (e == cudaSuccess) e = upload(t.units, &t.d_units);
+            if (e == cudaSuccess) e = upload(t.blks, &t.d_blks);
+            if (e == cudaSuccess) e = upload(t.ents, &t.d_ents);
+            if (e == cudaSuccess) e = upload(t.comps, &t.d_comps);
+        }
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -514,6 +525,9 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
         cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);
         cudaFree(d->d_stasks); cudaFree(d->d_scomps); cudaFree(d->d_etasks); cudaFree(d->d_ecomps); cudaFree(d->d_zb_off);
         cudaFree(d->d_fstages); cudaFree(d->d_fs_begin); cudaFree(d->d_fs_count); cudaFree(d->d_fk_off);
+        for (TcSets& t : d->tc) {
+            cudaFree(t.d_sets); cudaFree(t.d_units); cudaFree(t.d_blks); cudaFree(t.d_ents); cudaFree(t.d_comps);
+        }
     }
     (void)cudaGetLastError();
     delete p;

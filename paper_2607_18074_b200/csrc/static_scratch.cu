@@ -82,7 +82,7 @@ extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, 
     for (int64_t n0 = 0; n0 < g->N; n0 += chunk) {
         const int64_t nn = std::min(chunk, g->N - n0);
         // every element of the chunk's state that the contraction reads is overwritten first
-        CKS(launch_stream(p, dir, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, zh, zl, s));
+        CKS(launch_stream(p, dir, rv, n0, nn, x, nullptr, SplitSrc{}, Y, nullptr, phi, nullptr, 0, zh, zl, (int*)base, s));
         for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
             const DGroup& G = dir.groups[gi];
             if (G.path_end == G.path_begin) continue;
