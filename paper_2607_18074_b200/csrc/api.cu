@@ -28,6 +28,7 @@ struct Workspace {
     uint16_t *gbh, *gbl;      // bf16 (hi, lo) rows of the chunk's output adjoint
     // bf16 (hi, lo) copies of x, gy and vx, [N][C] each: the gathered operand of the tensor-core stream
     uint16_t *xsh, *xsl, *gsh, *gsl, *vsh, *vsl;
+    uint16_t *zqh, *zql;      // bf16 (hi, lo) adjoint state of one chunk (input of the tensor-core edge pass)
     int64_t chunk;
     size_t bytes;
 };
@@ -72,11 +73,15 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
         w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
     }
-    if (p->use_tc_stream) {
+    if (order >= 1 && p->use_tc_edge && p->fwd.etc[0].ok) {
+        w.zqh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.zb_elems * 2);
+        w.zql = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.zb_elems * 2);
+    }
+    if (p->use_tc_stream || (p->use_tc_edge && p->fwd.etc[0].ok)) {
         const size_t nx = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 2, ny = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 2;
-        if (p->fwd.tc[0].ok || (order >= 2 && p->fwd.tc[1].ok)) { w.xsh = (uint16_t*)take(nx); w.xsl = (uint16_t*)take(nx); }
+        if (p->fwd.tc[0].ok || (order >= 2 && p->fwd.tc[1].ok) || (order >= 1 && w.zqh)) { w.xsh = (uint16_t*)take(nx); w.xsl = (uint16_t*)take(nx); }
         if (order >= 1 && (p->tr.tc[0].ok || (order >= 2 && p->tr.tc[1].ok))) { w.gsh = (uint16_t*)take(ny); w.gsl = (uint16_t*)take(ny); }
-        if (order >= 2 && p->fwd.tc[1].ok) { w.vsh = (uint16_t*)take(nx); w.vsl = (uint16_t*)take(nx); }
+        if (order >= 2 && (p->fwd.tc[1].ok || (w.zqh && p->fwd.etc[1].ok))) { w.vsh = (uint16_t*)take(nx); w.vsl = (uint16_t*)take(nx); }
     }
     w.bytes = off;
     return w;
@@ -156,15 +161,23 @@ cudaError_t mix_tc(const sobek_plan* p, const Direction& dir, int64_t n0, int64_
 }
 
 // Zbar_g = gy_g * Rp_g^T       (Eq. receiver_adjoint)
+// With zqh / zql the result is written as bf16 (hi, lo) rows in the layout of the stream's state instead.
 cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t nn, const uint16_t* gh,
                              const uint16_t* gl, const uint16_t* knh, const uint16_t* knl, float* Zbar, int* status,
-                             cudaStream_t s0) {
+                             cudaStream_t s0, uint16_t* zqh = nullptr, uint16_t* zql = nullptr) {
     Fork fork(p, s0);
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
         cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
-        cudaError_t e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+        cudaError_t e;
+        if (zqh)
+            e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                               knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi], nullptr, dir.nk_ld[gi], 0, 1,
+                               nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, zqh + nn * dir.zb_off[gi],
+                               zql + nn * dir.zb_off[gi]);
+        else
+            e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
                                        knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi],
                                        Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s);
         if (e != cudaSuccess) return e;
@@ -262,7 +275,8 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     }
     const EdgeView rv = receiver_view(g);
     SplitSrc xs{}, gs{};
-    if (w.xsh && gR) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
+    const bool tc_edge = w.zqh != nullptr;
+    if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     if (w.gsh && gx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (gR || gphi || gY) {
         if (gphi || gY) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
@@ -275,9 +289,15 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
                 CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
             }
             if (gphi || gY) {
-                CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
-                CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
-                                    gphi ? 1 : 0, gY ? 1 : 0, s));
+                if (tc_edge) {
+                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, nullptr, w.status, s, w.zqh, w.zql));
+                    CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql, gphi, gY,
+                                           gphi ? 1 : 0, gY ? 1 : 0, w.status, s));
+                } else {
+                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
+                                        gphi ? 1 : 0, gY ? 1 : 0, s));
+                }
             }
         }
         if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
@@ -334,7 +354,8 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
 
     const EdgeView rv = receiver_view(g);
     SplitSrc xs{}, gs{};
-    if (w.xsh && (ggy || hR)) {
+    const bool tc_edge_plain = w.zqh != nullptr, tc_edge_dual = tc_edge_plain && p->fwd.etc[1].ok && (!vx || w.vsh);
+    if (w.xsh && (ggy || hR || ((hphi || hY) && tc_edge_plain))) {
         CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl;
         if (vx && w.vsh) { CK(split_features(vx, g->N, p->C_x, w.vsh, w.vsl, s)); xs.vh = w.vsh; xs.vl = w.vsl; }
     }
@@ -381,15 +402,28 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate
                 if (any_edge_dir) {
                     // the three direction terms that share Zbar = gy R^T, in one pass
-                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
-                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbar, hphi, hY,
-                                        hphi ? pm : 0, hY ? ym : 0, s));
+                    if (tc_edge_dual) {
+                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, nullptr, w.status, s, w.zqh, w.zql));
+                        CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, vY, phi, vphi, 1, w.zqh, w.zql, hphi, hY,
+                                               hphi ? pm : 0, hY ? ym : 0, w.status, s));
+                    } else {
+                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbar, hphi, hY,
+                                            hphi ? pm : 0, hY ? ym : 0, s));
+                    }
                     pm = ym = 2;
                 }
                 if (vR) {   // the term through dZbar = gy vR^T
-                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
-                    CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, hphi, hY,
-                                        hphi ? pm : 0, hY ? ym : 0, s));
+                    if (tc_edge_plain) {
+                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, nullptr, w.status, s, w.zqh, w.zql));
+                        SplitSrc xp{}; xp.h = xs.h; xp.l = xs.l;
+                        CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xp, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql, hphi, hY,
+                                               hphi ? pm : 0, hY ? ym : 0, w.status, s));
+                    } else {
+                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
+                        CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, hphi, hY,
+                                            hphi ? pm : 0, hY ? ym : 0, s));
+                    }
                 }
             }
         }

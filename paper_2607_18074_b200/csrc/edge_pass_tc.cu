@@ -1,0 +1,714 @@
+// Receiver-owned edge pass on the tensor cores (sm_100a, tcgen05 / TMEM), warp-specialised.
+//
+// The two edge outputs of the backward program (Section "Receiver-factorized backward";
+// Eqs. streamed_radial_adjoints, streamed_operand_adjoints) share, per receiver i, source irrep block and
+// batch of 16 edges, the dense contraction over the multiplicity u
+//     D[(s,e), (comp,q)] = sum_u x_{src(e)}[s,u] * Zbar_i[(comp,q), u]
+// whose operands are plain copies: the gathered bf16 (hi, lo) sender rows (rows (s,e), K-major) and the
+// bf16 (hi, lo) rows of the adjoint state Zbar = gy R^T of the receiver (rows (comp,q), K-major), both in
+// the 128-byte-swizzled layout that tcgen05.mma reads.  The FP32 pipes only run the epilogue
+//     gM_e[s,comp] = sum_q phi_e[q] * D[(s,e),(comp,q)]          -> gY_e[b]  = sum c[s,b,comp] gM_e[s,comp]
+//     gphi_e[q]    = sum_{s,comp} M_e[s,comp] * D[(s,e),(comp,q)]
+// with one thread per accumulator row (s,e).  fp32 parity comes from the split-bf16 product
+// a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo.  Every output element has exactly one writer and every sum
+// runs in a fixed order (bitwise reproducible).
+//
+// With DUAL the pass evaluates the second-order terms that share Zbar (Eq. streamed_operand_second_adjoints)
+//     hphi_e += <Zbar, C(vx,Y) + C(x,vY)>,   hY_e += CG^T_Y(vx, phi Zbar) + CG^T_Y(x, vphi Zbar)
+// from D (sender rows of x) and Dv (sender rows of vx):
+//     gM = sum_q ( vphi[q] D + phi[q] Dv ),   gphi[q] += dM D + M Dv.
+//
+// Roles of a CTA (one receiver at a time, its edges in groups of 64 and batches of 16, the accumulator
+// tiles of the profile in sets): loader warps (cp.async of the Zbar slabs of a set, of the batch's phi / Y
+// rows and of the sender rows into a two-stage ring), one MMA thread (two TMEM accumulator buffers), and
+// compute warps (coupling matrices M_e from the sparse CG table, epilogue, fixed-order reductions, output).
+// Every mbarrier wait is bounded.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace sobek {
+namespace {
+
+using namespace ptx;
+
+constexpr int TB = 16;          // edges per batch
+constexpr int EG = 64;          // edges per group (outputs of a group are accumulated in shared memory)
+constexpr int NCW = 8;          // compute warps
+constexpr int NLW = 2;          // loader warps
+constexpr int TT = (NCW + NLW + 1) * 32;
+constexpr int NS = 2;           // ring stages
+constexpr int PS = 20;          // row pitch (floats) of the [.][16 edges] stages
+
+struct EtArgs {
+    const TSet* sets;
+    const TUnit* units;
+    const TBlk* blks;
+    const TEnt* ents;
+    const SComp* comps;
+    const int32_t* inv_ptr;     // per set: dsh+1 offsets into inv_ent / inv_coef (b -> terms (entry, coef))
+    const int32_t* inv_ent;
+    const float* inv_coef;
+    const int64_t* zb_off;
+    const int32_t* zb_ld;
+    const int32_t* tab_ptr;
+    const int32_t* tab_idx;
+    const float* tab_coef;
+    const int64_t* row_ptr;
+    const int32_t* col;
+    int64_t node0, n_nodes;
+    const __nv_bfloat16* sh;
+    const __nv_bfloat16* sl;
+    const __nv_bfloat16* vsh;
+    const __nv_bfloat16* vsl;
+    const float* Y;
+    const float* vY;
+    const float* phi;
+    const float* vphi;
+    const __nv_bfloat16* zqh;   // bf16 (hi, lo) adjoint state of the chunk, laid out like the stream's state
+    const __nv_bfloat16* zql;
+    float* gphi;
+    float* gY;
+    int32_t phi_mode, Y_mode;   // 0 skip, 1 overwrite, 2 accumulate
+    int32_t K, dsh, C_src, nsets;
+    int32_t x_cap, z_cap, max_ent, tmem_cols, acc_cols, n_units;
+    int* status;
+};
+
+struct UInfo {     // what the MMA thread needs of a unit, kept in shared memory
+    uint32_t idesc, z_off, z_kb, x_off, x_kb, ksteps, nmt, npad;
+};
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__host__ __device__ inline int raw_floats(int KP, bool dual, int dsh) {
+    const int n = dual ? 2 : 1;
+    return n * TB * KP + n * TB * (dsh + 1);
+}
+
+template <int KP, bool DUAL>
+__global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr int NOP = DUAL ? 2 : 1;
+    const int YS = a.dsh + 1;
+    const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023);
+    const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.x_cap) + raw_bytes;
+    uint8_t* sRing = smem;                                     // stages: X1h X1l (X2h X2l) raw
+    uint8_t* sZ = sRing + (size_t)NS * stage_bytes;            // Zbar slabs of the current set: hi, lo
+    uint8_t* meta = sZ + (size_t)2 * a.z_cap;
+    float* sPhiT = reinterpret_cast<float*>(meta);             // [KP][PS]
+    float* sVphiT = sPhiT + KP * PS;
+    float* sYT = sVphiT + (DUAL ? KP * PS : 0);                // [dsh][PS]
+    float* sVYT = sYT + a.dsh * PS;
+    float* sM = sVYT + (DUAL ? a.dsh * PS : 0);                // [max_ent][PS]
+    float* sdM = sM + (size_t)a.max_ent * PS;
+    float* sGM = sdM + (DUAL ? (size_t)a.max_ent * PS : 0);    // [max_ent][PS]
+    float* sPphi = sGM + (size_t)a.max_ent * PS;               // [NCW*16][KP]: one row per (warp, edge)
+    float* accPhi = sPphi + NCW * 16 * KP;                     // [EG][KP]
+    float* accY = accPhi + EG * KP;                            // [EG][dsh]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(accY + ((EG * a.dsh + 1) & ~1));
+    // bars: full[NS], free[NS], zfull, zfree, acc_full[2], acc_free[2]
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
+    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_zfull = bar0 + 16 * NS, bar_zfree = bar_zfull + 8,
+                   bar_accfull = bar_zfull + 16, bar_accfree = bar_zfull + 32;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool has_vx = DUAL && a.vsh != nullptr, has_vY = DUAL && a.vY != nullptr, has_vphi = DUAL && a.vphi != nullptr;
+    const bool use_x = !DUAL || has_vY || has_vphi;     // D (rows of x) is needed
+    const bool use_vx = has_vx;                         // Dv (rows of vx) is needed
+    const bool any_op = use_x || use_vx;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 2); }
+        mbar_init(bar_zfull, NLW * 32);
+        mbar_init(bar_zfree, 1);
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW * 32); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // zero what is never written later: the raw rows of padded radial components / absent directions, and the
+    // Zbar slab rows of padded radial components (they meet zeros of phi, but must stay finite)
+    {
+        const int words = (int)(stage_bytes / 4), x_words = 2 * NOP * a.x_cap / 4;
+        for (int i = tid; i < NS * words; i += TT) {
+            const int st = i / words, w = i - st * words;
+            if (w >= x_words) reinterpret_cast<uint32_t*>(sRing + (size_t)st * stage_bytes)[w] = 0u;
+        }
+        for (int i = tid; i < 2 * a.z_cap / 4; i += TT) reinterpret_cast<uint32_t*>(sZ)[i] = 0u;
+    }
+    for (int i = tid; i < a.n_units; i += TT) {
+        const TUnit U = a.units[i];
+        const TBlk B = a.blks[U.blk];
+        UInfo u;
+        u.npad = (uint32_t)U.pad[0];
+        // D = F32, A = B = BF16, both K-major, M = 128, N = npad
+        u.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((u.npad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        u.z_off = (uint32_t)U.a_off; u.z_kb = (uint32_t)U.slab_stride;
+        u.x_off = (uint32_t)B.b_off; u.x_kb = (uint32_t)B.atom_stride;
+        u.ksteps = (uint32_t)(B.c_src >> 4); u.nmt = (uint32_t)((B.d_src * TB + 127) / 128);
+        sU[i] = u;
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp >= NCW && warp < NCW + NLW) {
+        // =========================== loader warps ===========================
+        const int lt = (warp - NCW) * 32 + lane;
+        uint32_t it = 0, zi = 0;
+        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+            const int64_t node = a.node0 + nl;
+            const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
+            for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
+                const int64_t g1 = min(seg1, g0 + EG);
+                for (int si = 0; si < a.nsets; ++si, ++zi) {
+                    const TSet S = a.sets[si];
+                    // ---- Zbar slabs of the set (once the previous set's MMAs have read theirs)
+                    if (zi > 0) mbar_wait(bar_zfree, (zi - 1) & 1, a.status);
+                    for (int ui = 0; ui < S.nunit; ++ui) {
+                        const TUnit U = a.units[S.unit_begin + ui];
+                        const TBlk B = a.blks[U.blk];
+                        const int cpr = B.c_src >> 3;
+                        const int n_it = U.ncomp * a.K * cpr;
+                        for (int i = lt; i < n_it; i += NLW * 32) {
+                            const int rowi = i / cpr, j = i - rowi * cpr;
+                            const int cl = rowi / a.K, q = rowi - cl * a.K;
+                            const SComp cp = a.comps[U.comp_begin + cl];
+                            const int64_t g = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * (int64_t)a.zb_ld[cp.group] +
+                                              cp.koff + (int64_t)q * B.c_src + 8 * j;
+                            const int r = cl * KP + q, u = 8 * j;
+                            const uint32_t d = smem_u32(sZ) + (uint32_t)(U.a_off + (u >> 6) * U.slab_stride + r * 128 +
+                                                                        ((((u & 63) >> 3) ^ (r & 7)) << 4));
+                            cp_async16_zfill(d, a.zqh + g, 16);
+                            cp_async16_zfill(d + (uint32_t)a.z_cap, a.zql + g, 16);
+                        }
+                    }
+                    cp_async_arrive(bar_zfull);
+                    // ---- the batches of the group
+                    for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
+                        const int nb = (int)min((int64_t)TB, g1 - b0);
+                        int64_t eid = 0; int32_t sn = 0;
+                        if (lane < nb) { eid = b0 + lane; sn = a.col[eid]; }
+                        const int st = (int)(it % NS);
+                        if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
+                        const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                        const uint32_t raw_u = stage_u + (uint32_t)(2 * NOP * a.x_cap);
+                        {
+                            const bool v16 = (a.K & 3) == 0;
+                            const int per = v16 ? a.K / 4 : a.K;
+                            const int n_it = TB * per;
+                            for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
+                                const int i = i0 + lt;
+                                const int e = min(i / per, TB - 1), j = i - (i / per) * per;
+                                const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
+                                if (i < n_it) {
+                                    const uint32_t ok = e < nb ? 1u : 0u;
+                                    if (v16) {
+                                        cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
+                                        if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(TB * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
+                                    } else {
+                                        cp_async4_zfill(raw_u + (uint32_t)(e * KP + j) * 4, a.phi + ee * a.K + j, ok * 4);
+                                        if (has_vphi) cp_async4_zfill(raw_u + (uint32_t)(TB * KP + e * KP + j) * 4, a.vphi + ee * a.K + j, ok * 4);
+                                    }
+                                }
+                            }
+                        }
+                        {
+                            const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
+                            const int n_it = TB * a.dsh;
+                            for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
+                                const int i = i0 + lt;
+                                const int e = min(i / a.dsh, TB - 1), b = i - (i / a.dsh) * a.dsh;
+                                const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
+                                if (i < n_it) {
+                                    const uint32_t ok = e < nb ? 4u : 0u;
+                                    cp_async4_zfill(y_u + (uint32_t)(e * YS + b) * 4, a.Y + ee * a.dsh + b, ok);
+                                    if (has_vY) cp_async4_zfill(y_u + (uint32_t)(TB * YS + e * YS + b) * 4, a.vY + ee * a.dsh + b, ok);
+                                }
+                            }
+                        }
+                        // sender rows: rows (s, e) of 128 bytes per 64 multiplicities, 128-byte swizzle
+                        for (int bi = 0; bi < S.nblk; ++bi) {
+                            const TBlk B = a.blks[S.blk_begin + bi];
+                            const int cpr = B.c_src >> 3;
+                            const int npair = TB * cpr;
+                            for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
+                                const int pr = p0 + lt;
+                                const int e = min(pr / cpr, TB - 1), j = pr - (pr / cpr) * cpr;
+                                const int32_t sne = __shfl_sync(0xffffffffu, sn, e);
+                                if (pr < npair) {
+                                    const uint32_t ok = e < nb ? 16u : 0u;
+                                    const int u = 8 * j;
+                                    uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
+                                    const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
+                                    const __nv_bfloat16* ph = a.sh + g;
+                                    const __nv_bfloat16* pl = a.sl + g;
+                                    const __nv_bfloat16* vh = use_vx ? a.vsh + g : nullptr;
+                                    const __nv_bfloat16* vl = use_vx ? a.vsl + g : nullptr;
+                                    for (int sdx = 0; sdx < B.d_src; ++sdx) {
+                                        if (use_x) {
+                                            cp_async16_zfill(d, ph, ok);
+                                            cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
+                                        }
+                                        if (use_vx) {
+                                            cp_async16_zfill(d + 2u * (uint32_t)a.x_cap, vh, ok);
+                                            cp_async16_zfill(d + 3u * (uint32_t)a.x_cap, vl, ok);
+                                            vh += B.c_src; vl += B.c_src;
+                                        }
+                                        d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                                    }
+                                }
+                            }
+                        }
+                        cp_async_arrive(bar_full + 8 * st);
+                    }
+                }
+            }
+        }
+    } else if (warp == NCW + NLW) {
+        // =========================== MMA warp ===========================
+        if (lane == 0) {
+            uint32_t it = 0, zi = 0, ai = 0;
+            const uint32_t sZ_u = smem_u32(sZ);
+            for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+                const int64_t node = a.node0 + nl;
+                const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
+                for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
+                    const int64_t g1 = min(seg1, g0 + EG);
+                    for (int si = 0; si < a.nsets; ++si, ++zi) {
+                        const TSet S = a.sets[si];
+                        mbar_wait(bar_zfull, zi & 1, a.status);
+                        for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
+                            const int st = (int)(it % NS);
+                            mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
+                            fence_async_smem();
+                            tc_fence_after();
+                            const uint32_t sX_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                            for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
+                                const UInfo U = sU[S.unit_begin + ui];
+                                const uint32_t buf = ai & 1;
+                                if (ai >= 2) mbar_wait(bar_accfree + 8 * buf, ((ai >> 1) & 1) ^ 1, a.status);
+                                tc_fence_after();
+#pragma unroll
+                                for (int op = 0; op < NOP; ++op) {
+                                    if (op == 0 ? !use_x : !use_vx) continue;
+                                    for (uint32_t mt = 0; mt < U.nmt; ++mt) {
+                                        const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + ((uint32_t)op * U.nmt + mt) * U.npad;
+                                        for (uint32_t ks = 0; ks < U.ksteps; ++ks) {
+                                            const uint32_t kb = ks >> 2, kk = ks & 3;
+                                            const uint32_t xh = sX_u + (uint32_t)(2 * op) * a.x_cap + U.x_off + kb * U.x_kb + mt * (128u * 128u) + 32u * kk;
+                                            const uint32_t xl = xh + a.x_cap;
+                                            const uint32_t zh = sZ_u + U.z_off + kb * U.z_kb + 32u * kk;
+                                            const uint32_t zl = zh + a.z_cap;
+                                            const uint64_t dXh = make_desc(xh, 16, 1024), dXl = make_desc(xl, 16, 1024);
+                                            const uint64_t dZh = make_desc(zh, 16, 1024), dZl = make_desc(zl, 16, 1024);
+                                            tc_mma_bf16(d_tmem, dXh, dZh, U.idesc, ks > 0 ? 1u : 0u);
+                                            tc_mma_bf16(d_tmem, dXl, dZh, U.idesc, 1u);
+                                            tc_mma_bf16(d_tmem, dXh, dZl, U.idesc, 1u);
+                                        }
+                                    }
+                                }
+                                tc_commit(bar_accfull + 8 * buf);
+                            }
+                            tc_commit(bar_free + 8 * st);
+                        }
+                        tc_commit(bar_zfree);
+                    }
+                }
+            }
+        }
+    } else {
+        // =========================== compute warps ===========================
+        uint32_t it = 0, ai = 0;
+        const int quarter = warp & 3, half = warp >> 2;
+        const int e = lane & 15;                     // the edge of this thread's accumulator rows
+        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+            const int64_t node = a.node0 + nl;
+            const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
+            for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
+                const int64_t g1 = min(seg1, g0 + EG);
+                for (int i = tid; i < EG * KP; i += NCW * 32) accPhi[i] = 0.f;
+                for (int i = tid; i < EG * a.dsh; i += NCW * 32) accY[i] = 0.f;
+                for (int si = 0; si < a.nsets; ++si) {
+                    const TSet S = a.sets[si];
+                    for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
+                        const int st = (int)(it % NS);
+                        const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
+                        mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
+                        const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.x_cap);
+                        const float* rawY = raw + NOP * TB * KP;
+                        compute_sync();     // the previous batch's reductions are done with the stages below
+                        for (int i = tid; i < TB * KP; i += NCW * 32) {
+                            const int ee = i / KP, q = i - ee * KP;
+                            sPhiT[q * PS + ee] = raw[i];
+                            if (DUAL) sVphiT[q * PS + ee] = raw[TB * KP + i];
+                        }
+                        for (int i = tid; i < TB * a.dsh; i += NCW * 32) {
+                            const int ee = i / a.dsh, b = i - ee * a.dsh;
+                            sYT[b * PS + ee] = rawY[ee * YS + b];
+                            if (DUAL) sVYT[b * PS + ee] = rawY[TB * YS + ee * YS + b];
+                        }
+                        compute_sync();
+                        // the raw rows of the stage are consumed: one of the two releases of the stage (the other
+                        // is the commit of the batch's MMAs, which read the sender rows)
+                        if (tid == 0) mbar_arrive(bar_free + 8 * st);
+                        // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
+                        for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
+                            const int j = i >> 1, h = i & 1;
+                            const TEnt en = a.ents[S.ent_begin + j];
+                            const int t0 = __ldg(a.tab_ptr + en.tab), t1 = __ldg(a.tab_ptr + en.tab + 1);
+                            float m[8], dm[8];
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) { m[x] = 0.f; dm[x] = 0.f; }
+                            for (int k = t0; k < t1; ++k) {
+                                const float cf = __ldg(a.tab_coef + k);
+                                const int b = en.sh_off + __ldg(a.tab_idx + k);
+                                float y[8];
+                                *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h);
+                                *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h + 4);
+#pragma unroll
+                                for (int x = 0; x < 8; ++x) m[x] = fmaf(cf, y[x], m[x]);
+                                if (DUAL) {
+                                    *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sVYT + b * PS + 8 * h);
+                                    *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sVYT + b * PS + 8 * h + 4);
+#pragma unroll
+                                    for (int x = 0; x < 8; ++x) dm[x] = fmaf(cf, y[x], dm[x]);
+                                }
+                            }
+                            *reinterpret_cast<float4*>(sM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(m);
+                            *reinterpret_cast<float4*>(sM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(m + 4);
+                            if (DUAL) {
+                                *reinterpret_cast<float4*>(sdM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(dm);
+                                *reinterpret_cast<float4*>(sdM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(dm + 4);
+                            }
+                        }
+                        compute_sync();
+                        // ---- epilogue of the batch: this thread owns accumulator rows (s, e) with e = lane & 15
+                        float ph[KP], vph[KP], pphi[KP];
+#pragma unroll
+                        for (int q = 0; q < KP; ++q) {
+                            ph[q] = sPhiT[q * PS + e];
+                            vph[q] = DUAL ? sVphiT[q * PS + e] : 0.f;
+                            pphi[q] = 0.f;
+                        }
+                        int ent_u = 0;                // first entry of the unit inside the set
+                        for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
+                            const TUnit U = a.units[S.unit_begin + ui];
+                            const TBlk B = a.blks[U.blk];
+                            const int npad = U.pad[0];
+                            const int nmt = (B.d_src * TB + 127) / 128;
+                            const uint32_t buf = ai & 1;
+                            mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
+                            tc_fence_after();
+                            const int chalf = (U.ncomp + 1) >> 1;
+                            const int c_lo = half * chalf, c_hi = min(U.ncomp, c_lo + chalf);
+                            for (int mt = 0; mt < nmt; ++mt) {
+                                const int row = mt * 128 + quarter * 32 + lane;
+                                const int s = row >> 4;
+                                const bool rv = s < B.d_src;
+                                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
+                                for (int cl = c_lo; cl < c_hi; ++cl) {
+                                    const int ent = ent_u + cl * B.d_src + s;
+                                    const float mw = rv ? sM[ent * PS + e] : 0.f;
+                                    const float dmw = (DUAL && rv) ? sdM[ent * PS + e] : 0.f;
+                                    float gm = 0.f;
+#pragma unroll
+                                    for (int q8 = 0; q8 < KP; q8 += 8) {
+                                        float v[8], v2[8];
+                                        if (use_x) tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
+                                        if (DUAL && use_vx) tc_ld8(t0 + (uint32_t)((nmt + mt) * npad + cl * KP + q8), v2);
+                                        if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
+#pragma unroll
+                                        for (int x = 0; x < 8; ++x) {
+                                            if (!DUAL) {
+                                                gm = fmaf(ph[q8 + x], v[x], gm);
+                                                pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
+                                            } else {
+                                                if (has_vphi) gm = fmaf(vph[q8 + x], v[x], gm);
+                                                if (has_vY) pphi[q8 + x] = fmaf(dmw, v[x], pphi[q8 + x]);
+                                                if (use_vx) {
+                                                    gm = fmaf(ph[q8 + x], v2[x], gm);
+                                                    pphi[q8 + x] = fmaf(mw, v2[x], pphi[q8 + x]);
+                                                }
+                                            }
+                                        }
+                                        }
+                                    }
+                                    if (rv) sGM[ent * PS + e] = gm;
+                                }
+                            }
+                            tc_fence_before();
+                            mbar_arrive(bar_accfree + 8 * buf);
+                            ent_u += U.ncomp * B.d_src;
+                        }
+                        // lanes l and l+16 of a warp hold rows of the same edge
+#pragma unroll
+                        for (int q = 0; q < KP; ++q) {
+                            const float o = __shfl_xor_sync(0xffffffffu, pphi[q], 16);
+                            if (lane < 16) sPphi[(warp * 16 + lane) * KP + q] = pphi[q] + o;
+                        }
+                        compute_sync();
+                        // ---- fixed-order reductions into the group's accumulators
+                        for (int i = tid; i < TB * KP; i += NCW * 32) {
+                            const int ee = i / KP, q = i - ee * KP;
+                            float v = 0.f;
+#pragma unroll
+                            for (int j = 0; j < NCW; ++j) v += sPphi[(j * 16 + ee) * KP + q];
+                            accPhi[(bg + ee) * KP + q] += v;
+                        }
+                        for (int i = tid; i < 2 * a.dsh; i += NCW * 32) {
+                            const int b = i >> 1, h = i & 1;
+                            const int k0 = a.inv_ptr[si * (a.dsh + 1) + b], k1 = a.inv_ptr[si * (a.dsh + 1) + b + 1];
+                            float g[8];
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) g[x] = 0.f;
+                            for (int k = k0; k < k1; ++k) {
+                                const float cf = __ldg(a.inv_coef + k);
+                                const int ent = __ldg(a.inv_ent + k);
+                                float gm[8];
+                                *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + ent * PS + 8 * h);
+                                *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + ent * PS + 8 * h + 4);
+#pragma unroll
+                                for (int x = 0; x < 8; ++x) g[x] = fmaf(cf, gm[x], g[x]);
+                            }
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) accY[(bg + 8 * h + x) * a.dsh + b] += g[x];
+                        }
+                    }
+                }
+                compute_sync();
+                // ---- outputs of the group (edge id = position in the receiver-sorted order)
+                const int ng = (int)(g1 - g0);
+                if (a.phi_mode)
+                    for (int i = tid; i < ng * a.K; i += NCW * 32) {
+                        const int ee = i / a.K, q = i - ee * a.K;
+                        float* p = a.gphi + (g0 + ee) * a.K + q;
+                        *p = (a.phi_mode == 2 ? *p : 0.f) + accPhi[ee * KP + q];
+                    }
+                if (a.Y_mode)
+                    for (int i = tid; i < ng * a.dsh; i += NCW * 32) {
+                        float* p = a.gY + g0 * a.dsh + i;
+                        *p = (a.Y_mode == 2 ? *p : 0.f) + accY[i];
+                    }
+                compute_sync();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+    }
+}
+
+int smem_need(int KP, bool dual, int dsh, int x_cap, int z_cap, int max_ent, int n_units) {
+    const int nop = dual ? 2 : 1;
+    const int stage = 2 * nop * x_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
+    size_t meta = (size_t)nop * KP * PS + (size_t)nop * dsh * PS + (size_t)(nop + 1) * max_ent * PS + (size_t)NCW * 16 * KP +
+                  (size_t)EG * KP + (size_t)((EG * dsh + 1) & ~1);
+    return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + n_units * 32;
+}
+
+}  // namespace
+
+// Units and sets of the tensor-core edge pass (receiver direction) for the plain ([0]) and dual ([1]) pass.
+void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
+    const int KP = p->K <= 8 ? 8 : 16;
+    for (int dual = 0; dual < 2; ++dual) {
+        TcSets& T = dir.etc[dual];
+        T = TcSets{};
+        if (p->K > 16) continue;
+        bool ok = true;
+        for (const DPath& P : dir.paths)
+            if ((P.c_src & 15) || P.c_src > 128 || (P.src_off & 7)) ok = false;
+        if (!ok || (dir.C_src & 7) || dir.paths.empty()) continue;
+        const int nop = dual ? 2 : 1;
+        struct Blk { int so, c_src, d_src; std::vector<SComp> comps; };
+        std::vector<Blk> blocks;
+        for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+            const DGroup& G = dir.groups[gi];
+            for (int k = G.path_begin; k < G.path_end; ++k) {
+                const DPath& P = dir.paths[k];
+                auto it = std::find_if(blocks.begin(), blocks.end(), [&](const Blk& b) { return b.so == P.src_off; });
+                if (it == blocks.end()) { blocks.push_back(Blk{P.src_off, P.c_src, P.d_src, {}}); it = blocks.end() - 1; }
+                for (int o = 0; o < G.d_dst; ++o)
+                    it->comps.push_back(SComp{P.tabM + o, G.d_dst, P.sh_off, (int)gi, o, P.koff, G.d_dst, 0});
+            }
+        }
+        std::sort(blocks.begin(), blocks.end(), [](const Blk& x, const Blk& y) { return x.so < y.so; });
+        struct Cand { int blk, c0, nc; };
+        std::vector<Cand> cands;
+        const int comps_per_tile = 128 / KP;
+        for (size_t b = 0; b < blocks.size(); ++b) {
+            const int nc = (int)blocks[b].comps.size();
+            const int ntile = (nc + comps_per_tile - 1) / comps_per_tile;
+            const int per = (nc + ntile - 1) / ntile;
+            for (int c0 = 0; c0 < nc; c0 += per) cands.push_back(Cand{(int)b, c0, std::min(per, nc - c0)});
+        }
+        auto nkb = [&](int b) { return (blocks[b].c_src + 63) / 64; };
+        auto npad = [&](const Cand& c) { return (c.nc * KP + 15) & ~15; };
+        auto unit_z = [&](const Cand& c) { return npad(c) * 128 * nkb(c.blk); };
+        auto blk_x = [&](int b) { return blocks[b].d_src * 2048 * nkb(b); };
+        auto nmt = [&](int b) { return (blocks[b].d_src * TB + 127) / 128; };
+        auto unit_cols = [&](const Cand& c) { return nop * nmt(c.blk) * npad(c); };
+        // sets: at most `maxu` units each, the largest grouping that fits two CTAs per SM, else one CTA per SM
+        for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
+            const int attempt = trial / (int)cands.size();
+            const int maxu = (int)cands.size() - trial % (int)cands.size();
+            const int budget = (attempt == 0 ? 113 : 226) * 1024;
+            const int col_budget = attempt == 0 ? 128 : 256;
+            T = TcSets{};
+            bool fits = true;
+            size_t i = 0;
+            while (i < cands.size() && fits) {
+                int z_bytes = 0, x_bytes = 0, nent = 0;
+                std::vector<int> set_blks;
+                size_t j = i;
+                for (; j < cands.size() && (int)(j - i) < maxu; ++j) {
+                    const Cand& c = cands[j];
+                    const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
+                    const int z2 = z_bytes + unit_z(c), x2 = x_bytes + (new_blk ? blk_x(c.blk) : 0);
+                    const int e2 = nent + c.nc * blocks[c.blk].d_src;
+                    // a 128-row MMA tile may read past the rows of a block: whatever follows in shared memory (the next
+                    // copy, the next stage, the Zbar slabs) is at least 16 KiB, see the floor on z_cap below
+                    const int xcap = std::max(T.a_cap, (x2 + 1023) & ~1023), zcap = std::max(T.b_cap, std::max(8192, (z2 + 1023) & ~1023));
+                    const int need = smem_need(KP, dual, p->dim_sh, xcap, zcap, std::max(T.max_ent, e2), (int)cands.size());
+                    if (need > budget || unit_cols(c) > col_budget) break;
+                    z_bytes = z2; x_bytes = x2; nent = e2;
+                    if (new_blk) set_blks.push_back(c.blk);
+                }
+                if (j == i) { fits = false; break; }
+                TSet S{};
+                S.unit_begin = (int)T.units.size(); S.blk_begin = (int)T.blks.size(); S.ent_begin = (int)T.ents.size();
+                int z_off = 0, x_off = 0;
+                std::vector<int> local_blk;
+                for (size_t k = i; k < j; ++k) {
+                    const Cand& c = cands[k];
+                    const Blk& Bk = blocks[c.blk];
+                    int bi = -1;
+                    for (size_t m = 0; m < local_blk.size(); ++m) if (local_blk[m] == c.blk) bi = S.blk_begin + (int)m;
+                    if (bi < 0) {
+                        TBlk tb{};
+                        tb.src_off = Bk.so; tb.c_src = Bk.c_src; tb.d_src = Bk.d_src; tb.ncols = 0;
+                        tb.b_off = x_off; tb.slab_bytes = 2048; tb.atom_stride = Bk.d_src * 2048;
+                        x_off += blk_x(c.blk);
+                        bi = (int)T.blks.size();
+                        T.blks.push_back(tb);
+                        local_blk.push_back(c.blk);
+                    }
+                    TUnit U{};
+                    U.blk = bi; U.comp_begin = (int)T.comps.size(); U.ncomp = c.nc; U.a_off = z_off;
+                    U.slab_stride = npad(c) * 128; U.tmem_col = 0; U.pad[0] = npad(c);
+                    for (int cl = 0; cl < c.nc; ++cl) {
+                        const SComp& cp = Bk.comps[c.c0 + cl];
+                        T.comps.push_back(cp);
+                        for (int s = 0; s < Bk.d_src; ++s) T.ents.push_back(TEnt{cp.tab0 + s * cp.tstride, cp.sh_off, 0, 0});
+                    }
+                    z_off += unit_z(c);
+                    T.acc_cols = std::max(T.acc_cols, unit_cols(c));
+                    T.units.push_back(U);
+                }
+                S.nunit = (int)T.units.size() - S.unit_begin; S.nblk = (int)T.blks.size() - S.blk_begin;
+                S.nent = (int)T.ents.size() - S.ent_begin;
+                T.sets.push_back(S);
+                T.a_cap = std::max(T.a_cap, (x_off + 1023) & ~1023);                       // x_cap
+                T.b_cap = std::max(T.b_cap, std::max(8192, (z_off + 1023) & ~1023));       // z_cap (two copies >= 16 KiB)
+                T.max_ent = std::max(T.max_ent, S.nent);
+                i = j;
+            }
+            if (!fits) continue;
+            int tc = 32; while (tc < 2 * T.acc_cols) tc <<= 1;
+            T.tmem_cols = tc;
+            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size());
+            if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
+            T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
+            // inverse sparse tables per set: b -> (entry inside the set, coef)
+            const int dsh = p->dim_sh;
+            T.inv_ptr.clear(); T.inv_ent.clear(); T.inv_coef.clear();
+            for (const TSet& S : T.sets) {
+                for (int b = 0; b < dsh; ++b) {
+                    T.inv_ptr.push_back((int)T.inv_ent.size());
+                    for (int en = 0; en < S.nent; ++en) {
+                        const TEnt& E = T.ents[S.ent_begin + en];
+                        for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k)
+                            if (E.sh_off + p->tab_idx[k] == b) { T.inv_ent.push_back(en); T.inv_coef.push_back(p->tab_coef[k]); }
+                    }
+                }
+                T.inv_ptr.push_back((int)T.inv_ent.size());
+            }
+            T.ok = true;
+            if (getenv("SOBEK_DEBUG_TC")) fprintf(stderr, "[etc] dual=%d sets=%zu x_cap=%d z_cap=%d ent=%d tmem=%d smem=%d ctas=%d\n", dual, T.sets.size(), T.a_cap, T.b_cap, T.max_ent, T.tmem_cols, T.smem_bytes, T.ctas_per_sm);
+        }
+    }
+}
+
+cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
+                                int64_t n_nodes, const SplitSrc& ss, const float* Y, const float* vY, const float* phi,
+                                const float* vphi, int dual, const void* zqh, const void* zql, float* gphi, float* gY,
+                                int phi_mode, int Y_mode, int* status, cudaStream_t s) {
+    const TcSets& T = dir.etc[dual ? 1 : 0];
+    if (!T.ok || !ss.h || !ss.l) return cudaErrorInvalidValue;
+    if (n_nodes <= 0) return cudaSuccess;
+    EtArgs a{};
+    a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.ents = T.d_ents; a.comps = T.d_comps;
+    a.inv_ptr = T.d_inv_ptr; a.inv_ent = T.d_inv_ent; a.inv_coef = T.d_inv_coef;
+    a.zb_off = dir.d_zb_off; a.zb_ld = dir.d_nk_ld;
+    a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
+    a.row_ptr = ev.ptr; a.col = ev.col; a.node0 = node0; a.n_nodes = n_nodes;
+    a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
+    a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
+    a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
+    a.zqh = (const __nv_bfloat16*)zqh; a.zql = (const __nv_bfloat16*)zql;
+    a.gphi = gphi; a.gY = gY; a.phi_mode = phi_mode; a.Y_mode = Y_mode;
+    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
+    a.x_cap = T.a_cap; a.z_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols;
+    a.n_units = (int)T.units.size();
+    a.status = status;
+    const bool k8 = p->K <= 8;
+    void (*kern)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true> : k_edge_tc<8, false>)
+                                    : (dual ? k_edge_tc<16, true> : k_edge_tc<16, false>);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T.smem_bytes);
+    if (e != cudaSuccess) return e;
+    const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * T.ctas_per_sm);
+    KernelTimer kt(K_EDGE, s);
+    kern<<<grid, TT, T.smem_bytes, s>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace sobek

@@ -35,6 +35,8 @@ constexpr int TC_THREADS = 192;
 
 struct TcArgs {
     float* C;
+    __nv_bfloat16* Ch;          // when set, the result is written as bf16 (hi, lo) at the same indices instead of C
+    __nv_bfloat16* Cl;
     int64_t c_outer, c_inner;   // C(m,n) = C[(m/c_d)*c_outer + (m%c_d)*c_inner + n]
     int32_t c_d;
     int32_t accumulate;
@@ -165,12 +167,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
         for (int r = 0; r < 32; ++r) {
             const int64_t m = (int64_t)m0 + q * 32 + r;
             if (m >= g.M) break;
-            float* crow = g.C + blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+            const int64_t rbase = blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+            float* crow = g.C + rbase;
             for (int c = lane; c < g.BN; c += 32) {
                 const int64_t n = (int64_t)n0 + c;
                 if (n < g.N) {
                     const float v = num_kb > 0 ? park[r * (g.BN + 1) + c] : 0.f;
-                    crow[n] = g.accumulate ? crow[n] + v : v;
+                    if (g.Ch) {
+                        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                        g.Ch[rbase + n] = h;
+                        g.Cl[rbase + n] = __float2bfloat16_rn(v - __bfloat162float(h));
+                    } else {
+                        crow[n] = g.accumulate ? crow[n] + v : v;
+                    }
                 }
             }
         }
@@ -279,10 +288,10 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
-                           int64_t split_stride) {
+                           int64_t split_stride, void* Chi, void* Clo) {
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
     TcArgs g{};
-    g.C = C; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate;
+    g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate;
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
     g.splits = std::max(1, std::min<int>(splits, (int)((Kd + BK - 1) / BK))); g.split_stride = split_stride;
     int BN;

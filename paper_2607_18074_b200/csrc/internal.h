@@ -103,8 +103,9 @@ struct TBlk {
     int32_t src_off, c_src, d_src;
     int32_t ncols;         // accumulator columns = c_src rounded up to 16
     int32_t b_off;         // byte offset of the block's slab 0 inside one B copy
-    int32_t slab_bytes;    // bytes of one (s, 16 edges) slab = 2048 * ceil(c_src / 64)
-    int32_t pad[2];
+    int32_t slab_bytes;    // bytes between consecutive s slabs of the gathered rows
+    int32_t atom_stride;   // bytes between the 64-multiplicity column blocks of a slab
+    int32_t pad;
 };
 struct TSet {
     int32_t unit_begin, nunit, blk_begin, nblk, ent_begin, nent;
@@ -123,6 +124,10 @@ struct TcSets {
     TBlk* d_blks = nullptr;
     TEnt* d_ents = nullptr;
     SComp* d_comps = nullptr;
+    std::vector<int32_t> inv_ptr, inv_ent;   // edge pass: per set, b -> (entry, coef) terms
+    std::vector<float> inv_coef;
+    int32_t *d_inv_ptr = nullptr, *d_inv_ent = nullptr;
+    float* d_inv_coef = nullptr;
     int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
@@ -159,6 +164,7 @@ struct Direction {
     STask* d_stasks = nullptr;
     SComp* d_scomps = nullptr;
     TcSets tc[2];                     // tensor-core stream: [0] plain, [1] dual
+    TcSets etc[2];                    // tensor-core edge pass: [0] plain, [1] dual
     // receiver-owned edge pass: source-major tasks over all multiplicities
     std::vector<STask> etasks;
     std::vector<SComp> ecomps;
@@ -205,6 +211,7 @@ struct sobek_plan {
     float* d_tab_coef = nullptr;
     int device = -1;
     bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
+    bool use_tc_edge = true;     // edge pass on the tensor cores where the profile allows it
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -220,7 +227,7 @@ namespace sobek {
 // bytes reserved at the start of every workspace for the device status word
 constexpr size_t kHeaderBytes = 256;
 // budget for the bounded node-state buffer (floats of Z / V held at once)
-constexpr size_t kStateBudgetBytes = size_t(256) << 20;
+constexpr size_t kStateBudgetBytes = size_t(1024) << 20;
 constexpr int64_t kMinChunkNodes = 512;
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);
@@ -292,6 +299,12 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
                           int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,
                           const float* vY, const float* phi, const float* vphi, int dual, void* zh, void* zl,
                           int* status, cudaStream_t s);
+// --- edge_pass_tc.cu ------------------------------------------------------------------
+void build_tc_edge_sets(const sobek_plan* p, Direction& dir);
+cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
+                                int64_t n_nodes, const SplitSrc& ss, const float* Y, const float* vY, const float* phi,
+                                const float* vphi, int dual, const void* zqh, const void* zql, float* gphi, float* gY,
+                                int phi_mode, int Y_mode, int* status, cudaStream_t s);
 // --- stream_tc.cu ---------------------------------------------------------------------
 void build_tc_sets(const sobek_plan* p, Direction& dir);
 cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
@@ -359,7 +372,7 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
-                           int64_t split_stride = 0);
+                           int64_t split_stride = 0, void* Chi = nullptr, void* Clo = nullptr);
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer

@@ -451,6 +451,8 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     if (const char* e = getenv("SOBEK_TC_STREAM")) p->use_tc_stream = atoi(e) != 0;
     build_tc_sets(p, p->fwd);
     build_tc_sets(p, p->tr);
+    if (const char* e = getenv("SOBEK_TC_EDGE")) p->use_tc_edge = atoi(e) != 0;
+    build_tc_edge_sets(p, p->fwd);
     build_edge_tasks(p, p->fwd);
     build_fused_stages(p, p->fwd);
     build_fused_stages(p, p->tr);
@@ -484,8 +486,12 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         if (e == cudaSuccess) e = upload(d->fs_begin, &d->d_fs_begin);
         if (e == cudaSuccess) e = upload(d->fs_count, &d->d_fs_count);
         if (e == cudaSuccess) e = upload(d->fk_off, &d->d_fk_off);
-        for (TcSets& t : d->tc) {
+        for (TcSets* tp : {&d->tc[0], &d->tc[1], &d->etc[0], &d->etc[1]}) {
+            TcSets& t = *tp;
             if (!t.ok) continue;
+            if (e == cudaSuccess) e = upload(t.inv_ptr, &t.d_inv_ptr);
+            if (e == cudaSuccess) e = upload(t.inv_ent, &t.d_inv_ent);
+            if (e == cudaSuccess) e = upload(t.inv_coef, &t.d_inv_coef);
             if (e == cudaSuccess) e = upload(t.sets, &t.d_sets);
             if (e == cudaSuccess) e = upload(t.units, &t.d_units);
             if (e == cudaSuccess) e = upload(t.blks, &t.d_blks);
@@ -525,7 +531,9 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
         cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);
         cudaFree(d->d_stasks); cudaFree(d->d_scomps); cudaFree(d->d_etasks); cudaFree(d->d_ecomps); cudaFree(d->d_zb_off);
         cudaFree(d->d_fstages); cudaFree(d->d_fs_begin); cudaFree(d->d_fs_count); cudaFree(d->d_fk_off);
-        for (TcSets& t : d->tc) {
+        for (TcSets* tp : {&d->tc[0], &d->tc[1], &d->etc[0], &d->etc[1]}) {
+            TcSets& t = *tp;
+            cudaFree(t.d_inv_ptr); cudaFree(t.d_inv_ent); cudaFree(t.d_inv_coef);
             cudaFree(t.d_sets); cudaFree(t.d_units); cudaFree(t.d_blks); cudaFree(t.d_ents); cudaFree(t.d_comps);
         }
     }

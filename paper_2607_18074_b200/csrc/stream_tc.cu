@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     if (pr < npair) {
                         const uint32_t ok = e < nb ? 16u : 0u;
                         const int u = 8 * j;
-                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * 2048 + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
+                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
                         const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
                         const __nv_bfloat16* ph = a.sh + g;
                         const __nv_bfloat16* pl = a.sl + g;
@@ -632,7 +632,7 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
                     if (bi < 0) {
                         TBlk tb{};
                         tb.src_off = Bk.so; tb.c_src = Bk.c_src; tb.d_src = Bk.d_src; tb.ncols = ncols(c.blk);
-                        tb.b_off = b_off; tb.slab_bytes = 2048 * ((Bk.c_src + 63) / 64);
+                        tb.b_off = b_off; tb.slab_bytes = 2048 * ((Bk.c_src + 63) / 64); tb.atom_stride = 2048;
                         b_off += blk_b(c.blk);
                         S.b_items += Bk.d_src * TB * (Bk.c_src / 8);
                         bi = (int)T.blks.size();
