@@ -26,8 +26,6 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
-#include <cstdio>
-#include <cstdlib>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -49,16 +47,11 @@ struct EtArgs {
     const TSet* sets;
     const TUnit* units;
     const TBlk* blks;
-    const TEnt* ents;
-    const SComp* comps;
-    const int32_t* inv_ptr;     // per set: dsh+1 offsets into inv_ent / inv_coef (b -> terms (entry, coef))
-    const int32_t* inv_ent;
-    const float* inv_coef;
-    const int64_t* zb_off;
-    const int32_t* zb_ld;
-    const int32_t* tab_ptr;
-    const int32_t* tab_idx;
-    const float* tab_coef;
+    const EntS* ents;           // of the launch's set
+    const NzS* nz;
+    const CompS* comps;
+    const int32_t* inv_ptr;     // of the launch's set: dsh+1 offsets into inv (b -> terms (entry, coef))
+    const NzS* inv;             // terms: b field = entry inside the set
     const int64_t* row_ptr;
     const int32_t* col;
     int64_t node0, n_nodes;
@@ -75,13 +68,15 @@ struct EtArgs {
     float* gphi;
     float* gY;
     int32_t phi_mode, Y_mode;   // 0 skip, 1 overwrite, 2 accumulate
-    int32_t K, dsh, C_src, nsets;
-    int32_t x_cap, z_cap, max_ent, tmem_cols, acc_cols, n_units;
+    int32_t K, dsh, C_src, set;
+    int32_t x_cap, z_cap, max_ent, tmem_cols, acc_cols, max_nz, max_inv, max_units;
     int* status;
 };
 
-struct UInfo {     // what the MMA thread needs of a unit, kept in shared memory
-    uint32_t idesc, z_off, z_kb, x_off, x_kb, ksteps, nmt, npad;
+// Everything the roles look up per batch or row lives in shared memory (with most of the SM's L1 given to
+// the operand regions, table reads from global memory would mostly go to L2).
+struct UInfo {     // a unit of the launch's set
+    uint32_t idesc, z_off, z_kb, x_off, x_kb, ksteps, nmt, npad, ncomp, comp_begin, d_src, c_src;
 };
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -105,9 +100,10 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// per-stage raw area (floats): phi rows [TB][KP], (vphi), and Y written transposed [dsh][PS], (vY)
 __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh) {
     const int n = dual ? 2 : 1;
-    return n * TB * KP + n * TB * (dsh + 1);
+    return n * TB * KP + n * dsh * PS;
 }
 
 template <int KP, bool DUAL>
@@ -115,26 +111,27 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int NOP = DUAL ? 2 : 1;
-    const int YS = a.dsh + 1;
     const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023);
     const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.x_cap) + raw_bytes;
     uint8_t* sRing = smem;                                     // stages: X1h X1l (X2h X2l) raw
-    uint8_t* sZ = sRing + (size_t)NS * stage_bytes;            // Zbar slabs of the current set: hi, lo
+    uint8_t* sZ = sRing + (size_t)NS * stage_bytes;            // Zbar slabs of the set: hi, lo
     uint8_t* meta = sZ + (size_t)2 * a.z_cap;
-    float* sPhiT = reinterpret_cast<float*>(meta);             // [KP][PS]
-    float* sVphiT = sPhiT + KP * PS;
-    float* sYT = sVphiT + (DUAL ? KP * PS : 0);                // [dsh][PS]
-    float* sVYT = sYT + a.dsh * PS;
-    float* sM = sVYT + (DUAL ? a.dsh * PS : 0);                // [max_ent][PS]
-    float* sdM = sM + (size_t)a.max_ent * PS;
-    float* sGM = sdM + (DUAL ? (size_t)a.max_ent * PS : 0);    // [max_ent][PS]
+    float* sM0 = reinterpret_cast<float*>(meta);               // [2][max_ent][PS] coupling matrices, double buffered
+    float* sdM0 = sM0 + (size_t)2 * a.max_ent * PS;            // DUAL
+    float* sGM = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [max_ent][PS]
     float* sPphi = sGM + (size_t)a.max_ent * PS;               // [NCW*16][KP]: one row per (warp, edge)
     float* accPhi = sPphi + NCW * 16 * KP;                     // [EG][KP]
     float* accY = accPhi + EG * KP;                            // [EG][dsh]
     uint64_t* bars = reinterpret_cast<uint64_t*>(accY + ((EG * a.dsh + 1) & ~1));
     // bars: full[NS], free[NS], zfull, zfree, acc_full[2], acc_free[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
-    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);
+    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [max_units]
+    TBlk* sBlk = reinterpret_cast<TBlk*>(sU + a.max_units);            // [max_units]
+    CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.max_units);       // [128 / KP * max_units]
+    EntS* sEnt = reinterpret_cast<EntS*>(sComp + (128 / KP) * a.max_units);   // [max_ent]
+    NzS* sNz = reinterpret_cast<NzS*>(sEnt + a.max_ent);               // [max_nz]
+    NzS* sInv = sNz + a.max_nz;                                        // [max_inv]
+    int32_t* sInvPtr = reinterpret_cast<int32_t*>(sInv + a.max_inv);   // [dsh + 1]
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_zfull = bar0 + 16 * NS, bar_zfree = bar_zfull + 8,
                    bar_accfull = bar_zfull + 16, bar_accfree = bar_zfull + 32;
@@ -144,9 +141,11 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     const bool use_x = !DUAL || has_vY || has_vphi;     // D (rows of x) is needed
     const bool use_vx = has_vx;                         // Dv (rows of vx) is needed
     const bool any_op = use_x || use_vx;
+    const TSet S = a.sets[a.set];
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 2); }
+        // a stage is released by the commit of the batch's MMAs and by every compute thread (raw rows read)
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 1 + NCW * 32); }
         mbar_init(bar_zfull, NLW * 32);
         mbar_init(bar_zfree, 1);
         for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW * 32); }
@@ -162,8 +161,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         }
         for (int i = tid; i < 2 * a.z_cap / 4; i += TT) reinterpret_cast<uint32_t*>(sZ)[i] = 0u;
     }
-    for (int i = tid; i < a.n_units; i += TT) {
-        const TUnit U = a.units[i];
+    // tables of the set
+    for (int i = tid; i < S.nunit; i += TT) {
+        const TUnit U = a.units[S.unit_begin + i];
         const TBlk B = a.blks[U.blk];
         UInfo u;
         u.npad = (uint32_t)U.pad[0];
@@ -172,8 +172,20 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         u.z_off = (uint32_t)U.a_off; u.z_kb = (uint32_t)U.slab_stride;
         u.x_off = (uint32_t)B.b_off; u.x_kb = (uint32_t)B.atom_stride;
         u.ksteps = (uint32_t)(B.c_src >> 4); u.nmt = (uint32_t)((B.d_src * TB + 127) / 128);
+        u.ncomp = (uint32_t)U.ncomp; u.comp_begin = (uint32_t)(U.comp_begin - a.units[S.unit_begin].comp_begin);
+        u.d_src = (uint32_t)B.d_src; u.c_src = (uint32_t)B.c_src;
         sU[i] = u;
     }
+    for (int i = tid; i < S.nblk; i += TT) sBlk[i] = a.blks[S.blk_begin + i];
+    {
+        const int c0 = a.units[S.unit_begin].comp_begin;
+        const TUnit UL = a.units[S.unit_begin + S.nunit - 1];
+        for (int i = tid; i < UL.comp_begin + UL.ncomp - c0; i += TT) sComp[i] = a.comps[c0 + i];
+    }
+    for (int i = tid; i < S.nent; i += TT) sEnt[i] = a.ents[i];
+    for (int i = tid; i < S.pad; i += TT) sNz[i] = a.nz[i];
+    for (int i = tid; i <= a.dsh; i += TT) sInvPtr[i] = a.inv_ptr[i];
+    for (int i = tid; i < a.inv_ptr[a.dsh]; i += TT) sInv[i] = a.inv[i];
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)a.tmem_cols) : "memory");
@@ -192,110 +204,104 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
             const int64_t node = a.node0 + nl;
             const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
-            for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
-                const int64_t g1 = min(seg1, g0 + EG);
-                for (int si = 0; si < a.nsets; ++si, ++zi) {
-                    const TSet S = a.sets[si];
-                    // ---- Zbar slabs of the set (once the previous set's MMAs have read theirs)
-                    if (zi > 0) mbar_wait(bar_zfree, (zi - 1) & 1, a.status);
-                    for (int ui = 0; ui < S.nunit; ++ui) {
-                        const TUnit U = a.units[S.unit_begin + ui];
-                        const TBlk B = a.blks[U.blk];
-                        const int cpr = B.c_src >> 3;
-                        const int n_it = U.ncomp * a.K * cpr;
-                        for (int i = lt; i < n_it; i += NLW * 32) {
-                            const int rowi = i / cpr, j = i - rowi * cpr;
-                            const int cl = rowi / a.K, q = rowi - cl * a.K;
-                            const SComp cp = a.comps[U.comp_begin + cl];
-                            const int64_t g = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * (int64_t)a.zb_ld[cp.group] +
-                                              cp.koff + (int64_t)q * B.c_src + 8 * j;
-                            const int r = cl * KP + q, u = 8 * j;
-                            const uint32_t d = smem_u32(sZ) + (uint32_t)(U.a_off + (u >> 6) * U.slab_stride + r * 128 +
-                                                                        ((((u & 63) >> 3) ^ (r & 7)) << 4));
-                            cp_async16_zfill(d, a.zqh + g, 16);
-                            cp_async16_zfill(d + (uint32_t)a.z_cap, a.zql + g, 16);
-                        }
-                    }
-                    cp_async_arrive(bar_zfull);
-                    // ---- the batches of the group
-                    for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
-                        const int nb = (int)min((int64_t)TB, g1 - b0);
-                        int64_t eid = 0; int32_t sn = 0;
-                        if (lane < nb) { eid = b0 + lane; sn = a.col[eid]; }
-                        const int st = (int)(it % NS);
-                        if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
-                        const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
-                        const uint32_t raw_u = stage_u + (uint32_t)(2 * NOP * a.x_cap);
-                        {
-                            const bool v16 = (a.K & 3) == 0;
-                            const int per = v16 ? a.K / 4 : a.K;
-                            const int n_it = TB * per;
-                            for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
-                                const int i = i0 + lt;
-                                const int e = min(i / per, TB - 1), j = i - (i / per) * per;
-                                const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
-                                if (i < n_it) {
-                                    const uint32_t ok = e < nb ? 1u : 0u;
-                                    if (v16) {
-                                        cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
-                                        if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(TB * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
-                                    } else {
-                                        cp_async4_zfill(raw_u + (uint32_t)(e * KP + j) * 4, a.phi + ee * a.K + j, ok * 4);
-                                        if (has_vphi) cp_async4_zfill(raw_u + (uint32_t)(TB * KP + e * KP + j) * 4, a.vphi + ee * a.K + j, ok * 4);
-                                    }
-                                }
+            if (seg1 <= seg0) continue;
+            // ---- Zbar slabs of the receiver (once the previous receiver's MMAs have read theirs)
+            if (zi > 0) mbar_wait(bar_zfree, (zi - 1) & 1, a.status);
+            for (int ui = 0; ui < S.nunit; ++ui) {
+                const UInfo U = sU[ui];
+                const int cpr = (int)U.c_src >> 3;
+                const int n_it = (int)U.ncomp * a.K * cpr;
+                for (int i = lt; i < n_it; i += NLW * 32) {
+                    const int rowi = i / cpr, j = i - rowi * cpr;
+                    const int cl = rowi / a.K, q = rowi - cl * a.K;
+                    const CompS cp = sComp[U.comp_begin + cl];
+                    const int64_t g = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff +
+                                      (int64_t)q * U.c_src + 8 * j;
+                    const int r = cl * KP + q, u = 8 * j;
+                    const uint32_t d = smem_u32(sZ) + (uint32_t)(U.z_off + (u >> 6) * U.z_kb + r * 128 + ((((u & 63) >> 3) ^ (r & 7)) << 4));
+                    cp_async16_zfill(d, a.zqh + g, 16);
+                    cp_async16_zfill(d + (uint32_t)a.z_cap, a.zql + g, 16);
+                }
+            }
+            cp_async_arrive(bar_zfull);
+            ++zi;
+            // ---- the batches of the receiver
+            for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
+                const int nb = (int)min((int64_t)TB, seg1 - b0);
+                int64_t eid = 0; int32_t sn = 0;
+                if (lane < nb) { eid = b0 + lane; sn = a.col[eid]; }
+                const int st = (int)(it % NS);
+                if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
+                const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                const uint32_t raw_u = stage_u + (uint32_t)(2 * NOP * a.x_cap);
+                {
+                    const bool v16 = (a.K & 3) == 0;
+                    const int per = v16 ? a.K / 4 : a.K;
+                    const int n_it = TB * per;
+                    for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
+                        const int i = i0 + lt;
+                        const int e = min(i / per, TB - 1), j = i - (i / per) * per;
+                        const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
+                        if (i < n_it) {
+                            const uint32_t ok = e < nb ? 1u : 0u;
+                            if (v16) {
+                                cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
+                                if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(TB * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
+                            } else {
+                                cp_async4_zfill(raw_u + (uint32_t)(e * KP + j) * 4, a.phi + ee * a.K + j, ok * 4);
+                                if (has_vphi) cp_async4_zfill(raw_u + (uint32_t)(TB * KP + e * KP + j) * 4, a.vphi + ee * a.K + j, ok * 4);
                             }
                         }
-                        {
-                            const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
-                            const int n_it = TB * a.dsh;
-                            for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
-                                const int i = i0 + lt;
-                                const int e = min(i / a.dsh, TB - 1), b = i - (i / a.dsh) * a.dsh;
-                                const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
-                                if (i < n_it) {
-                                    const uint32_t ok = e < nb ? 4u : 0u;
-                                    cp_async4_zfill(y_u + (uint32_t)(e * YS + b) * 4, a.Y + ee * a.dsh + b, ok);
-                                    if (has_vY) cp_async4_zfill(y_u + (uint32_t)(TB * YS + e * YS + b) * 4, a.vY + ee * a.dsh + b, ok);
-                                }
-                            }
-                        }
-                        // sender rows: rows (s, e) of 128 bytes per 64 multiplicities, 128-byte swizzle
-                        for (int bi = 0; bi < S.nblk; ++bi) {
-                            const TBlk B = a.blks[S.blk_begin + bi];
-                            const int cpr = B.c_src >> 3;
-                            const int npair = TB * cpr;
-                            for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
-                                const int pr = p0 + lt;
-                                const int e = min(pr / cpr, TB - 1), j = pr - (pr / cpr) * cpr;
-                                const int32_t sne = __shfl_sync(0xffffffffu, sn, e);
-                                if (pr < npair) {
-                                    const uint32_t ok = e < nb ? 16u : 0u;
-                                    const int u = 8 * j;
-                                    uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
-                                    const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
-                                    const __nv_bfloat16* ph = a.sh + g;
-                                    const __nv_bfloat16* pl = a.sl + g;
-                                    const __nv_bfloat16* vh = use_vx ? a.vsh + g : nullptr;
-                                    const __nv_bfloat16* vl = use_vx ? a.vsl + g : nullptr;
-                                    for (int sdx = 0; sdx < B.d_src; ++sdx) {
-                                        if (use_x) {
-                                            cp_async16_zfill(d, ph, ok);
-                                            cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
-                                        }
-                                        if (use_vx) {
-                                            cp_async16_zfill(d + 2u * (uint32_t)a.x_cap, vh, ok);
-                                            cp_async16_zfill(d + 3u * (uint32_t)a.x_cap, vl, ok);
-                                            vh += B.c_src; vl += B.c_src;
-                                        }
-                                        d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
-                                    }
-                                }
-                            }
-                        }
-                        cp_async_arrive(bar_full + 8 * st);
                     }
                 }
+                {   // Y (and vY), transposed: raw[b][PS + e]
+                    const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
+                    const int n_it = TB * a.dsh;
+                    for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
+                        const int i = i0 + lt;
+                        const int e = min(i / a.dsh, TB - 1), b = i - (i / a.dsh) * a.dsh;
+                        const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
+                        if (i < n_it) {
+                            const uint32_t ok = e < nb ? 4u : 0u;
+                            cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
+                            if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
+                        }
+                    }
+                }
+                // sender rows: rows (s, e) of 128 bytes per 64 multiplicities, 128-byte swizzle
+                for (int bi = 0; bi < S.nblk; ++bi) {
+                    const TBlk B = sBlk[bi];
+                    const int cpr = B.c_src >> 3;
+                    const int npair = TB * cpr;
+                    for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
+                        const int pr = p0 + lt;
+                        const int e = min(pr / cpr, TB - 1), j = pr - (pr / cpr) * cpr;
+                        const int32_t sne = __shfl_sync(0xffffffffu, sn, e);
+                        if (pr < npair) {
+                            const uint32_t ok = e < nb ? 16u : 0u;
+                            const int u = 8 * j;
+                            uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
+                            const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
+                            const __nv_bfloat16* ph = a.sh + g;
+                            const __nv_bfloat16* pl = a.sl + g;
+                            const __nv_bfloat16* vh = use_vx ? a.vsh + g : nullptr;
+                            const __nv_bfloat16* vl = use_vx ? a.vsl + g : nullptr;
+                            for (int sdx = 0; sdx < B.d_src; ++sdx) {
+                                if (use_x) {
+                                    cp_async16_zfill(d, ph, ok);
+                                    cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
+                                }
+                                if (use_vx) {
+                                    cp_async16_zfill(d + 2u * (uint32_t)a.x_cap, vh, ok);
+                                    cp_async16_zfill(d + 3u * (uint32_t)a.x_cap, vl, ok);
+                                    vh += B.c_src; vl += B.c_src;
+                                }
+                                d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                            }
+                        }
+                    }
+                }
+                cp_async_arrive(bar_full + 8 * st);
             }
         }
     } else if (warp == NCW + NLW) {
@@ -306,48 +312,44 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
                 const int64_t node = a.node0 + nl;
                 const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
-                for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
-                    const int64_t g1 = min(seg1, g0 + EG);
-                    for (int si = 0; si < a.nsets; ++si, ++zi) {
-                        const TSet S = a.sets[si];
-                        mbar_wait(bar_zfull, zi & 1, a.status);
-                        for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
-                            const int st = (int)(it % NS);
-                            mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
-                            fence_async_smem();
-                            tc_fence_after();
-                            const uint32_t sX_u = smem_u32(sRing + (size_t)st * stage_bytes);
-                            for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
-                                const UInfo U = sU[S.unit_begin + ui];
-                                const uint32_t buf = ai & 1;
-                                if (ai >= 2) mbar_wait(bar_accfree + 8 * buf, ((ai >> 1) & 1) ^ 1, a.status);
-                                tc_fence_after();
+                if (seg1 <= seg0) continue;
+                mbar_wait(bar_zfull, zi & 1, a.status);
+                ++zi;
+                for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
+                    const int st = (int)(it % NS);
+                    mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
+                    fence_async_smem();
+                    tc_fence_after();
+                    const uint32_t sX_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                    for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
+                        const UInfo U = sU[ui];
+                        const uint32_t buf = ai & 1;
+                        if (ai >= 2) mbar_wait(bar_accfree + 8 * buf, ((ai >> 1) & 1) ^ 1, a.status);
+                        tc_fence_after();
 #pragma unroll
-                                for (int op = 0; op < NOP; ++op) {
-                                    if (op == 0 ? !use_x : !use_vx) continue;
-                                    for (uint32_t mt = 0; mt < U.nmt; ++mt) {
-                                        const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + ((uint32_t)op * U.nmt + mt) * U.npad;
-                                        for (uint32_t ks = 0; ks < U.ksteps; ++ks) {
-                                            const uint32_t kb = ks >> 2, kk = ks & 3;
-                                            const uint32_t xh = sX_u + (uint32_t)(2 * op) * a.x_cap + U.x_off + kb * U.x_kb + mt * (128u * 128u) + 32u * kk;
-                                            const uint32_t xl = xh + a.x_cap;
-                                            const uint32_t zh = sZ_u + U.z_off + kb * U.z_kb + 32u * kk;
-                                            const uint32_t zl = zh + a.z_cap;
-                                            const uint64_t dXh = make_desc(xh, 16, 1024), dXl = make_desc(xl, 16, 1024);
-                                            const uint64_t dZh = make_desc(zh, 16, 1024), dZl = make_desc(zl, 16, 1024);
-                                            tc_mma_bf16(d_tmem, dXh, dZh, U.idesc, ks > 0 ? 1u : 0u);
-                                            tc_mma_bf16(d_tmem, dXl, dZh, U.idesc, 1u);
-                                            tc_mma_bf16(d_tmem, dXh, dZl, U.idesc, 1u);
-                                        }
-                                    }
+                        for (int op = 0; op < NOP; ++op) {
+                            if (op == 0 ? !use_x : !use_vx) continue;
+                            for (uint32_t mt = 0; mt < U.nmt; ++mt) {
+                                const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + ((uint32_t)op * U.nmt + mt) * U.npad;
+                                for (uint32_t ks = 0; ks < U.ksteps; ++ks) {
+                                    const uint32_t kb = ks >> 2, kk = ks & 3;
+                                    const uint32_t xh = sX_u + (uint32_t)(2 * op) * a.x_cap + U.x_off + kb * U.x_kb + mt * (128u * 128u) + 32u * kk;
+                                    const uint32_t xl = xh + a.x_cap;
+                                    const uint32_t zh = sZ_u + U.z_off + kb * U.z_kb + 32u * kk;
+                                    const uint32_t zl = zh + a.z_cap;
+                                    const uint64_t dXh = make_desc(xh, 16, 1024), dXl = make_desc(xl, 16, 1024);
+                                    const uint64_t dZh = make_desc(zh, 16, 1024), dZl = make_desc(zl, 16, 1024);
+                                    tc_mma_bf16(d_tmem, dXh, dZh, U.idesc, ks > 0 ? 1u : 0u);
+                                    tc_mma_bf16(d_tmem, dXl, dZh, U.idesc, 1u);
+                                    tc_mma_bf16(d_tmem, dXh, dZl, U.idesc, 1u);
                                 }
-                                tc_commit(bar_accfull + 8 * buf);
                             }
-                            tc_commit(bar_free + 8 * st);
                         }
-                        tc_commit(bar_zfree);
+                        tc_commit(bar_accfull + 8 * buf);
                     }
+                    tc_commit(bar_free + 8 * st);
                 }
+                tc_commit(bar_zfree);
             }
         }
     } else {
@@ -360,97 +362,83 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
             for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
                 const int64_t g1 = min(seg1, g0 + EG);
+                compute_sync();     // the previous group's outputs have been written
                 for (int i = tid; i < EG * KP; i += NCW * 32) accPhi[i] = 0.f;
                 for (int i = tid; i < EG * a.dsh; i += NCW * 32) accY[i] = 0.f;
-                for (int si = 0; si < a.nsets; ++si) {
-                    const TSet S = a.sets[si];
-                    for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
-                        const int st = (int)(it % NS);
-                        const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
-                        mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
-                        const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.x_cap);
-                        const float* rawY = raw + NOP * TB * KP;
-                        compute_sync();     // the previous batch's reductions are done with the stages below
-                        for (int i = tid; i < TB * KP; i += NCW * 32) {
-                            const int ee = i / KP, q = i - ee * KP;
-                            sPhiT[q * PS + ee] = raw[i];
-                            if (DUAL) sVphiT[q * PS + ee] = raw[TB * KP + i];
-                        }
-                        for (int i = tid; i < TB * a.dsh; i += NCW * 32) {
-                            const int ee = i / a.dsh, b = i - ee * a.dsh;
-                            sYT[b * PS + ee] = rawY[ee * YS + b];
-                            if (DUAL) sVYT[b * PS + ee] = rawY[TB * YS + ee * YS + b];
-                        }
-                        compute_sync();
-                        // the raw rows of the stage are consumed: one of the two releases of the stage (the other
-                        // is the commit of the batch's MMAs, which read the sender rows)
-                        if (tid == 0) mbar_arrive(bar_free + 8 * st);
-                        // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
-                        for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
-                            const int j = i >> 1, h = i & 1;
-                            const TEnt en = a.ents[S.ent_begin + j];
-                            const int t0 = __ldg(a.tab_ptr + en.tab), t1 = __ldg(a.tab_ptr + en.tab + 1);
-                            float m[8], dm[8];
+                for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
+                    const int st = (int)(it % NS);
+                    const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
+                    mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
+                    const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.x_cap);
+                    const float* sYT = raw + NOP * TB * KP;
+                    const float* sVYT = sYT + a.dsh * PS;
+                    float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
+                    float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
+                    // ---- this thread's radial weights, then the coupling matrices: thread <-> (entry, 8 edges)
+                    float ph[KP], vph[KP], pphi[KP];
 #pragma unroll
-                            for (int x = 0; x < 8; ++x) { m[x] = 0.f; dm[x] = 0.f; }
-                            for (int k = t0; k < t1; ++k) {
-                                const float cf = __ldg(a.tab_coef + k);
-                                const int b = en.sh_off + __ldg(a.tab_idx + k);
-                                float y[8];
-                                *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h);
-                                *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h + 4);
+                    for (int q = 0; q < KP; ++q) {
+                        ph[q] = raw[e * KP + q];
+                        vph[q] = DUAL ? raw[TB * KP + e * KP + q] : 0.f;
+                        pphi[q] = 0.f;
+                    }
+                    for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
+                        const int j = i >> 1, h = i & 1;
+                        const EntS en = sEnt[j];
+                        float m[8], dm[8];
 #pragma unroll
-                                for (int x = 0; x < 8; ++x) m[x] = fmaf(cf, y[x], m[x]);
-                                if (DUAL) {
-                                    *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sVYT + b * PS + 8 * h);
-                                    *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sVYT + b * PS + 8 * h + 4);
+                        for (int x = 0; x < 8; ++x) { m[x] = 0.f; dm[x] = 0.f; }
+                        for (int k = en.nz_begin; k < en.nz_begin + en.nz_count; ++k) {
+                            const NzS t = sNz[k];
+                            float y[8];
+                            *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + t.b * PS + 8 * h);
+                            *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + t.b * PS + 8 * h + 4);
 #pragma unroll
-                                    for (int x = 0; x < 8; ++x) dm[x] = fmaf(cf, y[x], dm[x]);
-                                }
-                            }
-                            *reinterpret_cast<float4*>(sM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(m);
-                            *reinterpret_cast<float4*>(sM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(m + 4);
+                            for (int x = 0; x < 8; ++x) m[x] = fmaf(t.coef, y[x], m[x]);
                             if (DUAL) {
-                                *reinterpret_cast<float4*>(sdM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(dm);
-                                *reinterpret_cast<float4*>(sdM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(dm + 4);
+                                *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + 8 * h);
+                                *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + 8 * h + 4);
+#pragma unroll
+                                for (int x = 0; x < 8; ++x) dm[x] = fmaf(t.coef, y[x], dm[x]);
                             }
                         }
-                        compute_sync();
-                        // ---- epilogue of the batch: this thread owns accumulator rows (s, e) with e = lane & 15
-                        float ph[KP], vph[KP], pphi[KP];
-#pragma unroll
-                        for (int q = 0; q < KP; ++q) {
-                            ph[q] = sPhiT[q * PS + e];
-                            vph[q] = DUAL ? sVphiT[q * PS + e] : 0.f;
-                            pphi[q] = 0.f;
+                        *reinterpret_cast<float4*>(sM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(m);
+                        *reinterpret_cast<float4*>(sM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(m + 4);
+                        if (DUAL) {
+                            *reinterpret_cast<float4*>(sdM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(dm);
+                            *reinterpret_cast<float4*>(sdM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(dm + 4);
                         }
-                        int ent_u = 0;                // first entry of the unit inside the set
-                        for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
-                            const TUnit U = a.units[S.unit_begin + ui];
-                            const TBlk B = a.blks[U.blk];
-                            const int npad = U.pad[0];
-                            const int nmt = (B.d_src * TB + 127) / 128;
-                            const uint32_t buf = ai & 1;
-                            mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
-                            tc_fence_after();
-                            const int chalf = (U.ncomp + 1) >> 1;
-                            const int c_lo = half * chalf, c_hi = min(U.ncomp, c_lo + chalf);
-                            for (int mt = 0; mt < nmt; ++mt) {
-                                const int row = mt * 128 + quarter * 32 + lane;
-                                const int s = row >> 4;
-                                const bool rv = s < B.d_src;
-                                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
-                                for (int cl = c_lo; cl < c_hi; ++cl) {
-                                    const int ent = ent_u + cl * B.d_src + s;
-                                    const float mw = rv ? sM[ent * PS + e] : 0.f;
-                                    const float dmw = (DUAL && rv) ? sdM[ent * PS + e] : 0.f;
-                                    float gm = 0.f;
+                    }
+                    // the raw rows of the stage are consumed by this thread (the stage is released when all compute
+                    // threads have said so and the batch's MMAs, which read the sender rows, have retired)
+                    mbar_arrive(bar_free + 8 * st);
+                    compute_sync();     // coupling matrices complete; the previous batch's reductions are done
+                    // ---- epilogue of the batch: this thread owns accumulator rows (s, e) with e = lane & 15
+                    int ent_u = 0;                // first entry of the unit inside the set
+                    for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
+                        const UInfo U = sU[ui];
+                        const int npad = (int)U.npad, nmt = (int)U.nmt, d_src = (int)U.d_src;
+                        const uint32_t buf = ai & 1;
+                        mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
+                        tc_fence_after();
+                        const int chalf = ((int)U.ncomp + 1) >> 1;
+                        const int c_lo = half * chalf, c_hi = min((int)U.ncomp, c_lo + chalf);
+                        for (int mt = 0; mt < nmt; ++mt) {
+                            const int row = mt * 128 + quarter * 32 + lane;
+                            const int s = row >> 4;
+                            const bool rv = s < d_src;
+                            const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
+                            for (int cl = c_lo; cl < c_hi; ++cl) {
+                                const int ent = ent_u + cl * d_src + s;
+                                const float mw = rv ? sM[ent * PS + e] : 0.f;
+                                const float dmw = (DUAL && rv) ? sdM[ent * PS + e] : 0.f;
+                                float gm = 0.f;
 #pragma unroll
-                                    for (int q8 = 0; q8 < KP; q8 += 8) {
-                                        float v[8], v2[8];
-                                        if (use_x) tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
-                                        if (DUAL && use_vx) tc_ld8(t0 + (uint32_t)((nmt + mt) * npad + cl * KP + q8), v2);
-                                        if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
+                                for (int q8 = 0; q8 < KP; q8 += 8) {
+                                    float v[8], v2[8];
+                                    if (use_x) tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
+                                    if (DUAL && use_vx) tc_ld8(t0 + (uint32_t)((nmt + mt) * npad + cl * KP + q8), v2);
+                                    if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
 #pragma unroll
                                         for (int x = 0; x < 8; ++x) {
                                             if (!DUAL) {
@@ -465,48 +453,45 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                                                 }
                                             }
                                         }
-                                        }
                                     }
-                                    if (rv) sGM[ent * PS + e] = gm;
                                 }
+                                if (rv) sGM[ent * PS + e] = gm;
                             }
-                            tc_fence_before();
-                            mbar_arrive(bar_accfree + 8 * buf);
-                            ent_u += U.ncomp * B.d_src;
                         }
-                        // lanes l and l+16 of a warp hold rows of the same edge
+                        tc_fence_before();
+                        mbar_arrive(bar_accfree + 8 * buf);
+                        ent_u += (int)U.ncomp * d_src;
+                    }
+                    // lanes l and l+16 of a warp hold rows of the same edge
 #pragma unroll
-                        for (int q = 0; q < KP; ++q) {
-                            const float o = __shfl_xor_sync(0xffffffffu, pphi[q], 16);
-                            if (lane < 16) sPphi[(warp * 16 + lane) * KP + q] = pphi[q] + o;
+                    for (int q = 0; q < KP; ++q) {
+                        const float o = __shfl_xor_sync(0xffffffffu, pphi[q], 16);
+                        if (lane < 16) sPphi[(warp * 16 + lane) * KP + q] = pphi[q] + o;
+                    }
+                    compute_sync();
+                    // ---- fixed-order reductions into the group's accumulators
+                    for (int i = tid; i < TB * KP; i += NCW * 32) {
+                        const int ee = i / KP, q = i - ee * KP;
+                        float v = 0.f;
+#pragma unroll
+                        for (int j = 0; j < NCW; ++j) v += sPphi[(j * 16 + ee) * KP + q];
+                        accPhi[(bg + ee) * KP + q] += v;
+                    }
+                    for (int i = tid; i < 2 * a.dsh; i += NCW * 32) {
+                        const int b = i >> 1, h = i & 1;
+                        float g[8];
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) g[x] = 0.f;
+                        for (int k = sInvPtr[b]; k < sInvPtr[b + 1]; ++k) {
+                            const NzS t = sInv[k];
+                            float gm[8];
+                            *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + t.b * PS + 8 * h);
+                            *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + t.b * PS + 8 * h + 4);
+#pragma unroll
+                            for (int x = 0; x < 8; ++x) g[x] = fmaf(t.coef, gm[x], g[x]);
                         }
-                        compute_sync();
-                        // ---- fixed-order reductions into the group's accumulators
-                        for (int i = tid; i < TB * KP; i += NCW * 32) {
-                            const int ee = i / KP, q = i - ee * KP;
-                            float v = 0.f;
 #pragma unroll
-                            for (int j = 0; j < NCW; ++j) v += sPphi[(j * 16 + ee) * KP + q];
-                            accPhi[(bg + ee) * KP + q] += v;
-                        }
-                        for (int i = tid; i < 2 * a.dsh; i += NCW * 32) {
-                            const int b = i >> 1, h = i & 1;
-                            const int k0 = a.inv_ptr[si * (a.dsh + 1) + b], k1 = a.inv_ptr[si * (a.dsh + 1) + b + 1];
-                            float g[8];
-#pragma unroll
-                            for (int x = 0; x < 8; ++x) g[x] = 0.f;
-                            for (int k = k0; k < k1; ++k) {
-                                const float cf = __ldg(a.inv_coef + k);
-                                const int ent = __ldg(a.inv_ent + k);
-                                float gm[8];
-                                *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + ent * PS + 8 * h);
-                                *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + ent * PS + 8 * h + 4);
-#pragma unroll
-                                for (int x = 0; x < 8; ++x) g[x] = fmaf(cf, gm[x], g[x]);
-                            }
-#pragma unroll
-                            for (int x = 0; x < 8; ++x) accY[(bg + 8 * h + x) * a.dsh + b] += g[x];
-                        }
+                        for (int x = 0; x < 8; ++x) accY[(bg + 8 * h + x) * a.dsh + b] += g[x];
                     }
                 }
                 compute_sync();
@@ -523,7 +508,6 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                         float* p = a.gY + g0 * a.dsh + i;
                         *p = (a.Y_mode == 2 ? *p : 0.f) + accY[i];
                     }
-                compute_sync();
             }
         }
     }
@@ -536,12 +520,14 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     }
 }
 
-int smem_need(int KP, bool dual, int dsh, int x_cap, int z_cap, int max_ent, int n_units) {
+int smem_need(int KP, bool dual, int dsh, int x_cap, int z_cap, int max_ent, int max_units, int max_nz, int max_inv) {
     const int nop = dual ? 2 : 1;
     const int stage = 2 * nop * x_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
-    size_t meta = (size_t)nop * KP * PS + (size_t)nop * dsh * PS + (size_t)(nop + 1) * max_ent * PS + (size_t)NCW * 16 * KP +
-                  (size_t)EG * KP + (size_t)((EG * dsh + 1) & ~1);
-    return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + n_units * 32;
+    const size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)max_ent * PS + (size_t)NCW * 16 * KP + (size_t)EG * KP +
+                        (size_t)((EG * dsh + 1) & ~1);
+    const int tables = max_units * (int)(sizeof(UInfo) + sizeof(TBlk) + (128 / KP) * sizeof(CompS)) + max_ent * (int)sizeof(EntS) +
+                       (max_nz + max_inv) * (int)sizeof(NzS) + (dsh + 2) * 4;
+    return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
 }
 
 }  // namespace
@@ -586,6 +572,17 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         auto blk_x = [&](int b) { return blocks[b].d_src * 2048 * nkb(b); };
         auto nmt = [&](int b) { return (blocks[b].d_src * TB + 127) / 128; };
         auto unit_cols = [&](const Cand& c) { return nop * nmt(c.blk) * npad(c); };
+        auto cand_nz = [&](const Cand& c) {
+            int n = 0;
+            for (int cl = 0; cl < c.nc; ++cl) {
+                const SComp& cp = blocks[c.blk].comps[c.c0 + cl];
+                for (int sdx = 0; sdx < blocks[c.blk].d_src; ++sdx) {
+                    const int t = cp.tab0 + sdx * cp.tstride;
+                    n += p->tab_ptr[t + 1] - p->tab_ptr[t];
+                }
+            }
+            return n;
+        };
         // sets: at most `maxu` units each, the largest grouping that fits two CTAs per SM, else one CTA per SM
         for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
             const int attempt = trial / (int)cands.size();
@@ -595,21 +592,24 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
             T = TcSets{};
             bool fits = true;
             size_t i = 0;
+            int maxu_seen = 0;
             while (i < cands.size() && fits) {
-                int z_bytes = 0, x_bytes = 0, nent = 0;
+                int z_bytes = 0, x_bytes = 0, nent = 0, nnz = 0;
                 std::vector<int> set_blks;
                 size_t j = i;
                 for (; j < cands.size() && (int)(j - i) < maxu; ++j) {
                     const Cand& c = cands[j];
                     const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
                     const int z2 = z_bytes + unit_z(c), x2 = x_bytes + (new_blk ? blk_x(c.blk) : 0);
-                    const int e2 = nent + c.nc * blocks[c.blk].d_src;
+                    const int e2 = nent + c.nc * blocks[c.blk].d_src, n2 = nnz + cand_nz(c);
                     // a 128-row MMA tile may read past the rows of a block: whatever follows in shared memory (the next
                     // copy, the next stage, the Zbar slabs) is at least 16 KiB, see the floor on z_cap below
                     const int xcap = std::max(T.a_cap, (x2 + 1023) & ~1023), zcap = std::max(T.b_cap, std::max(8192, (z2 + 1023) & ~1023));
-                    const int need = smem_need(KP, dual, p->dim_sh, xcap, zcap, std::max(T.max_ent, e2), (int)cands.size());
+                    // (the inverse table of a set has as many terms as its forward table)
+                    const int need = smem_need(KP, dual, p->dim_sh, xcap, zcap, std::max(T.max_ent, e2), std::max(maxu_seen, (int)(j - i) + 1),
+                                               std::max(T.max_nz, n2), std::max(T.max_nz, n2));
                     if (need > budget || unit_cols(c) > col_budget) break;
-                    z_bytes = z2; x_bytes = x2; nent = e2;
+                    z_bytes = z2; x_bytes = x2; nent = e2; nnz = n2;
                     if (new_blk) set_blks.push_back(c.blk);
                 }
                 if (j == i) { fits = false; break; }
@@ -649,30 +649,44 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
                 T.a_cap = std::max(T.a_cap, (x_off + 1023) & ~1023);                       // x_cap
                 T.b_cap = std::max(T.b_cap, std::max(8192, (z_off + 1023) & ~1023));       // z_cap (two copies >= 16 KiB)
                 T.max_ent = std::max(T.max_ent, S.nent);
+                T.max_nz = std::max(T.max_nz, nnz);
+                maxu_seen = std::max(maxu_seen, S.nunit);
                 i = j;
             }
             if (!fits) continue;
             int tc = 32; while (tc < 2 * T.acc_cols) tc <<= 1;
             T.tmem_cols = tc;
-            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size());
+            T.max_units = maxu_seen;
+            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, T.max_units, T.max_nz, T.max_nz);
             if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
             T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
-            // inverse sparse tables per set: b -> (entry inside the set, coef)
+            // shared-memory images of the tables, per set: entries with their sparse terms, the inverse table
+            // b -> (entry inside the set, coef), and the components with their group layout resolved
             const int dsh = p->dim_sh;
-            T.inv_ptr.clear(); T.inv_ent.clear(); T.inv_coef.clear();
-            for (const TSet& S : T.sets) {
+            for (TSet& S : T.sets) {
+                S.b_items = (int)T.nz.size();
+                for (int j = 0; j < S.nent; ++j) {
+                    const TEnt& E = T.ents[S.ent_begin + j];
+                    EntS es{0, (int)T.nz.size() - S.b_items, p->tab_ptr[E.tab + 1] - p->tab_ptr[E.tab], 0};
+                    for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k) T.nz.push_back(NzS{E.sh_off + p->tab_idx[k], p->tab_coef[k]});
+                    T.ents_s.push_back(es);
+                }
+                S.pad = (int)T.nz.size() - S.b_items;
+                T.inv_base.push_back((int)T.inv.size());
+                const int base = (int)T.inv.size();
                 for (int b = 0; b < dsh; ++b) {
-                    T.inv_ptr.push_back((int)T.inv_ent.size());
+                    T.inv_ptr.push_back((int)T.inv.size() - base);
                     for (int en = 0; en < S.nent; ++en) {
                         const TEnt& E = T.ents[S.ent_begin + en];
                         for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k)
-                            if (E.sh_off + p->tab_idx[k] == b) { T.inv_ent.push_back(en); T.inv_coef.push_back(p->tab_coef[k]); }
+                            if (E.sh_off + p->tab_idx[k] == b) T.inv.push_back(NzS{en, p->tab_coef[k]});
                     }
                 }
-                T.inv_ptr.push_back((int)T.inv_ent.size());
+                T.inv_ptr.push_back((int)T.inv.size() - base);
             }
+            for (const SComp& cp : T.comps)
+                T.comps_s.push_back(CompS{dir.zb_off[cp.group], dir.nk_ld[cp.group], cp.d_dst, cp.o, cp.koff, {0, 0}});
             T.ok = true;
-            if (getenv("SOBEK_DEBUG_TC")) fprintf(stderr, "[etc] dual=%d sets=%zu x_cap=%d z_cap=%d ent=%d tmem=%d smem=%d ctas=%d\n", dual, T.sets.size(), T.a_cap, T.b_cap, T.max_ent, T.tmem_cols, T.smem_bytes, T.ctas_per_sm);
         }
     }
 }
@@ -685,19 +699,16 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     if (!T.ok || !ss.h || !ss.l) return cudaErrorInvalidValue;
     if (n_nodes <= 0) return cudaSuccess;
     EtArgs a{};
-    a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.ents = T.d_ents; a.comps = T.d_comps;
-    a.inv_ptr = T.d_inv_ptr; a.inv_ent = T.d_inv_ent; a.inv_coef = T.d_inv_coef;
-    a.zb_off = dir.d_zb_off; a.zb_ld = dir.d_nk_ld;
-    a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
+    a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.comps = T.d_comps_s;
     a.row_ptr = ev.ptr; a.col = ev.col; a.node0 = node0; a.n_nodes = n_nodes;
     a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zqh = (const __nv_bfloat16*)zqh; a.zql = (const __nv_bfloat16*)zql;
-    a.gphi = gphi; a.gY = gY; a.phi_mode = phi_mode; a.Y_mode = Y_mode;
-    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
+    a.gphi = gphi; a.gY = gY;
+    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
     a.x_cap = T.a_cap; a.z_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols;
-    a.n_units = (int)T.units.size();
+    a.max_nz = T.max_nz; a.max_inv = T.max_nz; a.max_units = T.max_units;
     a.status = status;
     const bool k8 = p->K <= 8;
     void (*kern)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true> : k_edge_tc<8, false>)
@@ -705,10 +716,21 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T.smem_bytes);
     if (e != cudaSuccess) return e;
     const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * T.ctas_per_sm);
-    KernelTimer kt(K_EDGE, s);
-    kern<<<grid, TT, T.smem_bytes, s>>>(a);
-    count_launch();
-    return cudaGetLastError();
+    // one launch per set of accumulator tiles: the first writes in the caller's mode, the others accumulate
+    for (size_t si = 0; si < T.sets.size(); ++si) {
+        const TSet& S = T.sets[si];
+        a.set = (int)si;
+        a.ents = T.d_ents_s + S.ent_begin; a.nz = T.d_nz + S.b_items;
+        a.inv_ptr = T.d_inv_ptr + si * (size_t)(p->dim_sh + 1); a.inv = T.d_inv + T.inv_base[si];
+        a.phi_mode = phi_mode ? (si == 0 ? phi_mode : 2) : 0;
+        a.Y_mode = Y_mode ? (si == 0 ? Y_mode : 2) : 0;
+        KernelTimer kt(K_EDGE, s);
+        kern<<<grid, TT, T.smem_bytes, s>>>(a);
+        count_launch();
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace sobek

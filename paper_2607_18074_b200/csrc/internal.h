@@ -112,6 +112,18 @@ struct TSet {
     int32_t b_items;       // float4 pieces of sender rows gathered per 16-edge batch
     int32_t pad;
 };
+struct EntS {          // a (unit, component, s) entry of a set, as the kernels keep it in shared memory
+    int32_t a_off, nz_begin, nz_count, pad;   // nz_begin is relative to the set's first term
+};
+struct NzS {           // one sparse CG term of an entry: Y index and coefficient
+    int32_t b;
+    float coef;
+};
+struct CompS {         // an output component with the layout of its destination group resolved
+    int64_t zoff;      // bf16 state offset per node of the group
+    int32_t ld, d_dst, o, koff;
+    int32_t pad[2];
+};
 struct TcSets {
     bool ok = false;       // the tensor-core stream supports this direction
     std::vector<TSet> sets;
@@ -124,10 +136,18 @@ struct TcSets {
     TBlk* d_blks = nullptr;
     TEnt* d_ents = nullptr;
     SComp* d_comps = nullptr;
-    std::vector<int32_t> inv_ptr, inv_ent;   // edge pass: per set, b -> (entry, coef) terms
-    std::vector<float> inv_coef;
-    int32_t *d_inv_ptr = nullptr, *d_inv_ent = nullptr;
-    float* d_inv_coef = nullptr;
+    std::vector<EntS> ents_s;                // per set (TSet::ent_begin); TSet::b_items / TSet::pad = first term / terms
+    std::vector<NzS> nz;
+    std::vector<CompS> comps_s;              // parallel to comps
+    EntS* d_ents_s = nullptr;
+    NzS* d_nz = nullptr;
+    CompS* d_comps_s = nullptr;
+    int32_t max_nz = 0;
+    std::vector<int32_t> inv_ptr, inv_base;  // edge pass: per set, dsh+1 relative offsets / first term of the set
+    std::vector<NzS> inv;                    //   b -> terms (entry inside the set, coef)
+    int32_t* d_inv_ptr = nullptr;
+    NzS* d_inv = nullptr;
+    int32_t max_units = 0;
     int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)

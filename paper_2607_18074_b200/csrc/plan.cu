@@ -489,9 +489,11 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         for (TcSets* tp : {&d->tc[0], &d->tc[1], &d->etc[0], &d->etc[1]}) {
             TcSets& t = *tp;
             if (!t.ok) continue;
+            if (e == cudaSuccess) e = upload(t.ents_s, &t.d_ents_s);
+            if (e == cudaSuccess) e = upload(t.nz, &t.d_nz);
+            if (e == cudaSuccess) e = upload(t.comps_s, &t.d_comps_s);
             if (e == cudaSuccess) e = upload(t.inv_ptr, &t.d_inv_ptr);
-            if (e == cudaSuccess) e = upload(t.inv_ent, &t.d_inv_ent);
-            if (e == cudaSuccess) e = upload(t.inv_coef, &t.d_inv_coef);
+            if (e == cudaSuccess) e = upload(t.inv, &t.d_inv);
             if (e == cudaSuccess) e = upload(t.sets, &t.d_sets);
             if (e == cudaSuccess) e = upload(t.units, &t.d_units);
             if (e == cudaSuccess) e = upload(t.blks, &t.d_blks);
@@ -533,7 +535,8 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
         cudaFree(d->d_fstages); cudaFree(d->d_fs_begin); cudaFree(d->d_fs_count); cudaFree(d->d_fk_off);
         for (TcSets* tp : {&d->tc[0], &d->tc[1], &d->etc[0], &d->etc[1]}) {
             TcSets& t = *tp;
-            cudaFree(t.d_inv_ptr); cudaFree(t.d_inv_ent); cudaFree(t.d_inv_coef);
+            cudaFree(t.d_inv_ptr); cudaFree(t.d_inv);
+            cudaFree(t.d_ents_s); cudaFree(t.d_nz); cudaFree(t.d_comps_s);
             cudaFree(t.d_sets); cudaFree(t.d_units); cudaFree(t.d_blks); cudaFree(t.d_ents); cudaFree(t.d_comps);
         }
     }

@@ -21,21 +21,32 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One poll of the barrier phase.  The suspend-time hint lets the hardware park the thread until the
+// phase completes (or the hint, in nanoseconds, runs out) instead of returning at once, so that waiting
+// warps do not take issue slots from the warps that do the work.
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
     return ok != 0;
 }
-// Bounded wait.  A healthy wait ends after a handful of polls; the limit only exists so that a
-// broken pipeline cannot spin for ever.  On give-up the status word is set and the caller goes on.
+// Bounded wait.  A healthy wait ends after a handful of polls; the limit (about two seconds of wall
+// time, checked every 64 polls) only exists so that a broken pipeline cannot wait for ever.  On give-up
+// the status word is set and the caller goes on.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
+    if (mbar_try(bar, parity)) return;
+    uint64_t t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try(bar, parity)) return;
-        if (it > 4096) __nanosleep(256);
+        if ((it & 63u) == 0) {
+            uint64_t t1;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            if (t1 - t0 > 2000000000ull) break;
+        }
     }
     atomicExch(status, (int)SOBEK_ERR_DEVICE_TIMEOUT);
 }

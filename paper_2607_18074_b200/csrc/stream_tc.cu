@@ -47,13 +47,9 @@ struct TcArgs {
     const TSet* sets;
     const TUnit* units;
     const TBlk* blks;
-    const TEnt* ents;
-    const SComp* comps;
-    const int64_t* zb_off;
-    const int32_t* zb_ld;
-    const int32_t* tab_ptr;
-    const int32_t* tab_idx;
-    const float* tab_coef;
+    const EntS* ents;      // per set (TSet::ent_begin)
+    const NzS* nz;         // per set (TSet::b_items = first term, TSet::pad = number of terms)
+    const CompS* comps;
     EdgeView ev;
     int64_t node0, n_nodes;
     const __nv_bfloat16* sh;    // bf16 hi / lo copies of the source features [N][C_src]
@@ -67,7 +63,7 @@ struct TcArgs {
     __nv_bfloat16* zh;
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
-    int32_t a_cap, b_cap, max_ent, tmem_cols, acc_cols, n_units;
+    int32_t a_cap, b_cap, max_ent, tmem_cols, acc_cols, n_units, n_blks, n_comps, max_nz;
     int* status;
 };
 
@@ -80,10 +76,11 @@ __device__ __forceinline__ int64_t owner_of(const int64_t* __restrict__ row_ptr,
     return lo;
 }
 
-struct UInfo {     // what the MMA thread needs of a unit, kept in shared memory
-    uint32_t idesc, tmem_col, a_off, slab_stride, b_off, slab_bytes, d_src, pad;
+// Everything the roles look up per item, batch or row lives in shared memory: with most of the SM's
+// L1 given to the operand regions, table reads from global memory would mostly go to L2.
+struct UInfo {     // a unit, as the MMA thread and the drain need it
+    uint32_t idesc, tmem_col, a_off, slab_stride, b_off, slab_bytes, d_src, comp_begin, ncomp, c_src, ncols, pad;
 };
-
 // shared-memory operand descriptor without swizzle (K-major core matrices of 8 rows x 16 bytes)
 __device__ __forceinline__ uint64_t make_desc_none(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
@@ -134,10 +131,10 @@ __device__ __forceinline__ void split8(const float* p, uint4& h, uint4& l) {
     split2(p[6], p[7], h.w, l.w);
 }
 
-// per-stage raw area (floats): phi [TB][KP], (vphi), Y [TB][YS], (vY)
+// per-stage raw area (floats): phi rows [TB][KP], (vphi), and Y written transposed [dsh][PS], (vY)
 __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh) {
     const int n = dual ? 2 : 1;
-    return n * TB * KP + n * TB * (dsh + 1);
+    return n * TB * KP + n * dsh * PS;
 }
 
 template <int KP, bool DUAL>
@@ -152,16 +149,18 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.b_cap + ((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023));
     uint8_t* sRing = sA + (size_t)2 * NOP * a.a_cap;
     uint8_t* meta = sRing + (size_t)NS * stage_bytes;
-    float* sPhiT = reinterpret_cast<float*>(meta);           // [KP][PS]
-    float* sVphiT = sPhiT + KP * PS;                         // DUAL
-    float* sYT = sVphiT + (DUAL ? KP * PS : 0);              // [dsh][PS]
-    float* sVYT = sYT + a.dsh * PS;                          // DUAL
-    float* sM = sVYT + (DUAL ? a.dsh * PS : 0);              // [max_ent][PS]
-    float* sdM = sM + (size_t)a.max_ent * PS;                // DUAL
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sdM + (DUAL ? (size_t)a.max_ent * PS : 0));
+    float* sM0 = reinterpret_cast<float*>(meta);             // [2][max_ent][PS]: coupling matrices, double buffered
+    float* sdM0 = sM0 + (size_t)2 * a.max_ent * PS;          // DUAL
+    float* sPhiT0 = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [2][NOP][KP][PS]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sPhiT0 + 2 * NOP * KP * PS);
     // bars: full[NS], freeS[NS], ready, afree, acc_full[2], acc_free[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
-    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);
+    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [n_units]
+    TSet* sSet = reinterpret_cast<TSet*>(sU + a.n_units);               // [nsets]
+    TBlk* sBlk = reinterpret_cast<TBlk*>(sSet + a.nsets);               // [n_blks]
+    CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.n_blks);           // [n_comps]
+    EntS* sEnt = reinterpret_cast<EntS*>(sComp + a.n_comps);            // [max_ent]  (current set)
+    NzS* sNz = reinterpret_cast<NzS*>(sEnt + a.max_ent);                // [max_nz]   (current set)
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_ready = bar0 + 16 * NS, bar_afree = bar_ready + 8,
                    bar_accfull = bar_ready + 16, bar_accfree = bar_ready + 32;
@@ -194,9 +193,14 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         // D = F32, A = B = BF16, A K-major, B MN-major, M = 128, N = ncols
         u.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(B.ncols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         u.tmem_col = (uint32_t)U.tmem_col; u.a_off = (uint32_t)U.a_off; u.slab_stride = (uint32_t)U.slab_stride;
-        u.b_off = (uint32_t)B.b_off; u.slab_bytes = (uint32_t)B.slab_bytes; u.d_src = (uint32_t)B.d_src; u.pad = 0;
+        u.b_off = (uint32_t)B.b_off; u.slab_bytes = (uint32_t)B.slab_bytes; u.d_src = (uint32_t)B.d_src;
+        u.comp_begin = (uint32_t)U.comp_begin; u.ncomp = (uint32_t)U.ncomp; u.c_src = (uint32_t)B.c_src;
+        u.ncols = (uint32_t)B.ncols; u.pad = 0;
         sU[i] = u;
     }
+    for (int i = tid; i < a.nsets; i += TT) sSet[i] = a.sets[i];
+    for (int i = tid; i < a.n_blks; i += TT) sBlk[i] = a.blks[i];
+    for (int i = tid; i < a.n_comps; i += TT) sComp[i] = a.comps[i];
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)a.tmem_cols) : "memory");
@@ -217,7 +221,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         int64_t p_item = blockIdx.x, p_seg0 = 0, p_seg1 = 0;     // prefetched item
         auto prefetch_item = [&]() {
             if (p_item < total) {
-                const int64_t node = a.node0 + p_item / a.nsets;
+                const int64_t node = a.node0 + p_item % a.n_nodes;
                 p_seg0 = a.ev.ptr[node];
                 p_seg1 = any_op ? a.ev.ptr[node + 1] : p_seg0;
             }
@@ -229,7 +233,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             while (first || c.b0 >= c.seg1) {
                 first = false;
                 if (p_item >= total) return false;
-                c.set = (int)(p_item % a.nsets); c.b0 = p_seg0; c.seg1 = p_seg1;
+                c.set = (int)(p_item / a.n_nodes); c.b0 = p_seg0; c.seg1 = p_seg1;
                 p_item += gridDim.x;
                 prefetch_item();
             }
@@ -252,7 +256,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             const bool have_n = next_batch(nxt, false);
             int64_t eid_n = 0; int32_t sn_n = 0;
             if (have_n) load_ids(nxt, eid_n, sn_n);
-            const TSet S = a.sets[cur.set];
+            const TSet S = sSet[cur.set];
             const int nb = (int)min((int64_t)TB, cur.seg1 - cur.b0);
             const int st = (int)(it % NS);
             if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
@@ -279,7 +283,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     }
                 }
             }
-            // Y (and vY) rows: raw[e][YS]
+            // Y (and vY), transposed: raw[b][PS + e]
             {
                 const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
                 const int n_it = TB * a.dsh;
@@ -289,15 +293,15 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
                     if (i < n_it) {
                         const uint32_t ok = e < nb ? 4u : 0u;
-                        cp_async4_zfill(y_u + (uint32_t)(e * YS + b) * 4, a.Y + ee * a.dsh + b, ok);
-                        if (has_vY) cp_async4_zfill(y_u + (uint32_t)(TB * YS + e * YS + b) * 4, a.vY + ee * a.dsh + b, ok);
+                        cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
+                        if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
                     }
                 }
             }
             // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy: a thread owns an
             // (edge, piece) pair of a block and walks its d_src rows with constant strides
             for (int bi = 0; bi < S.nblk; ++bi) {
-                const TBlk B = a.blks[S.blk_begin + bi];
+                const TBlk B = sBlk[S.blk_begin + bi];
                 const int cpr = B.c_src >> 3;                  // 16-byte pieces per row
                 const int npair = TB * cpr;
                 for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
@@ -337,8 +341,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         if (lane == 0) {
             uint32_t it = 0, mi = 0;
             for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-                const int64_t nl = item / a.nsets;
-                const TSet S = a.sets[(int)(item - nl * a.nsets)];
+                const int64_t nl = item % a.n_nodes;
+                const TSet S = sSet[(int)(item / a.n_nodes)];
                 const int64_t node = a.node0 + nl;
                 const int64_t seg0 = a.ev.ptr[node], seg1 = any_op ? a.ev.ptr[node + 1] : seg0;
                 if (seg1 <= seg0) continue;
@@ -382,11 +386,12 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     } else {
         // =========================== compute warps ===========================
         uint32_t it = 0, mi = 0;
+        int cur_set = -1;
         // the item whose accumulator is drained next (one behind the one being built)
         int64_t p_nl = -1; int p_set = 0; uint32_t p_mi = 0; bool p_wrote = false;
 
         auto drain = [&](int64_t nl, int set, uint32_t dmi, bool wrote) {
-            const TSet S = a.sets[set];
+            const TSet S = sSet[set];
             const uint32_t buf = dmi & 1;
             if (wrote) {
                 mbar_wait(bar_accfull + 8 * buf, (dmi >> 1) & 1, a.status);
@@ -394,31 +399,50 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
             const int quarter = warp & 3, half = warp >> 2;
             for (int ui = 0; ui < S.nunit; ++ui) {
-                const TUnit U = a.units[S.unit_begin + ui];
-                const TBlk B = a.blks[U.blk];
+                const UInfo U = sU[S.unit_begin + ui];
+                struct { int ncols, c_src; } B{(int)U.ncols, (int)U.c_src};
                 const int r = quarter * 32 + lane;
                 const int cl = r / KP, q = r - cl * KP;
-                const bool rv = cl < U.ncomp && q < a.K;
+                const bool rv = cl < (int)U.ncomp && q < a.K;
                 int64_t off = 0;
                 if (rv) {
-                    const SComp cp = a.comps[U.comp_begin + cl];
-                    off = a.n_nodes * a.zb_off[cp.group] + (nl * cp.d_dst + cp.o) * (int64_t)a.zb_ld[cp.group] + cp.koff +
-                          (int64_t)q * B.c_src;
+                    const CompS cp = sComp[U.comp_begin + cl];
+                    off = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff + (int64_t)q * B.c_src;
                 }
                 const int hc = B.ncols >> 1;       // columns per warp half (multiple of 8)
-                for (int cc = half * hc; cc < (half + 1) * hc; cc += 8) {
-                    float v[8];
-                    if (wrote) tc_ld8(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols +
-                                      (uint32_t)(U.tmem_col + cc), v);
-                    else {
+                const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols + U.tmem_col;
+                if ((hc & 15) == 0) {              // 16 columns per TMEM load: half as many load round trips
+                    for (int cc = half * hc; cc < (half + 1) * hc; cc += 16) {
+                        float v[16];
+                        if (wrote) tc_ld16(trow + (uint32_t)cc, v);
+                        else {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+                            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                        }
+#pragma unroll
+                        for (int g8 = 0; g8 < 16; g8 += 8) {
+                            if (rv && cc + g8 < B.c_src) {
+                                uint4 h, l;
+                                split8(v + g8, h, l);
+                                *reinterpret_cast<uint4*>(a.zh + off + cc + g8) = h;
+                                *reinterpret_cast<uint4*>(a.zl + off + cc + g8) = l;
+                            }
+                        }
                     }
-                    if (rv && cc < B.c_src) {
-                        uint4 h, l;
-                        split8(v, h, l);
-                        *reinterpret_cast<uint4*>(a.zh + off + cc) = h;
-                        *reinterpret_cast<uint4*>(a.zl + off + cc) = l;
+                } else {
+                    for (int cc = half * hc; cc < (half + 1) * hc; cc += 8) {
+                        float v[8];
+                        if (wrote) tc_ld8(trow + (uint32_t)cc, v);
+                        else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+                        }
+                        if (rv && cc < B.c_src) {
+                            uint4 h, l;
+                            split8(v, h, l);
+                            *reinterpret_cast<uint4*>(a.zh + off + cc) = h;
+                            *reinterpret_cast<uint4*>(a.zl + off + cc) = l;
+                        }
                     }
                 }
             }
@@ -429,40 +453,45 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         };
 
         for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-            const int64_t nl = item / a.nsets;
-            const int set = (int)(item - nl * a.nsets);
-            const TSet S = a.sets[set];
+            const int64_t nl = item % a.n_nodes;
+            const int set = (int)(item / a.n_nodes);
+            const TSet S = sSet[set];
             const int64_t node = a.node0 + nl;
             const int64_t seg0 = a.ev.ptr[node], seg1 = any_op ? a.ev.ptr[node + 1] : seg0;
+            if (set != cur_set && seg1 > seg0) {     // entry and sparse-term tables of the set
+                compute_sync();
+                for (int i = tid; i < S.nent; i += NCW * 32) sEnt[i] = a.ents[S.ent_begin + i];
+                for (int i = tid; i < S.pad; i += NCW * 32) sNz[i] = a.nz[S.b_items + i];
+                compute_sync();
+                cur_set = set;
+            }
             for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
                 const int st = (int)(it % NS);
                 mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
-                compute_sync();     // everyone is done with the transposed stages of the previous batch
                 const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.b_cap);
-                const float* rawY = raw + NOP * TB * KP;
-                // ---- transpose phi and Y: [e][.] -> [.][e]
+                const float* sYT = raw + NOP * TB * KP;
+                const float* sVYT = sYT + a.dsh * PS;
+                float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
+                float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
+                float* sPhiT = sPhiT0 + (size_t)(it & 1) * NOP * KP * PS;      // [KP][PS] (+ vphi)
+                float* sVphiT = sPhiT + KP * PS;
+                // ---- transpose phi: [e][q] -> [q][e]   (same double buffer and barrier as the coupling matrices)
                 for (int i = tid; i < TB * KP; i += NCW * 32) {
                     const int e = i / KP, q = i - e * KP;
                     sPhiT[q * PS + e] = raw[i];
                     if (DUAL) sVphiT[q * PS + e] = raw[TB * KP + i];
                 }
-                for (int i = tid; i < TB * a.dsh; i += NCW * 32) {
-                    const int e = i / a.dsh, b = i - e * a.dsh;
-                    sYT[b * PS + e] = rawY[e * YS + b];
-                    if (DUAL) sVYT[b * PS + e] = rawY[TB * YS + e * YS + b];
-                }
-                compute_sync();
                 // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
                 for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
                     const int j = i >> 1, h = i & 1;
-                    const TEnt en = a.ents[S.ent_begin + j];
-                    const int t0 = __ldg(a.tab_ptr + en.tab), t1 = __ldg(a.tab_ptr + en.tab + 1);
+                    const EntS en = sEnt[j];
                     float m[8], dm[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) { m[e] = 0.f; dm[e] = 0.f; }
-                    for (int k = t0; k < t1; ++k) {
-                        const float cf = __ldg(a.tab_coef + k);
-                        const int b = en.sh_off + __ldg(a.tab_idx + k);
+                    for (int k = en.nz_begin; k < en.nz_begin + en.nz_count; ++k) {
+                        const NzS t = sNz[k];
+                        const float cf = t.coef;
+                        const int b = t.b;
                         float y[8];
                         *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h);
                         *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + b * PS + 8 * h + 4);
@@ -488,7 +517,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 // ---- A slabs: thread <-> (entry, q), both 8-edge halves
                 for (int i = tid; i < S.nent * KP; i += NCW * 32) {
                     const int j = i / KP, q = i - j * KP;
-                    const int a_off = a.ents[S.ent_begin + j].a_off + (q >> 3) * 256 + (q & 7) * 16;
+                    const int a_off = sEnt[j].a_off + (q >> 3) * 256 + (q & 7) * 16;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         float mv[8], ph[8], p1[8];
@@ -546,12 +575,15 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
 }
 
 // shared bytes of the kernel for given region sizes
-int smem_need(int KP, bool dual, int dsh, int a_cap, int b_cap, int max_ent, int n_units) {
+int smem_need(int KP, bool dual, int dsh, int a_cap, int b_cap, int max_ent, int n_units, int n_sets, int n_comps, int max_nz) {
     const int nop = dual ? 2 : 1;
     const int stage = 2 * nop * b_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
-    size_t meta = (size_t)nop * KP * PS + (size_t)nop * dsh * PS + (size_t)nop * max_ent * PS;
+    size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)2 * nop * KP * PS;
     meta = (meta + 1) & ~size_t(1);
-    return 1024 + 2 * nop * a_cap + NS * stage + (int)(meta * 4) + (2 * NS + 8) * 8 + n_units * 32;
+    // tables: units (and at most as many blocks), sets, components, entries and sparse terms of one set
+    const int tables = n_units * (int)(sizeof(UInfo) + sizeof(TBlk)) + n_sets * (int)sizeof(TSet) + n_comps * (int)sizeof(CompS) +
+                       max_ent * (int)sizeof(EntS) + max_nz * (int)sizeof(NzS);
+    return 1024 + 2 * nop * a_cap + NS * stage + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
 }
 
 }  // namespace
@@ -595,6 +627,19 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
         auto blk_b = [&](int b) { return blocks[b].d_src * 2048 * ((blocks[b].c_src + 63) / 64); };
         auto ncols = [&](int b) { return (blocks[b].c_src + 15) & ~15; };
         auto cols32 = [&](int b) { return (ncols(b) + 31) & ~31; };
+        auto cand_nz = [&](const Cand& c) {
+            int n = 0;
+            for (int cl = 0; cl < c.nc; ++cl) {
+                const SComp& cp = blocks[c.blk].comps[c.c0 + cl];
+                for (int sdx = 0; sdx < blocks[c.blk].d_src; ++sdx) {
+                    const int t = cp.tab0 + sdx * cp.tstride;
+                    n += p->tab_ptr[t + 1] - p->tab_ptr[t];
+                }
+            }
+            return n;
+        };
+        int n_comps_total = 0;
+        for (const Blk& b : blocks) n_comps_total += (int)b.comps.size();
         // greedy packing under a shared-memory budget: first for two CTAs per SM, else for one
         for (int attempt = 0; attempt < 2 && !T.ok; ++attempt) {
             const int budget = (attempt == 0 ? 113 : 226) * 1024;
@@ -603,19 +648,20 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
             bool fits = true;
             size_t i = 0;
             while (i < cands.size() && fits) {
-                int a_bytes = 0, b_bytes = 0, cols = 0, nent = 0;
+                int a_bytes = 0, b_bytes = 0, cols = 0, nent = 0, nnz = 0;
                 std::vector<int> set_blks;
                 size_t j = i;
                 for (; j < cands.size(); ++j) {
                     const Cand& c = cands[j];
                     const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
                     const int a2 = a_bytes + unit_a(c), b2 = b_bytes + (new_blk ? blk_b(c.blk) : 0);
-                    const int c2 = cols + cols32(c.blk), e2 = nent + c.nc * blocks[c.blk].d_src;
+                    const int c2 = cols + cols32(c.blk), e2 = nent + c.nc * blocks[c.blk].d_src, n2 = nnz + cand_nz(c);
                     // the kernel sizes its regions by the maxima over all sets
                     const int acap = std::max(T.a_cap, (a2 + 4096 + 1023) & ~1023), bcap = std::max(T.b_cap, (b2 + 1023) & ~1023);
-                    const int need = smem_need(KP, dual, p->dim_sh, acap, bcap, std::max(T.max_ent, e2), (int)cands.size());
+                    const int need = smem_need(KP, dual, p->dim_sh, acap, bcap, std::max(T.max_ent, e2), (int)cands.size(), (int)cands.size(),
+                                               n_comps_total, std::max(T.max_nz, n2));
                     if (need > budget || c2 > col_budget) break;
-                    a_bytes = a2; b_bytes = b2; cols = c2; nent = e2;
+                    a_bytes = a2; b_bytes = b2; cols = c2; nent = e2; nnz = n2;
                     if (new_blk) set_blks.push_back(c.blk);
                 }
                 if (j == i) { fits = false; break; }
@@ -658,15 +704,29 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
                 T.a_cap = std::max(T.a_cap, (a_off + 4096 + 1023) & ~1023);
                 T.b_cap = std::max(T.b_cap, (b_off + 1023) & ~1023);
                 T.max_ent = std::max(T.max_ent, S.nent);
+                T.max_nz = std::max(T.max_nz, nnz);
                 T.acc_cols = std::max(T.acc_cols, col);
                 i = j;
             }
             if (!fits) continue;
             int tc = 32; while (tc < 2 * T.acc_cols) tc <<= 1;
             T.tmem_cols = tc;
-            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size());
+            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size(), (int)cands.size(), n_comps_total, T.max_nz);
             if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
             T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
+            // shared-memory images of the tables
+            for (TSet& S : T.sets) {
+                S.b_items = (int)T.nz.size();
+                for (int j = 0; j < S.nent; ++j) {
+                    const TEnt& E = T.ents[S.ent_begin + j];
+                    EntS es{E.a_off, (int)T.nz.size() - S.b_items, p->tab_ptr[E.tab + 1] - p->tab_ptr[E.tab], 0};
+                    for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k) T.nz.push_back(NzS{E.sh_off + p->tab_idx[k], p->tab_coef[k]});
+                    T.ents_s.push_back(es);
+                }
+                S.pad = (int)T.nz.size() - S.b_items;
+            }
+            for (const SComp& cp : T.comps)
+                T.comps_s.push_back(CompS{dir.zb_off[cp.group], dir.nk_ld[cp.group], cp.d_dst, cp.o, cp.koff, {0, 0}});
             T.ok = true;
         }
     }
@@ -679,16 +739,14 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     if (!T.ok || !ss.h || !ss.l) return cudaErrorInvalidValue;
     if (n_nodes <= 0) return cudaSuccess;
     TcArgs a{};
-    a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.ents = T.d_ents; a.comps = T.d_comps;
-    a.zb_off = dir.d_zb_off; a.zb_ld = dir.d_nk_ld;
-    a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
+    a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.ents = T.d_ents_s; a.nz = T.d_nz; a.comps = T.d_comps_s;
     a.ev = ev; a.node0 = node0; a.n_nodes = n_nodes;
     a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
-    a.a_cap = T.a_cap; a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols; a.n_units = (int)T.units.size();
+    a.a_cap = T.a_cap; a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols; a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
     a.status = status;
     const bool k8 = p->K <= 8;
     void (*kern)(const TcArgs) = k8 ? (dual ? k_stream_tc<8, true> : k_stream_tc<8, false>)
