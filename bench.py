@@ -227,7 +227,8 @@ def main():
     rp = torch.from_numpy(d.row_ptr.astype(np.int64)).to(dev)
     col = torch.from_numpy(d.col.astype(np.int32)).to(dev)
     sp, perm = sb.graph_prepare(rp, col)
-    g = sb.make_graph(rp, col, sp, perm)
+    recv = sb.graph_receivers(rp, perm)
+    g = sb.make_graph(rp, col, sp, perm, recv)
     in_bytes = torch.cuda.memory_allocated(dev) - base_alloc
     new = lambda *s: torch.empty(*s, dtype=torch.float32, device=dev)
     out = {"y": new(N, i.C_y), "gx": new(N, i.C_x), "gY": new(E, i.dim_sh), "gphi": new(E, i.K),

@@ -128,6 +128,8 @@ typedef struct {
     const int32_t* col;      /* [E]   sender of each edge                                   */
     const int64_t* src_ptr;  /* [N+1] sender-sorted view; may be NULL if gx/hx not wanted   */
     const int32_t* src_perm; /* [E]   edge ids grouped by sender, increasing inside a group */
+    const int32_t* src_recv; /* [E]   optional: receiver of edge src_perm[p] at position p (see
+                                      sobek_graph_receivers); NULL = looked up in row_ptr when needed */
 } sobek_graph;
 
 /*
@@ -143,9 +145,19 @@ int sobek_graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int3
                         void* stream);
 
 /*
+ * sobek_graph_receivers -- fills src_recv[p] = receiver of edge src_perm[p], the column array of the
+ * sender-sorted view (it makes that view a plain CSR, so that the source-owned traversal reads its
+ * neighbour ids instead of searching row_ptr for them).  Integer work, unique result.  Only enqueues.
+ */
+int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* src_perm,
+                          int32_t* src_recv, void* stream);
+
+/*
  * Workspace needed by one call of the given order (0 = fwd, 1 = bwd, 2 = dbwd).  It holds
- * re-laid-out copies of R, the bounded receiver/sender state of one node chunk and a
- * status word.  It depends on the plan and on min(N, chunk size) only -- never on E.
+ * re-laid-out copies of R, the bounded receiver/sender state of one node chunk (at most 1 GiB,
+ * whatever the graph), a status word and, for the tensor-core edge kernels, bf16 (hi, lo)
+ * copies of the node features they gather from (4 bytes per feature of x, and of gy / vx for
+ * orders 1 / 2).  It depends on the plan and on N only -- never on E.
  * The pointer passed as `ws` must be 256-byte aligned.
  */
 size_t sobek_workspace_bytes(const sobek_plan* plan, int64_t N, int64_t E, int order);

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsobek.so")
 
 EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
-    "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_workspace_bytes", "sobek_conv_fwd",
+    "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_graph_receivers", "sobek_workspace_bytes", "sobek_conv_fwd",
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static",
@@ -49,7 +49,7 @@ class PathInfo(Structure):
 
 class Graph(Structure):
     _fields_ = [("N", c_int64), ("E", c_int64), ("row_ptr", c_void_p), ("col", c_void_p),
-                ("src_ptr", c_void_p), ("src_perm", c_void_p)]
+                ("src_ptr", c_void_p), ("src_perm", c_void_p), ("src_recv", c_void_p)]
 
 
 _lib = None
@@ -73,6 +73,7 @@ def lib():
         L.sobek_graph_prepare_bytes.argtypes = [c_int64, c_int64]
         L.sobek_graph_prepare_bytes.restype = c_size_t
         L.sobek_graph_prepare.argtypes = [c_int64, c_int64] + [c_void_p] * 5 + [c_size_t, c_void_p]
+        L.sobek_graph_receivers.argtypes = [c_int64, c_int64] + [c_void_p] * 4
         L.sobek_workspace_bytes.argtypes = [c_void_p, c_int64, c_int64, c_int]
         L.sobek_workspace_bytes.restype = c_size_t
         L.sobek_conv_fwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6 + [c_size_t, c_void_p]
@@ -199,8 +200,19 @@ def graph_prepare(row_ptr, col):
     return src_ptr, src_perm
 
 
-def make_graph(row_ptr, col, src_ptr=None, src_perm=None) -> Graph:
-    return Graph(row_ptr.numel() - 1, col.numel(), _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm))
+def graph_receivers(row_ptr, src_perm):
+    """src_recv int32[E]: the receiver of edge src_perm[p] at every position p of the sender-sorted view."""
+    import torch
+    N, E = row_ptr.numel() - 1, src_perm.numel()
+    src_recv = torch.empty(E, dtype=torch.int32, device=row_ptr.device)
+    _check(lib().sobek_graph_receivers(N, E, _ptr(row_ptr), _ptr(src_perm), _ptr(src_recv), _stream()),
+           "sobek_graph_receivers")
+    return src_recv
+
+
+def make_graph(row_ptr, col, src_ptr=None, src_perm=None, src_recv=None) -> Graph:
+    return Graph(row_ptr.numel() - 1, col.numel(), _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm),
+                 _ptr(src_recv))
 
 
 def workspace_bytes(plan: Plan, N: int, E: int, order: int) -> int:

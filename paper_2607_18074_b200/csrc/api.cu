@@ -117,7 +117,7 @@ EdgeView receiver_view(const sobek_graph* g) {
     return EdgeView{g->row_ptr, nullptr, g->col, g->row_ptr, g->N, g->E, 0};
 }
 EdgeView sender_view(const sobek_graph* g) {
-    return EdgeView{g->src_ptr, g->src_perm, g->col, g->row_ptr, g->N, g->E, 1};
+    return EdgeView{g->src_ptr, g->src_perm, g->col, g->row_ptr, g->N, g->E, 1, g->src_recv};
 }
 
 bool has_uncovered(const Direction& d) {
@@ -226,6 +226,11 @@ extern "C" int sobek_graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr,
                                    int64_t* src_ptr, int32_t* src_perm, void* ws, size_t ws_bytes,
                                    void* stream) {
     return graph_prepare(N, E, row_ptr, col, src_ptr, src_perm, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+extern "C" int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* src_perm,
+                                     int32_t* src_recv, void* stream) {
+    return graph_receivers(N, E, row_ptr, src_perm, src_recv, (cudaStream_t)stream);
 }
 
 extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,

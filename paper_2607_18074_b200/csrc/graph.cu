@@ -165,4 +165,31 @@ int graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* c
     return SOBEK_OK;
 }
 
+namespace {
+// src_recv[p] = receiver of edge src_perm[p]: the row of the receiver CSR that holds that edge id
+__global__ void k_receivers(int64_t N, int64_t E, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ src_perm,
+                            int32_t* __restrict__ src_recv) {
+    for (int64_t p = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; p < E; p += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = src_perm[p];
+        int64_t lo = 0, hi = N;   // row_ptr[lo] <= e < row_ptr[hi]
+        while (hi - lo > 1) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (row_ptr[mid] <= e) lo = mid; else hi = mid;
+        }
+        src_recv[p] = (int32_t)lo;
+    }
+}
+}  // namespace
+
+int graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* src_perm, int32_t* src_recv,
+                    cudaStream_t s) {
+    if (N < 0 || E < 0 || (E > 0 && (N == 0 || !row_ptr || !src_perm || !src_recv))) return SOBEK_ERR_INVALID_ARG;
+    if (E == 0) return SOBEK_OK;
+    const int grid = (int)std::min<int64_t>((E + 255) / 256, 148 * 16);
+    k_receivers<<<grid, 256, 0, s>>>(N, E, row_ptr, src_perm, src_recv);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return SOBEK_ERR_CUDA;
+    return SOBEK_OK;
+}
+
 }  // namespace sobek

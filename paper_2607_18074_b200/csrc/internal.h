@@ -399,6 +399,8 @@ constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its p
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);
+int graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* src_perm, int32_t* src_recv,
+                    cudaStream_t s);
 int graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* col, int64_t* src_ptr,
                   int32_t* src_perm, void* ws, size_t ws_bytes, cudaStream_t s);
 

@@ -34,7 +34,8 @@ class Case:
         self.x, self.Y, self.phi, self.R, self.gy = t(d.x), t(d.Y), t(d.phi), t(d.R), t(d.gy)
         self.vx, self.vY, self.vphi, self.vR = t(d.vx), t(d.vY), t(d.vphi), t(d.vR)
         self.src_ptr, self.src_perm = sb.graph_prepare(self.row_ptr, self.col)
-        self.graph = sb.make_graph(self.row_ptr, self.col, self.src_ptr, self.src_perm)
+        self.src_recv = sb.graph_receivers(self.row_ptr, self.src_perm)
+        self.graph = sb.make_graph(self.row_ptr, self.col, self.src_ptr, self.src_perm, self.src_recv)
         self.N, self.E = d.N, d.E
         self._ws = {}
 

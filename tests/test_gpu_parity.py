@@ -102,6 +102,9 @@ def test_graph_prepare_bit_exact(cases):
         sp, perm = oconv.sender_view(c.d.row_ptr, c.d.col)
         assert np.array_equal(c.src_ptr.cpu().numpy(), sp)
         assert np.array_equal(c.src_perm.cpu().numpy(), perm)
+        # receiver of every edge of the sender-sorted view
+        recv_of_edge = np.repeat(np.arange(c.d.N), np.diff(c.d.row_ptr))
+        assert np.array_equal(c.src_recv.cpu().numpy(), recv_of_edge[perm].astype(np.int32))
 
 
 def test_graph_prepare_large_and_hub():
