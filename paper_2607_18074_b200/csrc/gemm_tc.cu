@@ -50,7 +50,7 @@ struct TcArgs {
     int* status;
 };
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
           const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const TcArgs g) {
     extern __shared__ uint8_t smem_raw[];
@@ -164,6 +164,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
             for (int j = 0; j < 16; ++j) park[lane * (g.BN + 1) + c0 + j] = v[j];
         }
         __syncwarp();
+        if (g.Ch && (g.N & 7) == 0) {
+            // bf16 (hi, lo) output: a lane converts 8 consecutive columns and writes them as two 16-byte stores
+            for (int r = 0; r < 32; ++r) {
+                const int64_t m = (int64_t)m0 + q * 32 + r;
+                if (m >= g.M) break;
+                const int64_t rbase = blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+                for (int c8 = lane; c8 < g.BN / 8; c8 += 32) {
+                    const int64_t n = (int64_t)n0 + 8 * c8;
+                    if (n < g.N) {
+                        __align__(16) __nv_bfloat16 h[8], l[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float v = num_kb > 0 ? park[r * (g.BN + 1) + 8 * c8 + j] : 0.f;
+                            h[j] = __float2bfloat16_rn(v);
+                            l[j] = __float2bfloat16_rn(v - __bfloat162float(h[j]));
+                        }
+                        *reinterpret_cast<uint4*>(g.Ch + rbase + n) = *reinterpret_cast<const uint4*>(h);
+                        *reinterpret_cast<uint4*>(g.Cl + rbase + n) = *reinterpret_cast<const uint4*>(l);
+                    }
+                }
+            }
+        } else {
         for (int r = 0; r < 32; ++r) {
             const int64_t m = (int64_t)m0 + q * 32 + r;
             if (m >= g.M) break;
@@ -182,6 +204,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
                     }
                 }
             }
+        }
         }
     }
     tc_fence_before();
@@ -299,7 +322,9 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
     else BN = (int)std::min<int64_t>(256, (N + 15) / 16 * 16);
     g.BN = BN;
     const size_t stage = 2 * (size_t)BM * BK * 2 + 2 * (size_t)BN * BK * 2;
-    int stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
+    // two CTAs per SM where two stages of the ring fit twice (more loads in flight per SM), else one CTA with a deeper ring
+    int stages = (int)std::min<size_t>(4, (108 * 1024) / stage);
+    if (stages < 2) stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
     g.stages = std::max(stages, 2);
     int cols = 32;
     while (cols < BN) cols <<= 1;
