@@ -33,10 +33,11 @@ METRIC = "edges/s (one step = fwd + bwd + double-bwd)"
 FP32_FMA_LANES = 148 * 128            # SMs x FP32 lanes
 L2_FLUSH_BYTES = 512 << 20
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the edge-stream kernel,
-# from the ncu capture summarised in profiles/ncu_edge_stream_cfg2.md (average of the two kernel
-# classes of one pass).  Only known for the workload that was captured.
-NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 31.0e6, ("cfg2", "edge_pass"): 91.6e6}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from the ncu captures summarised
+# under profiles/ (average over the launches of the class in one step).  Only known for the workload
+# that was captured.
+NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 144.0e6, ("cfg2", "edge_pass"): 82.0e6,
+                     ("cfg2", "node_gemm"): 26.6e6}
 
 
 def measured_peaks():
@@ -348,20 +349,30 @@ def main():
     dom = max(classes, key=lambda k: classes[k][0])
     dom_ms, dom_launches = classes[dom]
     steps_timed = args.steps
-    if dom == "node_gemm":
-        fmas = 3 * (node_w["fwd"] + node_w["bwd"] + node_w["dbwd"]) * N * steps_timed   # three bf16 passes
-    else:
-        fmas = cls_w.get(dom, 0) * E * steps_timed
     alu_peak = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
-    achieved = 2.0 * fmas / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
-    roofline = {"kernel": dom, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                "frac": achieved / alu_peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
-                "peak_source": f"derived: 148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz "
-                               f"(HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_tflops']} TFLOP/s {peaks['source']})",
+    if dom == "node_gemm":
+        # the node contractions stream the bounded state once per pass (4 bytes per state element as bf16
+        # hi + lo, read or written): HBM-bound; passes per step: 8 over the receiver state, 3 over the sender state
+        info = plan.info
+        nbytes = 4.0 * (8 * info.state_floats_fwd + 3 * info.state_floats_bwd) * N * steps_timed
+        achieved = nbytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+                    "peak_source": f"HBM copy bandwidth, {peaks['source']}"}
+    else:
+        # the edge kernels: algorithmic multiply-adds of the method per edge against the FP32 pipes (the
+        # tensor-core kernels move the part that scales with the multiplicity off those pipes)
+        fmas = cls_w.get(dom, 0) * E * steps_timed
+        achieved = 2.0 * fmas / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
+        roofline = {"kernel": dom, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                    "frac": achieved / alu_peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+                    "peak_source": f"derived: 148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz "
+                                   f"(HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_tflops']} TFLOP/s {peaks['source']})"}
+    roofline.update({
                 "avg_launch_ms": dom_ms / max(dom_launches, 1), "launches": int(dom_launches),
                 "share_of_kernel_time": dom_ms / tot_cls,
                 "classes": {k: {"ms_per_step": v[0] / steps_timed, "launches_per_step": v[1] / steps_timed}
-                            for k, v in classes.items()}}
+                            for k, v in classes.items()}})
 
     res = {
         "metric": METRIC, "value": E_total / (step_ms * 1e-3), "unit": "edges/s", "n_gpus": world,

@@ -10,14 +10,17 @@
 // split-bf16 product a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo (fp32 accumulation in TMEM); the sender
 // rows are read from bf16 (hi, lo) copies of the source features made once per call.
 //
-// A CTA works through (receiver, set of accumulator tiles) items, edges in batches of 16, with three roles:
-//   loader warps  run ahead: edge / sender ids, then cp.async of the batch's phi and Y rows and of the
-//                 sender rows straight into the B slabs (16 edges x c_src, MN-major, 128-byte swizzle)
-//                 of a two-stage ring;
-//   compute warps transpose phi / Y, expand the coupling matrices M_e[s,comp] of the set from the sparse
-//                 CG table, build the A slabs (one per s: 128 rows x 16 edges, K-major, no swizzle, bf16
-//                 hi / lo), and - one item behind - drain the finished accumulator (tcgen05.ld), split
-//                 it into bf16 hi / lo and write the rows of the node GEMM's A operand;
+// A CTA works through (set of accumulator tiles, receiver) items in set-major order, edges in batches of 16,
+// with three roles:
+//   loader warps  run ahead (segment bounds and edge / sender ids are requested one step early): cp.async of
+//                 the batch's phi rows, of its Y rows (written transposed) and of the sender rows straight
+//                 into the B slabs (16 edges x c_src, MN-major, 128-byte swizzle) of a two-stage ring; the
+//                 copies signal the stage's mbarrier themselves when they land;
+//   compute warps expand the coupling matrices M_e[s,comp] of the set from the sparse CG table (kept in shared
+//                 memory, like every other table the kernel looks up), build the A slabs (one per s: 128 rows
+//                 x 16 edges, K-major, no swizzle, bf16 hi / lo), and - one item behind - drain the finished
+//                 accumulator (tcgen05.ld), split it into bf16 hi / lo and write the rows of the node GEMM's
+//                 A operand (contraction index k = koff + q*c_src + u, so a row of 16-byte pieces per thread);
 //   MMA warp      one thread issues the batch's MMAs into one of two TMEM accumulator buffers and commits
 //                 to the mbarriers that release the A region, the ring stage and the accumulator.
 // With DUAL the kernel produces the directional state of the double backward
@@ -641,7 +644,10 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
         int n_comps_total = 0;
         for (const Blk& b : blocks) n_comps_total += (int)b.comps.size();
         // greedy packing under a shared-memory budget: first for two CTAs per SM, else for one
-        for (int attempt = 0; attempt < 2 && !T.ok; ++attempt) {
+        // sets of at most `maxu` units: the largest grouping that fits two CTAs per SM, else one CTA per SM
+        for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
+            const int attempt = trial / (int)cands.size();
+            const int maxu = (int)cands.size() - trial % (int)cands.size();
             const int budget = (attempt == 0 ? 113 : 226) * 1024;
             const int col_budget = attempt == 0 ? 128 : 256;     // two accumulator buffers per CTA
             T = TcSets{};
@@ -651,7 +657,7 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
                 int a_bytes = 0, b_bytes = 0, cols = 0, nent = 0, nnz = 0;
                 std::vector<int> set_blks;
                 size_t j = i;
-                for (; j < cands.size(); ++j) {
+                for (; j < cands.size() && (int)(j - i) < maxu; ++j) {
                     const Cand& c = cands[j];
                     const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
                     const int a2 = a_bytes + unit_a(c), b2 = b_bytes + (new_blk ? blk_b(c.blk) : 0);

@@ -248,3 +248,33 @@ def test_fused_schedule(name, monkeypatch):
     assert rel_err(ggy.cpu().numpy(), ref[0]) <= BWD_TOL and rel_err(hx.cpu().numpy(), ref[1]) <= BWD_TOL
     for got, r, nm in zip(c.dbwd(), ref, ("ggy", "hx", "hY", "hphi", "hR")):
         assert rel_err(got, r) <= BWD_TOL, nm
+
+
+# ---------------------------------------------------------------------------------------
+# the FP32-pipe edge kernels (used where the tensor-core kernels do not apply), forced for whole plans
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["cfg1", "cfg2_N200", "cfg4_N150", "ragged"])
+def test_fp32_pipe_edge_kernels(name, monkeypatch):
+    """SOBEK_TC_STREAM=0 / SOBEK_TC_EDGE=0 at plan creation select the FP32-pipe stream and edge pass for
+    every traversal; all three orders must match the oracle to the same tolerances."""
+    monkeypatch.setenv("SOBEK_TC_STREAM", "0")
+    monkeypatch.setenv("SOBEK_TC_EDGE", "0")
+    c = Case(CASES[name])
+    monkeypatch.delenv("SOBEK_TC_STREAM")
+    monkeypatch.delenv("SOBEK_TC_EDGE")
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+    for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+    for got, ref, nm in zip(c.dbwd(), c.o_dbwd(), ("ggy", "hx", "hY", "hphi", "hR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+
+
+def test_sender_view_without_receiver_ids(cases):
+    """src_recv is optional: without it the transposed traversal looks the receivers up in row_ptr."""
+    import paper_2607_18074_b200 as sb
+    c = get(cases, "cfg2_N200")
+    g = sb.make_graph(c.row_ptr, c.col, c.src_ptr, c.src_perm)
+    import torch
+    gx = torch.full((c.N, c.plan.info.C_x), float("nan"), dtype=torch.float32, device="cuda:0")
+    sb.conv_bwd(c.plan, g, c.x, c.Y, c.phi, c.R, c.gy, gx, None, None, None, c.ws(1))
+    assert rel_err(gx.cpu().numpy(), c.o_bwd()[0]) <= BWD_TOL
