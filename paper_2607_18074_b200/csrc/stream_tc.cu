@@ -144,7 +144,8 @@ template <int KP, bool DUAL>
 __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int NOP = DUAL ? 2 : 1;
+    constexpr int NOP = 1;                 // operand pairs held at once (the dual stream runs its two pairs in turn)
+    constexpr int NRAW = DUAL ? 2 : 1;     // raw / transposed stages: phi and Y, plus their directions
     const int YS = a.dsh + 1;
     // A region (single buffer): A1h A1l (A2h A2l)
     uint8_t* sA = smem;
@@ -154,8 +155,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     uint8_t* meta = sRing + (size_t)NS * stage_bytes;
     float* sM0 = reinterpret_cast<float*>(meta);             // [2][max_ent][PS]: coupling matrices, double buffered
     float* sdM0 = sM0 + (size_t)2 * a.max_ent * PS;          // DUAL
-    float* sPhiT0 = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [2][NOP][KP][PS]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sPhiT0 + 2 * NOP * KP * PS);
+    float* sPhiT0 = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [2][NRAW][KP][PS]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sPhiT0 + 2 * NRAW * KP * PS);
     // bars: full[NS], freeS[NS], ready, afree, acc_full[2], acc_free[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
     UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [n_units]
@@ -173,6 +174,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     const bool has_a1 = !DUAL || has_vY || has_vphi;   // operand 1: [phi*M] (plain) or [vphi*M + phi*dM] (dual), times x
     const bool has_a2 = has_vx;                        // operand 2 (dual): [phi*M] times vx
     const bool any_op = has_a1 || has_a2;
+    // sub-batches per batch of edges: one per operand pair that is present (op = 0: x rows, op = 1: vx rows)
+    const int nsub = (has_a1 ? 1 : 0) + (has_a2 ? 1 : 0);
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 1); }
@@ -230,13 +233,16 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
         };
         prefetch_item();
-        struct Cur { int set; int64_t b0, seg1; };
+        struct Cur { int set; int64_t b0, seg1; int sub; };
         auto next_batch = [&](Cur& c, bool first) -> bool {
-            if (!first) c.b0 += TB;
+            if (!first) {
+                if (c.sub + 1 < nsub) { ++c.sub; return true; }
+                c.sub = 0; c.b0 += TB;
+            }
             while (first || c.b0 >= c.seg1) {
                 first = false;
                 if (p_item >= total) return false;
-                c.set = (int)(p_item / a.n_nodes); c.b0 = p_seg0; c.seg1 = p_seg1;
+                c.set = (int)(p_item / a.n_nodes); c.b0 = p_seg0; c.seg1 = p_seg1; c.sub = 0;
                 p_item += gridDim.x;
                 prefetch_item();
             }
@@ -250,7 +256,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 sn = a.ev.transposed ? (a.ev.recv ? a.ev.recv[pos] : (int32_t)owner_of(a.ev.row_ptr, a.ev.N, eid)) : a.ev.col[eid];
             }
         };
-        Cur cur{0, 0, 0};
+        Cur cur{0, 0, 0, 0};
         bool have = next_batch(cur, true);
         int64_t eid = 0; int32_t sn = 0;
         if (have) load_ids(cur, eid, sn);
@@ -260,6 +266,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             int64_t eid_n = 0; int32_t sn_n = 0;
             if (have_n) load_ids(nxt, eid_n, sn_n);
             const TSet S = sSet[cur.set];
+            const int op = has_a1 ? cur.sub : 1;
             const int nb = (int)min((int64_t)TB, cur.seg1 - cur.b0);
             const int st = (int)(it % NS);
             if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
@@ -288,7 +295,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
             // Y (and vY), transposed: raw[b][PS + e]
             {
-                const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
+                const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
                 const int n_it = TB * a.dsh;
                 for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
                     const int i = i0 + lt;
@@ -316,20 +323,11 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                         const int u = 8 * j;
                         uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
                         const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
-                        const __nv_bfloat16* ph = a.sh + g;
-                        const __nv_bfloat16* pl = a.sl + g;
-                        const __nv_bfloat16* vh = has_a2 ? a.vsh + g : nullptr;
-                        const __nv_bfloat16* vl = has_a2 ? a.vsl + g : nullptr;
+                        const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
+                        const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
                         for (int sdx = 0; sdx < B.d_src; ++sdx) {
-                            if (has_a1) {
-                                cp_async16_zfill(d, ph, ok);
-                                cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
-                            }
-                            if (has_a2) {
-                                cp_async16_zfill(d + 2u * (uint32_t)a.b_cap, vh, ok);
-                                cp_async16_zfill(d + 3u * (uint32_t)a.b_cap, vl, ok);
-                                vh += B.c_src; vl += B.c_src;
-                            }
+                            cp_async16_zfill(d, ph, ok);
+                            cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
                             d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
                         }
                     }
@@ -352,23 +350,21 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 const uint32_t buf = mi & 1;
                 if (mi >= 2) mbar_wait(bar_accfree + 8 * buf, ((mi >> 1) & 1) ^ 1, a.status);
                 tc_fence_after();
-                for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
-                    const int st = (int)(it % NS);
-                    mbar_wait(bar_ready, it & 1, a.status);
-                    tc_fence_after();
-                    const uint32_t sA_u = smem_u32(sA);
-                    const uint32_t sB_u = smem_u32(sRing + (size_t)st * stage_bytes);
-                    for (int ui = 0; ui < S.nunit; ++ui) {
-                        const UInfo U = sU[S.unit_begin + ui];
-                        const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + U.tmem_col;
-                        uint32_t acc = b0 == seg0 ? 0u : 1u;
-                        for (uint32_t s = 0; s < U.d_src; ++s) {
-#pragma unroll
-                            for (int op = 0; op < NOP; ++op) {
-                                if (op == 0 ? !has_a1 : !has_a2) continue;
-                                const uint32_t ah = sA_u + (uint32_t)(2 * op) * a.a_cap + U.a_off + s * U.slab_stride;
+                for (int64_t b0 = seg0; b0 < seg1; b0 += TB) {
+                    for (int sb = 0; sb < nsub; ++sb, ++it) {
+                        const int st = (int)(it % NS);
+                        mbar_wait(bar_ready, it & 1, a.status);
+                        tc_fence_after();
+                        const uint32_t sA_u = smem_u32(sA);
+                        const uint32_t sB_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                        for (int ui = 0; ui < S.nunit; ++ui) {
+                            const UInfo U = sU[S.unit_begin + ui];
+                            const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + U.tmem_col;
+                            uint32_t acc = (b0 == seg0 && sb == 0) ? 0u : 1u;
+                            for (uint32_t s = 0; s < U.d_src; ++s) {
+                                const uint32_t ah = sA_u + U.a_off + s * U.slab_stride;
                                 const uint32_t al = ah + a.a_cap;
-                                const uint32_t bh = sB_u + (uint32_t)(2 * op) * a.b_cap + U.b_off + s * U.slab_bytes;
+                                const uint32_t bh = sB_u + U.b_off + s * U.slab_bytes;
                                 const uint32_t bl = bh + a.b_cap;
                                 const uint64_t dAh = make_desc_none(ah, 128, 256), dAl = make_desc_none(al, 128, 256);
                                 const uint64_t dBh = make_desc(bh, 2048, 1024), dBl = make_desc(bl, 2048, 1024);
@@ -378,10 +374,10 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                                 acc = 1u;
                             }
                         }
+                        tc_commit(bar_afree);
+                        tc_commit(bar_free + 8 * st);
+                        if (b0 + TB >= seg1 && sb == nsub - 1) tc_commit(bar_accfull + 8 * buf);
                     }
-                    tc_commit(bar_afree);
-                    tc_commit(bar_free + 8 * st);
-                    if (b0 + TB >= seg1) tc_commit(bar_accfull + 8 * buf);
                 }
                 ++mi;
             }
@@ -468,15 +464,17 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 compute_sync();
                 cur_set = set;
             }
-            for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
+            for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
+            for (int sb = 0; sb < nsub; ++sb, ++it) {
+                const int op = has_a1 ? sb : 1;          // which operand pair this sub-batch builds
                 const int st = (int)(it % NS);
                 mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
                 const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.b_cap);
-                const float* sYT = raw + NOP * TB * KP;
+                const float* sYT = raw + NRAW * TB * KP;
                 const float* sVYT = sYT + a.dsh * PS;
                 float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
                 float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
-                float* sPhiT = sPhiT0 + (size_t)(it & 1) * NOP * KP * PS;      // [KP][PS] (+ vphi)
+                float* sPhiT = sPhiT0 + (size_t)(it & 1) * NRAW * KP * PS;     // [KP][PS] (+ vphi)
                 float* sVphiT = sPhiT + KP * PS;
                 // ---- transpose phi: [e][q] -> [q][e]   (same double buffer and barrier as the coupling matrices)
                 for (int i = tid; i < TB * KP; i += NCW * 32) {
@@ -535,26 +533,23 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                             split8(p1, hh, ll);
                             *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
                             *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
+                        } else if (op == 0) {
+                            float dmv[8], vph[8];
+                            *reinterpret_cast<float4*>(dmv) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h);
+                            *reinterpret_cast<float4*>(dmv + 4) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h + 4);
+                            *reinterpret_cast<float4*>(vph) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h);
+                            *reinterpret_cast<float4*>(vph + 4) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h + 4);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) p1[e] = fmaf(vph[e], mv[e], ph[e] * dmv[e]);
+                            split8(p1, hh, ll);
+                            *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
+                            *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
                         } else {
-                            if (has_a1) {
-                                float dmv[8], vph[8];
-                                *reinterpret_cast<float4*>(dmv) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h);
-                                *reinterpret_cast<float4*>(dmv + 4) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h + 4);
-                                *reinterpret_cast<float4*>(vph) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h);
-                                *reinterpret_cast<float4*>(vph + 4) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h + 4);
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) p1[e] = fmaf(vph[e], mv[e], ph[e] * dmv[e]);
-                                split8(p1, hh, ll);
-                                *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
-                                *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
-                            }
-                            if (has_a2) {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) p1[e] = ph[e] * mv[e];
-                                split8(p1, hh, ll);
-                                *reinterpret_cast<uint4*>(sA + 2 * a.a_cap + a_off + 128 * h) = hh;
-                                *reinterpret_cast<uint4*>(sA + 3 * a.a_cap + a_off + 128 * h) = ll;
-                            }
+                            for (int e = 0; e < 8; ++e) p1[e] = ph[e] * mv[e];
+                            split8(p1, hh, ll);
+                            *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
+                            *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
                         }
                     }
                 }
@@ -579,14 +574,14 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
 
 // shared bytes of the kernel for given region sizes
 int smem_need(int KP, bool dual, int dsh, int a_cap, int b_cap, int max_ent, int n_units, int n_sets, int n_comps, int max_nz) {
-    const int nop = dual ? 2 : 1;
-    const int stage = 2 * nop * b_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
+    const int nop = dual ? 2 : 1;     // phi / Y / M come with their directions in the dual stream
+    const int stage = 2 * b_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
     size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)2 * nop * KP * PS;
     meta = (meta + 1) & ~size_t(1);
     // tables: units (and at most as many blocks), sets, components, entries and sparse terms of one set
     const int tables = n_units * (int)(sizeof(UInfo) + sizeof(TBlk)) + n_sets * (int)sizeof(TSet) + n_comps * (int)sizeof(CompS) +
                        max_ent * (int)sizeof(EntS) + max_nz * (int)sizeof(NzS);
-    return 1024 + 2 * nop * a_cap + NS * stage + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
+    return 1024 + 2 * a_cap + NS * stage + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
 }
 
 }  // namespace
