@@ -110,7 +110,8 @@ template <int KP, bool DUAL>
 __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int NOP = DUAL ? 2 : 1;
+    constexpr int NOP = 1;                 // operand pairs held at once (the dual pass runs D and Dv in turn)
+    constexpr int NRAW = DUAL ? 2 : 1;     // raw stages: phi and Y, plus their directions
     const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023);
     const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.x_cap) + raw_bytes;
     uint8_t* sRing = smem;                                     // stages: X1h X1l (X2h X2l) raw
@@ -141,6 +142,8 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     const bool use_x = !DUAL || has_vY || has_vphi;     // D (rows of x) is needed
     const bool use_vx = has_vx;                         // Dv (rows of vx) is needed
     const bool any_op = use_x || use_vx;
+    // sub-batches per batch of edges: one per product that is needed (op = 0: rows of x, op = 1: rows of vx)
+    const int nsub = (use_x ? 1 : 0) + (use_vx ? 1 : 0);
     const TSet S = a.sets[a.set];
 
     if (tid == 0) {
@@ -226,7 +229,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             cp_async_arrive(bar_zfull);
             ++zi;
             // ---- the batches of the receiver
-            for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
+            for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
+            for (int sb = 0; sb < nsub; ++sb, ++it) {
+                const int op = use_x ? sb : 1;
                 const int nb = (int)min((int64_t)TB, seg1 - b0);
                 int64_t eid = 0; int32_t sn = 0;
                 if (lane < nb) { eid = b0 + lane; sn = a.col[eid]; }
@@ -255,7 +260,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                     }
                 }
                 {   // Y (and vY), transposed: raw[b][PS + e]
-                    const uint32_t y_u = raw_u + (uint32_t)(NOP * TB * KP) * 4;
+                    const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
                     const int n_it = TB * a.dsh;
                     for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
                         const int i = i0 + lt;
@@ -282,20 +287,11 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                             const int u = 8 * j;
                             uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
                             const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
-                            const __nv_bfloat16* ph = a.sh + g;
-                            const __nv_bfloat16* pl = a.sl + g;
-                            const __nv_bfloat16* vh = use_vx ? a.vsh + g : nullptr;
-                            const __nv_bfloat16* vl = use_vx ? a.vsl + g : nullptr;
+                            const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
+                            const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
                             for (int sdx = 0; sdx < B.d_src; ++sdx) {
-                                if (use_x) {
-                                    cp_async16_zfill(d, ph, ok);
-                                    cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
-                                }
-                                if (use_vx) {
-                                    cp_async16_zfill(d + 2u * (uint32_t)a.x_cap, vh, ok);
-                                    cp_async16_zfill(d + 3u * (uint32_t)a.x_cap, vl, ok);
-                                    vh += B.c_src; vl += B.c_src;
-                                }
+                                cp_async16_zfill(d, ph, ok);
+                                cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
                                 d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
                             }
                         }
@@ -315,7 +311,8 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 if (seg1 <= seg0) continue;
                 mbar_wait(bar_zfull, zi & 1, a.status);
                 ++zi;
-                for (int64_t b0 = seg0; b0 < seg1; b0 += TB, ++it) {
+                for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
+                for (int sb = 0; sb < nsub; ++sb, ++it) {
                     const int st = (int)(it % NS);
                     mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
                     fence_async_smem();
@@ -326,23 +323,19 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                         const uint32_t buf = ai & 1;
                         if (ai >= 2) mbar_wait(bar_accfree + 8 * buf, ((ai >> 1) & 1) ^ 1, a.status);
                         tc_fence_after();
-#pragma unroll
-                        for (int op = 0; op < NOP; ++op) {
-                            if (op == 0 ? !use_x : !use_vx) continue;
-                            for (uint32_t mt = 0; mt < U.nmt; ++mt) {
-                                const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + ((uint32_t)op * U.nmt + mt) * U.npad;
-                                for (uint32_t ks = 0; ks < U.ksteps; ++ks) {
-                                    const uint32_t kb = ks >> 2, kk = ks & 3;
-                                    const uint32_t xh = sX_u + (uint32_t)(2 * op) * a.x_cap + U.x_off + kb * U.x_kb + mt * (128u * 128u) + 32u * kk;
-                                    const uint32_t xl = xh + a.x_cap;
-                                    const uint32_t zh = sZ_u + U.z_off + kb * U.z_kb + 32u * kk;
-                                    const uint32_t zl = zh + a.z_cap;
-                                    const uint64_t dXh = make_desc(xh, 16, 1024), dXl = make_desc(xl, 16, 1024);
-                                    const uint64_t dZh = make_desc(zh, 16, 1024), dZl = make_desc(zl, 16, 1024);
-                                    tc_mma_bf16(d_tmem, dXh, dZh, U.idesc, ks > 0 ? 1u : 0u);
-                                    tc_mma_bf16(d_tmem, dXl, dZh, U.idesc, 1u);
-                                    tc_mma_bf16(d_tmem, dXh, dZl, U.idesc, 1u);
-                                }
+                        for (uint32_t mt = 0; mt < U.nmt; ++mt) {
+                            const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + mt * U.npad;
+                            for (uint32_t ks = 0; ks < U.ksteps; ++ks) {
+                                const uint32_t kb = ks >> 2, kk = ks & 3;
+                                const uint32_t xh = sX_u + U.x_off + kb * U.x_kb + mt * (128u * 128u) + 32u * kk;
+                                const uint32_t xl = xh + a.x_cap;
+                                const uint32_t zh = sZ_u + U.z_off + kb * U.z_kb + 32u * kk;
+                                const uint32_t zl = zh + a.z_cap;
+                                const uint64_t dXh = make_desc(xh, 16, 1024), dXl = make_desc(xl, 16, 1024);
+                                const uint64_t dZh = make_desc(zh, 16, 1024), dZl = make_desc(zl, 16, 1024);
+                                tc_mma_bf16(d_tmem, dXh, dZh, U.idesc, ks > 0 ? 1u : 0u);
+                                tc_mma_bf16(d_tmem, dXl, dZh, U.idesc, 1u);
+                                tc_mma_bf16(d_tmem, dXh, dZl, U.idesc, 1u);
                             }
                         }
                         tc_commit(bar_accfull + 8 * buf);
@@ -365,23 +358,26 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 compute_sync();     // the previous group's outputs have been written
                 for (int i = tid; i < EG * KP; i += NCW * 32) accPhi[i] = 0.f;
                 for (int i = tid; i < EG * a.dsh; i += NCW * 32) accY[i] = 0.f;
-                for (int64_t b0 = g0; b0 < g1; b0 += TB, ++it) {
-                    const int st = (int)(it % NS);
+                for (int64_t b0 = g0; b0 < g1; b0 += TB) {
                     const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
+                    float pphi[KP];
+#pragma unroll
+                    for (int q = 0; q < KP; ++q) pphi[q] = 0.f;
+                    for (int sb = 0; sb < nsub; ++sb, ++it) {
+                    const int op = use_x ? sb : 1;           // D (rows of x) or Dv (rows of vx)
+                    const int st = (int)(it % NS);
                     mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
                     const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.x_cap);
-                    const float* sYT = raw + NOP * TB * KP;
+                    const float* sYT = raw + NRAW * TB * KP;
                     const float* sVYT = sYT + a.dsh * PS;
                     float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
                     float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
                     // ---- this thread's radial weights, then the coupling matrices: thread <-> (entry, 8 edges)
-                    float ph[KP], vph[KP], pphi[KP];
+                    // weights of this sub-batch: gM += sum_q aw[q] * D,  gphi[q] += mw * D
+                    //   plain: aw = phi, mw = M;   dual, op 0: aw = vphi, mw = dM;   dual, op 1: aw = phi, mw = M
+                    float aw[KP];
 #pragma unroll
-                    for (int q = 0; q < KP; ++q) {
-                        ph[q] = raw[e * KP + q];
-                        vph[q] = DUAL ? raw[TB * KP + e * KP + q] : 0.f;
-                        pphi[q] = 0.f;
-                    }
+                    for (int q = 0; q < KP; ++q) aw[q] = (DUAL && op == 0) ? raw[TB * KP + e * KP + q] : raw[e * KP + q];
                     for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
                         const int j = i >> 1, h = i & 1;
                         const EntS en = sEnt[j];
@@ -430,38 +426,28 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                             const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
                             for (int cl = c_lo; cl < c_hi; ++cl) {
                                 const int ent = ent_u + cl * d_src + s;
-                                const float mw = rv ? sM[ent * PS + e] : 0.f;
-                                const float dmw = (DUAL && rv) ? sdM[ent * PS + e] : 0.f;
+                                const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
                                 float gm = 0.f;
 #pragma unroll
                                 for (int q8 = 0; q8 < KP; q8 += 8) {
-                                    float v[8], v2[8];
-                                    if (use_x) tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
-                                    if (DUAL && use_vx) tc_ld8(t0 + (uint32_t)((nmt + mt) * npad + cl * KP + q8), v2);
+                                    float v[8];
+                                    tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
                                     if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
 #pragma unroll
                                         for (int x = 0; x < 8; ++x) {
-                                            if (!DUAL) {
-                                                gm = fmaf(ph[q8 + x], v[x], gm);
-                                                pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
-                                            } else {
-                                                if (has_vphi) gm = fmaf(vph[q8 + x], v[x], gm);
-                                                if (has_vY) pphi[q8 + x] = fmaf(dmw, v[x], pphi[q8 + x]);
-                                                if (use_vx) {
-                                                    gm = fmaf(ph[q8 + x], v2[x], gm);
-                                                    pphi[q8 + x] = fmaf(mw, v2[x], pphi[q8 + x]);
-                                                }
-                                            }
+                                            gm = fmaf(aw[q8 + x], v[x], gm);
+                                            pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
                                         }
                                     }
                                 }
-                                if (rv) sGM[ent * PS + e] = gm;
+                                if (rv) sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                             }
                         }
                         tc_fence_before();
                         mbar_arrive(bar_accfree + 8 * buf);
                         ent_u += (int)U.ncomp * d_src;
                     }
+                    }   // sub-batches
                     // lanes l and l+16 of a warp hold rows of the same edge
 #pragma unroll
                     for (int q = 0; q < KP; ++q) {
@@ -522,7 +508,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
 
 int smem_need(int KP, bool dual, int dsh, int x_cap, int z_cap, int max_ent, int max_units, int max_nz, int max_inv) {
     const int nop = dual ? 2 : 1;
-    const int stage = 2 * nop * x_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
+    const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
     const size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)max_ent * PS + (size_t)NCW * 16 * KP + (size_t)EG * KP +
                         (size_t)((EG * dsh + 1) & ~1);
     const int tables = max_units * (int)(sizeof(UInfo) + sizeof(TBlk) + (128 / KP) * sizeof(CompS)) + max_ent * (int)sizeof(EntS) +
@@ -571,7 +557,7 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         auto unit_z = [&](const Cand& c) { return npad(c) * 128 * nkb(c.blk); };
         auto blk_x = [&](int b) { return blocks[b].d_src * 2048 * nkb(b); };
         auto nmt = [&](int b) { return (blocks[b].d_src * TB + 127) / 128; };
-        auto unit_cols = [&](const Cand& c) { return nop * nmt(c.blk) * npad(c); };
+        auto unit_cols = [&](const Cand& c) { return nmt(c.blk) * npad(c); };
         auto cand_nz = [&](const Cand& c) {
             int n = 0;
             for (int cl = 0; cl < c.nc; ++cl) {
