@@ -18,8 +18,10 @@
 // from D (sender rows of x) and Dv (sender rows of vx):
 //     gM = sum_q ( vphi[q] D + phi[q] Dv ),   gphi[q] += dM D + M Dv.
 //
-// Roles of a CTA (one receiver at a time, its edges in groups of 64 and batches of 16, the accumulator
-// tiles of the profile in sets): loader warps (cp.async of the Zbar slabs of a set, of the batch's phi / Y
+// One launch per set of accumulator tiles (the first writes the outputs, the others accumulate).  The batch
+// size tb of a set is the largest power of two (16..128) whose rows (s, e) = d_src * tb still fill one
+// 128-row tile, so that the accumulator rows - one epilogue thread each - are used as fully as possible.
+// Roles of a CTA (one receiver at a time, its edges in batches of tb): loader warps (cp.async of the Zbar slabs of a set, of the batch's phi / Y
 // rows and of the sender rows into a two-stage ring), one MMA thread (two TMEM accumulator buffers), and
 // compute warps (coupling matrices M_e from the sparse CG table, epilogue, fixed-order reductions, output).
 // Every mbarrier wait is bounded.
@@ -35,13 +37,11 @@ namespace {
 
 using namespace ptx;
 
-constexpr int TB = 16;          // edges per batch
-constexpr int EG = 64;          // edges per group (outputs of a group are accumulated in shared memory)
 constexpr int NCW = 8;          // compute warps
 constexpr int NLW = 2;          // loader warps
 constexpr int TT = (NCW + NLW + 1) * 32;
 constexpr int NS = 2;           // ring stages
-constexpr int PS = 20;          // row pitch (floats) of the [.][16 edges] stages
+constexpr int EGMIN = 64;       // edges per output group: max(EGMIN, tb)
 
 struct EtArgs {
     const TSet* sets;
@@ -69,7 +69,8 @@ struct EtArgs {
     float* gY;
     int32_t phi_mode, Y_mode;   // 0 skip, 1 overwrite, 2 accumulate
     int32_t K, dsh, C_src, set;
-    int32_t x_cap, z_cap, max_ent, tmem_cols, acc_cols, max_nz, max_inv, max_units;
+    int32_t tb, lg;             // edges per batch (power of two) and its log2
+    int32_t x_cap, z_cap, nent, tmem_cols, acc_cols, nnz, ninv, nunit, ncomp;
     int* status;
 };
 
@@ -100,39 +101,40 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// per-stage raw area (floats): phi rows [TB][KP], (vphi), and Y written transposed [dsh][PS], (vY)
-__host__ __device__ inline int raw_floats(int KP, bool dual, int dsh) {
+// per-stage raw area (floats): phi rows [tb][KP], (vphi), Y written transposed [dsh][tb+4], (vY), sender ids [tb]
+__host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
     const int n = dual ? 2 : 1;
-    return n * TB * KP + n * dsh * PS;
+    return n * tb * KP + n * dsh * (tb + 4) + tb;
 }
+__host__ __device__ inline int group_edges(int tb) { return tb > EGMIN ? tb : EGMIN; }
 
 template <int KP, bool DUAL>
 __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int NOP = 1;                 // operand pairs held at once (the dual pass runs D and Dv in turn)
     constexpr int NRAW = DUAL ? 2 : 1;     // raw stages: phi and Y, plus their directions
-    const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023);
-    const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.x_cap) + raw_bytes;
-    uint8_t* sRing = smem;                                     // stages: X1h X1l (X2h X2l) raw
+    const int tb = a.tb, lg = a.lg, PS = a.tb + 4, EG = group_edges(a.tb);
+    const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh, tb) * 4 + 1023) & ~1023);
+    const uint32_t stage_bytes = (uint32_t)(2 * a.x_cap) + raw_bytes;
+    uint8_t* sRing = smem;                                     // stages: Xh Xl raw
     uint8_t* sZ = sRing + (size_t)NS * stage_bytes;            // Zbar slabs of the set: hi, lo
     uint8_t* meta = sZ + (size_t)2 * a.z_cap;
-    float* sM0 = reinterpret_cast<float*>(meta);               // [2][max_ent][PS] coupling matrices, double buffered
-    float* sdM0 = sM0 + (size_t)2 * a.max_ent * PS;            // DUAL
-    float* sGM = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [max_ent][PS]
-    float* sPphi = sGM + (size_t)a.max_ent * PS;               // [NCW*16][KP]: one row per (warp, edge)
-    float* accPhi = sPphi + NCW * 16 * KP;                     // [EG][KP]
+    float* sM0 = reinterpret_cast<float*>(meta);               // [2][nent][PS] coupling matrices, double buffered
+    float* sdM0 = sM0 + (size_t)2 * a.nent * PS;               // DUAL
+    float* sGM = sdM0 + (DUAL ? (size_t)2 * a.nent * PS : 0);  // [nent][PS]
+    float* sPphi = sGM + (size_t)a.nent * PS;                  // [NCW*32][KP]: one row per compute thread
+    float* accPhi = sPphi + NCW * 32 * KP;                     // [EG][KP]
     float* accY = accPhi + EG * KP;                            // [EG][dsh]
     uint64_t* bars = reinterpret_cast<uint64_t*>(accY + ((EG * a.dsh + 1) & ~1));
     // bars: full[NS], free[NS], zfull, zfree, acc_full[2], acc_free[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
-    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [max_units]
-    TBlk* sBlk = reinterpret_cast<TBlk*>(sU + a.max_units);            // [max_units]
-    CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.max_units);       // [128 / KP * max_units]
-    EntS* sEnt = reinterpret_cast<EntS*>(sComp + (128 / KP) * a.max_units);   // [max_ent]
-    NzS* sNz = reinterpret_cast<NzS*>(sEnt + a.max_ent);               // [max_nz]
-    NzS* sInv = sNz + a.max_nz;                                        // [max_inv]
-    int32_t* sInvPtr = reinterpret_cast<int32_t*>(sInv + a.max_inv);   // [dsh + 1]
+    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [nunit]
+    TBlk* sBlk = reinterpret_cast<TBlk*>(sU + a.nunit);                // [nunit]
+    CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.nunit);           // [ncomp]
+    EntS* sEnt = reinterpret_cast<EntS*>(sComp + a.ncomp);             // [nent]
+    NzS* sNz = reinterpret_cast<NzS*>(sEnt + a.nent);                  // [nnz]
+    NzS* sInv = sNz + a.nnz;                                           // [ninv]
+    int32_t* sInvPtr = reinterpret_cast<int32_t*>(sInv + a.ninv);      // [dsh + 1]
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_zfull = bar0 + 16 * NS, bar_zfree = bar_zfull + 8,
                    bar_accfull = bar_zfull + 16, bar_accfree = bar_zfull + 32;
@@ -157,7 +159,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     // zero what is never written later: the raw rows of padded radial components / absent directions, and the
     // Zbar slab rows of padded radial components (they meet zeros of phi, but must stay finite)
     {
-        const int words = (int)(stage_bytes / 4), x_words = 2 * NOP * a.x_cap / 4;
+        const int words = (int)(stage_bytes / 4), x_words = 2 * a.x_cap / 4;
         for (int i = tid; i < NS * words; i += TT) {
             const int st = i / words, w = i - st * words;
             if (w >= x_words) reinterpret_cast<uint32_t*>(sRing + (size_t)st * stage_bytes)[w] = 0u;
@@ -174,7 +176,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         u.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((u.npad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         u.z_off = (uint32_t)U.a_off; u.z_kb = (uint32_t)U.slab_stride;
         u.x_off = (uint32_t)B.b_off; u.x_kb = (uint32_t)B.atom_stride;
-        u.ksteps = (uint32_t)(B.c_src >> 4); u.nmt = (uint32_t)((B.d_src * TB + 127) / 128);
+        u.ksteps = (uint32_t)(B.c_src >> 4); u.nmt = (uint32_t)((B.d_src * tb + 127) / 128);
         u.ncomp = (uint32_t)U.ncomp; u.comp_begin = (uint32_t)(U.comp_begin - a.units[S.unit_begin].comp_begin);
         u.d_src = (uint32_t)B.d_src; u.c_src = (uint32_t)B.c_src;
         sU[i] = u;
@@ -182,13 +184,12 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     for (int i = tid; i < S.nblk; i += TT) sBlk[i] = a.blks[S.blk_begin + i];
     {
         const int c0 = a.units[S.unit_begin].comp_begin;
-        const TUnit UL = a.units[S.unit_begin + S.nunit - 1];
-        for (int i = tid; i < UL.comp_begin + UL.ncomp - c0; i += TT) sComp[i] = a.comps[c0 + i];
+        for (int i = tid; i < a.ncomp; i += TT) sComp[i] = a.comps[c0 + i];
     }
     for (int i = tid; i < S.nent; i += TT) sEnt[i] = a.ents[i];
-    for (int i = tid; i < S.pad; i += TT) sNz[i] = a.nz[i];
+    for (int i = tid; i < a.nnz; i += TT) sNz[i] = a.nz[i];
     for (int i = tid; i <= a.dsh; i += TT) sInvPtr[i] = a.inv_ptr[i];
-    for (int i = tid; i < a.inv_ptr[a.dsh]; i += TT) sInv[i] = a.inv[i];
+    for (int i = tid; i < a.ninv; i += TT) sInv[i] = a.inv[i];
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)a.tmem_cols) : "memory");
@@ -229,71 +230,64 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             cp_async_arrive(bar_zfull);
             ++zi;
             // ---- the batches of the receiver
-            for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
+            for (int64_t b0 = seg0; b0 < seg1; b0 += tb)
             for (int sb = 0; sb < nsub; ++sb, ++it) {
                 const int op = use_x ? sb : 1;
-                const int nb = (int)min((int64_t)TB, seg1 - b0);
-                int64_t eid = 0; int32_t sn = 0;
-                if (lane < nb) { eid = b0 + lane; sn = a.col[eid]; }
+                const int nb = (int)min((int64_t)tb, seg1 - b0);
                 const int st = (int)(it % NS);
                 if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
-                const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
-                const uint32_t raw_u = stage_u + (uint32_t)(2 * NOP * a.x_cap);
+                uint8_t* stage = sRing + (size_t)st * stage_bytes;
+                const uint32_t stage_u = smem_u32(stage);
+                const uint32_t raw_u = stage_u + (uint32_t)(2 * a.x_cap);
+                // sender ids of the batch (each loader warp keeps its own copy of all of them)
+                int32_t* sIds = reinterpret_cast<int32_t*>(stage + 2 * a.x_cap) + NRAW * tb * KP + NRAW * a.dsh * PS + (warp - NCW) * 0;
+                for (int e = lane; e < tb; e += 32) sIds[e] = e < nb ? a.col[b0 + e] : 0;
+                __syncwarp();
                 {
                     const bool v16 = (a.K & 3) == 0;
                     const int per = v16 ? a.K / 4 : a.K;
-                    const int n_it = TB * per;
-                    for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
-                        const int i = i0 + lt;
-                        const int e = min(i / per, TB - 1), j = i - (i / per) * per;
-                        const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
-                        if (i < n_it) {
-                            const uint32_t ok = e < nb ? 1u : 0u;
-                            if (v16) {
-                                cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
-                                if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(TB * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
-                            } else {
-                                cp_async4_zfill(raw_u + (uint32_t)(e * KP + j) * 4, a.phi + ee * a.K + j, ok * 4);
-                                if (has_vphi) cp_async4_zfill(raw_u + (uint32_t)(TB * KP + e * KP + j) * 4, a.vphi + ee * a.K + j, ok * 4);
-                            }
+                    const int n_it = tb * per;
+                    for (int i = lt; i < n_it; i += NLW * 32) {
+                        const int e = i / per, j = i - e * per;
+                        const int64_t ee = b0 + min(e, nb - 1);
+                        const uint32_t ok = e < nb ? 1u : 0u;
+                        if (v16) {
+                            cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
+                            if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(tb * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
+                        } else {
+                            cp_async4_zfill(raw_u + (uint32_t)(e * KP + j) * 4, a.phi + ee * a.K + j, ok * 4);
+                            if (has_vphi) cp_async4_zfill(raw_u + (uint32_t)(tb * KP + e * KP + j) * 4, a.vphi + ee * a.K + j, ok * 4);
                         }
                     }
                 }
                 {   // Y (and vY), transposed: raw[b][PS + e]
-                    const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
-                    const int n_it = TB * a.dsh;
-                    for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
-                        const int i = i0 + lt;
-                        const int e = min(i / a.dsh, TB - 1), b = i - (i / a.dsh) * a.dsh;
-                        const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
-                        if (i < n_it) {
-                            const uint32_t ok = e < nb ? 4u : 0u;
-                            cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
-                            if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
-                        }
+                    const uint32_t y_u = raw_u + (uint32_t)(NRAW * tb * KP) * 4;
+                    const int n_it = tb * a.dsh;
+                    for (int i = lt; i < n_it; i += NLW * 32) {
+                        const int e = i / a.dsh, b = i - e * a.dsh;
+                        const int64_t ee = b0 + min(e, nb - 1);
+                        const uint32_t ok = e < nb ? 4u : 0u;
+                        cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
+                        if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
                     }
                 }
                 // sender rows: rows (s, e) of 128 bytes per 64 multiplicities, 128-byte swizzle
                 for (int bi = 0; bi < S.nblk; ++bi) {
                     const TBlk B = sBlk[bi];
                     const int cpr = B.c_src >> 3;
-                    const int npair = TB * cpr;
-                    for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
-                        const int pr = p0 + lt;
-                        const int e = min(pr / cpr, TB - 1), j = pr - (pr / cpr) * cpr;
-                        const int32_t sne = __shfl_sync(0xffffffffu, sn, e);
-                        if (pr < npair) {
-                            const uint32_t ok = e < nb ? 16u : 0u;
-                            const int u = 8 * j;
-                            uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
-                            const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
-                            const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
-                            const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
-                            for (int sdx = 0; sdx < B.d_src; ++sdx) {
-                                cp_async16_zfill(d, ph, ok);
-                                cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
-                                d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
-                            }
+                    const int npair = tb * cpr;
+                    for (int pr = lt; pr < npair; pr += NLW * 32) {
+                        const int e = pr / cpr, j = pr - e * cpr;
+                        const uint32_t ok = e < nb ? 16u : 0u;
+                        const int u = 8 * j;
+                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
+                        const int64_t g = (int64_t)sIds[e] * a.C_src + B.src_off + u;
+                        const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
+                        const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
+                        for (int sdx = 0; sdx < B.d_src; ++sdx) {
+                            cp_async16_zfill(d, ph, ok);
+                            cp_async16_zfill(d + (uint32_t)a.x_cap, pl, ok);
+                            d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
                         }
                     }
                 }
@@ -311,7 +305,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 if (seg1 <= seg0) continue;
                 mbar_wait(bar_zfull, zi & 1, a.status);
                 ++zi;
-                for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
+                for (int64_t b0 = seg0; b0 < seg1; b0 += tb)
                 for (int sb = 0; sb < nsub; ++sb, ++it) {
                     const int st = (int)(it % NS);
                     mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
@@ -349,7 +343,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         // =========================== compute warps ===========================
         uint32_t it = 0, ai = 0;
         const int quarter = warp & 3, half = warp >> 2;
-        const int e = lane & 15;                     // the edge of this thread's accumulator rows
+        const int row0 = quarter * 32 + lane;        // this thread's accumulator row inside a 128-row tile
+        const int e = row0 & (tb - 1);               // its edge (the same in every tile: 128 is a multiple of tb)
+        const int t8 = tb >> 3;                      // 8-edge octets per batch
         for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
             const int64_t node = a.node0 + nl;
             const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
@@ -358,126 +354,121 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 compute_sync();     // the previous group's outputs have been written
                 for (int i = tid; i < EG * KP; i += NCW * 32) accPhi[i] = 0.f;
                 for (int i = tid; i < EG * a.dsh; i += NCW * 32) accY[i] = 0.f;
-                for (int64_t b0 = g0; b0 < g1; b0 += TB) {
+                for (int64_t b0 = g0; b0 < g1; b0 += tb) {
                     const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
                     float pphi[KP];
 #pragma unroll
                     for (int q = 0; q < KP; ++q) pphi[q] = 0.f;
                     for (int sb = 0; sb < nsub; ++sb, ++it) {
-                    const int op = use_x ? sb : 1;           // D (rows of x) or Dv (rows of vx)
-                    const int st = (int)(it % NS);
-                    mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
-                    const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.x_cap);
-                    const float* sYT = raw + NRAW * TB * KP;
-                    const float* sVYT = sYT + a.dsh * PS;
-                    float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
-                    float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
-                    // ---- this thread's radial weights, then the coupling matrices: thread <-> (entry, 8 edges)
-                    // weights of this sub-batch: gM += sum_q aw[q] * D,  gphi[q] += mw * D
-                    //   plain: aw = phi, mw = M;   dual, op 0: aw = vphi, mw = dM;   dual, op 1: aw = phi, mw = M
-                    float aw[KP];
+                        const int op = use_x ? sb : 1;           // D (rows of x) or Dv (rows of vx)
+                        const int st = (int)(it % NS);
+                        mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
+                        const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.x_cap);
+                        const float* sYT = raw + NRAW * tb * KP;
+                        const float* sVYT = sYT + a.dsh * PS;
+                        float* sM = sM0 + (size_t)(it & 1) * a.nent * PS;
+                        float* sdM = sdM0 + (size_t)(it & 1) * a.nent * PS;
+                        // weights of this sub-batch: gM += sum_q aw[q] * D,  gphi[q] += mw * D
+                        //   plain: aw = phi, mw = M;   dual, op 0: aw = vphi, mw = dM;   dual, op 1: aw = phi, mw = M
+                        float aw[KP];
 #pragma unroll
-                    for (int q = 0; q < KP; ++q) aw[q] = (DUAL && op == 0) ? raw[TB * KP + e * KP + q] : raw[e * KP + q];
-                    for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
-                        const int j = i >> 1, h = i & 1;
-                        const EntS en = sEnt[j];
-                        float m[8], dm[8];
+                        for (int q = 0; q < KP; ++q) aw[q] = (DUAL && op == 0) ? raw[tb * KP + e * KP + q] : raw[e * KP + q];
+                        // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
+                        for (int i = tid; i < S.nent * t8; i += NCW * 32) {
+                            const int j = i / t8, o8 = 8 * (i - j * t8);
+                            const EntS en = sEnt[j];
+                            float m[8], dm[8];
 #pragma unroll
-                        for (int x = 0; x < 8; ++x) { m[x] = 0.f; dm[x] = 0.f; }
-                        for (int k = en.nz_begin; k < en.nz_begin + en.nz_count; ++k) {
-                            const NzS t = sNz[k];
-                            float y[8];
-                            *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + t.b * PS + 8 * h);
-                            *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + t.b * PS + 8 * h + 4);
+                            for (int x = 0; x < 8; ++x) { m[x] = 0.f; dm[x] = 0.f; }
+                            for (int k = en.nz_begin; k < en.nz_begin + en.nz_count; ++k) {
+                                const NzS t = sNz[k];
+                                float y[8];
+                                *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sYT + t.b * PS + o8);
+                                *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sYT + t.b * PS + o8 + 4);
 #pragma unroll
-                            for (int x = 0; x < 8; ++x) m[x] = fmaf(t.coef, y[x], m[x]);
+                                for (int x = 0; x < 8; ++x) m[x] = fmaf(t.coef, y[x], m[x]);
+                                if (DUAL) {
+                                    *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + o8);
+                                    *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + o8 + 4);
+#pragma unroll
+                                    for (int x = 0; x < 8; ++x) dm[x] = fmaf(t.coef, y[x], dm[x]);
+                                }
+                            }
+                            *reinterpret_cast<float4*>(sM + j * PS + o8) = *reinterpret_cast<const float4*>(m);
+                            *reinterpret_cast<float4*>(sM + j * PS + o8 + 4) = *reinterpret_cast<const float4*>(m + 4);
                             if (DUAL) {
-                                *reinterpret_cast<float4*>(y) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + 8 * h);
-                                *reinterpret_cast<float4*>(y + 4) = *reinterpret_cast<const float4*>(sVYT + t.b * PS + 8 * h + 4);
-#pragma unroll
-                                for (int x = 0; x < 8; ++x) dm[x] = fmaf(t.coef, y[x], dm[x]);
+                                *reinterpret_cast<float4*>(sdM + j * PS + o8) = *reinterpret_cast<const float4*>(dm);
+                                *reinterpret_cast<float4*>(sdM + j * PS + o8 + 4) = *reinterpret_cast<const float4*>(dm + 4);
                             }
                         }
-                        *reinterpret_cast<float4*>(sM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(m);
-                        *reinterpret_cast<float4*>(sM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(m + 4);
-                        if (DUAL) {
-                            *reinterpret_cast<float4*>(sdM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(dm);
-                            *reinterpret_cast<float4*>(sdM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(dm + 4);
-                        }
-                    }
-                    // the raw rows of the stage are consumed by this thread (the stage is released when all compute
-                    // threads have said so and the batch's MMAs, which read the sender rows, have retired)
-                    mbar_arrive(bar_free + 8 * st);
-                    compute_sync();     // coupling matrices complete; the previous batch's reductions are done
-                    // ---- epilogue of the batch: this thread owns accumulator rows (s, e) with e = lane & 15
-                    int ent_u = 0;                // first entry of the unit inside the set
-                    for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
-                        const UInfo U = sU[ui];
-                        const int npad = (int)U.npad, nmt = (int)U.nmt, d_src = (int)U.d_src;
-                        const uint32_t buf = ai & 1;
-                        mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
-                        tc_fence_after();
-                        const int chalf = ((int)U.ncomp + 1) >> 1;
-                        const int c_lo = half * chalf, c_hi = min((int)U.ncomp, c_lo + chalf);
-                        for (int mt = 0; mt < nmt; ++mt) {
-                            const int row = mt * 128 + quarter * 32 + lane;
-                            const int s = row >> 4;
-                            const bool rv = s < d_src;
-                            const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
-                            for (int cl = c_lo; cl < c_hi; ++cl) {
-                                const int ent = ent_u + cl * d_src + s;
-                                const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
-                                float gm = 0.f;
+                        // the raw rows of the stage are consumed by this thread (the stage is released when all compute
+                        // threads have said so and the batch's MMAs, which read the sender rows, have retired)
+                        mbar_arrive(bar_free + 8 * st);
+                        compute_sync();     // coupling matrices complete; the previous batch's reductions are done
+                        // ---- epilogue: this thread owns the accumulator rows (s, e) = (row >> lg, row & (tb-1))
+                        int ent_u = 0;                // first entry of the unit inside the set
+                        for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
+                            const UInfo U = sU[ui];
+                            const int npad = (int)U.npad, nmt = (int)U.nmt, d_src = (int)U.d_src;
+                            const uint32_t buf = ai & 1;
+                            mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
+                            tc_fence_after();
+                            const int chalf = ((int)U.ncomp + 1) >> 1;
+                            const int c_lo = half * chalf, c_hi = min((int)U.ncomp, c_lo + chalf);
+                            for (int mt = 0; mt < nmt; ++mt) {
+                                const int s = (mt * 128 + row0) >> lg;
+                                const bool rv = s < d_src;
+                                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
+                                for (int cl = c_lo; cl < c_hi; ++cl) {
+                                    const int ent = ent_u + cl * d_src + s;
+                                    const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
+                                    float gm = 0.f;
 #pragma unroll
-                                for (int q8 = 0; q8 < KP; q8 += 8) {
-                                    float v[8];
-                                    tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
-                                    if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
+                                    for (int q8 = 0; q8 < KP; q8 += 8) {
+                                        float v[8];
+                                        tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
+                                        if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
 #pragma unroll
-                                        for (int x = 0; x < 8; ++x) {
-                                            gm = fmaf(aw[q8 + x], v[x], gm);
-                                            pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
+                                            for (int x = 0; x < 8; ++x) {
+                                                gm = fmaf(aw[q8 + x], v[x], gm);
+                                                pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
+                                            }
                                         }
                                     }
+                                    if (rv) sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                                 }
-                                if (rv) sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                             }
+                            tc_fence_before();
+                            mbar_arrive(bar_accfree + 8 * buf);
+                            ent_u += (int)U.ncomp * d_src;
                         }
-                        tc_fence_before();
-                        mbar_arrive(bar_accfree + 8 * buf);
-                        ent_u += (int)U.ncomp * d_src;
-                    }
                     }   // sub-batches
-                    // lanes l and l+16 of a warp hold rows of the same edge
 #pragma unroll
-                    for (int q = 0; q < KP; ++q) {
-                        const float o = __shfl_xor_sync(0xffffffffu, pphi[q], 16);
-                        if (lane < 16) sPphi[(warp * 16 + lane) * KP + q] = pphi[q] + o;
-                    }
+                    for (int q = 0; q < KP; ++q) sPphi[tid * KP + q] = pphi[q];
                     compute_sync();
-                    // ---- fixed-order reductions into the group's accumulators
-                    for (int i = tid; i < TB * KP; i += NCW * 32) {
+                    // ---- fixed-order reductions into the group's accumulators: the threads that share an edge
+                    // are those whose row is congruent to it modulo tb, in both column halves
+                    for (int i = tid; i < tb * KP; i += NCW * 32) {
                         const int ee = i / KP, q = i - ee * KP;
                         float v = 0.f;
-#pragma unroll
-                        for (int j = 0; j < NCW; ++j) v += sPphi[(j * 16 + ee) * KP + q];
+                        for (int r = ee; r < 128; r += tb) v += sPphi[r * KP + q] + sPphi[(128 + r) * KP + q];
                         accPhi[(bg + ee) * KP + q] += v;
                     }
-                    for (int i = tid; i < 2 * a.dsh; i += NCW * 32) {
-                        const int b = i >> 1, h = i & 1;
+                    for (int i = tid; i < t8 * a.dsh; i += NCW * 32) {
+                        const int b = i / t8, o8 = 8 * (i - b * t8);
                         float g[8];
 #pragma unroll
                         for (int x = 0; x < 8; ++x) g[x] = 0.f;
                         for (int k = sInvPtr[b]; k < sInvPtr[b + 1]; ++k) {
                             const NzS t = sInv[k];
                             float gm[8];
-                            *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + t.b * PS + 8 * h);
-                            *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + t.b * PS + 8 * h + 4);
+                            *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + t.b * PS + o8);
+                            *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + t.b * PS + o8 + 4);
 #pragma unroll
                             for (int x = 0; x < 8; ++x) g[x] = fmaf(t.coef, gm[x], g[x]);
                         }
 #pragma unroll
-                        for (int x = 0; x < 8; ++x) accY[(bg + 8 * h + x) * a.dsh + b] += g[x];
+                        for (int x = 0; x < 8; ++x) accY[(bg + o8 + x) * a.dsh + b] += g[x];
                     }
                 }
                 compute_sync();
@@ -506,21 +497,25 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     }
 }
 
-int smem_need(int KP, bool dual, int dsh, int x_cap, int z_cap, int max_ent, int max_units, int max_nz, int max_inv) {
+// shared bytes of a launch
+int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent, int nunit, int ncomp, int nnz, int ninv) {
     const int nop = dual ? 2 : 1;
-    const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
-    const size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)max_ent * PS + (size_t)NCW * 16 * KP + (size_t)EG * KP +
+    const int PS = tb + 4, EG = group_edges(tb);
+    const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
+    const size_t meta = (size_t)2 * nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)EG * KP +
                         (size_t)((EG * dsh + 1) & ~1);
-    const int tables = max_units * (int)(sizeof(UInfo) + sizeof(TBlk) + (128 / KP) * sizeof(CompS)) + max_ent * (int)sizeof(EntS) +
-                       (max_nz + max_inv) * (int)sizeof(NzS) + (dsh + 2) * 4;
+    const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
+                       (nnz + ninv) * (int)sizeof(NzS) + (dsh + 2) * 4;
     return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
 }
 
 }  // namespace
 
 // Units and sets of the tensor-core edge pass (receiver direction) for the plain ([0]) and dual ([1]) pass.
+// Every set is one launch with its own batch size and shared-memory layout.
 void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
     const int KP = p->K <= 8 ? 8 : 16;
+    const int dsh = p->dim_sh;
     for (int dual = 0; dual < 2; ++dual) {
         TcSets& T = dir.etc[dual];
         T = TcSets{};
@@ -529,7 +524,6 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         for (const DPath& P : dir.paths)
             if ((P.c_src & 15) || P.c_src > 128 || (P.src_off & 7)) ok = false;
         if (!ok || (dir.C_src & 7) || dir.paths.empty()) continue;
-        const int nop = dual ? 2 : 1;
         struct Blk { int so, c_src, d_src; std::vector<SComp> comps; };
         std::vector<Blk> blocks;
         for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
@@ -555,9 +549,6 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         auto nkb = [&](int b) { return (blocks[b].c_src + 63) / 64; };
         auto npad = [&](const Cand& c) { return (c.nc * KP + 15) & ~15; };
         auto unit_z = [&](const Cand& c) { return npad(c) * 128 * nkb(c.blk); };
-        auto blk_x = [&](int b) { return blocks[b].d_src * 2048 * nkb(b); };
-        auto nmt = [&](int b) { return (blocks[b].d_src * TB + 127) / 128; };
-        auto unit_cols = [&](const Cand& c) { return nmt(c.blk) * npad(c); };
         auto cand_nz = [&](const Cand& c) {
             int n = 0;
             for (int cl = 0; cl < c.nc; ++cl) {
@@ -569,6 +560,37 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
             }
             return n;
         };
+        // batch size of a set: the largest power of two in 16..128 whose rows d_src * tb fit one 128-row tile
+        auto batch_of = [&](int d_src_max) { int tb = 16; while (tb < 128 && d_src_max * tb * 2 <= 128) tb *= 2; return tb; };
+        struct Par { int tb, x, z, nent, nnz, ncomp, cols, need; };
+        // the launch parameters of the set of candidates [i, j): the largest batch size (at most the one that
+        // fills a 128-row tile) whose shared memory stays within the budget
+        auto eval = [&](size_t i, size_t j, int budget) {
+            int dmax = 0;
+            std::vector<int> blks;
+            for (size_t k = i; k < j; ++k) {
+                dmax = std::max(dmax, blocks[cands[k].blk].d_src);
+                if (std::find(blks.begin(), blks.end(), cands[k].blk) == blks.end()) blks.push_back(cands[k].blk);
+            }
+            Par r{};
+            for (int tb = batch_of(dmax); tb >= 16; tb >>= 1) {
+                r = Par{};
+                r.tb = tb;
+                for (int b : blks) r.x += blocks[b].d_src * r.tb * 128 * nkb(b);
+                for (size_t k = i; k < j; ++k) {
+                    const Cand& c = cands[k];
+                    r.z += unit_z(c); r.nent += c.nc * blocks[c.blk].d_src; r.nnz += cand_nz(c); r.ncomp += c.nc;
+                    r.cols = std::max(r.cols, ((blocks[c.blk].d_src * r.tb + 127) / 128) * npad(c));
+                }
+                // a 128-row MMA tile may read past the rows of a block: what follows in shared memory (the other
+                // copy, the next stage, the Zbar slabs) is at least 16 KiB, hence the floor on the slab size
+                r.x = (r.x + 1023) & ~1023;
+                r.z = std::max(8192, (r.z + 1023) & ~1023);
+                r.need = smem_need(KP, dual, dsh, r.tb, r.x, r.z, r.nent, (int)(j - i), r.ncomp, r.nnz, r.nnz);
+                if (r.need <= budget) break;
+            }
+            return r;
+        };
         // sets: at most `maxu` units each, the largest grouping that fits two CTAs per SM, else one CTA per SM
         for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
             const int attempt = trial / (int)cands.size();
@@ -578,27 +600,15 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
             T = TcSets{};
             bool fits = true;
             size_t i = 0;
-            int maxu_seen = 0;
             while (i < cands.size() && fits) {
-                int z_bytes = 0, x_bytes = 0, nent = 0, nnz = 0;
-                std::vector<int> set_blks;
                 size_t j = i;
-                for (; j < cands.size() && (int)(j - i) < maxu; ++j) {
-                    const Cand& c = cands[j];
-                    const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
-                    const int z2 = z_bytes + unit_z(c), x2 = x_bytes + (new_blk ? blk_x(c.blk) : 0);
-                    const int e2 = nent + c.nc * blocks[c.blk].d_src, n2 = nnz + cand_nz(c);
-                    // a 128-row MMA tile may read past the rows of a block: whatever follows in shared memory (the next
-                    // copy, the next stage, the Zbar slabs) is at least 16 KiB, see the floor on z_cap below
-                    const int xcap = std::max(T.a_cap, (x2 + 1023) & ~1023), zcap = std::max(T.b_cap, std::max(8192, (z2 + 1023) & ~1023));
-                    // (the inverse table of a set has as many terms as its forward table)
-                    const int need = smem_need(KP, dual, p->dim_sh, xcap, zcap, std::max(T.max_ent, e2), std::max(maxu_seen, (int)(j - i) + 1),
-                                               std::max(T.max_nz, n2), std::max(T.max_nz, n2));
-                    if (need > budget || unit_cols(c) > col_budget) break;
-                    z_bytes = z2; x_bytes = x2; nent = e2; nnz = n2;
-                    if (new_blk) set_blks.push_back(c.blk);
+                while (j < cands.size() && (int)(j - i) < maxu) {
+                    const Par r = eval(i, j + 1, budget);
+                    if (r.need > budget || r.cols > col_budget) break;
+                    ++j;
                 }
                 if (j == i) { fits = false; break; }
+                const Par r = eval(i, j, budget);
                 TSet S{};
                 S.unit_begin = (int)T.units.size(); S.blk_begin = (int)T.blks.size(); S.ent_begin = (int)T.ents.size();
                 int z_off = 0, x_off = 0;
@@ -611,8 +621,8 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
                     if (bi < 0) {
                         TBlk tb{};
                         tb.src_off = Bk.so; tb.c_src = Bk.c_src; tb.d_src = Bk.d_src; tb.ncols = 0;
-                        tb.b_off = x_off; tb.slab_bytes = 2048; tb.atom_stride = Bk.d_src * 2048;
-                        x_off += blk_x(c.blk);
+                        tb.b_off = x_off; tb.slab_bytes = r.tb * 128; tb.atom_stride = Bk.d_src * r.tb * 128;
+                        x_off += Bk.d_src * r.tb * 128 * nkb(c.blk);
                         bi = (int)T.blks.size();
                         T.blks.push_back(tb);
                         local_blk.push_back(c.blk);
@@ -626,29 +636,24 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
                         for (int s = 0; s < Bk.d_src; ++s) T.ents.push_back(TEnt{cp.tab0 + s * cp.tstride, cp.sh_off, 0, 0});
                     }
                     z_off += unit_z(c);
-                    T.acc_cols = std::max(T.acc_cols, unit_cols(c));
                     T.units.push_back(U);
                 }
                 S.nunit = (int)T.units.size() - S.unit_begin; S.nblk = (int)T.blks.size() - S.blk_begin;
                 S.nent = (int)T.ents.size() - S.ent_begin;
                 T.sets.push_back(S);
-                T.a_cap = std::max(T.a_cap, (x_off + 1023) & ~1023);                       // x_cap
-                T.b_cap = std::max(T.b_cap, std::max(8192, (z_off + 1023) & ~1023));       // z_cap (two copies >= 16 KiB)
-                T.max_ent = std::max(T.max_ent, S.nent);
-                T.max_nz = std::max(T.max_nz, nnz);
-                maxu_seen = std::max(maxu_seen, S.nunit);
+                int lg = 0; while ((1 << lg) < r.tb) ++lg;
+                int tc = 32; while (tc < 2 * r.cols) tc <<= 1;
+                TcSets::ESetPar ep{};
+                ep.tb = r.tb; ep.lg = lg; ep.x_cap = r.x; ep.z_cap = r.z; ep.smem = r.need; ep.tmem_cols = tc; ep.acc_cols = r.cols;
+                ep.ctas = (r.need <= 113 * 1024 && tc <= 256) ? 2 : 1;
+                ep.nnz = r.nnz; ep.ninv = r.nnz; ep.ncomp = r.ncomp;
+                T.epar.push_back(ep);
+                if (r.need > 227 * 1024 || tc > 512) fits = false;
                 i = j;
             }
             if (!fits) continue;
-            int tc = 32; while (tc < 2 * T.acc_cols) tc <<= 1;
-            T.tmem_cols = tc;
-            T.max_units = maxu_seen;
-            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, T.max_units, T.max_nz, T.max_nz);
-            if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
-            T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
             // shared-memory images of the tables, per set: entries with their sparse terms, the inverse table
             // b -> (entry inside the set, coef), and the components with their group layout resolved
-            const int dsh = p->dim_sh;
             for (TSet& S : T.sets) {
                 S.b_items = (int)T.nz.size();
                 for (int j = 0; j < S.nent; ++j) {
@@ -693,25 +698,28 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     a.zqh = (const __nv_bfloat16*)zqh; a.zql = (const __nv_bfloat16*)zql;
     a.gphi = gphi; a.gY = gY;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
-    a.x_cap = T.a_cap; a.z_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols;
-    a.max_nz = T.max_nz; a.max_inv = T.max_nz; a.max_units = T.max_units;
     a.status = status;
     const bool k8 = p->K <= 8;
     void (*kern)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true> : k_edge_tc<8, false>)
                                     : (dual ? k_edge_tc<16, true> : k_edge_tc<16, false>);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T.smem_bytes);
+    int max_smem = 0;
+    for (const auto& ep : T.epar) max_smem = std::max(max_smem, ep.smem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (e != cudaSuccess) return e;
-    const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * T.ctas_per_sm);
     // one launch per set of accumulator tiles: the first writes in the caller's mode, the others accumulate
     for (size_t si = 0; si < T.sets.size(); ++si) {
         const TSet& S = T.sets[si];
+        const TcSets::ESetPar& ep = T.epar[si];
         a.set = (int)si;
+        a.tb = ep.tb; a.lg = ep.lg; a.x_cap = ep.x_cap; a.z_cap = ep.z_cap; a.nent = S.nent;
+        a.tmem_cols = ep.tmem_cols; a.acc_cols = ep.acc_cols; a.nnz = ep.nnz; a.ninv = ep.ninv; a.nunit = S.nunit; a.ncomp = ep.ncomp;
         a.ents = T.d_ents_s + S.ent_begin; a.nz = T.d_nz + S.b_items;
         a.inv_ptr = T.d_inv_ptr + si * (size_t)(p->dim_sh + 1); a.inv = T.d_inv + T.inv_base[si];
         a.phi_mode = phi_mode ? (si == 0 ? phi_mode : 2) : 0;
         a.Y_mode = Y_mode ? (si == 0 ? Y_mode : 2) : 0;
+        const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * ep.ctas);
         KernelTimer kt(K_EDGE, s);
-        kern<<<grid, TT, T.smem_bytes, s>>>(a);
+        kern<<<grid, TT, ep.smem, s>>>(a);
         count_launch();
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;

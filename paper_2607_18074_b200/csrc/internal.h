@@ -148,6 +148,8 @@ struct TcSets {
     int32_t* d_inv_ptr = nullptr;
     NzS* d_inv = nullptr;
     int32_t max_units = 0;
+    struct ESetPar { int32_t tb, lg, x_cap, z_cap, smem, ctas, tmem_cols, acc_cols, nnz, ninv, ncomp; };
+    std::vector<ESetPar> epar;               // edge pass: launch parameters of every set (one launch per set)
     int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
