@@ -119,9 +119,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     uint8_t* sRing = smem;                                     // stages: Xh Xl raw
     uint8_t* sZ = sRing + (size_t)NS * stage_bytes;            // Zbar slabs of the set: hi, lo
     uint8_t* meta = sZ + (size_t)2 * a.z_cap;
-    float* sM0 = reinterpret_cast<float*>(meta);               // [2][nent][PS] coupling matrices, double buffered
-    float* sdM0 = sM0 + (size_t)2 * a.nent * PS;               // DUAL
-    float* sGM = sdM0 + (DUAL ? (size_t)2 * a.nent * PS : 0);  // [nent][PS]
+    float* sM = reinterpret_cast<float*>(meta);                // [nent][PS] coupling matrices of the batch
+    float* sdM = sM + (size_t)a.nent * PS;                     // DUAL
+    float* sGM = sdM + (DUAL ? (size_t)a.nent * PS : 0);       // [nent][PS]
     float* sPphi = sGM + (size_t)a.nent * PS;                  // [NCW*32][KP]: one row per compute thread
     float* accPhi = sPphi + NCW * 32 * KP;                     // [EG][KP]
     float* accY = accPhi + EG * KP;                            // [EG][dsh]
@@ -366,14 +366,14 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                         const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.x_cap);
                         const float* sYT = raw + NRAW * tb * KP;
                         const float* sVYT = sYT + a.dsh * PS;
-                        float* sM = sM0 + (size_t)(it & 1) * a.nent * PS;
-                        float* sdM = sdM0 + (size_t)(it & 1) * a.nent * PS;
                         // weights of this sub-batch: gM += sum_q aw[q] * D,  gphi[q] += mw * D
                         //   plain: aw = phi, mw = M;   dual, op 0: aw = vphi, mw = dM;   dual, op 1: aw = phi, mw = M
                         float aw[KP];
 #pragma unroll
                         for (int q = 0; q < KP; ++q) aw[q] = (DUAL && op == 0) ? raw[tb * KP + e * KP + q] : raw[e * KP + q];
-                        // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
+                        // ---- coupling matrices of the set, once per batch (both sub-batches share them; the previous
+                        // batch's readers are all past the barrier that follows its epilogue): thread <-> (entry, 8 edges)
+                        if (sb == 0)
                         for (int i = tid; i < S.nent * t8; i += NCW * 32) {
                             const int j = i / t8, o8 = 8 * (i - j * t8);
                             const EntS en = sEnt[j];
@@ -502,7 +502,7 @@ int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent
     const int nop = dual ? 2 : 1;
     const int PS = tb + 4, EG = group_edges(tb);
     const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
-    const size_t meta = (size_t)2 * nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)EG * KP +
+    const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)EG * KP +
                         (size_t)((EG * dsh + 1) & ~1);
     const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
                        (nnz + ninv) * (int)sizeof(NzS) + (dsh + 2) * 4;
@@ -591,10 +591,11 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
             }
             return r;
         };
-        // sets: at most `maxu` units each, the largest grouping that fits two CTAs per SM, else one CTA per SM
-        for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
-            const int attempt = trial / (int)cands.size();
-            const int maxu = (int)cands.size() - trial % (int)cands.size();
+        // sets of at most `maxu` units each: the largest grouping that fits the budget of two CTAs per SM
+        // (attempt 0) or of one CTA per SM (attempt 1)
+        auto pack = [&](int attempt) {
+          TcSets T;
+          for (int maxu = (int)cands.size(); maxu >= 1 && !T.ok; --maxu) {
             const int budget = (attempt == 0 ? 113 : 226) * 1024;
             const int col_budget = attempt == 0 ? 128 : 256;
             T = TcSets{};
@@ -678,7 +679,13 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
             for (const SComp& cp : T.comps)
                 T.comps_s.push_back(CompS{dir.zb_off[cp.group], dir.nk_ld[cp.group], cp.d_dst, cp.o, cp.koff, {0, 0}});
             T.ok = true;
-        }
+          }
+          return T;
+        };
+        // two CTAs per SM hide the latency of the short batches better, unless that takes many more sets (each set
+        // is a launch of its own that stages the edge data again)
+        TcSets T0 = pack(0), T1 = pack(1);
+        T = (T0.ok && (!T1.ok || T0.sets.size() <= T1.sets.size() + 2)) ? T0 : T1;
     }
 }
 
