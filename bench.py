@@ -36,8 +36,8 @@ L2_FLUSH_BYTES = 512 << 20
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from the ncu captures summarised
 # under profiles/ (average over the launches of the class in one step).  Only known for the workload
 # that was captured.
-NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 144.0e6, ("cfg2", "edge_pass"): 82.0e6,
-                     ("cfg2", "node_gemm"): 26.6e6}
+NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 144.0e6, ("cfg2", "edge_pass"): 137.0e6,
+                     ("cfg2", "node_gemm"): 48.4e6}
 
 
 def measured_peaks():

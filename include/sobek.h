@@ -84,7 +84,10 @@ enum { SOBEK_MAX_L = 4 };
  * the radial embedding.  `flags` must be 0.  If the environment variable SOBEK_FUSED is set to a
  * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
  * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise
- * by the stream -> bounded state -> GEMM schedule, which is the faster one at present.
+ * by the stream -> bounded state -> GEMM schedule, which is the faster one at present.  In that schedule
+ * the edge stream and the edge pass run on the tensor cores where the profile allows it (multiplicities
+ * that are multiples of 8 / 16, at most 128, K <= 16); SOBEK_TC_STREAM=0 / SOBEK_TC_EDGE=0 at plan
+ * creation select the FP32-pipe kernels instead (same results within the tolerances).
  * Errors: INVALID_ARG (null, mul < 1, parity not +-1, K < 1), UNSUPPORTED (l or l_max >
  * SOBEK_MAX_L, or no valid path), CUDA.
  */
