@@ -538,8 +538,10 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         }
         std::sort(blocks.begin(), blocks.end(), [](const Blk& x, const Blk& y) { return x.so < y.so; });
         struct Cand { int blk, c0, nc; };
+        // accumulator tiles of up to 16 components (128 columns at K <= 8, 256 above); if the wide tiles of a
+        // K > 8 profile do not fit shared memory, tiles of 8 components
+        for (int comps_per_tile = 16; comps_per_tile >= 128 / KP && !T.ok; comps_per_tile >>= 1) {
         std::vector<Cand> cands;
-        const int comps_per_tile = 128 / KP;
         for (size_t b = 0; b < blocks.size(); ++b) {
             const int nc = (int)blocks[b].comps.size();
             const int ntile = (nc + comps_per_tile - 1) / comps_per_tile;
@@ -686,6 +688,7 @@ void build_tc_edge_sets(const sobek_plan* p, Direction& dir) {
         // is a launch of its own that stages the edge data again)
         TcSets T0 = pack(0), T1 = pack(1);
         T = (T0.ok && (!T1.ok || T0.sets.size() <= T1.sets.size() + 2)) ? T0 : T1;
+        }   // tile widths
     }
 }
 
