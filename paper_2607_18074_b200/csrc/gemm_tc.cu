@@ -43,6 +43,7 @@ struct TcArgs {
     int64_t M, N, Kd;
     int32_t BN;                 // tile width (multiple of 16, <= 256)
     int32_t stages;
+    int32_t ring_bytes;         // bytes of the operand ring = what the epilogue may use as its staging area
     int32_t tmem_cols;          // power of two >= max(32, BN)
     int32_t mn_major;           // 0: A[M,Kd], B[N,Kd] row-major;  1: A^T[Kd,M], B^T[Kd,N] row-major
     int32_t splits;             // gridDim.z: the contraction range is cut into this many pieces,
@@ -59,7 +60,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
     const uint32_t a_bytes = BM * BK * 2;             // 16 KiB
     const uint32_t b_bytes = (uint32_t)g.BN * BK * 2;
     const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;
-    uint64_t* bars = (uint64_t*)(smem + (size_t)g.stages * stage_bytes);
+    uint64_t* bars = (uint64_t*)(smem + (size_t)g.ring_bytes);
     // bars[0..S) full, bars[S..2S) empty, bars[2S] accumulator ready; then the TMEM base word
     uint32_t* tmem_holder = (uint32_t*)(bars + 2 * g.stages + 1);
     const uint32_t sbase = smem_u32(smem);
@@ -318,14 +319,19 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
     g.splits = std::max(1, std::min<int>(splits, (int)((Kd + BK - 1) / BK))); g.split_stride = split_stride;
     int BN;
+    const int num_kb = (int)((Kd + BK - 1) / BK);
     if (mn_major) BN = N <= 64 ? 64 : (N <= 128 ? 128 : 256);     // whole 64-wide boxes
-    else BN = (int)std::min<int64_t>(256, (N + 15) / 16 * 16);
+    else BN = (int)std::min<int64_t>(num_kb == 1 ? 128 : 256, (N + 15) / 16 * 16);   // a single k-block is all epilogue: narrower tiles, more CTAs
     g.BN = BN;
     const size_t stage = 2 * (size_t)BM * BK * 2 + 2 * (size_t)BN * BK * 2;
-    // two CTAs per SM where two stages of the ring fit twice (more loads in flight per SM), else one CTA with a deeper ring
+    // two (or more) CTAs per SM where the ring fits twice (more loads and epilogues in flight per SM), else one
+    // CTA with a deeper ring; never more stages than k-blocks
     int stages = (int)std::min<size_t>(4, (108 * 1024) / stage);
     if (stages < 2) stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
-    g.stages = std::max(stages, 2);
+    stages = std::max(1, std::min(stages, (num_kb + g.splits - 1) / g.splits));
+    g.stages = stages;
+    const size_t park = (size_t)4 * 32 * (BN + 1) * sizeof(float);       // epilogue staging of the four drain warps
+    g.ring_bytes = (int32_t)((std::max(park, (size_t)stages * stage) + 1023) & ~size_t(1023));
     int cols = 32;
     while (cols < BN) cols <<= 1;
     g.tmem_cols = cols;
@@ -339,7 +345,7 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
              make_map(&tBh, Bhi, N, Kd, ldb, 64, BK) && make_map(&tBl, Blo, N, Kd, ldb, 64, BK);
     }
     if (!ok) return cudaErrorInvalidValue;
-    const size_t sh = (size_t)g.stages * stage + 1024 + 8 * (2 * g.stages + 1) + 16;
+    const size_t sh = (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
