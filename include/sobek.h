@@ -157,7 +157,7 @@ int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const in
 
 /*
  * Workspace needed by one call of the given order (0 = fwd, 1 = bwd, 2 = dbwd).  It holds
- * re-laid-out copies of R, the bounded receiver/sender state of one node chunk (at most 1 GiB,
+ * re-laid-out copies of R, the bounded receiver/sender state of one node chunk (at most 2 GiB,
  * whatever the graph), a status word and, for the tensor-core edge kernels, bf16 (hi, lo)
  * copies of the node features they gather from (4 bytes per feature of x, and of gy / vx for
  * orders 1 / 2).  It depends on the plan and on N only -- never on E.

@@ -249,7 +249,7 @@ namespace sobek {
 // bytes reserved at the start of every workspace for the device status word
 constexpr size_t kHeaderBytes = 256;
 // budget for the bounded node-state buffer (floats of Z / V held at once)
-constexpr size_t kStateBudgetBytes = size_t(1024) << 20;
+constexpr size_t kStateBudgetBytes = size_t(2048) << 20;
 constexpr int64_t kMinChunkNodes = 512;
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);

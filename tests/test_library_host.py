@@ -89,13 +89,13 @@ def test_workspace_does_not_grow_with_edges():
         per_node = 4 * (C_x + (C_y if order >= 1 else 0) + (C_x if order >= 2 else 0))
         grow = sb.workspace_bytes(plan, 3 * 10**6, 10**8, order) - sb.workspace_bytes(plan, 10**6, 10**8, order)
         assert abs(grow - 2 * 10**6 * per_node) < 4096
-        assert sb.workspace_bytes(plan, 10**6, 10**8, order) - 10**6 * per_node < 2200 * 2**20
-    # the widest benchmark contract: bounded by 512 nodes of state plus the feature copies, whatever the edge count
+        assert sb.workspace_bytes(plan, 10**6, 10**8, order) - 10**6 * per_node < 4300 * 2**20
+    # the widest benchmark contract: bounded by the state budget (or 512 nodes) plus the feature copies, whatever the edge count
     w = synth.config("cfg5")
     plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
     a = sb.workspace_bytes(plan, 50000, 2 * 10**6, 2)
     assert a == sb.workspace_bytes(plan, 50000, 4 * 10**8, 2)
-    assert a - 50000 * 4 * (2 * plan.info.C_x + plan.info.C_y) < 2800 * 2**20
+    assert a - 50000 * 4 * (2 * plan.info.C_x + plan.info.C_y) < 5400 * 2**20
 
 
 def test_argument_errors_are_status_codes():
