@@ -120,12 +120,12 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
 
 // (hi, lo) bf16 split of two floats: hi pair, lo pair (element 0 in the low half)
 __device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo) {
-    // hi = the upper 16 bits of each float (bf16 by truncation), lo = bf16 of the exact remainder, again by truncation
-    const uint32_t ua = __float_as_uint(a), ub = __float_as_uint(b);
-    hi = __byte_perm(ua, ub, 0x7632);
-    const float ra = a - __uint_as_float(ua & 0xffff0000u);
-    const float rb = b - __uint_as_float(ub & 0xffff0000u);
-    lo = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    const float ra = a - __uint_as_float(hi << 16);
+    const float rb = b - __uint_as_float(hi & 0xffff0000u);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(ra, rb);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 __device__ __forceinline__ void split8(const float* p, uint4& h, uint4& l) {
     split2(p[0], p[1], h.x, l.x);
