@@ -25,6 +25,11 @@ def small_cases():
     c["ragged"] = synth.Workload("ragged", P("5x0e+3x1o+2x1e+33x2e"), P("7x0e+1x0o+35x1o+2x2e+3x3o+2x4e"),
                                  3, 3, 40, 4.0, 1.9, "gaussian", seed=3)
     c["K20"] = synth.Workload("K20", P("6x0e+4x1o"), P("6x0e+4x1o+2x2e"), 2, 20, 50, 4.0, 1.8, "bessel", seed=4)
+    # tensor-core kernels off their main path: K below the padded width (and not a multiple of 4), multiplicities
+    # that are multiples of 16 but not of 32, and receivers with well over 64 / 128 edges (several output groups)
+    c["tc_K6_dense"] = synth.Workload("tc_K6_dense", P("16x0e+16x1o"), P("16x0e+16x1o+16x2e"), 2, 6, 160, 4.0, 3.6,
+                                      "gaussian", seed=5)
+    c["tc_K12"] = synth.Workload("tc_K12", P("48x0e+16x1o+16x2e"), P("16x0e+48x1o"), 2, 12, 70, 4.0, 2.2, "bessel", seed=6)
     return c
 
 
