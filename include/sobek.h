@@ -88,6 +88,10 @@ enum { SOBEK_MAX_L = 4 };
  * the edge stream and the edge pass run on the tensor cores where the profile allows it (multiplicities
  * that are multiples of 8 / 16, at most 128, K <= 16); SOBEK_TC_STREAM=0 / SOBEK_TC_EDGE=0 at plan
  * creation select the FP32-pipe kernels instead (same results within the tolerances).
+ * SOBEK_STATE_BUDGET_MB (an integer number of MiB, default 2048) at plan creation sets the scratch
+ * budget (section "Runtime scratch-budget policy"; the paper measures with 128 MiB): the bytes of receiver (or sender) state held at once.  Nodes
+ * are processed in chunks that fit the budget, but never fewer than 512 at a time; the results do not
+ * depend on the budget beyond the summation order of gR / hR across chunks.
  * Errors: INVALID_ARG (null, mul < 1, parity not +-1, K < 1), UNSUPPORTED (l or l_max >
  * SOBEK_MAX_L, or no valid path), CUDA.
  */

@@ -234,6 +234,7 @@ struct sobek_plan {
     int device = -1;
     bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
     bool use_tc_edge = true;     // edge pass on the tensor cores where the profile allows it
+    size_t state_budget = size_t(2048) << 20;   // bytes of receiver / sender state held at once (the scratch budget)
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -249,7 +250,6 @@ namespace sobek {
 // bytes reserved at the start of every workspace for the device status word
 constexpr size_t kHeaderBytes = 256;
 // budget for the bounded node-state buffer (floats of Z / V held at once)
-constexpr size_t kStateBudgetBytes = size_t(2048) << 20;
 constexpr int64_t kMinChunkNodes = 512;
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order);

@@ -374,7 +374,7 @@ int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order) {
     per = std::max<int64_t>(per, 1);
     // the budget bounds the chunk, but a chunk never has fewer than kMinChunkNodes nodes: below that the
     // node-side kernels cannot fill the machine
-    int64_t n = (int64_t)(kStateBudgetBytes / (size_t)per);
+    int64_t n = (int64_t)(p->state_budget / (size_t)per);
     n = std::max<int64_t>(n, kMinChunkNodes);
     return std::min<int64_t>(std::max<int64_t>(N, 1), n);
 }
@@ -444,6 +444,10 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         for (double& v : p->paths[k].cg) v *= nrm;
     }
     if (const char* e = getenv("SOBEK_FUSED")) p->use_fused = atoi(e) != 0;
+    if (const char* e = getenv("SOBEK_STATE_BUDGET_MB")) {
+        const long mb = atol(e);
+        if (mb >= 1 && mb <= (1L << 20)) p->state_budget = size_t(mb) << 20;
+    }
     build_direction(p, 0, p->fwd);
     build_direction(p, 1, p->tr);
     build_stream_tasks(p, p->fwd);

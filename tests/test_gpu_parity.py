@@ -283,3 +283,81 @@ def test_sender_view_without_receiver_ids(cases):
     gx = torch.full((c.N, c.plan.info.C_x), float("nan"), dtype=torch.float32, device="cuda:0")
     sb.conv_bwd(c.plan, g, c.x, c.Y, c.phi, c.R, c.gy, gx, None, None, None, c.ws(1))
     assert rel_err(gx.cpu().numpy(), c.o_bwd()[0]) <= BWD_TOL
+
+
+# ---------------------------------------------------------------------------------------
+# the paper's scaling axes (section "Scaling axes"): long neighbourhoods, many small graphs
+# ---------------------------------------------------------------------------------------
+AXES = {
+    "deg_4": (6, (0, 1, 2)),         # mean degree 4: isolated receivers and receivers with one edge
+    "deg_1023": (2, (0, 1, 2)),      # 341 ... 1850 edges per receiver (dozens of edge batches each)
+    "graphs_31": (6, (0, 1, 2)),     # one 128-node graph repeated 31 times
+}
+
+
+@pytest.mark.parametrize("name", list(AXES))
+def test_scaling_axes_sampled(name):
+    n_sample, orders = AXES[name]
+    FULL[name] = (synth.config(name), n_sample, orders)
+    try:
+        test_full_size_sampled(name)
+    finally:
+        del FULL[name]
+
+
+def test_scratch_budget(monkeypatch):
+    """The scratch budget (section "Runtime scratch-budget policy") only changes the chunking: with the
+    paper's 128 MiB the workspace shrinks and every output still matches the oracle."""
+    import paper_2607_18074_b200 as sb
+    w = synth.scaled(synth.config("cfg4", edges=1e5), 1500)
+    big = Case(w)
+    monkeypatch.setenv("SOBEK_STATE_BUDGET_MB", "128")
+    small = Case(w, inputs=big.d)
+    monkeypatch.delenv("SOBEK_STATE_BUDGET_MB")
+    for order in (0, 1, 2):
+        assert sb.workspace_bytes(small.plan, w.N, small.E, order) < sb.workspace_bytes(big.plan, w.N, big.E, order)
+    rng = np.random.default_rng(5)
+    act = np.unique(np.concatenate([[0, big.N - 1], rng.choice(big.N, size=6, replace=False)]))
+    ed = big.edges_into(act)
+    assert rel_err(small.fwd()[act], big.o_fwd(act)[act]) <= FWD_TOL
+    assert np.array_equal(small.fwd(), big.fwd())            # the forward does not depend on the chunking at all
+    got = small.bwd(gy=small.masked_gy(act))
+    ref = big.o_bwd(act)
+    assert rel_err(got[0], ref[0]) <= BWD_TOL and rel_err(got[3], ref[3]) <= BWD_TOL
+    assert rel_err(got[1][ed], ref[1][ed]) <= BWD_TOL and rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL
+    got = small.dbwd(gy=small.masked_gy(act))
+    ref = big.o_dbwd(act)
+    assert rel_err(got[0][act], ref[0][act]) <= BWD_TOL
+    assert rel_err(got[1], ref[1]) <= BWD_TOL and rel_err(got[4], ref[4]) <= BWD_TOL
+    assert rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL and rel_err(got[3][ed], ref[3][ed]) <= BWD_TOL
+
+
+def test_cuda_graph_capture(cases):
+    """A call neither allocates nor synchronises, and its side streams fork from and join the caller's
+    stream with events, so the three orders can be captured into one CUDA graph and replayed."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    c = get(cases, "cfg2_N200")
+    i = c.plan.info
+    eager = [c.fwd()] + c.bwd() + c.dbwd()
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    y = new(c.N, i.C_y)
+    gx, gY, gphi, gR = new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)
+    ggy, hx, hY, hphi, hR = new(c.N, i.C_y), new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)
+    ws = c.ws(2)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sb.conv_fwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, y, ws)
+        sb.conv_bwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, gx, gY, gphi, gR, ws)
+        sb.conv_dbwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, c.vx, c.vY, c.vphi, c.vR,
+                     ggy, hx, hY, hphi, hR, ws)
+    outs = (y, gx, gY, gphi, gR, ggy, hx, hY, hphi, hR)
+    for _ in range(2):
+        for t in outs:
+            t.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert sb.last_device_status(ws) == 0
+        for got, ref in zip(outs, eager):
+            assert np.array_equal(got.cpu().numpy(), ref)

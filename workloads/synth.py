@@ -170,6 +170,7 @@ class Workload:
     orders: tuple = (0, 1, 2)
     seed: int = 0
     note: str = ""
+    copies: int = 1  # the graph of N nodes repeated this many times (disjoint copies, one batch)
 
 
 def _cube(N, rho):
@@ -205,6 +206,23 @@ def config(name: str, **kw) -> Workload:
         N = 50000
         L = _cube(N, 0.1)
         return Workload("cfg5", ir, ir, 4, 16, N, L, cutoff_for_edges(N, 40.0 * N, L), "bessel")
+    if name.startswith("deg_") or name.startswith("graphs_"):
+        # the paper's two scaling axes (section "Scaling axes"), on its 128/64/64 profile with K = 16:
+        # longer neighbourhoods on 2,048 nodes, or one 128-node graph of mean degree 32 repeated B times
+        ir = P("128x0e+64x1o+64x2e")
+        v = int(name.split("_")[1])
+        if name.startswith("deg_"):
+            N, deg, copies = 2048, float(v), 1
+        else:
+            N, deg, copies = 128, 32.0, v
+        L = _cube(N, 0.1)
+        # cutoff from the realised positions (same seeded draw as make_inputs), so that the mean degree is exact
+        pos = L * np.random.default_rng(np.random.SeedSequence(0).spawn(8)[0]).random((N, 3))
+        iu = np.triu_indices(N, 1)
+        dist = np.sort(np.linalg.norm(pos[iu[0]] - pos[iu[1]], axis=1))
+        n_pairs = min(int(round(deg * N / 2)), dist.size - 1)
+        r_c = 0.5 * (dist[n_pairs - 1] + dist[n_pairs])
+        return Workload(name, ir, ir, 2, 16, N, L, float(r_c), "bessel", copies=copies)
     raise KeyError(name)
 
 
@@ -252,6 +270,15 @@ def make_inputs(w: Workload, col_std: np.ndarray, dtype=np.float32,
     s_pos, s_x, s_R, s_gy, s_vx, s_vY, s_vphi, s_vR = [np.random.default_rng(s) for s in ss.spawn(8)]
     pos = w.L * s_pos.random((w.N, 3))
     row_ptr, col, recv = radius_graph(pos, w.r_c)
+    if w.copies > 1:
+        # disjoint copies of the same graph: node ids of copy b are shifted by b * N
+        n1, e1, B = w.N, int(col.shape[0]), int(w.copies)
+        shift = (np.arange(B, dtype=np.int64) * n1)[:, None]
+        col = (col[None, :].astype(np.int64) + shift).reshape(-1).astype(np.int32)
+        recv = (recv[None, :].astype(np.int64) + shift).reshape(-1).astype(np.int32)
+        row_ptr = np.concatenate([[0], (row_ptr[None, 1:] + (np.arange(B, dtype=np.int64) * e1)[:, None]).reshape(-1)])
+        pos = np.tile(pos, (B, 1))
+    N_tot = w.N * max(1, int(w.copies))
     E = int(col.shape[0])
     rij = pos[col] - pos[recv]
     r = np.linalg.norm(rij, axis=1)
@@ -261,17 +288,17 @@ def make_inputs(w: Workload, col_std: np.ndarray, dtype=np.float32,
     else:
         phi = bessel_basis(r, w.K, w.r_c)
     C_x, C_y = irreps_dim(w.irreps_in), irreps_dim(w.irreps_out)
-    x = s_x.standard_normal((w.N, C_x))
+    x = s_x.standard_normal((N_tot, C_x))
     R = s_R.standard_normal((w.K, N_w)) * col_std[None, :]
     vR = s_vR.standard_normal((w.K, N_w)) * col_std[None, :]
-    gy = s_gy.standard_normal((w.N, C_y))
+    gy = s_gy.standard_normal((N_tot, C_y))
     dsh = (w.l_max + 1) ** 2
     if with_cotangents:
-        vx = s_vx.standard_normal((w.N, C_x))
+        vx = s_vx.standard_normal((N_tot, C_x))
         vY = s_vY.standard_normal((E, dsh))
         vphi = s_vphi.standard_normal((E, w.K))
     else:
         vx = np.zeros((0, C_x)); vY = np.zeros((0, dsh)); vphi = np.zeros((0, w.K))
     c = lambda a: np.ascontiguousarray(a.astype(dtype))
-    return Inputs(w, w.N, E, row_ptr, col, recv, c(x), c(Y), c(phi), c(R), c(gy), c(vx), c(vY),
+    return Inputs(w, N_tot, E, row_ptr, col, recv, c(x), c(Y), c(phi), c(R), c(gy), c(vx), c(vY),
                   c(vphi), c(vR), pos)
