@@ -56,23 +56,25 @@ def _d(a):
 
 
 class Oracle:
-    def __init__(self, irreps_in, irreps_out, l_max: int, K: int):
+    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, mode: str = "uvw"):
         self.irreps_in, self.irreps_out, self.l_max, self.K = list(irreps_in), list(irreps_out), l_max, K
-        self.paths, self.N_w = tables.enumerate_paths(irreps_in, irreps_out, l_max)
+        self.mode = mode   # "uvw" (Eq. uvw_connection) or "uvu" (Eq. uvu_connection)
+        self.paths, self.N_w = tables.enumerate_paths(irreps_in, irreps_out, l_max, mode)
         self.C_x = sum(c * (2 * l + 1) for c, l, _ in irreps_in)
         self.C_y = sum(c * (2 * l + 1) for c, l, _ in irreps_out)
         self.dsh = (l_max + 1) ** 2
         rows, cg, off = [], [], 0
         for p in self.paths:
             di, ds, do = 2 * p.l_in + 1, 2 * p.l_sh + 1, 2 * p.l_out + 1
-            rows.append([p.in_off, p.c_in, di, p.sh_off, ds, p.out_off, p.c_out, do, p.w_off, off])
+            rows.append([p.in_off, p.c_in, di, p.sh_off, ds, p.out_off, p.c_out, do, p.w_off, off,
+                         1 if mode == "uvu" else 0])
             cg.append(p.cg.ravel())
             off += di * ds * do
-        self._P = np.ascontiguousarray(np.array(rows, dtype=np.int64).reshape(-1, 10))
+        self._P = np.ascontiguousarray(np.array(rows, dtype=np.int64).reshape(-1, 11))
         self._cg = np.ascontiguousarray(np.concatenate(cg)) if cg else np.zeros(1)
 
     def col_std(self):
-        return tables.weight_col_std(self.irreps_in, self.irreps_out, self.l_max, self.K)
+        return tables.weight_col_std(self.irreps_in, self.irreps_out, self.l_max, self.K, self.mode)
 
     # -- helpers ------------------------------------------------------------
     def _graph(self, row_ptr, col, act):
@@ -133,8 +135,12 @@ class Oracle:
             C = np.einsum("abo,eau,eb->euo", p.cg, xs, Ys)            # angular contraction
             S = np.zeros((N, self.K, p.c_in, do))
             np.add.at(S, recv, phi[:, :, None, None] * C[:, None, :, :])  # receiver state
-            A = R[:, p.w_off:p.w_off + p.c_in * p.c_out].reshape(self.K, p.c_in, p.c_out)
-            m = np.einsum("iquo,quw->iow", S, A)                        # channel mixing
+            if self.mode == "uvu":
+                A = R[:, p.w_off:p.w_off + p.c_in]
+                m = np.einsum("iquo,qu->iou", S, A)                     # tied channels: no mixing
+            else:
+                A = R[:, p.w_off:p.w_off + p.c_in * p.c_out].reshape(self.K, p.c_in, p.c_out)
+                m = np.einsum("iquo,quw->iow", S, A)                    # channel mixing
             y[:, p.out_off:p.out_off + do * p.c_out] += m.reshape(N, -1)
         return y
 

@@ -21,6 +21,10 @@
  * Layouts: features [N, C] in ir_mul order (block offset + m*mult + u); Y [E, dsh];
  * phi [E, K]; A [K, N_w] with column w_off(pi) + u*C_out + w.
  *
+ * Channelwise mode (Eq. uvu_connection): a path marked `tied` couples input multiplicity u
+ * only to output multiplicity u (C_out = C_in) and owns C_in weights, column w_off(pi) + u.
+ * Every loop over the output multiplicity w below then runs over the single value w = u.
+ *
  * Every routine works on a list of ACTIVE RECEIVERS: only edges into those nodes are
  * visited.  With the full list this is the whole operator; with a sample it gives the
  * rows of y / the edge outputs for that sample, and the node/parameter adjoints that
@@ -34,8 +38,15 @@
 #endif
 
 typedef struct {
-    int64_t in_off, c_in, d_in, sh_off, d_sh, out_off, c_out, d_out, w_off, cg_off;
+    int64_t in_off, c_in, d_in, sh_off, d_sh, out_off, c_out, d_out, w_off, cg_off, tied;
 } opath;
+
+/* range of output multiplicities coupled to input multiplicity u, and the weight column of (u, w) */
+static int64_t w_lo(const opath* p, int64_t u) { return p->tied ? u : 0; }
+static int64_t w_hi(const opath* p, int64_t u) { return p->tied ? u + 1 : p->c_out; }
+static int64_t w_col(const opath* p, int64_t u, int64_t w) {
+    return p->tied ? p->w_off + u : p->w_off + u * p->c_out + w;
+}
 
 static int nthreads(void) {
 #ifdef _OPENMP
@@ -101,8 +112,8 @@ void oracle_fwd(int64_t n_act, const int64_t* act, const int64_t* row_ptr, const
                     const opath* p = P + k;
                     angular(p, cg, x + j * C_x + p->in_off, Y + e * dsh + p->sh_off, t);
                     for (int64_t u = 0; u < p->c_in; ++u)
-                        for (int64_t w = 0; w < p->c_out; ++w) {
-                            const double Wuw = W[p->w_off + u * p->c_out + w];
+                        for (int64_t w = w_lo(p, u); w < w_hi(p, u); ++w) {
+                            const double Wuw = W[w_col(p, u, w)];
                             for (int64_t o = 0; o < p->d_out; ++o)
                                 M[p->out_off + o * p->c_out + w] += Wuw * t[u * p->d_out + o];
                         }
@@ -156,15 +167,15 @@ void oracle_bwd(int64_t n_act, const int64_t* act, const int64_t* row_ptr, const
                         /* h = <mbar_i, T_{pi,(u,w)}>  and  s = sum_w W mbar (weighted adjoint
                            of the angular contraction) */
                         for (int64_t o = 0; o < p->d_out; ++o) s[u * p->d_out + o] = 0.0;
-                        for (int64_t w = 0; w < p->c_out; ++w) {
+                        for (int64_t w = w_lo(p, u); w < w_hi(p, u); ++w) {
                             double acc = 0.0;
-                            const double Wuw = W[p->w_off + u * p->c_out + w];
+                            const double Wuw = W[w_col(p, u, w)];
                             for (int64_t o = 0; o < p->d_out; ++o) {
                                 const double g = gyi[p->out_off + o * p->c_out + w];
                                 acc += g * t[u * p->d_out + o];
                                 s[u * p->d_out + o] += Wuw * g;
                             }
-                            h[p->w_off + u * p->c_out + w] = acc;
+                            h[w_col(p, u, w)] = acc;
                         }
                         /* operand adjoints: D_x T^* and D_Y T^* applied to s */
                         for (int64_t a = 0; a < p->d_in; ++a) {
@@ -263,8 +274,8 @@ void oracle_dbwd(int64_t n_act, const int64_t* act, const int64_t* row_ptr, cons
                             s[u * p->d_out + o] = 0.0;
                             ds[u * p->d_out + o] = 0.0;
                         }
-                        for (int64_t w = 0; w < p->c_out; ++w) {
-                            const int64_t n = p->w_off + u * p->c_out + w;
+                        for (int64_t w = w_lo(p, u); w < w_hi(p, u); ++w) {
+                            const int64_t n = w_col(p, u, w);
                             double a0 = 0.0, a1 = 0.0;
                             for (int64_t o = 0; o < p->d_out; ++o) {
                                 const int64_t yo = p->out_off + o * p->c_out + w;

@@ -123,10 +123,14 @@ class Path:
                 f"l={self.l_out}, {self.c_in}x{self.c_out} @ {self.w_off})")
 
 
-def enumerate_paths(irreps_in, irreps_out, l_max: int):
+def enumerate_paths(irreps_in, irreps_out, l_max: int, mode: str = "uvw"):
     """All (input irrep, SH order, output irrep) triples allowed by
     Eq. cg_selection_rules; SH irreps are one copy per order with parity (-1)^l.
-    Returns (paths, N_w)."""
+    mode "uvw": C_in*C_out weights per path (Eq. uvw_connection); mode "uvu": the output
+    multiplicity is tied to the input one, C_in weights per path (Eq. uvu_connection), and
+    a path between blocks of different multiplicity is an error.  Returns (paths, N_w)."""
+    if mode not in ("uvw", "uvu"):
+        raise ValueError(mode)
     in_offs, o = [], 0
     for c, l, p in irreps_in:
         in_offs.append(o)
@@ -147,7 +151,12 @@ def enumerate_paths(irreps_in, irreps_out, l_max: int):
                     p.in_off, p.sh_off, p.out_off = in_offs[ii], ls * ls, out_offs[io]
                     p.w_off = w_off
                     p.cg = path_cg(li, ls, lo)
-                    w_off += ci * co
+                    if mode == "uvu":
+                        if ci != co:
+                            raise ValueError("uvu needs equal input and output multiplicity on every path")
+                        w_off += ci
+                    else:
+                        w_off += ci * co
                     paths.append(p)
     return paths, w_off
 
@@ -156,18 +165,19 @@ def n_weights_uvu(irreps_in, irreps_out, l_max: int) -> int:
     """Weight count of the channelwise mode (Eq. uvu_connection): C_in per path,
     paths restricted to equal input/output multiplicity blocks.  Used only to pin
     the path enumeration against the counts the paper prints for that mode."""
-    paths, _ = enumerate_paths(irreps_in, irreps_out, l_max)
-    return sum(p.c_in for p in paths)
+    return enumerate_paths(irreps_in, irreps_out, l_max, "uvu")[1]
 
 
-def weight_col_std(irreps_in, irreps_out, l_max: int, K: int) -> np.ndarray:
+def weight_col_std(irreps_in, irreps_out, l_max: int, K: int, mode: str = "uvw") -> np.ndarray:
     """Per-column standard deviation 1/sqrt(fan_in) for drawing R, with
-    fan_in = K * (sum of input multiplicities over the paths into that output block)."""
-    paths, n_w = enumerate_paths(irreps_in, irreps_out, l_max)
+    fan_in = K * (sum of input multiplicities over the paths into that output block); in the
+    channelwise mode an output channel is fed by one channel per path: fan_in = K * (paths into the block)."""
+    paths, n_w = enumerate_paths(irreps_in, irreps_out, l_max, mode)
     fan = {}
     for p in paths:
-        fan[p.i_out] = fan.get(p.i_out, 0) + p.c_in
+        fan[p.i_out] = fan.get(p.i_out, 0) + (1 if mode == "uvu" else p.c_in)
     std = np.zeros(n_w)
     for p in paths:
-        std[p.w_off:p.w_off + p.c_in * p.c_out] = 1.0 / math.sqrt(K * fan[p.i_out])
+        n = p.c_in if mode == "uvu" else p.c_in * p.c_out
+        std[p.w_off:p.w_off + n] = 1.0 / math.sqrt(K * fan[p.i_out])
     return std

@@ -268,3 +268,106 @@ def test_empty_receivers_self_loops_duplicates():
     Ysame = Y.copy(); Ysame[2] = Y[1]; phis = phi.copy(); phis[2] = phi[1]
     phi2[1] *= 2
     assert np.allclose(o.fwd(row_ptr, col, x, Ysame, phis, R), o.fwd(rp2, cl2, x, Y2, phi2, R), atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# channelwise (uvu) mode, Eq. uvu_connection
+# ---------------------------------------------------------------------------------------
+UVU_CASES = [
+    (P("3x0e+3x1o"), 1, 3),
+    (P("2x0e+2x1o+2x2e"), 2, 2),
+]
+
+
+def _uvu_pair(ir, l_max, K, seed=2):
+    """A uvu oracle, a uvw oracle on the same irreps, inputs for the first, and the map that embeds
+    the tied weights on the diagonal of the fully connected ones: A[q, pi, u, w] = delta_uw a[q, pi, u]."""
+    w = synth.Workload("t", ir, ir, l_max, K, 7, 1.0, 0.75, "gaussian", seed=seed)
+    try:
+        ou = conv.Oracle(ir, ir, l_max, K, mode="uvu")
+    except ValueError:
+        return None
+    ow = conv.Oracle(ir, ir, l_max, K)
+    inp = synth.make_inputs(w, ou.col_std(), dtype=np.float64)
+
+    def embed(a):
+        A = np.zeros((K, ow.N_w))
+        for pu, pw in zip(ou.paths, ow.paths):
+            for u in range(pu.c_in):
+                A[:, pw.w_off + u * pw.c_out + u] = a[:, pu.w_off + u]
+        return A
+
+    def diag(A):
+        a = np.zeros((K, ou.N_w))
+        for pu, pw in zip(ou.paths, ow.paths):
+            for u in range(pu.c_in):
+                a[:, pu.w_off + u] = A[:, pw.w_off + u * pw.c_out + u]
+        return a
+
+    return ou, ow, inp, embed, diag
+
+
+def test_uvu_rejects_unequal_multiplicities():
+    with pytest.raises(ValueError):
+        conv.Oracle(P("2x0e+3x1o"), P("2x0e+3x1o"), 1, 2, mode="uvu")     # 0e x 1o -> 1o couples 2 with 3
+    with pytest.raises(ValueError):
+        conv.Oracle(P("2x0e+3x1o"), P("2x0e+3x1o+1x2e"), 2, 2, mode="uvu")
+    conv.Oracle(P("3x0e+3x1o"), P("3x0e+3x1o"), 1, 2, mode="uvu")
+
+
+@pytest.mark.parametrize("case", UVU_CASES)
+def test_uvu_is_uvw_with_diagonal_weights(case):
+    """The tied mode is the fully connected one restricted to weights that vanish off the diagonal u = w
+    (Eqs. uvw_connection, uvu_connection): all three orders must agree, with the weight adjoints read off the
+    diagonal.  This pins the uvu oracle to the uvw oracle, which the tests above pin independently."""
+    ir, l_max, K = case
+    ou, ow, d, embed, diag = _uvu_pair(ir, l_max, K)
+    assert ou.N_w == sum(p.c_in for p in ou.paths) and len(ou.paths) == len(ow.paths)
+    A, vA = embed(d.R), embed(d.vR)
+    g = (d.row_ptr, d.col, d.x, d.Y, d.phi)
+    assert np.allclose(ou.fwd(*g, d.R), ow.fwd(*g, A), rtol=1e-12, atol=1e-13)
+    bu, bw = ou.bwd(*g, d.R, d.gy), ow.bwd(*g, A, d.gy)
+    for a, b in zip(bu[:3], bw[:3]):
+        assert np.allclose(a, b, rtol=1e-12, atol=1e-13)
+    assert np.allclose(bu[3], diag(bw[3]), rtol=1e-12, atol=1e-13)
+    du = ou.dbwd(*g, d.R, d.gy, d.vx, d.vY, d.vphi, d.vR)
+    dw = ow.dbwd(*g, A, d.gy, d.vx, d.vY, d.vphi, vA)
+    for a, b in zip(du[:4], dw[:4]):
+        assert np.allclose(a, b, rtol=1e-12, atol=1e-13)
+    assert np.allclose(du[4], diag(dw[4]), rtol=1e-12, atol=1e-13)
+    assert np.abs(du[0]).max() > 1e-3 and np.abs(du[4]).max() > 1e-3
+
+
+@pytest.mark.parametrize("case", UVU_CASES)
+def test_uvu_materialised_equals_reassociated(case):
+    ir, l_max, K = case
+    ou, _, d, _, _ = _uvu_pair(ir, l_max, K)
+    g = (d.row_ptr, d.col, d.x, d.Y, d.phi, d.R)
+    assert np.allclose(ou.fwd(*g), ou.reassociated_fwd(*g), rtol=1e-11, atol=1e-12)
+
+
+def test_uvu_channels_do_not_mix():
+    """Changing input channel u changes output channel u only, in every block."""
+    ir, l_max, K = UVU_CASES[1]
+    ou, _, d, _, _ = _uvu_pair(ir, l_max, K)
+    g = (d.row_ptr, d.col)
+    y0 = ou.fwd(*g, d.x, d.Y, d.phi, d.R)
+    x1 = d.x.copy()
+    o = 0
+    for c, l, _ in ir:                      # perturb channel 0 of every input block
+        for m in range(2 * l + 1):
+            x1[:, o + m * c + 0] += 1.0
+        o += c * (2 * l + 1)
+    dy = ou.fwd(*g, x1, d.Y, d.phi, d.R) - y0
+    o = 0
+    for c, l, _ in ir:
+        blk = dy[:, o:o + c * (2 * l + 1)].reshape(-1, 2 * l + 1, c)
+        assert np.abs(blk[:, :, 1:]).max() == 0.0 and np.abs(blk[:, :, 0]).max() > 0.0
+        o += c * (2 * l + 1)
+
+
+def test_uvu_mixed_multiplicity_blocks_that_do_not_couple():
+    """Blocks of different multiplicity are allowed as long as no path joins them."""
+    ir = P("2x0e+3x1e")          # 0e x l_sh -> needs parity (-1)^l_sh: with l_max = 0 only 0e->0e and 1e->1e
+    ou = conv.Oracle(ir, ir, 0, 2, mode="uvu")
+    assert [(p.c_in, p.c_out) for p in ou.paths] == [(2, 2), (3, 3)] and ou.N_w == 5
