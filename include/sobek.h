@@ -74,6 +74,9 @@ typedef struct sobek_plan sobek_plan; /* opaque; host-owned; immutable after cre
 
 enum { SOBEK_MAX_L = 4 };
 
+/* plan flags */
+#define SOBEK_FLAG_UVU 1u   /* channelwise multiplicity mode, Eq. uvu_connection */
+
 /*
  * sobek_plan_create -- the static contract of one layer (Section "Generated
  * deterministic runtime and execution contracts"): enumerates the paths allowed by the
@@ -81,7 +84,12 @@ enum { SOBEK_MAX_L = 4 };
  * l = 0..l_max, computes the real Clebsch-Gordan tensors and uploads the sparse tables to
  * the current CUDA device (the only device allocation the library ever makes; it is
  * released by sobek_plan_destroy).  `in`/`out` are host arrays.  K >= 1 is the width of
- * the radial embedding.  `flags` must be 0.  If the environment variable SOBEK_FUSED is set to a
+ * the radial embedding.  `flags` is 0 for fully connected multiplicity mixing (Eq. uvw_connection:
+ * C_in*C_out weights per path, column w_off + u*C_out + w of R) or SOBEK_FLAG_UVU for the channelwise
+ * mode (Eq. uvu_connection: output multiplicity tied to the input one, C_in weights per path, column
+ * w_off + u; N_w = sum of C_in over the paths; a path between blocks of different multiplicity makes the
+ * call fail with UNSUPPORTED).  Every other argument, layout and entry point is the same in both modes.
+ * If the environment variable SOBEK_FUSED is set to a
  * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
  * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise
  * by the stream -> bounded state -> GEMM schedule, which is the faster one at present.  In that schedule

@@ -16,6 +16,8 @@ from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsobek.so")
 
+FLAG_UVU = 1   # SOBEK_FLAG_UVU: channelwise multiplicity mode
+
 EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
     "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_graph_receivers", "sobek_workspace_bytes", "sobek_conv_fwd",
@@ -126,9 +128,15 @@ def _irreps(seq):
 
 
 class Plan:
-    """sobek_plan: irreps are sequences of (mul, l, parity) with parity +1 / -1."""
+    """sobek_plan: irreps are sequences of (mul, l, parity) with parity +1 / -1.  mode "uvw" is the fully
+    connected multiplicity mixing, "uvu" the channelwise one (SOBEK_FLAG_UVU)."""
 
-    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0):
+    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0, mode: str = "uvw"):
+        if mode not in ("uvw", "uvu"):
+            raise ValueError(mode)
+        if mode == "uvu":
+            flags |= FLAG_UVU
+        self.mode = "uvu" if flags & FLAG_UVU else "uvw"
         self._h = c_void_p()
         a, b = _irreps(irreps_in), _irreps(irreps_out)
         _check(lib().sobek_plan_create(a, len(irreps_in), b, len(irreps_out), l_max, K, flags,
@@ -161,15 +169,17 @@ class Plan:
 
     def col_std(self):
         """1/sqrt(fan_in) per column of R (fan_in = K * sum of input multiplicities over the
-        paths into the column's output block): the scale used for synthetic weights."""
+        paths into the column's output block; K * number of those paths in the channelwise mode):
+        the scale used for synthetic weights."""
         import numpy as np
         paths = [self.path(k) for k in range(self.info.n_paths)]
+        uvu = self.mode == "uvu"
         fan = {}
         for p in paths:
-            fan[p.i_out] = fan.get(p.i_out, 0) + p.c_in
+            fan[p.i_out] = fan.get(p.i_out, 0) + (1 if uvu else p.c_in)
         std = np.zeros(self.info.N_w)
         for p in paths:
-            std[p.w_off:p.w_off + p.c_in * p.c_out] = (self.info.K * fan[p.i_out]) ** -0.5
+            std[p.w_off:p.w_off + (p.c_in if uvu else p.c_in * p.c_out)] = (self.info.K * fan[p.i_out]) ** -0.5
         return std
 
 

@@ -50,15 +50,19 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         w.bytes = off;
         return w;
     }
-    w.fNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.fNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
+    const bool gemm = !p->uvu;   // the channelwise mode has no GEMM, hence no operand copies of R
+    if (gemm) { w.fNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.fNKl = (uint16_t*)take(p->fwd.nk_elems * 2); }
     if (order >= 1) {
-        w.fKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.fKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
-        w.tNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.tNKl = (uint16_t*)take(p->tr.nk_elems * 2);
+        if (gemm) {
+            w.fKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.fKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
+            w.tNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.tNKl = (uint16_t*)take(p->tr.nk_elems * 2);
+        }
         w.gRp = (float*)take((size_t)p->K * (size_t)p->N_w * 4);
-        w.splits = (int)std::max<size_t>(1, std::min<size_t>(kMaxSplits, kPartBudgetBytes / ((size_t)p->K * (size_t)p->N_w * 4)));
+        w.splits = (int)std::max<size_t>(1, std::min<size_t>(gemm ? kMaxSplits : kMaxSplitsUvu,
+                                                             kPartBudgetBytes / ((size_t)p->K * (size_t)p->N_w * 4)));
         w.part = (float*)take((size_t)w.splits * (size_t)p->K * (size_t)p->N_w * 4);
     }
-    if (order >= 2) {
+    if (order >= 2 && gemm) {
         w.vfNKh = (uint16_t*)take(p->fwd.nk_elems * 2); w.vfNKl = (uint16_t*)take(p->fwd.nk_elems * 2);
         w.vfKNh = (uint16_t*)take(p->fwd.kn_elems * 2); w.vfKNl = (uint16_t*)take(p->fwd.kn_elems * 2);
         w.vtNKh = (uint16_t*)take(p->tr.nk_elems * 2); w.vtNKl = (uint16_t*)take(p->tr.nk_elems * 2);
@@ -70,8 +74,10 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     w.zbl = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
     if (order >= 1) {
         w.zbar = (float*)take((size_t)w.chunk * (size_t)p->fwd.state_floats * 4);
-        w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
-        w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
+        if (gemm) {
+            w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
+            w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
+        }
     }
     if (order >= 1 && p->use_tc_edge && p->fwd.etc[0].ok) {
         w.zqh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.zb_elems * 2);
@@ -209,6 +215,41 @@ cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn
     return fork.join();
 }
 
+// ---- the node-side steps in either multiplicity mode: tensor-core GEMMs on the packed copies of R (uvw), or
+// the elementwise kernels on R itself (uvu, Eq. uvu_connection) --------------------------------------------
+cudaError_t pack_R(const sobek_plan* p, const Direction& dir, int transposed, int n_major, const float* R, void* hi,
+                   void* lo, cudaStream_t s) {
+    return p->uvu ? cudaSuccess : launch_pack_R_bf16(p, dir, transposed, n_major, R, hi, lo, s);
+}
+cudaError_t split_gy(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const float* gdst,
+                     uint16_t* gh, uint16_t* gl, cudaStream_t s) {
+    return p->uvu ? cudaSuccess : split_adjoint(p, dir, n0, nn, gdst, gh, gl, s);
+}
+cudaError_t mix(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh,
+                const uint16_t* zl, const uint16_t* nkh, const uint16_t* nkl, const float* Rraw, float* dst,
+                int accumulate, int* status, cudaStream_t s) {
+    if (p->uvu) return launch_uvu_mix(p, dir, n0, nn, zh, zl, Rraw, dst, accumulate, s);
+    return mix_tc(p, dir, n0, nn, zh, zl, nkh, nkl, dst, accumulate, status, s);
+}
+cudaError_t state_adjoint(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const uint16_t* gh,
+                          const uint16_t* gl, const uint16_t* knh, const uint16_t* knl, const float* gy,
+                          const float* Rraw, float* Zbar, int* status, cudaStream_t s, uint16_t* zqh = nullptr,
+                          uint16_t* zql = nullptr) {
+    if (p->uvu) return launch_uvu_zbar(p, dir, n0, nn, gy, Rraw, Zbar, zqh, zql, s);
+    return state_adjoint_tc(p, dir, nn, gh, gl, knh, knl, Zbar, status, s, zqh, zql);
+}
+cudaError_t weight_grad(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh,
+                        const uint16_t* zl, const uint16_t* gh, const uint16_t* gl, const float* gy, float* gRp,
+                        float* part, int splits, int* status, cudaStream_t s) {
+    if (p->uvu) return launch_uvu_wgrad(p, dir, n0, nn, zh, zl, gy, gRp, part, splits, s);
+    return weight_grad_tc(p, dir, nn, zh, zl, gh, gl, gRp, part, splits, status, s);
+}
+// the accumulated weight adjoint -> the caller's [K, N_w] array (already in that layout in the uvu mode)
+cudaError_t unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R, cudaStream_t s) {
+    if (p->uvu) return cudaMemcpyAsync(R, Rp, (size_t)p->K * (size_t)p->N_w * 4, cudaMemcpyDeviceToDevice, s);
+    return launch_unpack_R(p, dir, Rp, R, s);
+}
+
 }  // namespace
 
 extern "C" size_t sobek_workspace_bytes(const sobek_plan* p, int64_t N, int64_t E, int order) {
@@ -251,13 +292,13 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
         CK(launch_fused(p, p->fwd, rv, x, nullptr, Y, nullptr, phi, nullptr, 0, w.fFKh, w.fFKl, y, 0, w.status, s));
         return SOBEK_OK;
     }
-    CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+    CK(pack_R(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     SplitSrc xs{};
     if (w.xsh) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
         CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
-        CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, y, 0, w.status, s));
+        CK(mix(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, R, y, 0, w.status, s));
     }
     return SOBEK_OK;
 }
@@ -284,28 +325,28 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     if (w.gsh && gx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (gR || gphi || gY) {
-        if (gphi || gY) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
+        if (gphi || gY) CK(pack_R(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
         if (gR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            CK(split_gy(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
-                CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
+                CK(weight_grad(p, p->fwd, n0, nn, w.zbh, w.zbl, w.gbh, w.gbl, gy, w.gRp, w.part, w.splits, w.status, s));
             }
             if (gphi || gY) {
                 if (tc_edge) {
-                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, nullptr, w.status, s, w.zqh, w.zql));
+                    CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, nullptr, w.status, s, w.zqh, w.zql));
                     CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql, gphi, gY,
                                            gphi ? 1 : 0, gY ? 1 : 0, w.status, s));
                 } else {
-                    CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                    CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, w.zbar, w.status, s));
                     CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
                                         gphi ? 1 : 0, gY ? 1 : 0, s));
                 }
             }
         }
-        if (gR) CK(launch_unpack_R(p, p->fwd, w.gRp, gR, s));
+        if (gR) CK(unpack_R(p, p->fwd, w.gRp, gR, s));
     }
     if (gx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(gx, g->N * (int64_t)p->C_x, s));
@@ -314,11 +355,11 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
             CK(launch_pack_R_fused(p, p->tr, 1, R, w.tFKh, w.tFKl, s));
             CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.tFKh, w.tFKl, gx, 0, w.status, s));
         } else {
-            CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
+            CK(pack_R(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
             for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
                 const int64_t nn = std::min(w.chunk, g->N - n0);
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
-                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, gx, 0, w.status, s));
+                CK(mix(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, R, gx, 0, w.status, s));
             }
         }
     }
@@ -382,37 +423,37 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             CK(launch_fused(p, p->fwd, rv, x, vx, Y, vY, phi, vphi, 1, w.fFKh, w.fFKl, ggy, ggy_done, w.status, s));
             ggy_done = 1;
         }
-        if (ggy && any_edge_dir && !fuse_dz) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
-        if (ggy && vR && !fuse_ggy) CK(launch_pack_R_bf16(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
-        if ((hphi || hY) && any_edge_dir) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
-        if ((hphi || hY) && vR) CK(launch_pack_R_bf16(p, p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl, s));
+        if (ggy && any_edge_dir && !fuse_dz) CK(pack_R(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
+        if (ggy && vR && !fuse_ggy) CK(pack_R(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
+        if ((hphi || hY) && any_edge_dir) CK(pack_R(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
+        if ((hphi || hY) && vR) CK(pack_R(p, p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl, s));
         if (hR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
-            if (hR || hphi || hY) CK(split_adjoint(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
+            if (hR || hphi || hY) CK(split_gy(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
             // ggy = Z vR + dZ R,  hR = dZ^T gy      (Eq. receiver_double_adjoint with d(gy) = 0)
             int ggy_written = ggy_done;
             if (ggy && vR && !fuse_ggy) {
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
-                CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, ggy, 0, w.status, s));
+                CK(mix(p, p->fwd, n0, nn, w.zbh, w.zbl, w.vfNKh, w.vfNKl, vR, ggy, 0, w.status, s));
                 ggy_written = 1;
             }
             if (((ggy && !fuse_dz) || hR) && any_edge_dir) {
                 // dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [C(vx,Y) + C(x,vY)] ) in one pass
                 CK(launch_stream(p, p->fwd, rv, n0, nn, x, vx, xs, Y, vY, phi, vphi, 1, w.zbh, w.zbl, w.status, s));
-                if (ggy && !fuse_dz) CK(mix_tc(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, ggy, ggy_written, w.status, s));
-                if (hR) CK(weight_grad_tc(p, p->fwd, nn, w.zbh, w.zbl, w.gbh, w.gbl, w.gRp, w.part, w.splits, w.status, s));
+                if (ggy && !fuse_dz) CK(mix(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, R, ggy, ggy_written, w.status, s));
+                if (hR) CK(weight_grad(p, p->fwd, n0, nn, w.zbh, w.zbl, w.gbh, w.gbl, gy, w.gRp, w.part, w.splits, w.status, s));
             }
             if (hphi || hY) {
                 int pm = 1, ym = 1;   // first writer overwrites, later ones accumulate
                 if (any_edge_dir) {
                     // the three direction terms that share Zbar = gy R^T, in one pass
                     if (tc_edge_dual) {
-                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, nullptr, w.status, s, w.zqh, w.zql));
+                        CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, nullptr, w.status, s, w.zqh, w.zql));
                         CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, vY, phi, vphi, 1, w.zqh, w.zql, hphi, hY,
                                                hphi ? pm : 0, hY ? ym : 0, w.status, s));
                     } else {
-                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, w.zbar, w.status, s));
+                        CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, w.zbar, w.status, s));
                         CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbar, hphi, hY,
                                             hphi ? pm : 0, hY ? ym : 0, s));
                     }
@@ -420,19 +461,19 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
                 }
                 if (vR) {   // the term through dZbar = gy vR^T
                     if (tc_edge_plain) {
-                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, nullptr, w.status, s, w.zqh, w.zql));
+                        CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, gy, vR, nullptr, w.status, s, w.zqh, w.zql));
                         SplitSrc xp{}; xp.h = xs.h; xp.l = xs.l;
                         CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xp, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql, hphi, hY,
                                                hphi ? pm : 0, hY ? ym : 0, w.status, s));
                     } else {
-                        CK(state_adjoint_tc(p, p->fwd, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, w.zbar, w.status, s));
+                        CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, gy, vR, w.zbar, w.status, s));
                         CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, hphi, hY,
                                             hphi ? pm : 0, hY ? ym : 0, s));
                     }
                 }
             }
         }
-        if (hR) CK(launch_unpack_R(p, p->fwd, w.gRp, hR, s));
+        if (hR) CK(unpack_R(p, p->fwd, w.gRp, hR, s));
     }
     if (hx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(hx, g->N * (int64_t)p->C_x, s));
@@ -450,19 +491,19 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
             }
             return SOBEK_OK;
         }
-        if (vY || vphi) CK(launch_pack_R_bf16(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
-        if (vR) CK(launch_pack_R_bf16(p, p->tr, 1, 1, vR, w.vtNKh, w.vtNKl, s));
+        if (vY || vphi) CK(pack_R(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
+        if (vR) CK(pack_R(p, p->tr, 1, 1, vR, w.vtNKh, w.vtNKl, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             int wrote = 0;
             if (vY || vphi) {   // dV = V(gy; vY, phi) + V(gy; Y, vphi) in one pass
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, vY, phi, vphi, 1, w.zbh, w.zbl, w.status, s));
-                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, hx, 0, w.status, s));
+                CK(mix(p, p->tr, n0, nn, w.zbh, w.zbl, w.tNKh, w.tNKl, R, hx, 0, w.status, s));
                 wrote = 1;
             }
             if (vR) {
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
-                CK(mix_tc(p, p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, hx, wrote, w.status, s));
+                CK(mix(p, p->tr, n0, nn, w.zbh, w.zbl, w.vtNKh, w.vtNKl, vR, hx, wrote, w.status, s));
             }
         }
     }

@@ -235,6 +235,7 @@ struct sobek_plan {
     bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
     bool use_tc_edge = true;     // edge pass on the tensor cores where the profile allows it
     size_t state_budget = size_t(2048) << 20;   // bytes of receiver / sender state held at once (the scratch budget)
+    bool uvu = false;         // channelwise mode (Eq. uvu_connection): tied multiplicities, C_in weights per path
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -398,6 +399,16 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
+
+// --- node_uvu.cu: the node-side steps of the channelwise mode (no GEMM) ---------------
+cudaError_t launch_uvu_mix(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
+                           const void* zl, const float* R, float* dst, int accumulate, cudaStream_t s0);
+cudaError_t launch_uvu_zbar(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const float* gy,
+                            const float* R, float* Zbar, void* zqh, void* zql, cudaStream_t s0);
+cudaError_t launch_uvu_wgrad(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
+                             const void* zl, const float* gy, float* gR_acc, float* part, int splits,
+                             cudaStream_t s0);
+constexpr int kMaxSplitsUvu = 64;                              // node slices of the channelwise weight adjoint
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);

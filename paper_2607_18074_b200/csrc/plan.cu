@@ -385,7 +385,7 @@ using namespace sobek;
 
 extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
                                  int l_max, int K, uint32_t flags, sobek_plan** plan) {
-    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || flags != 0 || l_max < 0)
+    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU)) != 0 || l_max < 0)
         return SOBEK_ERR_INVALID_ARG;
     *plan = nullptr;
     if (l_max > SOBEK_MAX_L) return SOBEK_ERR_UNSUPPORTED;
@@ -403,6 +403,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     p->out.assign(out, out + n_out);
     p->l_max = l_max;
     p->K = K;
+    p->uvu = (flags & SOBEK_FLAG_UVU) != 0;
     p->dim_sh = (l_max + 1) * (l_max + 1);
     std::vector<int> in_off(n_in), out_off(n_out);
     for (int i = 0; i < n_in; ++i) { in_off[i] = p->C_x; p->C_x += in[i].mul * (2 * in[i].l + 1); }
@@ -418,7 +419,13 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
                 HPath hp;
                 hp.info = sobek_path_info{ii, ls, io, li, lo, in[ii].mul, out[io].mul, in_off[ii], ls * ls,
                                           out_off[io], p->N_w};
-                p->N_w += int64_t(in[ii].mul) * out[io].mul;
+                if (p->uvu) {
+                    // tied multiplicities: the instruction needs C_out = C_in and owns C_in weights
+                    if (in[ii].mul != out[io].mul) { delete p; return SOBEK_ERR_UNSUPPORTED; }
+                    p->N_w += in[ii].mul;
+                } else {
+                    p->N_w += int64_t(in[ii].mul) * out[io].mul;
+                }
                 p->paths.push_back(hp);
                 triples.push_back(li); triples.push_back(ls); triples.push_back(lo);
             }
@@ -444,6 +451,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         for (double& v : p->paths[k].cg) v *= nrm;
     }
     if (const char* e = getenv("SOBEK_FUSED")) p->use_fused = atoi(e) != 0;
+    if (p->uvu) p->use_fused = false;   // the fused kernels contain the channel-mixing GEMM
     if (const char* e = getenv("SOBEK_STATE_BUDGET_MB")) {
         const long mb = atol(e);
         if (mb >= 1 && mb <= (1L << 20)) p->state_budget = size_t(mb) << 20;

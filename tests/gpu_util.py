@@ -24,8 +24,8 @@ class Case:
         import paper_2607_18074_b200 as sb
         self.sb, self.torch = sb, torch
         self.w = w
-        self.oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
-        self.plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+        self.oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
+        self.plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
         self.d = inputs if inputs is not None else synth.make_inputs(w, self.oracle.col_std())
         d = self.d
         dev = "cuda:0"

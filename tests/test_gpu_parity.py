@@ -361,3 +361,95 @@ def test_cuda_graph_capture(cases):
         assert sb.last_device_status(ws) == 0
         for got, ref in zip(outs, eager):
             assert np.array_equal(got.cpu().numpy(), ref)
+
+
+# ---------------------------------------------------------------------------------------
+# channelwise (uvu) mode, Eq. uvu_connection: same edge kernels, elementwise node-side steps
+# ---------------------------------------------------------------------------------------
+def uvu_cases():
+    W = synth.Workload
+    c = {}
+    # tensor-core edge kernels (multiplicities that are multiples of 16), several node chunks' worth of rows
+    c["uvu_16x3"] = W("uvu_16x3", P("16x0e+16x1o+16x2e"), P("16x0e+16x1o+16x2e"), 2, 8, 150, 4.0, 1.5, "bessel", seed=7,
+                      mode="uvu")
+    c["uvu_32x4_K16"] = W("uvu_32x4_K16", P("32x0e+32x1o+32x2e+32x3o"), P("32x0e+32x1o+32x2e+32x3o"), 3, 16, 80, 4.0, 1.7,
+                          "bessel", seed=8, mode="uvu")
+    # FP32-pipe edge kernels: odd multiplicities, blocks of different multiplicity that no path couples, an
+    # output block without an input twin (3x3e, fed by 4e only), a multiplicity above 128
+    c["uvu_ragged"] = W("uvu_ragged", P("5x0e+5x1o+3x4e+2x0o"), P("5x0e+5x1o+3x4e+3x3e+2x0o"), 2, 3, 40, 4.0, 1.9,
+                        "gaussian", seed=9, mode="uvu")
+    c["uvu_wide"] = W("uvu_wide", P("144x0e+144x1o"), P("144x0e+144x1o"), 1, 8, 60, 4.0, 1.8, "bessel", seed=10, mode="uvu")
+    return c
+
+
+UVU = uvu_cases()
+
+
+@pytest.fixture(scope="module")
+def ucases():
+    return {}
+
+
+def uget(ucases, name):
+    if name not in ucases:
+        ucases[name] = Case(UVU[name])
+    return ucases[name]
+
+
+@pytest.mark.parametrize("name", list(UVU))
+def test_uvu_forward(ucases, name):
+    c = uget(ucases, name)
+    assert c.plan.info.N_w == c.oracle.N_w
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+
+
+@pytest.mark.parametrize("name", list(UVU))
+def test_uvu_backward(ucases, name):
+    c = uget(ucases, name)
+    for got, ref in zip(c.bwd(), c.o_bwd()):
+        assert rel_err(got, ref) <= BWD_TOL
+
+
+@pytest.mark.parametrize("name", list(UVU))
+def test_uvu_double_backward(ucases, name):
+    c = uget(ucases, name)
+    for got, ref in zip(c.dbwd(), c.o_dbwd()):
+        assert rel_err(got, ref) <= BWD_TOL
+
+
+@pytest.mark.parametrize("dirs", [(1, 0, 0, 0), (0, 1, 0, 0), (0, 0, 1, 0), (0, 0, 0, 1)])
+def test_uvu_double_backward_single_directions(ucases, dirs):
+    c = uget(ucases, "uvu_16x3")
+    for got, ref in zip(c.dbwd(dirs=dirs), c.o_dbwd(dirs=dirs)):
+        assert rel_err(got, ref) <= BWD_TOL
+
+
+def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases, monkeypatch):
+    c = uget(ucases, "uvu_16x3")
+    for a, b in zip([c.fwd()] + c.bwd() + c.dbwd(), [c.fwd()] + c.bwd() + c.dbwd()):
+        assert np.array_equal(a, b)
+    monkeypatch.setenv("SOBEK_TC_STREAM", "0")
+    monkeypatch.setenv("SOBEK_TC_EDGE", "0")
+    f = Case(UVU["uvu_16x3"], inputs=c.d)
+    assert rel_err(f.fwd(), c.o_fwd()) <= FWD_TOL
+    for got, ref in zip(f.bwd(), c.o_bwd()):
+        assert rel_err(got, ref) <= BWD_TOL
+    for got, ref in zip(f.dbwd(), c.o_dbwd()):
+        assert rel_err(got, ref) <= BWD_TOL
+
+
+def test_uvu_full_size_sampled():
+    """The paper's 128/128/128 channelwise profile (K = 16) on 31 copies of its 128-node graph."""
+    FULL["uvu_128x3_31"] = (synth.config("uvu_128x3_31"), 6, (0, 1, 2))
+    try:
+        test_full_size_sampled("uvu_128x3_31")
+    finally:
+        del FULL["uvu_128x3_31"]
+
+
+def test_uvu_plan_contract():
+    import paper_2607_18074_b200 as sb
+    ir = P("64x0e+64x1o+64x2e+64x3o")
+    assert sb.Plan(ir, ir, 3, 16, mode="uvu").info.N_w == 1472          # Table uvu_capacity_matched
+    with pytest.raises(sb.SobekError):
+        sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")      # 0e x 1o -> 1o would tie 8 to 4

@@ -115,3 +115,36 @@ def test_argument_errors_are_status_codes():
     assert L.sobek_plan_path(plan.handle, 99, ctypes.byref(sb.PathInfo())) == -1
     assert sb.workspace_bytes(plan, 4, 0, 7) == 0
     assert L.sobek_last_device_status(None, None) == -1
+
+
+def test_uvu_plan_weight_counts_match_the_paper():
+    """Channelwise mode (Eq. uvu_connection): N_w = sum of C_in over the paths; the paper prints it for nine
+    profiles (Table uvu_capacity_matched)."""
+    n = 0
+    for line in open(os.path.join(ROOT, "tests", "golden", "paper_weight_counts.txt")):
+        tok = line.split()
+        if not tok or tok[0] != "uvu":
+            continue
+        mults = [int(v) for v in tok[1].split("/")]
+        ir = [(m, l, 1 if l % 2 == 0 else -1) for l, m in enumerate(mults)]
+        plan = sb.Plan(ir, ir, len(mults) - 1, 16, mode="uvu")
+        assert plan.info.N_w == int(tok[2])
+        paths, n_w = tables.enumerate_paths(ir, ir, len(mults) - 1, "uvu")
+        assert [plan.path(k).w_off for k in range(plan.info.n_paths)] == [p.w_off for p in paths]
+        n += 1
+    assert n == 9
+
+
+def test_uvu_plan_errors_and_workspace():
+    P = synth.parse_irreps
+    with pytest.raises(sb.SobekError):
+        sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")       # 0e x 1o -> 1o would tie 8 channels to 4
+    with pytest.raises(sb.SobekError):
+        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=2)                    # unknown flag bit
+    ir = P("64x0e+64x1o+64x2e")
+    u, w = sb.Plan(ir, ir, 2, 16, mode="uvu"), sb.Plan(ir, ir, 2, 16)
+    assert u.mode == "uvu" and w.mode == "uvw" and u.info.C_y == w.info.C_y
+    for order in (0, 1, 2):
+        a = sb.workspace_bytes(u, 3125, 10**5, order)
+        assert a == sb.workspace_bytes(u, 3125, 10**9, order)            # nothing edge-sized
+        assert a <= sb.workspace_bytes(w, 3125, 10**5, order)            # no GEMM operand copies of R

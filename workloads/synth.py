@@ -171,6 +171,7 @@ class Workload:
     seed: int = 0
     note: str = ""
     copies: int = 1  # the graph of N nodes repeated this many times (disjoint copies, one batch)
+    mode: str = "uvw"  # multiplicity mode of the operator: "uvw" fully connected, "uvu" channelwise
 
 
 def _cube(N, rho):
@@ -206,6 +207,14 @@ def config(name: str, **kw) -> Workload:
         N = 50000
         L = _cube(N, 0.1)
         return Workload("cfg5", ir, ir, 4, 16, N, L, cutoff_for_edges(N, 40.0 * N, L), "bessel")
+    if name.startswith("uvu_"):
+        # channelwise mode on the paper's fixed 128-node, degree-32 graph repeated B times (appendix "Native
+        # Channelwise Throughput"): uvu_<mult>x<blocks>_<B>, e.g. uvu_128x3_511 = profile 128/128/128, K = 16
+        _, prof, B = name.split("_")
+        mult, nb = (int(v) for v in prof.split("x"))
+        base = config(f"graphs_{int(B)}")
+        ir = [(mult, l, 1 if l % 2 == 0 else -1) for l in range(nb)]
+        return Workload(name, ir, ir, nb - 1, 16, base.N, base.L, base.r_c, "bessel", copies=base.copies, mode="uvu")
     if name.startswith("deg_") or name.startswith("graphs_"):
         # the paper's two scaling axes (section "Scaling axes"), on its 128/64/64 profile with K = 16:
         # longer neighbourhoods on 2,048 nodes, or one 128-node graph of mean degree 32 repeated B times
