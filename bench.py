@@ -63,8 +63,9 @@ def work_model(plan):
         KFt += K * p.c_out * di
         CG += p.c_in * nnz
         CGt += p.c_out * nnz
-        Gf += K * p.c_in * p.c_out * do
-        Gt += K * p.c_in * p.c_out * di
+        co = 1 if plan.mode == "uvu" else p.c_out      # tied multiplicities: no sum over a second channel index
+        Gf += K * p.c_in * co * do
+        Gt += K * p.c_in * co * di
     edge = {"fwd": KF + CG, "bwd": 3 * KF + KFt + 3 * CG + CGt, "dbwd": 8 * KF + 3 * KFt + 5 * CG + 2 * CGt}
     node = {"fwd": Gf, "bwd": 2 * Gf + Gt, "dbwd": 5 * Gf + 2 * Gt}
     # split of the edge work between the two edge-stream kernel classes
@@ -153,7 +154,7 @@ def run_reference(args):
         return
     from oracle import conv as oconv
     w = synth.config(args.workload)
-    oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
     d = synth.make_inputs(w, oracle.col_std())
     cores = oconv.threads()
     # one step = fwd+bwd+dbwd on a bounded contiguous receiver sample
@@ -213,7 +214,7 @@ def main():
         dist = dist_mod
 
     w = synth.config(args.workload)
-    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
     # replicas only: every rank runs the same workload on its own GPU (different seed per rank)
     w.seed = rank
     d = synth.make_inputs(w, plan.col_std())
@@ -378,7 +379,7 @@ def main():
         "metric": METRIC, "value": E_total / (step_ms * 1e-3), "unit": "edges/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "N": N, "E": E, "K": i.K, "N_w": int(i.N_w), "C_x": i.C_x, "C_y": i.C_y,
+        "config": {"workload": w.name, "mode": w.mode, "N": N, "E": E, "K": i.K, "N_w": int(i.N_w), "C_x": i.C_x, "C_y": i.C_y,
                    "l_max": i.l_max, "replicas": world, "l2": f"flushed before every order ({L2_FLUSH_BYTES >> 20} MiB write)"},
         "orders": {nm: {"edges_per_s": E_total / (ms * 1e-3), "ms": float(ms),
                         "edge_fma_per_edge": edge_w[nm], "node_fma_per_node": node_w[nm]}
@@ -394,7 +395,7 @@ def main():
     }
     if not args.no_cpu_baseline and world == 1:
         from oracle import conv as oconv
-        oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
+        oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
         rate, edges, secs, tt, nrecv, cores = oracle_sample_rate(w, d, oracle)
         res["cpu_baseline"] = {"value": rate, "unit": "edges/s", "cores": cores, "kind": "oracle",
                                "sample": f"first {nrecv} receivers ({edges} edges) of {w.name}, fwd+bwd+dbwd, {secs:.1f} s",

@@ -24,11 +24,19 @@ __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf1(uint16_t v) { return __uint_as_float((uint32_t)v << 16); }
 
-// V consecutive multiplicities of the state, hi + lo, starting at element index i (i even when V == 2)
+// V consecutive multiplicities of the state, hi + lo, starting at element index i (a multiple of V)
 template <int V>
 __device__ __forceinline__ void load_state(const uint16_t* __restrict__ zh, const uint16_t* __restrict__ zl, int64_t i,
                                            float* z) {
-    if (V == 2) {
+    if (V == 8) {
+        const uint4 h = *reinterpret_cast<const uint4*>(zh + i), l = *reinterpret_cast<const uint4*>(zl + i);
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w}, lw[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            z[2 * j] = bf_lo(hw[j]) + bf_lo(lw[j]);
+            z[2 * j + 1] = bf_hi(hw[j]) + bf_hi(lw[j]);
+        }
+    } else if (V == 2) {
         const uint32_t h = *reinterpret_cast<const uint32_t*>(zh + i), l = *reinterpret_cast<const uint32_t*>(zl + i);
         z[0] = bf_lo(h) + bf_lo(l);
         z[1] = bf_hi(h) + bf_hi(l);
@@ -106,7 +114,17 @@ __global__ void k_uvu_zbar(UvuGroup g, const float* __restrict__ gy, const float
                 h[v] = __float2bfloat16_rn(val[v]);
                 l[v] = __float2bfloat16_rn(val[v] - __bfloat162float(h[v]));
             }
-            if (V == 2) {
+            if (V == 8) {
+                uint32_t hw[4], lw[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const __nv_bfloat162 hp = __halves2bfloat162(h[2 * j], h[2 * j + 1]), lp = __halves2bfloat162(l[2 * j], l[2 * j + 1]);
+                    hw[j] = *reinterpret_cast<const uint32_t*>(&hp);
+                    lw[j] = *reinterpret_cast<const uint32_t*>(&lp);
+                }
+                *reinterpret_cast<uint4*>(zh + r * g.ld + k) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                *reinterpret_cast<uint4*>(zl + r * g.ld + k) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            } else if (V == 2) {
                 *reinterpret_cast<__nv_bfloat162*>(zh + r * g.ld + k) = __halves2bfloat162(h[0], h[1]);
                 *reinterpret_cast<__nv_bfloat162*>(zl + r * g.ld + k) = __halves2bfloat162(l[0], l[1]);
             } else {
@@ -179,7 +197,8 @@ cudaError_t launch_uvu_mix(const sobek_plan* p, const Direction& dir, int64_t n0
         const uint16_t* l = (const uint16_t*)zl + nn * dir.zb_off[gi];
         float* d = dst + n0 * dir.C_dst + G.dst_off;
         KernelTimer kt(K_GEMM, s);
-        if (g.c % 2 == 0) k_uvu_mix<2><<<grid_for(g.rows * (g.c / 2)), 256, 0, s>>>(g, h, l, R, d, accumulate);
+        if (g.c % 8 == 0) k_uvu_mix<8><<<grid_for(g.rows * (g.c / 8)), 256, 0, s>>>(g, h, l, R, d, accumulate);
+        else if (g.c % 2 == 0) k_uvu_mix<2><<<grid_for(g.rows * (g.c / 2)), 256, 0, s>>>(g, h, l, R, d, accumulate);
         else k_uvu_mix<1><<<grid_for(g.rows * g.c), 256, 0, s>>>(g, h, l, R, d, accumulate);
         count_launch();
         cudaError_t e = cudaGetLastError();
@@ -202,7 +221,8 @@ cudaError_t launch_uvu_zbar(const sobek_plan* p, const Direction& dir, int64_t n
         uint16_t* l = zqh ? (uint16_t*)zql + nn * dir.zb_off[gi] : nullptr;
         const int64_t total = g.rows * (int64_t)g.np * g.K * g.c;
         KernelTimer kt(K_GEMM, s);
-        if (g.c % 2 == 0) k_uvu_zbar<2><<<grid_for(total / 2), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
+        if (g.c % 8 == 0) k_uvu_zbar<8><<<grid_for(total / 8), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
+        else if (g.c % 2 == 0) k_uvu_zbar<2><<<grid_for(total / 2), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
         else k_uvu_zbar<1><<<grid_for(total), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
         count_launch();
         cudaError_t e = cudaGetLastError();
@@ -226,11 +246,12 @@ cudaError_t launch_uvu_wgrad(const sobek_plan* p, const Direction& dir, int64_t 
             const uint16_t* h = (const uint16_t*)zh + nn * dir.zb_off[gi];
             const uint16_t* l = (const uint16_t*)zl + nn * dir.zb_off[gi];
             const float* gsrc = gy + n0 * dir.C_dst + G.dst_off;
-            const int V = g.c % 2 == 0 ? 2 : 1;
+            const int V = g.c % 8 == 0 ? 8 : g.c % 2 == 0 ? 2 : 1;
             const int64_t cols = (int64_t)g.np * g.K * (g.c / V);
             dim3 grid((unsigned)std::max<int64_t>(1, (cols + 127) / 128), (unsigned)sp);
             KernelTimer kt(K_GEMM, s);
-            if (V == 2) k_uvu_wgrad<2><<<grid, 128, 0, s>>>(g, h, l, gsrc, part, KN, sp);
+            if (V == 8) k_uvu_wgrad<8><<<grid, 128, 0, s>>>(g, h, l, gsrc, part, KN, sp);
+            else if (V == 2) k_uvu_wgrad<2><<<grid, 128, 0, s>>>(g, h, l, gsrc, part, KN, sp);
             else k_uvu_wgrad<1><<<grid, 128, 0, s>>>(g, h, l, gsrc, part, KN, sp);
             count_launch();
             cudaError_t e = cudaGetLastError();
