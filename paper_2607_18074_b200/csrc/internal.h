@@ -408,7 +408,7 @@ cudaError_t launch_uvu_zbar(const sobek_plan* p, const Direction& dir, int64_t n
 cudaError_t launch_uvu_wgrad(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
                              const void* zl, const float* gy, float* gR_acc, float* part, int splits,
                              cudaStream_t s0);
-constexpr int kMaxSplitsUvu = 64;                              // node slices of the channelwise weight adjoint
+constexpr int kMaxSplitsUvu = 256;                             // node slices of the channelwise weight adjoint
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);

@@ -72,6 +72,7 @@ __global__ void k_uvu_mix(UvuGroup g, const uint16_t* __restrict__ zh, const uin
         for (int pl = 0; pl < g.np; ++pl) {
             const int64_t wcol = g.paths[pl].w_off + u;
             const int64_t zp = zrow + (int64_t)pl * g.K * g.c;
+#pragma unroll 4
             for (int q = 0; q < g.K; ++q) {
                 float z[V];
                 load_state<V>(zh, zl, zp + (int64_t)q * g.c, z);
@@ -166,6 +167,53 @@ __global__ void k_uvu_wgrad(UvuGroup g, const uint16_t* __restrict__ zh, const u
     }
 }
 
+// ---- multiplicities that are multiples of 8: one block per state row, threads (x = 8 multiplicities, y = (path, q)) ----
+// Zbar row = gy row (x) R as bf16 (hi, lo) or fp32: thread (x, y) keeps its 8 output-adjoint values and walks the
+// (path, q) pairs pq = y, y + blockDim.y, ...
+__global__ void k_uvu_zbar_row(UvuGroup g, const float* __restrict__ gy, const float* __restrict__ R,
+                               float* __restrict__ zf, int64_t ldf, uint16_t* __restrict__ zh, uint16_t* __restrict__ zl) {
+    const int cv = g.c >> 3;
+    const int64_t r = blockIdx.x;
+    const float* gr = gy + (r / g.d) * g.C_dst + (r % g.d) * g.c;
+    for (int x = threadIdx.x; x < cv; x += blockDim.x) {
+        const int u = x << 3;
+        float gv[8];
+#pragma unroll
+        for (int v = 0; v < 8; ++v) gv[v] = gr[u + v];
+        for (int pq = threadIdx.y; pq < g.np * g.K; pq += blockDim.y) {
+            const int pl = pq / g.K, q = pq - pl * g.K;
+            const float* Rr = R + q * g.N_w + g.paths[pl].w_off + u;
+            float val[8];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) val[v] = gv[v] * __ldg(Rr + v);
+            const int64_t k = (int64_t)pq * g.c + u;
+            if (zf) {
+#pragma unroll
+                for (int v = 0; v < 8; ++v) zf[r * ldf + k + v] = val[v];
+            } else {
+                uint32_t hw[4], lw[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const __nv_bfloat162 hp = __floats2bfloat162_rn(val[2 * j], val[2 * j + 1]);
+                    const float2 hf = __bfloat1622float2(hp);
+                    const __nv_bfloat162 lp = __floats2bfloat162_rn(val[2 * j] - hf.x, val[2 * j + 1] - hf.y);
+                    hw[j] = *reinterpret_cast<const uint32_t*>(&hp);
+                    lw[j] = *reinterpret_cast<const uint32_t*>(&lp);
+                }
+                *reinterpret_cast<uint4*>(zh + r * g.ld + k) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                *reinterpret_cast<uint4*>(zl + r * g.ld + k) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
+        }
+    }
+}
+
+// block shape of the row kernels: x covers the 8-multiplicity pieces of a row (at most 32), y the rest of 256 threads
+dim3 row_block(int c, int ny_max) {
+    const int bx = std::max(1, std::min(c / 8, 32));
+    const int by = std::max(1, std::min(ny_max, 256 / bx));
+    return dim3((unsigned)bx, (unsigned)by);
+}
+
 UvuGroup make_group(const sobek_plan* p, const Direction& dir, size_t gi, int64_t nn) {
     const DGroup& G = dir.groups[gi];
     UvuGroup g{};
@@ -221,7 +269,7 @@ cudaError_t launch_uvu_zbar(const sobek_plan* p, const Direction& dir, int64_t n
         uint16_t* l = zqh ? (uint16_t*)zql + nn * dir.zb_off[gi] : nullptr;
         const int64_t total = g.rows * (int64_t)g.np * g.K * g.c;
         KernelTimer kt(K_GEMM, s);
-        if (g.c % 8 == 0) k_uvu_zbar<8><<<grid_for(total / 8), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
+        if (g.c % 8 == 0) k_uvu_zbar_row<<<(unsigned)g.rows, row_block(g.c, g.np * g.K), 0, s>>>(g, gsrc, R, zf, G.D, h, l);
         else if (g.c % 2 == 0) k_uvu_zbar<2><<<grid_for(total / 2), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
         else k_uvu_zbar<1><<<grid_for(total), 256, 0, s>>>(g, gsrc, R, zf, G.D, h, l);
         count_launch();
