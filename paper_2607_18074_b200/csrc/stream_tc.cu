@@ -83,6 +83,9 @@ __device__ __forceinline__ int64_t owner_of(const int64_t* __restrict__ row_ptr,
 // L1 given to the operand regions, table reads from global memory would mostly go to L2.
 struct UInfo {     // a unit, as the MMA thread and the drain need it
     uint32_t idesc, tmem_col, a_off, slab_stride, b_off, slab_bytes, d_src, comp_begin, ncomp, c_src, ncols, pad;
+    // operand descriptors of slab 0 (hi copies; stage 0 of the ring for B): the other slabs, copies and stages differ
+    // only in the 16-byte-granular address field, so the MMA thread reaches them with one addition each
+    uint64_t dA0, dB0;
 };
 // shared-memory operand descriptor without swizzle (K-major core matrices of 8 rows x 16 bytes)
 __device__ __forceinline__ uint64_t make_desc_none(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -202,6 +205,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         u.b_off = (uint32_t)B.b_off; u.slab_bytes = (uint32_t)B.slab_bytes; u.d_src = (uint32_t)B.d_src;
         u.comp_begin = (uint32_t)U.comp_begin; u.ncomp = (uint32_t)U.ncomp; u.c_src = (uint32_t)B.c_src;
         u.ncols = (uint32_t)B.ncols; u.pad = 0;
+        u.dA0 = make_desc_none(smem_u32(sA) + u.a_off, 128, 256);
+        u.dB0 = make_desc(smem_u32(sRing) + u.b_off, 2048, 1024);
         sU[i] = u;
     }
     for (int i = tid; i < a.nsets; i += TT) sSet[i] = a.sets[i];
@@ -217,6 +222,12 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
     const int64_t total = a.n_nodes * a.nsets;
+    // (local node, set) of an item, advanced without divisions: items are set-major, a CTA takes every gridDim.x-th
+    struct ItemPos {
+        int64_t nl; int set;
+        __device__ void init(int64_t item, int64_t n) { nl = item % n; set = (int)(item / n); }
+        __device__ void step(int64_t by, int64_t n) { nl += by; while (nl >= n) { nl -= n; ++set; } }
+    };
 
     if (warp >= NCW && warp < NCW + NLW) {
         // =========================== loader warps ===========================
@@ -225,9 +236,10 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         // signal the stage's mbarrier when they land (no wait in this warp).
         const int lt = (warp - NCW) * 32 + lane;   // thread index among the loaders
         int64_t p_item = blockIdx.x, p_seg0 = 0, p_seg1 = 0;     // prefetched item
+        ItemPos lp; lp.init(p_item, a.n_nodes);
         auto prefetch_item = [&]() {
             if (p_item < total) {
-                const int64_t node = a.node0 + p_item % a.n_nodes;
+                const int64_t node = a.node0 + lp.nl;
                 p_seg0 = a.ev.ptr[node];
                 p_seg1 = any_op ? a.ev.ptr[node + 1] : p_seg0;
             }
@@ -242,8 +254,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             while (first || c.b0 >= c.seg1) {
                 first = false;
                 if (p_item >= total) return false;
-                c.set = (int)(p_item / a.n_nodes); c.b0 = p_seg0; c.seg1 = p_seg1; c.sub = 0;
-                p_item += gridDim.x;
+                c.set = lp.set; c.b0 = p_seg0; c.seg1 = p_seg1; c.sub = 0;
+                p_item += gridDim.x; lp.step(gridDim.x, a.n_nodes);
                 prefetch_item();
             }
             return true;
@@ -293,38 +305,37 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     }
                 }
             }
-            // Y (and vY), transposed: raw[b][PS + e]
+            // Y (and vY), transposed: raw[b][PS + e].  Thread <-> (edge e = lane mod 16, b = lt / 16, + 4, ...)
+            const int le = lane & (TB - 1);
+            const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
             {
                 const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
-                const int n_it = TB * a.dsh;
-                for (int i0 = 0; i0 < n_it; i0 += NLW * 32) {
-                    const int i = i0 + lt;
-                    const int e = min(i / a.dsh, TB - 1), b = i - (i / a.dsh) * a.dsh;
-                    const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
-                    if (i < n_it) {
-                        const uint32_t ok = e < nb ? 4u : 0u;
-                        cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
-                        if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
-                    }
+                const uint32_t ok = le < nb ? 4u : 0u;
+                const float* yr = a.Y + ee_own * a.dsh;
+                const float* vyr = has_vY ? a.vY + ee_own * a.dsh : nullptr;
+                for (int b = lt >> 4; b < a.dsh; b += NLW * 32 / TB) {
+                    cp_async4_zfill(y_u + (uint32_t)(b * PS + le) * 4, yr + b, ok);
+                    if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + le) * 4, vyr + b, ok);
                 }
             }
-            // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy: a thread owns an
-            // (edge, piece) pair of a block and walks its d_src rows with constant strides
-            for (int bi = 0; bi < S.nblk; ++bi) {
-                const TBlk B = sBlk[S.blk_begin + bi];
-                const int cpr = B.c_src >> 3;                  // 16-byte pieces per row
-                const int npair = TB * cpr;
-                for (int p0 = 0; p0 < npair; p0 += NLW * 32) {
-                    const int pr = p0 + lt;
-                    const int e = min(pr / cpr, TB - 1), j = pr - (pr / cpr) * cpr;
-                    const int32_t sne = __shfl_sync(0xffffffffu, sn, e);
-                    if (pr < npair) {
-                        const uint32_t ok = e < nb ? 16u : 0u;
+            // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy
+            {
+                // lanes 2e, 2e+1 of each loader warp serve edge e; a thread walks pieces j0, j0 + 4, ... of the row
+                const int re = (lane >> 1) & (TB - 1);
+                const int32_t sne = __shfl_sync(0xffffffffu, sn, re);
+                const uint32_t ok = re < nb ? 16u : 0u;
+                const int j0 = (lane & 1) | ((lt >> 5) << 1);
+                const int64_t grow = (int64_t)sne * a.C_src;
+                const __nv_bfloat16* srch = (op == 0 ? a.sh : a.vsh) + grow;
+                const __nv_bfloat16* srcl = (op == 0 ? a.sl : a.vsl) + grow;
+                for (int bi = 0; bi < S.nblk; ++bi) {
+                    const TBlk B = sBlk[S.blk_begin + bi];
+                    const int cpr = B.c_src >> 3;                  // 16-byte pieces per row
+                    for (int j = j0; j < cpr; j += 2 * NLW) {
                         const int u = 8 * j;
-                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
-                        const int64_t g = (int64_t)sne * a.C_src + B.src_off + u;
-                        const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
-                        const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
+                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + re * 128 + ((((u & 63) >> 3) ^ (re & 7)) << 4));
+                        const __nv_bfloat16* ph = srch + B.src_off + u;
+                        const __nv_bfloat16* pl = srcl + B.src_off + u;
                         for (int sdx = 0; sdx < B.d_src; ++sdx) {
                             cp_async16_zfill(d, ph, ok);
                             cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
@@ -341,11 +352,18 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         // =========================== MMA warp ===========================
         if (lane == 0) {
             uint32_t it = 0, mi = 0;
+            int64_t nx0 = 0, nx1 = 0;
+            ItemPos mp; mp.init(blockIdx.x, a.n_nodes);      // position of the item whose bounds are in flight
+            if ((int64_t)blockIdx.x < total) { const int64_t nn = a.node0 + mp.nl; nx0 = a.ev.ptr[nn]; nx1 = a.ev.ptr[nn + 1]; }
+            const uint64_t acap16 = (uint64_t)(a.a_cap >> 4), bcap16 = (uint64_t)(a.b_cap >> 4);
             for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-                const int64_t nl = item % a.n_nodes;
-                const TSet S = sSet[(int)(item / a.n_nodes)];
-                const int64_t node = a.node0 + nl;
-                const int64_t seg0 = a.ev.ptr[node], seg1 = any_op ? a.ev.ptr[node + 1] : seg0;
+                const TSet S = sSet[mp.set];
+                const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
+                mp.step(gridDim.x, a.n_nodes);
+                if (item + gridDim.x < total) {     // the next item's bounds, requested one item ahead
+                    const int64_t nn = a.node0 + mp.nl;
+                    nx0 = a.ev.ptr[nn]; nx1 = a.ev.ptr[nn + 1];
+                }
                 if (seg1 <= seg0) continue;
                 const uint32_t buf = mi & 1;
                 if (mi >= 2) mbar_wait(bar_accfree + 8 * buf, ((mi >> 1) & 1) ^ 1, a.status);
@@ -355,23 +373,22 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                         const int st = (int)(it % NS);
                         mbar_wait(bar_ready, it & 1, a.status);
                         tc_fence_after();
-                        const uint32_t sA_u = smem_u32(sA);
-                        const uint32_t sB_u = smem_u32(sRing + (size_t)st * stage_bytes);
+                        const uint64_t st16 = (uint64_t)((uint32_t)st * (stage_bytes >> 4));
+                        const uint32_t acc0 = (b0 == seg0 && sb == 0) ? 0u : 1u;
                         for (int ui = 0; ui < S.nunit; ++ui) {
-                            const UInfo U = sU[S.unit_begin + ui];
+                            const UInfo& U = sU[S.unit_begin + ui];
                             const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + U.tmem_col;
-                            uint32_t acc = (b0 == seg0 && sb == 0) ? 0u : 1u;
-                            for (uint32_t s = 0; s < U.d_src; ++s) {
-                                const uint32_t ah = sA_u + U.a_off + s * U.slab_stride;
-                                const uint32_t al = ah + a.a_cap;
-                                const uint32_t bh = sB_u + U.b_off + s * U.slab_bytes;
-                                const uint32_t bl = bh + a.b_cap;
-                                const uint64_t dAh = make_desc_none(ah, 128, 256), dAl = make_desc_none(al, 128, 256);
-                                const uint64_t dBh = make_desc(bh, 2048, 1024), dBl = make_desc(bl, 2048, 1024);
-                                tc_mma_bf16(d_tmem, dAh, dBh, U.idesc, acc);
-                                tc_mma_bf16(d_tmem, dAl, dBh, U.idesc, 1u);
-                                tc_mma_bf16(d_tmem, dAh, dBl, U.idesc, 1u);
-                                acc = 1u;
+                            const uint32_t idesc = U.idesc, nslab = U.d_src;
+                            const uint64_t sa16 = U.slab_stride >> 4, sb16 = U.slab_bytes >> 4;
+                            uint64_t dAh = U.dA0, dBh = U.dB0 + st16;
+                            tc_mma_bf16(d_tmem, dAh, dBh, idesc, acc0);
+                            tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dAh, dBh + bcap16, idesc, 1u);
+                            for (uint32_t s = 1; s < nslab; ++s) {
+                                dAh += sa16; dBh += sb16;
+                                tc_mma_bf16(d_tmem, dAh, dBh, idesc, 1u);
+                                tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
+                                tc_mma_bf16(d_tmem, dAh, dBh + bcap16, idesc, 1u);
                             }
                         }
                         tc_commit(bar_afree);
@@ -386,6 +403,9 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         // =========================== compute warps ===========================
         uint32_t it = 0, mi = 0;
         int cur_set = -1;
+        int64_t cx0 = 0, cx1 = 0;
+        ItemPos cp_; cp_.init(blockIdx.x, a.n_nodes);        // position of the item whose bounds are in flight
+        if ((int64_t)blockIdx.x < total) { const int64_t nn = a.node0 + cp_.nl; cx0 = a.ev.ptr[nn]; cx1 = a.ev.ptr[nn + 1]; }
         // the item whose accumulator is drained next (one behind the one being built)
         int64_t p_nl = -1; int p_set = 0; uint32_t p_mi = 0; bool p_wrote = false;
 
@@ -452,11 +472,15 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         };
 
         for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-            const int64_t nl = item % a.n_nodes;
-            const int set = (int)(item / a.n_nodes);
+            const int64_t nl = cp_.nl;
+            const int set = cp_.set;
             const TSet S = sSet[set];
-            const int64_t node = a.node0 + nl;
-            const int64_t seg0 = a.ev.ptr[node], seg1 = any_op ? a.ev.ptr[node + 1] : seg0;
+            const int64_t seg0 = cx0, seg1 = any_op ? cx1 : cx0;
+            cp_.step(gridDim.x, a.n_nodes);
+            if (item + gridDim.x < total) {     // the next item's bounds, requested one item ahead
+                const int64_t nn = a.node0 + cp_.nl;
+                cx0 = a.ev.ptr[nn]; cx1 = a.ev.ptr[nn + 1];
+            }
             if (set != cur_set && seg1 > seg0) {     // entry and sparse-term tables of the set
                 compute_sync();
                 for (int i = tid; i < S.nent; i += NCW * 32) sEnt[i] = a.ents[S.ent_begin + i];
