@@ -419,23 +419,28 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                                 const int s = (mt * 128 + row0) >> lg;
                                 const bool rv = s < d_src;
                                 const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
-                                for (int cl = c_lo; cl < c_hi; ++cl) {
-                                    const int ent = ent_u + cl * d_src + s;
-                                    const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
-                                    float gm = 0.f;
+                                // 16 accumulator columns per TMEM load: two components at KP = 8, one at KP = 16
+                                constexpr int CPL = 16 / KP;
+                                for (int cl = c_lo; cl < c_hi; cl += CPL) {
+                                    float v[16];
+                                    const bool full = cl + CPL <= c_hi;        // warp-uniform
+                                    if (full) tc_ld16(t0 + (uint32_t)(mt * npad + cl * KP), v);
+                                    else tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP), v);
 #pragma unroll
-                                    for (int q8 = 0; q8 < KP; q8 += 8) {
-                                        float v[8];
-                                        tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP + q8), v);
+                                    for (int c2 = 0; c2 < CPL; ++c2) {
+                                        if (c2 > 0 && !full) break;
+                                        const int ent = ent_u + (cl + c2) * d_src + s;
+                                        const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
                                         if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
+                                            float gm = 0.f;
 #pragma unroll
-                                            for (int x = 0; x < 8; ++x) {
-                                                gm = fmaf(aw[q8 + x], v[x], gm);
-                                                pphi[q8 + x] = fmaf(mw, v[x], pphi[q8 + x]);
+                                            for (int x = 0; x < KP; ++x) {
+                                                gm = fmaf(aw[x], v[c2 * KP + x], gm);
+                                                pphi[x] = fmaf(mw, v[c2 * KP + x], pphi[x]);
                                             }
+                                            sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                                         }
                                     }
-                                    if (rv) sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                                 }
                             }
                             tc_fence_before();
