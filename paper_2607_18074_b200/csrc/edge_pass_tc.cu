@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int NRAW = DUAL ? 2 : 1;     // raw stages: phi and Y, plus their directions
-    const int tb = a.tb, lg = a.lg, PS = a.tb + 4, EG = group_edges(a.tb);
+    const int tb = a.tb, lg = a.lg, PS = a.tb + 4;
     const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh, tb) * 4 + 1023) & ~1023);
     const uint32_t stage_bytes = (uint32_t)(2 * a.x_cap) + raw_bytes;
     uint8_t* sRing = smem;                                     // stages: Xh Xl raw
@@ -123,9 +123,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     float* sdM = sM + (size_t)a.nent * PS;                     // DUAL
     float* sGM = sdM + (DUAL ? (size_t)a.nent * PS : 0);       // [nent][PS]
     float* sPphi = sGM + (size_t)a.nent * PS;                  // [NCW*32][KP]: one row per compute thread
-    float* accPhi = sPphi + NCW * 32 * KP;                     // [EG][KP]
-    float* accY = accPhi + EG * KP;                            // [EG][dsh]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(accY + ((EG * a.dsh + 1) & ~1));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sPphi + NCW * 32 * KP);
     // bars: full[NS], free[NS], zfull, zfree, acc_full[2], acc_free[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
     UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [nunit]
@@ -346,16 +344,15 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         const int row0 = quarter * 32 + lane;        // this thread's accumulator row inside a 128-row tile
         const int e = row0 & (tb - 1);               // its edge (the same in every tile: 128 is a multiple of tb)
         const int t8 = tb >> 3;                      // 8-edge octets per batch
+        // bounds of the next receiver, requested one receiver ahead
+        int64_t nx0 = 0, nx1 = 0;
+        if ((int64_t)blockIdx.x < a.n_nodes) { nx0 = a.row_ptr[a.node0 + blockIdx.x]; nx1 = a.row_ptr[a.node0 + blockIdx.x + 1]; }
         for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
-            const int64_t node = a.node0 + nl;
-            const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
-            for (int64_t g0 = seg0; g0 < seg1; g0 += EG) {
-                const int64_t g1 = min(seg1, g0 + EG);
-                compute_sync();     // the previous group's outputs have been written
-                for (int i = tid; i < EG * KP; i += NCW * 32) accPhi[i] = 0.f;
-                for (int i = tid; i < EG * a.dsh; i += NCW * 32) accY[i] = 0.f;
-                for (int64_t b0 = g0; b0 < g1; b0 += tb) {
-                    const int bg = (int)(b0 - g0);           // first edge of the batch inside the group
+            const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
+            if (nl + gridDim.x < a.n_nodes) { nx0 = a.row_ptr[a.node0 + nl + gridDim.x]; nx1 = a.row_ptr[a.node0 + nl + gridDim.x + 1]; }
+            {
+                for (int64_t b0 = seg0; b0 < seg1; b0 += tb) {
+                    const int nb = (int)min((int64_t)tb, seg1 - b0);     // edges of the batch
                     float pphi[KP];
 #pragma unroll
                     for (int q = 0; q < KP; ++q) pphi[q] = 0.f;
@@ -451,45 +448,34 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
 #pragma unroll
                     for (int q = 0; q < KP; ++q) sPphi[tid * KP + q] = pphi[q];
                     compute_sync();
-                    // ---- fixed-order reductions into the group's accumulators: the threads that share an edge
-                    // are those whose row is congruent to it modulo tb, in both column halves
-                    for (int i = tid; i < tb * KP; i += NCW * 32) {
-                        const int ee = i / KP, q = i - ee * KP;
-                        float v = 0.f;
-                        for (int r = ee; r < 128; r += tb) v += sPphi[r * KP + q] + sPphi[(128 + r) * KP + q];
-                        accPhi[(bg + ee) * KP + q] += v;
-                    }
-                    for (int i = tid; i < t8 * a.dsh; i += NCW * 32) {
-                        const int b = i / t8, o8 = 8 * (i - b * t8);
-                        float g[8];
-#pragma unroll
-                        for (int x = 0; x < 8; ++x) g[x] = 0.f;
-                        for (int k = sInvPtr[b]; k < sInvPtr[b + 1]; ++k) {
-                            const NzS t = sInv[k];
-                            float gm[8];
-                            *reinterpret_cast<float4*>(gm) = *reinterpret_cast<const float4*>(sGM + t.b * PS + o8);
-                            *reinterpret_cast<float4*>(gm + 4) = *reinterpret_cast<const float4*>(sGM + t.b * PS + o8 + 4);
-#pragma unroll
-                            for (int x = 0; x < 8; ++x) g[x] = fmaf(t.coef, gm[x], g[x]);
+                    // ---- fixed-order reductions, written straight to the outputs: every (edge, q) and (edge, b) of the
+                    // batch is produced here exactly once per launch (edge id = position in the receiver-sorted order).
+                    // The threads that share an edge are those whose row is congruent to it modulo tb, in both column halves.
+                    if (a.phi_mode)
+                        for (int i = tid; i < tb * KP; i += NCW * 32) {
+                            const int ee = i / KP, q = i - ee * KP;
+                            if (ee < nb && q < a.K) {
+                                float v = 0.f;
+                                for (int r = ee; r < 128; r += tb) v += sPphi[r * KP + q] + sPphi[(128 + r) * KP + q];
+                                float* p = a.gphi + (b0 + ee) * a.K + q;
+                                *p = a.phi_mode == 2 ? *p + v : v;
+                            }
                         }
-#pragma unroll
-                        for (int x = 0; x < 8; ++x) accY[(bg + o8 + x) * a.dsh + b] += g[x];
-                    }
+                    // gY: thread <-> (b, edge); the sparse terms of b are the same for the lanes that share it
+                    if (a.Y_mode)
+                        for (int i = tid; i < a.dsh * tb; i += NCW * 32) {
+                            const int b = i >> lg, ee = i & (tb - 1);
+                            if (ee < nb) {
+                                float g = 0.f;
+                                for (int k = sInvPtr[b]; k < sInvPtr[b + 1]; ++k) {
+                                    const NzS t = sInv[k];
+                                    g = fmaf(t.coef, sGM[t.b * PS + ee], g);
+                                }
+                                float* p = a.gY + (b0 + ee) * a.dsh + b;
+                                *p = a.Y_mode == 2 ? *p + g : g;
+                            }
+                        }
                 }
-                compute_sync();
-                // ---- outputs of the group (edge id = position in the receiver-sorted order)
-                const int ng = (int)(g1 - g0);
-                if (a.phi_mode)
-                    for (int i = tid; i < ng * a.K; i += NCW * 32) {
-                        const int ee = i / a.K, q = i - ee * a.K;
-                        float* p = a.gphi + (g0 + ee) * a.K + q;
-                        *p = (a.phi_mode == 2 ? *p : 0.f) + accPhi[ee * KP + q];
-                    }
-                if (a.Y_mode)
-                    for (int i = tid; i < ng * a.dsh; i += NCW * 32) {
-                        float* p = a.gY + g0 * a.dsh + i;
-                        *p = (a.Y_mode == 2 ? *p : 0.f) + accY[i];
-                    }
             }
         }
     }
@@ -505,10 +491,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
 // shared bytes of a launch
 int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent, int nunit, int ncomp, int nnz, int ninv) {
     const int nop = dual ? 2 : 1;
-    const int PS = tb + 4, EG = group_edges(tb);
+    const int PS = tb + 4;
     const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
-    const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)EG * KP +
-                        (size_t)((EG * dsh + 1) & ~1);
+    const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP;
     const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
                        (nnz + ninv) * (int)sizeof(NzS) + (dsh + 2) * 4;
     return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
