@@ -41,7 +41,6 @@ constexpr int NCW = 8;          // compute warps
 constexpr int NLW = 2;          // loader warps
 constexpr int TT = (NCW + NLW + 1) * 32;
 constexpr int NS = 2;           // ring stages
-constexpr int EGMIN = 64;       // edges per output group: max(EGMIN, tb)
 
 struct EtArgs {
     const TSet* sets;
@@ -106,7 +105,6 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
     const int n = dual ? 2 : 1;
     return n * tb * KP + n * dsh * (tb + 4) + tb;
 }
-__host__ __device__ inline int group_edges(int tb) { return tb > EGMIN ? tb : EGMIN; }
 
 template <int KP, bool DUAL>
 __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
