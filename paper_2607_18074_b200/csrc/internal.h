@@ -153,6 +153,7 @@ struct TcSets {
     int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
+    int32_t concat = 0;               // stream: the lo copy of the gathered rows sits beside the hi copy (see stream_tc.cu)
     int32_t smem_bytes = 0, ctas_per_sm = 1;
 };
 

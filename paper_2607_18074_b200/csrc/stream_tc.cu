@@ -67,6 +67,7 @@ struct TcArgs {
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
     int32_t a_cap, b_cap, max_ent, tmem_cols, acc_cols, n_units, n_blks, n_comps, max_nz;
+    int32_t concat;        // 1: multiplicities <= 32, the lo copy of a gathered row sits 32 columns beside the hi copy
     int* status;
 };
 
@@ -86,6 +87,7 @@ struct UInfo {     // a unit, as the MMA thread and the drain need it
     // operand descriptors of slab 0 (hi copies; stage 0 of the ring for B): the other slabs, copies and stages differ
     // only in the 16-byte-granular address field, so the MMA thread reaches them with one addition each
     uint64_t dA0, dB0;
+    uint32_t idesc_wide, pad2;   // concat: the same instruction with N = 64 columns ([B_hi | B_lo])
 };
 // shared-memory operand descriptor without swizzle (K-major core matrices of 8 rows x 16 bytes)
 __device__ __forceinline__ uint64_t make_desc_none(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -205,6 +207,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         u.b_off = (uint32_t)B.b_off; u.slab_bytes = (uint32_t)B.slab_bytes; u.d_src = (uint32_t)B.d_src;
         u.comp_begin = (uint32_t)U.comp_begin; u.ncomp = (uint32_t)U.ncomp; u.c_src = (uint32_t)B.c_src;
         u.ncols = (uint32_t)B.ncols; u.pad = 0;
+        u.idesc_wide = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        u.pad2 = 0;
         u.dA0 = make_desc_none(smem_u32(sA) + u.a_off, 128, 256);
         u.dB0 = make_desc(smem_u32(sRing) + u.b_off, 2048, 1024);
         sU[i] = u;
@@ -336,10 +340,13 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                         uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + re * 128 + ((((u & 63) >> 3) ^ (re & 7)) << 4));
                         const __nv_bfloat16* ph = srch + B.src_off + u;
                         const __nv_bfloat16* pl = srcl + B.src_off + u;
+                        // the lo copy: a slab of its own, or (concat) columns 32.. of the same swizzled row
+                        uint32_t dl = a.concat ? stage_u + (uint32_t)(B.b_off + re * 128 + ((((u >> 3) + 4) ^ (re & 7)) << 4))
+                                               : d + (uint32_t)a.b_cap;
                         for (int sdx = 0; sdx < B.d_src; ++sdx) {
                             cp_async16_zfill(d, ph, ok);
-                            cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
-                            d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                            cp_async16_zfill(dl, pl, ok);
+                            d += (uint32_t)B.slab_bytes; dl += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
                         }
                     }
                 }
@@ -381,6 +388,20 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                             const uint32_t idesc = U.idesc, nslab = U.d_src;
                             const uint64_t sa16 = U.slab_stride >> 4, sb16 = U.slab_bytes >> 4;
                             uint64_t dAh = U.dA0, dBh = U.dB0 + st16;
+                            if (a.concat) {
+                                // two instructions per slab instead of three: A_hi x [B_hi | B_lo] (64 columns; the second
+                                // 32 are summed into the first at the drain) and A_lo x B_hi.  An MMA of up to 64 columns
+                                // costs the same fixed time, so this takes a third off the tensor-pipe time.
+                                const uint32_t iw = U.idesc_wide;
+                                tc_mma_bf16(d_tmem, dAh, dBh, iw, acc0);
+                                tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
+                                for (uint32_t s = 1; s < nslab; ++s) {
+                                    dAh += sa16; dBh += sb16;
+                                    tc_mma_bf16(d_tmem, dAh, dBh, iw, 1u);
+                                    tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
+                                }
+                                continue;
+                            }
                             tc_mma_bf16(d_tmem, dAh, dBh, idesc, acc0);
                             tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
                             tc_mma_bf16(d_tmem, dAh, dBh + bcap16, idesc, 1u);
@@ -433,8 +454,15 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 if ((hc & 15) == 0) {              // 16 columns per TMEM load: half as many load round trips
                     for (int cc = half * hc; cc < (half + 1) * hc; cc += 16) {
                         float v[16];
-                        if (wrote) tc_ld16(trow + (uint32_t)cc, v);
-                        else {
+                        if (wrote) {
+                            tc_ld16(trow + (uint32_t)cc, v);
+                            if (a.concat) {     // + A_hi x B_lo, accumulated 32 columns further on
+                                float w[16];
+                                tc_ld16(trow + 32u + (uint32_t)cc, w);
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) v[i] += w[i];
+                            }
+                        } else {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) v[i] = 0.f;
                         }
@@ -451,8 +479,15 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 } else {
                     for (int cc = half * hc; cc < (half + 1) * hc; cc += 8) {
                         float v[8];
-                        if (wrote) tc_ld8(trow + (uint32_t)cc, v);
-                        else {
+                        if (wrote) {
+                            tc_ld8(trow + (uint32_t)cc, v);
+                            if (a.concat) {
+                                float w[8];
+                                tc_ld8(trow + 32u + (uint32_t)cc, w);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) v[i] += w[i];
+                            }
+                        } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) v[i] = 0.f;
                         }
@@ -648,7 +683,11 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
         auto unit_a = [&](const Cand& c) { return blocks[c.blk].d_src * (c.nc * KP) * 32; };
         auto blk_b = [&](int b) { return blocks[b].d_src * 2048 * ((blocks[b].c_src + 63) / 64); };
         auto ncols = [&](int b) { return (blocks[b].c_src + 15) & ~15; };
-        auto cols32 = [&](int b) { return (ncols(b) + 31) & ~31; };
+        // with every multiplicity <= 32 the lo copy of a gathered row fits beside the hi copy inside one 64-column
+        // swizzle row: [B_hi | B_lo] is then one 64-column operand and a tile takes 64 accumulator columns
+        bool concat = true;
+        for (const Blk& b : blocks) concat = concat && b.c_src <= 32;
+        auto cols32 = [&](int b) { return concat ? 64 : (ncols(b) + 31) & ~31; };
         auto cand_nz = [&](const Cand& c) {
             int n = 0;
             for (int cl = 0; cl < c.nc; ++cl) {
@@ -739,6 +778,7 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
             T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size(), (int)cands.size(), n_comps_total, T.max_nz);
             if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
             T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
+            T.concat = concat ? 1 : 0;
             // shared-memory images of the tables
             for (TSet& S : T.sets) {
                 S.b_items = (int)T.nz.size();
@@ -771,7 +811,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
-    a.a_cap = T.a_cap; a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols; a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
+    a.a_cap = T.a_cap; a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols; a.concat = T.concat; a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
     a.status = status;
     const bool k8 = p->K <= 8;
     void (*kern)(const TcArgs) = k8 ? (dual ? k_stream_tc<8, true> : k_stream_tc<8, false>)
