@@ -75,7 +75,8 @@ typedef struct sobek_plan sobek_plan; /* opaque; host-owned; immutable after cre
 enum { SOBEK_MAX_L = 4 };
 
 /* plan flags */
-#define SOBEK_FLAG_UVU 1u   /* channelwise multiplicity mode, Eq. uvu_connection */
+#define SOBEK_FLAG_UVU 1u      /* channelwise multiplicity mode, Eq. uvu_connection */
+#define SOBEK_FLAG_MUL_IR 2u   /* node features cross the boundary in mul_ir order (see sobek_plan_create) */
 
 /*
  * sobek_plan_create -- the static contract of one layer (Section "Generated
@@ -89,6 +90,11 @@ enum { SOBEK_MAX_L = 4 };
  * mode (Eq. uvu_connection: output multiplicity tied to the input one, C_in weights per path, column
  * w_off + u; N_w = sum of C_in over the paths; a path between blocks of different multiplicity makes the
  * call fail with UNSUPPORTED).  Every other argument, layout and entry point is the same in both modes.
+ * SOBEK_FLAG_MUL_IR (may be combined with the above) selects the mul_ir order for every node feature array
+ * at the boundary (x, y, gy, gx, vx, ggy, hx): inside an irrep block of multiplicity C the element (u, m) sits at
+ * u*(2l+1) + m instead of m*C + u (Section "Generated deterministic runtime and execution contracts": the kernels
+ * work in ir_mul, the other order is transposed at the boundary).  The calls then re-lay the arrays through the
+ * workspace, which grows by 4 bytes per node feature and array; Y, phi and R are unaffected.
  * If the environment variable SOBEK_FUSED is set to a
  * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
  * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise

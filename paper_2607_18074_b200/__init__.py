@@ -16,7 +16,8 @@ from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsobek.so")
 
-FLAG_UVU = 1   # SOBEK_FLAG_UVU: channelwise multiplicity mode
+FLAG_UVU = 1      # SOBEK_FLAG_UVU: channelwise multiplicity mode
+FLAG_MUL_IR = 2   # SOBEK_FLAG_MUL_IR: node features cross the boundary in mul_ir order
 
 EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
@@ -129,13 +130,21 @@ def _irreps(seq):
 
 class Plan:
     """sobek_plan: irreps are sequences of (mul, l, parity) with parity +1 / -1.  mode "uvw" is the fully
-    connected multiplicity mixing, "uvu" the channelwise one (SOBEK_FLAG_UVU)."""
+    connected multiplicity mixing, "uvu" the channelwise one (SOBEK_FLAG_UVU).  layout "ir_mul" (block offset +
+    m*mul + u) is the kernels' own order of node features, "mul_ir" (block offset + u*(2l+1) + m) is transposed at the
+    boundary (SOBEK_FLAG_MUL_IR)."""
 
-    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0, mode: str = "uvw"):
+    def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0, mode: str = "uvw",
+                 layout: str = "ir_mul"):
         if mode not in ("uvw", "uvu"):
             raise ValueError(mode)
+        if layout not in ("ir_mul", "mul_ir"):
+            raise ValueError(layout)
         if mode == "uvu":
             flags |= FLAG_UVU
+        if layout == "mul_ir":
+            flags |= FLAG_MUL_IR
+        self.layout = "mul_ir" if flags & FLAG_MUL_IR else "ir_mul"
         self.mode = "uvu" if flags & FLAG_UVU else "uvw"
         self._h = c_void_p()
         a, b = _irreps(irreps_in), _irreps(irreps_out)

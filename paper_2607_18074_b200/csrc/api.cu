@@ -29,6 +29,8 @@ struct Workspace {
     // bf16 (hi, lo) copies of x, gy and vx, [N][C] each: the gathered operand of the tensor-core stream
     uint16_t *xsh, *xsl, *gsh, *gsl, *vsh, *vsl;
     uint16_t *zqh, *zql;      // bf16 (hi, lo) adjoint state of one chunk (input of the tensor-core edge pass)
+    // mul_ir plans: ir_mul copies of the node feature arrays of a call (inputs x, gy, vx; outputs on C_y, on C_x)
+    float *lx, *lgy, *lvx, *ly, *lgx;
     int64_t chunk;
     size_t bytes;
 };
@@ -47,6 +49,10 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     if (w.fused_t && order >= 2) { w.vtFKh = (uint16_t*)take(p->tr.fk_elems * 2); w.vtFKl = (uint16_t*)take(p->tr.fk_elems * 2); }
     if (order == 0 && w.fused_f) {   // the forward needs nothing else: the state stays on chip
         w.chunk = 0;
+        if (p->mul_ir) {
+            w.lx = (float*)take((size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 4);
+            w.ly = (float*)take((size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 4);
+        }
         w.bytes = off;
         return w;
     }
@@ -88,6 +94,13 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         if (p->fwd.tc[0].ok || (order >= 2 && p->fwd.tc[1].ok) || (order >= 1 && w.zqh)) { w.xsh = (uint16_t*)take(nx); w.xsl = (uint16_t*)take(nx); }
         if (order >= 1 && (p->tr.tc[0].ok || (order >= 2 && p->tr.tc[1].ok))) { w.gsh = (uint16_t*)take(ny); w.gsl = (uint16_t*)take(ny); }
         if (order >= 2 && (p->fwd.tc[1].ok || (w.zqh && p->fwd.etc[1].ok))) { w.vsh = (uint16_t*)take(nx); w.vsl = (uint16_t*)take(nx); }
+    }
+    if (p->mul_ir) {
+        const size_t nx = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 4, ny = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 4;
+        w.lx = (float*)take(nx);
+        w.ly = (float*)take(ny);            // y (order 0), ggy (order 2)
+        if (order >= 1) { w.lgy = (float*)take(ny); w.lgx = (float*)take(nx); }
+        if (order >= 2) w.lvx = (float*)take(nx);
     }
     w.bytes = off;
     return w;
@@ -274,9 +287,10 @@ extern "C" int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_pt
     return graph_receivers(N, E, row_ptr, src_perm, src_recv, (cudaStream_t)stream);
 }
 
-extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
-                              const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
-                              void* stream) {
+namespace {
+int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                  const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
+                  void* stream) {
     int rc = check_common(p, g, ws, ws_bytes, 0);
     if (rc) return rc;
     if (!y || !R || (g->N > 0 && !x) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
@@ -303,9 +317,9 @@ extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const f
     return SOBEK_OK;
 }
 
-extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
-                              const float* phi, const float* R, const float* gy, float* gx, float* gY,
-                              float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream) {
+int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                  const float* phi, const float* R, const float* gy, float* gx, float* gY,
+                  float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_common(p, g, ws, ws_bytes, 1);
     if (rc) return rc;
     if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
@@ -366,11 +380,11 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     return SOBEK_OK;
 }
 
-extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
-                               const float* phi, const float* R, const float* gy, const float* vx,
-                               const float* vY, const float* vphi, const float* vR, float* ggy,
-                               float* hx, float* hY, float* hphi, float* hR, void* ws, size_t ws_bytes,
-                               void* stream) {
+int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                   const float* phi, const float* R, const float* gy, const float* vx,
+                   const float* vY, const float* vphi, const float* vR, float* ggy,
+                   float* hx, float* hY, float* hphi, float* hR, void* ws, size_t ws_bytes,
+                   void* stream) {
     int rc = check_common(p, g, ws, ws_bytes, 2);
     if (rc) return rc;
     if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
@@ -508,6 +522,86 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
         }
     }
     return SOBEK_OK;
+}
+
+// ---- boundary layout: a mul_ir plan re-lays the node feature arrays through the workspace around the ir_mul core
+struct Relay {
+    const sobek_plan* p; int64_t N; cudaStream_t s;
+    // ir_mul copy of an input on C_x (in = 1) or C_y columns; NULL stays NULL
+    int in_x(const float* src, float* tmp, const float** out) const {
+        *out = src;
+        if (!src || !p->mul_ir) return SOBEK_OK;
+        CK(launch_relayout(src, tmp, N, p->C_x, p->d_in_blocks, (int)p->in.size(), 1, s));
+        *out = tmp; return SOBEK_OK;
+    }
+    int in_y(const float* src, float* tmp, const float** out) const {
+        *out = src;
+        if (!src || !p->mul_ir) return SOBEK_OK;
+        CK(launch_relayout(src, tmp, N, p->C_y, p->d_out_blocks, (int)p->out.size(), 1, s));
+        *out = tmp; return SOBEK_OK;
+    }
+    int out_x(const float* tmp, float* dst) const {
+        if (!dst || !p->mul_ir) return SOBEK_OK;
+        CK(launch_relayout(tmp, dst, N, p->C_x, p->d_in_blocks, (int)p->in.size(), 0, s));
+        return SOBEK_OK;
+    }
+    int out_y(const float* tmp, float* dst) const {
+        if (!dst || !p->mul_ir) return SOBEK_OK;
+        CK(launch_relayout(tmp, dst, N, p->C_y, p->d_out_blocks, (int)p->out.size(), 0, s));
+        return SOBEK_OK;
+    }
+};
+}  // namespace
+
+extern "C" int sobek_conv_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                              const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
+                              void* stream) {
+    if (!p || !p->mul_ir) return conv_fwd_core(p, g, x, Y, phi, R, y, ws, ws_bytes, stream);
+    int rc = check_common(p, g, ws, ws_bytes, 0);
+    if (rc) return rc;
+    if (!y || (g->N > 0 && !x)) return SOBEK_ERR_INVALID_ARG;
+    const Workspace w = carve(p, g->N, 0, ws);
+    const Relay r{p, g->N, (cudaStream_t)stream};
+    const float* xi;
+    if ((rc = r.in_x(x, w.lx, &xi))) return rc;
+    if ((rc = conv_fwd_core(p, g, xi, Y, phi, R, w.ly, ws, ws_bytes, stream))) return rc;
+    return r.out_y(w.ly, y);
+}
+
+extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                              const float* phi, const float* R, const float* gy, float* gx, float* gY,
+                              float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream) {
+    if (!p || !p->mul_ir) return conv_bwd_core(p, g, x, Y, phi, R, gy, gx, gY, gphi, gR, ws, ws_bytes, stream);
+    int rc = check_common(p, g, ws, ws_bytes, 1);
+    if (rc) return rc;
+    if (g->N > 0 && (!x || !gy)) return SOBEK_ERR_INVALID_ARG;
+    const Workspace w = carve(p, g->N, 1, ws);
+    const Relay r{p, g->N, (cudaStream_t)stream};
+    const float *xi, *gyi;
+    if ((rc = r.in_x(x, w.lx, &xi)) || (rc = r.in_y(gy, w.lgy, &gyi))) return rc;
+    if ((rc = conv_bwd_core(p, g, xi, Y, phi, R, gyi, gx ? w.lgx : nullptr, gY, gphi, gR, ws, ws_bytes, stream))) return rc;
+    return r.out_x(w.lgx, gx);
+}
+
+extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                               const float* phi, const float* R, const float* gy, const float* vx,
+                               const float* vY, const float* vphi, const float* vR, float* ggy,
+                               float* hx, float* hY, float* hphi, float* hR, void* ws, size_t ws_bytes,
+                               void* stream) {
+    if (!p || !p->mul_ir)
+        return conv_dbwd_core(p, g, x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi, hR, ws, ws_bytes, stream);
+    int rc = check_common(p, g, ws, ws_bytes, 2);
+    if (rc) return rc;
+    if (g->N > 0 && (!x || !gy)) return SOBEK_ERR_INVALID_ARG;
+    const Workspace w = carve(p, g->N, 2, ws);
+    const Relay r{p, g->N, (cudaStream_t)stream};
+    const float *xi, *gyi, *vxi;
+    if ((rc = r.in_x(x, w.lx, &xi)) || (rc = r.in_y(gy, w.lgy, &gyi)) || (rc = r.in_x(vx, w.lvx, &vxi))) return rc;
+    if ((rc = conv_dbwd_core(p, g, xi, Y, phi, R, gyi, vxi, vY, vphi, vR, ggy ? w.ly : nullptr, hx ? w.lgx : nullptr, hY, hphi,
+                             hR, ws, ws_bytes, stream)))
+        return rc;
+    if ((rc = r.out_y(w.ly, ggy))) return rc;
+    return r.out_x(w.lgx, hx);
 }
 
 extern "C" int sobek_last_device_status(void* ws, void* stream) {

@@ -236,6 +236,9 @@ struct sobek_plan {
     bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
     bool use_tc_edge = true;     // edge pass on the tensor cores where the profile allows it
     size_t state_budget = size_t(2048) << 20;   // bytes of receiver / sender state held at once (the scratch budget)
+    bool mul_ir = false;      // node features cross the boundary in mul_ir order and are re-laid through the workspace
+    int4* d_in_blocks = nullptr;    // {offset, multiplicity, 2l+1, 0} of the irrep blocks of x / of y (device), for the re-layout
+    int4* d_out_blocks = nullptr;
     bool uvu = false;         // channelwise mode (Eq. uvu_connection): tied multiplicities, C_in weights per path
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
@@ -308,6 +311,9 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
                              float* gY, int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
                              cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
+// [N][C] node features between the two block orders: to_ir_mul = 1: dst[m*C_b + u] = src[u*d + m] inside every block
+cudaError_t launch_relayout(const float* src, float* dst, int64_t N, int C, const int4* blocks, int nblk, int to_ir_mul,
+                            cudaStream_t s);
 
 // --- edge_stream.cu ---------------------------------------------------------------
 void build_stream_tasks(const sobek_plan* p, Direction& dir);

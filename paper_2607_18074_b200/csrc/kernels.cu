@@ -157,6 +157,35 @@ cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+namespace {
+// one thread per element of the ir_mul side (block offset + m*c + u); the mul_ir partner is block offset + u*d + m
+__global__ void k_relayout(const float* __restrict__ src, float* __restrict__ dst, int64_t N, int C,
+                           const int4* __restrict__ blocks, int nblk, int to_ir_mul) {
+    const int64_t total = N * C;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t n = i / C;
+        const int col = (int)(i - n * C);
+        int b = 0;
+        while (b + 1 < nblk && blocks[b + 1].x <= col) ++b;
+        const int4 B = blocks[b];
+        const int r = col - B.x, m = r / B.y, u = r - m * B.y;      // ir_mul position inside the block
+        const int64_t other = n * C + B.x + u * B.z + m;
+        if (to_ir_mul) dst[i] = src[other];
+        else dst[other] = src[i];
+    }
+}
+}  // namespace
+
+cudaError_t launch_relayout(const float* src, float* dst, int64_t N, int C, const int4* blocks, int nblk, int to_ir_mul,
+                            cudaStream_t s) {
+    if (N <= 0 || C <= 0) return cudaSuccess;
+    const int nb = (int)std::min<int64_t>((N * C + 255) / 256, 148 * 16);
+    KernelTimer kt(K_PACK, s);
+    k_relayout<<<nb, 256, 0, s>>>(src, dst, N, C, blocks, nblk, to_ir_mul);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const float* Rp, float* R,
                             cudaStream_t s) {
     dim3 grid(32, (unsigned)dir.paths.size());

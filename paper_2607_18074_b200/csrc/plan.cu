@@ -385,7 +385,7 @@ using namespace sobek;
 
 extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
                                  int l_max, int K, uint32_t flags, sobek_plan** plan) {
-    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU)) != 0 || l_max < 0)
+    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR)) != 0 || l_max < 0)
         return SOBEK_ERR_INVALID_ARG;
     *plan = nullptr;
     if (l_max > SOBEK_MAX_L) return SOBEK_ERR_UNSUPPORTED;
@@ -404,6 +404,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     p->l_max = l_max;
     p->K = K;
     p->uvu = (flags & SOBEK_FLAG_UVU) != 0;
+    p->mul_ir = (flags & SOBEK_FLAG_MUL_IR) != 0;
     p->dim_sh = (l_max + 1) * (l_max + 1);
     std::vector<int> in_off(n_in), out_off(n_out);
     for (int i = 0; i < n_in; ++i) { in_off[i] = p->C_x; p->C_x += in[i].mul * (2 * in[i].l + 1); }
@@ -480,6 +481,13 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     if (e == cudaSuccess) e = upload(p->tab_ptr, &p->d_tab_ptr);
     if (e == cudaSuccess) e = upload(p->tab_idx, &p->d_tab_idx);
     if (e == cudaSuccess) e = upload(p->tab_coef, &p->d_tab_coef);
+    {
+        std::vector<int4> bi, bo;
+        for (int i = 0; i < n_in; ++i) bi.push_back(make_int4(in_off[i], in[i].mul, 2 * in[i].l + 1, 0));
+        for (int i = 0; i < n_out; ++i) bo.push_back(make_int4(out_off[i], out[i].mul, 2 * out[i].l + 1, 0));
+        if (e == cudaSuccess) e = upload(bi, &p->d_in_blocks);
+        if (e == cudaSuccess) e = upload(bo, &p->d_out_blocks);
+    }
     for (Direction* d : {&p->fwd, &p->tr}) {
         if (e == cudaSuccess) e = upload(d->paths, &d->d_paths);
         if (e == cudaSuccess) e = upload(d->groups, &d->d_groups);
@@ -540,6 +548,7 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
     }
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     cudaFree(p->d_tab_ptr); cudaFree(p->d_tab_idx); cudaFree(p->d_tab_coef);
+    cudaFree(p->d_in_blocks); cudaFree(p->d_out_blocks);
     for (Direction* d : {&p->fwd, &p->tr}) {
         cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);
         cudaFree(d->d_kn_off); cudaFree(d->d_nk_off); cudaFree(d->d_kn_ld); cudaFree(d->d_nk_ld); cudaFree(d->d_path_group);

@@ -37,7 +37,7 @@ extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, 
     if (!y || !R || (g->N > 0 && (!x || !g->row_ptr)) || (g->E > 0 && (!Y || !phi || !g->col)))
         return SOBEK_ERR_INVALID_ARG;
     if (p->device < 0) return SOBEK_ERR_CUDA;
-    if (p->uvu) return SOBEK_ERR_UNSUPPORTED;   // this entry point covers the fully connected mode only
+    if (p->uvu || p->mul_ir) return SOBEK_ERR_UNSUPPORTED;   // this entry point covers the fully connected mode in ir_mul order only
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         (void)cudaGetLastError();

@@ -453,3 +453,56 @@ def test_uvu_plan_contract():
     assert sb.Plan(ir, ir, 3, 16, mode="uvu").info.N_w == 1472          # Table uvu_capacity_matched
     with pytest.raises(sb.SobekError):
         sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")      # 0e x 1o -> 1o would tie 8 to 4
+
+
+# ---------------------------------------------------------------------------------------
+# mul_ir boundary layout (SOBEK_FLAG_MUL_IR): the same operator with node features transposed per block
+# ---------------------------------------------------------------------------------------
+def _to_mul_ir(a, irreps):
+    """[N, C] in ir_mul order (block offset + m*c + u) -> mul_ir order (block offset + u*d + m)."""
+    out = np.empty_like(a)
+    o = 0
+    for c, l, _ in irreps:
+        d = 2 * l + 1
+        out[:, o:o + c * d] = a[:, o:o + c * d].reshape(-1, d, c).transpose(0, 2, 1).reshape(-1, c * d)
+        o += c * d
+    return out
+
+
+@pytest.mark.parametrize("name,mode", [("cfg2_N200", "uvw"), ("ragged", "uvw"), ("uvu_16x3", "uvu")])
+def test_mul_ir_layout(name, mode):
+    import torch
+    import paper_2607_18074_b200 as sb
+    w = (UVU if mode == "uvu" else CASES)[name]
+    ref = Case(w)                                   # ir_mul plan: outputs to compare with
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=mode, layout="mul_ir")
+    assert plan.layout == "mul_ir" and plan.info.N_w == ref.plan.info.N_w
+    d, i = ref.d, plan.info
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
+    x, gy, vx = t(_to_mul_ir(d.x, w.irreps_in)), t(_to_mul_ir(d.gy, w.irreps_out)), t(_to_mul_ir(d.vx, w.irreps_in))
+    ws = torch.empty(sb.workspace_bytes(plan, d.N, d.E, 2), dtype=torch.uint8, device="cuda:0")
+    assert ws.numel() > sb.workspace_bytes(ref.plan, d.N, d.E, 2)
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    y = new(d.N, i.C_y)
+    sb.conv_fwd(plan, ref.graph, x, ref.Y, ref.phi, ref.R, y, ws)
+    assert np.array_equal(y.cpu().numpy(), _to_mul_ir(ref.fwd(), w.irreps_out))       # same kernels, same bits
+    gx, gY, gphi, gR = new(d.N, i.C_x), new(d.E, i.dim_sh), new(d.E, i.K), new(i.K, i.N_w)
+    sb.conv_bwd(plan, ref.graph, x, ref.Y, ref.phi, ref.R, gy, gx, gY, gphi, gR, ws)
+    rb = ref.bwd()
+    assert np.array_equal(gx.cpu().numpy(), _to_mul_ir(rb[0], w.irreps_in))
+    for got, r in zip((gY, gphi, gR), rb[1:]):
+        assert np.array_equal(got.cpu().numpy(), r)
+    ggy, hx, hY, hphi, hR = new(d.N, i.C_y), new(d.N, i.C_x), new(d.E, i.dim_sh), new(d.E, i.K), new(i.K, i.N_w)
+    sb.conv_dbwd(plan, ref.graph, x, ref.Y, ref.phi, ref.R, gy, vx, ref.vY, ref.vphi, ref.vR, ggy, hx, hY, hphi, hR, ws)
+    rd = ref.dbwd()
+    assert np.array_equal(ggy.cpu().numpy(), _to_mul_ir(rd[0], w.irreps_out))
+    assert np.array_equal(hx.cpu().numpy(), _to_mul_ir(rd[1], w.irreps_in))
+    for got, r in zip((hY, hphi, hR), rd[2:]):
+        assert np.array_equal(got.cpu().numpy(), r)
+    assert sb.last_device_status(ws) == 0
+    # and against the oracle directly (forward), so that the layout itself is pinned, not only its consistency
+    assert rel_err(y.cpu().numpy(), _to_mul_ir(ref.o_fwd(), w.irreps_out)) <= FWD_TOL
+    # partial outputs through the re-layout: only hx
+    hx2 = new(d.N, i.C_x)
+    sb.conv_dbwd(plan, ref.graph, x, ref.Y, ref.phi, ref.R, gy, vx, ref.vY, ref.vphi, ref.vR, None, hx2, None, None, None, ws)
+    assert np.array_equal(hx2.cpu().numpy(), hx.cpu().numpy())

@@ -140,7 +140,7 @@ def test_uvu_plan_errors_and_workspace():
     with pytest.raises(sb.SobekError):
         sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")       # 0e x 1o -> 1o would tie 8 channels to 4
     with pytest.raises(sb.SobekError):
-        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=2)                    # unknown flag bit
+        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=4)                    # unknown flag bit
     ir = P("64x0e+64x1o+64x2e")
     u, w = sb.Plan(ir, ir, 2, 16, mode="uvu"), sb.Plan(ir, ir, 2, 16)
     assert u.mode == "uvu" and w.mode == "uvw" and u.info.C_y == w.info.C_y
@@ -148,3 +148,18 @@ def test_uvu_plan_errors_and_workspace():
         a = sb.workspace_bytes(u, 3125, 10**5, order)
         assert a == sb.workspace_bytes(u, 3125, 10**9, order)            # nothing edge-sized
         assert a <= sb.workspace_bytes(w, 3125, 10**5, order)            # no GEMM operand copies of R
+
+
+def test_mul_ir_flag_and_workspace():
+    P = synth.parse_irreps
+    ir = P("32x0e+32x1o+32x2e")
+    a, b = sb.Plan(ir, ir, 2, 8), sb.Plan(ir, ir, 2, 8, layout="mul_ir")
+    assert (a.layout, b.layout) == ("ir_mul", "mul_ir") and a.info.N_w == b.info.N_w
+    N = 5000
+    # the re-layout copies: x, y | + gy, gx | + vx   (4 bytes per node feature and array, 256-byte aligned)
+    al = lambda n: (n + 255) & ~255
+    cx = cy = a.info.C_x
+    extra = [al(4 * N * cx) + al(4 * N * cy), 2 * (al(4 * N * cx) + al(4 * N * cy)), 3 * al(4 * N * cx) + 2 * al(4 * N * cy)]
+    for order in (0, 1, 2):
+        assert sb.workspace_bytes(b, N, 10**5, order) - sb.workspace_bytes(a, N, 10**5, order) == extra[order]
+    assert sb.Plan(ir, ir, 2, 8, mode="uvu", layout="mul_ir").mode == "uvu"
