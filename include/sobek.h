@@ -230,6 +230,13 @@ int sobek_conv_fwd_static(const sobek_plan* plan, const sobek_graph* g,
                           const float* x, const float* Y, const float* phi, const float* R,
                           float* y, void* stream);
 
+/* Self-test of the bounded device-side waits: enqueues a one-thread kernel that waits on a barrier nothing ever
+ * completes.  The wait gives up after `limit_ms` (1..2000) milliseconds, writes SOBEK_ERR_DEVICE_TIMEOUT into the
+ * status word at the start of `ws` (at least 256 bytes, 256-byte aligned) and the kernel returns normally: the
+ * same code path every mbarrier wait of the tensor-core kernels takes if its partner never arrives.  Read the
+ * result with sobek_last_device_status.  Errors: INVALID_ARG, CUDA. */
+int sobek_selftest_wait_timeout(void* ws, unsigned limit_ms, void* stream);
+
 /* Synchronises `stream`, then returns the status word the kernels of earlier calls wrote
  * into `ws` (0, or SOBEK_ERR_DEVICE_TIMEOUT / SOBEK_ERR_GRAPH ...). */
 int sobek_last_device_status(void* ws, void* stream);

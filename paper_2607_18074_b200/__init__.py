@@ -24,7 +24,7 @@ EXPORTS = [
     "sobek_graph_prepare_bytes", "sobek_graph_prepare", "sobek_graph_receivers", "sobek_workspace_bytes", "sobek_conv_fwd",
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
-    "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static",
+    "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
 ]
 
 
@@ -266,6 +266,11 @@ def conv_dbwd(plan, graph, x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi
                                  _ptr(vx), _ptr(vY), _ptr(vphi), _ptr(vR), _ptr(ggy), _ptr(hx), _ptr(hY),
                                  _ptr(hphi), _ptr(hR), _ptr(ws), ws.numel() * ws.element_size(),
                                  _stream()), "sobek_conv_dbwd")
+
+
+def selftest_wait_timeout(ws, limit_ms: int = 200):
+    """Enqueue the bounded-wait self-test; read its result with last_device_status(ws)."""
+    _check(lib().sobek_selftest_wait_timeout(_ptr(ws), int(limit_ms), _stream()), "sobek_selftest_wait_timeout")
 
 
 def last_device_status(ws) -> int:

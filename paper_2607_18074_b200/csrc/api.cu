@@ -604,6 +604,14 @@ extern "C" int sobek_conv_dbwd(const sobek_plan* p, const sobek_graph* g, const 
     return r.out_x(w.lgx, hx);
 }
 
+extern "C" int sobek_selftest_wait_timeout(void* ws, unsigned limit_ms, void* stream) {
+    if (!ws || ((uintptr_t)ws & 255) || limit_ms == 0 || limit_ms > 2000) return SOBEK_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    CK(cudaMemsetAsync(ws, 0, kHeaderBytes, s));
+    CK(launch_wait_selftest((int*)ws, (uint64_t)limit_ms * 1000000ull, s));
+    return SOBEK_OK;
+}
+
 extern "C" int sobek_last_device_status(void* ws, void* stream) {
     if (!ws) return SOBEK_ERR_INVALID_ARG;
     int h = 0;

@@ -276,6 +276,25 @@ __global__ void k_reduce_parts(float* __restrict__ dst, const float* __restrict_
 }
 }  // namespace
 
+namespace {
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever completes; the wait gives up after
+// `limit_ns`, records SOBEK_ERR_DEVICE_TIMEOUT in the status word and the kernel returns normally.
+__global__ void k_wait_selftest(int* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0, status, limit_ns);
+    }
+}
+}  // namespace
+
+cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s) {
+    k_wait_selftest<<<1, 32, 0, s>>>(status, limit_ns);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s) {
     if (n <= 0 || splits <= 0) return cudaSuccess;
     const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);

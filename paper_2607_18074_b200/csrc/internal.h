@@ -404,6 +404,7 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
                            int64_t split_stride = 0, void* Chi = nullptr, void* Clo = nullptr);
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
+cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s);
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
 

@@ -36,7 +36,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  A healthy wait ends after a handful of polls; the limit (about two seconds of wall
 // time, checked every 64 polls) only exists so that a broken pipeline cannot wait for ever.  On give-up
 // the status word is set and the caller goes on.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status, uint64_t limit_ns = 2000000000ull) {
     if (mbar_try(bar, parity)) return;
     uint64_t t0;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
@@ -45,7 +45,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* st
         if ((it & 63u) == 0) {
             uint64_t t1;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-            if (t1 - t0 > 2000000000ull) break;
+            if (t1 - t0 > limit_ns) break;
         }
     }
     atomicExch(status, (int)SOBEK_ERR_DEVICE_TIMEOUT);

@@ -506,3 +506,20 @@ def test_mul_ir_layout(name, mode):
     hx2 = new(d.N, i.C_x)
     sb.conv_dbwd(plan, ref.graph, x, ref.Y, ref.phi, ref.R, gy, vx, ref.vY, ref.vphi, ref.vR, None, hx2, None, None, None, ws)
     assert np.array_equal(hx2.cpu().numpy(), hx.cpu().numpy())
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A device-side wait whose partner never arrives runs out after its limit, records DEVICE_TIMEOUT in the status
+    word and the kernel returns: the context stays usable (the next call computes correct results)."""
+    import time
+    import torch
+    import paper_2607_18074_b200 as sb
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda:0")
+    t0 = time.time()
+    sb.selftest_wait_timeout(ws, 200)
+    assert sb.last_device_status(ws) == -7            # SOBEK_ERR_DEVICE_TIMEOUT
+    dt = time.time() - t0
+    assert 0.15 < dt < 5.0
+    assert "timeout" in sb.status_string(-7).lower() or "wait" in sb.status_string(-7).lower()
+    c = Case(CASES["cfg1"])
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
