@@ -49,6 +49,7 @@ struct EdgeArgs {
     int K, dsh, C_src, phi_mode, Y_mode;
     int warp_floats;     // shared floats per warp
     int zslab;           // floats of one Zbar slab buffer
+    int zvec;            // 1: every row pitch and offset of Zbar is a multiple of 4 floats (16-byte pieces may be copied)
 };
 
 __device__ __forceinline__ void cp_async4(float* dst, const float* src) {
@@ -67,7 +68,9 @@ __device__ __forceinline__ void cp_async16(float* dst, const float* src) {
 template <int CAP, int KC>
 __device__ __forceinline__ void stage_zbar(const EdgeArgs& a, const STask& T, const SComp* comps, const int64_t nl,
                                            int u0, int q0, float* sZ, int lane) {
-    const bool vec = (T.c_src & 3) == 0;       // then every row pitch and offset is a multiple of 4 floats
+    // 16-byte pieces need the group's row pitch D, the path offset koff and the task's own stride to be multiples of
+    // 4 floats: true when every multiplicity of the direction is (a.zvec), not when only this task's is
+    const bool vec = a.zvec && (T.c_src & 3) == 0;
     if (vec) {
         for (int i = lane; i < T.ncomp * KC; i += 32) {
             const int c = i / KC, q = i - c * KC;
@@ -401,6 +404,8 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
     a.src = src; a.vsrc = vsrc; a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.Zbar = Zbar; a.gphi = gphi; a.gY = gY;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
+    a.zvec = 1;      // koff = K * (sum of earlier multiplicities) and D = K * (sum of all): multiples of 4 iff every one is
+    for (const DPath& P : dir.paths) if (P.c_src & 3) a.zvec = 0;
     const bool k16 = p->K > 8;
     bool first = true;
     for (const auto& c : dir.eclasses) {

@@ -29,6 +29,9 @@ def small_cases():
     # that are multiples of 16 but not of 32, and receivers with well over 64 / 128 edges (several output groups)
     c["tc_K6_dense"] = synth.Workload("tc_K6_dense", P("16x0e+16x1o"), P("16x0e+16x1o+16x2e"), 2, 6, 160, 4.0, 3.6,
                                       "gaussian", seed=5)
+    # a group whose paths mix a multiplicity that is a multiple of 4 with one that is not (row pitch and path offset
+    # of the adjoint state are then odd): FP32-pipe kernels one way, tensor-core stream the other way
+    c["mixed_align"] = synth.Workload("mixed_align", P("5x0e+96x1o"), P("16x0e+96x2e"), 2, 3, 114, 4.0, 1.9, "bessel", seed=11)
     c["tc_K12"] = synth.Workload("tc_K12", P("48x0e+16x1o+16x2e"), P("16x0e+48x1o"), 2, 12, 70, 4.0, 2.2, "bessel", seed=6)
     return c
 
