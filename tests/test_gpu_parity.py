@@ -526,3 +526,55 @@ def test_bounded_wait_gives_up_and_reports():
     assert "timeout" in sb.status_string(-7).lower() or "wait" in sb.status_string(-7).lower()
     c = Case(CASES["cfg1"])
     assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+
+
+# ---------------------------------------------------------------------------------------
+# randomised profiles: multiplicities, orders, parities, K, mode and graph drawn from a seed
+# ---------------------------------------------------------------------------------------
+def _random_workload(rng, it):
+    mults = [8, 16, 24, 32, 48, 64, 96, 128, 5, 12]
+    mode = "uvu" if rng.random() < 0.35 else "uvw"
+    l_max = int(rng.integers(1, 4))
+    K = int(rng.choice([3, 4, 8, 11, 16, 20]))
+
+    def irreps(n, fixed=None):
+        out = []
+        for l in sorted(rng.choice(np.arange(0, 4), size=n, replace=False).tolist()):
+            par = 1 if l % 2 == 0 else -1
+            if rng.random() < 0.15:
+                par = -par
+            out.append((fixed if fixed is not None else int(rng.choice(mults)), int(l), par))
+        return out
+
+    n_in, n_out = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    m = int(rng.choice(mults)) if mode == "uvu" else None
+    ir_in, ir_out = irreps(n_in, m), irreps(n_out, m)
+    big = rng.random() < 0.15
+    N = int(rng.integers(600, 1200)) if big else int(rng.integers(20, 120))
+    deg = float(rng.choice([3, 12])) if big else float(rng.choice([3, 12, 40]))
+    L = 4.0 * (N / 60.0) ** (1 / 3)
+    return synth.Workload(f"rnd{it}", ir_in, ir_out, l_max, K, N, L, float(synth.cutoff_for_edges(N, deg * N, L)), "bessel",
+                          seed=int(rng.integers(1 << 30)), mode=mode)
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_profiles(seed):
+    """Profiles nobody hand-picked: mixed and odd multiplicities, sparse path sets, both modes, K off the padded
+    widths, tiny and multi-chunk graphs.  (A sweep of this kind found the odd-row-pitch profile `mixed_align`.)"""
+    import paper_2607_18074_b200 as sb
+    rng = np.random.default_rng(seed)
+    ran = 0
+    for it in range(45):
+        w = _random_workload(rng, it)
+        try:
+            c = Case(w)
+        except (sb.SobekError, ValueError):
+            continue                  # no allowed path, or a uvu path between unequal multiplicities
+        tag = f"seed {seed} case {it}: {w.mode} {w.irreps_in} -> {w.irreps_out} l_max={w.l_max} K={w.K} N={w.N}"
+        assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL, tag
+        for got, ref in zip(c.bwd(), c.o_bwd()):
+            assert rel_err(got, ref) <= BWD_TOL, tag
+        for got, ref in zip(c.dbwd(), c.o_dbwd()):
+            assert rel_err(got, ref) <= BWD_TOL, tag
+        ran += 1
+    assert ran >= 25
