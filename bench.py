@@ -75,6 +75,20 @@ def work_model(plan):
     return edge, node, cls
 
 
+def aggregate_over_ranks(dist, device, step_ms, e2e_ms, order_ms, E):
+    """Replicas only: every rank times its own copy of the workload.  The job's step time is the MAX over the ranks
+    (the slowest replica), its work the SUM of the ranks' edges.  `dist` is torch.distributed with an initialised
+    process group, or None for a single process.  Returns (step_ms, e2e_ms, order_ms[3], E_total)."""
+    if dist is None:
+        return float(step_ms), float(e2e_ms), np.asarray(order_ms, dtype=np.float64), float(E)
+    import torch
+    v = torch.tensor([step_ms, e2e_ms] + list(order_ms), device=device, dtype=torch.float64)
+    dist.all_reduce(v, op=dist.ReduceOp.MAX)
+    es = torch.tensor([E], device=device, dtype=torch.float64)
+    dist.all_reduce(es, op=dist.ReduceOp.SUM)
+    return float(v[0]), float(v[1]), v[2:].cpu().numpy(), float(es[0])
+
+
 class ClockSampler:
     def __init__(self, device_index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
@@ -328,16 +342,7 @@ def main():
     d2h = out_bytes
 
     # ---- max over ranks ------------------------------------------------------------------
-    if dist is not None:
-        v = torch.tensor([step_ms, e2e_ms] + list(order_ms), device=dev, dtype=torch.float64)
-        dist.all_reduce(v, op=dist.ReduceOp.MAX)
-        step_ms, e2e_ms = float(v[0]), float(v[1])
-        order_ms = v[2:].cpu().numpy()
-        es = torch.tensor([E], device=dev, dtype=torch.float64)
-        dist.all_reduce(es, op=dist.ReduceOp.SUM)
-        E_total = float(es[0])
-    else:
-        E_total = float(E)
+    step_ms, e2e_ms, order_ms, E_total = aggregate_over_ranks(dist, dev, step_ms, e2e_ms, order_ms, E)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
