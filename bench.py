@@ -319,6 +319,23 @@ def main():
     classes = sb.timing_collect()
     clocks = sampler.stop() if sampler else None
 
+    # ---- backward after a retaining forward (extra figure, not part of the step): the forward leaves the receiver
+    # state in the workspace when all nodes fit one chunk, and the backward then skips its own edge stream for gR
+    bwd_retained_ms = None
+    if world == 1:
+        ms = []
+        for _ in range(max(3, args.steps)):
+            kept = sb.conv_fwd_retain(plan, g, t["x"], t["Y"], t["phi"], t["R"], out["y"], ws)
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            sb.conv_bwd_retained(plan, g, t["x"], t["Y"], t["phi"], t["R"], t["gy"], out["gx"], out["gY"], out["gphi"],
+                                 out["gR"], ws, kept)
+            b.record()
+            torch.cuda.synchronize(dev)
+            ms.append(a.elapsed_time(b))
+        bwd_retained_ms = (float(np.mean(ms[1:])), int(kept))
+
     # ---- end to end: host buffers in, host buffers out ---------------------------------
     def e2e_step():
         for k, v in host.items():
@@ -391,6 +408,8 @@ def main():
                    for (nm, _), ms in zip(orders, order_ms)},
         "e2e": {"value": E_total / (e2e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "bwd_after_retaining_fwd": None if bwd_retained_ms is None else {
+            "edges_per_s": E_total / (bwd_retained_ms[0] * 1e-3), "ms": bwd_retained_ms[0], "state_retained": bwd_retained_ms[1]},
         "gpu_launches": int(launches),
         "wall_s_timed_region": wall,
         "peak_bytes": {"total": int(peak_bytes), "inputs_and_graph": int(in_bytes), "outputs": int(out_bytes),

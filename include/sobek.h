@@ -196,6 +196,26 @@ int sobek_conv_bwd(const sobek_plan* plan, const sobek_graph* g,
                    float* gx, float* gY, float* gphi, float* gR,
                    void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Retaining the receiver state from the forward for the backward (Section "Runtime scratch-budget policy": a
+ * forward-retained primal state is reused when it covers all groups and all receivers in one chunk).
+ * sobek_conv_fwd_retain is sobek_conv_fwd on a workspace of at least sobek_workspace_bytes(plan, N, E, 1) bytes, laid
+ * out as the backward lays it out; it sets *retained to 1 when the state Z of every receiver is left in `ws` (all
+ * nodes fit one chunk of the scratch budget and the state schedule is in use), else to 0.
+ * sobek_conv_bwd_retained is sobek_conv_bwd with that value passed back: with retained = 1 the caller asserts that
+ * `ws` has not been used since by any other call and that plan, graph, x, Y and phi are the ones of the retaining
+ * forward; the backward then computes gR from the state in place instead of streaming the edges again.  The call
+ * itself consumes the state (one backward per retaining forward).  Results are bitwise those of sobek_conv_bwd.
+ * With retained = 0 the two calls are sobek_conv_fwd / sobek_conv_bwd.  Errors: as for those, INVALID_ARG for a
+ * null `retained`.
+ */
+int sobek_conv_fwd_retain(const sobek_plan* plan, const sobek_graph* g, const float* x, const float* Y,
+                          const float* phi, const float* R, float* y, void* ws, size_t ws_bytes, void* stream,
+                          int* retained);
+int sobek_conv_bwd_retained(const sobek_plan* plan, const sobek_graph* g, const float* x, const float* Y,
+                            const float* phi, const float* R, const float* gy, float* gx, float* gY, float* gphi,
+                            float* gR, void* ws, size_t ws_bytes, void* stream, int retained);
+
 /* Double backward (Eqs. streamed_directional_terms .. streamed_operand_second_adjoints,
  * receiver_double_adjoint) with the direction on gy equal to zero: for the backward map
  * b(x,Y,phi,R; gy) = (gx,gY,gphi,gR) and cotangents v = (vx,vY,vphi,vR) it returns

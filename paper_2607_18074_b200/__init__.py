@@ -25,6 +25,7 @@ EXPORTS = [
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
+    "sobek_conv_fwd_retain", "sobek_conv_bwd_retained",
 ]
 
 
@@ -259,6 +260,23 @@ def conv_bwd(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws):
     _check(lib().sobek_conv_bwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(gy),
                                 _ptr(gx), _ptr(gY), _ptr(gphi), _ptr(gR), _ptr(ws),
                                 ws.numel() * ws.element_size(), _stream()), "sobek_conv_bwd")
+
+
+def conv_fwd_retain(plan, graph, x, Y, phi, R, y, ws) -> int:
+    """sobek_conv_fwd_retain: forward on an order-1 workspace; returns 1 if the state of all receivers stays in ws."""
+    from ctypes import c_int
+    kept = c_int(0)
+    _check(lib().sobek_conv_fwd_retain(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(y),
+                                       _ptr(ws), ws.numel() * ws.element_size(), _stream(), byref(kept)),
+           "sobek_conv_fwd_retain")
+    return int(kept.value)
+
+
+def conv_bwd_retained(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws, retained: int):
+    _check(lib().sobek_conv_bwd_retained(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(gy),
+                                         _ptr(gx), _ptr(gY), _ptr(gphi), _ptr(gR), _ptr(ws),
+                                         ws.numel() * ws.element_size(), _stream(), int(retained)),
+           "sobek_conv_bwd_retained")
 
 
 def conv_dbwd(plan, graph, x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi, hR, ws):

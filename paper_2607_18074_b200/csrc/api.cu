@@ -288,14 +288,17 @@ extern "C" int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_pt
 }
 
 namespace {
+// `order` is the workspace layout to use (0, or 1 when the state is to be found by a following backward call);
+// *retained is set to 1 when the state of every receiver is left in the workspace (one chunk, state schedule)
 int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
                   const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
-                  void* stream) {
-    int rc = check_common(p, g, ws, ws_bytes, 0);
+                  void* stream, int order = 0, int* retained = nullptr) {
+    if (retained) *retained = 0;
+    int rc = check_common(p, g, ws, ws_bytes, order);
     if (rc) return rc;
     if (!y || !R || (g->N > 0 && !x) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    Workspace w = carve(p, g->N, 0, ws);
+    Workspace w = carve(p, g->N, order, ws);
     CK(cudaMemsetAsync(w.status, 0, kHeaderBytes, s));
     if (g->N == 0) return SOBEK_OK;
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
@@ -314,12 +317,14 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
         CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
         CK(mix(p, p->fwd, n0, nn, w.zbh, w.zbl, w.fNKh, w.fNKl, R, y, 0, w.status, s));
     }
+    if (retained && w.chunk >= g->N) *retained = 1;
     return SOBEK_OK;
 }
 
+// z_valid: the workspace still holds the state Z of all receivers, left by conv_fwd_core(order = 1) on the same inputs
 int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
                   const float* phi, const float* R, const float* gy, float* gx, float* gY,
-                  float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream) {
+                  float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream, int z_valid = 0) {
     int rc = check_common(p, g, ws, ws_bytes, 1);
     if (rc) return rc;
     if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
@@ -344,8 +349,9 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             CK(split_gy(p, p->fwd, n0, nn, gy, w.gbh, w.gbl, s));
-            if (gR) {     // gR = Z^T gy with Z re-streamed (never retained across calls)
-                CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
+            if (gR) {     // gR = Z^T gy with Z re-streamed, unless the forward left it in place for all receivers
+                if (!(z_valid && w.chunk >= g->N))
+                    CK(launch_stream(p, p->fwd, rv, n0, nn, x, nullptr, xs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
                 CK(weight_grad(p, p->fwd, n0, nn, w.zbh, w.zbl, w.gbh, w.gbl, gy, w.gRp, w.part, w.splits, w.status, s));
             }
             if (gphi || gY) {
@@ -580,6 +586,38 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     const float *xi, *gyi;
     if ((rc = r.in_x(x, w.lx, &xi)) || (rc = r.in_y(gy, w.lgy, &gyi))) return rc;
     if ((rc = conv_bwd_core(p, g, xi, Y, phi, R, gyi, gx ? w.lgx : nullptr, gY, gphi, gR, ws, ws_bytes, stream))) return rc;
+    return r.out_x(w.lgx, gx);
+}
+
+extern "C" int sobek_conv_fwd_retain(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                                     const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
+                                     void* stream, int* retained) {
+    if (!retained) return SOBEK_ERR_INVALID_ARG;
+    *retained = 0;
+    if (!p || !p->mul_ir) return conv_fwd_core(p, g, x, Y, phi, R, y, ws, ws_bytes, stream, 1, retained);
+    int rc = check_common(p, g, ws, ws_bytes, 1);
+    if (rc) return rc;
+    if (!y || (g->N > 0 && !x)) return SOBEK_ERR_INVALID_ARG;
+    const Workspace w = carve(p, g->N, 1, ws);
+    const Relay r{p, g->N, (cudaStream_t)stream};
+    const float* xi;
+    if ((rc = r.in_x(x, w.lx, &xi))) return rc;
+    if ((rc = conv_fwd_core(p, g, xi, Y, phi, R, w.ly, ws, ws_bytes, stream, 1, retained))) return rc;
+    return r.out_y(w.ly, y);
+}
+
+extern "C" int sobek_conv_bwd_retained(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                                       const float* phi, const float* R, const float* gy, float* gx, float* gY,
+                                       float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream, int retained) {
+    if (!p || !p->mul_ir) return conv_bwd_core(p, g, x, Y, phi, R, gy, gx, gY, gphi, gR, ws, ws_bytes, stream, retained);
+    int rc = check_common(p, g, ws, ws_bytes, 1);
+    if (rc) return rc;
+    if (g->N > 0 && (!x || !gy)) return SOBEK_ERR_INVALID_ARG;
+    const Workspace w = carve(p, g->N, 1, ws);
+    const Relay r{p, g->N, (cudaStream_t)stream};
+    const float *xi, *gyi;
+    if ((rc = r.in_x(x, w.lx, &xi)) || (rc = r.in_y(gy, w.lgy, &gyi))) return rc;
+    if ((rc = conv_bwd_core(p, g, xi, Y, phi, R, gyi, gx ? w.lgx : nullptr, gY, gphi, gR, ws, ws_bytes, stream, retained))) return rc;
     return r.out_x(w.lgx, gx);
 }
 

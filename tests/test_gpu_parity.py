@@ -578,3 +578,42 @@ def test_random_profiles(seed):
             assert rel_err(got, ref) <= BWD_TOL, tag
         ran += 1
     assert ran >= 25
+
+
+@pytest.mark.parametrize("name,mode", [("cfg2_N200", "uvw"), ("ragged", "uvw"), ("uvu_16x3", "uvu")])
+def test_state_retained_from_forward(name, mode, monkeypatch):
+    """sobek_conv_fwd_retain leaves the receiver state in the workspace; sobek_conv_bwd_retained then computes gR
+    from it without streaming the edges again: same bits as the plain calls, one stream launch fewer."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    c = Case((UVU if mode == "uvu" else CASES)[name])
+    i = c.plan.info
+    y_ref, b_ref = c.fwd(), c.bwd()
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    ws = c.ws(1)
+    y = new(c.N, i.C_y)
+    kept = sb.conv_fwd_retain(c.plan, c.graph, c.x, c.Y, c.phi, c.R, y, ws)
+    assert kept == 1 and np.array_equal(y.cpu().numpy(), y_ref)
+    outs = [new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)]
+    l0 = sb.launch_count()
+    sb.conv_bwd_retained(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, *outs, ws, kept)
+    n_ret = sb.launch_count() - l0
+    assert sb.last_device_status(ws) == 0
+    for got, ref in zip(outs, b_ref):
+        assert np.array_equal(got.cpu().numpy(), ref)
+    l0 = sb.launch_count()
+    sb.conv_bwd(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, *outs, ws)
+    assert sb.launch_count() - l0 > n_ret               # the plain call streams the edges once more
+    # retained = 0 is the plain backward
+    sb.conv_bwd_retained(c.plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, *outs, ws, 0)
+    for got, ref in zip(outs, b_ref):
+        assert np.array_equal(got.cpu().numpy(), ref)
+    # a scratch budget that needs several chunks: nothing is retained, the results stay right
+    if c.N >= 100:
+        monkeypatch.setenv("SOBEK_STATE_BUDGET_MB", "1")
+        w2 = synth.scaled(synth.config("cfg2"), 1300)
+        c2 = Case(w2)
+        monkeypatch.delenv("SOBEK_STATE_BUDGET_MB")
+        y2 = new(c2.N, c2.plan.info.C_y)
+        assert sb.conv_fwd_retain(c2.plan, c2.graph, c2.x, c2.Y, c2.phi, c2.R, y2, c2.ws(1)) == 0
+        assert np.array_equal(y2.cpu().numpy(), c2.fwd())
