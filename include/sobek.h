@@ -77,6 +77,7 @@ enum { SOBEK_MAX_L = 4 };
 /* plan flags */
 #define SOBEK_FLAG_UVU 1u      /* channelwise multiplicity mode, Eq. uvu_connection */
 #define SOBEK_FLAG_MUL_IR 2u   /* node features cross the boundary in mul_ir order (see sobek_plan_create) */
+#define SOBEK_FLAG_FAST_GEMM 4u /* node-side GEMMs as plain bf16 products: lower precision, optional */
 
 /*
  * sobek_plan_create -- the static contract of one layer (Section "Generated
@@ -95,6 +96,10 @@ enum { SOBEK_MAX_L = 4 };
  * u*(2l+1) + m instead of m*C + u (Section "Generated deterministic runtime and execution contracts": the kernels
  * work in ir_mul, the other order is transposed at the boundary).  The calls then re-lay the arrays through the
  * workspace, which grows by 4 bytes per node feature and array; Y, phi and R are unaffected.
+ * SOBEK_FLAG_FAST_GEMM replaces the three-pass split-bf16 product of the node-side GEMMs (fp32-faithful, the default
+ * and what every stated tolerance refers to) by the single bf16 product a_hi*b_hi with fp32 accumulation: the optional
+ * reduced-precision channel GEMM of the paper's runtime contract.  Relative errors of about 1e-2 of the largest output
+ * are to be expected; the edge kernels keep their three-pass products; the flag has no effect in the uvu mode.
  * If the environment variable SOBEK_FUSED is set to a
  * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
  * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsobek.so")
 
 FLAG_UVU = 1      # SOBEK_FLAG_UVU: channelwise multiplicity mode
 FLAG_MUL_IR = 2   # SOBEK_FLAG_MUL_IR: node features cross the boundary in mul_ir order
+FLAG_FAST_GEMM = 4  # SOBEK_FLAG_FAST_GEMM: node-side GEMMs as plain bf16 products (optional, lower precision)
 
 EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",

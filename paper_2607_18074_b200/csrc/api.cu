@@ -173,7 +173,7 @@ cudaError_t mix_tc(const sobek_plan* p, const Direction& dir, int64_t n0, int64_
         cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
                                        nkh + dir.nk_off[gi], nkl + dir.nk_off[gi], dir.nk_ld[gi],
                                        dst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst,
-                                       nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s);
+                                       nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s, 1, 0, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
     return fork.join();
@@ -194,11 +194,12 @@ cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t 
             e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
                                knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi], nullptr, dir.nk_ld[gi], 0, 1,
                                nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, zqh + nn * dir.zb_off[gi],
-                               zql + nn * dir.zb_off[gi]);
+                               zql + nn * dir.zb_off[gi], p->gemm_passes);
         else
             e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
                                        knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi],
-                                       Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s);
+                                       Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, nullptr, nullptr,
+                                       p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
     return fork.join();
@@ -220,7 +221,7 @@ cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn
         cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
                                        gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
                                        part + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 0, 1, status, s,
-                                       sp, KN);
+                                       sp, KN, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
         e = launch_reduce_parts(gRp + G.rp_off, part + G.rp_off, (int64_t)G.D * G.c_dst, KN, sp, s);
         if (e != cudaSuccess) return e;

@@ -40,6 +40,7 @@ struct TcArgs {
     int64_t c_outer, c_inner;   // C(m,n) = C[(m/c_d)*c_outer + (m%c_d)*c_inner + n]
     int32_t c_d;
     int32_t accumulate;
+    int32_t passes;             // 3: split-bf16 product (fp32-faithful); 1: the hi x hi product only (plain bf16 GEMM)
     int64_t M, N, Kd;
     int32_t BN;                 // tile width (multiple of 16, <= 256)
     int32_t stages;
@@ -95,22 +96,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
                 const uint32_t ph = (kb / S) & 1;
                 mbar_wait(bar0 + 8 * (S + s), ph ^ 1, g.status);        // slot free
                 const uint32_t full = bar0 + 8 * s;
-                mbar_expect_tx(full, stage_bytes);
+                mbar_expect_tx(full, g.passes == 1 ? a_bytes + b_bytes : stage_bytes);
                 const uint32_t sa = sbase + s * stage_bytes;
                 if (!g.mn_major) {
                     tma_load_2d(sa, &tmAh, (kb_first + kb) * BK, m0, full);
-                    tma_load_2d(sa + a_bytes, &tmAl, (kb_first + kb) * BK, m0, full);
                     tma_load_2d(sa + 2 * a_bytes, &tmBh, (kb_first + kb) * BK, n0, full);
-                    tma_load_2d(sa + 2 * a_bytes + b_bytes, &tmBl, (kb_first + kb) * BK, n0, full);
+                    if (g.passes != 1) {
+                        tma_load_2d(sa + a_bytes, &tmAl, (kb_first + kb) * BK, m0, full);
+                        tma_load_2d(sa + 2 * a_bytes + b_bytes, &tmBl, (kb_first + kb) * BK, n0, full);
+                    }
                 } else {
                     // operands stored [Kd rows][M or N contiguous]: boxes of 64 MN-elements x 64 k-rows
                     for (int j = 0; j < BM / 64; ++j) {
                         tma_load_2d(sa + j * (64 * BK * 2), &tmAh, m0 + 64 * j, (kb_first + kb) * BK, full);
-                        tma_load_2d(sa + a_bytes + j * (64 * BK * 2), &tmAl, m0 + 64 * j, (kb_first + kb) * BK, full);
+                        if (g.passes != 1) tma_load_2d(sa + a_bytes + j * (64 * BK * 2), &tmAl, m0 + 64 * j, (kb_first + kb) * BK, full);
                     }
                     for (int j = 0; j < g.BN / 64; ++j) {
                         tma_load_2d(sa + 2 * a_bytes + j * (64 * BK * 2), &tmBh, n0 + 64 * j, (kb_first + kb) * BK, full);
-                        tma_load_2d(sa + 2 * a_bytes + b_bytes + j * (64 * BK * 2), &tmBl, n0 + 64 * j, (kb_first + kb) * BK, full);
+                        if (g.passes != 1) tma_load_2d(sa + 2 * a_bytes + b_bytes + j * (64 * BK * 2), &tmBl, n0 + 64 * j, (kb_first + kb) * BK, full);
                     }
                 }
             }
@@ -142,8 +145,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
                     }
                     const uint32_t first = (kb > 0 || k > 0) ? 1u : 0u;
                     tc_mma_bf16(tmem_base, dAh, dBh, idesc, first);
-                    tc_mma_bf16(tmem_base, dAl, dBh, idesc, 1u);
-                    tc_mma_bf16(tmem_base, dAh, dBl, idesc, 1u);
+                    if (g.passes != 1) {
+                        tc_mma_bf16(tmem_base, dAl, dBh, idesc, 1u);
+                        tc_mma_bf16(tmem_base, dAh, dBl, idesc, 1u);
+                    }
                 }
                 tc_commit(bar0 + 8 * (S + s));                           // frees the slot when the MMAs retire
             }
@@ -331,10 +336,10 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
-                           int64_t split_stride, void* Chi, void* Clo) {
+                           int64_t split_stride, void* Chi, void* Clo, int passes) {
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
     TcArgs g{};
-    g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate;
+    g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate; g.passes = passes == 1 ? 1 : 3;
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
     g.splits = std::max(1, std::min<int>(splits, (int)((Kd + BK - 1) / BK))); g.split_stride = split_stride;
     int BN;

@@ -236,6 +236,7 @@ struct sobek_plan {
     bool use_tc_stream = true;   // edge stream on the tensor cores where the profile allows it
     bool use_tc_edge = true;     // edge pass on the tensor cores where the profile allows it
     size_t state_budget = size_t(2048) << 20;   // bytes of receiver / sender state held at once (the scratch budget)
+    int gemm_passes = 3;      // 3: split-bf16 node GEMMs (fp32-faithful); 1: plain bf16 GEMMs (SOBEK_FLAG_FAST_GEMM)
     bool mul_ir = false;      // node features cross the boundary in mul_ir order and are re-laid through the workspace
     int4* d_in_blocks = nullptr;    // {offset, multiplicity, 2l+1, 0} of the irrep blocks of x / of y (device), for the re-layout
     int4* d_out_blocks = nullptr;
@@ -402,7 +403,7 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
-                           int64_t split_stride = 0, void* Chi = nullptr, void* Clo = nullptr);
+                           int64_t split_stride = 0, void* Chi = nullptr, void* Clo = nullptr, int passes = 3);
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
 cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s);
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM

@@ -385,7 +385,7 @@ using namespace sobek;
 
 extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
                                  int l_max, int K, uint32_t flags, sobek_plan** plan) {
-    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR)) != 0 || l_max < 0)
+    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR | SOBEK_FLAG_FAST_GEMM)) != 0 || l_max < 0)
         return SOBEK_ERR_INVALID_ARG;
     *plan = nullptr;
     if (l_max > SOBEK_MAX_L) return SOBEK_ERR_UNSUPPORTED;
@@ -405,6 +405,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     p->K = K;
     p->uvu = (flags & SOBEK_FLAG_UVU) != 0;
     p->mul_ir = (flags & SOBEK_FLAG_MUL_IR) != 0;
+    p->gemm_passes = (flags & SOBEK_FLAG_FAST_GEMM) ? 1 : 3;
     p->dim_sh = (l_max + 1) * (l_max + 1);
     std::vector<int> in_off(n_in), out_off(n_out);
     for (int i = 0; i < n_in; ++i) { in_off[i] = p->C_x; p->C_x += in[i].mul * (2 * in[i].l + 1); }

@@ -617,3 +617,29 @@ def test_state_retained_from_forward(name, mode, monkeypatch):
         y2 = new(c2.N, c2.plan.info.C_y)
         assert sb.conv_fwd_retain(c2.plan, c2.graph, c2.x, c2.Y, c2.phi, c2.R, y2, c2.ws(1)) == 0
         assert np.array_equal(y2.cpu().numpy(), c2.fwd())
+
+
+def test_fast_gemm_flag(cases):
+    """SOBEK_FLAG_FAST_GEMM: the node-side GEMMs as single bf16 products.  Optional and outside the stated tolerances:
+    close to the oracle at bf16 level, and not the same numbers as the default three-pass plan."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    c = get(cases, "cfg2_N200")
+    w = c.w
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, flags=sb.FLAG_FAST_GEMM)
+    i = plan.info
+    ws = torch.empty(sb.workspace_bytes(plan, c.N, c.E, 2), dtype=torch.uint8, device="cuda:0")
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    y = new(c.N, i.C_y)
+    sb.conv_fwd(plan, c.graph, c.x, c.Y, c.phi, c.R, y, ws)
+    e = rel_err(y.cpu().numpy(), c.o_fwd())
+    assert FWD_TOL < e < 2e-2
+    outs = [new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)]
+    sb.conv_bwd(plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, *outs, ws)
+    for got, ref in zip(outs, c.o_bwd()):
+        assert rel_err(got.cpu().numpy(), ref) < 2e-2
+    outs = [new(c.N, i.C_y), new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)]
+    sb.conv_dbwd(plan, c.graph, c.x, c.Y, c.phi, c.R, c.gy, c.vx, c.vY, c.vphi, c.vR, *outs, ws)
+    for got, ref in zip(outs, c.o_dbwd()):
+        assert rel_err(got.cpu().numpy(), ref) < 2e-2
+    assert sb.last_device_status(ws) == 0

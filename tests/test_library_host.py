@@ -140,7 +140,7 @@ def test_uvu_plan_errors_and_workspace():
     with pytest.raises(sb.SobekError):
         sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")       # 0e x 1o -> 1o would tie 8 channels to 4
     with pytest.raises(sb.SobekError):
-        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=4)                    # unknown flag bit
+        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=8)                    # unknown flag bit
     ir = P("64x0e+64x1o+64x2e")
     u, w = sb.Plan(ir, ir, 2, 16, mode="uvu"), sb.Plan(ir, ir, 2, 16)
     assert u.mode == "uvu" and w.mode == "uvw" and u.info.C_y == w.info.C_y
