@@ -337,26 +337,74 @@ def main():
         bwd_retained_ms = (float(np.mean(ms[1:])), int(kept))
 
     # ---- end to end: host buffers in, host buffers out ---------------------------------
-    def e2e_step():
-        for k, v in host.items():
-            t[k].copy_(v, non_blocking=True)
-        fwd(); bwd(); dbwd()
-        for k, v in out.items():
-            host_out[k].copy_(v, non_blocking=True)
+    # Every step copies all of its inputs from pinned host memory and all of its outputs back, through the public
+    # API.  Where device memory allows a second set of input / output buffers, the copies run on two copy streams
+    # and overlap the previous / next step's kernels (double buffering); otherwise everything is serial.
+    def run_orders(tt, oo):
+        sb.conv_fwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], oo["y"], ws)
+        sb.conv_bwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], oo["gx"], oo["gY"], oo["gphi"], oo["gR"], ws)
+        sb.conv_dbwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], tt["vx"], tt["vY"], tt["vphi"], tt["vR"],
+                     oo["ggy"], oo["hx"], oo["hY"], oo["hphi"], oo["hR"], ws)
 
-    e2e_step()
+    h2d = sum(v.numel() * 4 for v in host.values())
+    d2h = out_bytes
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    pipelined = free_b > 1.25 * (h2d + d2h) + (1 << 30)
+    if pipelined:
+        t_sets = [t, {k: torch.empty_like(v) for k, v in t.items()}]
+        o_sets = [out, {k: torch.empty_like(v) for k, v in out.items()}]
+        s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        main = torch.cuda.current_stream(dev)
+
+        def e2e_run(n):
+            in_ready = [torch.cuda.Event(), torch.cuda.Event()]
+            done = [torch.cuda.Event(), torch.cuda.Event()]
+            with torch.cuda.stream(s_in):                      # inputs of step 0
+                s_in.wait_stream(main)
+                for k, v in host.items():
+                    t_sets[0][k].copy_(v, non_blocking=True)
+                in_ready[0].record(s_in)
+            for i in range(n):
+                cur = i & 1
+                flush.fill_(1)
+                main.wait_event(in_ready[cur])
+                if i >= 2:
+                    main.wait_stream(s_out)                    # the outputs of step i-2 have left o_sets[cur]
+                run_orders(t_sets[cur], o_sets[cur])
+                done[cur].record(main)
+                with torch.cuda.stream(s_out):                 # outputs of step i go back while step i+1 runs
+                    s_out.wait_event(done[cur])
+                    for k, v in o_sets[cur].items():
+                        host_out[k].copy_(v, non_blocking=True)
+                if i + 1 < n:
+                    with torch.cuda.stream(s_in):              # inputs of step i+1 come in while step i runs
+                        if i >= 1:
+                            s_in.wait_event(done[1 - cur])     # step i-1 no longer reads t_sets[1-cur]
+                        for k, v in host.items():
+                            t_sets[1 - cur][k].copy_(v, non_blocking=True)
+                        in_ready[1 - cur].record(s_in)
+            main.wait_stream(s_out)
+            main.wait_stream(s_in)
+    else:
+        def e2e_run(n):
+            for _ in range(n):
+                flush.fill_(1)
+                for k, v in host.items():
+                    t[k].copy_(v, non_blocking=True)
+                run_orders(t, out)
+                for k, v in out.items():
+                    host_out[k].copy_(v, non_blocking=True)
+
+    e2e_run(2)
     torch.cuda.synchronize(dev)
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
-    for _ in range(args.steps):
-        flush.fill_(1)
-        e2e_step()
+    e2e_run(args.steps)
     b.record()
     barrier()
     e2e_ms = a.elapsed_time(b) / args.steps
-    h2d = sum(v.numel() * 4 for v in host.values())
-    d2h = out_bytes
+    assert sb.last_device_status(ws) == 0
 
     # ---- max over ranks ------------------------------------------------------------------
     step_ms, e2e_ms, order_ms, E_total = aggregate_over_ranks(dist, dev, step_ms, e2e_ms, order_ms, E)
@@ -407,7 +455,8 @@ def main():
                         "edge_fma_per_edge": edge_w[nm], "node_fma_per_node": node_w[nm]}
                    for (nm, _), ms in zip(orders, order_ms)},
         "e2e": {"value": E_total / (e2e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                "copies": "double-buffered on two copy streams" if pipelined else "serial"},
         "bwd_after_retaining_fwd": None if bwd_retained_ms is None else {
             "edges_per_s": E_total / (bwd_retained_ms[0] * 1e-3), "ms": bwd_retained_ms[0], "state_retained": bwd_retained_ms[1]},
         "gpu_launches": int(launches),
