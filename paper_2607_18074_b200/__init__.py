@@ -11,7 +11,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_uint, c_uint32, c_void_p
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsobek.so")
@@ -84,6 +84,9 @@ def lib():
         L.sobek_conv_fwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6 + [c_size_t, c_void_p]
         L.sobek_conv_bwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 10 + [c_size_t, c_void_p]
         L.sobek_conv_dbwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 15 + [c_size_t, c_void_p]
+        L.sobek_conv_fwd_retain.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6 + [c_size_t, c_void_p, POINTER(c_int)]
+        L.sobek_conv_bwd_retained.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 10 + [c_size_t, c_void_p, c_int]
+        L.sobek_selftest_wait_timeout.argtypes = [c_void_p, c_uint, c_void_p]
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
         L.sobek_static_scratch_bytes.restype = c_size_t
         L.sobek_conv_fwd_static.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6

@@ -163,3 +163,14 @@ def test_mul_ir_flag_and_workspace():
     for order in (0, 1, 2):
         assert sb.workspace_bytes(b, N, 10**5, order) - sb.workspace_bytes(a, N, 10**5, order) == extra[order]
     assert sb.Plan(ir, ir, 2, 8, mode="uvu", layout="mul_ir").mode == "uvu"
+
+
+def test_binding_declares_every_signature():
+    """ctypes without argtypes passes Python ints as 32-bit C ints: a workspace size above 4 GiB would be truncated.
+    Every exported entry point that takes arguments must have its signature declared."""
+    L = sb.lib()
+    no_args = {"sobek_static_scratch_bytes", "sobek_launch_count", "sobek_timing_classes"}
+    for name in sb.EXPORTS:
+        if name in no_args:
+            continue
+        assert getattr(L, name).argtypes is not None, name
