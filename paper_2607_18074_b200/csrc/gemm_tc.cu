@@ -162,6 +162,47 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
         // The pipeline buffers are idle now: each warp parks its 32 x BN block there (row pitch BN+1, so
         // that both the row-wise writes and the column-wise reads are bank-conflict free) and then writes
         // C row by row with the lanes along the columns (coalesced).
+        if (g.Ch && (g.N & 7) == 0) {
+            // bf16 (hi, lo) output.  The warp parks its 32 x BN block with a row pitch of BN + 4 floats (16-byte
+            // pieces, conflict-free), then writes two rows per step: lanes 0-15 and 16-31 each convert 8 consecutive
+            // columns of their row into two 16-byte stores, so that a row leaves as contiguous 256-byte runs.
+            const int P4 = g.BN + 4;
+            float* pk = reinterpret_cast<float*>(smem) + (size_t)q * 32 * P4;
+            for (int c0 = 0; c0 < g.BN; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);   // warp-collective
+#pragma unroll
+                for (int j = 0; j < 16; j += 4)
+                    *reinterpret_cast<float4*>(pk + lane * P4 + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            }
+            __syncwarp();
+            const int half = lane >> 4, l16 = lane & 15;
+            for (int r = half; r < 32; r += 2) {
+                const int64_t m = (int64_t)m0 + q * 32 + r;
+                if (m >= g.M) continue;
+                const int64_t rbase = blockIdx.z * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
+                for (int c8 = l16; c8 < g.BN / 8; c8 += 16) {
+                    const int64_t n = (int64_t)n0 + 8 * c8;
+                    if (n < g.N) {
+                        const float4 x0 = *reinterpret_cast<const float4*>(pk + r * P4 + 8 * c8);
+                        const float4 x1 = *reinterpret_cast<const float4*>(pk + r * P4 + 8 * c8 + 4);
+                        const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                        uint32_t hw[4], lw[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float a0 = num_kb > 0 ? xv[2 * j] : 0.f, a1 = num_kb > 0 ? xv[2 * j + 1] : 0.f;
+                            const __nv_bfloat162 hp = __floats2bfloat162_rn(a0, a1);
+                            const float2 hf = __bfloat1622float2(hp);
+                            const __nv_bfloat162 lp = __floats2bfloat162_rn(a0 - hf.x, a1 - hf.y);
+                            hw[j] = *reinterpret_cast<const uint32_t*>(&hp);
+                            lw[j] = *reinterpret_cast<const uint32_t*>(&lp);
+                        }
+                        *reinterpret_cast<uint4*>(g.Ch + rbase + n) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        *reinterpret_cast<uint4*>(g.Cl + rbase + n) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    }
+                }
+            }
+        } else {
         float* park = reinterpret_cast<float*>(smem) + (size_t)q * 32 * (g.BN + 1);
         for (int c0 = 0; c0 < g.BN; c0 += 16) {
             float v[16];
@@ -170,32 +211,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
             for (int j = 0; j < 16; ++j) park[lane * (g.BN + 1) + c0 + j] = v[j];
         }
         __syncwarp();
-        if (g.Ch && (g.N & 7) == 0) {
-            // bf16 (hi, lo) output: a lane converts 8 consecutive columns and writes them as two 16-byte stores
-            for (int r = 0; r < 32; ++r) {
-                const int64_t m = (int64_t)m0 + q * 32 + r;
-                if (m >= g.M) break;
-                const int64_t rbase = blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
-                for (int c8 = lane; c8 < g.BN / 8; c8 += 32) {
-                    const int64_t n = (int64_t)n0 + 8 * c8;
-                    if (n < g.N) {
-                        __align__(16) __nv_bfloat16 h[8], l[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float v = num_kb > 0 ? park[r * (g.BN + 1) + 8 * c8 + j] : 0.f;
-                            h[j] = __float2bfloat16_rn(v);
-                            l[j] = __float2bfloat16_rn(v - __bfloat162float(h[j]));
-                        }
-                        *reinterpret_cast<uint4*>(g.Ch + rbase + n) = *reinterpret_cast<const uint4*>(h);
-                        *reinterpret_cast<uint4*>(g.Cl + rbase + n) = *reinterpret_cast<const uint4*>(l);
-                    }
-                }
-            }
-        } else {
         for (int r = 0; r < 32; ++r) {
             const int64_t m = (int64_t)m0 + q * 32 + r;
             if (m >= g.M) break;
-            const int64_t rbase = blockIdx.z * g.split_stride + (m / g.c_d) * g.c_outer + (m % g.c_d) * g.c_inner;
+            const int64_t rbase = blockIdx.z * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
             float* crow = g.C + rbase;
             for (int c = lane; c < g.BN; c += 32) {
                 const int64_t n = (int64_t)n0 + c;
@@ -338,6 +357,7 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
                            int64_t split_stride, void* Chi, void* Clo, int passes) {
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
+    if (M >= (int64_t(1) << 32)) return cudaErrorInvalidValue;   // the epilogue maps rows with 32-bit divisions
     TcArgs g{};
     g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate; g.passes = passes == 1 ? 1 : 3;
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
@@ -354,7 +374,7 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
     if (stages < 2) stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
     stages = std::max(1, std::min(stages, (num_kb + g.splits - 1) / g.splits));
     g.stages = stages;
-    const size_t park = (size_t)4 * 32 * (BN + 1) * sizeof(float);       // epilogue staging of the four drain warps
+    const size_t park = (size_t)4 * 32 * (BN + 4) * sizeof(float);       // epilogue staging of the four drain warps
     g.ring_bytes = (int32_t)((std::max(park, (size_t)stages * stage) + 1023) & ~size_t(1023));
     int cols = 32;
     while (cols < BN) cols <<= 1;
