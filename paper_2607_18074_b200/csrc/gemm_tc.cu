@@ -159,9 +159,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
         const int q = warp & 3;
         mbar_wait(bar0 + 8 * 2 * S, 0, g.status);
         tc_fence_after();
-        // The pipeline buffers are idle now: each warp parks its 32 x BN block there (row pitch BN+1, so
-        // that both the row-wise writes and the column-wise reads are bank-conflict free) and then writes
-        // C row by row with the lanes along the columns (coalesced).
+        // The pipeline buffers are idle now: each warp parks its 32 x BN block there and then writes C row by row
+        // with the lanes along the columns (coalesced).
         if (g.Ch && (g.N & 7) == 0) {
             // bf16 (hi, lo) output.  The warp parks its 32 x BN block with a row pitch of BN + 4 floats (16-byte
             // pieces, conflict-free), then writes two rows per step: lanes 0-15 and 16-31 each convert 8 consecutive
@@ -203,12 +202,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
                 }
             }
         } else {
-        float* park = reinterpret_cast<float*>(smem) + (size_t)q * 32 * (g.BN + 1);
+        const int P4 = g.BN + 4;      // 16-byte-aligned pitch: conflict-free 16-byte writes, conflict-free row reads
+        float* park = reinterpret_cast<float*>(smem) + (size_t)q * 32 * P4;
         for (int c0 = 0; c0 < g.BN; c0 += 16) {
             float v[16];
             tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);   // warp-collective
 #pragma unroll
-            for (int j = 0; j < 16; ++j) park[lane * (g.BN + 1) + c0 + j] = v[j];
+            for (int j = 0; j < 16; j += 4)
+                *reinterpret_cast<float4*>(park + lane * P4 + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
         }
         __syncwarp();
         for (int r = 0; r < 32; ++r) {
@@ -219,7 +220,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
             for (int c = lane; c < g.BN; c += 32) {
                 const int64_t n = (int64_t)n0 + c;
                 if (n < g.N) {
-                    const float v = num_kb > 0 ? park[r * (g.BN + 1) + c] : 0.f;
+                    const float v = num_kb > 0 ? park[r * P4 + c] : 0.f;
                     if (g.Ch) {
                         const __nv_bfloat16 h = __float2bfloat16_rn(v);
                         g.Ch[rbase + n] = h;
