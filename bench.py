@@ -33,11 +33,12 @@ METRIC = "edges/s (one step = fwd + bwd + double-bwd)"
 FP32_FMA_LANES = 148 * 128            # SMs x FP32 lanes
 L2_FLUSH_BYTES = 512 << 20
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from the ncu captures summarised
-# under profiles/ (average over the launches of the class in one step).  Only known for the workload
-# that was captured.
-NCU_TRAFFIC_BYTES = {("cfg2", "edge_stream_state"): 144.0e6, ("cfg2", "edge_pass"): 137.0e6,
-                     ("cfg2", "node_gemm"): 48.4e6}
+DTYPE = "f32 storage; products as split bf16 x3 (hi*hi + lo*hi + hi*lo) with f32 accumulation (tcgen05)"
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel class, measured with ncu
+# on the named workload.  A capture on a scaled-down graph of the same profile is stored per edge and multiplied by
+# the edges of a launch (the traffic of these kernels grows in proportion to the edges).
+NCU_TRAFFIC_BYTES_PER_EDGE = {}
 
 
 def measured_peaks():
@@ -72,7 +73,16 @@ def work_model(plan):
     cls = {"edge_stream_state": (KF + CG) + (KF + CG + KFt + CGt) + (3 * KF + 2 * CG + 3 * KFt + 2 * CGt),
            "edge_pass": (2 * KF + 2 * CG) + (5 * KF + 3 * CG),
            "fused_stream_gemm": 0}
-    return edge, node, cls
+    # algorithmic HBM bytes per edge and step of the same classes (edge inputs read once per launch, one gathered
+    # feature row per edge; the bounded state and the node-sized outputs are not edge-sized and not counted)
+    i = plan.info
+    e_in = 4 * i.dim_sh + 4 * K
+    b_r, b_s = 4 + e_in + 4 * i.C_x, 8 + e_in + 4 * i.C_y
+    cls_bytes = {"edge_stream_state": 3 * b_r + (4 + 2 * e_in + 8 * i.C_x) + 2 * b_s + (8 + 2 * e_in + 4 * i.C_y),
+                 # gphi / gY (hphi / hY) written, the dual pass reads both copies of the edge inputs and of x
+                 "edge_pass": 2 * (b_r + e_in) + (4 + 3 * e_in + 8 * i.C_x),
+                 "fused_stream_gemm": 0}
+    return edge, node, cls, cls_bytes
 
 
 def aggregate_over_ranks(dist, device, step_ms, e2e_ms, order_ms, E):
@@ -199,14 +209,111 @@ def run_reference(args):
     }))
 
 
+class Run:
+    """One workload resident on the device, with the three calls of a step bound to its buffers."""
+
+    def __init__(self, sb, torch, dev, w, seed):
+        self.sb, self.torch, self.dev, self.w = sb, torch, dev, w
+        self.plan = plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
+        w.seed = seed
+        self.d = d = synth.make_inputs(w, synth.plan_col_std(plan))
+        self.info = i = plan.info
+        self.N, self.E = N, E = d.N, d.E
+        self.host = {k: torch.from_numpy(np.ascontiguousarray(getattr(d, k))).pin_memory()
+                     for k in ("x", "Y", "phi", "R", "gy", "vx", "vY", "vphi", "vR")}
+        torch.cuda.reset_peak_memory_stats(dev)
+        self.base_alloc = torch.cuda.memory_allocated(dev)
+        self.t = {k: v.to(dev) for k, v in self.host.items()}
+        rp = torch.from_numpy(d.row_ptr.astype(np.int64)).to(dev)
+        col = torch.from_numpy(d.col.astype(np.int32)).to(dev)
+        sp, perm = sb.graph_prepare(rp, col)
+        recv = sb.graph_receivers(rp, perm)
+        self.g = sb.make_graph(rp, col, sp, perm, recv)
+        self.in_bytes = torch.cuda.memory_allocated(dev) - self.base_alloc
+        new = lambda *s: torch.empty(*s, dtype=torch.float32, device=dev)
+        self.out = {"y": new(N, i.C_y), "gx": new(N, i.C_x), "gY": new(E, i.dim_sh), "gphi": new(E, i.K),
+                    "gR": new(i.K, i.N_w), "ggy": new(N, i.C_y), "hx": new(N, i.C_x), "hY": new(E, i.dim_sh),
+                    "hphi": new(E, i.K), "hR": new(i.K, i.N_w)}
+        self.out_bytes = sum(v.numel() * 4 for v in self.out.values())
+        self.ws_bytes = sb.workspace_bytes(plan, N, E, 2)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def run_orders(self, tt, oo, which=(0, 1, 2)):
+        sb, plan, g, ws = self.sb, self.plan, self.g, self.ws
+        if 0 in which:
+            sb.conv_fwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], oo["y"], ws)
+        if 1 in which:
+            sb.conv_bwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], oo["gx"], oo["gY"], oo["gphi"],
+                        oo["gR"], ws)
+        if 2 in which:
+            sb.conv_dbwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], tt["vx"], tt["vY"], tt["vphi"],
+                         tt["vR"], oo["ggy"], oo["hx"], oo["hY"], oo["hphi"], oo["hR"], ws)
+
+    def timed_step(self):
+        """One step; returns per-order device milliseconds.  L2 is flushed (a buffer larger than L2 is
+        overwritten) before every order, outside the event brackets."""
+        torch = self.torch
+        evs = []
+        for o in (0, 1, 2):
+            self.flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            self.run_orders(self.t, self.out, (o,))
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize(self.dev)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def class_times(self, steps):
+        """{kernel class: (device ms, launches)} over `steps` steps, CUDA events around every launch."""
+        self.sb.timing_enable(True)
+        for _ in range(steps):
+            for o in (0, 1, 2):
+                self.flush.fill_(1)
+                self.run_orders(self.t, self.out, (o,))
+        self.torch.cuda.synchronize(self.dev)
+        self.sb.timing_enable(False)
+        return self.sb.timing_collect()
+
+
+ORDER_NAMES = ("fwd", "bwd", "dbwd")
+
+
+def side_table(sb, torch, dev, names, steps=5, warmup=3):
+    """The other single-GPU configurations, measured in the same process with the same protocol (median of
+    `steps` steps after `warmup`): edges/s per order and per step, and the edge-stream class time."""
+    rows = {}
+    for name in names:
+        r = Run(sb, torch, dev, synth.config(name), 0)
+        for _ in range(warmup):
+            r.timed_step()
+        per = np.array([r.timed_step() for _ in range(steps)])
+        assert sb.last_device_status(r.ws) == 0
+        cls = r.class_times(2)
+        _, _, cls_w, _ = work_model(r.plan)
+        ms = np.median(per, axis=0)
+        st_ms = cls["edge_stream_state"][0] / 2
+        rows[r.w.name] = {
+            "N": r.N, "E": r.E, "ms_per_step": float(np.median(per.sum(axis=1))),
+            "edges_per_s": {nm: r.E / (m * 1e-3) for nm, m in zip(ORDER_NAMES, ms)},
+            "step_edges_per_s": r.E / (float(np.median(per.sum(axis=1))) * 1e-3),
+            "edge_stream_state_tflops": 2.0 * cls_w["edge_stream_state"] * r.E / (st_ms * 1e-3) / 1e12 if st_ms > 0 else None,
+            "workspace_bytes": int(r.ws_bytes), "steps": steps}
+        del r
+        torch.cuda.empty_cache()
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="skip the table of the other configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -227,61 +334,10 @@ def main():
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
 
-    w = synth.config(args.workload)
-    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
     # replicas only: every rank runs the same workload on its own GPU (different seed per rank)
-    w.seed = rank
-    d = synth.make_inputs(w, plan.col_std())
-    i = plan.info
-    N, E = d.N, d.E
-
-    host = {k: torch.from_numpy(np.ascontiguousarray(getattr(d, k))).pin_memory()
-            for k in ("x", "Y", "phi", "R", "gy", "vx", "vY", "vphi", "vR")}
-    torch.cuda.reset_peak_memory_stats(dev)
-    base_alloc = torch.cuda.memory_allocated(dev)
-    t = {k: v.to(dev) for k, v in host.items()}
-    rp = torch.from_numpy(d.row_ptr.astype(np.int64)).to(dev)
-    col = torch.from_numpy(d.col.astype(np.int32)).to(dev)
-    sp, perm = sb.graph_prepare(rp, col)
-    recv = sb.graph_receivers(rp, perm)
-    g = sb.make_graph(rp, col, sp, perm, recv)
-    in_bytes = torch.cuda.memory_allocated(dev) - base_alloc
-    new = lambda *s: torch.empty(*s, dtype=torch.float32, device=dev)
-    out = {"y": new(N, i.C_y), "gx": new(N, i.C_x), "gY": new(E, i.dim_sh), "gphi": new(E, i.K),
-           "gR": new(i.K, i.N_w), "ggy": new(N, i.C_y), "hx": new(N, i.C_x), "hY": new(E, i.dim_sh),
-           "hphi": new(E, i.K), "hR": new(i.K, i.N_w)}
-    out_bytes = sum(v.numel() * 4 for v in out.values())
-    ws_bytes = sb.workspace_bytes(plan, N, E, 2)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    r = Run(sb, torch, dev, synth.config(args.workload), rank)
+    w, plan, i, N, E, t, out, ws, g, host, flush = r.w, r.plan, r.info, r.N, r.E, r.t, r.out, r.ws, r.g, r.host, r.flush
     host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
-
-    def fwd():
-        sb.conv_fwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], out["y"], ws)
-
-    def bwd():
-        sb.conv_bwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], t["gy"], out["gx"], out["gY"], out["gphi"],
-                    out["gR"], ws)
-
-    def dbwd():
-        sb.conv_dbwd(plan, g, t["x"], t["Y"], t["phi"], t["R"], t["gy"], t["vx"], t["vY"], t["vphi"], t["vR"],
-                     out["ggy"], out["hx"], out["hY"], out["hphi"], out["hR"], ws)
-
-    orders = [("fwd", fwd), ("bwd", bwd), ("dbwd", dbwd)]
-
-    def timed_step():
-        """One step; returns per-order device milliseconds.  L2 is flushed (a buffer larger than
-        L2 is overwritten) before every order, outside the event brackets."""
-        evs = []
-        for _, fn in orders:
-            flush.fill_(1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            b.record()
-            evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        return [a.elapsed_time(b) for a, b in evs]
 
     def barrier():
         if dist is not None:
@@ -289,42 +345,44 @@ def main():
         torch.cuda.synchronize(dev)
 
     for _ in range(args.warmup):
-        timed_step()
+        r.timed_step()
     assert sb.last_device_status(ws) == 0
-    peak_bytes = torch.cuda.max_memory_allocated(dev) - base_alloc
+    peak_bytes = torch.cuda.max_memory_allocated(dev) - r.base_alloc
 
-    # ---- timed region: exactly K steps -------------------------------------------------
+    # ---- timed region: exactly K steps; every step is one sample, the reported time is their median ----
     sampler = ClockSampler(local) if rank == 0 else None
     barrier()
     l0 = sb.launch_count()
     per = []
     wall0 = time.perf_counter()
     for _ in range(args.steps):
-        per.append(timed_step())
+        per.append(r.timed_step())
     barrier()
     wall = time.perf_counter() - wall0
     launches = sb.launch_count() - l0
     per = np.array(per)                                  # [steps, 3] device ms
-    step_ms = float(per.sum(axis=1).mean())
-    order_ms = per.mean(axis=0)
+    step_ms = float(np.median(per.sum(axis=1)))
+    step_ms_mean = float(per.sum(axis=1).mean())
+    order_ms = np.median(per, axis=0)
 
-    # ---- per-kernel-class device time over K more steps (events around every launch)
-    sb.timing_enable(True)
-    for _ in range(args.steps):
-        for _, fn in orders:
-            flush.fill_(1)
-            fn()
-    torch.cuda.synchronize(dev)
-    sb.timing_enable(False)
-    classes = sb.timing_collect()
+    # ---- per-kernel-class device time over a few more steps (events around every launch)
+    cls_steps = min(args.steps, 5)
+    classes = r.class_times(cls_steps)
     clocks = sampler.stop() if sampler else None
+
+    # ---- the FP32 multiply-add rate of this GPU, measured for about a second, with the SM clock sampled meanwhile
+    fp32_peak, fp32_clock = None, None
+    if rank == 0:
+        cs = ClockSampler(local)
+        fp32_peak = sb.measure_fp32_peak(1.0)
+        fp32_clock = cs.stop()
 
     # ---- backward after a retaining forward (extra figure, not part of the step): the forward leaves the receiver
     # state in the workspace when all nodes fit one chunk, and the backward then skips its own edge stream for gR
     bwd_retained_ms = None
     if world == 1:
         ms = []
-        for _ in range(max(3, args.steps)):
+        for _ in range(4):
             kept = sb.conv_fwd_retain(plan, g, t["x"], t["Y"], t["phi"], t["R"], out["y"], ws)
             flush.fill_(1)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -334,20 +392,15 @@ def main():
             b.record()
             torch.cuda.synchronize(dev)
             ms.append(a.elapsed_time(b))
-        bwd_retained_ms = (float(np.mean(ms[1:])), int(kept))
+        bwd_retained_ms = (float(np.median(ms[1:])), int(kept))
 
     # ---- end to end: host buffers in, host buffers out ---------------------------------
     # Every step copies all of its inputs from pinned host memory and all of its outputs back, through the public
     # API.  Where device memory allows a second set of input / output buffers, the copies run on two copy streams
     # and overlap the previous / next step's kernels (double buffering); otherwise everything is serial.
-    def run_orders(tt, oo):
-        sb.conv_fwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], oo["y"], ws)
-        sb.conv_bwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], oo["gx"], oo["gY"], oo["gphi"], oo["gR"], ws)
-        sb.conv_dbwd(plan, g, tt["x"], tt["Y"], tt["phi"], tt["R"], tt["gy"], tt["vx"], tt["vY"], tt["vphi"], tt["vR"],
-                     oo["ggy"], oo["hx"], oo["hY"], oo["hphi"], oo["hR"], ws)
-
+    run_orders = r.run_orders
     h2d = sum(v.numel() * 4 for v in host.values())
-    d2h = out_bytes
+    d2h = r.out_bytes
     free_b, _ = torch.cuda.mem_get_info(dev)
     pipelined = free_b > 1.25 * (h2d + d2h) + (1 << 30)
     if pipelined:
@@ -414,13 +467,16 @@ def main():
         return
 
     peaks = measured_peaks()
-    edge_w, node_w, cls_w = work_model(plan)
+    edge_w, node_w, cls_w, cls_b = work_model(plan)
     # dominant kernel class and its roofline
     tot_cls = sum(v[0] for v in classes.values()) or 1.0
     dom = max(classes, key=lambda k: classes[k][0])
     dom_ms, dom_launches = classes[dom]
-    steps_timed = args.steps
-    alu_peak = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
+    steps_timed = cls_steps
+    alu_derived = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
+    alu_peak = fp32_peak if fp32_peak else alu_derived
+    traffic_pe = NCU_TRAFFIC_BYTES_PER_EDGE.get((w.name.split("_N")[0], dom))
+    traffic = None if traffic_pe is None else traffic_pe * E
     if dom == "node_gemm":
         # the node contractions stream the bounded state once per pass (4 bytes per state element as bf16
         # hi + lo, read or written): HBM-bound; passes per step: 8 over the receiver state, 3 over the sender state
@@ -428,17 +484,26 @@ def main():
         nbytes = 4.0 * (8 * info.state_floats_fwd + 3 * info.state_floats_bwd) * N * steps_timed
         achieved = nbytes / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
         roofline = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic,
                     "peak_source": f"HBM copy bandwidth, {peaks['source']}"}
     else:
-        # the edge kernels: algorithmic multiply-adds of the method per edge against the FP32 pipes (the
-        # tensor-core kernels move the part that scales with the multiplicity off those pipes)
+        # the edge kernels: algorithmic multiply-adds of the method per edge against the FP32 multiply-add rate
+        # measured on this GPU in this run (the tensor-core kernels move the part of the work that scales with the
+        # multiplicity off those pipes, so the fraction may pass 1); beside it the same launches' algorithmic HBM
+        # bytes against the measured copy bandwidth
         fmas = cls_w.get(dom, 0) * E * steps_timed
         achieved = 2.0 * fmas / (dom_ms * 1e-3) / 1e12 if dom_ms > 0 else 0.0
+        hbm = cls_b.get(dom, 0) * E * steps_timed / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
         roofline = {"kernel": dom, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                    "frac": achieved / alu_peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
-                    "peak_source": f"derived: 148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz "
-                                   f"(HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_tflops']} TFLOP/s {peaks['source']})"}
+                    "frac": achieved / alu_peak, "traffic": traffic,
+                    "peak_source": ("measured: independent FP32 fused multiply-add chains on all SMs for 1 s, CUDA events"
+                                    if fp32_peak else "derived"),
+                    "peak_derived": alu_derived,
+                    "peak_derived_source": f"148 SMs x 128 FP32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz",
+                    "frac_of_derived": achieved / alu_derived,
+                    "fp32_peak_clocks": fp32_clock,
+                    "hbm": {"algorithmic_gbs": hbm, "peak_gbs": peaks["hbm_gbs"], "frac": hbm / peaks["hbm_gbs"],
+                            "peak_source": f"copy bandwidth, {peaks['source']}"}}
     roofline.update({
                 "avg_launch_ms": dom_ms / max(dom_launches, 1), "launches": int(dom_launches),
                 "share_of_kernel_time": dom_ms / tot_cls,
@@ -448,12 +513,14 @@ def main():
     res = {
         "metric": METRIC, "value": E_total / (step_ms * 1e-3), "unit": "edges/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": w.name, "mode": w.mode, "N": N, "E": E, "K": i.K, "N_w": int(i.N_w), "C_x": i.C_x, "C_y": i.C_y,
-                   "l_max": i.l_max, "replicas": world, "l2": f"flushed before every order ({L2_FLUSH_BYTES >> 20} MiB write)"},
+                   "l_max": i.l_max, "replicas": world, "l2": f"flushed before every order ({L2_FLUSH_BYTES >> 20} MiB write)",
+                   "timing": "every step is one sample (CUDA events per order); ms_per_step and the per-order times are medians"},
+        "ms_per_step_mean": step_ms_mean, "timed_ms_total": float(per.sum()),
         "orders": {nm: {"edges_per_s": E_total / (ms * 1e-3), "ms": float(ms),
                         "edge_fma_per_edge": edge_w[nm], "node_fma_per_node": node_w[nm]}
-                   for (nm, _), ms in zip(orders, order_ms)},
+                   for nm, ms in zip(ORDER_NAMES, order_ms)},
         "e2e": {"value": E_total / (e2e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "copies": "double-buffered on two copy streams" if pipelined else "serial"},
@@ -461,18 +528,26 @@ def main():
             "edges_per_s": E_total / (bwd_retained_ms[0] * 1e-3), "ms": bwd_retained_ms[0], "state_retained": bwd_retained_ms[1]},
         "gpu_launches": int(launches),
         "wall_s_timed_region": wall,
-        "peak_bytes": {"total": int(peak_bytes), "inputs_and_graph": int(in_bytes), "outputs": int(out_bytes),
-                       "workspace": int(ws_bytes), "l2_flush_buffer": L2_FLUSH_BYTES},
+        "peak_bytes": {"total": int(peak_bytes), "inputs_and_graph": int(r.in_bytes), "outputs": int(r.out_bytes),
+                       "workspace": int(r.ws_bytes), "l2_flush_buffer": L2_FLUSH_BYTES},
         "roofline": roofline,
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
         from oracle import conv as oconv
         oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
-        rate, edges, secs, tt, nrecv, cores = oracle_sample_rate(w, d, oracle)
+        rate, edges, secs, tt, nrecv, cores = oracle_sample_rate(w, r.d, oracle)
         res["cpu_baseline"] = {"value": rate, "unit": "edges/s", "cores": cores, "kind": "oracle",
                                "sample": f"first {nrecv} receivers ({edges} edges) of {w.name}, fwd+bwd+dbwd, {secs:.1f} s",
                                "seconds": {k: round(v, 3) for k, v in tt.items()}}
+    if world == 1 and not args.no_table and args.workload == "cfg5":
+        # the other single-GPU configurations, same process and protocol
+        del t, out, ws, g, host, flush, host_out, run_orders
+        if pipelined:
+            del t_sets, o_sets
+        del r
+        torch.cuda.empty_cache()
+        res["other_configs"] = side_table(sb, torch, dev, ["cfg2", "cfg3", "cfg4_1e6"])
     print(json.dumps(res))
     if dist is not None:
         dist.destroy_process_group()

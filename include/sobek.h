@@ -18,6 +18,8 @@
  *   - All array arguments of the sobek_conv_* / sobek_graph_prepare calls are DEVICE
  *     pointers owned by the caller and must stay valid until the work queued on
  *     `stream` (a cudaStream_t passed as void*; NULL = default stream) has finished.
+ *     Every floating-point array must start on a 16-byte boundary (the kernels copy 16-byte pieces of
+ *     phi / vphi rows and of feature rows); a pointer that does not is refused with INVALID_ARG.
  *     Plan handles and descriptor arrays are HOST memory.
  *   - fp32 data, row-major.  Node features x[N,C_x], y/gy/ggy[N,C_y] use the `ir_mul`
  *     layout (Section "Generated deterministic runtime and execution contracts"):
@@ -78,6 +80,11 @@ enum { SOBEK_MAX_L = 4 };
 #define SOBEK_FLAG_UVU 1u      /* channelwise multiplicity mode, Eq. uvu_connection */
 #define SOBEK_FLAG_MUL_IR 2u   /* node features cross the boundary in mul_ir order (see sobek_plan_create) */
 #define SOBEK_FLAG_FAST_GEMM 4u /* node-side GEMMs as plain bf16 products: lower precision, optional */
+#define SOBEK_FLAG_FUSED_FP32 8u   /* schedule: FP32-pipe edge stream feeding the tensor core inside one kernel */
+#define SOBEK_FLAG_FP32_STREAM 16u /* edge stream on the FP32 pipes even where the tensor-core kernel applies */
+#define SOBEK_FLAG_FP32_EDGE 32u   /* edge pass on the FP32 pipes even where the tensor-core kernel applies */
+/* scratch budget in MiB (1 .. 2^20 - 1) in bits 12..31 of the flags word; 0 = the default */
+#define SOBEK_FLAG_STATE_BUDGET_MIB(mb) (((uint32_t)(mb) & 0xFFFFFu) << 12)
 
 /*
  * sobek_plan_create -- the static contract of one layer (Section "Generated
@@ -100,17 +107,16 @@ enum { SOBEK_MAX_L = 4 };
  * and what every stated tolerance refers to) by the single bf16 product a_hi*b_hi with fp32 accumulation: the optional
  * reduced-precision channel GEMM of the paper's runtime contract.  Relative errors of about 1e-2 of the largest output
  * are to be expected; the edge kernels keep their three-pass products; the flag has no effect in the uvu mode.
- * If the environment variable SOBEK_FUSED is set to a
- * non-zero integer when the plan is created, y / gx / ggy / hx are computed by the fused kernels (edge
- * stream feeding the tensor core inside one kernel, receiver state never written to memory); otherwise
- * by the stream -> bounded state -> GEMM schedule, which is the faster one at present.  In that schedule
- * the edge stream and the edge pass run on the tensor cores where the profile allows it (multiplicities
- * that are multiples of 8 / 16, at most 128, K <= 16); SOBEK_TC_STREAM=0 / SOBEK_TC_EDGE=0 at plan
- * creation select the FP32-pipe kernels instead (same results within the tolerances).
- * SOBEK_STATE_BUDGET_MB (an integer number of MiB, default 2048) at plan creation sets the scratch
- * budget (section "Runtime scratch-budget policy"; the paper measures with 128 MiB): the bytes of receiver (or sender) state held at once.  Nodes
- * are processed in chunks that fit the budget, but never fewer than 512 at a time; the results do not
- * depend on the budget beyond the summation order of gR / hR across chunks.
+ * SOBEK_FLAG_FUSED_FP32 selects the fused schedule for y / gx / ggy / hx (FP32-pipe edge stream feeding the tensor
+ * core inside one kernel, receiver state never written to memory); the default is the stream -> bounded state ->
+ * GEMM schedule, which is the faster one at present.  In the default schedule the edge stream and the edge pass run
+ * on the tensor cores where the profile allows it (multiplicities that are multiples of 8 / 16, at most 128,
+ * K <= 16); SOBEK_FLAG_FP32_STREAM / SOBEK_FLAG_FP32_EDGE select the FP32-pipe kernels instead (same results
+ * within the tolerances).
+ * SOBEK_FLAG_STATE_BUDGET_MIB(mb) sets the scratch budget (section "Runtime scratch-budget policy"; the paper
+ * measures with 128 MiB): the bytes of receiver (or sender) state held at once.  Nodes are processed in chunks that
+ * fit the budget, but never fewer than 512 at a time; the results do not depend on the budget beyond the summation
+ * order of gR / hR across chunks.  Without it the budget is 2048 MiB.
  * Errors: INVALID_ARG (null, mul < 1, parity not +-1, K < 1), UNSUPPORTED (l or l_max >
  * SOBEK_MAX_L, or no valid path), CUDA.
  */
@@ -237,7 +243,9 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
  * allocation of any kind (the paper has no counterpart; it exists for hosts of this library
  * that cannot allocate device memory when they run the operator: code running inside another
  * framework's fixed memory plan, real-time loops, processes whose device memory was handed out
- * completely at start-up).  Same inputs, output and results as sobek_conv_fwd.  The scratch that
+ * completely at start-up).  Same inputs and output as sobek_conv_fwd, and the same results within the stated
+ * tolerance (this path always uses the FP32-pipe edge stream and three-pass GEMMs; SOBEK_FLAG_FAST_GEMM is not
+ * honoured; fully connected mode and ir_mul layout only, else UNSUPPORTED).  The scratch that
  * sobek_conv_fwd takes from the caller lives in a fixed array inside the library image:
  * sobek_static_scratch_bytes() bytes (32 MiB) on every GPU that loads the library, held until the
  * process exits.  The call makes no cudaMalloc / cudaFree and calls no allocating routine.
@@ -249,8 +257,13 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
  *   - Every call on a device shares the one array, and the array keeps the previous call's
  *     contents: the call clears what must start at zero itself, but two calls whose kernels
  *     overlap on the GPU (different streams) race.  Serialise them.
+ *   - The plan must have been created on the device that is current at the call (else INVALID_ARG).
+ *   - sobek_static_last_status synchronises `stream` and returns the status word that the kernels of the last
+ *     sobek_conv_fwd_static call on the current device left in the array (0, SOBEK_ERR_DEVICE_TIMEOUT,
+ *     SOBEK_ERR_GRAPH); CUDA if no such call has been made on this device.
  */
 size_t sobek_static_scratch_bytes(void);
+int sobek_static_last_status(void* stream);
 int sobek_conv_fwd_static(const sobek_plan* plan, const sobek_graph* g,
                           const float* x, const float* Y, const float* phi, const float* R,
                           float* y, void* stream);
@@ -263,7 +276,9 @@ int sobek_conv_fwd_static(const sobek_plan* plan, const sobek_graph* g,
 int sobek_selftest_wait_timeout(void* ws, unsigned limit_ms, void* stream);
 
 /* Synchronises `stream`, then returns the status word the kernels of earlier calls wrote
- * into `ws` (0, or SOBEK_ERR_DEVICE_TIMEOUT / SOBEK_ERR_GRAPH ...). */
+ * into `ws`: 0, SOBEK_ERR_DEVICE_TIMEOUT (a bounded wait gave up), or SOBEK_ERR_GRAPH: a segment bound or an
+ * id that a kernel read from row_ptr / col / src_ptr / src_perm / src_recv was out of range.  Such a value is
+ * never used as an index (the edge is skipped or reads row 0 instead), so the outputs are finite but wrong. */
 int sobek_last_device_status(void* ws, void* stream);
 
 const char* sobek_status_string(int status);
@@ -283,6 +298,15 @@ int sobek_timing_enable(int on);
 int sobek_timing_classes(void);
 const char* sobek_timing_class_name(int cls);
 int sobek_timing_collect(double* total_ms, int64_t* launches);
+
+/*
+ * Measures the sustained FP32 multiply-add rate of the current device (instrumentation for the roofline of the
+ * edge kernels; the paper has no counterpart): launches a kernel of independent fused multiply-add chains over and
+ * over for about `seconds` (0 < seconds <= 10) of device time, times it with CUDA events and writes the rate in
+ * TFLOP/s (2 flops per multiply-add) to *tflops (host).  `scratch` is a device buffer of at least
+ * 8192 * (number of SMs) floats that the kernel writes.  Synchronises `stream`.  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+int sobek_measure_fp32_peak(double seconds, float* scratch, size_t scratch_floats, double* tflops, void* stream);
 
 #ifdef __cplusplus
 }

@@ -16,7 +16,7 @@ What is here
     Clebsch-Gordan coefficient with the path normalisation" of
     Eq. angular_path_contraction.
 
-Readings of points the paper leaves open (each also listed in the design notes):
+Readings of points the paper leaves open:
   real basis m = -l..l with sine-type components at m < 0, Condon-Shortley phase
   cancelled (l = 1 is (y, z, x)); unit Frobenius norm for the 3j tensor; sign fixed
   so that the first nonzero entry in lexicographic (m_in, m_sh, m_out) order is

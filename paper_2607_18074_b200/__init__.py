@@ -19,6 +19,16 @@ LIB_PATH = os.path.join(_HERE, "libsobek.so")
 FLAG_UVU = 1      # SOBEK_FLAG_UVU: channelwise multiplicity mode
 FLAG_MUL_IR = 2   # SOBEK_FLAG_MUL_IR: node features cross the boundary in mul_ir order
 FLAG_FAST_GEMM = 4  # SOBEK_FLAG_FAST_GEMM: node-side GEMMs as plain bf16 products (optional, lower precision)
+FLAG_FUSED_FP32 = 8    # SOBEK_FLAG_FUSED_FP32: fused FP32-pipe stream + contraction schedule
+FLAG_FP32_STREAM = 16  # SOBEK_FLAG_FP32_STREAM: edge stream on the FP32 pipes
+FLAG_FP32_EDGE = 32    # SOBEK_FLAG_FP32_EDGE: edge pass on the FP32 pipes
+
+
+def flag_state_budget_mib(mb: int) -> int:
+    """SOBEK_FLAG_STATE_BUDGET_MIB: the scratch budget in MiB, carried in bits 12..31 of the flags word."""
+    if not 1 <= int(mb) < (1 << 20):
+        raise ValueError(mb)
+    return int(mb) << 12
 
 EXPORTS = [
     "sobek_plan_create", "sobek_plan_destroy", "sobek_plan_info", "sobek_plan_path", "sobek_plan_cg",
@@ -26,7 +36,7 @@ EXPORTS = [
     "sobek_conv_bwd", "sobek_conv_dbwd", "sobek_last_device_status", "sobek_status_string",
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
-    "sobek_conv_fwd_retain", "sobek_conv_bwd_retained",
+    "sobek_conv_fwd_retain", "sobek_conv_bwd_retained", "sobek_static_last_status", "sobek_measure_fp32_peak",
 ]
 
 
@@ -90,6 +100,8 @@ def lib():
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
         L.sobek_static_scratch_bytes.restype = c_size_t
         L.sobek_conv_fwd_static.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6
+        L.sobek_static_last_status.argtypes = [c_void_p]
+        L.sobek_measure_fp32_peak.argtypes = [c_double, c_void_p, c_size_t, POINTER(c_double), c_void_p]
         L.sobek_status_string.argtypes = [c_int]
         L.sobek_status_string.restype = c_char_p
         L.sobek_launch_count.restype = c_int64
@@ -137,10 +149,12 @@ class Plan:
     """sobek_plan: irreps are sequences of (mul, l, parity) with parity +1 / -1.  mode "uvw" is the fully
     connected multiplicity mixing, "uvu" the channelwise one (SOBEK_FLAG_UVU).  layout "ir_mul" (block offset +
     m*mul + u) is the kernels' own order of node features, "mul_ir" (block offset + u*(2l+1) + m) is transposed at the
-    boundary (SOBEK_FLAG_MUL_IR)."""
+    boundary (SOBEK_FLAG_MUL_IR).  fused / tc_stream / tc_edge / state_budget_mib map to SOBEK_FLAG_FUSED_FP32,
+    SOBEK_FLAG_FP32_STREAM, SOBEK_FLAG_FP32_EDGE and SOBEK_FLAG_STATE_BUDGET_MIB."""
 
     def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0, mode: str = "uvw",
-                 layout: str = "ir_mul"):
+                 layout: str = "ir_mul", fused: bool = False, tc_stream: bool = True, tc_edge: bool = True,
+                 state_budget_mib: int | None = None):
         if mode not in ("uvw", "uvu"):
             raise ValueError(mode)
         if layout not in ("ir_mul", "mul_ir"):
@@ -149,6 +163,14 @@ class Plan:
             flags |= FLAG_UVU
         if layout == "mul_ir":
             flags |= FLAG_MUL_IR
+        if fused:
+            flags |= FLAG_FUSED_FP32
+        if not tc_stream:
+            flags |= FLAG_FP32_STREAM
+        if not tc_edge:
+            flags |= FLAG_FP32_EDGE
+        if state_budget_mib is not None:
+            flags |= flag_state_budget_mib(state_budget_mib)
         self.layout = "mul_ir" if flags & FLAG_MUL_IR else "ir_mul"
         self.mode = "uvu" if flags & FLAG_UVU else "uvw"
         self._h = c_void_p()
@@ -180,21 +202,6 @@ class Plan:
         out = np.zeros(shape, dtype=np.float64)
         _check(lib().sobek_plan_cg(self._h, k, out.ctypes.data_as(POINTER(c_double))), "sobek_plan_cg")
         return out
-
-    def col_std(self):
-        """1/sqrt(fan_in) per column of R (fan_in = K * sum of input multiplicities over the
-        paths into the column's output block; K * number of those paths in the channelwise mode):
-        the scale used for synthetic weights."""
-        import numpy as np
-        paths = [self.path(k) for k in range(self.info.n_paths)]
-        uvu = self.mode == "uvu"
-        fan = {}
-        for p in paths:
-            fan[p.i_out] = fan.get(p.i_out, 0) + (1 if uvu else p.c_in)
-        std = np.zeros(self.info.N_w)
-        for p in paths:
-            std[p.w_off:p.w_off + (p.c_in if uvu else p.c_in * p.c_out)] = (self.info.K * fan[p.i_out]) ** -0.5
-        return std
 
 
 def _ptr(t):
@@ -235,8 +242,12 @@ def graph_receivers(row_ptr, src_perm):
 
 
 def make_graph(row_ptr, col, src_ptr=None, src_perm=None, src_recv=None) -> Graph:
-    return Graph(row_ptr.numel() - 1, col.numel(), _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm),
-                 _ptr(src_recv))
+    """The sobek_graph descriptor of five CUDA tensors.  The descriptor holds raw device addresses, so the
+    returned object also keeps references to the tensors: they stay allocated for as long as it lives."""
+    g = Graph(row_ptr.numel() - 1, col.numel(), _ptr(row_ptr), _ptr(col), _ptr(src_ptr), _ptr(src_perm),
+              _ptr(src_recv))
+    g.tensors = (row_ptr, col, src_ptr, src_perm, src_recv)
+    return g
 
 
 def workspace_bytes(plan: Plan, N: int, E: int, order: int) -> int:
@@ -258,6 +269,11 @@ def conv_fwd_static(plan, graph, x, Y, phi, R, y):
     sobek_conv_fwd_static in include/sobek.h for the size limit and the sharing rules)."""
     _check(lib().sobek_conv_fwd_static(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R),
                                        _ptr(y), _stream()), "sobek_conv_fwd_static")
+
+
+def static_last_status() -> int:
+    """Status word left by the kernels of the last conv_fwd_static call on the current device (synchronises)."""
+    return int(lib().sobek_static_last_status(_stream()))
 
 
 def conv_bwd(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws):
@@ -288,6 +304,17 @@ def conv_dbwd(plan, graph, x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi
                                  _ptr(vx), _ptr(vY), _ptr(vphi), _ptr(vR), _ptr(ggy), _ptr(hx), _ptr(hY),
                                  _ptr(hphi), _ptr(hR), _ptr(ws), ws.numel() * ws.element_size(),
                                  _stream()), "sobek_conv_dbwd")
+
+
+def measure_fp32_peak(seconds: float = 1.0) -> float:
+    """Sustained FP32 multiply-add rate of the current device in TFLOP/s (sobek_measure_fp32_peak)."""
+    import torch
+    n = 8192 * torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    scratch = torch.empty(n, dtype=torch.float32, device="cuda")
+    out = c_double(0.0)
+    _check(lib().sobek_measure_fp32_peak(float(seconds), _ptr(scratch), n, byref(out), _stream()),
+           "sobek_measure_fp32_peak")
+    return float(out.value)
 
 
 def selftest_wait_timeout(ws, limit_ms: int = 200):

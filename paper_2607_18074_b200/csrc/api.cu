@@ -123,6 +123,14 @@ int check_common(const sobek_plan* p, const sobek_graph* g, void* ws, size_t ws_
     return SOBEK_OK;
 }
 
+// every floating-point array argument must start on a 16-byte boundary (NULL passes: "not given")
+template <class... P>
+bool aligned16(P... ptrs) {
+    uintptr_t m = 0;
+    ((m |= (uintptr_t)ptrs), ...);
+    return (m & 15) == 0;
+}
+
 #define CK(expr)                                              \
     do {                                                      \
         cudaError_t e__ = (expr);                             \
@@ -298,6 +306,7 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     int rc = check_common(p, g, ws, ws_bytes, order);
     if (rc) return rc;
     if (!y || !R || (g->N > 0 && !x) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!aligned16(x, Y, phi, R, y)) return SOBEK_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, order, ws);
     CK(cudaMemsetAsync(w.status, 0, kHeaderBytes, s));
@@ -329,6 +338,7 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     int rc = check_common(p, g, ws, ws_bytes, 1);
     if (rc) return rc;
     if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!aligned16(x, Y, phi, R, gy, gx, gY, gphi, gR)) return SOBEK_ERR_INVALID_ARG;
     if (gx && g->E > 0 && (!g->src_ptr || !g->src_perm)) return SOBEK_ERR_NEED_TRANSPOSE;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, 1, ws);
@@ -363,7 +373,7 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
                 } else {
                     CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, w.zbar, w.status, s));
                     CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
-                                        gphi ? 1 : 0, gY ? 1 : 0, s));
+                                        gphi ? 1 : 0, gY ? 1 : 0, w.status, s));
                 }
             }
         }
@@ -395,6 +405,7 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
     int rc = check_common(p, g, ws, ws_bytes, 2);
     if (rc) return rc;
     if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!aligned16(x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi, hR)) return SOBEK_ERR_INVALID_ARG;
     if (hx && g->E > 0 && (!g->src_ptr || !g->src_perm)) return SOBEK_ERR_NEED_TRANSPOSE;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, 2, ws);
@@ -476,7 +487,7 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
                     } else {
                         CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, w.zbar, w.status, s));
                         CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, vx, Y, vY, phi, vphi, 1, w.zbar, hphi, hY,
-                                            hphi ? pm : 0, hY ? ym : 0, s));
+                                            hphi ? pm : 0, hY ? ym : 0, w.status, s));
                     }
                     pm = ym = 2;
                 }
@@ -489,7 +500,7 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
                     } else {
                         CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.vfKNh, w.vfKNl, gy, vR, w.zbar, w.status, s));
                         CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, hphi, hY,
-                                            hphi ? pm : 0, hY ? ym : 0, s));
+                                            hphi ? pm : 0, hY ? ym : 0, w.status, s));
                     }
                 }
             }

@@ -20,6 +20,7 @@
 //     hphi_e += <Zbar, C(vx,Y) + C(x,vY)>,   hY_e += CG^T_Y(vx, phi Zbar) + CG^T_Y(x, vphi Zbar).
 #include <algorithm>
 
+#include "guard.cuh"
 #include "internal.h"
 
 namespace sobek {
@@ -49,6 +50,7 @@ struct EdgeArgs {
     int K, dsh, C_src, phi_mode, Y_mode;
     int warp_floats;     // shared floats per warp
     int zslab;           // floats of one Zbar slab buffer
+    int* status;         // device status word (range guards report SOBEK_ERR_GRAPH there)
     int zvec;            // 1: every row pitch and offset of Zbar is a multiple of 4 floats (16-byte pieces may be copied)
 };
 
@@ -273,11 +275,13 @@ k_edge_pass(const EdgeArgs a, const int t_begin, const int t_count) {
     const int nw = blockDim.x >> 5;
     for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
         const int64_t node = a.node0 + nl;
-        const int64_t seg0 = a.ev.ptr[node], seg1 = a.ev.ptr[node + 1];
+        int64_t seg0, seg1;
+        seg_bounds(a.ev.ptr, node, a.ev.E, a.status, seg0, seg1);
         for (int64_t b0 = seg0; b0 < seg1; b0 += 32) {
             const int64_t e = b0 + lane;
             const bool valid = e < seg1;
-            const int64_t sn = (int64_t)a.ev.col[valid ? e : seg0];
+            int64_t sn = (int64_t)a.ev.col[valid ? e : seg0];   // e < seg1 <= E, or seg0 < seg1
+            if (!id_ok(sn, a.ev.N, a.status)) sn = 0;          // reported; the edge then reads node 0
             for (int b = 0; b < a.dsh; ++b) {
                 sY[b * 32 + lane] = valid ? a.Y[e * a.dsh + b] : 0.f;
                 if (has_vY) sVY[b * 32 + lane] = valid ? a.vY[e * a.dsh + b] : 0.f;
@@ -395,9 +399,10 @@ void build_edge_tasks(const sobek_plan* p, Direction& dir) {
 cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
                              int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
                              const float* phi, const float* vphi, int dual, const float* Zbar, float* gphi,
-                             float* gY, int phi_mode, int Y_mode, cudaStream_t s) {
+                             float* gY, int phi_mode, int Y_mode, int* status, cudaStream_t s) {
     if (n_nodes <= 0 || dir.etasks.empty()) return cudaSuccess;
     EdgeArgs a{};
+    a.status = status;
     a.tasks = dir.d_etasks; a.comps = dir.d_ecomps; a.groups = dir.d_groups;
     a.tab_ptr = p->d_tab_ptr; a.tab_idx = p->d_tab_idx; a.tab_coef = p->d_tab_coef;
     a.ev = ev; a.node0 = node0; a.n_nodes = n_nodes;

@@ -29,6 +29,7 @@
 
 #include <algorithm>
 
+#include "guard.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -54,6 +55,7 @@ struct EtArgs {
     const int64_t* row_ptr;
     const int32_t* col;
     int64_t node0, n_nodes;
+    int64_t N, E;               // sizes of the graph: every gathered id and segment bound is checked against them
     const __nv_bfloat16* sh;
     const __nv_bfloat16* sl;
     const __nv_bfloat16* vsh;
@@ -202,8 +204,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         const int lt = (warp - NCW) * 32 + lane;
         uint32_t it = 0, zi = 0;
         for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
-            const int64_t node = a.node0 + nl;
-            const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
+            int64_t seg0, seg1;
+            seg_bounds(a.row_ptr, a.node0 + nl, a.E, a.status, seg0, seg1);
+            if (!any_op) seg1 = seg0;
             if (seg1 <= seg0) continue;
             // ---- Zbar slabs of the receiver (once the previous receiver's MMAs have read theirs)
             if (zi > 0) mbar_wait(bar_zfree, (zi - 1) & 1, a.status);
@@ -237,7 +240,11 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 const uint32_t raw_u = stage_u + (uint32_t)(2 * a.x_cap);
                 // sender ids of the batch (each loader warp keeps its own copy of all of them)
                 int32_t* sIds = reinterpret_cast<int32_t*>(stage + 2 * a.x_cap) + NRAW * tb * KP + NRAW * a.dsh * PS + (warp - NCW) * 0;
-                for (int e = lane; e < tb; e += 32) sIds[e] = e < nb ? a.col[b0 + e] : 0;
+                for (int e = lane; e < tb; e += 32) {      // -1: no such edge, or a sender id out of range (reported)
+                    int32_t sid = -1;
+                    if (e < nb) { sid = a.col[b0 + e]; if (!id_ok(sid, a.N, a.status)) sid = -1; }
+                    sIds[e] = sid;
+                }
                 __syncwarp();
                 {
                     const bool v16 = (a.K & 3) == 0;
@@ -274,10 +281,11 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                     const int npair = tb * cpr;
                     for (int pr = lt; pr < npair; pr += NLW * 32) {
                         const int e = pr / cpr, j = pr - e * cpr;
-                        const uint32_t ok = e < nb ? 16u : 0u;
+                        const int32_t sid = sIds[e];
+                        const uint32_t ok = sid >= 0 ? 16u : 0u;
                         const int u = 8 * j;
                         uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + e * 128 + ((((u & 63) >> 3) ^ (e & 7)) << 4));
-                        const int64_t g = (int64_t)sIds[e] * a.C_src + B.src_off + u;
+                        const int64_t g = (int64_t)max(sid, 0) * a.C_src + B.src_off + u;
                         const __nv_bfloat16* ph = (op == 0 ? a.sh : a.vsh) + g;
                         const __nv_bfloat16* pl = (op == 0 ? a.sl : a.vsl) + g;
                         for (int sdx = 0; sdx < B.d_src; ++sdx) {
@@ -296,8 +304,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             uint32_t it = 0, zi = 0, ai = 0;
             const uint32_t sZ_u = smem_u32(sZ);
             for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
-                const int64_t node = a.node0 + nl;
-                const int64_t seg0 = a.row_ptr[node], seg1 = any_op ? a.row_ptr[node + 1] : seg0;
+                int64_t seg0, seg1;
+                seg_bounds(a.row_ptr, a.node0 + nl, a.E, nullptr, seg0, seg1);
+                if (!any_op) seg1 = seg0;
                 if (seg1 <= seg0) continue;
                 mbar_wait(bar_zfull, zi & 1, a.status);
                 ++zi;
@@ -344,10 +353,10 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
         const int t8 = tb >> 3;                      // 8-edge octets per batch
         // bounds of the next receiver, requested one receiver ahead
         int64_t nx0 = 0, nx1 = 0;
-        if ((int64_t)blockIdx.x < a.n_nodes) { nx0 = a.row_ptr[a.node0 + blockIdx.x]; nx1 = a.row_ptr[a.node0 + blockIdx.x + 1]; }
+        if ((int64_t)blockIdx.x < a.n_nodes) seg_bounds(a.row_ptr, a.node0 + blockIdx.x, a.E, nullptr, nx0, nx1);
         for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
             const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
-            if (nl + gridDim.x < a.n_nodes) { nx0 = a.row_ptr[a.node0 + nl + gridDim.x]; nx1 = a.row_ptr[a.node0 + nl + gridDim.x + 1]; }
+            if (nl + gridDim.x < a.n_nodes) seg_bounds(a.row_ptr, a.node0 + nl + gridDim.x, a.E, nullptr, nx0, nx1);
             {
                 for (int64_t b0 = seg0; b0 < seg1; b0 += tb) {
                     const int nb = (int)min((int64_t)tb, seg1 - b0);     // edges of the batch
@@ -689,7 +698,7 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     if (n_nodes <= 0) return cudaSuccess;
     EtArgs a{};
     a.sets = T.d_sets; a.units = T.d_units; a.blks = T.d_blks; a.comps = T.d_comps_s;
-    a.row_ptr = ev.ptr; a.col = ev.col; a.node0 = node0; a.n_nodes = n_nodes;
+    a.row_ptr = ev.ptr; a.col = ev.col; a.node0 = node0; a.n_nodes = n_nodes; a.N = ev.N; a.E = ev.E;
     a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;

@@ -72,7 +72,7 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
     a.ev = ev; a.node0 = node0; a.n_nodes = n_nodes;
     a.src = src; a.vsrc = vsrc; a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zh = zh; a.zl = zl;
-    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.warp_floats = 0;
+    a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.warp_floats = 0; a.status = status;
     Fork fork(p, s);   // the kernel classes touch disjoint parts of the state: run them concurrently
     for (const auto& c : dir.sclasses) {
         cudaStream_t cs = fork.pick();

@@ -24,6 +24,7 @@ struct StreamArgs {
     void* zl;
     int32_t K, dsh, C_src;
     int32_t warp_floats;       // shared floats per warp
+    int* status;               // device status word (range guards report SOBEK_ERR_GRAPH there); may be NULL
 };
 
 

@@ -19,6 +19,7 @@
 #include <cuda_bf16.h>
 
 #include "edge_stream_args.h"
+#include "guard.cuh"
 #include "internal.h"
 
 namespace sobek {
@@ -51,7 +52,8 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
     float* sVY = sVphi + S_EB * KC;                // DUAL: [EB][YS]
 
     const int64_t node = a.node0 + nl;
-    const int64_t seg0 = a.ev.ptr[node], seg1 = a.ev.ptr[node + 1];
+    int64_t seg0, seg1;
+    seg_bounds(a.ev.ptr, node, a.ev.E, a.status, seg0, seg1);
     const int u = T.u0 + lane;
     const bool act = u < T.c_src;
     const bool has_vx = DUAL && a.vsrc != nullptr, has_vY = DUAL && a.vY != nullptr,
@@ -71,9 +73,13 @@ __device__ __forceinline__ void run_task(const StreamArgs& a, const STask T, con
             __syncwarp();
             if (lane < nb) {
                 const int64_t pos = b0 + lane;
-                const int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
+                // an id out of range is reported; the edge then reads edge 0 / node 0 (valid memory, wrong data)
+                int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
+                if (!id_ok(eid, a.ev.E, a.status)) eid = 0;
                 sE[lane] = (int32_t)eid;
-                sSrc[lane] = a.ev.transposed ? (int32_t)owner_of(a.ev.row_ptr, a.ev.N, eid) : a.ev.col[eid];
+                int64_t sn = a.ev.transposed ? owner_of(a.ev.row_ptr, a.ev.N, eid) : (int64_t)a.ev.col[eid];
+                if (!id_ok(sn, a.ev.N, a.status)) sn = 0;
+                sSrc[lane] = (int32_t)sn;
             }
             __syncwarp();
             for (int i = lane; i < nb * a.dsh; i += 32) {

@@ -20,6 +20,7 @@
 #pragma once
 #include <cuda_bf16.h>
 
+#include "guard.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -69,7 +70,7 @@ __device__ __forceinline__ void produce(const FusedArgs& a, const FStage st, con
                has_vphi = DUAL && a.vphi != nullptr;
 
     int64_t seg0 = 0, seg1 = 0;
-    if (has_node) { seg0 = a.ev.ptr[n0 + t]; seg1 = a.ev.ptr[n0 + t + 1]; }
+    if (has_node) seg_bounds(a.ev.ptr, n0 + t, a.ev.E, a.status, seg0, seg1);
     int deg = (int)(seg1 - seg0);
     int maxdeg = deg;
 #pragma unroll
@@ -86,9 +87,13 @@ __device__ __forceinline__ void produce(const FusedArgs& a, const FStage st, con
         __syncwarp();
         if (ul < nb) {
             const int64_t pos = seg0 + b0 + ul;
-            const int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
+            // an id out of range is reported; the edge then reads edge 0 / node 0 (valid memory, wrong data)
+            int64_t eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
+            if (!id_ok(eid, a.ev.E, a.status)) eid = 0;
             sE[ul] = (int32_t)eid;
-            sSrc[ul] = a.ev.transposed ? (int32_t)f_owner_of(a.ev.row_ptr, a.ev.N, eid) : a.ev.col[eid];
+            int64_t sn = a.ev.transposed ? f_owner_of(a.ev.row_ptr, a.ev.N, eid) : (int64_t)a.ev.col[eid];
+            if (!id_ok(sn, a.ev.N, a.status)) sn = 0;
+            sSrc[ul] = (int32_t)sn;
         }
         __syncwarp();
         for (int i = ul; i < nb * a.dsh; i += US) {

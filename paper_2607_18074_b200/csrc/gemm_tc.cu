@@ -19,7 +19,6 @@
 // if it gives up it records SOBEK_ERR_DEVICE_TIMEOUT in the status word and carries on, so the
 // kernel always reaches its TMEM release and returns.
 #include <cuda_bf16.h>
-#include <stdio.h>
 
 #include "internal.h"
 #include "ptx.cuh"

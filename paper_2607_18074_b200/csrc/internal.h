@@ -310,7 +310,7 @@ cudaError_t launch_edge_pass(const sobek_plan* p, const Direction& dir, const Ed
                              int64_t n_nodes, const float* src, const float* vsrc, const float* Y, const float* vY,
                              const float* phi, const float* vphi, int dual, const float* Zbar, float* gphi,
                              float* gY, int phi_mode, int Y_mode /* 0 skip, 1 overwrite, 2 accumulate */,
-                             cudaStream_t s);
+                             int* status, cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, int64_t n, cudaStream_t s);
 // [N][C] node features between the two block orders: to_ir_mul = 1: dst[m*C_b + u] = src[u*d + m] inside every block
 cudaError_t launch_relayout(const float* src, float* dst, int64_t N, int C, const int4* blocks, int nblk, int to_ir_mul,

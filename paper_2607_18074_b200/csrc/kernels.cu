@@ -4,8 +4,8 @@
 //                           back into the layout of R[K, N_w]
 // (the edge stream lives in edge_stream*.cu, the receiver-owned edge pass in edge_pass.cu, the
 //  node-side contractions in gemm_tc.cu)
-#include <stdio.h>
 
+#include <algorithm>
 #include <atomic>
 #include <type_traits>
 #include <vector>
@@ -196,3 +196,65 @@ cudaError_t launch_unpack_R(const sobek_plan* p, const Direction& dir, const flo
 }
 
 }  // namespace sobek
+
+// ---- FP32 multiply-add peak of the device, measured (instrumentation; the paper has no counterpart) ----------
+// Every thread runs 16 independent fused multiply-add chains, so that the FP32 pipes never wait for a result:
+// 2 x 16 x FMA_ITERS flops per thread.  The accumulators are stored at the end so that the loop is not removed.
+namespace sobek {
+namespace {
+constexpr int FMA_ITERS = 1 << 14;
+__global__ void __launch_bounds__(1024) k_fma_peak(float* out, float a, float b) {
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = (float)(threadIdx.x + i);
+#pragma unroll 1
+    for (int it = 0; it < FMA_ITERS; it += 4) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], a, b);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += acc[i];
+    out[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+}  // namespace
+}  // namespace sobek
+
+extern "C" int sobek_measure_fp32_peak(double seconds, float* scratch, size_t scratch_floats, double* tflops, void* stream) {
+    using namespace sobek;
+    if (!tflops || !scratch || !(seconds > 0.0) || seconds > 10.0) return SOBEK_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SOBEK_ERR_CUDA;
+    }
+    const int blocks = sms * 2 * 4, threads = 1024;     // 2 resident CTAs of 1024 threads per SM, four waves
+    if (scratch_floats < (size_t)blocks * threads) return SOBEK_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { (void)cudaGetLastError(); return SOBEK_ERR_CUDA; }
+    const double flops_per_launch = 2.0 * 16.0 * FMA_ITERS * (double)blocks * threads;
+    double total_ms = 0.0, best = 0.0;
+    int launches = 0;
+    int rc = SOBEK_OK;
+    k_fma_peak<<<blocks, threads, 0, s>>>(scratch, 1.0000001f, 1e-7f);     // warm-up
+    while (total_ms < seconds * 1e3 && launches < 100000) {
+        cudaEventRecord(e0, s);
+        for (int r = 0; r < 8; ++r) k_fma_peak<<<blocks, threads, 0, s>>>(scratch, 1.0000001f, 1e-7f);
+        cudaEventRecord(e1, s);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { rc = SOBEK_ERR_CUDA; break; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        count_launch(8);
+        total_ms += ms; launches += 8;
+        if (ms > 0.f) best = std::max(best, 8.0 * flops_per_launch / (ms * 1e-3) / 1e12);
+    }
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (cudaGetLastError() != cudaSuccess) rc = SOBEK_ERR_CUDA;
+    // the sustained figure: all launches over all the time
+    *tflops = total_ms > 0.0 ? launches * flops_per_launch / (total_ms * 1e-3) / 1e12 : 0.0;
+    (void)best;
+    return rc;
+}

@@ -10,7 +10,6 @@
 // made positive, and the path normalisation sqrt(2 l_out + 1) of Eq. angular_path_contraction
 // is applied.
 #include <math.h>
-#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -385,7 +384,7 @@ using namespace sobek;
 
 extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
                                  int l_max, int K, uint32_t flags, sobek_plan** plan) {
-    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR | SOBEK_FLAG_FAST_GEMM)) != 0 || l_max < 0)
+    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & 0xFFFu & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR | SOBEK_FLAG_FAST_GEMM | SOBEK_FLAG_FUSED_FP32 | SOBEK_FLAG_FP32_STREAM | SOBEK_FLAG_FP32_EDGE)) != 0 || l_max < 0)
         return SOBEK_ERR_INVALID_ARG;
     *plan = nullptr;
     if (l_max > SOBEK_MAX_L) return SOBEK_ERR_UNSUPPORTED;
@@ -452,20 +451,16 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
         const double nrm = sqrt(2.0 * p->paths[k].info.l_out + 1.0);
         for (double& v : p->paths[k].cg) v *= nrm;
     }
-    if (const char* e = getenv("SOBEK_FUSED")) p->use_fused = atoi(e) != 0;
-    if (p->uvu) p->use_fused = false;   // the fused kernels contain the channel-mixing GEMM
-    if (const char* e = getenv("SOBEK_STATE_BUDGET_MB")) {
-        const long mb = atol(e);
-        if (mb >= 1 && mb <= (1L << 20)) p->state_budget = size_t(mb) << 20;
-    }
+    p->use_fused = (flags & SOBEK_FLAG_FUSED_FP32) != 0 && !p->uvu;   // the fused kernels contain the channel-mixing GEMM
+    p->use_tc_stream = (flags & SOBEK_FLAG_FP32_STREAM) == 0;
+    p->use_tc_edge = (flags & SOBEK_FLAG_FP32_EDGE) == 0;
+    if (const uint32_t mb = flags >> 12) p->state_budget = size_t(mb) << 20;
     build_direction(p, 0, p->fwd);
     build_direction(p, 1, p->tr);
     build_stream_tasks(p, p->fwd);
     build_stream_tasks(p, p->tr);
-    if (const char* e = getenv("SOBEK_TC_STREAM")) p->use_tc_stream = atoi(e) != 0;
     build_tc_sets(p, p->fwd);
     build_tc_sets(p, p->tr);
-    if (const char* e = getenv("SOBEK_TC_EDGE")) p->use_tc_edge = atoi(e) != 0;
     build_tc_edge_sets(p, p->fwd);
     build_edge_tasks(p, p->fwd);
     build_fused_stages(p, p->fwd);

@@ -29,6 +29,20 @@ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 extern "C" size_t sobek_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
+// The status word of the array on the current device (the kernels' bounded waits and range guards write it).
+extern "C" int sobek_static_last_status(void* stream) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices || !g_scratch_addr[dev]) {
+        (void)cudaGetLastError();
+        return SOBEK_ERR_CUDA;
+    }
+    int h = 0;
+    cudaError_t e = cudaMemcpyAsync(&h, g_scratch_addr[dev], sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return SOBEK_ERR_CUDA; }
+    return h;
+}
+
 extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, const float* x,
                                      const float* Y, const float* phi, const float* R, float* y,
                                      void* stream) {
@@ -43,6 +57,8 @@ extern "C" int sobek_conv_fwd_static(const sobek_plan* p, const sobek_graph* g, 
         (void)cudaGetLastError();
         return SOBEK_ERR_CUDA;
     }
+    if (dev != p->device) return SOBEK_ERR_INVALID_ARG;   // the plan's tables live on the device it was created on
+    if ((((uintptr_t)x | (uintptr_t)Y | (uintptr_t)phi | (uintptr_t)R | (uintptr_t)y) & 15) != 0) return SOBEK_ERR_INVALID_ARG;
     if (!g_scratch_addr[dev]) {   // set-up on the first call on this device
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {

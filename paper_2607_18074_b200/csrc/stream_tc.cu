@@ -31,6 +31,7 @@
 
 #include <algorithm>
 
+#include "guard.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -243,9 +244,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         ItemPos lp; lp.init(p_item, a.n_nodes);
         auto prefetch_item = [&]() {
             if (p_item < total) {
-                const int64_t node = a.node0 + lp.nl;
-                p_seg0 = a.ev.ptr[node];
-                p_seg1 = any_op ? a.ev.ptr[node + 1] : p_seg0;
+                seg_bounds(a.ev.ptr, a.node0 + lp.nl, a.ev.E, a.status, p_seg0, p_seg1);
+                if (!any_op) p_seg1 = p_seg0;
             }
         };
         prefetch_item();
@@ -264,26 +264,37 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
             return true;
         };
-        auto load_ids = [&](const Cur& c, int64_t& eid, int32_t& sn) {   // lane e < 16 holds edge e of the batch
+        // lane e < 16 holds edge e of the batch; bit e of msk says that the edge exists and that its ids are in
+        // range (an id that is not turns the edge's copies into zero fills and is reported in the status word)
+        auto load_ids = [&](const Cur& c, int64_t& eid, int32_t& sn, uint32_t& msk) {
             eid = 0; sn = 0;
+            bool ok = false;
             if (c.b0 + lane < c.seg1 && lane < TB) {
                 const int64_t pos = c.b0 + lane;
                 eid = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos;
-                sn = a.ev.transposed ? (a.ev.recv ? a.ev.recv[pos] : (int32_t)owner_of(a.ev.row_ptr, a.ev.N, eid)) : a.ev.col[eid];
+                ok = id_ok(eid, a.ev.E, a.status);
+                if (ok) {
+                    const int64_t v = a.ev.transposed ? (a.ev.recv ? (int64_t)a.ev.recv[pos] : owner_of(a.ev.row_ptr, a.ev.N, eid))
+                                                      : (int64_t)a.ev.col[eid];
+                    ok = id_ok(v, a.ev.N, a.status);
+                    sn = ok ? (int32_t)v : 0;
+                } else {
+                    eid = 0;
+                }
             }
+            msk = __ballot_sync(0xffffffffu, ok);
         };
         Cur cur{0, 0, 0, 0};
         bool have = next_batch(cur, true);
-        int64_t eid = 0; int32_t sn = 0;
-        if (have) load_ids(cur, eid, sn);
+        int64_t eid = 0; int32_t sn = 0; uint32_t msk = 0;
+        if (have) load_ids(cur, eid, sn, msk);
         for (uint32_t it = 0; have; ++it) {
             Cur nxt = cur;
             const bool have_n = next_batch(nxt, false);
-            int64_t eid_n = 0; int32_t sn_n = 0;
-            if (have_n) load_ids(nxt, eid_n, sn_n);
+            int64_t eid_n = 0; int32_t sn_n = 0; uint32_t msk_n = 0;
+            if (have_n) load_ids(nxt, eid_n, sn_n, msk_n);
             const TSet S = sSet[cur.set];
             const int op = has_a1 ? cur.sub : 1;
-            const int nb = (int)min((int64_t)TB, cur.seg1 - cur.b0);
             const int st = (int)(it % NS);
             if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
             const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
@@ -298,7 +309,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     const int e = min(i / per, TB - 1), j = i - (i / per) * per;
                     const int64_t ee = __shfl_sync(0xffffffffu, eid, e);
                     if (i < n_it) {
-                        const uint32_t ok = e < nb ? 1u : 0u;
+                        const uint32_t ok = (msk >> e) & 1u;
                         if (v16) {
                             cp_async16_zfill(raw_u + (uint32_t)(e * KP + 4 * j) * 4, a.phi + ee * a.K + 4 * j, ok * 16);
                             if (has_vphi) cp_async16_zfill(raw_u + (uint32_t)(TB * KP + e * KP + 4 * j) * 4, a.vphi + ee * a.K + 4 * j, ok * 16);
@@ -314,7 +325,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
             {
                 const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
-                const uint32_t ok = le < nb ? 4u : 0u;
+                const uint32_t ok = ((msk >> le) & 1u) * 4u;
                 const float* yr = a.Y + ee_own * a.dsh;
                 const float* vyr = has_vY ? a.vY + ee_own * a.dsh : nullptr;
                 for (int b = lt >> 4; b < a.dsh; b += NLW * 32 / TB) {
@@ -327,7 +338,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 // lanes 2e, 2e+1 of each loader warp serve edge e; a thread walks pieces j0, j0 + 4, ... of the row
                 const int re = (lane >> 1) & (TB - 1);
                 const int32_t sne = __shfl_sync(0xffffffffu, sn, re);
-                const uint32_t ok = re < nb ? 16u : 0u;
+                const uint32_t ok = ((msk >> re) & 1u) * 16u;
                 const int j0 = (lane & 1) | ((lt >> 5) << 1);
                 const int64_t grow = (int64_t)sne * a.C_src;
                 const __nv_bfloat16* srch = (op == 0 ? a.sh : a.vsh) + grow;
@@ -353,7 +364,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
             // this thread's arrival on the stage's barrier fires when all its copies above have landed
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_full + 8 * st) : "memory");
-            cur = nxt; have = have_n; eid = eid_n; sn = sn_n;
+            cur = nxt; have = have_n; eid = eid_n; sn = sn_n; msk = msk_n;
         }
     } else if (warp == NCW + NLW) {
         // =========================== MMA warp ===========================
@@ -361,16 +372,14 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             uint32_t it = 0, mi = 0;
             int64_t nx0 = 0, nx1 = 0;
             ItemPos mp; mp.init(blockIdx.x, a.n_nodes);      // position of the item whose bounds are in flight
-            if ((int64_t)blockIdx.x < total) { const int64_t nn = a.node0 + mp.nl; nx0 = a.ev.ptr[nn]; nx1 = a.ev.ptr[nn + 1]; }
+            if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
             const uint64_t acap16 = (uint64_t)(a.a_cap >> 4), bcap16 = (uint64_t)(a.b_cap >> 4);
             for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
                 const TSet S = sSet[mp.set];
                 const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
                 mp.step(gridDim.x, a.n_nodes);
-                if (item + gridDim.x < total) {     // the next item's bounds, requested one item ahead
-                    const int64_t nn = a.node0 + mp.nl;
-                    nx0 = a.ev.ptr[nn]; nx1 = a.ev.ptr[nn + 1];
-                }
+                if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
+                    seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
                 if (seg1 <= seg0) continue;
                 const uint32_t buf = mi & 1;
                 if (mi >= 2) mbar_wait(bar_accfree + 8 * buf, ((mi >> 1) & 1) ^ 1, a.status);
@@ -426,7 +435,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         int cur_set = -1;
         int64_t cx0 = 0, cx1 = 0;
         ItemPos cp_; cp_.init(blockIdx.x, a.n_nodes);        // position of the item whose bounds are in flight
-        if ((int64_t)blockIdx.x < total) { const int64_t nn = a.node0 + cp_.nl; cx0 = a.ev.ptr[nn]; cx1 = a.ev.ptr[nn + 1]; }
+        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
         // the item whose accumulator is drained next (one behind the one being built)
         int64_t p_nl = -1; int p_set = 0; uint32_t p_mi = 0; bool p_wrote = false;
 
@@ -512,10 +521,8 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             const TSet S = sSet[set];
             const int64_t seg0 = cx0, seg1 = any_op ? cx1 : cx0;
             cp_.step(gridDim.x, a.n_nodes);
-            if (item + gridDim.x < total) {     // the next item's bounds, requested one item ahead
-                const int64_t nn = a.node0 + cp_.nl;
-                cx0 = a.ev.ptr[nn]; cx1 = a.ev.ptr[nn + 1];
-            }
+            if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
+                seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
             if (set != cur_set && seg1 > seg0) {     // entry and sparse-term tables of the set
                 compute_sync();
                 for (int i = tid; i < S.nent; i += NCW * 32) sEnt[i] = a.ents[S.ent_begin + i];

@@ -19,13 +19,13 @@ def rel_err(got, ref):
 class Case:
     """One workload on the GPU and in the oracle."""
 
-    def __init__(self, w: synth.Workload, inputs=None):
+    def __init__(self, w: synth.Workload, inputs=None, **plan_options):
         import torch
         import paper_2607_18074_b200 as sb
         self.sb, self.torch = sb, torch
         self.w = w
         self.oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
-        self.plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
+        self.plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode, **plan_options)
         self.d = inputs if inputs is not None else synth.make_inputs(w, self.oracle.col_std())
         d = self.d
         dev = "cuda:0"

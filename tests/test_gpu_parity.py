@@ -190,6 +190,58 @@ def test_errors_on_device_calls(cases):
     assert ei.value.code == -5
 
 
+@pytest.mark.parametrize("fp32_pipe", [False, True])
+def test_stale_graph_arrays_are_reported_not_followed(fp32_pipe):
+    """The graph arrays are the caller's: an entry that is out of range when a kernel reads it (a freed or
+    overwritten buffer) must end in SOBEK_ERR_GRAPH in the status word with finite outputs, never in an
+    access through the bad value.  One corrupted entry per array, positive and negative, all three orders."""
+    import torch
+    opts = dict(tc_stream=False, tc_edge=False) if fp32_pipe else {}
+    c = Case(CASES["cfg1"], **opts)
+    sb, i = c.sb, c.plan.info
+    names = ("row_ptr", "col", "src_ptr", "src_perm", "src_recv")
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
+    for which, pos, bad in (("col", 5, c.N + 1000), ("col", 0, -3), ("src_recv", 7, 2 ** 30), ("src_recv", 1, -1),
+                            ("src_perm", 3, c.E + 5), ("src_perm", c.E - 1, -7), ("row_ptr", c.N, c.E + 1000),
+                            ("row_ptr", 3, -4), ("src_ptr", 2, 2 ** 40)):
+        arrs = {n: getattr(c, n).clone() for n in names}
+        arrs[which][pos] = bad
+        g = sb.make_graph(*[arrs[n] for n in names])
+        assert all(a is b for a, b in zip(g.tensors, [arrs[n] for n in names]))     # the descriptor keeps them alive
+        touched = {"col": (0, 1, 2), "row_ptr": (0, 1, 2)}.get(which, (1, 2))        # the forward reads only the receiver CSR
+        for order in (0, 1, 2):
+            ws = c.ws(order)
+            if order == 0:
+                outs = [new(c.N, i.C_y)]
+                sb.conv_fwd(c.plan, g, c.x, c.Y, c.phi, c.R, *outs, ws)
+            elif order == 1:
+                outs = [new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)]
+                sb.conv_bwd(c.plan, g, c.x, c.Y, c.phi, c.R, c.gy, *outs, ws)
+            else:
+                outs = [new(c.N, i.C_y), new(c.N, i.C_x), new(c.E, i.dim_sh), new(c.E, i.K), new(i.K, i.N_w)]
+                sb.conv_dbwd(c.plan, g, c.x, c.Y, c.phi, c.R, c.gy, c.vx, c.vY, c.vphi, c.vR, *outs, ws)
+            status = sb.last_device_status(ws)
+            assert status == (-4 if order in touched else 0), (which, pos, order, status)
+            for o in outs:
+                assert torch.isfinite(o).all(), (which, pos, order)
+    # and the context is intact: the untouched graph still gives the right answer
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+
+
+def test_misaligned_arrays_are_refused(cases):
+    """Floating-point arrays must start on a 16-byte boundary (16-byte pieces of their rows are copied)."""
+    import torch
+    c = get(cases, "cfg1")
+    sb = c.sb
+    y = torch.empty(c.N, c.plan.info.C_y, device="cuda:0")
+    buf = torch.empty(c.phi.numel() + 4, dtype=torch.float32, device="cuda:0")
+    phi1 = buf[1:1 + c.phi.numel()].view_as(c.phi)       # 4 bytes off
+    phi1.copy_(c.phi)
+    with pytest.raises(sb.SobekError) as ei:
+        sb.conv_fwd(c.plan, c.graph, c.x, c.Y, phi1, c.R, y, c.ws(0))
+    assert ei.value.code == -1
+
+
 # ---------------------------------------------------------------------------------------
 # benchmark-sized workloads, in the configuration bench.py times: sampled receivers
 # ---------------------------------------------------------------------------------------
@@ -236,12 +288,10 @@ def test_full_size_sampled(name):
 # the fused schedule (edge stream feeding the tensor core without leaving the SM)
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["cfg2_N200", "cfg4_N150", "cfg5_N60", "ragged", "K20"])
-def test_fused_schedule(name, monkeypatch):
-    """The plan-level schedule switch selects the fused stream+contraction kernels for y, gx, ggy
-    and hx; results must match the oracle to the same tolerances."""
-    monkeypatch.setenv("SOBEK_FUSED", "1")
-    c = Case(CASES[name])
-    monkeypatch.delenv("SOBEK_FUSED")
+def test_fused_schedule(name):
+    """The plan-level schedule switch (SOBEK_FLAG_FUSED_FP32) selects the fused stream+contraction kernels for
+    y, gx, ggy and hx; results must match the oracle to the same tolerances."""
+    c = Case(CASES[name], fused=True)
     assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
     for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
         assert rel_err(got, ref) <= BWD_TOL, nm
@@ -262,14 +312,10 @@ def test_fused_schedule(name, monkeypatch):
 # the FP32-pipe edge kernels (used where the tensor-core kernels do not apply), forced for whole plans
 # ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["cfg1", "cfg2_N200", "cfg4_N150", "ragged"])
-def test_fp32_pipe_edge_kernels(name, monkeypatch):
-    """SOBEK_TC_STREAM=0 / SOBEK_TC_EDGE=0 at plan creation select the FP32-pipe stream and edge pass for
-    every traversal; all three orders must match the oracle to the same tolerances."""
-    monkeypatch.setenv("SOBEK_TC_STREAM", "0")
-    monkeypatch.setenv("SOBEK_TC_EDGE", "0")
-    c = Case(CASES[name])
-    monkeypatch.delenv("SOBEK_TC_STREAM")
-    monkeypatch.delenv("SOBEK_TC_EDGE")
+def test_fp32_pipe_edge_kernels(name):
+    """SOBEK_FLAG_FP32_STREAM / SOBEK_FLAG_FP32_EDGE at plan creation select the FP32-pipe stream and edge pass
+    for every traversal; all three orders must match the oracle to the same tolerances."""
+    c = Case(CASES[name], tc_stream=False, tc_edge=False)
     assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
     for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
         assert rel_err(got, ref) <= BWD_TOL, nm
@@ -308,15 +354,13 @@ def test_scaling_axes_sampled(name):
         del FULL[name]
 
 
-def test_scratch_budget(monkeypatch):
+def test_scratch_budget():
     """The scratch budget (section "Runtime scratch-budget policy") only changes the chunking: with the
     paper's 128 MiB the workspace shrinks and every output still matches the oracle."""
     import paper_2607_18074_b200 as sb
     w = synth.scaled(synth.config("cfg4", edges=1e5), 1500)
     big = Case(w)
-    monkeypatch.setenv("SOBEK_STATE_BUDGET_MB", "128")
-    small = Case(w, inputs=big.d)
-    monkeypatch.delenv("SOBEK_STATE_BUDGET_MB")
+    small = Case(w, inputs=big.d, state_budget_mib=128)
     for order in (0, 1, 2):
         assert sb.workspace_bytes(small.plan, w.N, small.E, order) < sb.workspace_bytes(big.plan, w.N, big.E, order)
     rng = np.random.default_rng(5)
@@ -427,13 +471,11 @@ def test_uvu_double_backward_single_directions(ucases, dirs):
         assert rel_err(got, ref) <= BWD_TOL
 
 
-def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases, monkeypatch):
+def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases):
     c = uget(ucases, "uvu_16x3")
     for a, b in zip([c.fwd()] + c.bwd() + c.dbwd(), [c.fwd()] + c.bwd() + c.dbwd()):
         assert np.array_equal(a, b)
-    monkeypatch.setenv("SOBEK_TC_STREAM", "0")
-    monkeypatch.setenv("SOBEK_TC_EDGE", "0")
-    f = Case(UVU["uvu_16x3"], inputs=c.d)
+    f = Case(UVU["uvu_16x3"], inputs=c.d, tc_stream=False, tc_edge=False)
     assert rel_err(f.fwd(), c.o_fwd()) <= FWD_TOL
     for got, ref in zip(f.bwd(), c.o_bwd()):
         assert rel_err(got, ref) <= BWD_TOL
@@ -581,7 +623,7 @@ def test_random_profiles(seed):
 
 
 @pytest.mark.parametrize("name,mode", [("cfg2_N200", "uvw"), ("ragged", "uvw"), ("uvu_16x3", "uvu")])
-def test_state_retained_from_forward(name, mode, monkeypatch):
+def test_state_retained_from_forward(name, mode):
     """sobek_conv_fwd_retain leaves the receiver state in the workspace; sobek_conv_bwd_retained then computes gR
     from it without streaming the edges again: same bits as the plain calls, one stream launch fewer."""
     import torch
@@ -610,10 +652,8 @@ def test_state_retained_from_forward(name, mode, monkeypatch):
         assert np.array_equal(got.cpu().numpy(), ref)
     # a scratch budget that needs several chunks: nothing is retained, the results stay right
     if c.N >= 100:
-        monkeypatch.setenv("SOBEK_STATE_BUDGET_MB", "1")
         w2 = synth.scaled(synth.config("cfg2"), 1300)
-        c2 = Case(w2)
-        monkeypatch.delenv("SOBEK_STATE_BUDGET_MB")
+        c2 = Case(w2, state_budget_mib=1)
         y2 = new(c2.N, c2.plan.info.C_y)
         assert sb.conv_fwd_retain(c2.plan, c2.graph, c2.x, c2.Y, c2.phi, c2.R, y2, c2.ws(1)) == 0
         assert np.array_equal(y2.cpu().numpy(), c2.fwd())

@@ -51,7 +51,7 @@ def test_plan_paths_and_cg_match_oracle(name):
                 q.w_off) == (p.i_in, p.l_sh, p.i_out, p.l_in, p.l_out, p.c_in, p.c_out, p.in_off, p.sh_off,
                              p.out_off, p.w_off)
         assert np.abs(plan.cg(k) - p.cg).max() < 1e-9
-    assert np.allclose(plan.col_std(), tables.weight_col_std(w.irreps_in, w.irreps_out, w.l_max, w.K))
+    assert np.allclose(synth.plan_col_std(plan), tables.weight_col_std(w.irreps_in, w.irreps_out, w.l_max, w.K))
 
 
 def test_cg_all_triples_including_odd_sums():
@@ -140,7 +140,7 @@ def test_uvu_plan_errors_and_workspace():
     with pytest.raises(sb.SobekError):
         sb.Plan(P("8x0e+4x1o"), P("8x0e+4x1o"), 1, 4, mode="uvu")       # 0e x 1o -> 1o would tie 8 channels to 4
     with pytest.raises(sb.SobekError):
-        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=8)                    # unknown flag bit
+        sb.Plan(P("8x0e"), P("8x0e"), 0, 4, flags=1 << 10)              # unknown flag bit
     ir = P("64x0e+64x1o+64x2e")
     u, w = sb.Plan(ir, ir, 2, 16, mode="uvu"), sb.Plan(ir, ir, 2, 16)
     assert u.mode == "uvu" and w.mode == "uvw" and u.info.C_y == w.info.C_y
@@ -174,3 +174,27 @@ def test_binding_declares_every_signature():
         if name in no_args:
             continue
         assert getattr(L, name).argtypes is not None, name
+
+
+def test_graph_descriptor_keeps_its_tensors_alive():
+    """make_graph stores raw addresses in the C struct, so the returned object must hold the tensors."""
+    import torch
+    rp = torch.tensor([0, 1, 2], dtype=torch.int64)
+    col = torch.tensor([1, 0], dtype=torch.int32)
+    sp, perm, recv = rp.clone(), col.clone(), col.clone()
+    g = sb.make_graph(rp, col, sp, perm, recv)
+    assert g.N == 2 and g.E == 2
+    assert [id(t) for t in g.tensors] == [id(t) for t in (rp, col, sp, perm, recv)]
+    assert g.row_ptr == rp.data_ptr() and g.src_recv == recv.data_ptr()
+    g2 = sb.make_graph(rp, col)
+    assert g2.tensors[2] is None and not g2.src_ptr
+
+
+def test_plan_option_flags():
+    ir = [(8, 0, 1), (8, 1, -1)]
+    for kw in (dict(fused=True), dict(tc_stream=False), dict(tc_edge=False), dict(state_budget_mib=128)):
+        sb.Plan(ir, ir, 2, 8, **kw)
+    with pytest.raises(sb.SobekError):
+        sb.Plan(ir, ir, 2, 8, flags=1 << 11)            # an undefined flag bit
+    with pytest.raises(ValueError):
+        sb.Plan(ir, ir, 2, 8, state_budget_mib=0)

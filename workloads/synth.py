@@ -264,6 +264,25 @@ class Inputs:
     pos: np.ndarray = field(default=None, repr=False)
 
 
+def weight_col_std(paths, K: int, N_w: int, mode: str = "uvw") -> np.ndarray:
+    """1/sqrt(fan_in) per column of R, the scale of the synthetic weights: fan_in = K * (sum of the input
+    multiplicities over the paths into the column's output block; the number of those paths in the channelwise
+    mode).  `paths` is a sequence of records with fields i_out, c_in, c_out, w_off (the path table of a plan)."""
+    uvu = mode == "uvu"
+    fan = {}
+    for p in paths:
+        fan[p.i_out] = fan.get(p.i_out, 0) + (1 if uvu else p.c_in)
+    std = np.zeros(N_w)
+    for p in paths:
+        std[p.w_off:p.w_off + (p.c_in if uvu else p.c_in * p.c_out)] = (K * fan[p.i_out]) ** -0.5
+    return std
+
+
+def plan_col_std(plan) -> np.ndarray:
+    """weight_col_std for a library plan (anything with .info, .path(k) and .mode)."""
+    return weight_col_std([plan.path(k) for k in range(plan.info.n_paths)], plan.info.K, plan.info.N_w, plan.mode)
+
+
 def make_inputs(w: Workload, col_std: np.ndarray, dtype=np.float32,
                 with_cotangents: bool = True) -> Inputs:
     """Draw every input of one workload.
