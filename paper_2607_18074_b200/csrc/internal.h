@@ -111,6 +111,9 @@ struct TSet {
     int32_t unit_begin, nunit, blk_begin, nblk, ent_begin, nent;
     int32_t b_items;       // float4 pieces of sender rows gathered per 16-edge batch
     int32_t pad;
+    // stream: the set's slab list (TcSets::slabs, two words per slab), slabs per batch, first slab of each MMA thread
+    // (one byte each, 255: none) and the slots that a batch uses an odd number of times
+    int32_t sched_begin, nslab, mfirst, oddmask;
 };
 struct EntS {          // a (unit, component, s) entry of a set, as the kernels keep it in shared memory
     int32_t a_off, nz_begin, nz_count, pad;   // nz_begin is relative to the set's first term
@@ -139,6 +142,8 @@ struct TcSets {
     std::vector<EntS> ents_s;                // per set (TSet::ent_begin); TSet::b_items / TSet::pad = first term / terms
     std::vector<NzS> nz;
     std::vector<CompS> comps_s;              // parallel to comps
+    std::vector<uint32_t> slabs;             // stream: per set, two words per slab in build order (see stream_tc.cu)
+    uint32_t* d_slabs = nullptr;
     EntS* d_ents_s = nullptr;
     NzS* d_nz = nullptr;
     CompS* d_comps_s = nullptr;
@@ -147,13 +152,13 @@ struct TcSets {
     std::vector<NzS> inv;                    //   b -> terms (entry inside the set, coef)
     int32_t* d_inv_ptr = nullptr;
     NzS* d_inv = nullptr;
-    int32_t max_units = 0;
+    int32_t max_units = 0;                   // stream: slabs of a batch that one builder group builds, at most
     struct ESetPar { int32_t tb, lg, x_cap, z_cap, smem, ctas, tmem_cols, acc_cols, nnz, ninv, ncomp; };
     std::vector<ESetPar> epar;               // edge pass: launch parameters of every set (one launch per set)
-    int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets)
+    int32_t a_cap = 0, b_cap = 0;     // bytes of one A / B copy (max over sets; the stream keeps A in tensor memory)
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
-    int32_t concat = 0;               // stream: the lo copy of the gathered rows sits beside the hi copy (see stream_tc.cu)
+    int32_t ring_stages = 2;          // stream: stages of the shared-memory ring (as many as fit)
     int32_t smem_bytes = 0, ctas_per_sm = 1;
 };
 

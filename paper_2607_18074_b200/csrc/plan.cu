@@ -508,6 +508,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
             if (e == cudaSuccess) e = upload(t.ents_s, &t.d_ents_s);
             if (e == cudaSuccess) e = upload(t.nz, &t.d_nz);
             if (e == cudaSuccess) e = upload(t.comps_s, &t.d_comps_s);
+            if (e == cudaSuccess) e = upload(t.slabs, &t.d_slabs);
             if (e == cudaSuccess) e = upload(t.inv_ptr, &t.d_inv_ptr);
             if (e == cudaSuccess) e = upload(t.inv, &t.d_inv);
             if (e == cudaSuccess) e = upload(t.sets, &t.d_sets);
@@ -553,7 +554,7 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
         for (TcSets* tp : {&d->tc[0], &d->tc[1], &d->etc[0], &d->etc[1]}) {
             TcSets& t = *tp;
             cudaFree(t.d_inv_ptr); cudaFree(t.d_inv);
-            cudaFree(t.d_ents_s); cudaFree(t.d_nz); cudaFree(t.d_comps_s);
+            cudaFree(t.d_ents_s); cudaFree(t.d_nz); cudaFree(t.d_comps_s); cudaFree(t.d_slabs);
             cudaFree(t.d_sets); cudaFree(t.d_units); cudaFree(t.d_blks); cudaFree(t.d_ents); cudaFree(t.d_comps);
         }
     }

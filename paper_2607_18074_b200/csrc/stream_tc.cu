@@ -10,19 +10,31 @@
 // split-bf16 product a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo (fp32 accumulation in TMEM); the sender
 // rows are read from bf16 (hi, lo) copies of the source features made once per call.
 //
-// A CTA works through (set of accumulator tiles, receiver) items in set-major order, edges in batches of 16,
-// with three roles:
-//   loader warps  run ahead (segment bounds and edge / sender ids are requested one step early): cp.async of
-//                 the batch's phi rows, of its Y rows (written transposed) and of the sender rows straight
-//                 into the B slabs (16 edges x c_src, MN-major, 128-byte swizzle) of a two-stage ring; the
-//                 copies signal the stage's mbarrier themselves when they land;
-//   compute warps expand the coupling matrices M_e[s,comp] of the set from the sparse CG table (kept in shared
-//                 memory, like every other table the kernel looks up), build the A slabs (one per s: 128 rows
-//                 x 16 edges, K-major, no swizzle, bf16 hi / lo), and - one item behind - drain the finished
-//                 accumulator (tcgen05.ld), split it into bf16 hi / lo and write the rows of the node GEMM's
-//                 A operand (contraction index k = koff + q*c_src + u, so a row of 16-byte pieces per thread);
-//   MMA warp      one thread issues the batch's MMAs into one of two TMEM accumulator buffers and commits
-//                 to the mbarriers that release the A region, the ring stage and the accumulator.
+// The A operand never touches shared memory: the thread that owns accumulator row (comp,q) computes the 16
+// values of one slab (one s, 16 edges) in registers, splits them and stores them with tcgen05.st into a ring
+// of slab slots in tensor memory, from where tcgen05.mma reads them (A in TMEM, B from a shared-memory
+// descriptor).  Shared-memory bandwidth is then spent on the gathered rows only.
+//
+// One CTA per SM works through (pass, receiver) items in pass-major order (a pass = the accumulator tiles that
+// fit one of two TMEM accumulator buffers), edges in batches of 16, with four roles:
+//   loader warps   run ahead (segment bounds and edge / sender ids are requested one step early): cp.async of
+//                  the batch's phi rows, of its Y rows (written transposed) and of the sender rows straight
+//                  into the B slabs (16 edges x c_src, MN-major, 128-byte swizzle) of a ring of stages; the
+//                  copies signal the stage's mbarrier themselves when they land;
+//   builder warps  three groups of four (one warp per TMEM lane quarter).  Group g produces every third A slab of
+//                  the batch into its two TMEM slots (the slabs of a pass are listed tile after tile in turn, so
+//                  that the groups and the MMA threads are evenly loaded whatever the mix of source orders).  Per
+//                  batch it first expands the coupling values M_e[s,comp] of its own slabs from the sparse CG
+//                  table (kept in shared memory, like every other table the kernel looks up) into a buffer of
+//                  its own: one barrier among its 128 threads per batch, none with the other groups;
+//   MMA threads    three, in three warps (one thread gets a tcgen05.mma accepted every ~110 cycles whatever its
+//                  size, the pipe takes them three times as fast); thread t owns the accumulator tiles
+//                  unit = t mod 3 of the pass (a tile's products all come from one thread, in a fixed order), issues
+//                  the three products of a slab of theirs as soon as its slot is full, and commits to the
+//                  mbarriers that release the slot, the ring stage and the accumulator buffer;
+//   drain warps    read a finished accumulator (tcgen05.ld), split it into bf16 hi / lo and write the rows of
+//                  the node GEMM's A operand (contraction index k = koff + q*c_src + u, so a row of 16-byte
+//                  pieces per thread) while the next receiver's products run into the other buffer.
 // With DUAL the kernel produces the directional state of the double backward
 //     dZ = sum_e ( vphi (x) C(x,Y) + phi (x) [ C(vx,Y) + C(x,vY) ] )       (Eq. receiver_double_adjoint)
 // as  [vphi*M + phi*dM] x B(x)  +  [phi*M] x B(vx).
@@ -41,11 +53,20 @@ namespace {
 using namespace ptx;
 
 constexpr int TB = 16;          // edges per batch = k extent of one MMA
-constexpr int NCW = 8;          // compute warps
-constexpr int NLW = 2;          // loader warps
-constexpr int TT = (NCW + NLW + 1) * 32;   // threads per CTA
-constexpr int NS = 2;           // ring stages
+constexpr int NBG = 3;          // builder groups (four warps each: one per TMEM lane quarter)
+constexpr int NBW = 4 * NBG;    // builder warps
+constexpr int NDW = 4;          // drain warps
+constexpr int NLW = 4;          // loader warps
+constexpr int NMW = 3;          // MMA warps (one issuing thread each; a unit's products all come from one of them)
+constexpr int W_DRAIN = NBW, W_LOAD = NBW + NDW, W_MMA = NBW + NDW + NLW;
+constexpr int TT = (W_MMA + NMW + 1) * 32;   // threads per CTA (a multiple of 128; the last warp has no role)
+constexpr int MAXNS = 4;        // ring stages: 2..4, as many as shared memory holds
+constexpr int NSLOT = 2 * NBG;  // A slab slots in tensor memory, two per builder group: 16 columns each (8 hi + 8 lo)
+constexpr int TMEM_COLS = 512;
+constexpr int RING0 = TMEM_COLS - NSLOT * 16;      // first column of the slot ring
+constexpr int ACC_BUDGET = RING0 / 2;              // columns of one accumulator buffer (two buffers)
 constexpr int PS = 20;          // row pitch (floats) of the transposed stages: 16 values + 4 (bank spread)
+static_assert(NSLOT % NBG == 0, "slab j of a batch goes to slot j mod NSLOT, built by group j mod NBG");
 
 struct TcArgs {
     const TSet* sets;
@@ -67,8 +88,9 @@ struct TcArgs {
     __nv_bfloat16* zh;
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
-    int32_t a_cap, b_cap, max_ent, tmem_cols, acc_cols, n_units, n_blks, n_comps, max_nz;
-    int32_t concat;        // 1: multiplicities <= 32, the lo copy of a gathered row sits 32 columns beside the hi copy
+    int32_t b_cap, max_ent, acc_cols, n_units, n_blks, n_comps, max_nz, ns, n_slab;
+    int32_t max_own;        // slabs of a batch that one builder group builds, at most
+    const uint32_t* slabs;  // per set (TSet::sched_begin, nslab): two words per slab, in build order (see SlabW)
     int* status;
 };
 
@@ -81,27 +103,41 @@ __device__ __forceinline__ int64_t owner_of(const int64_t* __restrict__ row_ptr,
     return lo;
 }
 
-// Everything the roles look up per item, batch or row lives in shared memory: with most of the SM's
+// Everything the roles look up per item, batch or slab lives in shared memory: with most of the SM's
 // L1 given to the operand regions, table reads from global memory would mostly go to L2.
-struct UInfo {     // a unit, as the MMA thread and the drain need it
-    uint32_t idesc, tmem_col, a_off, slab_stride, b_off, slab_bytes, d_src, comp_begin, ncomp, c_src, ncols, pad;
-    // operand descriptors of slab 0 (hi copies; stage 0 of the ring for B): the other slabs, copies and stages differ
-    // only in the 16-byte-granular address field, so the MMA thread reaches them with one addition each
-    uint64_t dA0, dB0;
-    uint32_t idesc_wide, pad2;   // concat: the same instruction with N = 64 columns ([B_hi | B_lo])
+struct UInfo {     // a unit, as the MMA thread, the builders and the drain need it
+    uint32_t idesc, tmem_col, d_src, comp_begin, ncomp, c_src, ncols, ent0;
+    uint64_t dB0;    // operand descriptor of the unit's B slab 0 (hi copy, stage 0 of the ring): the other slabs,
+    uint64_t sb16;   // copies and stages differ only in the 16-byte-granular address field (sb16 per slab)
 };
-// shared-memory operand descriptor without swizzle (K-major core matrices of 8 rows x 16 bytes)
-__device__ __forceinline__ uint64_t make_desc_none(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;   // version
-    return d;
-}
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
+// hand-over by a count in shared memory that only grows: the producer adds with release semantics, the consumer
+// polls with acquire semantics until the count reaches its target (bounded like every other wait of the kernel)
+__device__ __forceinline__ void count_add(uint32_t addr) {
+    asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ void count_wait(uint32_t addr, uint32_t target, int* status) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t v;
+        asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+        if ((int32_t)(v - target) >= 0) return;
+        if ((it & 255u) == 0) {
+            uint64_t t1;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            if (it == 0) t0 = t1;
+            else if (t1 - t0 > 2000000000ull) break;
+        }
+    }
+    atomicExch(status, (int)SOBEK_ERR_DEVICE_TIMEOUT);
+}
+__device__ __forceinline__ void group_sync(int grp) { asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory"); }
+__device__ __forceinline__ void builder_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NBW * 32) : "memory"); }
+// A slab of a pass in build order, as two words.
+//   bw: (first entry of the tile + s) | d_src << 16 | ncomp << 24         what the builders need
+//   mw: tile in the pass | s << 8 | next slab of the same MMA thread << 16 (255: none)
+struct SlabW { uint32_t bw, mw; };
 
 // cp.async with zero fill: copies `bytes` (0 or the full size) and fills the rest with zeros
 __device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t bytes) {
@@ -109,19 +145,6 @@ __device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, 
 }
 __device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void* src, uint32_t bytes) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // (hi, lo) bf16 split of two floats: hi pair, lo pair (element 0 in the low half)
@@ -147,33 +170,39 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh) {
 }
 
 template <int KP, bool DUAL>
-__global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
+__global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int NOP = 1;                 // operand pairs held at once (the dual stream runs its two pairs in turn)
     constexpr int NRAW = DUAL ? 2 : 1;     // raw / transposed stages: phi and Y, plus their directions
-    const int YS = a.dsh + 1;
-    // A region (single buffer): A1h A1l (A2h A2l)
-    uint8_t* sA = smem;
-    // ring stages: B1h B1l (B2h B2l), then the raw phi / Y rows
-    const uint32_t stage_bytes = (uint32_t)(2 * NOP * a.b_cap + ((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023));
-    uint8_t* sRing = sA + (size_t)2 * NOP * a.a_cap;
+    const int NS = a.ns;
+    // ring stages: Bh Bl, then the raw phi / Y rows
+    const uint32_t stage_bytes = (uint32_t)(2 * a.b_cap + ((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023));
+    uint8_t* sRing = smem;
     uint8_t* meta = sRing + (size_t)NS * stage_bytes;
-    float* sM0 = reinterpret_cast<float*>(meta);             // [2][max_ent][PS]: coupling matrices, double buffered
-    float* sdM0 = sM0 + (size_t)2 * a.max_ent * PS;          // DUAL
-    float* sPhiT0 = sdM0 + (DUAL ? (size_t)2 * a.max_ent * PS : 0);   // [2][NRAW][KP][PS]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sPhiT0 + 2 * NRAW * KP * PS);
-    // bars: full[NS], freeS[NS], ready, afree, acc_full[2], acc_free[2]
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
-    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [n_units]
+    // coupling values of a group's own slabs of one batch, double buffered: [NBG][2][max_own][MC][PS] (+ directions)
+    constexpr int MC = 128 / KP;                              // components of a tile at most
+    const size_t mbuf_floats = (size_t)a.max_own * MC * PS;
+    float* sM0 = reinterpret_cast<float*>(meta);
+    float* sdM0 = sM0 + (size_t)NBG * 2 * mbuf_floats;        // DUAL
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sdM0 + (DUAL ? (size_t)NBG * 2 * mbuf_floats : 0));
+    // bars: full[MAXNS], sfree[MAXNS], slot_free[NSLOT], acc_full[2], acc_free[2]
+    constexpr int NBAR = 2 * MAXNS + NSLOT + 4;
+    // slot_fill[s]: warps that have finished storing into slot s, counted over the whole kernel (4 per use).  A slot is
+    // consumed by whichever MMA thread owns the slab's tile, so its hand-over is a count that only grows (an mbarrier's
+    // parity could be misread by a thread that is two uses ahead of another).
+    uint32_t* slot_fill = reinterpret_cast<uint32_t*>(bars + NBAR);
+    uint32_t* tmem_holder = slot_fill + NSLOT + (NSLOT & 1);
+    UInfo* sU = reinterpret_cast<UInfo*>(tmem_holder + 2);             // [n_units]
     TSet* sSet = reinterpret_cast<TSet*>(sU + a.n_units);               // [nsets]
     TBlk* sBlk = reinterpret_cast<TBlk*>(sSet + a.nsets);               // [n_blks]
     CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.n_blks);           // [n_comps]
     EntS* sEnt = reinterpret_cast<EntS*>(sComp + a.n_comps);            // [max_ent]  (current set)
     NzS* sNz = reinterpret_cast<NzS*>(sEnt + a.max_ent);                // [max_nz]   (current set)
+    SlabW* sSlab = reinterpret_cast<SlabW*>(sNz + a.max_nz);            // [n_slab]
     const uint32_t bar0 = smem_u32(bars);
-    const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_ready = bar0 + 16 * NS, bar_afree = bar_ready + 8,
-                   bar_accfull = bar_ready + 16, bar_accfree = bar_ready + 32;
+    const uint32_t bar_full = bar0, bar_sfree = bar0 + 8 * MAXNS, bar_slotfree = bar0 + 16 * MAXNS,
+                   bar_accfull = bar_slotfree + 8 * NSLOT, bar_accfree = bar_accfull + 16;
+    const uint32_t fill0 = smem_u32(slot_fill);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool has_vx = DUAL && a.vsh != nullptr, has_vY = DUAL && a.vY != nullptr, has_vphi = DUAL && a.vphi != nullptr;
@@ -184,15 +213,16 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
     const int nsub = (has_a1 ? 1 : 0) + (has_a2 ? 1 : 0);
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 1); }
-        mbar_init(bar_ready, NCW * 32);
-        mbar_init(bar_afree, 1);
-        for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW * 32); }
+        for (int s = 0; s < MAXNS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_sfree + 8 * s, NMW); }
+        for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_slotfree + 8 * s, 1); slot_fill[s] = 0u; }
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, NMW); mbar_init(bar_accfree + 8 * t, NDW); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // every slot starts out free: its first phase completes here, so that the builders wait on it like on any other
+        for (int s = 0; s < NSLOT; ++s) mbar_arrive(bar_slotfree + 8 * s);
     }
     // the raw rows of padded radial components (q >= K) and of absent directions stay zero for ever
     {
-        const int words = (int)(stage_bytes / 4), b_words = 2 * NOP * a.b_cap / 4;
+        const int words = (int)(stage_bytes / 4), b_words = 2 * a.b_cap / 4;
         for (int i = tid; i < NS * words; i += TT) {
             const int st = i / words, w = i - st * words;
             if (w >= b_words) reinterpret_cast<uint32_t*>(sRing + (size_t)st * stage_bytes)[w] = 0u;
@@ -202,24 +232,22 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         const TUnit U = a.units[i];
         const TBlk B = a.blks[U.blk];
         UInfo u;
-        // D = F32, A = B = BF16, A K-major, B MN-major, M = 128, N = ncols
+        // D = F32, A = B = BF16, A K-major (tensor memory), B MN-major, M = 128, N = ncols
         u.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(B.ncols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        u.tmem_col = (uint32_t)U.tmem_col; u.a_off = (uint32_t)U.a_off; u.slab_stride = (uint32_t)U.slab_stride;
-        u.b_off = (uint32_t)B.b_off; u.slab_bytes = (uint32_t)B.slab_bytes; u.d_src = (uint32_t)B.d_src;
+        u.tmem_col = (uint32_t)U.tmem_col; u.d_src = (uint32_t)B.d_src;
         u.comp_begin = (uint32_t)U.comp_begin; u.ncomp = (uint32_t)U.ncomp; u.c_src = (uint32_t)B.c_src;
-        u.ncols = (uint32_t)B.ncols; u.pad = 0;
-        u.idesc_wide = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        u.pad2 = 0;
-        u.dA0 = make_desc_none(smem_u32(sA) + u.a_off, 128, 256);
-        u.dB0 = make_desc(smem_u32(sRing) + u.b_off, 2048, 1024);
+        u.ncols = (uint32_t)B.ncols; u.ent0 = (uint32_t)U.a_off;
+        u.dB0 = make_desc(smem_u32(sRing) + (uint32_t)B.b_off, 2048, 1024);
+        u.sb16 = (uint64_t)(B.slab_bytes >> 4);
         sU[i] = u;
     }
     for (int i = tid; i < a.nsets; i += TT) sSet[i] = a.sets[i];
     for (int i = tid; i < a.n_blks; i += TT) sBlk[i] = a.blks[i];
     for (int i = tid; i < a.n_comps; i += TT) sComp[i] = a.comps[i];
+    for (int i = tid; i < 2 * a.n_slab; i += TT) reinterpret_cast<uint32_t*>(sSlab)[i] = a.slabs[i];
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)a.tmem_cols) : "memory");
+                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -234,12 +262,12 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         __device__ void step(int64_t by, int64_t n) { nl += by; while (nl >= n) { nl -= n; ++set; } }
     };
 
-    if (warp >= NCW && warp < NCW + NLW) {
+    if (warp >= W_LOAD && warp < W_LOAD + NLW) {
         // =========================== loader warps ===========================
         // The segment bounds of the next item and the ids of the next batch are requested one step ahead,
         // so that their latency overlaps the issue of the current batch's copies; the copies themselves
         // signal the stage's mbarrier when they land (no wait in this warp).
-        const int lt = (warp - NCW) * 32 + lane;   // thread index among the loaders
+        const int lt = (warp - W_LOAD) * 32 + lane;   // thread index among the loaders
         int64_t p_item = blockIdx.x, p_seg0 = 0, p_seg1 = 0;     // prefetched item
         ItemPos lp; lp.init(p_item, a.n_nodes);
         auto prefetch_item = [&]() {
@@ -288,17 +316,17 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
         bool have = next_batch(cur, true);
         int64_t eid = 0; int32_t sn = 0; uint32_t msk = 0;
         if (have) load_ids(cur, eid, sn, msk);
-        for (uint32_t it = 0; have; ++it) {
+        int st = 0; uint32_t round = 0;      // stage of the batch and how often the ring has wrapped
+        for (; have;) {
             Cur nxt = cur;
             const bool have_n = next_batch(nxt, false);
             int64_t eid_n = 0; int32_t sn_n = 0; uint32_t msk_n = 0;
             if (have_n) load_ids(nxt, eid_n, sn_n, msk_n);
             const TSet S = sSet[cur.set];
             const int op = has_a1 ? cur.sub : 1;
-            const int st = (int)(it % NS);
-            if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
+            if (round > 0) mbar_wait(bar_sfree + 8 * st, (round & 1) ^ 1, a.status);
             const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
-            const uint32_t raw_u = stage_u + (uint32_t)(2 * NOP * a.b_cap);
+            const uint32_t raw_u = stage_u + (uint32_t)(2 * a.b_cap);
             // phi (and vphi) rows: raw[e][KP]   (all lanes run every iteration: the loops hold shuffles)
             {
                 const bool v16 = (a.K & 3) == 0;
@@ -320,7 +348,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                     }
                 }
             }
-            // Y (and vY), transposed: raw[b][PS + e].  Thread <-> (edge e = lane mod 16, b = lt / 16, + 4, ...)
+            // Y (and vY), transposed: raw[b][PS + e].  Thread <-> (edge e = lane mod 16, b = lt / 16, + 8, ...)
             const int le = lane & (TB - 1);
             const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
             {
@@ -335,7 +363,7 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             }
             // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy
             {
-                // lanes 2e, 2e+1 of each loader warp serve edge e; a thread walks pieces j0, j0 + 4, ... of the row
+                // lanes 2e, 2e+1 of each loader warp serve edge e; a thread walks pieces j0, j0 + 2 NLW, ... of the row
                 const int re = (lane >> 1) & (TB - 1);
                 const int32_t sne = __shfl_sync(0xffffffffu, sn, re);
                 const uint32_t ok = ((msk >> re) & 1u) * 16u;
@@ -351,13 +379,10 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                         uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + re * 128 + ((((u & 63) >> 3) ^ (re & 7)) << 4));
                         const __nv_bfloat16* ph = srch + B.src_off + u;
                         const __nv_bfloat16* pl = srcl + B.src_off + u;
-                        // the lo copy: a slab of its own, or (concat) columns 32.. of the same swizzled row
-                        uint32_t dl = a.concat ? stage_u + (uint32_t)(B.b_off + re * 128 + ((((u >> 3) + 4) ^ (re & 7)) << 4))
-                                               : d + (uint32_t)a.b_cap;
                         for (int sdx = 0; sdx < B.d_src; ++sdx) {
                             cp_async16_zfill(d, ph, ok);
-                            cp_async16_zfill(dl, pl, ok);
-                            d += (uint32_t)B.slab_bytes; dl += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                            cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
+                            d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
                         }
                     }
                 }
@@ -365,15 +390,21 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             // this thread's arrival on the stage's barrier fires when all its copies above have landed
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_full + 8 * st) : "memory");
             cur = nxt; have = have_n; eid = eid_n; sn = sn_n; msk = msk_n;
+            if (++st == NS) { st = 0; ++round; }
         }
-    } else if (warp == NCW + NLW) {
-        // =========================== MMA warp ===========================
+    } else if (warp >= W_MMA && warp < W_MMA + NMW) {
+        // =========================== MMA warps ===========================
         if (lane == 0) {
-            uint32_t it = 0, mi = 0;
+            const uint32_t me = (uint32_t)(warp - W_MMA);
+            uint32_t mi = 0;
+            uint32_t uses[NSLOT];            // how often every slot has been used before the current batch
+#pragma unroll
+            for (int s = 0; s < NSLOT; ++s) uses[s] = 0u;
+            int st = 0; uint32_t round = 0;
             int64_t nx0 = 0, nx1 = 0;
             ItemPos mp; mp.init(blockIdx.x, a.n_nodes);      // position of the item whose bounds are in flight
             if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
-            const uint64_t acap16 = (uint64_t)(a.a_cap >> 4), bcap16 = (uint64_t)(a.b_cap >> 4);
+            const uint64_t bcap16 = (uint64_t)(a.b_cap >> 4);
             for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
                 const TSet S = sSet[mp.set];
                 const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
@@ -384,139 +415,123 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                 const uint32_t buf = mi & 1;
                 if (mi >= 2) mbar_wait(bar_accfree + 8 * buf, ((mi >> 1) & 1) ^ 1, a.status);
                 tc_fence_after();
+                const SlabW* slabs = sSlab + S.sched_begin;
+                const uint32_t j0 = ((uint32_t)S.mfirst >> (8 * me)) & 255u;     // first slab of this thread (255: none)
                 for (int64_t b0 = seg0; b0 < seg1; b0 += TB) {
-                    for (int sb = 0; sb < nsub; ++sb, ++it) {
-                        const int st = (int)(it % NS);
-                        mbar_wait(bar_ready, it & 1, a.status);
-                        tc_fence_after();
+                    for (int sb = 0; sb < nsub; ++sb) {
+                        mbar_wait(bar_full + 8 * st, round & 1, a.status);
+                        fence_async_smem();      // the gathered rows were written through the generic proxy
                         const uint64_t st16 = (uint64_t)((uint32_t)st * (stage_bytes >> 4));
-                        const uint32_t acc0 = (b0 == seg0 && sb == 0) ? 0u : 1u;
-                        for (int ui = 0; ui < S.nunit; ++ui) {
+                        const bool first = b0 == seg0 && sb == 0;
+                        for (uint32_t j = j0; j != 255u;) {
+                            const uint32_t mw = slabs[j].mw, ui = mw & 255u, sl = (mw >> 8) & 255u;
                             const UInfo& U = sU[S.unit_begin + ui];
                             const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + U.tmem_col;
-                            const uint32_t idesc = U.idesc, nslab = U.d_src;
-                            const uint64_t sa16 = U.slab_stride >> 4, sb16 = U.slab_bytes >> 4;
-                            uint64_t dAh = U.dA0, dBh = U.dB0 + st16;
-                            if (a.concat) {
-                                // two instructions per slab instead of three: A_hi x [B_hi | B_lo] (64 columns; the second
-                                // 32 are summed into the first at the drain) and A_lo x B_hi.  An MMA of up to 64 columns
-                                // costs the same fixed time, so this takes a third off the tensor-pipe time.
-                                const uint32_t iw = U.idesc_wide;
-                                tc_mma_bf16(d_tmem, dAh, dBh, iw, acc0);
-                                tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
-                                for (uint32_t s = 1; s < nslab; ++s) {
-                                    dAh += sa16; dBh += sb16;
-                                    tc_mma_bf16(d_tmem, dAh, dBh, iw, 1u);
-                                    tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
-                                }
-                                continue;
-                            }
-                            tc_mma_bf16(d_tmem, dAh, dBh, idesc, acc0);
-                            tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
-                            tc_mma_bf16(d_tmem, dAh, dBh + bcap16, idesc, 1u);
-                            for (uint32_t s = 1; s < nslab; ++s) {
-                                dAh += sa16; dBh += sb16;
-                                tc_mma_bf16(d_tmem, dAh, dBh, idesc, 1u);
-                                tc_mma_bf16(d_tmem, dAh + acap16, dBh, idesc, 1u);
-                                tc_mma_bf16(d_tmem, dAh, dBh + bcap16, idesc, 1u);
-                            }
+                            const uint64_t dBh = U.dB0 + st16 + sl * U.sb16;
+                            const uint32_t idesc = U.idesc;
+                            const uint32_t slot = j % NSLOT, use = j / NSLOT;
+                            uint32_t before = 0;
+#pragma unroll
+                            for (int s = 0; s < NSLOT; ++s) before = slot == (uint32_t)s ? uses[s] : before;
+                            count_wait(fill0 + 4 * slot, 4u * (before + use + 1u), a.status);
+                            tc_fence_after();
+                            const uint32_t a_h = tmem_base + (uint32_t)RING0 + slot * 16u, a_l = a_h + 8u;
+                            tc_mma_bf16_ts(d_tmem, a_h, dBh, idesc, (first && sl == 0) ? 0u : 1u);
+                            tc_mma_bf16_ts(d_tmem, a_l, dBh, idesc, 1u);
+                            tc_mma_bf16_ts(d_tmem, a_h, dBh + bcap16, idesc, 1u);
+                            tc_commit(bar_slotfree + 8 * slot);
+                            j = (mw >> 16) & 255u;
                         }
-                        tc_commit(bar_afree);
-                        tc_commit(bar_free + 8 * st);
+#pragma unroll
+                        for (int s = 0; s < NSLOT; ++s) uses[s] += (uint32_t)(S.nslab + NSLOT - 1 - s) / NSLOT;
+                        // (a commit with nothing outstanding arrives at once: every MMA thread takes part)
+                        tc_commit(bar_sfree + 8 * st);
                         if (b0 + TB >= seg1 && sb == nsub - 1) tc_commit(bar_accfull + 8 * buf);
+                        if (++st == NS) { st = 0; ++round; }
                     }
                 }
                 ++mi;
             }
         }
-    } else {
-        // =========================== compute warps ===========================
-        uint32_t it = 0, mi = 0;
-        int cur_set = -1;
-        int64_t cx0 = 0, cx1 = 0;
-        ItemPos cp_; cp_.init(blockIdx.x, a.n_nodes);        // position of the item whose bounds are in flight
-        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
-        // the item whose accumulator is drained next (one behind the one being built)
-        int64_t p_nl = -1; int p_set = 0; uint32_t p_mi = 0; bool p_wrote = false;
-
-        auto drain = [&](int64_t nl, int set, uint32_t dmi, bool wrote) {
-            const TSet S = sSet[set];
-            const uint32_t buf = dmi & 1;
+    } else if (warp >= W_DRAIN && warp < W_DRAIN + NDW) {
+        // =========================== drain warps ===========================
+        // one thread per accumulator row (TMEM lane); a warp reaches the 32 lanes of its quarter only
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;
+        const int cl = r / KP, q = r - cl * KP;
+        uint32_t mi = 0;
+        int64_t dx0 = 0, dx1 = 0;
+        ItemPos dp; dp.init(blockIdx.x, a.n_nodes);
+        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + dp.nl, a.ev.E, nullptr, dx0, dx1);
+        for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
+            const int64_t nl = dp.nl;
+            const TSet S = sSet[dp.set];
+            const int64_t seg0 = dx0, seg1 = any_op ? dx1 : dx0;
+            dp.step(gridDim.x, a.n_nodes);
+            if (item + gridDim.x < total) seg_bounds(a.ev.ptr, a.node0 + dp.nl, a.ev.E, nullptr, dx0, dx1);
+            const bool wrote = seg1 > seg0;      // a node without edges has a state of zeros
+            const uint32_t buf = mi & 1;
             if (wrote) {
-                mbar_wait(bar_accfull + 8 * buf, (dmi >> 1) & 1, a.status);
+                mbar_wait(bar_accfull + 8 * buf, (mi >> 1) & 1, a.status);
                 tc_fence_after();
             }
-            const int quarter = warp & 3, half = warp >> 2;
             for (int ui = 0; ui < S.nunit; ++ui) {
-                const UInfo U = sU[S.unit_begin + ui];
-                struct { int ncols, c_src; } B{(int)U.ncols, (int)U.c_src};
-                const int r = quarter * 32 + lane;
-                const int cl = r / KP, q = r - cl * KP;
+                const UInfo& U = sU[S.unit_begin + ui];
+                const int c_src = (int)U.c_src, ncols = (int)U.ncols;
                 const bool rv = cl < (int)U.ncomp && q < a.K;
                 int64_t off = 0;
                 if (rv) {
                     const CompS cp = sComp[U.comp_begin + cl];
-                    off = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff + (int64_t)q * B.c_src;
+                    off = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff + (int64_t)q * c_src;
                 }
-                const int hc = B.ncols >> 1;       // columns per warp half (multiple of 8)
                 const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols + U.tmem_col;
-                if ((hc & 15) == 0) {              // 16 columns per TMEM load: half as many load round trips
-                    for (int cc = half * hc; cc < (half + 1) * hc; cc += 16) {
-                        float v[16];
-                        if (wrote) {
-                            tc_ld16(trow + (uint32_t)cc, v);
-                            if (a.concat) {     // + A_hi x B_lo, accumulated 32 columns further on
-                                float w[16];
-                                tc_ld16(trow + 32u + (uint32_t)cc, w);
+#pragma unroll 1
+                for (int cc = 0; cc < ncols; cc += 16) {       // ncols is a multiple of 16, c_src of 8
+                    float v[16];
+                    if (wrote) {
+                        tc_ld16(trow + (uint32_t)cc, v);
+                    } else {
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] += w[i];
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                        }
-#pragma unroll
-                        for (int g8 = 0; g8 < 16; g8 += 8) {
-                            if (rv && cc + g8 < B.c_src) {
-                                uint4 h, l;
-                                split8(v + g8, h, l);
-                                *reinterpret_cast<uint4*>(a.zh + off + cc + g8) = h;
-                                *reinterpret_cast<uint4*>(a.zl + off + cc + g8) = l;
-                            }
-                        }
+                        for (int i = 0; i < 16; ++i) v[i] = 0.f;
                     }
-                } else {
-                    for (int cc = half * hc; cc < (half + 1) * hc; cc += 8) {
-                        float v[8];
-                        if (wrote) {
-                            tc_ld8(trow + (uint32_t)cc, v);
-                            if (a.concat) {
-                                float w[8];
-                                tc_ld8(trow + 32u + (uint32_t)cc, w);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) v[i] += w[i];
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) v[i] = 0.f;
-                        }
-                        if (rv && cc < B.c_src) {
-                            uint4 h, l;
-                            split8(v, h, l);
-                            *reinterpret_cast<uint4*>(a.zh + off + cc) = h;
-                            *reinterpret_cast<uint4*>(a.zl + off + cc) = l;
+                    if (rv && cc < c_src) {
+                        __nv_bfloat16* ph_ = a.zh + off + cc;
+                        __nv_bfloat16* pl_ = a.zl + off + cc;
+                        uint4 h, l;
+                        split8(v, h, l);
+                        *reinterpret_cast<uint4*>(ph_) = h;
+                        *reinterpret_cast<uint4*>(pl_) = l;
+                        if (cc + 8 < c_src) {
+                            split8(v + 8, h, l);
+                            *reinterpret_cast<uint4*>(ph_ + 8) = h;
+                            *reinterpret_cast<uint4*>(pl_ + 8) = l;
                         }
                     }
                 }
             }
             if (wrote) {
                 tc_fence_before();
-                mbar_arrive(bar_accfree + 8 * buf);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_accfree + 8 * buf);
+                ++mi;
             }
-        };
-
+        }
+    } else if (warp < NBW) {
+        // =========================== builder warps ===========================
+        // group grp = warp / 4 builds the slabs j = grp, grp + NBG, ... of every batch; its four warps cover the 128 rows
+        const int grp = warp >> 2, quarter = warp & 3;
+        const int r = quarter * 32 + lane;                    // this thread's accumulator row = TMEM lane
+        const int cl = r / KP, q = r - cl * KP;
+        const uint32_t ring_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)RING0;
+        const int gt = tid & 127;                             // thread index inside the group
+        uint32_t it = 0;
+        uint32_t par = 0;                // bit s: how often slot s has been used so far, modulo 2
+        int st = 0; uint32_t round = 0;
+        int cur_set = -1;
+        int64_t cx0 = 0, cx1 = 0;
+        ItemPos cp_; cp_.init(blockIdx.x, a.n_nodes);        // position of the item whose bounds are in flight
+        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
         for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-            const int64_t nl = cp_.nl;
             const int set = cp_.set;
             const TSet S = sSet[set];
             const int64_t seg0 = cx0, seg1 = any_op ? cx1 : cx0;
@@ -524,39 +539,35 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
             if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
                 seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
             if (set != cur_set && seg1 > seg0) {     // entry and sparse-term tables of the set
-                compute_sync();
-                for (int i = tid; i < S.nent; i += NCW * 32) sEnt[i] = a.ents[S.ent_begin + i];
-                for (int i = tid; i < S.pad; i += NCW * 32) sNz[i] = a.nz[S.b_items + i];
-                compute_sync();
+                builder_sync();
+                for (int i = tid; i < S.nent; i += NBW * 32) sEnt[i] = a.ents[S.ent_begin + i];
+                for (int i = tid; i < S.pad; i += NBW * 32) sNz[i] = a.nz[S.b_items + i];
+                builder_sync();
                 cur_set = set;
             }
+            const SlabW* slabs = sSlab + S.sched_begin;
             for (int64_t b0 = seg0; b0 < seg1; b0 += TB)
             for (int sb = 0; sb < nsub; ++sb, ++it) {
                 const int op = has_a1 ? sb : 1;          // which operand pair this sub-batch builds
-                const int st = (int)(it % NS);
-                mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
-                const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * NOP * a.b_cap);
+                mbar_wait(bar_full + 8 * st, round & 1, a.status);
+                const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.b_cap);
                 const float* sYT = raw + NRAW * TB * KP;
                 const float* sVYT = sYT + a.dsh * PS;
-                float* sM = sM0 + (size_t)(it & 1) * a.max_ent * PS;
-                float* sdM = sdM0 + (size_t)(it & 1) * a.max_ent * PS;
-                float* sPhiT = sPhiT0 + (size_t)(it & 1) * NRAW * KP * PS;     // [KP][PS] (+ vphi)
-                float* sVphiT = sPhiT + KP * PS;
-                // ---- transpose phi: [e][q] -> [q][e]   (same double buffer and barrier as the coupling matrices)
-                for (int i = tid; i < TB * KP; i += NCW * 32) {
-                    const int e = i / KP, q = i - e * KP;
-                    sPhiT[q * PS + e] = raw[i];
-                    if (DUAL) sVphiT[q * PS + e] = raw[TB * KP + i];
-                }
-                // ---- coupling matrices of the set: thread <-> (entry, 8 edges)
-                for (int i = tid; i < 2 * S.nent; i += NCW * 32) {
-                    const int j = i >> 1, h = i & 1;
-                    const EntS en = sEnt[j];
+                float* sM = sM0 + ((size_t)grp * 2 + (it & 1)) * mbuf_floats;
+                float* sdM = sdM0 + ((size_t)grp * 2 + (it & 1)) * mbuf_floats;
+                // ---- coupling values of this group's own slabs: thread <-> (own slab k, component c, 8 edges)
+                const int nown = (S.nslab - grp + NBG - 1) / NBG;
+#pragma unroll 1
+                for (int i = gt; i < nown * 2 * MC; i += 128) {
+                    const int k = i / (2 * MC), c = (i >> 1) & (MC - 1), h = i & 1;
+                    const uint32_t bw = slabs[grp + k * NBG].bw;
+                    if (c >= (int)(bw >> 24)) continue;
+                    const EntS en = sEnt[(int)(bw & 0xffffu) + c * (int)((bw >> 16) & 255u)];
                     float m[8], dm[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) { m[e] = 0.f; dm[e] = 0.f; }
-                    for (int k = en.nz_begin; k < en.nz_begin + en.nz_count; ++k) {
-                        const NzS t = sNz[k];
+                    for (int kk = en.nz_begin; kk < en.nz_begin + en.nz_count; ++kk) {
+                        const NzS t = sNz[kk];
                         const float cf = t.coef;
                         const int b = t.b;
                         float y[8];
@@ -571,88 +582,102 @@ __global__ void __launch_bounds__(TT, 2) k_stream_tc(const TcArgs a) {
                             for (int e = 0; e < 8; ++e) dm[e] = fmaf(cf, y[e], dm[e]);
                         }
                     }
-                    *reinterpret_cast<float4*>(sM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(m);
-                    *reinterpret_cast<float4*>(sM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(m + 4);
+                    float* d = sM + (size_t)(k * MC + c) * PS + 8 * h;
+                    *reinterpret_cast<float4*>(d) = *reinterpret_cast<const float4*>(m);
+                    *reinterpret_cast<float4*>(d + 4) = *reinterpret_cast<const float4*>(m + 4);
                     if (DUAL) {
-                        *reinterpret_cast<float4*>(sdM + j * PS + 8 * h) = *reinterpret_cast<const float4*>(dm);
-                        *reinterpret_cast<float4*>(sdM + j * PS + 8 * h + 4) = *reinterpret_cast<const float4*>(dm + 4);
+                        float* dd = sdM + (size_t)(k * MC + c) * PS + 8 * h;
+                        *reinterpret_cast<float4*>(dd) = *reinterpret_cast<const float4*>(dm);
+                        *reinterpret_cast<float4*>(dd + 4) = *reinterpret_cast<const float4*>(dm + 4);
                     }
                 }
-                compute_sync();
-                // the previous batch's MMAs must have read the A region before it is rewritten
-                if (it > 0) mbar_wait(bar_afree, (it - 1) & 1, a.status);
-                // ---- A slabs: thread <-> (entry, q), both 8-edge halves
-                for (int i = tid; i < S.nent * KP; i += NCW * 32) {
-                    const int j = i / KP, q = i - j * KP;
-                    const int a_off = sEnt[j].a_off + (q >> 3) * 256 + (q & 7) * 16;
+                group_sync(grp);
+                // ---- this row's radial factors of the 16 edges (rows of padded q read the zeros left at start-up)
+                float ph[TB];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        float mv[8], ph[8], p1[8];
-                        uint4 hh, ll;
-                        *reinterpret_cast<float4*>(mv) = *reinterpret_cast<const float4*>(sM + j * PS + 8 * h);
-                        *reinterpret_cast<float4*>(mv + 4) = *reinterpret_cast<const float4*>(sM + j * PS + 8 * h + 4);
-                        *reinterpret_cast<float4*>(ph) = *reinterpret_cast<const float4*>(sPhiT + q * PS + 8 * h);
-                        *reinterpret_cast<float4*>(ph + 4) = *reinterpret_cast<const float4*>(sPhiT + q * PS + 8 * h + 4);
-                        if (!DUAL) {
+                for (int e = 0; e < TB; ++e) ph[e] = raw[e * KP + q];
+                const float* vph = raw + TB * KP + q;      // DUAL: the direction's factors are read where they are used
+                // ---- this group's A slabs of the batch, one slot each.  The stores of a slab stay in flight while the
+                // next one is computed: its slot is handed over after that.
+                int pend = -1;
+                const float* mrow = sM + (size_t)cl * PS;
+                const float* dmrow = sdM + (size_t)cl * PS;
+#pragma unroll 1
+                for (int j = grp; j < S.nslab; j += NBG, mrow += MC * PS, dmrow += MC * PS) {
+                    const uint32_t bw = slabs[j].bw;
+                    const bool rv = cl < (int)(bw >> 24) && q < a.K;
+                    const uint32_t slot = (uint32_t)j % NSLOT, use = (uint32_t)j / NSLOT;
+                    mbar_wait(bar_slotfree + 8 * slot, ((par >> slot) ^ use) & 1u, a.status);
+                    tc_fence_after();
+                    uint32_t hl[16];                 // columns 0..7: hi pairs, 8..15: lo pairs
+                    uint32_t* const hi = hl;
+                    uint32_t* const lo = hl + 8;
+                    if (rv) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) p1[e] = ph[e] * mv[e];
-                            split8(p1, hh, ll);
-                            *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
-                            *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
-                        } else if (op == 0) {
-                            float dmv[8], vph[8];
-                            *reinterpret_cast<float4*>(dmv) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h);
-                            *reinterpret_cast<float4*>(dmv + 4) = *reinterpret_cast<const float4*>(sdM + j * PS + 8 * h + 4);
-                            *reinterpret_cast<float4*>(vph) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h);
-                            *reinterpret_cast<float4*>(vph + 4) = *reinterpret_cast<const float4*>(sVphiT + q * PS + 8 * h + 4);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) p1[e] = fmaf(vph[e], mv[e], ph[e] * dmv[e]);
-                            split8(p1, hh, ll);
-                            *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
-                            *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) p1[e] = ph[e] * mv[e];
-                            split8(p1, hh, ll);
-                            *reinterpret_cast<uint4*>(sA + a_off + 128 * h) = hh;
-                            *reinterpret_cast<uint4*>(sA + a.a_cap + a_off + 128 * h) = ll;
+                        for (int e4 = 0; e4 < TB; e4 += 4) {
+                            const float4 mv = *reinterpret_cast<const float4*>(mrow + e4);
+                            float p0, p1, p2, p3;
+                            if (DUAL && op == 0) {
+                                const float4 dv = *reinterpret_cast<const float4*>(dmrow + e4);
+                                p0 = fmaf(vph[e4 * KP], mv.x, ph[e4] * dv.x);
+                                p1 = fmaf(vph[(e4 + 1) * KP], mv.y, ph[e4 + 1] * dv.y);
+                                p2 = fmaf(vph[(e4 + 2) * KP], mv.z, ph[e4 + 2] * dv.z);
+                                p3 = fmaf(vph[(e4 + 3) * KP], mv.w, ph[e4 + 3] * dv.w);
+                            } else {
+                                p0 = ph[e4] * mv.x; p1 = ph[e4 + 1] * mv.y; p2 = ph[e4 + 2] * mv.z; p3 = ph[e4 + 3] * mv.w;
+                            }
+                            split2(p0, p1, hi[e4 >> 1], lo[e4 >> 1]);
+                            split2(p2, p3, hi[(e4 >> 1) + 1], lo[(e4 >> 1) + 1]);
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) hl[i] = 0u;
                     }
+                    __syncwarp();
+                    if (pend >= 0) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) count_add(fill0 + 4 * (uint32_t)pend);
+                    }
+                    tc_st16(ring_row + slot * 16u, hl);
+                    pend = (int)slot;
                 }
-                fence_async_smem();
-                mbar_arrive(bar_ready);
+                if (pend >= 0) {
+                    tc_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) count_add(fill0 + 4 * (uint32_t)pend);
+                }
+                par ^= (uint32_t)S.oddmask;
+                if (++st == NS) { st = 0; ++round; }
             }
-            // one item behind: the previous item's accumulator drains while this item's last MMAs run
-            if (p_nl >= 0) drain(p_nl, p_set, p_mi, p_wrote);
-            p_nl = nl; p_set = set; p_mi = mi; p_wrote = seg1 > seg0;
-            if (seg1 > seg0) ++mi;
         }
-        if (p_nl >= 0) drain(p_nl, p_set, p_mi, p_wrote);
     }
 
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
 // shared bytes of the kernel for given region sizes
-int smem_need(int KP, bool dual, int dsh, int a_cap, int b_cap, int max_ent, int n_units, int n_sets, int n_comps, int max_nz) {
-    const int nop = dual ? 2 : 1;     // phi / Y / M come with their directions in the dual stream
+int smem_need(int KP, bool dual, int dsh, int ns, int b_cap, int max_ent, int n_units, int n_sets, int n_comps, int max_nz, int n_slab, int max_own) {
+    const int nop = dual ? 2 : 1;     // M comes with its direction in the dual stream
     const int stage = 2 * b_cap + ((raw_floats(KP, dual, dsh) * 4 + 1023) & ~1023);
-    size_t meta = (size_t)2 * nop * max_ent * PS + (size_t)2 * nop * KP * PS;
+    size_t meta = (size_t)NBG * 2 * nop * max_own * (128 / KP) * PS;     // coupling values of a group's own slabs, double buffered
     meta = (meta + 1) & ~size_t(1);
-    // tables: units (and at most as many blocks), sets, components, entries and sparse terms of one set
+    // tables: units (and at most as many blocks), sets, components, entries and sparse terms of one set, slabs
     const int tables = n_units * (int)(sizeof(UInfo) + sizeof(TBlk)) + n_sets * (int)sizeof(TSet) + n_comps * (int)sizeof(CompS) +
-                       max_ent * (int)sizeof(EntS) + max_nz * (int)sizeof(NzS);
-    return 1024 + 2 * a_cap + NS * stage + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
+                       max_ent * (int)sizeof(EntS) + max_nz * (int)sizeof(NzS) + n_slab * (int)sizeof(SlabW) + 16;
+    return 1024 + ns * stage + (int)(meta * 4) + (2 * MAXNS + 2 * NSLOT + 4 + 4) * 8 + tables;
 }
 
 }  // namespace
 
-// Units, sets and entries of one direction for the plain ([0]) and the dual ([1]) stream.
+// Units, passes ("sets") and entries of one direction for the plain ([0]) and the dual ([1]) stream.
 void build_tc_sets(const sobek_plan* p, Direction& dir) {
     const int KP = p->K <= 8 ? 8 : 16;
     for (int dual = 0; dual < 2; ++dual) {
@@ -677,7 +702,7 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
             }
         }
         std::sort(blocks.begin(), blocks.end(), [](const Blk& x, const Blk& y) { return x.so < y.so; });
-        // candidate units
+        // candidate units: accumulator tiles of up to 128 / KP components of one source block, split evenly
         struct Cand { int blk, c0, nc; };
         std::vector<Cand> cands;
         const int comps_per_tile = 128 / KP;
@@ -687,14 +712,9 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
             const int per = (nc + ntile - 1) / ntile;
             for (int c0 = 0; c0 < nc; c0 += per) cands.push_back(Cand{(int)b, c0, std::min(per, nc - c0)});
         }
-        auto unit_a = [&](const Cand& c) { return blocks[c.blk].d_src * (c.nc * KP) * 32; };
         auto blk_b = [&](int b) { return blocks[b].d_src * 2048 * ((blocks[b].c_src + 63) / 64); };
         auto ncols = [&](int b) { return (blocks[b].c_src + 15) & ~15; };
-        // with every multiplicity <= 32 the lo copy of a gathered row fits beside the hi copy inside one 64-column
-        // swizzle row: [B_hi | B_lo] is then one 64-column operand and a tile takes 64 accumulator columns
-        bool concat = true;
-        for (const Blk& b : blocks) concat = concat && b.c_src <= 32;
-        auto cols32 = [&](int b) { return concat ? 64 : (ncols(b) + 31) & ~31; };
+        auto cols32 = [&](int b) { return (ncols(b) + 31) & ~31; };
         auto cand_nz = [&](const Cand& c) {
             int n = 0;
             for (int cl = 0; cl < c.nc; ++cl) {
@@ -706,101 +726,124 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
             }
             return n;
         };
-        int n_comps_total = 0;
+        int n_comps_total = 0, n_slab = 0;
         for (const Blk& b : blocks) n_comps_total += (int)b.comps.size();
-        // greedy packing under a shared-memory budget: first for two CTAs per SM, else for one
-        // sets of at most `maxu` units: the largest grouping that fits two CTAs per SM, else one CTA per SM
-        for (int trial = 0; trial < 2 * (int)cands.size() && !T.ok; ++trial) {
-            const int attempt = trial / (int)cands.size();
-            const int maxu = (int)cands.size() - trial % (int)cands.size();
-            const int budget = (attempt == 0 ? 113 : 226) * 1024;
-            const int col_budget = attempt == 0 ? 128 : 256;     // two accumulator buffers per CTA
-            T = TcSets{};
-            bool fits = true;
-            size_t i = 0;
-            while (i < cands.size() && fits) {
-                int a_bytes = 0, b_bytes = 0, cols = 0, nent = 0, nnz = 0;
-                std::vector<int> set_blks;
-                size_t j = i;
-                for (; j < cands.size() && (int)(j - i) < maxu; ++j) {
-                    const Cand& c = cands[j];
-                    const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
-                    const int a2 = a_bytes + unit_a(c), b2 = b_bytes + (new_blk ? blk_b(c.blk) : 0);
-                    const int c2 = cols + cols32(c.blk), e2 = nent + c.nc * blocks[c.blk].d_src, n2 = nnz + cand_nz(c);
-                    // the kernel sizes its regions by the maxima over all sets
-                    const int acap = std::max(T.a_cap, (a2 + 4096 + 1023) & ~1023), bcap = std::max(T.b_cap, (b2 + 1023) & ~1023);
-                    const int need = smem_need(KP, dual, p->dim_sh, acap, bcap, std::max(T.max_ent, e2), (int)cands.size(), (int)cands.size(),
-                                               n_comps_total, std::max(T.max_nz, n2));
-                    if (need > budget || c2 > col_budget) break;
-                    a_bytes = a2; b_bytes = b2; cols = c2; nent = e2; nnz = n2;
-                    if (new_blk) set_blks.push_back(c.blk);
-                }
-                if (j == i) { fits = false; break; }
-                // emit the set
-                TSet S{};
-                S.unit_begin = (int)T.units.size(); S.blk_begin = (int)T.blks.size(); S.ent_begin = (int)T.ents.size();
-                int a_off = 0, b_off = 0, col = 0;
-                std::vector<int> local_blk;   // block index -> index in T.blks
-                for (size_t k = i; k < j; ++k) {
-                    const Cand& c = cands[k];
-                    const Blk& Bk = blocks[c.blk];
-                    int bi = -1;
-                    for (size_t m = 0; m < local_blk.size(); ++m) if (local_blk[m] == c.blk) bi = S.blk_begin + (int)m;
-                    if (bi < 0) {
-                        TBlk tb{};
-                        tb.src_off = Bk.so; tb.c_src = Bk.c_src; tb.d_src = Bk.d_src; tb.ncols = ncols(c.blk);
-                        tb.b_off = b_off; tb.slab_bytes = 2048 * ((Bk.c_src + 63) / 64); tb.atom_stride = 2048;
-                        b_off += blk_b(c.blk);
-                        S.b_items += Bk.d_src * TB * (Bk.c_src / 8);
-                        bi = (int)T.blks.size();
-                        T.blks.push_back(tb);
-                        local_blk.push_back(c.blk);
-                    }
-                    TUnit U{};
-                    U.blk = bi; U.comp_begin = (int)T.comps.size(); U.ncomp = c.nc; U.a_off = a_off;
-                    U.slab_stride = c.nc * KP * 32; U.tmem_col = col;
-                    for (int cl = 0; cl < c.nc; ++cl) {
-                        const SComp& cp = Bk.comps[c.c0 + cl];
-                        T.comps.push_back(cp);
-                        for (int s = 0; s < Bk.d_src; ++s)
-                            T.ents.push_back(TEnt{cp.tab0 + s * cp.tstride, cp.sh_off, a_off + s * U.slab_stride + cl * KP * 32, 0});
-                    }
-                    a_off += unit_a(c);
-                    col += cols32(c.blk);
-                    T.units.push_back(U);
-                }
-                S.nunit = (int)T.units.size() - S.unit_begin; S.nblk = (int)T.blks.size() - S.blk_begin;
-                S.nent = (int)T.ents.size() - S.ent_begin;
-                T.sets.push_back(S);
-                T.a_cap = std::max(T.a_cap, (a_off + 4096 + 1023) & ~1023);
-                T.b_cap = std::max(T.b_cap, (b_off + 1023) & ~1023);
-                T.max_ent = std::max(T.max_ent, S.nent);
-                T.max_nz = std::max(T.max_nz, nnz);
-                T.acc_cols = std::max(T.acc_cols, col);
-                i = j;
+        for (const Cand& c : cands) n_slab += blocks[c.blk].d_src;        // one slab per (tile, s)
+        // greedy packing of consecutive units into passes: the accumulator tiles of a pass fit one of the two TMEM
+        // buffers and its operand regions fit shared memory with at least two ring stages
+        const int budget = 227 * 1024;
+        bool fits = true;
+        size_t i = 0;
+        while (i < cands.size() && fits) {
+            int b_bytes = 0, cols = 0, nent = 0, nnz = 0, slabs_in = 0;
+            std::vector<int> set_blks;
+            size_t j = i;
+            for (; j < cands.size(); ++j) {
+                const Cand& c = cands[j];
+                const bool new_blk = std::find(set_blks.begin(), set_blks.end(), c.blk) == set_blks.end();
+                const int b2 = b_bytes + (new_blk ? blk_b(c.blk) : 0);
+                const int c2 = cols + cols32(c.blk), e2 = nent + c.nc * blocks[c.blk].d_src, n2 = nnz + cand_nz(c);
+                // the kernel sizes its regions by the maxima over all passes
+                const int bcap = std::max(T.b_cap, (b2 + 1023) & ~1023);
+                const int own2 = (slabs_in + blocks[c.blk].d_src + NBG - 1) / NBG;
+                const int need = smem_need(KP, dual, p->dim_sh, 2, bcap, std::max(T.max_ent, e2), (int)cands.size(), (int)cands.size(),
+                                           n_comps_total, std::max(T.max_nz, n2), n_slab, std::max(T.max_units, own2));
+                if (need > budget || c2 > ACC_BUDGET) break;
+                b_bytes = b2; cols = c2; nent = e2; nnz = n2; slabs_in += blocks[c.blk].d_src;
+                if (new_blk) set_blks.push_back(c.blk);
             }
-            if (!fits) continue;
-            int tc = 32; while (tc < 2 * T.acc_cols) tc <<= 1;
-            T.tmem_cols = tc;
-            T.smem_bytes = smem_need(KP, dual, p->dim_sh, T.a_cap, T.b_cap, T.max_ent, (int)cands.size(), (int)cands.size(), n_comps_total, T.max_nz);
-            if (T.smem_bytes > 227 * 1024 || T.tmem_cols > 512) continue;
-            T.ctas_per_sm = (T.smem_bytes <= 113 * 1024 && T.tmem_cols <= 256) ? 2 : 1;
-            T.concat = concat ? 1 : 0;
-            // shared-memory images of the tables
-            for (TSet& S : T.sets) {
-                S.b_items = (int)T.nz.size();
-                for (int j = 0; j < S.nent; ++j) {
-                    const TEnt& E = T.ents[S.ent_begin + j];
-                    EntS es{E.a_off, (int)T.nz.size() - S.b_items, p->tab_ptr[E.tab + 1] - p->tab_ptr[E.tab], 0};
-                    for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k) T.nz.push_back(NzS{E.sh_off + p->tab_idx[k], p->tab_coef[k]});
-                    T.ents_s.push_back(es);
+            if (j == i) { fits = false; break; }
+            TSet S{};
+            S.unit_begin = (int)T.units.size(); S.blk_begin = (int)T.blks.size(); S.ent_begin = (int)T.ents.size();
+            int b_off = 0, col = 0, ent = 0;
+            std::vector<int> local_blk;   // block index -> index in T.blks
+            for (size_t k = i; k < j; ++k) {
+                const Cand& c = cands[k];
+                const Blk& Bk = blocks[c.blk];
+                int bi = -1;
+                for (size_t m = 0; m < local_blk.size(); ++m) if (local_blk[m] == c.blk) bi = S.blk_begin + (int)m;
+                if (bi < 0) {
+                    TBlk tb{};
+                    tb.src_off = Bk.so; tb.c_src = Bk.c_src; tb.d_src = Bk.d_src; tb.ncols = ncols(c.blk);
+                    tb.b_off = b_off; tb.slab_bytes = 2048 * ((Bk.c_src + 63) / 64); tb.atom_stride = 2048;
+                    b_off += blk_b(c.blk);
+                    bi = (int)T.blks.size();
+                    T.blks.push_back(tb);
+                    local_blk.push_back(c.blk);
                 }
-                S.pad = (int)T.nz.size() - S.b_items;
+                TUnit U{};
+                U.blk = bi; U.comp_begin = (int)T.comps.size(); U.ncomp = c.nc;
+                U.a_off = ent;                 // first entry of the unit inside the pass: entry = a_off + cl * d_src + s
+                U.slab_stride = 0; U.tmem_col = col;
+                for (int cl = 0; cl < c.nc; ++cl) {
+                    const SComp& cp = Bk.comps[c.c0 + cl];
+                    T.comps.push_back(cp);
+                    for (int s = 0; s < Bk.d_src; ++s) T.ents.push_back(TEnt{cp.tab0 + s * cp.tstride, cp.sh_off, 0, 0});
+                }
+                ent += c.nc * Bk.d_src;
+                col += cols32(c.blk);
+                T.units.push_back(U);
             }
-            for (const SComp& cp : T.comps)
-                T.comps_s.push_back(CompS{dir.zb_off[cp.group], dir.nk_ld[cp.group], cp.d_dst, cp.o, cp.koff, {0, 0}});
-            T.ok = true;
+            S.nunit = (int)T.units.size() - S.unit_begin; S.nblk = (int)T.blks.size() - S.blk_begin;
+            S.nent = (int)T.ents.size() - S.ent_begin;
+            // build order of the pass's slabs: tile after tile in turn (s = 0 of every tile, then s = 1, ...), so that
+            // the builder groups (slab j mod NBG) and the MMA threads (tile mod NMW) find work at the same rate
+            S.sched_begin = (int)T.slabs.size() / 2;
+            std::vector<uint32_t> order;      // (tile << 8) | s
+            for (int sdx = 0, more = 1; more; ++sdx) {
+                more = 0;
+                for (int u = 0; u < S.nunit; ++u)
+                    if (sdx < T.blks[T.units[S.unit_begin + u].blk].d_src) { order.push_back(((uint32_t)u << 8) | (uint32_t)sdx); more = 1; }
+            }
+            S.nslab = (int)order.size();
+            S.mfirst = 0x00ffffff;
+            S.oddmask = 0;
+            for (int sl = 0; sl < NSLOT; ++sl)
+                if (((S.nslab - sl + NSLOT - 1) / NSLOT) & 1) S.oddmask |= 1 << sl;      // slots used an odd number of times per batch
+            for (int j = 0; j < S.nslab; ++j) {
+                const int u = (int)(order[j] >> 8), sdx = (int)(order[j] & 255u);
+                const TUnit& Uu = T.units[S.unit_begin + u];
+                const int d = T.blks[Uu.blk].d_src;
+                uint32_t next = 255;
+                for (int k = j + 1; k < S.nslab && next == 255; ++k)
+                    if ((int)(order[k] >> 8) % NMW == u % NMW) next = (uint32_t)k;
+                T.slabs.push_back((uint32_t)(Uu.a_off + sdx) | ((uint32_t)d << 16) | ((uint32_t)Uu.ncomp << 24));
+                T.slabs.push_back((uint32_t)u | ((uint32_t)sdx << 8) | (next << 16));
+                const int t = u % NMW;
+                if (((S.mfirst >> (8 * t)) & 255) == 255) S.mfirst = (S.mfirst & ~(255 << (8 * t))) | (j << (8 * t));
+            }
+            if (S.nslab > 254) fits = false;
+            T.max_units = std::max(T.max_units, (S.nslab + NBG - 1) / NBG);      // own slabs of a builder group at most
+            T.sets.push_back(S);
+            T.b_cap = std::max(T.b_cap, (b_off + 1023) & ~1023);
+            T.max_ent = std::max(T.max_ent, S.nent);
+            T.max_nz = std::max(T.max_nz, nnz);
+            T.acc_cols = std::max(T.acc_cols, col);
+            i = j;
         }
+        if (!fits) { T = TcSets{}; continue; }
+        // as many ring stages as shared memory holds (the loaders run that many batches ahead)
+        int ns = 2;
+        while (ns < MAXNS && smem_need(KP, dual, p->dim_sh, ns + 1, T.b_cap, T.max_ent, (int)cands.size(), (int)cands.size(),
+                                       n_comps_total, T.max_nz, n_slab, T.max_units) <= budget) ++ns;
+        T.ctas_per_sm = 1;
+        T.ring_stages = ns;
+        T.tmem_cols = TMEM_COLS;
+        T.smem_bytes = smem_need(KP, dual, p->dim_sh, ns, T.b_cap, T.max_ent, (int)cands.size(), (int)cands.size(), n_comps_total, T.max_nz, n_slab, T.max_units);
+        // shared-memory images of the tables
+        for (TSet& S : T.sets) {
+            S.b_items = (int)T.nz.size();
+            for (int j = 0; j < S.nent; ++j) {
+                const TEnt& E = T.ents[S.ent_begin + j];
+                EntS es{0, (int)T.nz.size() - S.b_items, p->tab_ptr[E.tab + 1] - p->tab_ptr[E.tab], 0};
+                for (int k = p->tab_ptr[E.tab]; k < p->tab_ptr[E.tab + 1]; ++k) T.nz.push_back(NzS{E.sh_off + p->tab_idx[k], p->tab_coef[k]});
+                T.ents_s.push_back(es);
+            }
+            S.pad = (int)T.nz.size() - S.b_items;
+        }
+        for (const SComp& cp : T.comps)
+            T.comps_s.push_back(CompS{dir.zb_off[cp.group], dir.nk_ld[cp.group], cp.d_dst, cp.o, cp.koff, {0, 0}});
+        T.ok = true;
     }
 }
 
@@ -818,7 +861,9 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
-    a.a_cap = T.a_cap; a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.tmem_cols = T.tmem_cols; a.acc_cols = T.acc_cols; a.concat = T.concat; a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
+    a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages;
+    a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
+    a.slabs = T.d_slabs; a.n_slab = (int)T.slabs.size() / 2; a.max_own = T.max_units;
     a.status = status;
     const bool k8 = p->K <= 8;
     void (*kern)(const TcArgs) = k8 ? (dual ? k_stream_tc<8, true> : k_stream_tc<8, false>)
@@ -826,7 +871,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T.smem_bytes);
     if (e != cudaSuccess) return e;
     const int64_t total = n_nodes * a.nsets;
-    const int grid = (int)std::min<int64_t>(total, (int64_t)148 * T.ctas_per_sm);
+    const int grid = (int)std::min<int64_t>(total, (int64_t)148);
     KernelTimer kt(K_STATE, s);
     kern<<<grid, TT, T.smem_bytes, s>>>(a);
     count_launch();
