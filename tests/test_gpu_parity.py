@@ -252,6 +252,7 @@ FULL = {
     "cfg3": (synth.config("cfg3"), 6, (0, 1, 2)),
     "cfg4_1e5": (synth.config("cfg4", edges=1e5), 8, (0, 1)),
     "cfg4_1e6": (synth.config("cfg4", edges=1e6), 8, (0, 1)),
+    "cfg4t_10": (synth.config("cfg4t_10"), 8, (0, 1)),          # 1e7 edges: ten copies of the 1e6-edge graph
     "cfg5": (synth.config("cfg5"), 3, (0, 1, 2)),
 }
 
@@ -284,6 +285,85 @@ def test_full_size_sampled(name):
         assert rel_err(got[0][act], ref[0][act]) <= BWD_TOL
         assert rel_err(got[1], ref[1]) <= BWD_TOL and rel_err(got[4], ref[4]) <= BWD_TOL
         assert rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL and rel_err(got[3][ed], ref[3][ed]) <= BWD_TOL
+
+
+# ---------------------------------------------------------------------------------------
+# the top of the edge-scaling sweep (section "Scaling axes"): 5e7, 1e8 and 1.4e8 edges
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("copies", [50, 100, 140])
+def test_edge_sweep_top_sampled(copies):
+    """Forward and backward of the sweep profile on `copies` disjoint copies of its 1e6-edge graph (5.0e7 / 1.0e8 /
+    1.4e8 edges, up to 4.4 M nodes; with 140 copies E*K and N*C_x both pass 2^31, so that every offset of the kernels
+    has to be 64-bit).  A receiver only sees its own copy, so the oracle is run on single copies: on the sampled
+    receivers of three copies (first, middle, last) with that copy's features, with the output adjoint zero outside the
+    sample.  Checked: y of the sampled receivers, gY / gphi of their edges, gx of the three copies (and exact zeros in
+    the copies in between), gR (= the sum over the copies' oracle runs)."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    w = synth.config(f"cfg4t_{copies}")
+    oracle = oconv.Oracle(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    d = synth.make_inputs(w, oracle.col_std(), with_cotangents=False)
+    n1, B = w.N, copies
+    e1 = d.E // B
+    assert d.N == n1 * B and d.E == e1 * B
+    if copies == 140:
+        assert d.E * w.K > 2 ** 31 and d.N * plan.info.C_x > 2 ** 31
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(a).to(dev)
+    row_ptr, col = t(d.row_ptr.astype(np.int64)), t(d.col)
+    src_ptr, src_perm = sb.graph_prepare(row_ptr, col)
+    src_recv = sb.graph_receivers(row_ptr, src_perm)
+    g = sb.make_graph(row_ptr, col, src_ptr, src_perm, src_recv)
+    x, Y, phi, R = t(d.x), t(d.Y), t(d.phi), t(d.R)
+    rng = np.random.default_rng(7)
+    check = [0, B // 2, B - 1]
+    local = {b: np.unique(np.concatenate([[0, n1 - 1], rng.choice(n1, size=2, replace=False)])) for b in check}
+    i = plan.info
+    # ---- forward
+    ws = torch.empty(sb.workspace_bytes(plan, d.N, d.E, 0), dtype=torch.uint8, device=dev)
+    y = torch.full((d.N, i.C_y), float("nan"), dtype=torch.float32, device=dev)
+    sb.conv_fwd(plan, g, x, Y, phi, R, y, ws)
+    assert sb.last_device_status(ws) == 0
+    assert bool(torch.isfinite(y).all())
+    base_rp = d.row_ptr[:n1 + 1].astype(np.int64)
+    base_col = d.col[:e1].astype(np.int32)
+    for b in check:
+        act = local[b]
+        ref = oracle.fwd(base_rp, base_col, d.x[b * n1:(b + 1) * n1], d.Y[b * e1:(b + 1) * e1], d.phi[b * e1:(b + 1) * e1],
+                         d.R, act=act)
+        got = y[b * n1 + torch.from_numpy(act).to(dev)].cpu().numpy()
+        assert rel_err(got, ref[act]) <= FWD_TOL, b
+    del y, ws
+    torch.cuda.empty_cache()
+    # ---- backward, output adjoint supported on the sampled receivers
+    gy_host = np.zeros((d.N, i.C_y), dtype=np.float32)
+    for b in check:
+        gy_host[b * n1 + local[b]] = d.gy[b * n1 + local[b]]
+    gy = t(gy_host)
+    ws = torch.empty(sb.workspace_bytes(plan, d.N, d.E, 1), dtype=torch.uint8, device=dev)
+    new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device=dev)
+    gx, gY, gphi, gR = new(d.N, i.C_x), new(d.E, i.dim_sh), new(d.E, i.K), new(i.K, i.N_w)
+    sb.conv_bwd(plan, g, x, Y, phi, R, gy, gx, gY, gphi, gR, ws)
+    assert sb.last_device_status(ws) == 0
+    gR_ref = np.zeros((i.K, i.N_w))
+    for b in check:
+        act = local[b]
+        rx, rY, rphi, rR = oracle.bwd(base_rp, base_col, d.x[b * n1:(b + 1) * n1], d.Y[b * e1:(b + 1) * e1],
+                                      d.phi[b * e1:(b + 1) * e1], d.R, gy_host[b * n1:(b + 1) * n1], act=act)
+        gR_ref += rR
+        assert rel_err(gx[b * n1:(b + 1) * n1].cpu().numpy(), rx) <= BWD_TOL, b
+        ed = np.concatenate([np.arange(base_rp[r], base_rp[r + 1]) for r in act])
+        ge = torch.from_numpy(b * e1 + ed).to(dev)
+        assert rel_err(gY[ge].cpu().numpy(), rY[ed]) <= BWD_TOL, b
+        assert rel_err(gphi[ge].cpu().numpy(), rphi[ed]) <= BWD_TOL, b
+    assert rel_err(gR.cpu().numpy(), gR_ref) <= BWD_TOL
+    # copies without a sampled receiver get exact zeros
+    other = 1 if B > 3 else None
+    if other is not None:
+        assert float(gx[other * n1:(other + 1) * n1].abs().max()) == 0.0
+        assert float(gY[other * e1:(other + 1) * e1].abs().max()) == 0.0
+    assert bool(torch.isfinite(gx).all()) and bool(torch.isfinite(gphi).all())
 
 
 # ---------------------------------------------------------------------------------------

@@ -195,6 +195,13 @@ def config(name: str, **kw) -> Workload:
         L = _cube(N, 0.1)
         return Workload("cfg3", P("128x0e+128x1o"), P("128x0e+128x1o+128x2e+128x3o"), 3, 8, N, L,
                         cutoff_for_edges(N, 30.0 * N, L), "bessel")
+    if name.startswith("cfg4t_"):
+        # the edge-scaling sweep beyond 1e6 edges: the 1e6-edge graph of the sweep repeated B times (disjoint copies in
+        # one batch; the node features are drawn for every copy), so that 1e7 ... 1e8 edges are generated in seconds
+        base = config("cfg4", edges=1e6)
+        B = int(name.split("_")[1])
+        return Workload(name, base.irreps_in, base.irreps_out, 2, 16, base.N, base.L, base.r_c, "bessel", orders=(0, 1),
+                        copies=B, note=f"{B} copies of cfg4_1e6")
     if name.startswith("cfg4"):
         E = float(kw.get("edges", name.split("_")[1] if "_" in name else 1e5))
         ir = P("64x0e+64x1o+64x2e")
@@ -298,35 +305,42 @@ def make_inputs(w: Workload, col_std: np.ndarray, dtype=np.float32,
     s_pos, s_x, s_R, s_gy, s_vx, s_vY, s_vphi, s_vR = [np.random.default_rng(s) for s in ss.spawn(8)]
     pos = w.L * s_pos.random((w.N, 3))
     row_ptr, col, recv = radius_graph(pos, w.r_c)
+    # edge inputs of the base graph (computed once, then repeated with the graph)
+    e1 = int(col.shape[0])
+    rij = pos[col] - pos[recv]
+    r = np.linalg.norm(rij, axis=1)
+    dsh = (w.l_max + 1) ** 2
+    Y = real_sph_harm(w.l_max, rij) if e1 else np.zeros((0, dsh))
+    phi = gaussian_basis(r, w.K, w.r_c) if w.basis == "gaussian" else bessel_basis(r, w.K, w.r_c)
     if w.copies > 1:
-        # disjoint copies of the same graph: node ids of copy b are shifted by b * N
-        n1, e1, B = w.N, int(col.shape[0]), int(w.copies)
+        # disjoint copies of the same graph: node ids of copy b are shifted by b * N; the edge inputs repeat, the
+        # node features below are drawn for every node of every copy
+        n1, B = w.N, int(w.copies)
         shift = (np.arange(B, dtype=np.int64) * n1)[:, None]
         col = (col[None, :].astype(np.int64) + shift).reshape(-1).astype(np.int32)
         recv = (recv[None, :].astype(np.int64) + shift).reshape(-1).astype(np.int32)
         row_ptr = np.concatenate([[0], (row_ptr[None, 1:] + (np.arange(B, dtype=np.int64) * e1)[:, None]).reshape(-1)])
         pos = np.tile(pos, (B, 1))
+        Y = np.tile(Y.astype(dtype), (B, 1))
+        phi = np.tile(phi.astype(dtype), (B, 1))
     N_tot = w.N * max(1, int(w.copies))
     E = int(col.shape[0])
-    rij = pos[col] - pos[recv]
-    r = np.linalg.norm(rij, axis=1)
-    Y = real_sph_harm(w.l_max, rij) if E else np.zeros((0, (w.l_max + 1) ** 2))
-    if w.basis == "gaussian":
-        phi = gaussian_basis(r, w.K, w.r_c)
-    else:
-        phi = bessel_basis(r, w.K, w.r_c)
     C_x, C_y = irreps_dim(w.irreps_in), irreps_dim(w.irreps_out)
-    x = s_x.standard_normal((N_tot, C_x))
+    # node-sized Gaussians: in the target precision directly once they are large (the fp64 draw of a graph with millions
+    # of nodes would need tens of gigabytes of host memory)
+    big = N_tot * max(C_x, C_y) > 50_000_000
+    normal = (lambda g, shape: g.standard_normal(shape, dtype=np.float32)) if (big and dtype == np.float32) else \
+             (lambda g, shape: g.standard_normal(shape))
+    x = normal(s_x, (N_tot, C_x))
     R = s_R.standard_normal((w.K, N_w)) * col_std[None, :]
     vR = s_vR.standard_normal((w.K, N_w)) * col_std[None, :]
-    gy = s_gy.standard_normal((N_tot, C_y))
-    dsh = (w.l_max + 1) ** 2
+    gy = normal(s_gy, (N_tot, C_y))
     if with_cotangents:
-        vx = s_vx.standard_normal((N_tot, C_x))
-        vY = s_vY.standard_normal((E, dsh))
-        vphi = s_vphi.standard_normal((E, w.K))
+        vx = normal(s_vx, (N_tot, C_x))
+        vY = normal(s_vY, (E, dsh))
+        vphi = normal(s_vphi, (E, w.K))
     else:
         vx = np.zeros((0, C_x)); vY = np.zeros((0, dsh)); vphi = np.zeros((0, w.K))
-    c = lambda a: np.ascontiguousarray(a.astype(dtype))
+    c = lambda a: np.ascontiguousarray(a if a.dtype == dtype else a.astype(dtype))
     return Inputs(w, N_tot, E, row_ptr, col, recv, c(x), c(Y), c(phi), c(R), c(gy), c(vx), c(vY),
                   c(vphi), c(vR), pos)
