@@ -314,6 +314,8 @@ def main():
     ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="skip the table of the other configurations")
+    ap.add_argument("--nodes", type=int, default=0,
+                    help="run the workload's profile on a graph scaled to this many nodes (same density and degree): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -335,7 +337,10 @@ def main():
         dist = dist_mod
 
     # replicas only: every rank runs the same workload on its own GPU (different seed per rank)
-    r = Run(sb, torch, dev, synth.config(args.workload), rank)
+    wl = synth.config(args.workload)
+    if args.nodes > 0:
+        wl = synth.scaled(wl, args.nodes)
+    r = Run(sb, torch, dev, wl, rank)
     w, plan, i, N, E, t, out, ws, g, host, flush = r.w, r.plan, r.info, r.N, r.E, r.t, r.out, r.ws, r.g, r.host, r.flush
     host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
 

@@ -79,15 +79,18 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     w.zbh = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
     w.zbl = (uint16_t*)take((size_t)w.chunk * (size_t)zb * 2);
     if (order >= 1) {
-        w.zbar = (float*)take((size_t)w.chunk * (size_t)p->fwd.state_floats * 4);
         if (gemm) {
             w.gbh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
             w.gbl = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.gb_elems * 2);
         }
-    }
-    if (order >= 1 && p->use_tc_edge && p->fwd.etc[0].ok) {
-        w.zqh = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.zb_elems * 2);
-        w.zql = (uint16_t*)take((size_t)w.chunk * (size_t)p->fwd.zb_elems * 2);
+        if (p->use_tc_edge && p->fwd.etc[0].ok) {
+            // the adjoint state of a chunk is made after the chunk's state has been consumed (by the mixing and
+            // weight-adjoint contractions): the two share one buffer
+            w.zqh = w.zbh;
+            w.zql = w.zbl;
+        } else {
+            w.zbar = (float*)take((size_t)w.chunk * (size_t)p->fwd.state_floats * 4);
+        }
     }
     if (p->use_tc_stream || (p->use_tc_edge && p->fwd.etc[0].ok)) {
         const size_t nx = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 2, ny = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 2;

@@ -365,11 +365,12 @@ void build_direction(sobek_plan* p, int transposed, Direction& dir) {
 }  // namespace
 
 int64_t chunk_nodes(const sobek_plan* p, int64_t N, int order) {
-    // bytes per node held at once: the bf16 (hi, lo) state and, for orders >= 1, the fp32 adjoint
-    // state and the bf16 (hi, lo) rows of the output adjoint
+    // bytes per node held at once: the bf16 (hi, lo) state (its adjoint takes the same buffer in turn) and, for
+    // orders >= 1, the bf16 (hi, lo) rows of the output adjoint and - FP32-pipe edge pass only - the fp32 adjoint state
     int64_t zb = p->fwd.zb_elems;
     if (order >= 1) zb = std::max(zb, p->tr.zb_elems);
-    int64_t per = 4 * zb + (order >= 1 ? 4 * p->fwd.state_floats + 4 * p->fwd.gb_elems : 0);
+    const bool tc_edge = p->use_tc_edge && p->fwd.etc[0].ok;     // else the edge pass reads an fp32 adjoint state
+    int64_t per = 4 * zb + (order >= 1 ? (tc_edge ? 0 : 4 * p->fwd.state_floats) + 4 * p->fwd.gb_elems : 0);
     per = std::max<int64_t>(per, 1);
     // the budget bounds the chunk, but a chunk never has fewer than kMinChunkNodes nodes: below that the
     // node-side kernels cannot fill the machine
