@@ -124,9 +124,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     float* sGM = sdM + (DUAL ? (size_t)a.nent * PS : 0);       // [nent][PS]
     float* sPphi = sGM + (size_t)a.nent * PS;                  // [NCW*32][KP]: one row per compute thread
     uint64_t* bars = reinterpret_cast<uint64_t*>(sPphi + NCW * 32 * KP);
-    // bars: full[NS], free[NS], zfull, zfree, acc_full[2], acc_free[2]
+    // bars: full[NS], free[NS], acc_full[2], acc_free[2], (tmem address), zfull[nunit], zfree[nunit]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
-    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8);           // [nunit]
+    UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8 + 2 * a.nunit);     // [nunit]
     TBlk* sBlk = reinterpret_cast<TBlk*>(sU + a.nunit);                // [nunit]
     CompS* sComp = reinterpret_cast<CompS*>(sBlk + a.nunit);           // [ncomp]
     EntS* sEnt = reinterpret_cast<EntS*>(sComp + a.ncomp);             // [nent]
@@ -134,8 +134,10 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     NzS* sInv = sNz + a.nnz;                                           // [ninv]
     int32_t* sInvPtr = reinterpret_cast<int32_t*>(sInv + a.ninv);      // [dsh + 1]
     const uint32_t bar0 = smem_u32(bars);
-    const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_zfull = bar0 + 16 * NS, bar_zfree = bar_zfull + 8,
-                   bar_accfull = bar_zfull + 16, bar_accfree = bar_zfull + 32;
+    // the Zbar slabs of a unit have a pair of barriers of their own: a unit's slabs are refilled for the next receiver
+    // as soon as the last batch's MMAs of that unit have retired, while the later units are still being multiplied
+    const uint32_t bar_full = bar0, bar_free = bar0 + 8 * NS, bar_accfull = bar0 + 16 * NS, bar_accfree = bar_accfull + 16,
+                   bar_zfull = bar0 + 8 * (2 * NS + 8), bar_zfree = bar_zfull + 8 * (uint32_t)a.nunit;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool has_vx = DUAL && a.vsh != nullptr, has_vY = DUAL && a.vY != nullptr, has_vphi = DUAL && a.vphi != nullptr;
@@ -149,8 +151,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     if (tid == 0) {
         // a stage is released by the commit of the batch's MMAs and by every compute thread (raw rows read)
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 1 + NCW * 32); }
-        mbar_init(bar_zfull, NLW * 32);
-        mbar_init(bar_zfree, 1);
+        for (int u = 0; u < a.nunit; ++u) { mbar_init(bar_zfull + 8 * u, NLW * 32); mbar_init(bar_zfree + 8 * u, 1); }
         for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW * 32); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -208,29 +209,39 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
             seg_bounds(a.row_ptr, a.node0 + nl, a.E, a.status, seg0, seg1);
             if (!any_op) seg1 = seg0;
             if (seg1 <= seg0) continue;
-            // ---- Zbar slabs of the receiver (once the previous receiver's MMAs have read theirs)
-            if (zi > 0) mbar_wait(bar_zfree, (zi - 1) & 1, a.status);
-            for (int ui = 0; ui < S.nunit; ++ui) {
-                const UInfo U = sU[ui];
-                const int cpr = (int)U.c_src >> 3;
-                const int n_it = (int)U.ncomp * a.K * cpr;
-                for (int i = lt; i < n_it; i += NLW * 32) {
-                    const int rowi = i / cpr, j = i - rowi * cpr;
-                    const int cl = rowi / a.K, q = rowi - cl * a.K;
-                    const CompS cp = sComp[U.comp_begin + cl];
-                    const int64_t g = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff +
-                                      (int64_t)q * U.c_src + 8 * j;
-                    const int r = cl * KP + q, u = 8 * j;
-                    const uint32_t d = smem_u32(sZ) + (uint32_t)(U.z_off + (u >> 6) * U.z_kb + r * 128 + ((((u & 63) >> 3) ^ (r & 7)) << 4));
-                    cp_async16_zfill(d, a.zqh + g, 16);
-                    cp_async16_zfill(d + (uint32_t)a.z_cap, a.zql + g, 16);
+            // ---- Zbar slabs, unit by unit (each once the previous receiver's MMAs of that unit have read theirs);
+            // a loader warp takes whole components: K rows of c_src multiplicities, contiguous in the state
+            auto load_zbar = [&]() {
+                for (int ui = 0; ui < S.nunit; ++ui) {
+                    const UInfo U = sU[ui];
+                    if (zi > 0) mbar_wait(bar_zfree + 8 * ui, (zi - 1) & 1, a.status);
+                    const int cpr = (int)U.c_src >> 3;
+                    const int n_it = a.K * cpr;
+                    for (int cl = warp - NCW; cl < (int)U.ncomp; cl += NLW) {
+                        const CompS cp = sComp[U.comp_begin + cl];
+                        const int64_t g0 = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff;
+                        const __nv_bfloat16* gh = a.zqh + g0;
+                        const __nv_bfloat16* gl = a.zql + g0;
+                        const uint32_t d0 = smem_u32(sZ) + U.z_off + (uint32_t)(cl * KP) * 128u;
+                        for (int i = lane; i < n_it; i += 32) {
+                            const int q = i / cpr, j = i - q * cpr;
+                            const int r = cl * KP + q;
+                            const uint32_t d = d0 + (uint32_t)((j >> 3) * U.z_kb + q * 128 + (((j & 7) ^ (r & 7)) << 4));
+                            cp_async16_zfill(d, gh + 8 * i, 16);
+                            cp_async16_zfill(d + (uint32_t)a.z_cap, gl + 8 * i, 16);
+                        }
+                    }
+                    cp_async_arrive(bar_zfull + 8 * ui);
                 }
-            }
-            cp_async_arrive(bar_zfull);
-            ++zi;
-            // ---- the batches of the receiver
-            for (int64_t b0 = seg0; b0 < seg1; b0 += tb)
-            for (int sb = 0; sb < nsub; ++sb, ++it) {
+                ++zi;
+            };
+            // ---- the batches of the receiver; the first one is staged ahead of the Zbar slabs (its stage does not wait
+            // for the previous receiver's MMAs to end)
+            const int nbat = (int)((seg1 - seg0 + tb - 1) / tb) * nsub;
+            for (int bi_ = 0; bi_ < nbat; ++bi_, ++it) {
+                if (bi_ == 1) load_zbar();
+                const int64_t b0 = seg0 + (int64_t)(bi_ / nsub) * tb;
+                const int sb = bi_ - (bi_ / nsub) * nsub;
                 const int op = use_x ? sb : 1;
                 const int nb = (int)min((int64_t)tb, seg1 - b0);
                 const int st = (int)(it % NS);
@@ -297,6 +308,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 }
                 cp_async_arrive(bar_full + 8 * st);
             }
+            if (nbat == 1) load_zbar();
         }
     } else if (warp == NCW + NLW) {
         // =========================== MMA warp ===========================
@@ -308,10 +320,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                 seg_bounds(a.row_ptr, a.node0 + nl, a.E, nullptr, seg0, seg1);
                 if (!any_op) seg1 = seg0;
                 if (seg1 <= seg0) continue;
-                mbar_wait(bar_zfull, zi & 1, a.status);
-                ++zi;
                 for (int64_t b0 = seg0; b0 < seg1; b0 += tb)
                 for (int sb = 0; sb < nsub; ++sb, ++it) {
+                    const bool first = b0 == seg0 && sb == 0, last = b0 + tb >= seg1 && sb == nsub - 1;
                     const int st = (int)(it % NS);
                     mbar_wait(bar_full + 8 * st, (it / NS) & 1, a.status);
                     fence_async_smem();
@@ -320,7 +331,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                     for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
                         const UInfo U = sU[ui];
                         const uint32_t buf = ai & 1;
+                        if (first) mbar_wait(bar_zfull + 8 * ui, zi & 1, a.status);
                         if (ai >= 2) mbar_wait(bar_accfree + 8 * buf, ((ai >> 1) & 1) ^ 1, a.status);
+                        fence_async_smem();
                         tc_fence_after();
                         for (uint32_t mt = 0; mt < U.nmt; ++mt) {
                             const uint32_t d_tmem = tmem_base + buf * (uint32_t)a.acc_cols + mt * U.npad;
@@ -338,10 +351,11 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                             }
                         }
                         tc_commit(bar_accfull + 8 * buf);
+                        if (last) tc_commit(bar_zfree + 8 * ui);
                     }
                     tc_commit(bar_free + 8 * st);
                 }
-                tc_commit(bar_zfree);
+                ++zi;
             }
         }
     } else {
@@ -465,7 +479,8 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                                 float v = 0.f;
                                 for (int r = ee; r < 128; r += tb) v += sPphi[r * KP + q] + sPphi[(128 + r) * KP + q];
                                 float* p = a.gphi + (b0 + ee) * a.K + q;
-                                *p = a.phi_mode == 2 ? *p + v : v;
+                                // one add per element and launch, launches in stream order: the sum has a fixed order
+                                if (a.phi_mode == 2) atomicAdd(p, v); else *p = v;
                             }
                         }
                     // gY: thread <-> (b, edge); the sparse terms of b are the same for the lanes that share it
@@ -479,7 +494,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                                     g = fmaf(t.coef, sGM[t.b * PS + ee], g);
                                 }
                                 float* p = a.gY + (b0 + ee) * a.dsh + b;
-                                *p = a.Y_mode == 2 ? *p + g : g;
+                                if (a.Y_mode == 2) atomicAdd(p, g); else *p = g;
                             }
                         }
                 }
@@ -503,7 +518,7 @@ int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent
     const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP;
     const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
                        (nnz + ninv) * (int)sizeof(NzS) + (dsh + 2) * 4;
-    return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8) * 8 + tables;
+    return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8 + 2 * nunit) * 8 + tables;
 }
 
 }  // namespace
