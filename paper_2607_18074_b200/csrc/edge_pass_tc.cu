@@ -38,9 +38,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int NCW = 8;          // compute warps
-constexpr int NLW = 2;          // loader warps
-constexpr int TT = (NCW + NLW + 1) * 32;
+// Warps of a CTA: NCW = 8 compute warps, NLW loader warps, one MMA warp.  Two loader warps where two CTAs share an SM,
+// three (and the whole register file) where the shared memory of a set leaves room for one CTA only.
 constexpr int NS = 2;           // ring stages
 
 struct EtArgs {
@@ -82,6 +81,7 @@ struct UInfo {     // a unit of the launch's set
 };
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+template <int NCW>
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
 __device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
@@ -92,14 +92,23 @@ __device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void* src, u
 __device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+// the wait for the tensor-memory loads in flight; the loaded registers pass through it so that nothing that reads
+// them can be scheduled ahead of it
+__device__ __forceinline__ void tc_wait_ld16(float* v) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]),
+                   "+f"(v[8]), "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15])
+                 :: "memory");
+}
+__device__ __forceinline__ void tc_ld8_nowait(uint32_t taddr, float* v) {
     uint32_t r[8];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+#pragma unroll
+    for (int i = 8; i < 16; ++i) v[i] = 0.f;
 }
 
 // per-stage raw area (floats): phi rows [tb][KP], (vphi), Y written transposed [dsh][tb+4], (vY), sender ids [tb]
@@ -108,8 +117,10 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
     return n * tb * KP + n * dsh * (tb + 4) + tb;
 }
 
-template <int KP, bool DUAL>
-__global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
+template <int KP, bool DUAL, int NCW, int NLW>
+__global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge_tc(const EtArgs a) {
+    constexpr int TT = (NCW + NLW + 1) * 32;
+    constexpr int NH = NCW / 4;            // column parts of an accumulator tile: one per group of four compute warps
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int NRAW = DUAL ? 2 : 1;     // raw stages: phi and Y, plus their directions
@@ -150,9 +161,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
 
     if (tid == 0) {
         // a stage is released by the commit of the batch's MMAs and by every compute thread (raw rows read)
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 1 + NCW * 32); }
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 2); }
         for (int u = 0; u < a.nunit; ++u) { mbar_init(bar_zfull + 8 * u, NLW * 32); mbar_init(bar_zfree + 8 * u, 1); }
-        for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW * 32); }
+        for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero what is never written later: the raw rows of padded radial components / absent directions, and the
@@ -361,7 +372,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
     } else {
         // =========================== compute warps ===========================
         uint32_t it = 0, ai = 0;
-        const int quarter = warp & 3, half = warp >> 2;
+        const int quarter = warp & 3, half = warp >> 2;      // half: this warp's column part (0 .. NH-1)
         const int row0 = quarter * 32 + lane;        // this thread's accumulator row inside a 128-row tile
         const int e = row0 & (tb - 1);               // its edge (the same in every tile: 128 is a multiple of tb)
         const int t8 = tb >> 3;                      // 8-edge octets per batch
@@ -419,10 +430,10 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                                 *reinterpret_cast<float4*>(sdM + j * PS + o8 + 4) = *reinterpret_cast<const float4*>(dm + 4);
                             }
                         }
-                        // the raw rows of the stage are consumed by this thread (the stage is released when all compute
-                        // threads have said so and the batch's MMAs, which read the sender rows, have retired)
-                        mbar_arrive(bar_free + 8 * st);
-                        compute_sync();     // coupling matrices complete; the previous batch's reductions are done
+                        compute_sync<NCW>();     // coupling matrices complete; the previous batch's reductions are done
+                        // the raw rows of the stage are consumed by every compute thread (the stage is released when
+                        // they are and the batch's MMAs, which read the sender rows, have retired)
+                        if (tid == 0) mbar_arrive(bar_free + 8 * st);
                         // ---- epilogue: this thread owns the accumulator rows (s, e) = (row >> lg, row & (tb-1))
                         int ent_u = 0;                // first entry of the unit inside the set
                         for (int ui = 0; ui < S.nunit; ++ui, ++ai) {
@@ -431,44 +442,69 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                             const uint32_t buf = ai & 1;
                             mbar_wait(bar_accfull + 8 * buf, (ai >> 1) & 1, a.status);
                             tc_fence_after();
-                            const int chalf = ((int)U.ncomp + 1) >> 1;
+                            const int chalf = ((int)U.ncomp + NH - 1) / NH;
                             const int c_lo = half * chalf, c_hi = min((int)U.ncomp, c_lo + chalf);
-                            for (int mt = 0; mt < nmt; ++mt) {
+                            // 16 accumulator columns per TMEM load: two components at KP = 8, one at KP = 16.  The loads
+                            // of a tile whose rows of this warp carry no (s, e) are skipped; the others run one ahead of
+                            // the arithmetic (two register sets).
+                            constexpr int CPL = 16 / KP;
+                            const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
+                            const int ncl = (c_hi - c_lo + CPL - 1) / CPL;       // loads per tile
+                            int nmt_w = 0;                                       // tiles with rows of this warp (a prefix)
+                            for (int mt = 0; mt < nmt; ++mt) if (((mt * 128 + quarter * 32) >> lg) < d_src) nmt_w = mt + 1;
+                            const int nch = ncl > 0 ? ncl * nmt_w : 0;
+                            int mt_i = 0, cl_i = c_lo, mt_p = 0, cl_p = c_lo;      // the next load's and the next use's (tile, component)
+                            auto issue = [&](float* v) {
+                                const int mt = mt_i, cl = cl_i;
+                                cl_i += CPL; if (cl_i >= c_hi) { cl_i = c_lo; ++mt_i; }
+                                const uint32_t ad = t0 + (uint32_t)(mt * npad + cl * KP);
+                                if (cl + CPL <= c_hi) tc_ld16_nowait(ad, v); else tc_ld8_nowait(ad, v);     // warp-uniform
+                            };
+                            auto process = [&](const float* v) {
+                                const int mt = mt_p, cl = cl_p;
+                                cl_p += CPL; if (cl_p >= c_hi) { cl_p = c_lo; ++mt_p; }
                                 const int s = (mt * 128 + row0) >> lg;
-                                const bool rv = s < d_src;
-                                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols;
-                                // 16 accumulator columns per TMEM load: two components at KP = 8, one at KP = 16
-                                constexpr int CPL = 16 / KP;
-                                for (int cl = c_lo; cl < c_hi; cl += CPL) {
-                                    float v[16];
-                                    const bool full = cl + CPL <= c_hi;        // warp-uniform
-                                    if (full) tc_ld16(t0 + (uint32_t)(mt * npad + cl * KP), v);
-                                    else tc_ld8(t0 + (uint32_t)(mt * npad + cl * KP), v);
+                                if (s >= d_src) return;       // rows past the block's (s, e) range hold whatever the tile read
 #pragma unroll
-                                    for (int c2 = 0; c2 < CPL; ++c2) {
-                                        if (c2 > 0 && !full) break;
-                                        const int ent = ent_u + (cl + c2) * d_src + s;
-                                        const float mw = rv ? ((DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e]) : 0.f;
-                                        if (rv) {     // rows past the block's (s, e) range hold whatever the tile read
-                                            float gm = 0.f;
+                                for (int c2 = 0; c2 < CPL; ++c2) {
+                                    if (cl + c2 >= c_hi) break;
+                                    const int ent = ent_u + (cl + c2) * d_src + s;
+                                    const float mw = (DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e];
+                                    float gm = 0.f;
 #pragma unroll
-                                            for (int x = 0; x < KP; ++x) {
-                                                gm = fmaf(aw[x], v[c2 * KP + x], gm);
-                                                pphi[x] = fmaf(mw, v[c2 * KP + x], pphi[x]);
-                                            }
-                                            sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
-                                        }
+                                    for (int x = 0; x < KP; ++x) {
+                                        gm = fmaf(aw[x], v[c2 * KP + x], gm);
+                                        pphi[x] = fmaf(mw, v[c2 * KP + x], pphi[x]);
                                     }
+                                    sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
+                                }
+                            };
+                            float va[16];
+                            if constexpr (NLW == 2) {       // two CTAs per SM: half the registers, one load at a time
+                                for (int ch = 0; ch < nch; ++ch) { issue(va); tc_wait_ld16(va); process(va); }
+                            } else {
+                            float vb[16];
+                            if (nch > 0) issue(va);
+                            for (int ch = 0; ch < nch; ch += 2) {
+                                tc_wait_ld16(va);
+                                if (ch + 1 < nch) issue(vb);
+                                process(va);
+                                if (ch + 1 < nch) {
+                                    tc_wait_ld16(vb);
+                                    if (ch + 2 < nch) issue(va);
+                                    process(vb);
                                 }
                             }
+                            }
                             tc_fence_before();
-                            mbar_arrive(bar_accfree + 8 * buf);
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_accfree + 8 * buf);
                             ent_u += (int)U.ncomp * d_src;
                         }
                     }   // sub-batches
 #pragma unroll
                     for (int q = 0; q < KP; ++q) sPphi[tid * KP + q] = pphi[q];
-                    compute_sync();
+                    compute_sync<NCW>();
                     // ---- fixed-order reductions, written straight to the outputs: every (edge, q) and (edge, b) of the
                     // batch is produced here exactly once per launch (edge id = position in the receiver-sorted order).
                     // The threads that share an edge are those whose row is congruent to it modulo tb, in both column halves.
@@ -477,7 +513,9 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
                             const int ee = i / KP, q = i - ee * KP;
                             if (ee < nb && q < a.K) {
                                 float v = 0.f;
-                                for (int r = ee; r < 128; r += tb) v += sPphi[r * KP + q] + sPphi[(128 + r) * KP + q];
+                                for (int r = ee; r < 128; r += tb)
+#pragma unroll
+                                    for (int h = 0; h < NH; ++h) v += sPphi[(128 * h + r) * KP + q];
                                 float* p = a.gphi + (b0 + ee) * a.K + q;
                                 // one add per element and launch, launches in stream order: the sum has a fixed order
                                 if (a.phi_mode == 2) atomicAdd(p, v); else *p = v;
@@ -512,6 +550,7 @@ __global__ void __launch_bounds__(TT, 2) k_edge_tc(const EtArgs a) {
 
 // shared bytes of a launch
 int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent, int nunit, int ncomp, int nnz, int ninv) {
+    constexpr int NCW = 8;
     const int nop = dual ? 2 : 1;
     const int PS = tb + 4;
     const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
@@ -722,11 +761,14 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
     a.status = status;
     const bool k8 = p->K <= 8;
-    void (*kern)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true> : k_edge_tc<8, false>)
-                                    : (dual ? k_edge_tc<16, true> : k_edge_tc<16, false>);
+    void (*kern2)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 2> : k_edge_tc<8, false, 8, 2>)
+                                     : (dual ? k_edge_tc<16, true, 8, 2> : k_edge_tc<16, false, 8, 2>);
+    void (*kern1)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3> : k_edge_tc<8, false, 8, 3>)
+                                     : (dual ? k_edge_tc<16, true, 8, 3> : k_edge_tc<16, false, 8, 3>);
     int max_smem = 0;
     for (const auto& ep : T.epar) max_smem = std::max(max_smem, ep.smem);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaError_t e = cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (e != cudaSuccess) return e;
     // one launch per set of accumulator tiles: the first writes in the caller's mode, the others accumulate
     for (size_t si = 0; si < T.sets.size(); ++si) {
@@ -741,7 +783,8 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
         a.Y_mode = Y_mode ? (si == 0 ? Y_mode : 2) : 0;
         const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * ep.ctas);
         KernelTimer kt(K_EDGE, s);
-        kern<<<grid, TT, ep.smem, s>>>(a);
+        if (ep.ctas == 2) kern2<<<grid, (8 + 2 + 1) * 32, ep.smem, s>>>(a);
+        else kern1<<<grid, (8 + 3 + 1) * 32, ep.smem, s>>>(a);
         count_launch();
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
