@@ -81,6 +81,13 @@ struct UInfo {     // a unit of the launch's set
 };
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// i / d for the small index ranges of the loaders (0 <= i, i * d < 2^20) by one multiplication: an integer division
+// costs some thirty instructions, which the loader warps cannot hide
+struct SmallDiv {
+    uint32_t m;
+    __device__ __forceinline__ explicit SmallDiv(int d) : m((1u << 20) / (uint32_t)d + 1u) {}
+    __device__ __forceinline__ int operator()(int i) const { return (int)(((uint32_t)i * m) >> 20); }
+};
 template <int NCW>
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
 __device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t bytes) {
@@ -228,6 +235,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     if (zi > 0) mbar_wait(bar_zfree + 8 * ui, (zi - 1) & 1, a.status);
                     const int cpr = (int)U.c_src >> 3;
                     const int n_it = a.K * cpr;
+                    const SmallDiv by_cpr(cpr);
                     for (int cl = warp - NCW; cl < (int)U.ncomp; cl += NLW) {
                         const CompS cp = sComp[U.comp_begin + cl];
                         const int64_t g0 = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff;
@@ -235,7 +243,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                         const __nv_bfloat16* gl = a.zql + g0;
                         const uint32_t d0 = smem_u32(sZ) + U.z_off + (uint32_t)(cl * KP) * 128u;
                         for (int i = lane; i < n_it; i += 32) {
-                            const int q = i / cpr, j = i - q * cpr;
+                            const int q = by_cpr(i), j = i - q * cpr;
                             const int r = cl * KP + q;
                             const uint32_t d = d0 + (uint32_t)((j >> 3) * U.z_kb + q * 128 + (((j & 7) ^ (r & 7)) << 4));
                             cp_async16_zfill(d, gh + 8 * i, 16);
@@ -248,11 +256,12 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
             };
             // ---- the batches of the receiver; the first one is staged ahead of the Zbar slabs (its stage does not wait
             // for the previous receiver's MMAs to end)
-            const int nbat = (int)((seg1 - seg0 + tb - 1) / tb) * nsub;
+            const int nbat = (int)((seg1 - seg0 + tb - 1) >> lg) * nsub;
             for (int bi_ = 0; bi_ < nbat; ++bi_, ++it) {
                 if (bi_ == 1) load_zbar();
-                const int64_t b0 = seg0 + (int64_t)(bi_ / nsub) * tb;
-                const int sb = bi_ - (bi_ / nsub) * nsub;
+                const int bq = nsub == 2 ? bi_ >> 1 : bi_;
+                const int64_t b0 = seg0 + (int64_t)bq * tb;
+                const int sb = bi_ - bq * nsub;
                 const int op = use_x ? sb : 1;
                 const int nb = (int)min((int64_t)tb, seg1 - b0);
                 const int st = (int)(it % NS);
@@ -272,8 +281,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     const bool v16 = (a.K & 3) == 0;
                     const int per = v16 ? a.K / 4 : a.K;
                     const int n_it = tb * per;
+                    const SmallDiv by_per(per);
                     for (int i = lt; i < n_it; i += NLW * 32) {
-                        const int e = i / per, j = i - e * per;
+                        const int e = by_per(i), j = i - e * per;
                         const int64_t ee = b0 + min(e, nb - 1);
                         const uint32_t ok = e < nb ? 1u : 0u;
                         if (v16) {
@@ -288,8 +298,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                 {   // Y (and vY), transposed: raw[b][PS + e]
                     const uint32_t y_u = raw_u + (uint32_t)(NRAW * tb * KP) * 4;
                     const int n_it = tb * a.dsh;
+                    const SmallDiv by_dsh(a.dsh);
                     for (int i = lt; i < n_it; i += NLW * 32) {
-                        const int e = i / a.dsh, b = i - e * a.dsh;
+                        const int e = by_dsh(i), b = i - e * a.dsh;
                         const int64_t ee = b0 + min(e, nb - 1);
                         const uint32_t ok = e < nb ? 4u : 0u;
                         cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
@@ -301,8 +312,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     const TBlk B = sBlk[bi];
                     const int cpr = B.c_src >> 3;
                     const int npair = tb * cpr;
+                    const SmallDiv by_cpr(cpr);
                     for (int pr = lt; pr < npair; pr += NLW * 32) {
-                        const int e = pr / cpr, j = pr - e * cpr;
+                        const int e = by_cpr(pr), j = pr - e * cpr;
                         const int32_t sid = sIds[e];
                         const uint32_t ok = sid >= 0 ? 16u : 0u;
                         const int u = 8 * j;
@@ -404,7 +416,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                         // batch's readers are all past the barrier that follows its epilogue): thread <-> (entry, 8 edges)
                         if (sb == 0)
                         for (int i = tid; i < S.nent * t8; i += NCW * 32) {
-                            const int j = i / t8, o8 = 8 * (i - j * t8);
+                            const int j = i >> (lg - 3), o8 = 8 * (i - j * t8);
                             const EntS en = sEnt[j];
                             float m[8], dm[8];
 #pragma unroll
