@@ -239,6 +239,47 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
                     void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Geometry front end: the edge inputs recomputed from edge vectors inside the edge kernels, and the gradient
+ * that reaches the positions.  The graph inputs Y and phi are edge-sized and "any exact execution must either
+ * store or recompute them" (Section "Memory cost of edge-conditioned convolution"; Table memory_complexity lists
+ * the spherical harmonics as "stored or recomputed").  These entry points recompute them: the caller passes
+ * rvec [E][3], r_e = pos[sender(e)] - pos[receiver(e)] in the receiver-sorted edge order, and no array of width
+ * dim_sh or K per edge exists anywhere.  The backward returns the adjoint of the edge vectors g_rvec [E][3],
+ * from which the forces follow (Eq. energy_force_symmetry; Section "Introduction": energies and forces).
+ *   Y_e    real spherical harmonics of r_e / |r_e|, component normalisation (sum_m Y_lm^2 = 2l+1), no
+ *          Condon-Shortley sign, index l*l + l + m with the sine branch at negative m: the basis the coupling
+ *          tensors of the plan are expressed in.
+ *   phi_e  radial basis of |r_e| (the paper fixes none):
+ *          SOBEK_BASIS_BESSEL    sqrt(2/r_cut) sin(n pi r / r_cut) / r * u(r / r_cut), n = 1..K, with the polynomial
+ *                                envelope u(d) = 1 - (p+1)(p+2)/2 d^p + p(p+2) d^(p+1) - p(p+1)/2 d^(p+2);
+ *          SOBEK_BASIS_GAUSSIAN  exp(-(r - mu_q)^2 / (2 s^2)), mu_q = q s, s = r_cut / (K - 1), q = 0..K-1
+ *                                (envelope_p is ignored).
+ * Every r_e must be non-zero (an edge of length zero has no direction; nothing is checked).
+ * Plans: fully connected or channelwise, ir_mul layout, l_max <= 4, the tensor-core edge kernels in use (the
+ * default where the profile allows them: K <= 16, multiplicities multiples of 16 up to 128); otherwise UNSUPPORTED.
+ * Workspace: sobek_workspace_bytes(plan, N, E, 0) for the forward, (.., 1) for the backward.  Double backward
+ * through the geometry is not provided.  Errors as for sobek_conv_fwd / sobek_conv_bwd.
+ *
+ * sobek_edge_vectors       rvec[e] = pos[col[e]] - pos[receiver(e)]                       (pos [N][3], rvec [E][3])
+ * sobek_conv_geo_fwd       y of sobek_conv_fwd with Y, phi computed from rvec
+ * sobek_conv_geo_bwd       gx, gR as sobek_conv_bwd; g_rvec[e] = J_Y(r_e)^T gY_e + J_phi(r_e)^T gphi_e.  Any of
+ *                          gx, g_rvec, gR may be NULL (gx needs the sender view of the graph)
+ * sobek_position_gradient  gpos[n] = sum_{e: sender(e) = n} g_rvec[e] - sum_{e: receiver(e) = n} g_rvec[e], the
+ *                          adjoint of sobek_edge_vectors (forces are its negative); each node sums its own edges in
+ *                          a fixed order (needs src_ptr and src_perm).  Only enqueues.
+ */
+#define SOBEK_BASIS_BESSEL 0
+#define SOBEK_BASIS_GAUSSIAN 1
+int sobek_edge_vectors(const sobek_graph* g, const float* pos, float* rvec, void* stream);
+int sobek_conv_geo_fwd(const sobek_plan* plan, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                       int envelope_p, const float* x, const float* R, float* y, void* ws, size_t ws_bytes,
+                       void* stream);
+int sobek_conv_geo_bwd(const sobek_plan* plan, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                       int envelope_p, const float* x, const float* R, const float* gy, float* gx, float* g_rvec,
+                       float* gR, void* ws, size_t ws_bytes, void* stream);
+int sobek_position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, void* stream);
+
+/*
  * sobek_conv_fwd_static -- the forward convolution with NO workspace argument and no
  * allocation of any kind (the paper has no counterpart; it exists for hosts of this library
  * that cannot allocate device memory when they run the operator: code running inside another

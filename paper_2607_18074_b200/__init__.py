@@ -11,7 +11,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_uint, c_uint32, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_size_t, c_uint, c_uint32, c_void_p
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsobek.so")
@@ -37,7 +37,9 @@ EXPORTS = [
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
     "sobek_conv_fwd_retain", "sobek_conv_bwd_retained", "sobek_static_last_status", "sobek_measure_fp32_peak",
+    "sobek_edge_vectors", "sobek_conv_geo_fwd", "sobek_conv_geo_bwd", "sobek_position_gradient",
 ]
+BASIS_BESSEL, BASIS_GAUSSIAN = 0, 1
 
 
 class SobekError(RuntimeError):
@@ -96,6 +98,10 @@ def lib():
         L.sobek_conv_dbwd.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 15 + [c_size_t, c_void_p]
         L.sobek_conv_fwd_retain.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 6 + [c_size_t, c_void_p, POINTER(c_int)]
         L.sobek_conv_bwd_retained.argtypes = [c_void_p, POINTER(Graph)] + [c_void_p] * 10 + [c_size_t, c_void_p, c_int]
+        L.sobek_edge_vectors.argtypes = [POINTER(Graph), c_void_p, c_void_p, c_void_p]
+        L.sobek_position_gradient.argtypes = [POINTER(Graph), c_void_p, c_void_p, c_void_p]
+        L.sobek_conv_geo_fwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 4 + [c_size_t, c_void_p]
+        L.sobek_conv_geo_bwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 7 + [c_size_t, c_void_p]
         L.sobek_selftest_wait_timeout.argtypes = [c_void_p, c_uint, c_void_p]
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
         L.sobek_static_scratch_bytes.restype = c_size_t
@@ -280,6 +286,26 @@ def conv_bwd(plan, graph, x, Y, phi, R, gy, gx, gY, gphi, gR, ws):
     _check(lib().sobek_conv_bwd(plan.handle, byref(graph), _ptr(x), _ptr(Y), _ptr(phi), _ptr(R), _ptr(gy),
                                 _ptr(gx), _ptr(gY), _ptr(gphi), _ptr(gR), _ptr(ws),
                                 ws.numel() * ws.element_size(), _stream()), "sobek_conv_bwd")
+
+
+def edge_vectors(graph, pos, rvec):
+    _check(lib().sobek_edge_vectors(byref(graph), _ptr(pos), _ptr(rvec), _stream()), "sobek_edge_vectors")
+
+
+def position_gradient(graph, g_rvec, gpos):
+    _check(lib().sobek_position_gradient(byref(graph), _ptr(g_rvec), _ptr(gpos), _stream()), "sobek_position_gradient")
+
+
+def conv_geo_fwd(plan, graph, rvec, basis, r_cut, envelope_p, x, R, y, ws):
+    _check(lib().sobek_conv_geo_fwd(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
+                                    _ptr(x), _ptr(R), _ptr(y), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "sobek_conv_geo_fwd")
+
+
+def conv_geo_bwd(plan, graph, rvec, basis, r_cut, envelope_p, x, R, gy, gx, g_rvec, gR, ws):
+    _check(lib().sobek_conv_geo_bwd(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
+                                    _ptr(x), _ptr(R), _ptr(gy), _ptr(gx), _ptr(g_rvec), _ptr(gR), _ptr(ws),
+                                    ws.numel() * ws.element_size(), _stream()), "sobek_conv_geo_bwd")
 
 
 def conv_fwd_retain(plan, graph, x, Y, phi, R, y, ws) -> int:

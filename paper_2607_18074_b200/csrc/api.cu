@@ -300,18 +300,25 @@ extern "C" int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_pt
 }
 
 namespace {
+// Geometry mode (Y and phi recomputed from edge vectors inside the edge kernels) exists in the tensor-core edge
+// kernels only: the plan must run them in both directions, unfused, in the ir_mul layout, with l_max <= 4.
+bool geo_supported(const sobek_plan* p, const Workspace& w, int order) {
+    if (!p->use_tc_stream || !p->fwd.tc[0].ok || !w.xsh || w.fused_f || p->mul_ir || p->dim_sh > 25) return false;
+    return order == 0 || (p->tr.tc[0].ok && p->fwd.etc[0].ok && w.gsh && w.zqh && !w.fused_t);
+}
 // `order` is the workspace layout to use (0, or 1 when the state is to be found by a following backward call);
 // *retained is set to 1 when the state of every receiver is left in the workspace (one chunk, state schedule)
 int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
                   const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
-                  void* stream, int order = 0, int* retained = nullptr) {
+                  void* stream, int order = 0, int* retained = nullptr, const SplitSrc* geo = nullptr) {
     if (retained) *retained = 0;
     int rc = check_common(p, g, ws, ws_bytes, order);
     if (rc) return rc;
-    if (!y || !R || (g->N > 0 && !x) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!y || !R || (g->N > 0 && !x) || (g->E > 0 && !geo && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
     if (!aligned16(x, Y, phi, R, y)) return SOBEK_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, order, ws);
+    if (geo && !geo_supported(p, w, 0)) return SOBEK_ERR_UNSUPPORTED;
     CK(cudaMemsetAsync(w.status, 0, kHeaderBytes, s));
     if (g->N == 0) return SOBEK_OK;
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
@@ -324,6 +331,7 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     }
     CK(pack_R(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     SplitSrc xs{};
+    if (geo) xs = *geo;
     if (w.xsh) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
@@ -337,14 +345,16 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
 // z_valid: the workspace still holds the state Z of all receivers, left by conv_fwd_core(order = 1) on the same inputs
 int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
                   const float* phi, const float* R, const float* gy, float* gx, float* gY,
-                  float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream, int z_valid = 0) {
+                  float* gphi, float* gR, void* ws, size_t ws_bytes, void* stream, int z_valid = 0,
+                  const SplitSrc* geo = nullptr) {
     int rc = check_common(p, g, ws, ws_bytes, 1);
     if (rc) return rc;
-    if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && !geo && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
     if (!aligned16(x, Y, phi, R, gy, gx, gY, gphi, gR)) return SOBEK_ERR_INVALID_ARG;
     if (gx && g->E > 0 && (!g->src_ptr || !g->src_perm)) return SOBEK_ERR_NEED_TRANSPOSE;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, 1, ws);
+    if (geo && !geo_supported(p, w, 1)) return SOBEK_ERR_UNSUPPORTED;
     CK(cudaMemsetAsync(w.status, 0, kHeaderBytes, s));
     const int64_t KN = (int64_t)p->K * p->N_w;
     if (g->N == 0 || g->E == 0) {
@@ -354,6 +364,9 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     }
     const EdgeView rv = receiver_view(g);
     SplitSrc xs{}, gs{};
+    if (geo) { xs = *geo; gs = *geo; gs.g_rvec = nullptr; }
+    const bool g_edge = geo && geo->g_rvec;       // geometry mode: the edge pass writes the adjoint of the edge vectors
+    if (g_edge) { gphi = geo->g_rvec; gY = geo->g_rvec; }      // (stand-ins: "wanted"; the kernel writes g_rvec only)
     const bool tc_edge = w.zqh != nullptr;
     if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     if (w.gsh && gx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
@@ -371,8 +384,8 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
             if (gphi || gY) {
                 if (tc_edge) {
                     CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, nullptr, w.status, s, w.zqh, w.zql));
-                    CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql, gphi, gY,
-                                           gphi ? 1 : 0, gY ? 1 : 0, w.status, s));
+                    CK(launch_edge_pass_tc(p, p->fwd, rv, n0, nn, xs, Y, nullptr, phi, nullptr, 0, w.zqh, w.zql,
+                                           g_edge ? nullptr : gphi, g_edge ? nullptr : gY, gphi ? 1 : 0, gY ? 1 : 0, w.status, s));
                 } else {
                     CK(state_adjoint(p, p->fwd, n0, nn, w.gbh, w.gbl, w.fKNh, w.fKNl, gy, R, w.zbar, w.status, s));
                     CK(launch_edge_pass(p, p->fwd, rv, n0, nn, x, nullptr, Y, nullptr, phi, nullptr, 0, w.zbar, gphi, gY,
@@ -602,6 +615,43 @@ extern "C" int sobek_conv_bwd(const sobek_plan* p, const sobek_graph* g, const f
     if ((rc = r.in_x(x, w.lx, &xi)) || (rc = r.in_y(gy, w.lgy, &gyi))) return rc;
     if ((rc = conv_bwd_core(p, g, xi, Y, phi, R, gyi, gx ? w.lgx : nullptr, gY, gphi, gR, ws, ws_bytes, stream))) return rc;
     return r.out_x(w.lgx, gx);
+}
+
+namespace {
+int geo_source(const float* rvec, int basis, float r_cut, int envelope_p, SplitSrc* geo) {
+    if (!rvec || (basis != SOBEK_BASIS_BESSEL && basis != SOBEK_BASIS_GAUSSIAN) || !(r_cut > 0.f) ||
+        (basis == SOBEK_BASIS_BESSEL && (envelope_p < 1 || envelope_p > 16)))
+        return SOBEK_ERR_INVALID_ARG;
+    geo->rvec = rvec; geo->geo_basis = basis; geo->geo_rc = r_cut; geo->geo_p = envelope_p;
+    return SOBEK_OK;
+}
+}  // namespace
+
+extern "C" int sobek_edge_vectors(const sobek_graph* g, const float* pos, float* rvec, void* stream) {
+    return edge_vectors(g, pos, rvec, (cudaStream_t)stream);
+}
+
+extern "C" int sobek_position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, void* stream) {
+    return position_gradient(g, g_rvec, gpos, (cudaStream_t)stream);
+}
+
+extern "C" int sobek_conv_geo_fwd(const sobek_plan* p, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                                  int envelope_p, const float* x, const float* R, float* y, void* ws, size_t ws_bytes,
+                                  void* stream) {
+    SplitSrc geo{};
+    if (g && g->E > 0) { const int rc = geo_source(rvec, basis, r_cut, envelope_p, &geo); if (rc) return rc; }
+    else geo.rvec = rvec ? rvec : reinterpret_cast<const float*>(&geo);      // no edge is read
+    return conv_fwd_core(p, g, x, nullptr, nullptr, R, y, ws, ws_bytes, stream, 0, nullptr, &geo);
+}
+
+extern "C" int sobek_conv_geo_bwd(const sobek_plan* p, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                                  int envelope_p, const float* x, const float* R, const float* gy, float* gx,
+                                  float* g_rvec, float* gR, void* ws, size_t ws_bytes, void* stream) {
+    SplitSrc geo{};
+    if (g && g->E > 0) { const int rc = geo_source(rvec, basis, r_cut, envelope_p, &geo); if (rc) return rc; }
+    else geo.rvec = rvec ? rvec : reinterpret_cast<const float*>(&geo);
+    geo.g_rvec = g_rvec;
+    return conv_bwd_core(p, g, x, nullptr, nullptr, R, gy, gx, nullptr, nullptr, gR, ws, ws_bytes, stream, 0, &geo);
 }
 
 extern "C" int sobek_conv_fwd_retain(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,

@@ -29,6 +29,7 @@
 
 #include <algorithm>
 
+#include "geometry.cuh"
 #include "guard.cuh"
 #include "internal.h"
 #include "ptx.cuh"
@@ -67,6 +68,13 @@ struct EtArgs {
     const __nv_bfloat16* zql;
     float* gphi;
     float* gY;
+    // geometry mode: Y and phi are recomputed from the edge vectors [E][3] (Y, phi are NULL), and the adjoints of
+    // both are contracted with their Jacobians into the adjoint of the edge vectors g_rvec [E][3] (gphi, gY are NULL;
+    // phi_mode = Y_mode = mode of g_rvec)
+    const float* rvec;
+    float* g_rvec;
+    float geo_rc;
+    int32_t geo_basis, geo_p;
     int32_t phi_mode, Y_mode;   // 0 skip, 1 overwrite, 2 accumulate
     int32_t K, dsh, C_src, set;
     int32_t tb, lg;             // edges per batch (power of two) and its log2
@@ -124,7 +132,8 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
     return n * tb * KP + n * dsh * (tb + 4) + tb;
 }
 
-template <int KP, bool DUAL, int NCW, int NLW>
+// GEO: the geometry mode (edge inputs recomputed from edge vectors, adjoint of the edge vectors out); plain pass only
+template <int KP, bool DUAL, int NCW, int NLW, bool GEO>
 __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge_tc(const EtArgs a) {
     constexpr int TT = (NCW + NLW + 1) * 32;
     constexpr int NH = NCW / 4;            // column parts of an accumulator tile: one per group of four compute warps
@@ -141,7 +150,8 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
     float* sdM = sM + (size_t)a.nent * PS;                     // DUAL
     float* sGM = sdM + (DUAL ? (size_t)a.nent * PS : 0);       // [nent][PS]
     float* sPphi = sGM + (size_t)a.nent * PS;                  // [NCW*32][KP]: one row per compute thread
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sPphi + NCW * 32 * KP);
+    float* sGeo = sPphi + NCW * 32 * KP;                       // [tb][KP + dsh]: gphi and gY of the batch (geometry mode)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sGeo + (size_t)tb * (KP + a.dsh));
     // bars: full[NS], free[NS], acc_full[2], acc_free[2], (tmem address), zfull[nunit], zfree[nunit]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * NS + 6);
     UInfo* sU = reinterpret_cast<UInfo*>(bars + 2 * NS + 8 + 2 * a.nunit);     // [nunit]
@@ -277,6 +287,28 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     sIds[e] = sid;
                 }
                 __syncwarp();
+                if constexpr (GEO) {
+                    // recomputed from the edge vectors: thread <-> (edge, share of the radial indices and components)
+                    float* rawf = reinterpret_cast<float*>(stage + 2 * a.x_cap);       // phi rows [tb][KP]
+                    float* yT = rawf + NRAW * tb * KP;                                 // Y transposed [dsh][PS]
+                    const int nsh = max(1, (NLW * 32) >> lg);
+                    const int qw = (a.K + nsh - 1) / nsh, bw = (a.dsh + nsh - 1) / nsh;
+                    for (int i = lt; i < tb * nsh; i += NLW * 32) {
+                        const int e = i & (tb - 1), sh = i >> lg;
+                        const bool okb = e < nb;
+                        float rx = 0.f, ry = 0.f, rz = 1.f;
+                        if (okb) { const float* rp = a.rvec + (b0 + e) * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
+                        const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                        const int q_lo = sh * qw, q_hi = min(a.K, q_lo + qw), b_lo = sh * bw, b_hi = min(a.dsh, b_lo + bw);
+                        geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
+                            if (q >= q_lo && q < q_hi) rawf[e * KP + q] = okb ? f : 0.f;
+                        });
+                        geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
+                            if (b >= b_lo && b < b_hi) yT[b * PS + e] = okb ? yb : 0.f;
+                        });
+                    }
+                    __threadfence_block();       // the stores above are ordered before this thread's arrival on the stage
+                } else {
                 {
                     const bool v16 = (a.K & 3) == 0;
                     const int per = v16 ? a.K / 4 : a.K;
@@ -306,6 +338,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                         cp_async4_zfill(y_u + (uint32_t)(b * PS + e) * 4, a.Y + ee * a.dsh + b, ok);
                         if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + e) * 4, a.vY + ee * a.dsh + b, ok);
                     }
+                }
                 }
                 // sender rows: rows (s, e) of 128 bytes per 64 multiplicities, 128-byte swizzle
                 for (int bi = 0; bi < S.nblk; ++bi) {
@@ -388,6 +421,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
         const int row0 = quarter * 32 + lane;        // this thread's accumulator row inside a 128-row tile
         const int e = row0 & (tb - 1);               // its edge (the same in every tile: 128 is a multiple of tb)
         const int t8 = tb >> 3;                      // 8-edge octets per batch
+        const int GW = KP + a.dsh;                   // row pitch of sGeo
         // bounds of the next receiver, requested one receiver ahead
         int64_t nx0 = 0, nx1 = 0;
         if ((int64_t)blockIdx.x < a.n_nodes) seg_bounds(a.row_ptr, a.node0 + blockIdx.x, a.E, nullptr, nx0, nx1);
@@ -528,6 +562,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                                 for (int r = ee; r < 128; r += tb)
 #pragma unroll
                                     for (int h = 0; h < NH; ++h) v += sPphi[(128 * h + r) * KP + q];
+                                if constexpr (GEO) { sGeo[ee * GW + q] = v; continue; }
                                 float* p = a.gphi + (b0 + ee) * a.K + q;
                                 // one add per element and launch, launches in stream order: the sum has a fixed order
                                 if (a.phi_mode == 2) atomicAdd(p, v); else *p = v;
@@ -543,10 +578,33 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                                     const NzS t = sInv[k];
                                     g = fmaf(t.coef, sGM[t.b * PS + ee], g);
                                 }
+                                if constexpr (GEO) { sGeo[ee * GW + KP + b] = g; continue; }
                                 float* p = a.gY + (b0 + ee) * a.dsh + b;
                                 if (a.Y_mode == 2) atomicAdd(p, g); else *p = g;
                             }
                         }
+                    // geometry mode: g_r = (sum_q gphi_q dphi_q/dr) u + (I - u u^T) (sum_b gY_b grad F_b) / |r|, one thread per edge
+                    if constexpr (GEO) {
+                        compute_sync<NCW>();
+                        for (int ee = tid; ee < nb; ee += NCW * 32) {
+                            const float* rp = a.rvec + (b0 + ee) * 3;
+                            const float rx = __ldg(rp), ry = __ldg(rp + 1), rz = __ldg(rp + 2);
+                            const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                            const float ux = rx * ir, uy = ry * ir, uz = rz * ir;
+                            const float* ge = sGeo + ee * GW;
+                            float gr = 0.f, Gx = 0.f, Gy = 0.f, Gz = 0.f;
+                            geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float, float df) { gr = fmaf(ge[q], df, gr); });
+                            const int dsh = a.dsh;
+                            geo_sh(ux, uy, uz, [&](int b, float, float fx, float fy, float fz) {
+                                if (b < dsh) { const float w = ge[KP + b]; Gx = fmaf(w, fx, Gx); Gy = fmaf(w, fy, Gy); Gz = fmaf(w, fz, Gz); }
+                            });
+                            const float un = ux * Gx + uy * Gy + uz * Gz;
+                            const float o0 = gr * ux + (Gx - un * ux) * ir, o1 = gr * uy + (Gy - un * uy) * ir, o2 = gr * uz + (Gz - un * uz) * ir;
+                            float* p = a.g_rvec + (b0 + ee) * 3;
+                            if (a.phi_mode == 2) { atomicAdd(p, o0); atomicAdd(p + 1, o1); atomicAdd(p + 2, o2); }
+                            else { p[0] = o0; p[1] = o1; p[2] = o2; }
+                        }
+                    }
                 }
             }
         }
@@ -566,7 +624,7 @@ int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent
     const int nop = dual ? 2 : 1;
     const int PS = tb + 4;
     const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
-    const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP;
+    const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)tb * (KP + dsh);
     const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
                        (nnz + ninv) * (int)sizeof(NzS) + (dsh + 2) * 4;
     return 1024 + NS * stage + 2 * z_cap + (int)(meta * 4) + (2 * NS + 8 + 2 * nunit) * 8 + tables;
@@ -770,13 +828,19 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.zqh = (const __nv_bfloat16*)zqh; a.zql = (const __nv_bfloat16*)zql;
     a.gphi = gphi; a.gY = gY;
+    a.rvec = ss.rvec; a.g_rvec = ss.g_rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
     a.status = status;
     const bool k8 = p->K <= 8;
-    void (*kern2)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 2> : k_edge_tc<8, false, 8, 2>)
-                                     : (dual ? k_edge_tc<16, true, 8, 2> : k_edge_tc<16, false, 8, 2>);
-    void (*kern1)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3> : k_edge_tc<8, false, 8, 3>)
-                                     : (dual ? k_edge_tc<16, true, 8, 3> : k_edge_tc<16, false, 8, 3>);
+    if (ss.rvec && dual) return cudaErrorNotSupported;
+    void (*kern2)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 2, false> : k_edge_tc<8, false, 8, 2, false>)
+                                     : (dual ? k_edge_tc<16, true, 8, 2, false> : k_edge_tc<16, false, 8, 2, false>);
+    void (*kern1)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3, false> : k_edge_tc<8, false, 8, 3, false>)
+                                     : (dual ? k_edge_tc<16, true, 8, 3, false> : k_edge_tc<16, false, 8, 3, false>);
+    if (ss.rvec) {
+        kern2 = k8 ? k_edge_tc<8, false, 8, 2, true> : k_edge_tc<16, false, 8, 2, true>;
+        kern1 = k8 ? k_edge_tc<8, false, 8, 3, true> : k_edge_tc<16, false, 8, 3, true>;
+    }
     int max_smem = 0;
     for (const auto& ep : T.epar) max_smem = std::max(max_smem, ep.smem);
     cudaError_t e = cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);

@@ -64,6 +64,7 @@ cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeV
     // tensor-core stream when the profile allows it and the caller made the bf16 copies of the sources
     if (p->use_tc_stream && dir.tc[dual ? 1 : 0].ok && status && ss.h && ss.l && (!vsrc || (ss.vh && ss.vl)))
         return launch_stream_tc(p, dir, ev, node0, n_nodes, ss, Y, vY, phi, vphi, dual, zh, zl, status, s);
+    if (ss.rvec) return cudaErrorNotSupported;      // the geometry mode exists in the tensor-core kernels only
     const int KC = p->K <= 8 ? 8 : 16;
     StreamArgsHost a{};
     a.tasks = dir.d_stasks; a.comps = dir.d_scomps;

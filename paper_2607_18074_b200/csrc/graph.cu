@@ -192,4 +192,60 @@ int graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t*
     return SOBEK_OK;
 }
 
+namespace {
+// rvec[e] = pos[sender(e)] - pos[receiver(e)]: one warp per receiver walks its edge segment
+__global__ void k_edge_vectors(int64_t N, int64_t E, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                               const float* __restrict__ pos, float* __restrict__ rvec) {
+    const int lane = threadIdx.x & 31;
+    const int64_t w0 = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5, nw = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t n = w0; n < N; n += nw) {
+        const int64_t s0 = max((int64_t)0, min(row_ptr[n], E)), s1 = max(s0, min(row_ptr[n + 1], E));
+        const float px = pos[3 * n], py = pos[3 * n + 1], pz = pos[3 * n + 2];
+        for (int64_t e = s0 + lane; e < s1; e += 32) {
+            const int64_t j = col[e];
+            const bool ok = j >= 0 && j < N;      // an id out of range leaves a unit vector (and shows up in the conv calls)
+            rvec[3 * e] = ok ? pos[3 * j] - px : 0.f;
+            rvec[3 * e + 1] = ok ? pos[3 * j + 1] - py : 0.f;
+            rvec[3 * e + 2] = ok ? pos[3 * j + 2] - pz : 1.f;
+        }
+    }
+}
+// gpos[n] = sum over the edges n sends (sender view, in its order) - sum over the edges n receives (in edge order):
+// one thread per node, so that every sum has a fixed order
+__global__ void k_position_gradient(int64_t N, int64_t E, const int64_t* __restrict__ row_ptr, const int64_t* __restrict__ src_ptr,
+                                    const int32_t* __restrict__ src_perm, const float* __restrict__ g, float* __restrict__ gpos) {
+    for (int64_t n = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; n < N; n += (int64_t)gridDim.x * blockDim.x) {
+        float ax = 0.f, ay = 0.f, az = 0.f;
+        const int64_t p0 = max((int64_t)0, min(src_ptr[n], E)), p1 = max(p0, min(src_ptr[n + 1], E));
+        for (int64_t p = p0; p < p1; ++p) {
+            const int64_t e = src_perm[p];
+            if (e >= 0 && e < E) { ax += g[3 * e]; ay += g[3 * e + 1]; az += g[3 * e + 2]; }
+        }
+        const int64_t s0 = max((int64_t)0, min(row_ptr[n], E)), s1 = max(s0, min(row_ptr[n + 1], E));
+        for (int64_t e = s0; e < s1; ++e) { ax -= g[3 * e]; ay -= g[3 * e + 1]; az -= g[3 * e + 2]; }
+        gpos[3 * n] = ax; gpos[3 * n + 1] = ay; gpos[3 * n + 2] = az;
+    }
+}
+}  // namespace
+
+int edge_vectors(const sobek_graph* g, const float* pos, float* rvec, cudaStream_t s) {
+    if (!g || g->N < 0 || g->E < 0 || (g->E > 0 && (!g->row_ptr || !g->col || !pos || !rvec))) return SOBEK_ERR_INVALID_ARG;
+    if (g->E == 0) return SOBEK_OK;
+    const int grid = (int)std::min<int64_t>((g->N + 7) / 8, 148 * 16);
+    k_edge_vectors<<<grid, 256, 0, s>>>(g->N, g->E, g->row_ptr, g->col, pos, rvec);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SOBEK_OK : SOBEK_ERR_CUDA;
+}
+
+int position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, cudaStream_t s) {
+    if (!g || g->N < 0 || g->E < 0 || (g->N > 0 && !gpos) || (g->E > 0 && (!g->row_ptr || !g_rvec))) return SOBEK_ERR_INVALID_ARG;
+    if (g->E > 0 && (!g->src_ptr || !g->src_perm)) return SOBEK_ERR_NEED_TRANSPOSE;
+    if (g->N == 0) return SOBEK_OK;
+    if (g->E == 0) return cudaMemsetAsync(gpos, 0, (size_t)g->N * 12, s) == cudaSuccess ? SOBEK_OK : SOBEK_ERR_CUDA;
+    const int grid = (int)std::min<int64_t>((g->N + 127) / 128, 148 * 16);
+    k_position_gradient<<<grid, 128, 0, s>>>(g->N, g->E, g->row_ptr, g->src_ptr, g->src_perm, g_rvec, gpos);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SOBEK_OK : SOBEK_ERR_CUDA;
+}
+
 }  // namespace sobek

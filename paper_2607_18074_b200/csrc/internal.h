@@ -330,6 +330,12 @@ struct SplitSrc {
     const void* l = nullptr;
     const void* vh = nullptr;   // the same for the source direction of the dual stream (NULL without it)
     const void* vl = nullptr;
+    // geometry mode of the tensor-core edge kernels: edge vectors [E][3] from which Y and phi are recomputed (the Y and
+    // phi arguments are NULL then), and where the edge pass puts the adjoint of the edge vectors instead of gY, gphi
+    const float* rvec = nullptr;
+    float geo_rc = 0.f;
+    int geo_basis = 0, geo_p = 6;
+    float* g_rvec = nullptr;
 };
 cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
                           int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,
@@ -428,6 +434,8 @@ constexpr int kMaxSplitsUvu = 256;                             // node slices of
 size_t graph_prepare_bytes(int64_t N, int64_t E);
 int graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* src_perm, int32_t* src_recv,
                     cudaStream_t s);
+int edge_vectors(const sobek_graph* g, const float* pos, float* rvec, cudaStream_t s);
+int position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, cudaStream_t s);
 int graph_prepare(int64_t N, int64_t E, const int64_t* row_ptr, const int32_t* col, int64_t* src_ptr,
                   int32_t* src_perm, void* ws, size_t ws_bytes, cudaStream_t s);
 

@@ -43,6 +43,7 @@
 
 #include <algorithm>
 
+#include "geometry.cuh"
 #include "guard.cuh"
 #include "internal.h"
 #include "ptx.cuh"
@@ -85,6 +86,9 @@ struct TcArgs {
     const float* vY;
     const float* phi;
     const float* vphi;
+    const float* rvec;     // edge vectors [E][3]: when set, Y and phi are recomputed from them (Y, phi are NULL then)
+    float geo_rc;          // cutoff radius of the radial basis
+    int32_t geo_basis, geo_p;
     __nv_bfloat16* zh;
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
@@ -327,6 +331,26 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             if (round > 0) mbar_wait(bar_sfree + 8 * st, (round & 1) ^ 1, a.status);
             const uint32_t stage_u = smem_u32(sRing + (size_t)st * stage_bytes);
             const uint32_t raw_u = stage_u + (uint32_t)(2 * a.b_cap);
+            const int le = lane & (TB - 1);
+            const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
+            if (a.rvec) {
+                // recomputed from the edge vector: thread <-> (edge le, share g8 of the components and radial indices)
+                const int g8 = lt >> 4;
+                const bool okb = (msk >> le) & 1u;
+                float rx = 0.f, ry = 0.f, rz = 1.f;
+                if (okb) { const float* rp = a.rvec + ee_own * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
+                const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                float* rawf = reinterpret_cast<float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.b_cap);
+                float* yT = rawf + NRAW * TB * KP;
+                geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
+                    if ((q & 7) == g8) rawf[le * KP + q] = okb ? f : 0.f;
+                });
+                const int dsh = a.dsh;
+                geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
+                    if (b < dsh && (b & 7) == g8) yT[b * PS + le] = okb ? yb : 0.f;
+                });
+                __threadfence_block();       // the stores above are ordered before this thread's arrival on the stage
+            } else {
             // phi (and vphi) rows: raw[e][KP]   (all lanes run every iteration: the loops hold shuffles)
             {
                 const bool v16 = (a.K & 3) == 0;
@@ -349,8 +373,6 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                 }
             }
             // Y (and vY), transposed: raw[b][PS + e].  Thread <-> (edge e = lane mod 16, b = lt / 16, + 8, ...)
-            const int le = lane & (TB - 1);
-            const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
             {
                 const uint32_t y_u = raw_u + (uint32_t)(NRAW * TB * KP) * 4;
                 const uint32_t ok = ((msk >> le) & 1u) * 4u;
@@ -360,6 +382,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                     cp_async4_zfill(y_u + (uint32_t)(b * PS + le) * 4, yr + b, ok);
                     if (has_vY) cp_async4_zfill(y_u + (uint32_t)(a.dsh * PS + b * PS + le) * 4, vyr + b, ok);
                 }
+            }
             }
             // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy
             {
@@ -859,6 +882,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
+    a.rvec = ss.rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
     a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages;

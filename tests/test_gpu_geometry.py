@@ -1,0 +1,150 @@
+"""GPU parity of the geometry front end (Y and phi recomputed from edge vectors inside the edge kernels; the
+adjoint of the edge vectors and of the positions) against the fp64 geometry oracle, through the C ABI.
+Tolerances as for the convolution: forward 1e-4 * max|ref|, backward 5e-4 * max|ref|."""
+import numpy as np
+import pytest
+
+from oracle import geometry
+from tests.gpu_util import BWD_TOL, FWD_TOL, Case, rel_err
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+P = synth.parse_irreps
+
+
+def _cases():
+    c = {}
+    c["cfg2_N200"] = synth.scaled(synth.config("cfg2"), 200)
+    c["cfg3_N120"] = synth.scaled(synth.config("cfg3"), 120)
+    c["cfg4_N150"] = synth.scaled(synth.config("cfg4"), 150)           # K = 16
+    c["cfg5_N60"] = synth.scaled(synth.config("cfg5"), 60)             # l_max = 4, several sets per launch
+    c["tc_K6_dense"] = synth.Workload("tc_K6_dense", P("16x0e+16x1o"), P("16x0e+16x1o+16x2e"), 2, 6, 160, 4.0, 3.6,
+                                      "bessel", seed=5)                 # K not a multiple of 4, ~100 edges per receiver
+    c["gauss_K12"] = synth.Workload("gauss_K12", P("48x0e+16x1o+16x2e"), P("16x0e+48x1o"), 2, 12, 70, 4.0, 2.2,
+                                    "gaussian", seed=6)
+    return c
+
+
+CASES = _cases()
+
+
+class GeoCase(Case):
+    def __init__(self, w, **kw):
+        super().__init__(w, **kw)
+        import torch
+        d = self.d
+        self.basis = geometry.BESSEL if w.basis == "bessel" else geometry.GAUSSIAN
+        self.pos = torch.from_numpy(np.ascontiguousarray(d.pos, dtype=np.float32)).to("cuda:0")
+        self.rvec = self._new(self.E, 3)
+        self.sb.edge_vectors(self.graph, self.pos, self.rvec)
+        # the oracle starts from the same fp32 positions
+        self.o_rvec = geometry.edge_vectors(d.col, d.recv, self.pos.cpu().numpy().astype(np.float64))
+
+    def geo_fwd(self):
+        y = self._new(self.N, self.plan.info.C_y)
+        self.sb.conv_geo_fwd(self.plan, self.graph, self.rvec, self.basis, self.w.r_c, 6, self.x, self.R, y, self.ws(0))
+        assert self.sb.last_device_status(self.ws(0)) == 0
+        return y.cpu().numpy()
+
+    def geo_bwd(self, want=(True, True, True)):
+        i = self.plan.info
+        gx, g_rv, gR = self._new(self.N, i.C_x), self._new(self.E, 3), self._new(i.K, i.N_w)
+        out = [t if on else None for t, on in zip((gx, g_rv, gR), want)]
+        self.sb.conv_geo_bwd(self.plan, self.graph, self.rvec, self.basis, self.w.r_c, 6, self.x, self.R, self.gy,
+                             *out, self.ws(1))
+        assert self.sb.last_device_status(self.ws(1)) == 0
+        return [None if t is None else t.cpu().numpy() for t in out]
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_edge_vectors_and_forward(name):
+    c = GeoCase(CASES[name])
+    d = c.d
+    assert np.abs(c.rvec.cpu().numpy() - c.o_rvec).max() < 1e-6
+    y = c.geo_fwd()
+    ref = geometry.geo_fwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, c.w.r_c, c.basis)
+    assert np.isfinite(y).all() and np.abs(ref).max() > 1e-3
+    assert rel_err(y, ref) <= FWD_TOL
+    # and it is the stored-input forward on the same geometry (both within tolerance of the oracle)
+    assert rel_err(y, c.fwd()) <= 2 * FWD_TOL
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_backward_and_position_gradient(name):
+    c = GeoCase(CASES[name])
+    d = c.d
+    gx, g_rv, gR = c.geo_bwd()
+    rx, r_rv, rR = geometry.geo_bwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, d.gy, c.w.r_c, c.basis)
+    assert all(np.isfinite(a).all() for a in (gx, g_rv, gR))
+    assert rel_err(gx, rx) <= BWD_TOL and rel_err(gR, rR) <= BWD_TOL
+    assert np.abs(r_rv).max() > 1e-3 and rel_err(g_rv, r_rv) <= BWD_TOL
+    # positions: the fixed-order segment sums against numpy's scatter of the oracle's edge gradient
+    import torch
+    gpos = c._new(c.N, 3)
+    c.sb.position_gradient(c.graph, torch.from_numpy(r_rv.astype(np.float32)).to("cuda:0"), gpos)
+    ref = geometry.position_gradient(d.col, d.recv, r_rv, c.N)
+    assert rel_err(gpos.cpu().numpy(), ref) <= 1e-5
+    # bitwise the same on a second run (every sum has a fixed order)
+    again = c.geo_bwd()
+    assert all(np.array_equal(a, b) for a, b in zip((gx, g_rv, gR), again))
+
+
+def test_partial_outputs_and_argument_errors():
+    c = GeoCase(CASES["cfg3_N120"])
+    full = c.geo_bwd()
+    for want in [(True, False, False), (False, True, False), (False, False, True), (True, True, False)]:
+        got = c.geo_bwd(want)
+        for a, b, on in zip(got, full, want):
+            assert (a is None) == (not on)
+            if on:
+                assert np.array_equal(a, b)
+    sb = c.sb
+    y = c._new(c.N, c.plan.info.C_y)
+    for bad in [dict(basis=7), dict(r_cut=0.0), dict(p=0)]:
+        with pytest.raises(sb.SobekError) as e:
+            sb.conv_geo_fwd(c.plan, c.graph, c.rvec, bad.get("basis", 0), bad.get("r_cut", 1.0), bad.get("p", 6),
+                            c.x, c.R, y, c.ws(0))
+        assert e.value.code == -1
+    with pytest.raises(sb.SobekError) as e:
+        sb.conv_geo_fwd(c.plan, c.graph, None, 0, 1.0, 6, c.x, c.R, y, c.ws(0))
+    assert e.value.code == -1
+    # a plan that runs the FP32-pipe edge kernels has no geometry mode
+    c2 = GeoCase(CASES["cfg3_N120"], tc_stream=False)
+    with pytest.raises(sb.SobekError) as e:
+        c2.geo_fwd()
+    assert e.value.code == -2
+
+
+def test_forces_rotate_with_the_positions():
+    """Eq. energy_force_symmetry on the GPU path: the energy sum_i a . y_i[scalars] of invariant features is unchanged
+    by a rotation of the positions and the forces rotate with them."""
+    import torch
+    w = CASES["cfg3_N120"]
+    c = GeoCase(w)
+    i = c.plan.info
+    n0 = sum(m for m, l, p in w.irreps_out if l == 0)
+    c0 = sum(m for m, l, p in w.irreps_in if l == 0)
+    c.x[:, c0:] = 0
+    a = torch.randn(n0, generator=torch.Generator().manual_seed(1)).to("cuda:0")
+    c.gy.zero_(); c.gy[:, :n0] = a[None, :]
+
+    def energy_forces(pos):
+        c.sb.edge_vectors(c.graph, pos, c.rvec)
+        y = torch.from_numpy(c.geo_fwd()).to("cuda:0")
+        _, g_rv, _ = c.geo_bwd((False, True, False))
+        gpos = c._new(c.N, 3)
+        c.sb.position_gradient(c.graph, torch.from_numpy(g_rv).to("cuda:0"), gpos)
+        return float((y * c.gy).sum()), -gpos.cpu().numpy()
+
+    E0, F0 = energy_forces(c.pos)
+    q = np.random.default_rng(3).standard_normal(4); q /= np.linalg.norm(q)
+    a_, b_, c_, d_ = q
+    Rm = np.array([[a_*a_+b_*b_-c_*c_-d_*d_, 2*(b_*c_-a_*d_), 2*(b_*d_+a_*c_)],
+                   [2*(b_*c_+a_*d_), a_*a_-b_*b_+c_*c_-d_*d_, 2*(c_*d_-a_*b_)],
+                   [2*(b_*d_-a_*c_), 2*(c_*d_+a_*b_), a_*a_-b_*b_-c_*c_+d_*d_]], dtype=np.float32)
+    E1, F1 = energy_forces(c.pos @ torch.from_numpy(Rm.T.copy()).to("cuda:0"))
+    scale = np.abs(F0).max()
+    assert scale > 1e-3
+    assert abs(E1 - E0) <= 1e-4 * max(1.0, abs(E0))
+    assert np.abs(F1 - F0 @ Rm.T).max() <= 1e-3 * scale
+    assert np.abs(F0.sum(0)).max() <= 1e-3 * scale * np.sqrt(c.N)
