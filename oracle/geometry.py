@@ -98,18 +98,19 @@ def position_gradient(col, recv, g_rvec, N: int):
     return g
 
 
-def geo_fwd(orc, row_ptr, col, rvec, x, R, r_c: float, basis: int = BESSEL, p: int = 6):
-    """y of the convolution with Y, phi recomputed from the edge vectors; `orc` is a conv.Oracle."""
+def geo_fwd(orc, row_ptr, col, rvec, x, R, r_c: float, basis: int = BESSEL, p: int = 6, act=None):
+    """y of the convolution with Y, phi recomputed from the edge vectors; `orc` is a conv.Oracle, `act` an optional
+    subset of receivers (as in conv.Oracle.fwd)."""
     Y, phi = edge_inputs(rvec, orc.l_max, orc.K, r_c, basis, p)
-    return orc.fwd(row_ptr, col, x, Y, phi, R)
+    return orc.fwd(row_ptr, col, x, Y, phi, R, act=act)
 
 
-def geo_bwd(orc, row_ptr, col, rvec, x, R, gy, r_c: float, basis: int = BESSEL, p: int = 6):
+def geo_bwd(orc, row_ptr, col, rvec, x, R, gy, r_c: float, basis: int = BESSEL, p: int = 6, act=None):
     """(gx, g_rvec, gR): adjoints of geo_fwd.  g_rvec[e] = J_Y(r_e)^T gY_e + J_phi(r_e)^T gphi_e."""
     t = torch.as_tensor(np.asarray(rvec, dtype=np.float64)).clone().requires_grad_(True)
     Y = real_sh(t, orc.l_max)
     phi = radial(torch.linalg.norm(t, dim=-1), orc.K, r_c, basis, p)
-    gx, gY, gphi, gR = orc.bwd(row_ptr, col, x, Y.detach().numpy(), phi.detach().numpy(), R, gy)
+    gx, gY, gphi, gR = orc.bwd(row_ptr, col, x, Y.detach().numpy(), phi.detach().numpy(), R, gy, act=act)
     s = (Y * torch.as_tensor(gY)).sum() + (phi * torch.as_tensor(gphi)).sum()
     (g_rvec,) = torch.autograd.grad(s, t)
     return gx, g_rvec.numpy(), gR

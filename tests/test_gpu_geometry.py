@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from oracle import geometry
-from tests.gpu_util import BWD_TOL, FWD_TOL, Case, rel_err
+from gpu_util import BWD_TOL, FWD_TOL, Case, rel_err
 from workloads import synth
 
 pytestmark = pytest.mark.gpu
@@ -87,6 +87,33 @@ def test_backward_and_position_gradient(name):
     # bitwise the same on a second run (every sum has a fixed order)
     again = c.geo_bwd()
     assert all(np.array_equal(a, b) for a, b in zip((gx, g_rv, gR), again))
+
+
+FULL = {"cfg3": (synth.config("cfg3"), 6), "cfg4_1e6": (synth.config("cfg4", edges=1e6), 8), "cfg5": (synth.config("cfg5"), 3)}
+
+
+@pytest.mark.parametrize("name", list(FULL))
+def test_full_size_sampled(name):
+    """The benchmark configurations at full size: sampled receivers (first, last and some between, so that several
+    chunks are hit) against the oracle, output adjoint zero outside the sample."""
+    w, n_sample = FULL[name]
+    c = GeoCase(w)
+    d = c.d
+    act = np.sort(np.random.default_rng(123).choice(c.N, size=n_sample, replace=False))
+    act[0], act[-1] = 0, c.N - 1
+    act = np.unique(act)
+    ed = c.edges_into(act)
+    y = c.geo_fwd()
+    ref = geometry.geo_fwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, w.r_c, c.basis, act=act)
+    assert np.isfinite(y).all() and rel_err(y[act], ref[act]) <= FWD_TOL
+    c.gy = c.masked_gy(act)
+    gx, g_rv, gR = c.geo_bwd()
+    gym = c.gy.cpu().numpy().astype(np.float64)
+    rx, r_rv, rR = geometry.geo_bwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, gym, w.r_c, c.basis, act=act)
+    assert rel_err(gx, rx) <= BWD_TOL and rel_err(gR, rR) <= BWD_TOL
+    assert rel_err(g_rv[ed], r_rv[ed]) <= BWD_TOL
+    mask = np.ones(c.E, dtype=bool); mask[ed] = False
+    assert np.all(g_rv[mask] == 0)
 
 
 def test_partial_outputs_and_argument_errors():
