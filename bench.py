@@ -35,10 +35,16 @@ L2_FLUSH_BYTES = 512 << 20
 
 DTYPE = "f32 storage; products as split bf16 x3 (hi*hi + lo*hi + hi*lo) with f32 accumulation (tcgen05)"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel class, measured with ncu
-# on the named workload.  A capture on a scaled-down graph of the same profile is stored per edge and multiplied by
-# the edges of a launch (the traffic of these kernels grows in proportion to the edges).
-NCU_TRAFFIC_BYTES_PER_EDGE = {}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of an edge-kernel class, measured with
+# ncu on the named profile at 20,000 nodes and stored per edge of the launch (a launch of these classes processes
+# the edges of one node chunk once; its traffic grows in proportion to them).  At this profile the stream's figure is
+# the state of the chunk written once (0.92 MB per node as bf16 hi + lo, i.e. 23 KB per edge at 40 edges per node)
+# plus the gathered sender rows.
+NCU_TRAFFIC_BYTES_PER_EDGE = {
+    ("cfg5", "edge_stream_state"): (695.1e6 + 2081.8e6) / 90891.0,     # k_stream_tc, two launches
+    ("cfg5", "edge_pass"): (255.4e6 + 12.8e6) / 90891.0,                # k_edge_tc, three launches
+}
+STREAM_CALLS_PER_STEP = 7      # edge-stream passes over all edges per step: 1 fwd + 2 bwd + 4 dbwd
 
 
 def measured_peaks():
@@ -399,6 +405,36 @@ def main():
             ms.append(a.elapsed_time(b))
         bwd_retained_ms = (float(np.median(ms[1:])), int(kept))
 
+    # ---- geometry front end (extra figure, not part of the step): the same forward and backward with Y and phi
+    # recomputed from the edge vectors inside the edge kernels; outputs gx, the edge-vector adjoint and gR
+    geo = None
+    if world == 1 and w.mode == "uvw":
+        try:
+            pos = torch.from_numpy(np.ascontiguousarray(r.d.pos, dtype=np.float32)).to(dev)
+            rvec, g_rv = torch.empty(E, 3, device=dev), torch.empty(E, 3, device=dev)
+            sb.edge_vectors(g, pos, rvec)
+            basis = sb.BASIS_BESSEL if w.basis == "bessel" else sb.BASIS_GAUSSIAN
+            calls = (lambda: sb.conv_geo_fwd(plan, g, rvec, basis, w.r_c, 6, t["x"], t["R"], out["y"], ws),
+                     lambda: sb.conv_geo_bwd(plan, g, rvec, basis, w.r_c, 6, t["x"], t["R"], t["gy"], out["gx"], g_rv,
+                                             out["gR"], ws))
+            geo_ms = []
+            for f in calls:
+                ms = []
+                for _ in range(4):
+                    flush.fill_(1)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(); f(); b.record()
+                    torch.cuda.synchronize(dev)
+                    ms.append(a.elapsed_time(b))
+                geo_ms.append(float(np.median(ms[1:])))
+            assert sb.last_device_status(ws) == 0
+            geo = {"fwd_edges_per_s": E / (geo_ms[0] * 1e-3), "bwd_edges_per_s": E / (geo_ms[1] * 1e-3),
+                   "fwd_ms": geo_ms[0], "bwd_ms": geo_ms[1], "edge_input_bytes_per_edge": 12,
+                   "stored_edge_input_bytes_per_edge": 4 * (i.dim_sh + i.K)}
+            del pos, rvec, g_rv
+        except sb.SobekError as e:       # profiles without the tensor-core edge kernels have no geometry mode
+            geo = {"unavailable": str(e)}
+
     # ---- end to end: host buffers in, host buffers out ---------------------------------
     # Every step copies all of its inputs from pinned host memory and all of its outputs back, through the public
     # API.  Where device memory allows a second set of input / output buffers, the copies run on two copy streams
@@ -481,7 +517,9 @@ def main():
     alu_derived = FP32_FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12       # TFLOP/s at max clock
     alu_peak = fp32_peak if fp32_peak else alu_derived
     traffic_pe = NCU_TRAFFIC_BYTES_PER_EDGE.get((w.name.split("_N")[0], dom))
-    traffic = None if traffic_pe is None else traffic_pe * E
+    # edges of one launch = edges of one node chunk = E / chunks, chunks = stream launches per pass over the edges
+    n_chunks = max(1.0, classes["edge_stream_state"][1] / steps_timed / STREAM_CALLS_PER_STEP) if "edge_stream_state" in classes else 1.0
+    traffic = None if traffic_pe is None else traffic_pe * E / n_chunks
     if dom == "node_gemm":
         # the node contractions stream the bounded state once per pass (4 bytes per state element as bf16
         # hi + lo, read or written): HBM-bound; passes per step: 8 over the receiver state, 3 over the sender state
@@ -531,6 +569,7 @@ def main():
                 "copies": "double-buffered on two copy streams" if pipelined else "serial"},
         "bwd_after_retaining_fwd": None if bwd_retained_ms is None else {
             "edges_per_s": E_total / (bwd_retained_ms[0] * 1e-3), "ms": bwd_retained_ms[0], "state_retained": bwd_retained_ms[1]},
+        "geometry_front_end": geo,
         "gpu_launches": int(launches),
         "wall_s_timed_region": wall,
         "peak_bytes": {"total": int(peak_bytes), "inputs_and_graph": int(r.in_bytes), "outputs": int(r.out_bytes),

@@ -39,8 +39,9 @@ namespace {
 
 using namespace ptx;
 
-// Warps of a CTA: NCW = 8 compute warps, NLW loader warps, one MMA warp.  Two loader warps where two CTAs share an SM,
-// three (and the whole register file) where the shared memory of a set leaves room for one CTA only.
+// Warps of a CTA: NCW = 8 compute warps, NLW = 3 loader warps, one MMA warp (twelve warps: registers are handed out as
+// if a CTA had a multiple of four warps, so the third loader warp is free).  MINB = CTAs per SM the kernel is compiled
+// for: 2 where the shared memory of a set allows it, else 1 with the whole register file.
 constexpr int NS = 2;           // ring stages
 
 struct EtArgs {
@@ -133,9 +134,11 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
 }
 
 // GEO: the geometry mode (edge inputs recomputed from edge vectors, adjoint of the edge vectors out); plain pass only
-template <int KP, bool DUAL, int NCW, int NLW, bool GEO>
-__global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge_tc(const EtArgs a) {
+template <int KP, bool DUAL, int NCW, int NLW, bool GEO, int MINB>
+__global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const EtArgs a) {
     constexpr int TT = (NCW + NLW + 1) * 32;
+    // geometry mode: the last loader warp does not copy but recomputes phi and Y of every batch from the edge vectors
+    constexpr int NLG = GEO ? NLW - 1 : NLW;
     constexpr int NH = NCW / 4;            // column parts of an accumulator tile: one per group of four compute warps
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -179,7 +182,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
     if (tid == 0) {
         // a stage is released by the commit of the batch's MMAs and by every compute thread (raw rows read)
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_free + 8 * s, 2); }
-        for (int u = 0; u < a.nunit; ++u) { mbar_init(bar_zfull + 8 * u, NLW * 32); mbar_init(bar_zfree + 8 * u, 1); }
+        for (int u = 0; u < a.nunit; ++u) { mbar_init(bar_zfull + 8 * u, NLG * 32); mbar_init(bar_zfree + 8 * u, 1); }
         for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, 1); mbar_init(bar_accfree + 8 * t, NCW); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -228,7 +231,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    if (warp >= NCW && warp < NCW + NLW) {
+    if (warp >= NCW && warp < NCW + NLG) {
         // =========================== loader warps ===========================
         const int lt = (warp - NCW) * 32 + lane;
         uint32_t it = 0, zi = 0;
@@ -246,7 +249,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     const int cpr = (int)U.c_src >> 3;
                     const int n_it = a.K * cpr;
                     const SmallDiv by_cpr(cpr);
-                    for (int cl = warp - NCW; cl < (int)U.ncomp; cl += NLW) {
+                    for (int cl = warp - NCW; cl < (int)U.ncomp; cl += NLG) {
                         const CompS cp = sComp[U.comp_begin + cl];
                         const int64_t g0 = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff;
                         const __nv_bfloat16* gh = a.zqh + g0;
@@ -288,33 +291,14 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                 }
                 __syncwarp();
                 if constexpr (GEO) {
-                    // recomputed from the edge vectors: thread <-> (edge, share of the radial indices and components)
-                    float* rawf = reinterpret_cast<float*>(stage + 2 * a.x_cap);       // phi rows [tb][KP]
-                    float* yT = rawf + NRAW * tb * KP;                                 // Y transposed [dsh][PS]
-                    const int nsh = max(1, (NLW * 32) >> lg);
-                    const int qw = (a.K + nsh - 1) / nsh, bw = (a.dsh + nsh - 1) / nsh;
-                    for (int i = lt; i < tb * nsh; i += NLW * 32) {
-                        const int e = i & (tb - 1), sh = i >> lg;
-                        const bool okb = e < nb;
-                        float rx = 0.f, ry = 0.f, rz = 1.f;
-                        if (okb) { const float* rp = a.rvec + (b0 + e) * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
-                        const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
-                        const int q_lo = sh * qw, q_hi = min(a.K, q_lo + qw), b_lo = sh * bw, b_hi = min(a.dsh, b_lo + bw);
-                        geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
-                            if (q >= q_lo && q < q_hi) rawf[e * KP + q] = okb ? f : 0.f;
-                        });
-                        geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
-                            if (b >= b_lo && b < b_hi) yT[b * PS + e] = okb ? yb : 0.f;
-                        });
-                    }
-                    __threadfence_block();       // the stores above are ordered before this thread's arrival on the stage
+                    // phi and Y of the stage come from the geometry warp
                 } else {
                 {
                     const bool v16 = (a.K & 3) == 0;
                     const int per = v16 ? a.K / 4 : a.K;
                     const int n_it = tb * per;
                     const SmallDiv by_per(per);
-                    for (int i = lt; i < n_it; i += NLW * 32) {
+                    for (int i = lt; i < n_it; i += NLG * 32) {
                         const int e = by_per(i), j = i - e * per;
                         const int64_t ee = b0 + min(e, nb - 1);
                         const uint32_t ok = e < nb ? 1u : 0u;
@@ -331,7 +315,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     const uint32_t y_u = raw_u + (uint32_t)(NRAW * tb * KP) * 4;
                     const int n_it = tb * a.dsh;
                     const SmallDiv by_dsh(a.dsh);
-                    for (int i = lt; i < n_it; i += NLW * 32) {
+                    for (int i = lt; i < n_it; i += NLG * 32) {
                         const int e = by_dsh(i), b = i - e * a.dsh;
                         const int64_t ee = b0 + min(e, nb - 1);
                         const uint32_t ok = e < nb ? 4u : 0u;
@@ -346,7 +330,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                     const int cpr = B.c_src >> 3;
                     const int npair = tb * cpr;
                     const SmallDiv by_cpr(cpr);
-                    for (int pr = lt; pr < npair; pr += NLW * 32) {
+                    for (int pr = lt; pr < npair; pr += NLG * 32) {
                         const int e = by_cpr(pr), j = pr - e * cpr;
                         const int32_t sid = sIds[e];
                         const uint32_t ok = sid >= 0 ? 16u : 0u;
@@ -365,6 +349,40 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                 cp_async_arrive(bar_full + 8 * st);
             }
             if (nbat == 1) load_zbar();
+        }
+    } else if (GEO && warp == NCW + NLG) {
+        // =========================== geometry warp ===========================
+        // walks the same receivers and batches as the loaders; lane <-> (edge, share of the radial indices and components)
+        uint32_t it = 0;
+        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+            int64_t seg0, seg1;
+            seg_bounds(a.row_ptr, a.node0 + nl, a.E, nullptr, seg0, seg1);
+            if (!any_op) seg1 = seg0;
+            for (int64_t b0 = seg0; b0 < seg1; b0 += tb, ++it) {
+                const int nb = (int)min((int64_t)tb, seg1 - b0);
+                const int st = (int)(it % NS);
+                if (it >= NS) mbar_wait(bar_free + 8 * st, ((it / NS) & 1) ^ 1, a.status);
+                uint8_t* stage = sRing + (size_t)st * stage_bytes;
+                float* rawf = reinterpret_cast<float*>(stage + 2 * a.x_cap);       // phi rows [tb][KP]
+                float* yT = rawf + NRAW * tb * KP;                                 // Y transposed [dsh][PS]
+                const int nsh = max(1, 32 >> lg);
+                const int qw = (a.K + nsh - 1) / nsh, bw = (a.dsh + nsh - 1) / nsh;
+                for (int i = lane; i < tb * nsh; i += 32) {
+                    const int e = i & (tb - 1), sh = i >> lg;
+                    const bool okb = e < nb;
+                    float rx = 0.f, ry = 0.f, rz = 1.f;
+                    if (okb) { const float* rp = a.rvec + (b0 + e) * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
+                    const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                    const int q_lo = sh * qw, q_hi = min(a.K, q_lo + qw), b_lo = sh * bw, b_hi = min(a.dsh, b_lo + bw);
+                    geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
+                        if (q >= q_lo && q < q_hi) rawf[e * KP + q] = okb ? f : 0.f;
+                    });
+                    geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
+                        if (b >= b_lo && b < b_hi) yT[b * PS + e] = okb ? yb : 0.f;
+                    });
+                }
+                mbar_arrive(bar_full + 8 * st);      // release: the stores above are visible to whoever sees the stage full
+            }
         }
     } else if (warp == NCW + NLW) {
         // =========================== MMA warp ===========================
@@ -516,17 +534,18 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                                     if (cl + c2 >= c_hi) break;
                                     const int ent = ent_u + (cl + c2) * d_src + s;
                                     const float mw = (DUAL && op == 0) ? sdM[ent * PS + e] : sM[ent * PS + e];
-                                    float gm = 0.f;
+                                    float gp[4] = {0.f, 0.f, 0.f, 0.f};       // four partial sums: short dependent chains
 #pragma unroll
                                     for (int x = 0; x < KP; ++x) {
-                                        gm = fmaf(aw[x], v[c2 * KP + x], gm);
+                                        gp[x & 3] = fmaf(aw[x], v[c2 * KP + x], gp[x & 3]);
                                         pphi[x] = fmaf(mw, v[c2 * KP + x], pphi[x]);
                                     }
+                                    const float gm = (gp[0] + gp[1]) + (gp[2] + gp[3]);
                                     sGM[ent * PS + e] = (sb == 0 ? 0.f : sGM[ent * PS + e]) + gm;
                                 }
                             };
                             float va[16];
-                            if constexpr (NLW == 2) {       // two CTAs per SM: half the registers, one load at a time
+                            if constexpr (MINB == 2) {      // two CTAs per SM: half the registers, one load at a time
                                 for (int ch = 0; ch < nch; ++ch) { issue(va); tc_wait_ld16(va); process(va); }
                             } else {
                             float vb[16];
@@ -573,11 +592,16 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, NLW == 2 ? 2 : 1) k_edge
                         for (int i = tid; i < a.dsh * tb; i += NCW * 32) {
                             const int b = i >> lg, ee = i & (tb - 1);
                             if (ee < nb) {
-                                float g = 0.f;
-                                for (int k = sInvPtr[b]; k < sInvPtr[b + 1]; ++k) {
-                                    const NzS t = sInv[k];
-                                    g = fmaf(t.coef, sGM[t.b * PS + ee], g);
+                                float g0 = 0.f, g1 = 0.f;                  // two partial sums, fixed order
+                                const int k1 = sInvPtr[b + 1];
+                                int k = sInvPtr[b];
+                                for (; k + 1 < k1; k += 2) {
+                                    const NzS t0 = sInv[k], t1 = sInv[k + 1];
+                                    g0 = fmaf(t0.coef, sGM[t0.b * PS + ee], g0);
+                                    g1 = fmaf(t1.coef, sGM[t1.b * PS + ee], g1);
                                 }
+                                if (k < k1) { const NzS t0 = sInv[k]; g0 = fmaf(t0.coef, sGM[t0.b * PS + ee], g0); }
+                                const float g = g0 + g1;
                                 if constexpr (GEO) { sGeo[ee * GW + KP + b] = g; continue; }
                                 float* p = a.gY + (b0 + ee) * a.dsh + b;
                                 if (a.Y_mode == 2) atomicAdd(p, g); else *p = g;
@@ -833,13 +857,13 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     a.status = status;
     const bool k8 = p->K <= 8;
     if (ss.rvec && dual) return cudaErrorNotSupported;
-    void (*kern2)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 2, false> : k_edge_tc<8, false, 8, 2, false>)
-                                     : (dual ? k_edge_tc<16, true, 8, 2, false> : k_edge_tc<16, false, 8, 2, false>);
-    void (*kern1)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3, false> : k_edge_tc<8, false, 8, 3, false>)
-                                     : (dual ? k_edge_tc<16, true, 8, 3, false> : k_edge_tc<16, false, 8, 3, false>);
+    void (*kern2)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3, false, 2> : k_edge_tc<8, false, 8, 3, false, 2>)
+                                     : (dual ? k_edge_tc<16, true, 8, 3, false, 2> : k_edge_tc<16, false, 8, 3, false, 2>);
+    void (*kern1)(const EtArgs) = k8 ? (dual ? k_edge_tc<8, true, 8, 3, false, 1> : k_edge_tc<8, false, 8, 3, false, 1>)
+                                     : (dual ? k_edge_tc<16, true, 8, 3, false, 1> : k_edge_tc<16, false, 8, 3, false, 1>);
     if (ss.rvec) {
-        kern2 = k8 ? k_edge_tc<8, false, 8, 2, true> : k_edge_tc<16, false, 8, 2, true>;
-        kern1 = k8 ? k_edge_tc<8, false, 8, 3, true> : k_edge_tc<16, false, 8, 3, true>;
+        kern2 = k8 ? k_edge_tc<8, false, 8, 3, true, 2> : k_edge_tc<16, false, 8, 3, true, 2>;
+        kern1 = k8 ? k_edge_tc<8, false, 8, 3, true, 1> : k_edge_tc<16, false, 8, 3, true, 1>;
     }
     int max_smem = 0;
     for (const auto& ep : T.epar) max_smem = std::max(max_smem, ep.smem);
@@ -859,7 +883,7 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
         a.Y_mode = Y_mode ? (si == 0 ? Y_mode : 2) : 0;
         const int grid = (int)std::min<int64_t>(n_nodes, (int64_t)148 * ep.ctas);
         KernelTimer kt(K_EDGE, s);
-        if (ep.ctas == 2) kern2<<<grid, (8 + 2 + 1) * 32, ep.smem, s>>>(a);
+        if (ep.ctas == 2) kern2<<<grid, (8 + 3 + 1) * 32, ep.smem, s>>>(a);
         else kern1<<<grid, (8 + 3 + 1) * 32, ep.smem, s>>>(a);
         count_launch();
         e = cudaGetLastError();

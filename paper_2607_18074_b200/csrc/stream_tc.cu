@@ -60,7 +60,8 @@ constexpr int NDW = 4;          // drain warps
 constexpr int NLW = 4;          // loader warps
 constexpr int NMW = 3;          // MMA warps (one issuing thread each; a unit's products all come from one of them)
 constexpr int W_DRAIN = NBW, W_LOAD = NBW + NDW, W_MMA = NBW + NDW + NLW;
-constexpr int TT = (W_MMA + NMW + 1) * 32;   // threads per CTA (a multiple of 128; the last warp has no role)
+constexpr int W_GEO = W_MMA + NMW;           // the last warp: recomputes phi and Y from edge vectors in geometry mode, else idle
+constexpr int TT = (W_GEO + 1) * 32;         // threads per CTA (a multiple of 128)
 constexpr int MAXNS = 4;        // ring stages: 2..4, as many as shared memory holds
 constexpr int NSLOT = 2 * NBG;  // A slab slots in tensor memory, two per builder group: 16 columns each (8 hi + 8 lo)
 constexpr int TMEM_COLS = 512;
@@ -89,6 +90,9 @@ struct TcArgs {
     const float* rvec;     // edge vectors [E][3]: when set, Y and phi are recomputed from them (Y, phi are NULL then)
     float geo_rc;          // cutoff radius of the radial basis
     int32_t geo_basis, geo_p;
+    int32_t geo_inline;    // geometry mode: 0 = the geometry warp recomputes phi and Y (the default: nearly free, the warp has
+                           // nothing else to do); 1 = the loader warps do it themselves between their copies (measured
+                           // 5 - 20 % slower in the forward; the loader is close to the critical path)
     __nv_bfloat16* zh;
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
@@ -217,7 +221,8 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
     const int nsub = (has_a1 ? 1 : 0) + (has_a2 ? 1 : 0);
 
     if (tid == 0) {
-        for (int s = 0; s < MAXNS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32); mbar_init(bar_sfree + 8 * s, NMW); }
+        // a stage is full when every loader thread's copies have landed (and the geometry warp, where it runs, has stored phi and Y)
+        for (int s = 0; s < MAXNS; ++s) { mbar_init(bar_full + 8 * s, NLW * 32 + ((a.rvec && !a.geo_inline) ? 32 : 0)); mbar_init(bar_sfree + 8 * s, NMW); }
         for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_slotfree + 8 * s, 1); slot_fill[s] = 0u; }
         for (int t = 0; t < 2; ++t) { mbar_init(bar_accfull + 8 * t, NMW); mbar_init(bar_accfree + 8 * t, NDW); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -334,6 +339,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             const int le = lane & (TB - 1);
             const int64_t ee_own = __shfl_sync(0xffffffffu, eid, le);
             if (a.rvec) {
+                if (a.geo_inline) {
                 // recomputed from the edge vector: thread <-> (edge le, share g8 of the components and radial indices)
                 const int g8 = lt >> 4;
                 const bool okb = (msk >> le) & 1u;
@@ -350,6 +356,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                     if (b < dsh && (b & 7) == g8) yT[b * PS + le] = okb ? yb : 0.f;
                 });
                 __threadfence_block();       // the stores above are ordered before this thread's arrival on the stage
+                }
             } else {
             // phi (and vphi) rows: raw[e][KP]   (all lanes run every iteration: the loops hold shuffles)
             {
@@ -414,6 +421,56 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_full + 8 * st) : "memory");
             cur = nxt; have = have_n; eid = eid_n; sn = sn_n; msk = msk_n;
             if (++st == NS) { st = 0; ++round; }
+        }
+    } else if (warp == W_GEO) {
+        // =========================== geometry warp ===========================
+        // Walks the same batches as the loaders and fills the stage's phi rows and transposed Y from the edge vectors
+        // (lane <-> edge lane & 15, half of the radial indices / components each).
+        if (a.rvec != nullptr && !a.geo_inline) {
+            int64_t p_item = blockIdx.x, p_seg0 = 0, p_seg1 = 0;
+            ItemPos lp; lp.init(p_item, a.n_nodes);
+            auto prefetch_item = [&]() {
+                if (p_item < total) {
+                    seg_bounds(a.ev.ptr, a.node0 + lp.nl, a.ev.E, nullptr, p_seg0, p_seg1);
+                    if (!any_op) p_seg1 = p_seg0;
+                }
+            };
+            prefetch_item();
+            int64_t b0 = 0, seg1 = 0;
+            auto next_batch = [&](bool first) -> bool {
+                if (!first) b0 += TB;
+                while (first || b0 >= seg1) {
+                    first = false;
+                    if (p_item >= total) return false;
+                    b0 = p_seg0; seg1 = p_seg1;
+                    p_item += gridDim.x; lp.step(gridDim.x, a.n_nodes);
+                    prefetch_item();
+                }
+                return true;
+            };
+            const int le = lane & (TB - 1), hf = lane >> 4;
+            int st = 0; uint32_t round = 0;
+            for (bool have = next_batch(true); have; have = next_batch(false)) {
+                const int64_t pos = b0 + le;
+                bool okb = pos < seg1;
+                int64_t ee = 0;
+                if (okb) { ee = a.ev.perm ? (int64_t)a.ev.perm[pos] : pos; okb = ee >= 0 && ee < a.ev.E; }
+                float rx = 0.f, ry = 0.f, rz = 1.f;
+                if (okb) { const float* rp = a.rvec + ee * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
+                const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                if (round > 0) mbar_wait(bar_sfree + 8 * st, (round & 1) ^ 1, a.status);
+                float* rawf = reinterpret_cast<float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.b_cap);
+                float* yT = rawf + NRAW * TB * KP;
+                geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
+                    if ((q & 1) == hf) rawf[le * KP + q] = okb ? f : 0.f;
+                });
+                const int dsh = a.dsh;
+                geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
+                    if (b < dsh && (b & 1) == hf) yT[b * PS + le] = okb ? yb : 0.f;
+                });
+                mbar_arrive(bar_full + 8 * st);      // release: the stores above are visible to whoever sees the stage full
+                if (++st == NS) { st = 0; ++round; }
+            }
         }
     } else if (warp >= W_MMA && warp < W_MMA + NMW) {
         // =========================== MMA warps ===========================
@@ -882,7 +939,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.sh = (const __nv_bfloat16*)ss.h; a.sl = (const __nv_bfloat16*)ss.l;
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
-    a.rvec = ss.rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p;
+    a.rvec = ss.rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p; a.geo_inline = 0;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
     a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages;

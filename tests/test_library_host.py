@@ -115,6 +115,13 @@ def test_argument_errors_are_status_codes():
     assert L.sobek_plan_path(plan.handle, 99, ctypes.byref(sb.PathInfo())) == -1
     assert sb.workspace_bytes(plan, 4, 0, 7) == 0
     assert L.sobek_last_device_status(None, None) == -1
+    # geometry front end: null descriptors and arguments are refused before anything is launched
+    assert L.sobek_edge_vectors(None, None, None, None) == -1
+    assert L.sobek_position_gradient(None, None, None, None) == -1
+    assert L.sobek_conv_geo_fwd(None, ctypes.byref(g), None, 0, 1.0, 6, None, None, None, None, 0, None) == -1
+    g1 = sb.Graph(4, 1, None, None, None, None)
+    assert L.sobek_conv_geo_fwd(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, None, None, None, None, 0, None) == -1   # no rvec
+    assert L.sobek_conv_geo_bwd(plan.handle, ctypes.byref(g1), None, 5, 1.0, 6, None, None, None, None, None, None, None, 0, None) == -1
 
 
 def test_uvu_plan_weight_counts_match_the_paper():
