@@ -114,3 +114,17 @@ def geo_bwd(orc, row_ptr, col, rvec, x, R, gy, r_c: float, basis: int = BESSEL, 
     s = (Y * torch.as_tensor(gY)).sum() + (phi * torch.as_tensor(gphi)).sum()
     (g_rvec,) = torch.autograd.grad(s, t)
     return gx, g_rvec.numpy(), gR
+
+
+def geo_dbwd(orc, row_ptr, col, rvec, x, R, gy, vx, v_rvec, vR, r_c: float, basis: int = BESSEL, p: int = 6, act=None):
+    """(ggy, hx, hR): derivatives of  <vx, gx> + <v_rvec, g_rvec> + <vR, gR>  (the adjoints of geo_bwd) with respect to
+    gy, x and R -- what a loss on the forces needs for its parameter and feature gradients.  Since
+    <v_rvec, g_rvec> = <J_Y v_rvec, gY> + <J_phi v_rvec, gphi>, this is the double backward of the convolution with the
+    directions vY = J_Y v_rvec and vphi = J_phi v_rvec (Jacobian-vector products of the definitions above, by
+    torch.autograd).  The derivative with respect to rvec itself (second derivatives of both bases) is not provided."""
+    t = torch.as_tensor(np.asarray(rvec, dtype=np.float64))
+    v = torch.as_tensor(np.asarray(v_rvec, dtype=np.float64))
+    Y, vY = torch.autograd.functional.jvp(lambda r: real_sh(r, orc.l_max), t, v)
+    phi, vphi = torch.autograd.functional.jvp(lambda r: radial(torch.linalg.norm(r, dim=-1), orc.K, r_c, basis, p), t, v)
+    ggy, hx, _, _, hR = orc.dbwd(row_ptr, col, x, Y.numpy(), phi.numpy(), R, gy, vx, vY.numpy(), vphi.numpy(), vR, act=act)
+    return ggy, hx, hR

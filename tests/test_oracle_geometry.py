@@ -171,3 +171,33 @@ def test_energy_is_invariant_and_forces_rotate():
         dp = np.zeros_like(d.pos); dp[i, k] = h
         fd = (energy_forces(d.pos + dp)[0] - energy_forces(d.pos - dp)[0]) / (2 * h)
         assert abs(-fd - F0[i, k]) < 1e-6 * max(1.0, abs(fd))
+
+
+def test_force_loss_double_backward_by_central_differences():
+    """geo_dbwd against central differences of  Phi = <vx, gx> + <v_r, g_r> + <vR, gR>  evaluated with geo_bwd, with
+    respect to entries of x (hx), R (hR) and gy (ggy; Phi is linear in gy, so that one is exact up to rounding)."""
+    o, w, d = _tiny(seed=7)
+    rv = geometry.edge_vectors(d.col, d.recv, d.pos)
+    rng = np.random.default_rng(11)
+    v_r = rng.standard_normal(rv.shape)
+    ggy, hx, hR = geometry.geo_dbwd(o, d.row_ptr, d.col, rv, d.x, d.R, d.gy, d.vx, v_r, d.vR, w.r_c)
+
+    def Phi(x, R, gy):
+        gx, g_r, gR = geometry.geo_bwd(o, d.row_ptr, d.col, rv, x, R, gy, w.r_c)
+        return (d.vx * gx).sum() + (v_r * g_r).sum() + (d.vR * gR).sum()
+
+    h = 1e-5
+    for arr, grad, k in ((d.x, hx, 0), (d.R, hR, 1), (d.gy, ggy, 2)):
+        scale = np.abs(grad).max()
+        assert scale > 1e-6
+        for _ in range(6):
+            idx = tuple(rng.integers(n) for n in arr.shape)
+            dp = np.zeros_like(arr); dp[idx] = h
+            args = [d.x, d.R, d.gy]
+            args[k] = arr + dp; fp = Phi(*args)
+            args[k] = arr - dp; fm = Phi(*args)
+            assert abs((fp - fm) / (2 * h) - grad[idx]) < 1e-6 * scale + 1e-9
+    # with no direction on the edge vectors it is the stored-input double backward with vY = vphi = 0
+    g2 = geometry.geo_dbwd(o, d.row_ptr, d.col, rv, d.x, d.R, d.gy, d.vx, np.zeros_like(rv), d.vR, w.r_c)
+    ref = o.dbwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, d.vx, np.zeros_like(d.vY), np.zeros_like(d.vphi), d.vR)
+    assert np.allclose(g2[0], ref[0], atol=1e-11) and np.allclose(g2[1], ref[1], atol=1e-11) and np.allclose(g2[2], ref[4], atol=1e-11)
