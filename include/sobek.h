@@ -257,13 +257,19 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
  * Every r_e must be non-zero (an edge of length zero has no direction; nothing is checked).
  * Plans: fully connected or channelwise, ir_mul layout, l_max <= 4, the tensor-core edge kernels in use (the
  * default where the profile allows them: K <= 16, multiplicities multiples of 16 up to 128); otherwise UNSUPPORTED.
- * Workspace: sobek_workspace_bytes(plan, N, E, 0) for the forward, (.., 1) for the backward.  Double backward
- * through the geometry is not provided.  Errors as for sobek_conv_fwd / sobek_conv_bwd.
+ * Workspace: sobek_workspace_bytes(plan, N, E, 0) for the forward, (.., 1) for the backward, (.., 2) for the double
+ * backward.  Errors as for sobek_conv_fwd / sobek_conv_bwd / sobek_conv_dbwd.
  *
  * sobek_edge_vectors       rvec[e] = pos[col[e]] - pos[receiver(e)]                       (pos [N][3], rvec [E][3])
  * sobek_conv_geo_fwd       y of sobek_conv_fwd with Y, phi computed from rvec
  * sobek_conv_geo_bwd       gx, gR as sobek_conv_bwd; g_rvec[e] = J_Y(r_e)^T gY_e + J_phi(r_e)^T gphi_e.  Any of
  *                          gx, g_rvec, gR may be NULL (gx needs the sender view of the graph)
+ * sobek_conv_geo_dbwd      double backward for a loss on the forces: with cotangents (vx, v_rvec, vR) on the outputs
+ *                          (gx, g_rvec, gR) of sobek_conv_geo_bwd it returns ggy = d<v,b>/d gy, hx = d<v,b>/dx and
+ *                          hR = d<v,b>/dR (Eqs. streamed_directional_terms .. streamed_operand_second_adjoints with
+ *                          the directions vY = J_Y v_rvec, vphi = J_phi v_rvec, which the dual stream passes compute
+ *                          from rvec and v_rvec themselves).  Any of the cotangents and of the outputs may be NULL.  The
+ *                          derivative with respect to rvec itself (second derivatives of both bases) is not provided.
  * sobek_position_gradient  gpos[n] = sum_{e: sender(e) = n} g_rvec[e] - sum_{e: receiver(e) = n} g_rvec[e], the
  *                          adjoint of sobek_edge_vectors (forces are its negative); each node sums its own edges in
  *                          a fixed order (needs src_ptr and src_perm).  Only enqueues.
@@ -277,6 +283,10 @@ int sobek_conv_geo_fwd(const sobek_plan* plan, const sobek_graph* g, const float
 int sobek_conv_geo_bwd(const sobek_plan* plan, const sobek_graph* g, const float* rvec, int basis, float r_cut,
                        int envelope_p, const float* x, const float* R, const float* gy, float* gx, float* g_rvec,
                        float* gR, void* ws, size_t ws_bytes, void* stream);
+int sobek_conv_geo_dbwd(const sobek_plan* plan, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                        int envelope_p, const float* x, const float* R, const float* gy, const float* vx,
+                        const float* v_rvec, const float* vR, float* ggy, float* hx, float* hR, void* ws,
+                        size_t ws_bytes, void* stream);
 int sobek_position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, void* stream);
 
 /*

@@ -37,7 +37,7 @@ EXPORTS = [
     "sobek_launch_count", "sobek_timing_enable", "sobek_timing_classes", "sobek_timing_class_name",
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
     "sobek_conv_fwd_retain", "sobek_conv_bwd_retained", "sobek_static_last_status", "sobek_measure_fp32_peak",
-    "sobek_edge_vectors", "sobek_conv_geo_fwd", "sobek_conv_geo_bwd", "sobek_position_gradient",
+    "sobek_edge_vectors", "sobek_conv_geo_fwd", "sobek_conv_geo_bwd", "sobek_conv_geo_dbwd", "sobek_position_gradient",
 ]
 BASIS_BESSEL, BASIS_GAUSSIAN = 0, 1
 
@@ -102,6 +102,7 @@ def lib():
         L.sobek_position_gradient.argtypes = [POINTER(Graph), c_void_p, c_void_p, c_void_p]
         L.sobek_conv_geo_fwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 4 + [c_size_t, c_void_p]
         L.sobek_conv_geo_bwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 7 + [c_size_t, c_void_p]
+        L.sobek_conv_geo_dbwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 10 + [c_size_t, c_void_p]
         L.sobek_selftest_wait_timeout.argtypes = [c_void_p, c_uint, c_void_p]
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
         L.sobek_static_scratch_bytes.restype = c_size_t
@@ -306,6 +307,12 @@ def conv_geo_bwd(plan, graph, rvec, basis, r_cut, envelope_p, x, R, gy, gx, g_rv
     _check(lib().sobek_conv_geo_bwd(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
                                     _ptr(x), _ptr(R), _ptr(gy), _ptr(gx), _ptr(g_rvec), _ptr(gR), _ptr(ws),
                                     ws.numel() * ws.element_size(), _stream()), "sobek_conv_geo_bwd")
+
+
+def conv_geo_dbwd(plan, graph, rvec, basis, r_cut, envelope_p, x, R, gy, vx, v_rvec, vR, ggy, hx, hR, ws):
+    _check(lib().sobek_conv_geo_dbwd(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
+                                     _ptr(x), _ptr(R), _ptr(gy), _ptr(vx), _ptr(v_rvec), _ptr(vR), _ptr(ggy), _ptr(hx),
+                                     _ptr(hR), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "sobek_conv_geo_dbwd")
 
 
 def conv_fwd_retain(plan, graph, x, Y, phi, R, y, ws) -> int:

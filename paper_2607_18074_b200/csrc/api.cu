@@ -417,14 +417,21 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
                    const float* phi, const float* R, const float* gy, const float* vx,
                    const float* vY, const float* vphi, const float* vR, float* ggy,
                    float* hx, float* hY, float* hphi, float* hR, void* ws, size_t ws_bytes,
-                   void* stream) {
+                   void* stream, const SplitSrc* geo = nullptr) {
     int rc = check_common(p, g, ws, ws_bytes, 2);
     if (rc) return rc;
-    if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (!R || (g->N > 0 && (!x || !gy)) || (g->E > 0 && !geo && (!Y || !phi))) return SOBEK_ERR_INVALID_ARG;
+    if (geo) {
+        // geometry mode: the direction on the edge vectors stands for both vY and vphi (the dual stream passes compute
+        // J_Y v and J_phi v themselves); the second-order edge adjoints are not provided
+        if (hY || hphi) return SOBEK_ERR_UNSUPPORTED;
+        vY = vphi = geo->vrvec;
+    }
     if (!aligned16(x, Y, phi, R, gy, vx, vY, vphi, vR, ggy, hx, hY, hphi, hR)) return SOBEK_ERR_INVALID_ARG;
     if (hx && g->E > 0 && (!g->src_ptr || !g->src_perm)) return SOBEK_ERR_NEED_TRANSPOSE;
     cudaStream_t s = (cudaStream_t)stream;
     Workspace w = carve(p, g->N, 2, ws);
+    if (geo && !(geo_supported(p, w, 1) && p->fwd.tc[1].ok && p->tr.tc[1].ok && w.vsh)) return SOBEK_ERR_UNSUPPORTED;
     CK(cudaMemsetAsync(w.status, 0, kHeaderBytes, s));
     const int64_t KN = (int64_t)p->K * p->N_w;
     const bool any_edge_dir = vx || vY || vphi;
@@ -448,6 +455,7 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
 
     const EdgeView rv = receiver_view(g);
     SplitSrc xs{}, gs{};
+    if (geo) { xs = *geo; gs = *geo; }
     const bool tc_edge_plain = w.zqh != nullptr, tc_edge_dual = tc_edge_plain && p->fwd.etc[1].ok && (!vx || w.vsh);
     if (w.xsh && (ggy || hR || ((hphi || hY) && tc_edge_plain))) {
         CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl;
@@ -652,6 +660,18 @@ extern "C" int sobek_conv_geo_bwd(const sobek_plan* p, const sobek_graph* g, con
     else geo.rvec = rvec ? rvec : reinterpret_cast<const float*>(&geo);
     geo.g_rvec = g_rvec;
     return conv_bwd_core(p, g, x, nullptr, nullptr, R, gy, gx, nullptr, nullptr, gR, ws, ws_bytes, stream, 0, &geo);
+}
+
+extern "C" int sobek_conv_geo_dbwd(const sobek_plan* p, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                                   int envelope_p, const float* x, const float* R, const float* gy, const float* vx,
+                                   const float* v_rvec, const float* vR, float* ggy, float* hx, float* hR, void* ws,
+                                   size_t ws_bytes, void* stream) {
+    SplitSrc geo{};
+    if (g && g->E > 0) { const int rc = geo_source(rvec, basis, r_cut, envelope_p, &geo); if (rc) return rc; }
+    else geo.rvec = rvec ? rvec : reinterpret_cast<const float*>(&geo);
+    geo.vrvec = v_rvec;
+    return conv_dbwd_core(p, g, x, nullptr, nullptr, R, gy, vx, nullptr, nullptr, vR, ggy, hx, nullptr, nullptr, hR, ws,
+                          ws_bytes, stream, &geo);
 }
 
 extern "C" int sobek_conv_fwd_retain(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,

@@ -336,6 +336,7 @@ struct SplitSrc {
     float geo_rc = 0.f;
     int geo_basis = 0, geo_p = 6;
     float* g_rvec = nullptr;
+    const float* vrvec = nullptr;     // double backward: direction on the edge vectors (dual stream passes only)
 };
 cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
                           int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,

@@ -88,6 +88,7 @@ struct TcArgs {
     const float* phi;
     const float* vphi;
     const float* rvec;     // edge vectors [E][3]: when set, Y and phi are recomputed from them (Y, phi are NULL then)
+    const float* vrvec;    // DUAL, geometry mode: direction on the edge vectors; vY = J_Y vrvec, vphi = J_phi vrvec
     float geo_rc;          // cutoff radius of the radial basis
     int32_t geo_basis, geo_p;
     int32_t geo_inline;    // geometry mode: 0 = the geometry warp recomputes phi and Y (the default: nearly free, the warp has
@@ -213,7 +214,8 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
     const uint32_t fill0 = smem_u32(slot_fill);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool has_vx = DUAL && a.vsh != nullptr, has_vY = DUAL && a.vY != nullptr, has_vphi = DUAL && a.vphi != nullptr;
+    const bool has_vx = DUAL && a.vsh != nullptr, has_vY = DUAL && (a.rvec ? a.vrvec != nullptr : a.vY != nullptr),
+               has_vphi = DUAL && (a.rvec ? a.vrvec != nullptr : a.vphi != nullptr);
     const bool has_a1 = !DUAL || has_vY || has_vphi;   // operand 1: [phi*M] (plain) or [vphi*M + phi*dM] (dual), times x
     const bool has_a2 = has_vx;                        // operand 2 (dual): [phi*M] times vx
     const bool any_op = has_a1 || has_a2;
@@ -458,18 +460,37 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                 float rx = 0.f, ry = 0.f, rz = 1.f;
                 if (okb) { const float* rp = a.rvec + ee * 3; rx = __ldg(rp); ry = __ldg(rp + 1); rz = __ldg(rp + 2); }
                 const float r = sqrtf(rx * rx + ry * ry + rz * rz), ir = 1.f / r;
+                // every sub-batch of the batch (one per operand pair of the dual pass) has a stage of its own and needs the same rows
+                for (int sub = 0; sub < nsub; ++sub) {
                 if (round > 0) mbar_wait(bar_sfree + 8 * st, (round & 1) ^ 1, a.status);
                 float* rawf = reinterpret_cast<float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.b_cap);
                 float* yT = rawf + NRAW * TB * KP;
-                geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float) {
-                    if ((q & 1) == hf) rawf[le * KP + q] = okb ? f : 0.f;
+                const float ux = rx * ir, uy = ry * ir, uz = rz * ir;
+                // DUAL: the directions vphi = phi'(r) (u . v) and vY = grad F . (v - u (u . v)) / r of the edge-vector direction v
+                float uv = 0.f, tx = 0.f, ty = 0.f, tz = 0.f;
+                const bool dirs = DUAL && a.vrvec != nullptr;
+                if (dirs && okb) {
+                    const float* vp = a.vrvec + ee * 3;
+                    const float vx_ = __ldg(vp), vy_ = __ldg(vp + 1), vz_ = __ldg(vp + 2);
+                    uv = ux * vx_ + uy * vy_ + uz * vz_;
+                    tx = (vx_ - ux * uv) * ir; ty = (vy_ - uy * uv) * ir; tz = (vz_ - uz * uv) * ir;
+                }
+                geo_radial(r, a.K, a.geo_rc, a.geo_basis, a.geo_p, [&](int q, float f, float df) {
+                    if ((q & 1) == hf) {
+                        rawf[le * KP + q] = okb ? f : 0.f;
+                        if (dirs) rawf[TB * KP + le * KP + q] = okb ? df * uv : 0.f;
+                    }
                 });
                 const int dsh = a.dsh;
-                geo_sh(rx * ir, ry * ir, rz * ir, [&](int b, float yb, float, float, float) {
-                    if (b < dsh && (b & 1) == hf) yT[b * PS + le] = okb ? yb : 0.f;
+                geo_sh(ux, uy, uz, [&](int b, float yb, float fx, float fy, float fz) {
+                    if (b < dsh && (b & 1) == hf) {
+                        yT[b * PS + le] = okb ? yb : 0.f;
+                        if (dirs) yT[dsh * PS + b * PS + le] = okb ? fx * tx + fy * ty + fz * tz : 0.f;
+                    }
                 });
                 mbar_arrive(bar_full + 8 * st);      // release: the stores above are visible to whoever sees the stage full
                 if (++st == NS) { st = 0; ++round; }
+                }
             }
         }
     } else if (warp >= W_MMA && warp < W_MMA + NMW) {
@@ -940,6 +961,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.rvec = ss.rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p; a.geo_inline = 0;
+    a.vrvec = dual ? ss.vrvec : nullptr;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
     a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages;

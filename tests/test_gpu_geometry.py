@@ -116,6 +116,42 @@ def test_full_size_sampled(name):
     assert np.all(g_rv[mask] == 0)
 
 
+@pytest.mark.parametrize("name", list(CASES))
+def test_force_loss_double_backward(name):
+    """ggy, hx, hR for cotangents on (gx, g_rvec, gR): all three directions, single directions, partial outputs."""
+    import torch
+    c = GeoCase(CASES[name])
+    d, i = c.d, c.plan.info
+    v_r = np.random.default_rng(17).standard_normal((c.E, 3))
+    v_rt = torch.from_numpy(v_r.astype(np.float32)).to("cuda:0")
+    v_r = v_rt.cpu().numpy().astype(np.float64)
+
+    def run(dirs=(True, True, True), outs=(True, True, True)):
+        res = [c._new(c.N, i.C_y), c._new(c.N, i.C_x), c._new(i.K, i.N_w)]
+        o = [t if on else None for t, on in zip(res, outs)]
+        v = [t if on else None for t, on in zip((c.vx, v_rt, c.vR), dirs)]
+        c.sb.conv_geo_dbwd(c.plan, c.graph, c.rvec, c.basis, c.w.r_c, 6, c.x, c.R, c.gy, *v, *o, c.ws(2))
+        assert c.sb.last_device_status(c.ws(2)) == 0
+        return [None if t is None else t.cpu().numpy() for t in o]
+
+    def ref(dirs=(True, True, True)):
+        z = lambda a, on: a if on else np.zeros_like(a)
+        return geometry.geo_dbwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, d.gy, z(d.vx, dirs[0]), z(v_r, dirs[1]),
+                                 z(d.vR, dirs[2]), c.w.r_c, c.basis)
+
+    got, want = run(), ref()
+    for a, b in zip(got, want):
+        assert np.isfinite(a).all() and np.abs(b).max() > 1e-3 and rel_err(a, b) <= BWD_TOL
+    # the direction on the edge vectors alone (the force term proper), and without it
+    for dirs in [(False, True, False), (True, False, True)]:
+        got, want = run(dirs), ref(dirs)
+        for a, b in zip(got, want):
+            assert rel_err(a, b) <= BWD_TOL if np.abs(b).max() > 0 else np.all(a == 0)
+    full = run()
+    part = run(outs=(False, True, False))
+    assert part[0] is None and part[2] is None and np.array_equal(part[1], full[1])
+
+
 def test_partial_outputs_and_argument_errors():
     c = GeoCase(CASES["cfg3_N120"])
     full = c.geo_bwd()

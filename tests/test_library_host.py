@@ -122,6 +122,7 @@ def test_argument_errors_are_status_codes():
     g1 = sb.Graph(4, 1, None, None, None, None)
     assert L.sobek_conv_geo_fwd(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, None, None, None, None, 0, None) == -1   # no rvec
     assert L.sobek_conv_geo_bwd(plan.handle, ctypes.byref(g1), None, 5, 1.0, 6, None, None, None, None, None, None, None, 0, None) == -1
+    assert L.sobek_conv_geo_dbwd(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, *([None] * 10), 0, None) == -1
 
 
 def test_uvu_plan_weight_counts_match_the_paper():
