@@ -159,6 +159,7 @@ struct TcSets {
     int32_t max_ent = 0, tmem_cols = 32;
     int32_t acc_cols = 0;             // accumulator columns of one buffer (two buffers are allocated)
     int32_t ring_stages = 2;          // stream: stages of the shared-memory ring (as many as fit)
+    int32_t nbuf = 2;                 // stream: accumulator buffers in tensor memory (2, or 1 for wider sets)
     int32_t smem_bytes = 0, ctas_per_sm = 1;
 };
 

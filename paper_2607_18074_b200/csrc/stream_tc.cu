@@ -98,6 +98,8 @@ struct TcArgs {
     __nv_bfloat16* zl;
     int32_t K, dsh, C_src, nsets;
     int32_t b_cap, max_ent, acc_cols, n_units, n_blks, n_comps, max_nz, ns, n_slab;
+    int32_t nbuf;           // accumulator buffers: 2 (a set's tiles fit half of the accumulator columns; the drain of one item
+                            // overlaps the MMAs of the next) or 1 (wider sets, the MMAs wait for the drain)
     int32_t max_own;        // slabs of a batch that one builder group builds, at most
     const uint32_t* slabs;  // per set (TSet::sched_begin, nslab): two words per slab, in build order (see SlabW)
     int* status;
@@ -513,8 +515,8 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                 if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
                     seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
                 if (seg1 <= seg0) continue;
-                const uint32_t buf = mi & 1;
-                if (mi >= 2) mbar_wait(bar_accfree + 8 * buf, ((mi >> 1) & 1) ^ 1, a.status);
+                const uint32_t buf = a.nbuf == 2 ? (mi & 1) : 0u, gen = a.nbuf == 2 ? (mi >> 1) : mi;    // buffer and its use count
+                if (mi >= (uint32_t)a.nbuf) mbar_wait(bar_accfree + 8 * buf, (gen & 1) ^ 1, a.status);
                 tc_fence_after();
                 const SlabW* slabs = sSlab + S.sched_begin;
                 const uint32_t j0 = ((uint32_t)S.mfirst >> (8 * me)) & 255u;     // first slab of this thread (255: none)
@@ -571,9 +573,9 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             dp.step(gridDim.x, a.n_nodes);
             if (item + gridDim.x < total) seg_bounds(a.ev.ptr, a.node0 + dp.nl, a.ev.E, nullptr, dx0, dx1);
             const bool wrote = seg1 > seg0;      // a node without edges has a state of zeros
-            const uint32_t buf = mi & 1;
+            const uint32_t buf = a.nbuf == 2 ? (mi & 1) : 0u, gen = a.nbuf == 2 ? (mi >> 1) : mi;
             if (wrote) {
-                mbar_wait(bar_accfull + 8 * buf, (mi >> 1) & 1, a.status);
+                mbar_wait(bar_accfull + 8 * buf, gen & 1, a.status);
                 tc_fence_after();
             }
             for (int ui = 0; ui < S.nunit; ++ui) {
@@ -833,6 +835,15 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
         // greedy packing of consecutive units into passes: the accumulator tiles of a pass fit one of the two TMEM
         // buffers and its operand regions fit shared memory with at least two ring stages
         const int budget = 227 * 1024;
+        // Two accumulator buffers (the drain of one receiver overlaps the MMAs of the next) when at least two of the
+        // widest tiles fit half of the accumulator columns; else one buffer over all of them: with 128-column tiles a
+        // half holds a single tile, a set then has one to nine slabs per batch and most builder groups idle, which
+        // costs more than the wait for the drain (measured: 128-wide profiles 10 - 17 % faster with one buffer, 32- and
+        // 64-wide ones 2 - 10 % slower).
+        int widest = 0;
+        for (const Cand& c : cands) widest = std::max(widest, cols32(c.blk));
+        T.nbuf = 2 * widest > ACC_BUDGET ? 1 : 2;
+        const int acc_budget = T.nbuf == 2 ? ACC_BUDGET : RING0;
         bool fits = true;
         size_t i = 0;
         while (i < cands.size() && fits) {
@@ -849,7 +860,7 @@ void build_tc_sets(const sobek_plan* p, Direction& dir) {
                 const int own2 = (slabs_in + blocks[c.blk].d_src + NBG - 1) / NBG;
                 const int need = smem_need(KP, dual, p->dim_sh, 2, bcap, std::max(T.max_ent, e2), (int)cands.size(), (int)cands.size(),
                                            n_comps_total, std::max(T.max_nz, n2), n_slab, std::max(T.max_units, own2));
-                if (need > budget || c2 > ACC_BUDGET) break;
+                if (need > budget || c2 > acc_budget) break;
                 b_bytes = b2; cols = c2; nent = e2; nnz = n2; slabs_in += blocks[c.blk].d_src;
                 if (new_blk) set_blks.push_back(c.blk);
             }
@@ -964,7 +975,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.vrvec = dual ? ss.vrvec : nullptr;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();
-    a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages;
+    a.b_cap = T.b_cap; a.max_ent = T.max_ent; a.acc_cols = T.acc_cols; a.ns = T.ring_stages; a.nbuf = T.nbuf;
     a.n_units = (int)T.units.size(); a.n_blks = (int)T.blks.size(); a.n_comps = (int)T.comps.size(); a.max_nz = T.max_nz;
     a.slabs = T.d_slabs; a.n_slab = (int)T.slabs.size() / 2; a.max_own = T.max_units;
     a.status = status;
