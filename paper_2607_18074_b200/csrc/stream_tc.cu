@@ -66,6 +66,7 @@ constexpr int MAXNS = 4;        // ring stages: 2..4, as many as shared memory h
 constexpr int NSLOT = 2 * NBG;  // A slab slots in tensor memory, two per builder group: 16 columns each (8 hi + 8 lo)
 constexpr int TMEM_COLS = 512;
 constexpr int RING0 = TMEM_COLS - NSLOT * 16;      // first column of the slot ring
+constexpr int DRAIN_BYTES = NDW * 32 * 64 * 2;   // per drain warp: 32 rows x 32 columns, bf16 hi and lo
 constexpr int ACC_BUDGET = RING0 / 2;              // columns of one accumulator buffer (two buffers)
 constexpr int PS = 20;          // row pitch (floats) of the transposed stages: 16 values + 4 (bank spread)
 static_assert(NSLOT % NBG == 0, "slab j of a batch goes to slot j mod NSLOT, built by group j mod NBG");
@@ -189,7 +190,8 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
     // ring stages: Bh Bl, then the raw phi / Y rows
     const uint32_t stage_bytes = (uint32_t)(2 * a.b_cap + ((raw_floats(KP, DUAL, a.dsh) * 4 + 1023) & ~1023));
     uint8_t* sRing = smem;
-    uint8_t* meta = sRing + (size_t)NS * stage_bytes;
+    uint8_t* sDrain = sRing + (size_t)NS * stage_bytes;      // staging of the drain warps (DRAIN_BYTES)
+    uint8_t* meta = sDrain + DRAIN_BYTES;
     // coupling values of a group's own slabs of one batch, double buffered: [NBG][2][max_own][MC][PS] (+ directions)
     constexpr int MC = 128 / KP;                              // components of a tile at most
     const size_t mbuf_floats = (size_t)a.max_own * MC * PS;
@@ -578,38 +580,57 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                 mbar_wait(bar_accfull + 8 * buf, gen & 1, a.status);
                 tc_fence_after();
             }
+            // A lane owns an accumulator row, but 16-byte stores of 32 lanes to 32 different state rows cost the load/store
+            // unit 32 line requests per instruction.  So the warp stages 32 columns of its 32 rows in shared memory (bf16
+            // hi and lo, 64 bytes per row, 16-byte pieces XOR-swizzled: conflict-free both ways) and writes them back with
+            // four lanes per row: 64 contiguous bytes per row, eight rows per instruction.
+            uint8_t* stg = sDrain + (size_t)(warp - W_DRAIN) * (32 * 64 * 2);
+            const int wr = lane >> 2, wp = lane & 3;             // write-back: row wr (+ 8 per pass), piece wp
             for (int ui = 0; ui < S.nunit; ++ui) {
                 const UInfo& U = sU[S.unit_begin + ui];
                 const int c_src = (int)U.c_src, ncols = (int)U.ncols;
                 const bool rv = cl < (int)U.ncomp && q < a.K;
-                int64_t off = 0;
+                int64_t off = -1;
                 if (rv) {
                     const CompS cp = sComp[U.comp_begin + cl];
                     off = a.n_nodes * cp.zoff + (nl * cp.d_dst + cp.o) * (int64_t)cp.ld + cp.koff + (int64_t)q * c_src;
                 }
+                int64_t roff[4];                                 // state offsets of the four rows this lane writes back
+#pragma unroll
+                for (int t = 0; t < 4; ++t) roff[t] = __shfl_sync(0xffffffffu, off, 8 * t + wr);
                 const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)a.acc_cols + U.tmem_col;
 #pragma unroll 1
-                for (int cc = 0; cc < ncols; cc += 16) {       // ncols is a multiple of 16, c_src of 8
-                    float v[16];
-                    if (wrote) {
-                        tc_ld16(trow + (uint32_t)cc, v);
-                    } else {
+                for (int cc = 0; cc < ncols; cc += 32) {         // ncols is a multiple of 16, c_src of 8
+                    const int sw = (lane >> 1) & 3;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                    }
-                    if (rv && cc < c_src) {
-                        __nv_bfloat16* ph_ = a.zh + off + cc;
-                        __nv_bfloat16* pl_ = a.zl + off + cc;
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        float v[16];
+                        if (wrote && cc + 16 * h2 < ncols) {
+                            tc_ld16(trow + (uint32_t)(cc + 16 * h2), v);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                        }
                         uint4 h, l;
                         split8(v, h, l);
-                        *reinterpret_cast<uint4*>(ph_) = h;
-                        *reinterpret_cast<uint4*>(pl_) = l;
-                        if (cc + 8 < c_src) {
-                            split8(v + 8, h, l);
-                            *reinterpret_cast<uint4*>(ph_ + 8) = h;
-                            *reinterpret_cast<uint4*>(pl_ + 8) = l;
+                        *reinterpret_cast<uint4*>(stg + lane * 64 + (((2 * h2) ^ sw) << 4)) = h;
+                        *reinterpret_cast<uint4*>(stg + 2048 + lane * 64 + (((2 * h2) ^ sw) << 4)) = l;
+                        split8(v + 8, h, l);
+                        *reinterpret_cast<uint4*>(stg + lane * 64 + (((2 * h2 + 1) ^ sw) << 4)) = h;
+                        *reinterpret_cast<uint4*>(stg + 2048 + lane * 64 + (((2 * h2 + 1) ^ sw) << 4)) = l;
+                    }
+                    __syncwarp();
+                    const int col = cc + 8 * wp;
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int row = 8 * t + wr;
+                        if (roff[t] >= 0 && col < c_src) {
+                            const int so = row * 64 + ((wp ^ ((row >> 1) & 3)) << 4);
+                            *reinterpret_cast<uint4*>(a.zh + roff[t] + col) = *reinterpret_cast<const uint4*>(stg + so);
+                            *reinterpret_cast<uint4*>(a.zl + roff[t] + col) = *reinterpret_cast<const uint4*>(stg + 2048 + so);
                         }
                     }
+                    __syncwarp();
                 }
             }
             if (wrote) {
@@ -775,7 +796,7 @@ int smem_need(int KP, bool dual, int dsh, int ns, int b_cap, int max_ent, int n_
     // tables: units (and at most as many blocks), sets, components, entries and sparse terms of one set, slabs
     const int tables = n_units * (int)(sizeof(UInfo) + sizeof(TBlk)) + n_sets * (int)sizeof(TSet) + n_comps * (int)sizeof(CompS) +
                        max_ent * (int)sizeof(EntS) + max_nz * (int)sizeof(NzS) + n_slab * (int)sizeof(SlabW) + 16;
-    return 1024 + ns * stage + (int)(meta * 4) + (2 * MAXNS + 2 * NSLOT + 4 + 4) * 8 + tables;
+    return 1024 + ns * stage + DRAIN_BYTES + (int)(meta * 4) + (2 * MAXNS + 2 * NSLOT + 4 + 4) * 8 + tables;
 }
 
 }  // namespace
