@@ -399,26 +399,30 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             }
             // sender rows -> B slabs (hi and lo), 16 bytes = 8 multiplicities per copy
             {
-                // lanes 2e, 2e+1 of each loader warp serve edge e; a thread walks pieces j0, j0 + 2 NLW, ... of the row
-                const int re = (lane >> 1) & (TB - 1);
-                const int32_t sne = __shfl_sync(0xffffffffu, sn, re);
-                const uint32_t ok = ((msk >> re) & 1u) * 16u;
-                const int j0 = (lane & 1) | ((lt >> 5) << 1);
-                const int64_t grow = (int64_t)sne * a.C_src;
-                const __nv_bfloat16* srch = (op == 0 ? a.sh : a.vsh) + grow;
-                const __nv_bfloat16* srcl = (op == 0 ? a.sl : a.vsl) + grow;
+                // Eight consecutive loader threads serve one edge (four or two for blocks of fewer than 64 / 32
+                // multiplicities): a copy instruction then reads whole 128-byte runs of four sender rows instead of 32 bytes
+                // of sixteen.  A thread walks pieces j0, j0 + 8, ... of its edge's row.
+                const __nv_bfloat16* baseh = op == 0 ? a.sh : a.vsh;
+                const __nv_bfloat16* basel = op == 0 ? a.sl : a.vsl;
                 for (int bi = 0; bi < S.nblk; ++bi) {
                     const TBlk B = sBlk[S.blk_begin + bi];
                     const int cpr = B.c_src >> 3;                  // 16-byte pieces per row
-                    for (int j = j0; j < cpr; j += 2 * NLW) {
-                        const int u = 8 * j;
-                        uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + re * 128 + ((((u & 63) >> 3) ^ (re & 7)) << 4));
-                        const __nv_bfloat16* ph = srch + B.src_off + u;
-                        const __nv_bfloat16* pl = srcl + B.src_off + u;
-                        for (int sdx = 0; sdx < B.d_src; ++sdx) {
-                            cp_async16_zfill(d, ph, ok);
-                            cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
-                            d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                    const int lgp = cpr >= 8 ? 3 : (cpr >= 4 ? 2 : 1);
+                    const int re = lt >> lgp, j0 = lt & ((1 << lgp) - 1);
+                    const int32_t sne = __shfl_sync(0xffffffffu, sn, re & (TB - 1));
+                    if (re < TB) {
+                        const uint32_t ok = ((msk >> re) & 1u) * 16u;
+                        const int64_t grow = (int64_t)sne * a.C_src + B.src_off;
+                        for (int j = j0; j < cpr; j += 1 << lgp) {
+                            const int u = 8 * j;
+                            uint32_t d = stage_u + (uint32_t)(B.b_off + (u >> 6) * B.atom_stride + re * 128 + ((((u & 63) >> 3) ^ (re & 7)) << 4));
+                            const __nv_bfloat16* ph = baseh + grow + u;
+                            const __nv_bfloat16* pl = basel + grow + u;
+                            for (int sdx = 0; sdx < B.d_src; ++sdx) {
+                                cp_async16_zfill(d, ph, ok);
+                                cp_async16_zfill(d + (uint32_t)a.b_cap, pl, ok);
+                                d += (uint32_t)B.slab_bytes; ph += B.c_src; pl += B.c_src;
+                            }
                         }
                     }
                 }
