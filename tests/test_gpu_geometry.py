@@ -178,6 +178,47 @@ def test_partial_outputs_and_argument_errors():
     assert e.value.code == -2
 
 
+def test_graph_without_edges():
+    """E = 0: zeros out, no edge array needed; and receivers without edges inside a graph give zero rows."""
+    import torch
+    import paper_2607_18074_b200 as sb
+    w = CASES["cfg3_N120"]
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    i, N = plan.info, 9
+    dev = "cuda:0"
+    rp = torch.zeros(N + 1, dtype=torch.int64, device=dev)
+    col = torch.zeros(0, dtype=torch.int32, device=dev)
+    g = sb.make_graph(rp, col, rp.clone(), col.clone(), col.clone())
+    x = torch.randn(N, i.C_x, device=dev); R = torch.randn(i.K, i.N_w, device=dev); gy = torch.randn(N, i.C_y, device=dev)
+    nan = lambda *s: torch.full(s, float("nan"), device=dev)
+    ws = torch.empty(sb.workspace_bytes(plan, N, 0, 2), dtype=torch.uint8, device=dev)
+    y = nan(N, i.C_y)
+    sb.conv_geo_fwd(plan, g, None, 0, 1.0, 6, x, R, y, ws)
+    gx, gR = nan(N, i.C_x), nan(i.K, i.N_w)
+    sb.conv_geo_bwd(plan, g, None, 0, 1.0, 6, x, R, gy, gx, None, gR, ws)
+    ggy, hx, hR = nan(N, i.C_y), nan(N, i.C_x), nan(i.K, i.N_w)
+    sb.conv_geo_dbwd(plan, g, None, 0, 1.0, 6, x, R, gy, x, None, R, ggy, hx, hR, ws)
+    gpos = nan(N, 3)
+    sb.position_gradient(g, None, gpos)
+    for t in (y, gx, gR, ggy, hx, hR, gpos):
+        assert torch.all(t == 0)
+    # a real graph in which the last three receivers lose their edges
+    c = GeoCase(w)
+    d = c.d
+    cut = int(d.row_ptr[c.N - 3])
+    rp2 = torch.from_numpy(np.minimum(d.row_ptr, cut).astype(np.int64)).to(dev)
+    col2 = c.col[:cut].contiguous()
+    sp, perm = sb.graph_prepare(rp2, col2)
+    g2 = sb.make_graph(rp2, col2, sp, perm, sb.graph_receivers(rp2, perm))
+    rvec2 = c.rvec[:cut].contiguous()
+    y2 = c._new(c.N, c.plan.info.C_y)
+    ws2 = torch.empty(sb.workspace_bytes(c.plan, c.N, cut, 1), dtype=torch.uint8, device=dev)
+    sb.conv_geo_fwd(c.plan, g2, rvec2, c.basis, w.r_c, 6, c.x, c.R, y2, ws2)
+    assert sb.last_device_status(ws2) == 0
+    ref = geometry.geo_fwd(c.oracle, np.minimum(d.row_ptr, cut), d.col[:cut], c.o_rvec[:cut], d.x, d.R, w.r_c, c.basis)
+    assert torch.all(y2[c.N - 3:] == 0) and rel_err(y2.cpu().numpy(), ref) <= FWD_TOL
+
+
 def test_forces_rotate_with_the_positions():
     """Eq. energy_force_symmetry on the GPU path: the energy sum_i a . y_i[scalars] of invariant features is unchanged
     by a rotation of the positions and the forces rotate with them."""
