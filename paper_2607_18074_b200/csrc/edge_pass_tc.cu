@@ -127,10 +127,10 @@ __device__ __forceinline__ void tc_ld8_nowait(uint32_t taddr, float* v) {
     for (int i = 8; i < 16; ++i) v[i] = 0.f;
 }
 
-// per-stage raw area (floats): phi rows [tb][KP], (vphi), Y written transposed [dsh][tb+4], (vY), sender ids [tb]
+// per-stage raw area (floats): phi rows [tb][KP], (vphi), Y written transposed [dsh][tb], (vY), sender ids [tb]
 __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
     const int n = dual ? 2 : 1;
-    return n * tb * KP + n * dsh * (tb + 4) + tb;
+    return n * tb * KP + n * dsh * tb + tb;
 }
 
 // GEO: the geometry mode (edge inputs recomputed from edge vectors, adjoint of the edge vectors out); plain pass only
@@ -143,7 +143,8 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int NRAW = DUAL ? 2 : 1;     // raw stages: phi and Y, plus their directions
-    const int tb = a.tb, lg = a.lg, PS = a.tb + 4;
+    const int tb = a.tb, lg = a.lg, PS = a.tb;       // PS: row pitch of the per-entry arrays (a warp holds whole rows of tb
+                                                     // edges: no padding is needed, and shared memory decides the number of sets)
     const uint32_t raw_bytes = (uint32_t)((raw_floats(KP, DUAL, a.dsh, tb) * 4 + 1023) & ~1023);
     const uint32_t stage_bytes = (uint32_t)(2 * a.x_cap) + raw_bytes;
     uint8_t* sRing = smem;                                     // stages: Xh Xl raw
@@ -646,7 +647,7 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
 int smem_need(int KP, bool dual, int dsh, int tb, int x_cap, int z_cap, int nent, int nunit, int ncomp, int nnz, int ninv) {
     constexpr int NCW = 8;
     const int nop = dual ? 2 : 1;
-    const int PS = tb + 4;
+    const int PS = tb;
     const int stage = 2 * x_cap + ((raw_floats(KP, dual, dsh, tb) * 4 + 1023) & ~1023);
     const size_t meta = (size_t)nop * nent * PS + (size_t)nent * PS + (size_t)NCW * 32 * KP + (size_t)tb * (KP + dsh);
     const int tables = nunit * (int)(sizeof(UInfo) + sizeof(TBlk)) + ncomp * (int)sizeof(CompS) + nent * (int)sizeof(EntS) +
