@@ -681,12 +681,15 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                 const float* raw = reinterpret_cast<const float*>(sRing + (size_t)st * stage_bytes + (size_t)2 * a.b_cap);
                 const float* sYT = raw + NRAW * TB * KP;
                 const float* sVYT = sYT + a.dsh * PS;
-                float* sM = sM0 + ((size_t)grp * 2 + (it & 1)) * mbuf_floats;
-                float* sdM = sdM0 + ((size_t)grp * 2 + (it & 1)) * mbuf_floats;
+                // the two sub-batches of a batch of the dual pass share the coupling values: built with the first one
+                const uint32_t mpar = nsub == 2 ? (it >> 1) & 1u : it & 1u;
+                float* sM = sM0 + ((size_t)grp * 2 + mpar) * mbuf_floats;
+                float* sdM = sdM0 + ((size_t)grp * 2 + mpar) * mbuf_floats;
                 // ---- coupling values of this group's own slabs: thread <-> (own slab k, component c, 8 edges)
                 const int nown = (S.nslab - grp + NBG - 1) / NBG;
+                const bool build_m = nsub == 1 || sb == 0;
 #pragma unroll 1
-                for (int i = gt; i < nown * 2 * MC; i += 128) {
+                for (int i = gt; build_m && i < nown * 2 * MC; i += 128) {
                     const int k = i / (2 * MC), c = (i >> 1) & (MC - 1), h = i & 1;
                     const uint32_t bw = slabs[grp + k * NBG].bw;
                     if (c >= (int)(bw >> 24)) continue;
@@ -719,7 +722,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
                         *reinterpret_cast<float4*>(dd + 4) = *reinterpret_cast<const float4*>(dm + 4);
                     }
                 }
-                group_sync(grp);
+                if (build_m) group_sync(grp);
                 // ---- this row's radial factors of the 16 edges (rows of padded q read the zeros left at start-up)
                 float ph[TB];
 #pragma unroll
