@@ -178,6 +178,32 @@ def test_partial_outputs_and_argument_errors():
     assert e.value.code == -2
 
 
+@pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16"])
+def test_channelwise_mode(name):
+    """The geometry front end in the channelwise (uvu) mode: same edge kernels, elementwise node-side steps."""
+    import torch
+    W = synth.Workload
+    w = {"uvu_16x3": W("uvu_16x3", P("16x0e+16x1o+16x2e"), P("16x0e+16x1o+16x2e"), 2, 8, 150, 4.0, 1.5, "bessel", seed=7, mode="uvu"),
+         "uvu_32x4_K16": W("uvu_32x4_K16", P("32x0e+32x1o+32x2e+32x3o"), P("32x0e+32x1o+32x2e+32x3o"), 3, 16, 80, 4.0, 1.7, "bessel",
+                           seed=8, mode="uvu")}[name]
+    c = GeoCase(w)
+    d, i = c.d, c.plan.info
+    y = c.geo_fwd()
+    assert rel_err(y, geometry.geo_fwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, w.r_c, c.basis)) <= FWD_TOL
+    got = c.geo_bwd()
+    ref = geometry.geo_bwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, d.gy, w.r_c, c.basis)
+    for a, b in zip(got, ref):
+        assert np.abs(b).max() > 1e-4 and rel_err(a, b) <= BWD_TOL
+    v_rt = torch.randn(c.E, 3, generator=torch.Generator().manual_seed(3)).to("cuda:0")
+    ggy, hx, hR = c._new(c.N, i.C_y), c._new(c.N, i.C_x), c._new(i.K, i.N_w)
+    c.sb.conv_geo_dbwd(c.plan, c.graph, c.rvec, c.basis, w.r_c, 6, c.x, c.R, c.gy, c.vx, v_rt, c.vR, ggy, hx, hR, c.ws(2))
+    assert c.sb.last_device_status(c.ws(2)) == 0
+    ref = geometry.geo_dbwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, d.gy, d.vx, v_rt.cpu().numpy().astype(np.float64),
+                            d.vR, w.r_c, c.basis)
+    for a, b in zip((ggy, hx, hR), ref):
+        assert rel_err(a.cpu().numpy(), b) <= BWD_TOL
+
+
 def test_graph_without_edges():
     """E = 0: zeros out, no edge array needed; and receivers without edges inside a graph give zero rows."""
     import torch
