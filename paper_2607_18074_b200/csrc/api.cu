@@ -324,6 +324,11 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
     const EdgeView rv = receiver_view(g);
+    if (p->uvu && p->ud.ok && !p->uvu_state_fwd && !geo && order == 0) {
+        // channelwise mode, uniform natural-parity profile: the direct kernel (no state, no node-side pass)
+        CK(launch_uvu_direct_fwd(p, g, x, Y, phi, R, y, w.status, s));
+        return SOBEK_OK;
+    }
     if (w.fused_f) {
         CK(launch_pack_R_fused(p, p->fwd, 0, R, w.fFKh, w.fFKl, s));
         CK(launch_fused(p, p->fwd, rv, x, nullptr, Y, nullptr, phi, nullptr, 0, w.fFKh, w.fFKl, y, 0, w.status, s));

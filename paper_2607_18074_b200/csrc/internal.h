@@ -224,6 +224,18 @@ struct HPath {
 
 }  // namespace sobek
 
+// Direct forward of the channelwise mode (uvu_direct.cu): tables in the kernel's static path order
+struct UvuDirect {
+    bool ok = false;
+    int L = 0, C = 0, n_paths = 0, nM = 0;
+    std::vector<int32_t> woff;      // per path: first weight column
+    std::vector<int2> ent;          // per coupling-matrix entry: {first sparse term, number of terms}
+    std::vector<int2> nz;           // sparse terms: {index into a Y row, coefficient bits}
+    int32_t* d_woff = nullptr;
+    int2* d_ent = nullptr;
+    int2* d_nz = nullptr;
+};
+
 struct sobek_plan {
     std::vector<sobek_irrep> in, out;
     int l_max = 0, K = 0;
@@ -247,6 +259,8 @@ struct sobek_plan {
     int4* d_in_blocks = nullptr;    // {offset, multiplicity, 2l+1, 0} of the irrep blocks of x / of y (device), for the re-layout
     int4* d_out_blocks = nullptr;
     bool uvu = false;         // channelwise mode (Eq. uvu_connection): tied multiplicities, C_in weights per path
+    UvuDirect ud;             // its direct forward kernel, where the profile allows it
+    bool uvu_state_fwd = false;   // SOBEK_FLAG_UVU_STATE_FWD: forward through the receiver state even so
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -422,6 +436,10 @@ cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s)
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
 
+// --- uvu_direct.cu ------------------------------------------------------------------------
+void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out);
+cudaError_t launch_uvu_direct_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
+                                  const float* phi, const float* R, float* y, int* status, cudaStream_t s);
 // --- node_uvu.cu: the node-side steps of the channelwise mode (no GEMM) ---------------
 cudaError_t launch_uvu_mix(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
                            const void* zl, const float* R, float* dst, int accumulate, cudaStream_t s0);

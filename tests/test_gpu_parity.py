@@ -565,6 +565,19 @@ def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases):
         assert rel_err(got, ref) <= BWD_TOL
 
 
+@pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16"])
+def test_uvu_direct_forward_and_state_route_agree(name):
+    """Uniform natural-parity profiles take the direct channelwise forward kernel by default; the route through the
+    receiver state (SOBEK_FLAG_UVU_STATE_FWD) computes the same thing.  Both against the oracle."""
+    c = Case(UVU[name])
+    s = Case(UVU[name], inputs=c.d, uvu_state_fwd=True)
+    ref = c.o_fwd()
+    y_direct, y_state = c.fwd(), s.fwd()
+    assert rel_err(y_direct, ref) <= FWD_TOL and rel_err(y_state, ref) <= FWD_TOL
+    assert not np.array_equal(y_direct, y_state)        # two different kernels did run
+    assert np.array_equal(y_direct, c.fwd())            # and the direct one repeats bitwise
+
+
 def test_uvu_full_size_sampled():
     """The paper's 128/128/128 channelwise profile (K = 16) on 31 copies of its 128-node graph."""
     FULL["uvu_128x3_31"] = (synth.config("uvu_128x3_31"), 6, (0, 1, 2))
@@ -710,7 +723,8 @@ def test_state_retained_from_forward(name, mode):
     from it without streaming the edges again: same bits as the plain calls, one stream launch fewer."""
     import torch
     import paper_2607_18074_b200 as sb
-    c = Case((UVU if mode == "uvu" else CASES)[name])
+    # (a retaining forward goes through the state in either mode; the plain uvu forward compared with it must too)
+    c = Case(UVU[name], uvu_state_fwd=True) if mode == "uvu" else Case(CASES[name])
     i = c.plan.info
     y_ref, b_ref = c.fwd(), c.bwd()
     new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")
