@@ -83,7 +83,7 @@ enum { SOBEK_MAX_L = 4 };
 #define SOBEK_FLAG_FUSED_FP32 8u   /* schedule: FP32-pipe edge stream feeding the tensor core inside one kernel */
 #define SOBEK_FLAG_FP32_STREAM 16u /* edge stream on the FP32 pipes even where the tensor-core kernel applies */
 #define SOBEK_FLAG_FP32_EDGE 32u   /* edge pass on the FP32 pipes even where the tensor-core kernel applies */
-#define SOBEK_FLAG_UVU_STATE_FWD 64u /* channelwise mode: forward through the receiver state even where the direct kernel applies */
+#define SOBEK_FLAG_UVU_STATE 64u   /* channelwise mode: y and gx through the receiver state even where the direct kernel applies */
 /* scratch budget in MiB (1 .. 2^20 - 1) in bits 12..31 of the flags word; 0 = the default */
 #define SOBEK_FLAG_STATE_BUDGET_MIB(mb) (((uint32_t)(mb) & 0xFFFFFu) << 12)
 

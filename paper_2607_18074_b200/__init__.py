@@ -22,7 +22,7 @@ FLAG_FAST_GEMM = 4  # SOBEK_FLAG_FAST_GEMM: node-side GEMMs as plain bf16 produc
 FLAG_FUSED_FP32 = 8    # SOBEK_FLAG_FUSED_FP32: fused FP32-pipe stream + contraction schedule
 FLAG_FP32_STREAM = 16  # SOBEK_FLAG_FP32_STREAM: edge stream on the FP32 pipes
 FLAG_FP32_EDGE = 32    # SOBEK_FLAG_FP32_EDGE: edge pass on the FP32 pipes
-FLAG_UVU_STATE_FWD = 64    # SOBEK_FLAG_UVU_STATE_FWD: channelwise forward through the receiver state
+FLAG_UVU_STATE = 64        # SOBEK_FLAG_UVU_STATE: channelwise y and gx through the receiver state
 
 
 def flag_state_budget_mib(mb: int) -> int:
@@ -158,12 +158,12 @@ class Plan:
     connected multiplicity mixing, "uvu" the channelwise one (SOBEK_FLAG_UVU).  layout "ir_mul" (block offset +
     m*mul + u) is the kernels' own order of node features, "mul_ir" (block offset + u*(2l+1) + m) is transposed at the
     boundary (SOBEK_FLAG_MUL_IR).  fused / tc_stream / tc_edge / state_budget_mib map to SOBEK_FLAG_FUSED_FP32,
-    SOBEK_FLAG_FP32_STREAM, SOBEK_FLAG_FP32_EDGE and SOBEK_FLAG_STATE_BUDGET_MIB; uvu_state_fwd to
-    SOBEK_FLAG_UVU_STATE_FWD (channelwise forward through the receiver state even where the direct kernel applies)."""
+    SOBEK_FLAG_FP32_STREAM, SOBEK_FLAG_FP32_EDGE and SOBEK_FLAG_STATE_BUDGET_MIB; uvu_state to
+    SOBEK_FLAG_UVU_STATE (channelwise y and gx through the receiver state even where the direct kernel applies)."""
 
     def __init__(self, irreps_in, irreps_out, l_max: int, K: int, flags: int = 0, mode: str = "uvw",
                  layout: str = "ir_mul", fused: bool = False, tc_stream: bool = True, tc_edge: bool = True,
-                 state_budget_mib: int | None = None, uvu_state_fwd: bool = False):
+                 state_budget_mib: int | None = None, uvu_state: bool = False):
         if mode not in ("uvw", "uvu"):
             raise ValueError(mode)
         if layout not in ("ir_mul", "mul_ir"):
@@ -180,8 +180,8 @@ class Plan:
             flags |= FLAG_FP32_EDGE
         if state_budget_mib is not None:
             flags |= flag_state_budget_mib(state_budget_mib)
-        if uvu_state_fwd:
-            flags |= FLAG_UVU_STATE_FWD
+        if uvu_state:
+            flags |= FLAG_UVU_STATE
         self.layout = "mul_ir" if flags & FLAG_MUL_IR else "ir_mul"
         self.mode = "uvu" if flags & FLAG_UVU else "uvw"
         self._h = c_void_p()

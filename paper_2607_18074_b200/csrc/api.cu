@@ -324,9 +324,9 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     if (g->E == 0 || has_uncovered(p->fwd)) CK(launch_fill_zero(y, g->N * (int64_t)p->C_y, s));
     if (g->E == 0) return SOBEK_OK;
     const EdgeView rv = receiver_view(g);
-    if (p->uvu && p->ud.ok && !p->uvu_state_fwd && !geo && order == 0) {
+    if (p->uvu && p->ud.ok && !p->uvu_state && !geo && order == 0) {
         // channelwise mode, uniform natural-parity profile: the direct kernel (no state, no node-side pass)
-        CK(launch_uvu_direct_fwd(p, g, x, Y, phi, R, y, w.status, s));
+        CK(launch_uvu_direct(p, rv, 0, x, Y, phi, R, y, w.status, s));
         return SOBEK_OK;
     }
     if (w.fused_f) {
@@ -373,8 +373,9 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     const bool g_edge = geo && geo->g_rvec;       // geometry mode: the edge pass writes the adjoint of the edge vectors
     if (g_edge) { gphi = geo->g_rvec; gY = geo->g_rvec; }      // (stand-ins: "wanted"; the kernel writes g_rvec only)
     const bool tc_edge = w.zqh != nullptr;
+    const bool gx_direct = p->uvu && p->ud.ok && !p->uvu_state && !geo && g->src_recv;      // channelwise mode: no state for gx
     if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
-    if (w.gsh && gx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
+    if (w.gsh && gx && !w.fused_t && !gx_direct) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (gR || gphi || gY) {
         if (gphi || gY) CK(pack_R(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
         if (gR) CK(launch_fill_zero(w.gRp, KN, s));
@@ -403,7 +404,10 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     if (gx) {
         if (has_uncovered(p->tr)) CK(launch_fill_zero(gx, g->N * (int64_t)p->C_x, s));
         const EdgeView sv = sender_view(g);
-        if (w.fused_t) {
+        if (gx_direct) {
+            // channelwise mode, uniform natural-parity profile: the direct kernel on the sender view
+            CK(launch_uvu_direct(p, sv, 1, gy, Y, phi, R, gx, w.status, s));
+        } else if (w.fused_t) {
             CK(launch_pack_R_fused(p, p->tr, 1, R, w.tFKh, w.tFKl, s));
             CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.tFKh, w.tFKl, gx, 0, w.status, s));
         } else {

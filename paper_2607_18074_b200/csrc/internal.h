@@ -225,15 +225,18 @@ struct HPath {
 }  // namespace sobek
 
 // Direct forward of the channelwise mode (uvu_direct.cu): tables in the kernel's static path order
-struct UvuDirect {
-    bool ok = false;
-    int L = 0, C = 0, n_paths = 0, nM = 0;
+struct UvuDirectTables {
     std::vector<int32_t> woff;      // per path: first weight column
-    std::vector<int2> ent;          // per coupling-matrix entry: {first sparse term, number of terms}
+    std::vector<int2> ent;          // per stored coupling-matrix entry: {offset in the padded M_e | terms << 16, first term}
     std::vector<int2> nz;           // sparse terms: {index into a Y row, coefficient bits}
     int32_t* d_woff = nullptr;
     int2* d_ent = nullptr;
     int2* d_nz = nullptr;
+};
+struct UvuDirect {
+    bool ok = false;
+    int L = 0, C = 0;
+    UvuDirectTables dir[2];         // [0] y from x on the receiver view, [1] gx from gy on the sender view
 };
 
 struct sobek_plan {
@@ -259,8 +262,8 @@ struct sobek_plan {
     int4* d_in_blocks = nullptr;    // {offset, multiplicity, 2l+1, 0} of the irrep blocks of x / of y (device), for the re-layout
     int4* d_out_blocks = nullptr;
     bool uvu = false;         // channelwise mode (Eq. uvu_connection): tied multiplicities, C_in weights per path
-    UvuDirect ud;             // its direct forward kernel, where the profile allows it
-    bool uvu_state_fwd = false;   // SOBEK_FLAG_UVU_STATE_FWD: forward through the receiver state even so
+    UvuDirect ud;             // its direct kernel (y and gx), where the profile allows it
+    bool uvu_state = false;   // SOBEK_FLAG_UVU_STATE: through the receiver state even so
     bool use_fused = false;   // schedule choice: fused stream+contraction kernels vs. stream -> state -> GEMM
     // side streams used to run independent kernels of one call concurrently (joined back into the
     // caller's stream before the call returns control of ordering)
@@ -438,8 +441,9 @@ constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its p
 
 // --- uvu_direct.cu ------------------------------------------------------------------------
 void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out);
-cudaError_t launch_uvu_direct_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
-                                  const float* phi, const float* R, float* y, int* status, cudaStream_t s);
+// transposed = 0: y[N, C_y] from src = x on the receiver view; 1: gx[N, C_x] from src = gy on the sender view
+cudaError_t launch_uvu_direct(const sobek_plan* p, const EdgeView& ev, int transposed, const float* src, const float* Y,
+                              const float* phi, const float* R, float* dst, int* status, cudaStream_t s);
 // --- node_uvu.cu: the node-side steps of the channelwise mode (no GEMM) ---------------
 cudaError_t launch_uvu_mix(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
                            const void* zl, const float* R, float* dst, int accumulate, cudaStream_t s0);

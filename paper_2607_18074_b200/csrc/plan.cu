@@ -385,7 +385,7 @@ using namespace sobek;
 
 extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out,
                                  int l_max, int K, uint32_t flags, sobek_plan** plan) {
-    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & 0xFFFu & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR | SOBEK_FLAG_FAST_GEMM | SOBEK_FLAG_FUSED_FP32 | SOBEK_FLAG_FP32_STREAM | SOBEK_FLAG_FP32_EDGE | SOBEK_FLAG_UVU_STATE_FWD)) != 0 || l_max < 0)
+    if (!in || !out || !plan || n_in < 1 || n_out < 1 || K < 1 || (flags & 0xFFFu & ~uint32_t(SOBEK_FLAG_UVU | SOBEK_FLAG_MUL_IR | SOBEK_FLAG_FAST_GEMM | SOBEK_FLAG_FUSED_FP32 | SOBEK_FLAG_FP32_STREAM | SOBEK_FLAG_FP32_EDGE | SOBEK_FLAG_UVU_STATE)) != 0 || l_max < 0)
         return SOBEK_ERR_INVALID_ARG;
     *plan = nullptr;
     if (l_max > SOBEK_MAX_L) return SOBEK_ERR_UNSUPPORTED;
@@ -463,7 +463,7 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     build_tc_sets(p, p->fwd);
     build_tc_sets(p, p->tr);
     build_tc_edge_sets(p, p->fwd);
-    p->uvu_state_fwd = (flags & SOBEK_FLAG_UVU_STATE_FWD) != 0;
+    p->uvu_state = (flags & SOBEK_FLAG_UVU_STATE) != 0;
     build_uvu_direct(p, in, n_in, out, n_out);
     build_edge_tasks(p, p->fwd);
     build_fused_stages(p, p->fwd);
@@ -481,9 +481,11 @@ extern "C" int sobek_plan_create(const sobek_irrep* in, int n_in, const sobek_ir
     if (e == cudaSuccess) e = upload(p->tab_idx, &p->d_tab_idx);
     if (e == cudaSuccess) e = upload(p->tab_coef, &p->d_tab_coef);
     if (p->ud.ok) {
-        if (e == cudaSuccess) e = upload(p->ud.woff, &p->ud.d_woff);
-        if (e == cudaSuccess) e = upload(p->ud.ent, &p->ud.d_ent);
-        if (e == cudaSuccess) e = upload(p->ud.nz, &p->ud.d_nz);
+        for (UvuDirectTables& T : p->ud.dir) {
+            if (e == cudaSuccess) e = upload(T.woff, &T.d_woff);
+            if (e == cudaSuccess) e = upload(T.ent, &T.d_ent);
+            if (e == cudaSuccess) e = upload(T.nz, &T.d_nz);
+        }
     }
     {
         std::vector<int4> bi, bo;
@@ -553,7 +555,7 @@ extern "C" void sobek_plan_destroy(sobek_plan* p) {
     }
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     cudaFree(p->d_tab_ptr); cudaFree(p->d_tab_idx); cudaFree(p->d_tab_coef);
-    cudaFree(p->ud.d_woff); cudaFree(p->ud.d_ent); cudaFree(p->ud.d_nz);
+    for (UvuDirectTables& T : p->ud.dir) { cudaFree(T.d_woff); cudaFree(T.d_ent); cudaFree(T.d_nz); }
     cudaFree(p->d_in_blocks); cudaFree(p->d_out_blocks);
     for (Direction* d : {&p->fwd, &p->tr}) {
         cudaFree(d->d_paths); cudaFree(d->d_groups); cudaFree(d->d_wtasks);

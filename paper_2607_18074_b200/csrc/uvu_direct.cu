@@ -1,4 +1,4 @@
-// Direct forward of the channelwise (uvu) mode (Eq. uvu_connection), for profiles  C x 0e + C x 1o + ... + C x L  on
+// Direct kernel of the channelwise (uvu) mode (Eq. uvu_connection): y and gx, for profiles  C x 0e + C x 1o + ... + C x L  on
 // both sides with l_max = L:
 //   y_i[l_out, u, o] = sum_{e into i} sum_{paths (l_in, l_sh, l_out)} w_e[pi, u] * sum_a M_e^pi[a, o] x_{j(e)}[l_in, u, a],
 //   w_e[pi, u] = sum_q phi_e[q] R[q, w_off(pi) + u],        M_e^pi[a, o] = sum_b c^pi[a, b, o] Y_e[b].
@@ -21,6 +21,11 @@
 //                       contraction, with rows of M_e as broadcast 16-byte shared loads.
 // M_e per path is stored row-padded to four floats in the orientation with fewer rows to load; a path with
 // l_sh = 0 is a multiple of the identity and keeps one number.
+//
+// The input adjoint of the same operator, gx_j[l_in, u, a] = sum_{e out of j} sum_paths w_e[pi, u] sum_o M_e^pi[a, o]
+// gy_{i(e)}[l_out, u, o] (Eq. adjoints, channelwise), is the same kernel on the sender view of the graph: segments of
+// the senders, the receivers' gy rows gathered, phi and Y rows through the view's edge permutation, and host-built
+// tables in which the walk position (l_a, l_sh, l_b) stands for the path (l_in = l_b, l_out = l_a) with M_e transposed.
 #include <cuda_runtime.h>
 
 #include <string.h>
@@ -40,14 +45,15 @@ constexpr int KMAX = 16;
 constexpr int R_REG_BUDGET = 176;   // weights a thread may hold in registers
 
 struct UdArgs {
-    const int64_t* row_ptr;
-    const int32_t* col;
+    const int64_t* row_ptr;     // segments of the owning node (receivers; senders on the sender view)
+    const int32_t* ids;         // per position: the node whose row is gathered
+    const int32_t* perm;        // per position: the edge id (NULL: the position itself)
     int64_t N, E;
-    const float* x;
+    const float* x;             // gathered rows (x; gy on the sender view)
     const float* Y;
     const float* phi;
     const float* R;
-    float* y;
+    float* y;                   // rows of the owning nodes (y; gx on the sender view)
     const int32_t* woff;        // per path (static order): first weight column
     const int2* ent;            // per stored M entry: {offset in the padded M_e | number of terms << 16, first term}
     const int2* nz;             // terms: {index b into a Y row, coefficient bits}
@@ -95,6 +101,7 @@ struct UdSmem {           // carved from dynamic shared memory; every part a mul
     float* phi;           // [3][TB][KP]
     float* Y;             // [3][TB][DT]
     int32_t* sid;         // [3][TB]
+    int32_t* eid;         // [4][TB] edge ids of a batch (sender view), in step with desc
     float* M;             // [2][TB][MF]
     float* X;             // [2][TB][DT * C]
     float* out;           // [NG - 1][DT * C]
@@ -159,6 +166,8 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                 if (last) w_open = false;
             }
             sm.desc[d_slot] = d;
+            if (a.perm && d.w >= 0)
+                for (int i = 0; i < (d.z & 255); ++i) cp_async4(sm.eid + d_slot * TB + i, a.perm + (w_pos - (d.z & 255)) + i);
         }
         // ---- A: edge inputs of batch it + 2
         if (it >= -2) {
@@ -168,12 +177,18 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                 const int nb = d.z & 255;
                 float* dphi = sm.phi + r_slot2 * (TB * KP);
                 float* dY = sm.Y + r_slot2 * (TB * DT);
+                const int32_t* eid = sm.eid + ((d_slot + 3) & 3) * TB;
                 for (int i = tid; i < nb * KP; i += NT) {
                     const int e = i / KP, q = i - e * KP;
-                    if (q < a.K) cp_async4(dphi + i, a.phi + (b0 + e) * a.K + q);
+                    const int64_t ee = a.perm ? (int64_t)eid[e] : b0 + e;
+                    if (q < a.K && id_ok(ee, a.E, a.status)) cp_async4(dphi + i, a.phi + ee * a.K + q);
                 }
-                for (int i = tid; i < nb * DT; i += NT) cp_async4(dY + i, a.Y + b0 * DT + i);
-                if (tid < nb) cp_async4(sm.sid + r_slot2 * TB + tid, a.col + b0 + tid);
+                for (int i = tid; i < nb * DT; i += NT) {
+                    const int e = i / DT, b = i - e * DT;
+                    const int64_t ee = a.perm ? (int64_t)eid[e] : b0 + e;
+                    if (id_ok(ee, a.E, a.status)) cp_async4(dY + i, a.Y + ee * DT + b);
+                }
+                if (tid < nb) cp_async4(sm.sid + r_slot2 * TB + tid, a.ids + b0 + tid);
             }
         }
         // ---- B, C: sender rows and coupling matrices of batch it + 1
@@ -329,6 +344,7 @@ __global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
     sm.phi = reinterpret_cast<float*>(p); p += 3 * TB * KP * 4;
     sm.Y = reinterpret_cast<float*>(p); p += pad4(3 * TB * DT) * 4;
     sm.sid = reinterpret_cast<int32_t*>(p); p += 3 * TB * 4;
+    sm.eid = reinterpret_cast<int32_t*>(p); p += 4 * TB * 4;
     sm.M = reinterpret_cast<float*>(p); p += 2 * TB * MF * 4;
     sm.X = reinterpret_cast<float*>(p); p += (size_t)2 * TB * DT * C * 4;
     sm.out = reinterpret_cast<float*>(p); p += (size_t)(NG - 1) * DT * C * 4;
@@ -362,59 +378,68 @@ void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobe
         if (in[i].l != i || out[i].l != i || in[i].mul != C || out[i].mul != C || in[i].parity != par || out[i].parity != par) return;
     }
     const Direction& dir = p->fwd;
-    std::vector<int32_t> woff;
-    std::vector<int2> ent, nz;
-    int mo = 0;
-    for (int li = 0; li <= L; ++li)
-        for (int ls = 0; ls <= L; ++ls)
-            for (int lo = 0; lo <= L; ++lo) {
-                if (!path_ok(li, ls, lo, L)) continue;
-                const DPath* P = nullptr;
-                for (size_t gi = 0; gi < dir.groups.size() && !P; ++gi) {
-                    const DGroup& G = dir.groups[gi];
-                    if (G.dst_off != lo * lo * C || G.d_dst != 2 * lo + 1) continue;
-                    for (int k = G.path_begin; k < G.path_end; ++k) {
-                        const DPath& Q = dir.paths[k];
-                        if (Q.src_off == li * li * C && Q.d_src == 2 * li + 1 && Q.sh_off == ls * ls && Q.d_sh == 2 * ls + 1) { P = &Q; break; }
-                    }
-                }
-                if (!P || P->c_src != C || P->c_dst != C) return;
-                woff.push_back((int32_t)P->w_off);
-                const int di = P->d_src, dO = P->d_dst;
-                auto terms = [&](int s, int o) { const int t = P->tabM + s * dO + o; return std::make_pair(p->tab_ptr[t], p->tab_ptr[t + 1]); };
-                auto emit = [&](int s, int o, int dst) {
-                    const auto [k0, k1] = terms(s, o);
-                    ent.push_back(make_int2(dst | ((k1 - k0) << 16), (int)nz.size()));
-                    for (int k = k0; k < k1; ++k) {
-                        int bits; const float cf = p->tab_coef[k]; memcpy(&bits, &cf, 4);
-                        nz.push_back(make_int2(P->sh_off + p->tab_idx[k], bits));
-                    }
-                };
-                if (ls == 0) {
-                    // an equivariant map between equal irreps is a multiple of the identity; the kernel keeps only
-                    // that multiple, so check that the table says the same
-                    const auto [a0, a1] = terms(0, 0);
-                    if (a1 - a0 != 1) return;
-                    for (int s = 0; s < di; ++s)
-                        for (int o = 0; o < dO; ++o) {
-                            const auto [k0, k1] = terms(s, o);
-                            if (s != o) { if (k1 != k0) return; continue; }
-                            if (k1 - k0 != 1 || p->tab_idx[k0] != p->tab_idx[a0] ||
-                                std::fabs(p->tab_coef[k0] - p->tab_coef[a0]) > 1e-6f * std::fabs(p->tab_coef[a0])) return;
+    for (int tr = 0; tr < 2; ++tr) {
+        // tr = 1: the walk position (la, ls, lb) stands for the path (l_in = lb, l_sh = ls, l_out = la), whose coupling
+        // matrix is used transposed: gx_j[l_in, u, a] += w_e M_e[a, o] gy_i[l_out, u, o]
+        std::vector<int32_t> woff;
+        std::vector<int2> ent, nz;
+        int mo = 0;
+        for (int la = 0; la <= L; ++la)
+            for (int ls = 0; ls <= L; ++ls)
+                for (int lb = 0; lb <= L; ++lb) {
+                    if (!path_ok(la, ls, lb, L)) continue;
+                    const int li = tr ? lb : la, lo = tr ? la : lb;
+                    const DPath* P = nullptr;
+                    for (size_t gi = 0; gi < dir.groups.size() && !P; ++gi) {
+                        const DGroup& G = dir.groups[gi];
+                        if (G.dst_off != lo * lo * C || G.d_dst != 2 * lo + 1) continue;
+                        for (int k = G.path_begin; k < G.path_end; ++k) {
+                            const DPath& Q = dir.paths[k];
+                            if (Q.src_off == li * li * C && Q.d_src == 2 * li + 1 && Q.sh_off == ls * ls && Q.d_sh == 2 * ls + 1) { P = &Q; break; }
                         }
-                    emit(0, 0, mo);
-                } else if (!m_transposed(di, dO)) {
-                    for (int s = 0; s < di; ++s)
-                        for (int o = 0; o < dO; ++o) emit(s, o, mo + s * pad4(dO) + o);
-                } else {
-                    for (int s = 0; s < di; ++s)
-                        for (int o = 0; o < dO; ++o) emit(s, o, mo + o * pad4(di) + s);
+                    }
+                    if (!P || P->c_src != C || P->c_dst != C) return;
+                    woff.push_back((int32_t)P->w_off);
+                    const int dA = 2 * la + 1, dB = 2 * lb + 1;      // gathered side, accumulated side
+                    // sparse terms of the entry (a, b) of the walk's matrix
+                    auto terms = [&](int ia, int ib) {
+                        const int t = P->tabM + (tr ? ib * P->d_dst + ia : ia * P->d_dst + ib);
+                        return std::make_pair(p->tab_ptr[t], p->tab_ptr[t + 1]);
+                    };
+                    auto emit = [&](int ia, int ib, int dst) {
+                        const auto [k0, k1] = terms(ia, ib);
+                        ent.push_back(make_int2(dst | ((k1 - k0) << 16), (int)nz.size()));
+                        for (int k = k0; k < k1; ++k) {
+                            int bits; const float cf = p->tab_coef[k]; memcpy(&bits, &cf, 4);
+                            nz.push_back(make_int2(P->sh_off + p->tab_idx[k], bits));
+                        }
+                    };
+                    if (ls == 0) {
+                        // an equivariant map between equal irreps is a multiple of the identity; the kernel keeps only
+                        // that multiple, so check that the table says the same
+                        const auto [a0, a1] = terms(0, 0);
+                        if (a1 - a0 != 1) return;
+                        for (int ia = 0; ia < dA; ++ia)
+                            for (int ib = 0; ib < dB; ++ib) {
+                                const auto [k0, k1] = terms(ia, ib);
+                                if (ia != ib) { if (k1 != k0) return; continue; }
+                                if (k1 - k0 != 1 || p->tab_idx[k0] != p->tab_idx[a0] ||
+                                    std::fabs(p->tab_coef[k0] - p->tab_coef[a0]) > 1e-6f * std::fabs(p->tab_coef[a0])) return;
+                            }
+                        emit(0, 0, mo);
+                    } else if (!m_transposed(dA, dB)) {
+                        for (int ia = 0; ia < dA; ++ia)
+                            for (int ib = 0; ib < dB; ++ib) emit(ia, ib, mo + ia * pad4(dB) + ib);
+                    } else {
+                        for (int ia = 0; ia < dA; ++ia)
+                            for (int ib = 0; ib < dB; ++ib) emit(ia, ib, mo + ib * pad4(dA) + ia);
+                    }
+                    mo += m_block(la, ls, lb);
                 }
-                mo += m_block(li, ls, lo);
-            }
-    if (woff.size() != dir.paths.size() || mo != m_floats_c(L) || mo >= 65536 || nz.size() >= 32768) return;
-    D.L = L; D.C = C; D.n_paths = (int)woff.size(); D.nM = (int)ent.size();
-    D.woff = woff; D.ent = ent; D.nz = nz;
+        if (woff.size() != dir.paths.size() || mo != m_floats_c(L) || mo >= 65536 || nz.size() >= 32768) return;
+        D.dir[tr].woff = woff; D.dir[tr].ent = ent; D.dir[tr].nz = nz;
+    }
+    D.L = L; D.C = C;
     D.ok = true;
 }
 
@@ -423,7 +448,7 @@ template <int L, int KP>
 cudaError_t launch_ud(const UdArgs& a, size_t tables, cudaStream_t s) {
     constexpr int DT = (L + 1) * (L + 1), NG = n_groups_c(L, KP), MF = m_floats_c(L);
     const int NT = a.C * NG;
-    const size_t sh = 4 * sizeof(int4) + (size_t)3 * TB * KP * 4 + (size_t)pad4(3 * TB * DT) * 4 + 3 * TB * 4 + (size_t)2 * TB * MF * 4 +
+    const size_t sh = 4 * sizeof(int4) + (size_t)3 * TB * KP * 4 + (size_t)pad4(3 * TB * DT) * 4 + 7 * TB * 4 + (size_t)2 * TB * MF * 4 +
                       (size_t)2 * TB * DT * a.C * 4 + (size_t)(NG - 1) * DT * a.C * 4 + tables;
     auto kern = k_uvu_direct_fwd<L, KP>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
@@ -441,17 +466,18 @@ cudaError_t launch_ud(const UdArgs& a, size_t tables, cudaStream_t s) {
 }
 }  // namespace
 
-cudaError_t launch_uvu_direct_fwd(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
-                                  const float* phi, const float* R, float* y, int* status, cudaStream_t s) {
+cudaError_t launch_uvu_direct(const sobek_plan* p, const EdgeView& ev, int transposed, const float* src, const float* Y,
+                              const float* phi, const float* R, float* dst, int* status, cudaStream_t s) {
     const UvuDirect& D = p->ud;
-    if (!D.ok || !D.d_woff || !D.d_ent || !D.d_nz) return cudaErrorInvalidValue;
+    const UvuDirectTables& T = D.dir[transposed ? 1 : 0];
+    if (!D.ok || !T.d_woff || !T.d_ent || !T.d_nz || (transposed && (!ev.perm || !ev.recv))) return cudaErrorInvalidValue;
     UdArgs a{};
-    a.row_ptr = g->row_ptr; a.col = g->col; a.N = g->N; a.E = g->E;
-    a.x = x; a.Y = Y; a.phi = phi; a.R = R; a.y = y;
-    a.woff = D.d_woff; a.ent = D.d_ent; a.nz = D.d_nz; a.n_nz = (int32_t)D.nz.size();
-    a.C = D.C; a.K = p->K; a.nM = D.nM; a.N_w = (int32_t)p->N_w;
-    a.C_x = p->C_x; a.C_y = p->C_y; a.status = status;
-    const size_t tables = (size_t)(D.nM + D.nz.size()) * 8 + 16;
+    a.row_ptr = ev.ptr; a.ids = transposed ? ev.recv : ev.col; a.perm = transposed ? ev.perm : nullptr; a.N = ev.N; a.E = ev.E;
+    a.x = src; a.Y = Y; a.phi = phi; a.R = R; a.y = dst;
+    a.woff = T.d_woff; a.ent = T.d_ent; a.nz = T.d_nz; a.n_nz = (int32_t)T.nz.size();
+    a.C = D.C; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
+    a.C_x = transposed ? p->C_y : p->C_x; a.C_y = transposed ? p->C_x : p->C_y; a.status = status;
+    const size_t tables = (size_t)(T.ent.size() + T.nz.size()) * 8 + 16;
     KernelTimer kt(K_STATE, s);
     const bool k8 = p->K <= 8;
     cudaError_t e;

@@ -566,16 +566,24 @@ def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases):
 
 
 @pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16"])
-def test_uvu_direct_forward_and_state_route_agree(name):
-    """Uniform natural-parity profiles take the direct channelwise forward kernel by default; the route through the
-    receiver state (SOBEK_FLAG_UVU_STATE_FWD) computes the same thing.  Both against the oracle."""
+def test_uvu_direct_and_state_route_agree(name):
+    """Uniform natural-parity profiles take the direct channelwise kernel for y and gx by default; the route through
+    the receiver state (SOBEK_FLAG_UVU_STATE) computes the same thing.  Both against the oracle."""
     c = Case(UVU[name])
-    s = Case(UVU[name], inputs=c.d, uvu_state_fwd=True)
+    s = Case(UVU[name], inputs=c.d, uvu_state=True)
     ref = c.o_fwd()
     y_direct, y_state = c.fwd(), s.fwd()
     assert rel_err(y_direct, ref) <= FWD_TOL and rel_err(y_state, ref) <= FWD_TOL
     assert not np.array_equal(y_direct, y_state)        # two different kernels did run
     assert np.array_equal(y_direct, c.fwd())            # and the direct one repeats bitwise
+    b_direct, b_state, b_ref = c.bwd(), s.bwd(), c.o_bwd()
+    for got in (b_direct, b_state):
+        for g, r in zip(got, b_ref):
+            assert rel_err(g, r) <= BWD_TOL
+    assert not np.array_equal(b_direct[0], b_state[0])
+    assert np.array_equal(b_direct[0], c.bwd()[0])
+    for g, r in zip(b_direct[1:], b_state[1:]):         # gY, gphi, gR take the same kernels on both plans
+        assert np.array_equal(g, r)
 
 
 def test_uvu_full_size_sampled():
@@ -724,7 +732,7 @@ def test_state_retained_from_forward(name, mode):
     import torch
     import paper_2607_18074_b200 as sb
     # (a retaining forward goes through the state in either mode; the plain uvu forward compared with it must too)
-    c = Case(UVU[name], uvu_state_fwd=True) if mode == "uvu" else Case(CASES[name])
+    c = Case(UVU[name], uvu_state=True) if mode == "uvu" else Case(CASES[name])
     i = c.plan.info
     y_ref, b_ref = c.fwd(), c.bwd()
     new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")

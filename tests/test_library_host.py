@@ -200,7 +200,7 @@ def test_graph_descriptor_keeps_its_tensors_alive():
 
 def test_plan_option_flags():
     ir = [(8, 0, 1), (8, 1, -1)]
-    for kw in (dict(fused=True), dict(tc_stream=False), dict(tc_edge=False), dict(state_budget_mib=128)):
+    for kw in (dict(fused=True), dict(tc_stream=False), dict(tc_edge=False), dict(state_budget_mib=128), dict(mode="uvu", uvu_state=True)):
         sb.Plan(ir, ir, 2, 8, **kw)
     with pytest.raises(sb.SobekError):
         sb.Plan(ir, ir, 2, 8, flags=1 << 11)            # an undefined flag bit
