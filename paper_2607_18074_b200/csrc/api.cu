@@ -374,6 +374,14 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     if (g_edge) { gphi = geo->g_rvec; gY = geo->g_rvec; }      // (stand-ins: "wanted"; the kernel writes g_rvec only)
     const bool tc_edge = w.zqh != nullptr;
     const bool gx_direct = p->uvu && p->ud.ok && !p->uvu_state && !geo && g->src_recv;      // channelwise mode: no state for gx
+    const bool gR_direct = gR && p->uvu && p->ud.ok && !p->uvu_state && !geo && !z_valid;   // nor for gR
+    if (gR_direct) {
+        int n_parts = 0;
+        CK(launch_fill_zero(gR, KN, s));
+        CK(launch_uvu_direct_wgrad(p, rv, x, Y, phi, gy, w.part, w.splits, &n_parts, w.status, s));
+        CK(launch_reduce_parts(gR, w.part, KN, KN, n_parts, s));
+        gR = nullptr;
+    }
     if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     if (w.gsh && gx && !w.fused_t && !gx_direct) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
     if (gR || gphi || gY) {

@@ -444,6 +444,9 @@ void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobe
 // transposed = 0: y[N, C_y] from src = x on the receiver view; 1: gx[N, C_x] from src = gy on the sender view
 cudaError_t launch_uvu_direct(const sobek_plan* p, const EdgeView& ev, int transposed, const float* src, const float* Y,
                               const float* phi, const float* R, float* dst, int* status, cudaStream_t s);
+// part[0 .. *n_parts)[K * N_w]: per-CTA sums of the weight adjoint gR over the receivers (receiver view only)
+cudaError_t launch_uvu_direct_wgrad(const sobek_plan* p, const EdgeView& ev, const float* x, const float* Y, const float* phi,
+                                    const float* gy, float* part, int max_parts, int* n_parts, int* status, cudaStream_t s);
 // --- node_uvu.cu: the node-side steps of the channelwise mode (no GEMM) ---------------
 cudaError_t launch_uvu_mix(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
                            const void* zl, const float* R, float* dst, int accumulate, cudaStream_t s0);
@@ -452,7 +455,7 @@ cudaError_t launch_uvu_zbar(const sobek_plan* p, const Direction& dir, int64_t n
 cudaError_t launch_uvu_wgrad(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const void* zh,
                              const void* zl, const float* gy, float* gR_acc, float* part, int splits,
                              cudaStream_t s0);
-constexpr int kMaxSplitsUvu = 256;                             // node slices of the channelwise weight adjoint
+constexpr int kMaxSplitsUvu = 512;                             // node slices of the channelwise weight adjoint
 
 // --- graph.cu -----------------------------------------------------------------------
 size_t graph_prepare_bytes(int64_t N, int64_t E);

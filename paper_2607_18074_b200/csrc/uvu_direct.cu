@@ -54,6 +54,8 @@ struct UdArgs {
     const float* phi;
     const float* R;
     float* y;                   // rows of the owning nodes (y; gx on the sender view)
+    const float* own;           // weight adjoint: rows of the owning nodes that are read (gy), else NULL
+    float* part;                // weight adjoint: [gridDim.x][K * N_w] partial sums
     const int32_t* woff;        // per path (static order): first weight column
     const int2* ent;            // per stored M entry: {offset in the padded M_e | number of terms << 16, first term}
     const int2* nz;             // terms: {index b into a Y row, coefficient bits}
@@ -105,63 +107,50 @@ struct UdSmem {           // carved from dynamic shared memory; every part a mul
     float* M;             // [2][TB][MF]
     float* X;             // [2][TB][DT * C]
     float* out;           // [NG - 1][DT * C]
+    float* own;           // [2][DT * C] (weight adjoint)
     int2* ent;            // [nM]
     int2* nz;             // [n_nz]
 };
 
-// The work of one thread share G of NG: see the header.  All shares run the same barrier sequence.
-template <int L, int KP, int NG, int G>
-__device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& sm, const int u) {
-    constexpr int DT = (L + 1) * (L + 1);
-    constexpr int NP = n_paths_c(L);
-    constexpr int MF = m_floats_c(L);
-    constexpr int NPG = (NP + NG - 1) / NG;
-    const int C = a.C, NT = C * NG, tid = threadIdx.x;
-    const int row_chunks = DT * C / 4;            // 16-byte pieces of a feature row
-
-    // this channel's weights of the share's paths
-    float rw[NPG * KP];
-    {
-        int pi = 0, pl = 0;
-#pragma unroll
-        for (int li = 0; li <= L; ++li)
-#pragma unroll
-            for (int ls = 0; ls <= L; ++ls)
-#pragma unroll
-                for (int lo = 0; lo <= L; ++lo) {
-                    if (!path_ok(li, ls, lo, L)) continue;
-                    if (pi * NG / NP == G) {
-                        const float* Rp = a.R + __ldg(a.woff + pi) + u;
-#pragma unroll
-                        for (int q = 0; q < KP; ++q) rw[pl * KP + q] = q < a.K ? __ldg(Rp + (int64_t)q * a.N_w) : 0.f;
-                        ++pl;
-                    }
-                    ++pi;
-                }
-    }
-    float acc[DT];
-#pragma unroll
-    for (int i = 0; i < DT; ++i) acc[i] = 0.f;
-
+// The software pipeline both kernels share (see the header): prefetch(it) waits for the copies in flight, meets the
+// CTA barrier, and issues the work that runs ahead of batch `it`; the caller then consumes batch `it` and calls rotate().
+template <int L, int KP>
+struct UdPipe {
+    static constexpr int DT = (L + 1) * (L + 1);
+    static constexpr int MF = m_floats_c(L);
+    const UdArgs& a;
+    const UdSmem& sm;
+    const int NT, tid;
     // thread 0's CSR walk
-    int64_t w_node = (int64_t)blockIdx.x - gridDim.x, w_pos = 0, w_end = 0;
-    bool w_open = false;                          // a receiver is at hand and not yet closed by a `last` batch
+    int64_t w_node, w_pos = 0, w_end = 0;
+    bool w_open = false;                          // a node is at hand and not yet closed by a `last` batch
     int d_slot = 0;                               // ring slots of the batch `it + 3` (descriptor), `it + 2` (edge inputs),
     int r_slot2 = 2, r_slot1 = 1, r_slot0 = 0;    // `it + 1`, `it`; rotated at the end of an iteration
-    for (int it = -3;; ++it) {
+
+    __device__ __forceinline__ UdPipe(const UdArgs& a_, const UdSmem& sm_, int NT_)
+        : a(a_), sm(sm_), NT(NT_), tid(threadIdx.x), w_node((int64_t)blockIdx.x - gridDim.x) {}
+    __device__ __forceinline__ int4 desc_now() const { return sm.desc[(d_slot + 1) & 3]; }
+    __device__ __forceinline__ void rotate(int it) {
+        d_slot = (d_slot + 1) & 3;
+        if (it >= -2) { const int t = r_slot0; r_slot0 = r_slot1; r_slot1 = r_slot2; r_slot2 = t; }
+    }
+    __device__ __forceinline__ void prefetch(int it) {
+        const int C = a.C;
+        const int row_chunks = DT * C / 4;        // 16-byte pieces of a feature row
         cp_async_wait_all();
         __syncthreads();
         // ---- T: descriptor of batch it + 3
         if (tid == 0) {
+            bool first = false;
             if (!w_open) {
                 w_node += gridDim.x;
-                if (w_node < a.N) { seg_bounds(a.row_ptr, w_node, a.E, a.status, w_pos, w_end); w_open = true; }
+                if (w_node < a.N) { seg_bounds(a.row_ptr, w_node, a.E, a.status, w_pos, w_end); w_open = first = true; }
             }
             int4 d = make_int4(0, 0, 0, -1);
             if (w_open) {
                 const int nb = (int)min((int64_t)TB, w_end - w_pos);
                 const bool last = w_pos + nb >= w_end;
-                d = make_int4((int)(uint32_t)(uint64_t)w_pos, (int)((uint64_t)w_pos >> 32), nb | (last ? 256 : 0), (int)w_node);
+                d = make_int4((int)(uint32_t)(uint64_t)w_pos, (int)((uint64_t)w_pos >> 32), nb | (last ? 256 : 0) | (first ? 512 : 0), (int)w_node);
                 w_pos += nb;
                 if (last) w_open = false;
             }
@@ -206,6 +195,11 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                     float* dst = dX + e * DT * C;
                     for (int i = tid; i < row_chunks; i += NT) cp_async16(dst + 4 * i, src + 4 * i);
                 }
+                if (a.own && (d.z & 512)) {           // the owning node's row (weight adjoint), with its first batch
+                    const float* src = a.own + (int64_t)d.w * a.C_y;
+                    float* dst = sm.own + (size_t)buf * DT * C;
+                    for (int i = tid; i < row_chunks; i += NT) cp_async16(dst + 4 * i, src + 4 * i);
+                }
                 float* dM = sm.M + buf * (TB * MF);
                 const float* sY = sm.Y + r_slot1 * (TB * DT);
                 for (int m = tid; m < a.nM; m += NT) {
@@ -219,16 +213,55 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                 }
             }
         }
+    }
+};
+
+// The work of one thread share G of NG: see the header.  All shares run the same barrier sequence.
+template <int L, int KP, int NG, int G>
+__device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& sm, const int u) {
+    constexpr int DT = (L + 1) * (L + 1);
+    constexpr int NP = n_paths_c(L);
+    constexpr int MF = m_floats_c(L);
+    constexpr int NPG = (NP + NG - 1) / NG;
+    const int C = a.C, NT = C * NG;
+
+    // this channel's weights of the share's paths
+    float rw[NPG * KP];
+    {
+        int pi = 0, pl = 0;
+#pragma unroll
+        for (int li = 0; li <= L; ++li)
+#pragma unroll
+            for (int ls = 0; ls <= L; ++ls)
+#pragma unroll
+                for (int lo = 0; lo <= L; ++lo) {
+                    if (!path_ok(li, ls, lo, L)) continue;
+                    if (pi * NG / NP == G) {
+                        const float* Rp = a.R + __ldg(a.woff + pi) + u;
+#pragma unroll
+                        for (int q = 0; q < KP; ++q) rw[pl * KP + q] = q < a.K ? __ldg(Rp + (int64_t)q * a.N_w) : 0.f;
+                        ++pl;
+                    }
+                    ++pi;
+                }
+    }
+    float acc[DT];
+#pragma unroll
+    for (int i = 0; i < DT; ++i) acc[i] = 0.f;
+
+    UdPipe<L, KP> pipe(a, sm, NT);
+    for (int it = -3;; ++it) {
+        pipe.prefetch(it);
         // ---- D: batch it
         if (it >= 0) {
-            const int4 d = sm.desc[(d_slot + 1) & 3];
+            const int4 d = pipe.desc_now();
             if (d.w < 0) break;
             const int nb = d.z & 255;
             const int buf = it & 1;
             const float* bX = sm.X + (size_t)buf * TB * DT * C + u;
             const float* bM = sm.M + buf * (TB * MF);
-            const float* bphi = sm.phi + r_slot0 * (TB * KP);
-            const int32_t* sid = sm.sid + r_slot0 * TB;
+            const float* bphi = sm.phi + pipe.r_slot0 * (TB * KP);
+            const int32_t* sid = sm.sid + pipe.r_slot0 * TB;
             for (int e = 0; e < nb; ++e) {
                 if ((uint32_t)sid[e] >= (uint64_t)a.N) continue;
                 // w_e of the share's paths
@@ -326,20 +359,18 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                 for (int i = 0; i < DT; ++i) acc[i] = 0.f;
             }
         }
-        d_slot = (d_slot + 1) & 3;
-        if (it >= -2) { const int t = r_slot0; r_slot0 = r_slot1; r_slot1 = r_slot2; r_slot2 = t; }
+        pipe.rotate(it);
     }
 }
 
+// carves the dynamic shared memory, loads the tables; the first barrier of the pipeline orders these writes before use
 template <int L, int KP>
-__global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
+__device__ __forceinline__ UdSmem ud_setup(const UdArgs& a, unsigned char* p) {
     constexpr int DT = (L + 1) * (L + 1);
     constexpr int NG = n_groups_c(L, KP);
     constexpr int MF = m_floats_c(L);
-    extern __shared__ __align__(16) unsigned char smem_raw[];
     const int C = a.C, NT = C * NG, tid = threadIdx.x;
     UdSmem sm;
-    unsigned char* p = smem_raw;
     sm.desc = reinterpret_cast<int4*>(p); p += 4 * sizeof(int4);
     sm.phi = reinterpret_cast<float*>(p); p += 3 * TB * KP * 4;
     sm.Y = reinterpret_cast<float*>(p); p += pad4(3 * TB * DT) * 4;
@@ -348,17 +379,177 @@ __global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
     sm.M = reinterpret_cast<float*>(p); p += 2 * TB * MF * 4;
     sm.X = reinterpret_cast<float*>(p); p += (size_t)2 * TB * DT * C * 4;
     sm.out = reinterpret_cast<float*>(p); p += (size_t)(NG - 1) * DT * C * 4;
+    sm.own = reinterpret_cast<float*>(p); p += (size_t)2 * DT * C * 4;
     sm.ent = reinterpret_cast<int2*>(p); p += (size_t)a.nM * 8;
     sm.nz = reinterpret_cast<int2*>(p);
     for (int i = tid; i < 3 * TB * KP; i += NT) sm.phi[i] = 0.f;       // the columns q >= K stay zero
     for (int i = tid; i < a.nM; i += NT) sm.ent[i] = a.ent[i];
     for (int i = tid; i < a.n_nz; i += NT) sm.nz[i] = a.nz[i];
-    const int g = tid / C, u = tid - g * C;
-    // (the first barrier of the share's loop orders these writes before their first use)
+    return sm;
+}
+template <int L, int KP>
+constexpr size_t ud_smem_bytes(int C, size_t tables) {
+    constexpr int DT = (L + 1) * (L + 1), NG = n_groups_c(L, KP), MF = m_floats_c(L);
+    return 4 * sizeof(int4) + (size_t)3 * TB * KP * 4 + (size_t)pad4(3 * TB * DT) * 4 + 7 * TB * 4 + (size_t)2 * TB * MF * 4 +
+           (size_t)2 * TB * DT * C * 4 + (size_t)(NG - 1) * DT * C * 4 + (size_t)2 * DT * C * 4 + tables;
+}
+
+template <int L, int KP>
+__global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
+    constexpr int NG = n_groups_c(L, KP);
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const UdSmem sm = ud_setup<L, KP>(a, smem_raw);
+    const int g = threadIdx.x / a.C, u = threadIdx.x - g * a.C;
     if (NG == 1 || g == 0) uvu_direct_share<L, KP, NG, 0>(a, sm, u);
     else if (NG == 2 || g == 1) uvu_direct_share<L, KP, NG, (NG > 1 ? 1 : 0)>(a, sm, u);
     else if (NG == 3 || g == 2) uvu_direct_share<L, KP, NG, (NG > 2 ? 2 : 0)>(a, sm, u);
     else uvu_direct_share<L, KP, NG, (NG > 3 ? 3 : 0)>(a, sm, u);
+}
+
+// Weight adjoint of the channelwise mode on the same pipeline (Eq. adjoints):
+//   gR[q, w_off(pi) + u] = sum_e phi_e[q] gw_e[pi, u],   gw_e[pi, u] = sum_{a, o} M_e^pi[a, o] x_{j(e)}[l_in, u, a] gy_{i(e)}[l_out, u, o].
+// Thread (u, share) keeps the K x paths sums of its channel in registers over all receivers of its CTA and the
+// receiver's gy components beside them; the CTA's sums go to its own slice of `part`, summed over CTAs in a fixed
+// order by the caller.
+template <int L, int KP, int NG, int G>
+__device__ __forceinline__ void uvu_direct_wgrad_share(const UdArgs& a, const UdSmem& sm, const int u) {
+    constexpr int DT = (L + 1) * (L + 1);
+    constexpr int NP = n_paths_c(L);
+    constexpr int MF = m_floats_c(L);
+    constexpr int NPG = (NP + NG - 1) / NG;
+    const int C = a.C, NT = C * NG;
+    float ga[NPG * KP];
+#pragma unroll
+    for (int i = 0; i < NPG * KP; ++i) ga[i] = 0.f;
+    float gyr[DT];
+#pragma unroll
+    for (int i = 0; i < DT; ++i) gyr[i] = 0.f;
+    UdPipe<L, KP> pipe(a, sm, NT);
+    for (int it = -3;; ++it) {
+        pipe.prefetch(it);
+        if (it >= 0) {
+            const int4 d = pipe.desc_now();
+            if (d.w < 0) break;
+            const int nb = d.z & 255;
+            const int buf = it & 1;
+            const float* bX = sm.X + (size_t)buf * TB * DT * C + u;
+            const float* bM = sm.M + buf * (TB * MF);
+            const float* bphi = sm.phi + pipe.r_slot0 * (TB * KP);
+            const int32_t* sid = sm.sid + pipe.r_slot0 * TB;
+            if (d.z & 512) {                       // a new receiver: its gy components
+#pragma unroll
+                for (int i = 0; i < DT; ++i) gyr[i] = sm.own[((size_t)buf * DT + i) * C + u];
+            }
+            for (int e = 0; e < nb; ++e) {
+                if ((uint32_t)sid[e] >= (uint64_t)a.N) continue;
+                const float* eX = bX + e * DT * C;
+                const float* eM = bM + e * MF;
+                float gw[NPG];
+                int pi = 0, pl = 0, mo = 0, at_li = -1;
+                float xv[2 * L + 1];
+#pragma unroll
+                for (int li = 0; li <= L; ++li) {
+#pragma unroll
+                    for (int ls = 0; ls <= L; ++ls) {
+#pragma unroll
+                        for (int lo = 0; lo <= L; ++lo) {
+                            if (!path_ok(li, ls, lo, L)) continue;
+                            const int di = 2 * li + 1, dO = 2 * lo + 1;
+                            if (pi * NG / NP == G) {
+                                if (at_li != li) {
+#pragma unroll
+                                    for (int s = 0; s < di; ++s) xv[s] = eX[(li * li + s) * C];
+                                    at_li = li;
+                                }
+                                float c = 0.f;
+                                if (ls == 0) {
+#pragma unroll
+                                    for (int o = 0; o < dO; ++o) c = fmaf(xv[o], gyr[lo * lo + o], c);
+                                    c *= eM[mo];
+                                } else if (!m_transposed(di, dO)) {         // rows [a][o]
+#pragma unroll
+                                    for (int s = 0; s < di; ++s) {
+                                        float r = 0.f;
+#pragma unroll
+                                        for (int o4 = 0; o4 < dO; o4 += 4) {
+                                            const float4 m = *reinterpret_cast<const float4*>(eM + mo + s * pad4(dO) + o4);
+                                            r = fmaf(m.x, gyr[lo * lo + o4], r);
+                                            if (o4 + 1 < dO) r = fmaf(m.y, gyr[lo * lo + o4 + 1], r);
+                                            if (o4 + 2 < dO) r = fmaf(m.z, gyr[lo * lo + o4 + 2], r);
+                                            if (o4 + 3 < dO) r = fmaf(m.w, gyr[lo * lo + o4 + 3], r);
+                                        }
+                                        c = fmaf(r, xv[s], c);
+                                    }
+                                } else {                                     // rows [o][a]
+#pragma unroll
+                                    for (int o = 0; o < dO; ++o) {
+                                        float r = 0.f;
+#pragma unroll
+                                        for (int s4 = 0; s4 < di; s4 += 4) {
+                                            const float4 m = *reinterpret_cast<const float4*>(eM + mo + o * pad4(di) + s4);
+                                            r = fmaf(m.x, xv[s4], r);
+                                            if (s4 + 1 < di) r = fmaf(m.y, xv[s4 + 1], r);
+                                            if (s4 + 2 < di) r = fmaf(m.z, xv[s4 + 2], r);
+                                            if (s4 + 3 < di) r = fmaf(m.w, xv[s4 + 3], r);
+                                        }
+                                        c = fmaf(r, gyr[lo * lo + o], c);
+                                    }
+                                }
+                                gw[pl] = c;
+                                ++pl;
+                            }
+                            ++pi; mo += m_block(li, ls, lo);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q4 = 0; q4 < KP; q4 += 4) {
+                    const float4 f = *reinterpret_cast<const float4*>(bphi + e * KP + q4);
+#pragma unroll
+                    for (int i = 0; i < NPG; ++i) {
+                        if (i < pl) {
+                            ga[i * KP + q4] = fmaf(f.x, gw[i], ga[i * KP + q4]);
+                            ga[i * KP + q4 + 1] = fmaf(f.y, gw[i], ga[i * KP + q4 + 1]);
+                            ga[i * KP + q4 + 2] = fmaf(f.z, gw[i], ga[i * KP + q4 + 2]);
+                            ga[i * KP + q4 + 3] = fmaf(f.w, gw[i], ga[i * KP + q4 + 3]);
+                        }
+                    }
+                }
+            }
+        }
+        pipe.rotate(it);
+    }
+    // this CTA's sums
+    float* out = a.part + (int64_t)blockIdx.x * a.K * a.N_w + u;
+    int pi = 0, pl = 0;
+#pragma unroll
+    for (int li = 0; li <= L; ++li)
+#pragma unroll
+        for (int ls = 0; ls <= L; ++ls)
+#pragma unroll
+            for (int lo = 0; lo <= L; ++lo) {
+                if (!path_ok(li, ls, lo, L)) continue;
+                if (pi * NG / NP == G) {
+                    const int32_t wo = __ldg(a.woff + pi);
+#pragma unroll
+                    for (int q = 0; q < KP; ++q)
+                        if (q < a.K) out[(int64_t)q * a.N_w + wo] = ga[pl * KP + q];
+                    ++pl;
+                }
+                ++pi;
+            }
+}
+
+template <int L, int KP>
+__global__ void __launch_bounds__(256) k_uvu_direct_wgrad(const UdArgs a) {
+    constexpr int NG = n_groups_c(L, KP);
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const UdSmem sm = ud_setup<L, KP>(a, smem_raw);
+    const int g = threadIdx.x / a.C, u = threadIdx.x - g * a.C;
+    if (NG == 1 || g == 0) uvu_direct_wgrad_share<L, KP, NG, 0>(a, sm, u);
+    else if (NG == 2 || g == 1) uvu_direct_wgrad_share<L, KP, NG, (NG > 1 ? 1 : 0)>(a, sm, u);
+    else if (NG == 3 || g == 2) uvu_direct_wgrad_share<L, KP, NG, (NG > 2 ? 2 : 0)>(a, sm, u);
+    else uvu_direct_wgrad_share<L, KP, NG, (NG > 3 ? 3 : 0)>(a, sm, u);
 }
 
 }  // namespace
@@ -445,12 +636,11 @@ void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobe
 
 namespace {
 template <int L, int KP>
-cudaError_t launch_ud(const UdArgs& a, size_t tables, cudaStream_t s) {
-    constexpr int DT = (L + 1) * (L + 1), NG = n_groups_c(L, KP), MF = m_floats_c(L);
+cudaError_t launch_ud(const UdArgs& a, size_t tables, int max_grid, int* grid_out, cudaStream_t s) {
+    constexpr int NG = n_groups_c(L, KP);
     const int NT = a.C * NG;
-    const size_t sh = 4 * sizeof(int4) + (size_t)3 * TB * KP * 4 + (size_t)pad4(3 * TB * DT) * 4 + 7 * TB * 4 + (size_t)2 * TB * MF * 4 +
-                      (size_t)2 * TB * DT * a.C * 4 + (size_t)(NG - 1) * DT * a.C * 4 + tables;
-    auto kern = k_uvu_direct_fwd<L, KP>;
+    const size_t sh = ud_smem_bytes<L, KP>(a.C, tables);
+    auto kern = a.part ? k_uvu_direct_wgrad<L, KP> : k_uvu_direct_fwd<L, KP>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
@@ -460,9 +650,19 @@ cudaError_t launch_ud(const UdArgs& a, size_t tables, cudaStream_t s) {
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int grid = (int)std::min<int64_t>(a.N, (int64_t)sms * per_sm);
-    kern<<<grid, NT, sh, s>>>(a);
+    int64_t grid = std::min<int64_t>(a.N, (int64_t)sms * per_sm);
+    if (max_grid > 0) grid = std::min<int64_t>(grid, max_grid);
+    if (grid_out) *grid_out = (int)grid;
+    kern<<<(int)grid, NT, sh, s>>>(a);
     return cudaGetLastError();
+}
+cudaError_t dispatch_ud(int L, bool k8, const UdArgs& a, size_t tables, int max_grid, int* grid_out, cudaStream_t s) {
+    switch (L) {
+        case 0: return k8 ? launch_ud<0, 8>(a, tables, max_grid, grid_out, s) : launch_ud<0, 16>(a, tables, max_grid, grid_out, s);
+        case 1: return k8 ? launch_ud<1, 8>(a, tables, max_grid, grid_out, s) : launch_ud<1, 16>(a, tables, max_grid, grid_out, s);
+        case 2: return k8 ? launch_ud<2, 8>(a, tables, max_grid, grid_out, s) : launch_ud<2, 16>(a, tables, max_grid, grid_out, s);
+        default: return k8 ? launch_ud<3, 8>(a, tables, max_grid, grid_out, s) : launch_ud<3, 16>(a, tables, max_grid, grid_out, s);
+    }
 }
 }  // namespace
 
@@ -479,14 +679,27 @@ cudaError_t launch_uvu_direct(const sobek_plan* p, const EdgeView& ev, int trans
     a.C_x = transposed ? p->C_y : p->C_x; a.C_y = transposed ? p->C_x : p->C_y; a.status = status;
     const size_t tables = (size_t)(T.ent.size() + T.nz.size()) * 8 + 16;
     KernelTimer kt(K_STATE, s);
-    const bool k8 = p->K <= 8;
-    cudaError_t e;
-    switch (D.L) {
-        case 0: e = k8 ? launch_ud<0, 8>(a, tables, s) : launch_ud<0, 16>(a, tables, s); break;
-        case 1: e = k8 ? launch_ud<1, 8>(a, tables, s) : launch_ud<1, 16>(a, tables, s); break;
-        case 2: e = k8 ? launch_ud<2, 8>(a, tables, s) : launch_ud<2, 16>(a, tables, s); break;
-        default: e = k8 ? launch_ud<3, 8>(a, tables, s) : launch_ud<3, 16>(a, tables, s); break;
-    }
+    const cudaError_t e = dispatch_ud(D.L, p->K <= 8, a, tables, 0, nullptr, s);
+    count_launch();
+    return e;
+}
+
+// part[0 .. *n_parts)[K * N_w] = per-CTA sums of the weight adjoint over the receivers of `ev` (the receiver view);
+// at most max_parts slices are written.  The caller adds them up in order.
+cudaError_t launch_uvu_direct_wgrad(const sobek_plan* p, const EdgeView& ev, const float* x, const float* Y, const float* phi,
+                                    const float* gy, float* part, int max_parts, int* n_parts, int* status, cudaStream_t s) {
+    const UvuDirect& D = p->ud;
+    const UvuDirectTables& T = D.dir[0];
+    if (!D.ok || !T.d_woff || !T.d_ent || !T.d_nz || !part || max_parts < 1 || ev.perm) return cudaErrorInvalidValue;
+    UdArgs a{};
+    a.row_ptr = ev.ptr; a.ids = ev.col; a.perm = nullptr; a.N = ev.N; a.E = ev.E;
+    a.x = x; a.Y = Y; a.phi = phi; a.R = nullptr; a.y = nullptr; a.own = gy; a.part = part;
+    a.woff = T.d_woff; a.ent = T.d_ent; a.nz = T.d_nz; a.n_nz = (int32_t)T.nz.size();
+    a.C = D.C; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
+    a.C_x = p->C_x; a.C_y = p->C_y; a.status = status;
+    const size_t tables = (size_t)(T.ent.size() + T.nz.size()) * 8 + 16;
+    KernelTimer kt(K_STATE, s);
+    const cudaError_t e = dispatch_ud(D.L, p->K <= 8, a, tables, max_parts, n_parts, s);
     count_launch();
     return e;
 }

@@ -567,7 +567,7 @@ def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases):
 
 @pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16"])
 def test_uvu_direct_and_state_route_agree(name):
-    """Uniform natural-parity profiles take the direct channelwise kernel for y and gx by default; the route through
+    """Uniform natural-parity profiles take the direct channelwise kernels for y, gx and gR by default; the route through
     the receiver state (SOBEK_FLAG_UVU_STATE) computes the same thing.  Both against the oracle."""
     c = Case(UVU[name])
     s = Case(UVU[name], inputs=c.d, uvu_state=True)
@@ -580,10 +580,12 @@ def test_uvu_direct_and_state_route_agree(name):
     for got in (b_direct, b_state):
         for g, r in zip(got, b_ref):
             assert rel_err(g, r) <= BWD_TOL
-    assert not np.array_equal(b_direct[0], b_state[0])
-    assert np.array_equal(b_direct[0], c.bwd()[0])
-    for g, r in zip(b_direct[1:], b_state[1:]):         # gY, gphi, gR take the same kernels on both plans
-        assert np.array_equal(g, r)
+    again = c.bwd()
+    for k in (0, 3):                                    # gx and gR: direct kernels, repeatable bitwise
+        assert not np.array_equal(b_direct[k], b_state[k])
+        assert np.array_equal(b_direct[k], again[k])
+    for k in (1, 2):                                    # gY, gphi take the same kernels on both plans
+        assert np.array_equal(b_direct[k], b_state[k])
 
 
 def test_uvu_full_size_sampled():
