@@ -127,8 +127,12 @@ struct UdPipe {
     int d_slot = 0;                               // ring slots of the batch `it + 3` (descriptor), `it + 2` (edge inputs),
     int r_slot2 = 2, r_slot1 = 1, r_slot0 = 0;    // `it + 1`, `it`; rotated at the end of an iteration
 
+    int64_t n_s0 = 0, n_s1 = 0;                   // segment of the node after w_node, fetched ahead
+
     __device__ __forceinline__ UdPipe(const UdArgs& a_, const UdSmem& sm_, int NT_)
-        : a(a_), sm(sm_), NT(NT_), tid(threadIdx.x), w_node((int64_t)blockIdx.x - gridDim.x) {}
+        : a(a_), sm(sm_), NT(NT_), tid(threadIdx.x), w_node((int64_t)blockIdx.x - gridDim.x) {
+        if (tid == 0 && blockIdx.x < a.N) { n_s0 = a.row_ptr[blockIdx.x]; n_s1 = a.row_ptr[blockIdx.x + 1]; }
+    }
     __device__ __forceinline__ int4 desc_now() const { return sm.desc[(d_slot + 1) & 3]; }
     __device__ __forceinline__ void rotate(int it) {
         d_slot = (d_slot + 1) & 3;
@@ -144,7 +148,15 @@ struct UdPipe {
             bool first = false;
             if (!w_open) {
                 w_node += gridDim.x;
-                if (w_node < a.N) { seg_bounds(a.row_ptr, w_node, a.E, a.status, w_pos, w_end); w_open = first = true; }
+                if (w_node < a.N) {
+                    // the bounds were fetched when the node before was opened (no load latency under the CTA barrier)
+                    const int64_t s0 = n_s0 < 0 ? 0 : (n_s0 > a.E ? a.E : n_s0);
+                    const int64_t s1 = n_s1 < s0 ? s0 : (n_s1 > a.E ? a.E : n_s1);
+                    if ((s0 != n_s0 || s1 != n_s1) && a.status) atomicExch(a.status, (int)SOBEK_ERR_GRAPH);
+                    w_pos = s0; w_end = s1; w_open = first = true;
+                    const int64_t nx = w_node + gridDim.x;
+                    if (nx < a.N) { n_s0 = a.row_ptr[nx]; n_s1 = a.row_ptr[nx + 1]; }
+                }
             }
             int4 d = make_int4(0, 0, 0, -1);
             if (w_open) {
@@ -271,13 +283,15 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
 #pragma unroll
                 for (int q4 = 0; q4 < KP; q4 += 4) {
                     const float4 f = *reinterpret_cast<const float4*>(bphi + e * KP + q4);
+                    // (component by component: consecutive multiply-adds go to different sums)
 #pragma unroll
-                    for (int i = 0; i < NPG; ++i) {
-                        w[i] = fmaf(f.x, rw[i * KP + q4], w[i]);
-                        w[i] = fmaf(f.y, rw[i * KP + q4 + 1], w[i]);
-                        w[i] = fmaf(f.z, rw[i * KP + q4 + 2], w[i]);
-                        w[i] = fmaf(f.w, rw[i * KP + q4 + 3], w[i]);
-                    }
+                    for (int i = 0; i < NPG; ++i) w[i] = fmaf(f.x, rw[i * KP + q4], w[i]);
+#pragma unroll
+                    for (int i = 0; i < NPG; ++i) w[i] = fmaf(f.y, rw[i * KP + q4 + 1], w[i]);
+#pragma unroll
+                    for (int i = 0; i < NPG; ++i) w[i] = fmaf(f.z, rw[i * KP + q4 + 2], w[i]);
+#pragma unroll
+                    for (int i = 0; i < NPG; ++i) w[i] = fmaf(f.w, rw[i * KP + q4 + 3], w[i]);
                 }
                 const float* eX = bX + e * DT * C;
                 const float* eM = bM + e * MF;
