@@ -66,10 +66,19 @@ def work_model(plan):
         p = plan.path(k)
         di, do = 2 * p.l_in + 1, 2 * p.l_out + 1
         nnz = int((np.abs(plan.cg(k)) > 0).sum())
-        KF += K * p.c_in * do
-        KFt += K * p.c_out * di
-        CG += p.c_in * nnz
-        CGt += p.c_out * nnz
+        if plan.mode == "uvu":
+            # channelwise mode: the cheapest form of every pass is the direct one, K multiply-adds for the edge's weight
+            # of a channel and path plus d_in d_out for the contraction with the coupling matrix (both directions);
+            # passes that still go through the K-expanded state do more than this count credits them for
+            KF += K * p.c_in
+            KFt += K * p.c_in
+            CG += p.c_in * di * do
+            CGt += p.c_in * di * do
+        else:
+            KF += K * p.c_in * do
+            KFt += K * p.c_out * di
+            CG += p.c_in * nnz
+            CGt += p.c_out * nnz
         co = 1 if plan.mode == "uvu" else p.c_out      # tied multiplicities: no sum over a second channel index
         Gf += K * p.c_in * co * do
         Gt += K * p.c_in * co * di
