@@ -235,7 +235,7 @@ struct UvuDirectTables {
 };
 struct UvuDirect {
     bool ok = false;
-    int L = 0, C = 0;
+    int L = 0, C = 0, H = 1;        // H: channel slices, one CTA each (C / H channels x thread shares <= 256 threads)
     UvuDirectTables dir[2];         // [0] y from x on the receiver view, [1] gx from gy on the sender view
 };
 

@@ -59,7 +59,9 @@ struct UdArgs {
     const int32_t* woff;        // per path (static order): first weight column
     const int2* ent;            // per stored M entry: {offset in the padded M_e | number of terms << 16, first term}
     const int2* nz;             // terms: {index b into a Y row, coefficient bits}
-    int32_t C, K, nM, N_w, C_x, C_y, n_nz;
+    int32_t C;                  // channels of a CTA: slice blockIdx.x % H of the profile's Cf = C * H channels
+    int32_t Cf, H;
+    int32_t K, nM, N_w, C_x, C_y, n_nz;
     int* status;
 };
 
@@ -114,7 +116,8 @@ struct UdSmem {           // carved from dynamic shared memory; every part a mul
 
 // The software pipeline both kernels share (see the header): prefetch(it) waits for the copies in flight, meets the
 // CTA barrier, and issues the work that runs ahead of batch `it`; the caller then consumes batch `it` and calls rotate().
-template <int L, int KP>
+// SP: the channels are split into slices, one CTA each (else H = 1 is known at compile time)
+template <int L, int KP, bool SP>
 struct UdPipe {
     static constexpr int DT = (L + 1) * (L + 1);
     static constexpr int MF = m_floats_c(L);
@@ -130,8 +133,24 @@ struct UdPipe {
     int64_t n_s0 = 0, n_s1 = 0;                   // segment of the node after w_node, fetched ahead
 
     __device__ __forceinline__ UdPipe(const UdArgs& a_, const UdSmem& sm_, int NT_)
-        : a(a_), sm(sm_), NT(NT_), tid(threadIdx.x), w_node((int64_t)blockIdx.x - gridDim.x) {
-        if (tid == 0 && blockIdx.x < a.N) { n_s0 = a.row_ptr[blockIdx.x]; n_s1 = a.row_ptr[blockIdx.x + 1]; }
+        : a(a_), sm(sm_), NT(NT_), tid(threadIdx.x), w_node((int64_t)(blockIdx.x / (SP ? a_.H : 1)) - (int64_t)(gridDim.x / (SP ? a_.H : 1))) {
+        const int64_t n0 = blockIdx.x / (SP ? a.H : 1);
+        if (tid == 0 && n0 < a.N) { n_s0 = a.row_ptr[n0]; n_s1 = a.row_ptr[n0 + 1]; }
+    }
+    // copies the CTA's channels of a [DT][Cf] feature row into [DT][C] shared floats, 16 bytes at a time
+    __device__ __forceinline__ void copy_row(float* dst, const float* src) const {
+        const int C = a.C;
+        const int row_chunks = DT * C / 4;
+        if (!SP) {
+            for (int i = tid; i < row_chunks; i += NT) cp_async16(dst + 4 * i, src + 4 * i);
+        } else {
+            const int c4n = C / 4;
+            const float* s0 = src + (blockIdx.x % a.H) * C;
+            for (int i = tid; i < row_chunks; i += NT) {
+                const int t = i / c4n, c4 = i - t * c4n;
+                cp_async16(dst + 4 * i, s0 + t * a.Cf + 4 * c4);
+            }
+        }
     }
     __device__ __forceinline__ int4 desc_now() const { return sm.desc[(d_slot + 1) & 3]; }
     __device__ __forceinline__ void rotate(int it) {
@@ -140,21 +159,20 @@ struct UdPipe {
     }
     __device__ __forceinline__ void prefetch(int it) {
         const int C = a.C;
-        const int row_chunks = DT * C / 4;        // 16-byte pieces of a feature row
         cp_async_wait_all();
         __syncthreads();
         // ---- T: descriptor of batch it + 3
         if (tid == 0) {
             bool first = false;
             if (!w_open) {
-                w_node += gridDim.x;
+                w_node += gridDim.x / (SP ? a.H : 1);
                 if (w_node < a.N) {
                     // the bounds were fetched when the node before was opened (no load latency under the CTA barrier)
                     const int64_t s0 = n_s0 < 0 ? 0 : (n_s0 > a.E ? a.E : n_s0);
                     const int64_t s1 = n_s1 < s0 ? s0 : (n_s1 > a.E ? a.E : n_s1);
                     if ((s0 != n_s0 || s1 != n_s1) && a.status) atomicExch(a.status, (int)SOBEK_ERR_GRAPH);
                     w_pos = s0; w_end = s1; w_open = first = true;
-                    const int64_t nx = w_node + gridDim.x;
+                    const int64_t nx = w_node + gridDim.x / (SP ? a.H : 1);
                     if (nx < a.N) { n_s0 = a.row_ptr[nx]; n_s1 = a.row_ptr[nx + 1]; }
                 }
             }
@@ -203,14 +221,10 @@ struct UdPipe {
                 for (int e = 0; e < nb; ++e) {
                     const int32_t j = sid[e];
                     if (!id_ok(j, a.N, a.status)) continue;
-                    const float* src = a.x + (int64_t)j * a.C_x;
-                    float* dst = dX + e * DT * C;
-                    for (int i = tid; i < row_chunks; i += NT) cp_async16(dst + 4 * i, src + 4 * i);
+                    copy_row(dX + e * DT * C, a.x + (int64_t)j * a.C_x);
                 }
                 if (a.own && (d.z & 512)) {           // the owning node's row (weight adjoint), with its first batch
-                    const float* src = a.own + (int64_t)d.w * a.C_y;
-                    float* dst = sm.own + (size_t)buf * DT * C;
-                    for (int i = tid; i < row_chunks; i += NT) cp_async16(dst + 4 * i, src + 4 * i);
+                    copy_row(sm.own + (size_t)buf * DT * C, a.own + (int64_t)d.w * a.C_y);
                 }
                 float* dM = sm.M + buf * (TB * MF);
                 const float* sY = sm.Y + r_slot1 * (TB * DT);
@@ -229,7 +243,7 @@ struct UdPipe {
 };
 
 // The work of one thread share G of NG: see the header.  All shares run the same barrier sequence.
-template <int L, int KP, int NG, int G>
+template <int L, int KP, int NG, int G, bool SP>
 __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& sm, const int u) {
     constexpr int DT = (L + 1) * (L + 1);
     constexpr int NP = n_paths_c(L);
@@ -249,7 +263,7 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                 for (int lo = 0; lo <= L; ++lo) {
                     if (!path_ok(li, ls, lo, L)) continue;
                     if (pi * NG / NP == G) {
-                        const float* Rp = a.R + __ldg(a.woff + pi) + u;
+                        const float* Rp = a.R + __ldg(a.woff + pi) + (SP ? (blockIdx.x % a.H) * C : 0) + u;
 #pragma unroll
                         for (int q = 0; q < KP; ++q) rw[pl * KP + q] = q < a.K ? __ldg(Rp + (int64_t)q * a.N_w) : 0.f;
                         ++pl;
@@ -261,7 +275,7 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
 #pragma unroll
     for (int i = 0; i < DT; ++i) acc[i] = 0.f;
 
-    UdPipe<L, KP> pipe(a, sm, NT);
+    UdPipe<L, KP, SP> pipe(a, sm, NT);
     for (int it = -3;; ++it) {
         pipe.prefetch(it);
         // ---- D: batch it
@@ -360,13 +374,13 @@ __device__ __forceinline__ void uvu_direct_share(const UdArgs& a, const UdSmem& 
                     __syncthreads();
                 }
                 if (G == 0) {
-                    float* yp = a.y + (int64_t)d.w * a.C_y + u;
+                    float* yp = a.y + (int64_t)d.w * a.C_y + (SP ? (blockIdx.x % a.H) * C : 0) + u;
 #pragma unroll
                     for (int i = 0; i < DT; ++i) {
                         float v = acc[i];
 #pragma unroll
                         for (int g = 1; g < NG; ++g) v += sm.out[((g - 1) * DT + i) * C + u];
-                        yp[i * C] = v;
+                        yp[i * (SP ? a.Cf : C)] = v;
                     }
                 }
 #pragma unroll
@@ -408,16 +422,16 @@ constexpr size_t ud_smem_bytes(int C, size_t tables) {
            (size_t)2 * TB * DT * C * 4 + (size_t)(NG - 1) * DT * C * 4 + (size_t)2 * DT * C * 4 + tables;
 }
 
-template <int L, int KP>
+template <int L, int KP, bool SP>
 __global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
     constexpr int NG = n_groups_c(L, KP);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const UdSmem sm = ud_setup<L, KP>(a, smem_raw);
     const int g = threadIdx.x / a.C, u = threadIdx.x - g * a.C;
-    if (NG == 1 || g == 0) uvu_direct_share<L, KP, NG, 0>(a, sm, u);
-    else if (NG == 2 || g == 1) uvu_direct_share<L, KP, NG, (NG > 1 ? 1 : 0)>(a, sm, u);
-    else if (NG == 3 || g == 2) uvu_direct_share<L, KP, NG, (NG > 2 ? 2 : 0)>(a, sm, u);
-    else uvu_direct_share<L, KP, NG, (NG > 3 ? 3 : 0)>(a, sm, u);
+    if (NG == 1 || g == 0) uvu_direct_share<L, KP, NG, 0, SP>(a, sm, u);
+    else if (NG == 2 || g == 1) uvu_direct_share<L, KP, NG, (NG > 1 ? 1 : 0), SP>(a, sm, u);
+    else if (NG == 3 || g == 2) uvu_direct_share<L, KP, NG, (NG > 2 ? 2 : 0), SP>(a, sm, u);
+    else uvu_direct_share<L, KP, NG, (NG > 3 ? 3 : 0), SP>(a, sm, u);
 }
 
 // Weight adjoint of the channelwise mode on the same pipeline (Eq. adjoints):
@@ -425,7 +439,7 @@ __global__ void __launch_bounds__(256) k_uvu_direct_fwd(const UdArgs a) {
 // Thread (u, share) keeps the K x paths sums of its channel in registers over all receivers of its CTA and the
 // receiver's gy components beside them; the CTA's sums go to its own slice of `part`, summed over CTAs in a fixed
 // order by the caller.
-template <int L, int KP, int NG, int G>
+template <int L, int KP, int NG, int G, bool SP>
 __device__ __forceinline__ void uvu_direct_wgrad_share(const UdArgs& a, const UdSmem& sm, const int u) {
     constexpr int DT = (L + 1) * (L + 1);
     constexpr int NP = n_paths_c(L);
@@ -438,7 +452,7 @@ __device__ __forceinline__ void uvu_direct_wgrad_share(const UdArgs& a, const Ud
     float gyr[DT];
 #pragma unroll
     for (int i = 0; i < DT; ++i) gyr[i] = 0.f;
-    UdPipe<L, KP> pipe(a, sm, NT);
+    UdPipe<L, KP, SP> pipe(a, sm, NT);
     for (int it = -3;; ++it) {
         pipe.prefetch(it);
         if (it >= 0) {
@@ -534,7 +548,7 @@ __device__ __forceinline__ void uvu_direct_wgrad_share(const UdArgs& a, const Ud
         pipe.rotate(it);
     }
     // this CTA's sums
-    float* out = a.part + (int64_t)blockIdx.x * a.K * a.N_w + u;
+    float* out = a.part + (int64_t)(blockIdx.x / (SP ? a.H : 1)) * a.K * a.N_w + (SP ? (blockIdx.x % a.H) * C : 0) + u;
     int pi = 0, pl = 0;
 #pragma unroll
     for (int li = 0; li <= L; ++li)
@@ -554,22 +568,22 @@ __device__ __forceinline__ void uvu_direct_wgrad_share(const UdArgs& a, const Ud
             }
 }
 
-template <int L, int KP>
+template <int L, int KP, bool SP>
 __global__ void __launch_bounds__(256) k_uvu_direct_wgrad(const UdArgs a) {
     constexpr int NG = n_groups_c(L, KP);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const UdSmem sm = ud_setup<L, KP>(a, smem_raw);
     const int g = threadIdx.x / a.C, u = threadIdx.x - g * a.C;
-    if (NG == 1 || g == 0) uvu_direct_wgrad_share<L, KP, NG, 0>(a, sm, u);
-    else if (NG == 2 || g == 1) uvu_direct_wgrad_share<L, KP, NG, (NG > 1 ? 1 : 0)>(a, sm, u);
-    else if (NG == 3 || g == 2) uvu_direct_wgrad_share<L, KP, NG, (NG > 2 ? 2 : 0)>(a, sm, u);
-    else uvu_direct_wgrad_share<L, KP, NG, (NG > 3 ? 3 : 0)>(a, sm, u);
+    if (NG == 1 || g == 0) uvu_direct_wgrad_share<L, KP, NG, 0, SP>(a, sm, u);
+    else if (NG == 2 || g == 1) uvu_direct_wgrad_share<L, KP, NG, (NG > 1 ? 1 : 0), SP>(a, sm, u);
+    else if (NG == 3 || g == 2) uvu_direct_wgrad_share<L, KP, NG, (NG > 2 ? 2 : 0), SP>(a, sm, u);
+    else uvu_direct_wgrad_share<L, KP, NG, (NG > 3 ? 3 : 0), SP>(a, sm, u);
 }
 
 }  // namespace
 
 // Whether the plan's profile is  C x 0e + C x 1o + ... + C x L  on both sides with l_max = L <= 3, C a multiple of 16
-// and C x (thread shares) <= 256; fills the per-path and per-entry tables in the kernel's static path order and
+// that splits into slices of at most 256 / (thread shares) channels; fills the per-path and per-entry tables in the kernel's static path order and
 // padded M_e layout.
 void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out) {
     UvuDirect& D = p->ud;
@@ -577,7 +591,9 @@ void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobe
     if (!p->uvu || n_in != n_out || n_in < 1 || n_in > 4 || p->l_max != n_in - 1 || p->K > KMAX) return;
     const int L = n_in - 1, C = in[0].mul;
     const int NG = n_groups_c(L, p->K <= 8 ? 8 : 16);
-    if (C < 16 || (C & 15) || C * NG > 256 || NG > 4) return;
+    // a CTA takes C / H channels (a multiple of 16) so that its (channel, share) threads number at most 256
+    const int H = (C * NG + 255) / 256;
+    if (C < 16 || (C & 15) || NG > 4 || C % H != 0 || ((C / H) & 15)) return;
     for (int i = 0; i < n_in; ++i) {
         const int par = (i & 1) ? -1 : 1;
         if (in[i].l != i || out[i].l != i || in[i].mul != C || out[i].mul != C || in[i].parity != par || out[i].parity != par) return;
@@ -644,7 +660,7 @@ void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobe
         if (woff.size() != dir.paths.size() || mo != m_floats_c(L) || mo >= 65536 || nz.size() >= 32768) return;
         D.dir[tr].woff = woff; D.dir[tr].ent = ent; D.dir[tr].nz = nz;
     }
-    D.L = L; D.C = C;
+    D.L = L; D.C = C; D.H = H;
     D.ok = true;
 }
 
@@ -652,9 +668,10 @@ namespace {
 template <int L, int KP>
 cudaError_t launch_ud(const UdArgs& a, size_t tables, int max_grid, int* grid_out, cudaStream_t s) {
     constexpr int NG = n_groups_c(L, KP);
-    const int NT = a.C * NG;
+    const int NT = a.C * NG;                  // a.C: channels of a CTA
     const size_t sh = ud_smem_bytes<L, KP>(a.C, tables);
-    auto kern = a.part ? k_uvu_direct_wgrad<L, KP> : k_uvu_direct_fwd<L, KP>;
+    auto kern = a.part ? (a.H > 1 ? k_uvu_direct_wgrad<L, KP, true> : k_uvu_direct_wgrad<L, KP, false>)
+                       : (a.H > 1 ? k_uvu_direct_fwd<L, KP, true> : k_uvu_direct_fwd<L, KP, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
@@ -664,10 +681,11 @@ cudaError_t launch_ud(const UdArgs& a, size_t tables, int max_grid, int* grid_ou
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int64_t grid = std::min<int64_t>(a.N, (int64_t)sms * per_sm);
-    if (max_grid > 0) grid = std::min<int64_t>(grid, max_grid);
-    if (grid_out) *grid_out = (int)grid;
-    kern<<<(int)grid, NT, sh, s>>>(a);
+    // H CTAs (one per channel slice) walk the same nodes: the grid is a multiple of H
+    int64_t walks = std::min<int64_t>(a.N, std::max<int64_t>(1, (int64_t)sms * per_sm / a.H));
+    if (max_grid > 0) walks = std::min<int64_t>(walks, max_grid);
+    if (grid_out) *grid_out = (int)walks;
+    kern<<<(int)(walks * a.H), NT, sh, s>>>(a);
     return cudaGetLastError();
 }
 cudaError_t dispatch_ud(int L, bool k8, const UdArgs& a, size_t tables, int max_grid, int* grid_out, cudaStream_t s) {
@@ -689,7 +707,7 @@ cudaError_t launch_uvu_direct(const sobek_plan* p, const EdgeView& ev, int trans
     a.row_ptr = ev.ptr; a.ids = transposed ? ev.recv : ev.col; a.perm = transposed ? ev.perm : nullptr; a.N = ev.N; a.E = ev.E;
     a.x = src; a.Y = Y; a.phi = phi; a.R = R; a.y = dst;
     a.woff = T.d_woff; a.ent = T.d_ent; a.nz = T.d_nz; a.n_nz = (int32_t)T.nz.size();
-    a.C = D.C; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
+    a.C = D.C / D.H; a.Cf = D.C; a.H = D.H; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
     a.C_x = transposed ? p->C_y : p->C_x; a.C_y = transposed ? p->C_x : p->C_y; a.status = status;
     const size_t tables = (size_t)(T.ent.size() + T.nz.size()) * 8 + 16;
     KernelTimer kt(K_STATE, s);
@@ -709,7 +727,7 @@ cudaError_t launch_uvu_direct_wgrad(const sobek_plan* p, const EdgeView& ev, con
     a.row_ptr = ev.ptr; a.ids = ev.col; a.perm = nullptr; a.N = ev.N; a.E = ev.E;
     a.x = x; a.Y = Y; a.phi = phi; a.R = nullptr; a.y = nullptr; a.own = gy; a.part = part;
     a.woff = T.d_woff; a.ent = T.d_ent; a.nz = T.d_nz; a.n_nz = (int32_t)T.nz.size();
-    a.C = D.C; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
+    a.C = D.C / D.H; a.Cf = D.C; a.H = D.H; a.K = p->K; a.nM = (int32_t)T.ent.size(); a.N_w = (int32_t)p->N_w;
     a.C_x = p->C_x; a.C_y = p->C_y; a.status = status;
     const size_t tables = (size_t)(T.ent.size() + T.nz.size()) * 8 + 16;
     KernelTimer kt(K_STATE, s);

@@ -503,6 +503,9 @@ def uvu_cases():
                       mode="uvu")
     c["uvu_32x4_K16"] = W("uvu_32x4_K16", P("32x0e+32x1o+32x2e+32x3o"), P("32x0e+32x1o+32x2e+32x3o"), 3, 16, 80, 4.0, 1.7,
                           "bessel", seed=8, mode="uvu")
+    # 128 channels x 3 thread shares: the direct kernels split the channels into two slices of 64, one CTA each
+    c["uvu_128x4_K16"] = W("uvu_128x4_K16", P("128x0e+128x1o+128x2e+128x3o"), P("128x0e+128x1o+128x2e+128x3o"), 3, 16, 40,
+                           4.0, 1.7, "bessel", seed=11, mode="uvu")
     # FP32-pipe edge kernels: odd multiplicities, blocks of different multiplicity that no path couples, an
     # output block without an input twin (3x3e, fed by 4e only), a multiplicity above 128
     c["uvu_ragged"] = W("uvu_ragged", P("5x0e+5x1o+3x4e+2x0o"), P("5x0e+5x1o+3x4e+3x3e+2x0o"), 2, 3, 40, 4.0, 1.9,
@@ -565,7 +568,7 @@ def test_uvu_bitwise_reproducible_and_fp32_pipe_kernels(ucases):
         assert rel_err(got, ref) <= BWD_TOL
 
 
-@pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16"])
+@pytest.mark.parametrize("name", ["uvu_16x3", "uvu_32x4_K16", "uvu_128x4_K16"])
 def test_uvu_direct_and_state_route_agree(name):
     """Uniform natural-parity profiles take the direct channelwise kernels for y, gx and gR by default; the route through
     the receiver state (SOBEK_FLAG_UVU_STATE) computes the same thing.  Both against the oracle."""
