@@ -175,45 +175,43 @@ cudaError_t split_adjoint(const sobek_plan* p, const Direction& dir, int64_t n0,
 // dst_g (+)= Z_g * Rp_g        (Eq. receiver_matrix_product)
 cudaError_t mix_tc(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const uint16_t* zh,
                    const uint16_t* zl, const uint16_t* nkh, const uint16_t* nkl, float* dst, int accumulate,
-                   int* status, cudaStream_t s0) {
-    Fork fork(p, s0);
+                   int* status, cudaStream_t s) {
+    GemmBatch gb;                 // the groups' products run as one launch
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
-        cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
-                                       nkh + dir.nk_off[gi], nkl + dir.nk_off[gi], dir.nk_ld[gi],
-                                       dst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst,
-                                       nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s, 1, 0, nullptr, nullptr, p->gemm_passes);
+        cudaError_t e = gemm_tc_add(gb, zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
+                                    nkh + dir.nk_off[gi], nkl + dir.nk_off[gi], dir.nk_ld[gi],
+                                    dst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst,
+                                    nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s, 1, 0, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    return fork.join();
+    return gemm_tc_flush(gb, s);
 }
 
 // Zbar_g = gy_g * Rp_g^T       (Eq. receiver_adjoint)
 // With zqh / zql the result is written as bf16 (hi, lo) rows in the layout of the stream's state instead.
 cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t nn, const uint16_t* gh,
                              const uint16_t* gl, const uint16_t* knh, const uint16_t* knl, float* Zbar, int* status,
-                             cudaStream_t s0, uint16_t* zqh = nullptr, uint16_t* zql = nullptr) {
-    Fork fork(p, s0);
+                             cudaStream_t s, uint16_t* zqh = nullptr, uint16_t* zql = nullptr) {
+    GemmBatch gb;
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
         cudaError_t e;
         if (zqh)
-            e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
-                               knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi], nullptr, dir.nk_ld[gi], 0, 1,
-                               nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, zqh + nn * dir.zb_off[gi],
-                               zql + nn * dir.zb_off[gi], p->gemm_passes);
+            e = gemm_tc_add(gb, gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                            knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi], nullptr, dir.nk_ld[gi], 0, 1,
+                            nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, zqh + nn * dir.zb_off[gi],
+                            zql + nn * dir.zb_off[gi], p->gemm_passes);
         else
-            e = launch_gemm_tc(gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
-                                       knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi],
-                                       Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, nullptr, nullptr,
-                                       p->gemm_passes);
+            e = gemm_tc_add(gb, gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                            knh + dir.kn_off[gi], knl + dir.kn_off[gi], dir.kn_ld[gi],
+                            Zbar + nn * G.z_off, G.D, 0, 1, nn * G.d_dst, G.D, G.c_dst, 0, 0, status, s, 1, 0, nullptr, nullptr,
+                            p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    return fork.join();
+    return gemm_tc_flush(gb, s);
 }
 
 // gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint).  The contraction runs over every (node, component)
@@ -222,22 +220,35 @@ cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn
                            const uint16_t* zl, const uint16_t* gh, const uint16_t* gl, float* gRp, float* part,
                            int splits, int* status, cudaStream_t s0) {
     const int64_t KN = (int64_t)p->K * p->N_w;
-    Fork fork(p, s0);
+    GemmBatch gb;
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
-        cudaStream_t s = fork.pick();
         const int64_t kblocks = (nn * G.d_dst + 63) / 64;
         const int sp = (int)std::max<int64_t>(1, std::min<int64_t>(splits, kblocks));
-        cudaError_t e = launch_gemm_tc(zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
-                                       gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
-                                       part + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 0, 1, status, s,
-                                       sp, KN, nullptr, nullptr, p->gemm_passes);
-        if (e != cudaSuccess) return e;
-        e = launch_reduce_parts(gRp + G.rp_off, part + G.rp_off, (int64_t)G.D * G.c_dst, KN, sp, s);
+        cudaError_t e = gemm_tc_add(gb, zh + nn * dir.zb_off[gi], zl + nn * dir.zb_off[gi], dir.nk_ld[gi],
+                                    gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], dir.kn_ld[gi],
+                                    part + G.rp_off, G.c_dst, 0, 1, G.D, G.c_dst, nn * G.d_dst, 0, 1, status, s0,
+                                    sp, KN, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    return fork.join();
+    cudaError_t e = gemm_tc_flush(gb, s0);
+    if (e != cudaSuccess) return e;
+    // the pieces of every group, summed in a fixed order: one launch over the groups' column ranges
+    ReduceRange rr[kMaxReduceRanges];
+    int nr = 0;
+    for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
+        const DGroup& G = dir.groups[gi];
+        if (G.path_end == G.path_begin) continue;
+        const int64_t kblocks = (nn * G.d_dst + 63) / 64;
+        rr[nr++] = ReduceRange{G.rp_off, (int64_t)G.D * G.c_dst, (int)std::max<int64_t>(1, std::min<int64_t>(splits, kblocks))};
+        if (nr == kMaxReduceRanges) {
+            e = launch_reduce_ranges(gRp, part, KN, rr, nr, s0);
+            if (e != cudaSuccess) return e;
+            nr = 0;
+        }
+    }
+    return launch_reduce_ranges(gRp, part, KN, rr, nr, s0);
 }
 
 // ---- the node-side steps in either multiplicity mode: tensor-core GEMMs on the packed copies of R (uvw), or

@@ -51,9 +51,33 @@ struct TcArgs {
     int* status;
 };
 
+// One launch runs up to TC_MAX_BATCH independent products (the output groups of one node-side step): the CTAs
+// tile0[b] .. tile0[b+1]-1 belong to product b and number its (m tile, n tile, split) triples.
+constexpr int TC_MAX_BATCH = 5;
+struct alignas(64) TcProblem {
+    CUtensorMap tmAh, tmAl, tmBh, tmBl;
+    TcArgs g;
+    uint32_t gx, gy;            // m tiles, n tiles
+};
+struct TcBatch {
+    TcProblem p[TC_MAX_BATCH];
+    int32_t n;
+    uint32_t tile0[TC_MAX_BATCH + 1];
+};
+static_assert(sizeof(TcBatch) <= sizeof(GemmBatch::storage), "GemmBatch::storage holds a TcBatch");
+
 __global__ void __launch_bounds__(TC_THREADS, 2)
-k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
-          const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl, const TcArgs g) {
+k_gemm_tc(const __grid_constant__ TcBatch B) {
+    int bi = 0;
+    while (bi + 1 < B.n && blockIdx.x >= B.tile0[bi + 1]) ++bi;
+    const TcProblem& pr = B.p[bi];
+    const TcArgs& g = pr.g;
+    const CUtensorMap& tmAh = pr.tmAh;
+    const CUtensorMap& tmAl = pr.tmAl;
+    const CUtensorMap& tmBh = pr.tmBh;
+    const CUtensorMap& tmBl = pr.tmBl;
+    const uint32_t tile = blockIdx.x - B.tile0[bi];
+    const uint32_t bx = tile % pr.gx, by = (tile / pr.gx) % pr.gy, bz = tile / (pr.gx * pr.gy);
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment for the 128-byte swizzle atoms
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -67,10 +91,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
     const uint32_t bar0 = smem_u32(bars);
     const int S = g.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * g.BN;
+    const int m0 = (int)bx * BM, n0 = (int)by * g.BN;
     const int num_kb_all = (int)((g.Kd + BK - 1) / BK);
     const int kb_per = (num_kb_all + g.splits - 1) / g.splits;
-    const int kb_first = blockIdx.z * kb_per;
+    const int kb_first = (int)bz * kb_per;
     const int num_kb = max(0, min(kb_per, num_kb_all - kb_first));   // k-blocks of this piece
 
     if (threadIdx.x == 0) {
@@ -178,7 +202,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
             for (int r = half; r < 32; r += 2) {
                 const int64_t m = (int64_t)m0 + q * 32 + r;
                 if (m >= g.M) continue;
-                const int64_t rbase = blockIdx.z * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
+                const int64_t rbase = (int64_t)bz * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
                 for (int c8 = l16; c8 < g.BN / 8; c8 += 16) {
                     const int64_t n = (int64_t)n0 + 8 * c8;
                     if (n < g.N) {
@@ -214,7 +238,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUte
         for (int r = 0; r < 32; ++r) {
             const int64_t m = (int64_t)m0 + q * 32 + r;
             if (m >= g.M) break;
-            const int64_t rbase = blockIdx.z * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
+            const int64_t rbase = (int64_t)bz * g.split_stride + (int64_t)((uint32_t)m / (uint32_t)g.c_d) * g.c_outer + (int64_t)((uint32_t)m % (uint32_t)g.c_d) * g.c_inner;
             float* crow = g.C + rbase;
             for (int c = lane; c < g.BN; c += 32) {
                 const int64_t n = (int64_t)n0 + c;
@@ -298,6 +322,15 @@ __global__ void k_reduce_parts(float* __restrict__ dst, const float* __restrict_
         dst[i] = s;
     }
 }
+struct ReduceRanges { ReduceRange r[kMaxReduceRanges]; };
+__global__ void k_reduce_ranges(float* __restrict__ dst, const float* __restrict__ part, int64_t stride, const ReduceRanges R) {
+    const ReduceRange rg = R.r[blockIdx.y];
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < rg.n; i += (int64_t)gridDim.x * blockDim.x) {
+        float s = dst[rg.off + i];
+        for (int z = 0; z < rg.splits; ++z) s += part[z * stride + rg.off + i];
+        dst[rg.off + i] = s;
+    }
+}
 }  // namespace
 
 namespace {
@@ -328,6 +361,20 @@ cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_
     return cudaGetLastError();
 }
 
+cudaError_t launch_reduce_ranges(float* dst, const float* part, int64_t stride, const ReduceRange* r, int nr, cudaStream_t s) {
+    if (nr <= 0) return cudaSuccess;
+    if (nr > kMaxReduceRanges) return cudaErrorInvalidValue;
+    ReduceRanges R{};
+    int64_t nmax = 0;
+    for (int i = 0; i < nr; ++i) { R.r[i] = r[i]; nmax = std::max(nmax, r[i].n); }
+    if (nmax <= 0) return cudaSuccess;
+    dim3 grid((unsigned)std::min<int64_t>((nmax + 255) / 256, 148 * 4), (unsigned)nr);
+    KernelTimer kt(K_GEMM, s);
+    k_reduce_ranges<<<grid, 256, 0, s>>>(dst, part, stride, R);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int s_d, int64_t rows, int cols,
                          int64_t ld, void* hi, void* lo, cudaStream_t s) {
     if (rows <= 0 || cols <= 0) return cudaSuccess;
@@ -352,13 +399,21 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 
 // C[M,N] (+)= A * B^T on tensor cores.  mn_major = 0: A[M][lda], B[N][ldb] (rows contiguous in k).
 // mn_major = 1: A^T[Kd][lda] (contiguous in m), B^T[Kd][ldb] (contiguous in n).
-cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
-                           int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
-                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
-                           int64_t split_stride, void* Chi, void* Clo, int passes) {
+// gemm_tc_add queues one product (launching what is queued when the batch is full); gemm_tc_flush launches the queue.
+cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
+                        int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
+                        int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
+                        int64_t split_stride, void* Chi, void* Clo, int passes) {
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
     if (M >= (int64_t(1) << 32)) return cudaErrorInvalidValue;   // the epilogue maps rows with 32-bit divisions
-    TcArgs g{};
+    TcBatch& B = *reinterpret_cast<TcBatch*>(gb.storage);
+    if (gb.n == TC_MAX_BATCH) {
+        cudaError_t e = gemm_tc_flush(gb, s);
+        if (e != cudaSuccess) return e;
+    }
+    TcProblem& pr = B.p[gb.n];
+    TcArgs& g = pr.g;
+    g = TcArgs{};
     g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate; g.passes = passes == 1 ? 1 : 3;
     g.M = M; g.N = N; g.Kd = Kd; g.mn_major = mn_major; g.status = status;
     g.splits = std::max(1, std::min<int>(splits, (int)((Kd + BK - 1) / BK))); g.split_stride = split_stride;
@@ -379,28 +434,55 @@ cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const 
     int cols = 32;
     while (cols < BN) cols <<= 1;
     g.tmem_cols = cols;
-    CUtensorMap tAh, tAl, tBh, tBl;
     bool ok;
     if (!mn_major) {
-        ok = make_map(&tAh, Ahi, Kd, M, lda, BK, BM) && make_map(&tAl, Alo, Kd, M, lda, BK, BM) &&
-             make_map(&tBh, Bhi, Kd, N, ldb, BK, BN) && make_map(&tBl, Blo, Kd, N, ldb, BK, BN);
+        ok = make_map(&pr.tmAh, Ahi, Kd, M, lda, BK, BM) && make_map(&pr.tmAl, Alo, Kd, M, lda, BK, BM) &&
+             make_map(&pr.tmBh, Bhi, Kd, N, ldb, BK, BN) && make_map(&pr.tmBl, Blo, Kd, N, ldb, BK, BN);
     } else {
-        ok = make_map(&tAh, Ahi, M, Kd, lda, 64, BK) && make_map(&tAl, Alo, M, Kd, lda, 64, BK) &&
-             make_map(&tBh, Bhi, N, Kd, ldb, 64, BK) && make_map(&tBl, Blo, N, Kd, ldb, 64, BK);
+        ok = make_map(&pr.tmAh, Ahi, M, Kd, lda, 64, BK) && make_map(&pr.tmAl, Alo, M, Kd, lda, 64, BK) &&
+             make_map(&pr.tmBh, Bhi, N, Kd, ldb, 64, BK) && make_map(&pr.tmBl, Blo, N, Kd, ldb, 64, BK);
     }
     if (!ok) return cudaErrorInvalidValue;
-    const size_t sh = (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16;
+    pr.gx = (uint32_t)((M + BM - 1) / BM);
+    pr.gy = (uint32_t)((N + BN - 1) / BN);
+    const uint64_t tiles = (uint64_t)pr.gx * pr.gy * (uint64_t)g.splits;
+    if (gb.n == 0) B.tile0[0] = 0;
+    if (tiles + B.tile0[gb.n] >= (uint64_t(1) << 31)) return cudaErrorInvalidValue;
+    B.tile0[gb.n + 1] = B.tile0[gb.n] + (uint32_t)tiles;
+    gb.sh = std::max(gb.sh, (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16);
+    ++gb.n;
+    return cudaSuccess;
+}
+
+cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s) {
+    if (gb.n == 0) return cudaSuccess;
+    TcBatch& B = *reinterpret_cast<TcBatch*>(gb.storage);
+    B.n = gb.n;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid((unsigned)((M + BM - 1) / BM), (unsigned)((N + BN - 1) / BN), (unsigned)g.splits);
-    KernelTimer kt(K_GEMM, s);
-    k_gemm_tc<<<grid, TC_THREADS, sh, s>>>(tAh, tAl, tBh, tBl, g);
-    count_launch();
+    const unsigned grid = B.tile0[gb.n];
+    {
+        KernelTimer kt(K_GEMM, s);
+        k_gemm_tc<<<grid, TC_THREADS, gb.sh, s>>>(B);
+        count_launch();
+    }
+    gb.n = 0; gb.sh = 0;
     return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
+                           int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
+                           int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
+                           int64_t split_stride, void* Chi, void* Clo, int passes) {
+    GemmBatch gb;
+    cudaError_t e = gemm_tc_add(gb, Ahi, Alo, lda, Bhi, Blo, ldb, C, c_outer, c_inner, c_d, M, N, Kd, accumulate, mn_major, status, s,
+                                splits, split_stride, Chi, Clo, passes);
+    if (e != cudaSuccess) return e;
+    return gemm_tc_flush(gb, s);
 }
 
 }  // namespace sobek

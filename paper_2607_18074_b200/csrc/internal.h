@@ -430,11 +430,27 @@ cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int
                          int64_t ld, void* hi, void* lo, cudaStream_t s);
 cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int transposed, int n_major,
                                const float* R, void* hi, void* lo, cudaStream_t s);
+// a queue of tensor-core products that one launch runs (gemm_tc.cu); plain storage so that only gemm_tc.cu needs the
+// tensor-map type
+struct GemmBatch {
+    alignas(64) unsigned char storage[4096];
+    size_t sh = 0;      // dynamic shared memory the queued products need
+    int n = 0;
+};
+cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
+                        int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
+                        int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
+                        int64_t split_stride, void* Chi, void* Clo, int passes);
+cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s);
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
                            int64_t split_stride = 0, void* Chi = nullptr, void* Clo = nullptr, int passes = 3);
 cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_t stride, int splits, cudaStream_t s);
+// the same for several column ranges of one [splits][stride] buffer in one launch: dst[off + i] += sum_z part[z][off + i]
+struct ReduceRange { int64_t off, n; int splits; };
+constexpr int kMaxReduceRanges = 8;
+cudaError_t launch_reduce_ranges(float* dst, const float* part, int64_t stride, const ReduceRange* r, int nr, cudaStream_t s);
 cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s);
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
