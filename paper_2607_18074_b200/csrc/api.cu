@@ -114,6 +114,14 @@ cudaError_t split_features(const float* src, int64_t N, int C, uint16_t* h, uint
     return launch_split(src, C, 0, 1, N, C, C, h, l, s);
 }
 
+// several of them in one launch
+struct FeatureSplits {
+    SplitJob j[kMaxSplitJobs];
+    int n = 0;
+    void add(const float* src, int64_t N, int C, uint16_t* h, uint16_t* l) { j[n++] = SplitJob{src, C, 0, 1, N, C, C, h, l}; }
+    cudaError_t flush(cudaStream_t s) { const int k = n; n = 0; return launch_split_jobs(j, k, s); }
+};
+
 int check_common(const sobek_plan* p, const sobek_graph* g, void* ws, size_t ws_bytes, int order) {
     if (!p || !g) return SOBEK_ERR_INVALID_ARG;
     if (g->N < 0 || g->E < 0) return SOBEK_ERR_INVALID_ARG;
@@ -159,17 +167,21 @@ bool has_uncovered(const Direction& d) {
 
 // rows (node, o) of the chunk's output adjoint -> bf16 (hi, lo), group by group
 cudaError_t split_adjoint(const sobek_plan* p, const Direction& dir, int64_t n0, int64_t nn, const float* gdst,
-                          uint16_t* gh, uint16_t* gl, cudaStream_t s0) {
-    Fork fork(p, s0);
+                          uint16_t* gh, uint16_t* gl, cudaStream_t s) {
+    SplitJob jobs[kMaxSplitJobs];
+    int nj = 0;
     for (size_t gi = 0; gi < dir.groups.size(); ++gi) {
-        cudaStream_t s = fork.pick();
         const DGroup& G = dir.groups[gi];
         if (G.path_end == G.path_begin) continue;
-        cudaError_t e = launch_split(gdst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst, nn * G.d_dst,
-                                     G.c_dst, dir.kn_ld[gi], gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi], s);
-        if (e != cudaSuccess) return e;
+        jobs[nj++] = SplitJob{gdst + n0 * dir.C_dst + G.dst_off, dir.C_dst, G.c_dst, G.d_dst, nn * G.d_dst, G.c_dst, dir.kn_ld[gi],
+                              gh + nn * dir.gb_off[gi], gl + nn * dir.gb_off[gi]};
+        if (nj == kMaxSplitJobs) {
+            cudaError_t e = launch_split_jobs(jobs, nj, s);
+            if (e != cudaSuccess) return e;
+            nj = 0;
+        }
     }
-    return fork.join();
+    return launch_split_jobs(jobs, nj, s);
 }
 
 // dst_g (+)= Z_g * Rp_g        (Eq. receiver_matrix_product)
@@ -393,10 +405,15 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
         CK(launch_reduce_parts(gR, w.part, KN, KN, n_parts, s));
         gR = nullptr;
     }
-    if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
-    if (w.gsh && gx && !w.fused_t && !gx_direct) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
+    FeatureSplits fs;
+    if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { fs.add(x, g->N, p->C_x, w.xsh, w.xsl); xs.h = w.xsh; xs.l = w.xsl; }
+    if (w.gsh && gx && !w.fused_t && !gx_direct) { fs.add(gy, g->N, p->C_y, w.gsh, w.gsl); gs.h = w.gsh; gs.l = w.gsl; }
+    CK(fs.flush(s));
+    PackQueue pq(p);              // every operand layout of R this call needs, one launch
+    if (gphi || gY) pq.add(p->fwd, 0, 0, R, w.fKNh, w.fKNl);
+    if (gx && !gx_direct && !w.fused_t) pq.add(p->tr, 1, 1, R, w.tNKh, w.tNKl);
+    CK(pq.flush(s));
     if (gR || gphi || gY) {
-        if (gphi || gY) CK(pack_R(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
         if (gR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
@@ -430,7 +447,6 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
             CK(launch_pack_R_fused(p, p->tr, 1, R, w.tFKh, w.tFKl, s));
             CK(launch_fused(p, p->tr, sv, gy, nullptr, Y, nullptr, phi, nullptr, 0, w.tFKh, w.tFKl, gx, 0, w.status, s));
         } else {
-            CK(pack_R(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
             for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
                 const int64_t nn = std::min(w.chunk, g->N - n0);
                 CK(launch_stream(p, p->tr, sv, n0, nn, gy, nullptr, gs, Y, nullptr, phi, nullptr, 0, w.zbh, w.zbl, w.status, s));
@@ -485,11 +501,27 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
     SplitSrc xs{}, gs{};
     if (geo) { xs = *geo; gs = *geo; }
     const bool tc_edge_plain = w.zqh != nullptr, tc_edge_dual = tc_edge_plain && p->fwd.etc[1].ok && (!vx || w.vsh);
+    FeatureSplits fs;
     if (w.xsh && (ggy || hR || ((hphi || hY) && tc_edge_plain))) {
-        CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl;
-        if (vx && w.vsh) { CK(split_features(vx, g->N, p->C_x, w.vsh, w.vsl, s)); xs.vh = w.vsh; xs.vl = w.vsl; }
+        fs.add(x, g->N, p->C_x, w.xsh, w.xsl); xs.h = w.xsh; xs.l = w.xsl;
+        if (vx && w.vsh) { fs.add(vx, g->N, p->C_x, w.vsh, w.vsl); xs.vh = w.vsh; xs.vl = w.vsl; }
     }
-    if (w.gsh && hx && !w.fused_t) { CK(split_features(gy, g->N, p->C_y, w.gsh, w.gsl, s)); gs.h = w.gsh; gs.l = w.gsl; }
+    if (w.gsh && hx && !w.fused_t) { fs.add(gy, g->N, p->C_y, w.gsh, w.gsl); gs.h = w.gsh; gs.l = w.gsl; }
+    CK(fs.flush(s));
+    {
+        // every operand layout of R and vR this call needs, one launch (the fused schedule packs its own)
+        const bool fuse_ggy = ggy && w.fused_f, fuse_dz = fuse_ggy && !hR;
+        PackQueue pq(p);
+        if (ggy && any_edge_dir && !fuse_dz) pq.add(p->fwd, 0, 1, R, w.fNKh, w.fNKl);
+        if (ggy && vR && !fuse_ggy) pq.add(p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl);
+        if ((hphi || hY) && any_edge_dir) pq.add(p->fwd, 0, 0, R, w.fKNh, w.fKNl);
+        if ((hphi || hY) && vR) pq.add(p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl);
+        if (hx && !w.fused_t) {
+            if (vY || vphi) pq.add(p->tr, 1, 1, R, w.tNKh, w.tNKl);
+            if (vR) pq.add(p->tr, 1, 1, vR, w.vtNKh, w.vtNKl);
+        }
+        CK(pq.flush(s));
+    }
     if (ggy || hR || hphi || hY) {
         if (ggy && has_uncovered(p->fwd)) CK(launch_fill_zero(ggy, g->N * (int64_t)p->C_y, s));
         // ggy = Z vR + dZ R.  The fused kernels produce it without leaving the SM; when hR is wanted too the
@@ -507,10 +539,6 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
             CK(launch_fused(p, p->fwd, rv, x, vx, Y, vY, phi, vphi, 1, w.fFKh, w.fFKl, ggy, ggy_done, w.status, s));
             ggy_done = 1;
         }
-        if (ggy && any_edge_dir && !fuse_dz) CK(pack_R(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
-        if (ggy && vR && !fuse_ggy) CK(pack_R(p, p->fwd, 0, 1, vR, w.vfNKh, w.vfNKl, s));
-        if ((hphi || hY) && any_edge_dir) CK(pack_R(p, p->fwd, 0, 0, R, w.fKNh, w.fKNl, s));
-        if ((hphi || hY) && vR) CK(pack_R(p, p->fwd, 0, 0, vR, w.vfKNh, w.vfKNl, s));
         if (hR) CK(launch_fill_zero(w.gRp, KN, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
@@ -575,8 +603,6 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
             }
             return SOBEK_OK;
         }
-        if (vY || vphi) CK(pack_R(p, p->tr, 1, 1, R, w.tNKh, w.tNKl, s));
-        if (vR) CK(pack_R(p, p->tr, 1, 1, vR, w.vtNKh, w.vtNKl, s));
         for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
             const int64_t nn = std::min(w.chunk, g->N - n0);
             int wrote = 0;

@@ -281,6 +281,51 @@ __global__ void k_split(const float* __restrict__ src, int64_t s_outer, int64_t 
     }
 }
 
+// several such packings (directions, layouts, R or its direction vR) in one launch: blockIdx.z picks the job
+struct PackJobsArg { PackJob j[kMaxPackJobs]; int K; int64_t N_w; };
+__global__ void k_pack_R_jobs(const PackJobsArg J) {
+    const PackJob q = J.j[blockIdx.z];
+    if ((int)blockIdx.y >= q.n_paths) return;
+    const DPath P = q.paths[blockIdx.y];
+    const int gi = q.path_group[blockIdx.y];
+    const int64_t base = q.grp_off[gi];
+    const int64_t ld = q.grp_ld[gi];
+    const int K = J.K;
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(q.hi);
+    __nv_bfloat16* lo = reinterpret_cast<__nv_bfloat16*>(q.lo);
+    const int64_t total = (int64_t)K * P.c_src * P.c_dst;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(i % P.c_dst);
+        const int64_t r = i / P.c_dst;
+        const int k1 = (int)(r % K);
+        const int us = (int)(r / K);
+        const int u = q.transposed ? n : us, w = q.transposed ? us : n;
+        const float v = q.R[(int64_t)k1 * J.N_w + P.w_off + (int64_t)u * P.c_out + w];
+        const int64_t k = (int64_t)P.koff + (int64_t)k1 * P.c_src + us;
+        const int64_t o = q.n_major ? base + (int64_t)n * ld + k : base + k * ld + n;
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[o] = h;
+        lo[o] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// the same for several (source, destination) pairs in one launch: blockIdx.y picks the job
+struct SplitJobs { SplitJob j[kMaxSplitJobs]; };
+__global__ void k_split_jobs(const SplitJobs J) {
+    const SplitJob q = J.j[blockIdx.y];
+    const int64_t total = q.rows * q.cols;
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(q.hi);
+    __nv_bfloat16* lo = reinterpret_cast<__nv_bfloat16*>(q.lo);
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / q.cols;
+        const int c = (int)(i - r * q.cols);
+        const float v = q.src[(r / q.s_d) * q.s_outer + (r % q.s_d) * q.s_inner + c];
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[r * q.ld + c] = h;
+        lo[r * q.ld + c] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
 // R[K, N_w] -> bf16 hi/lo GEMM operands of one direction, per group g:
 //   layout KN (n_major = 0): [k][c_dst] rows of length ldn_g      (B operand of Zbar = gy Rp^T)
 //   layout NK (n_major = 1): [c_dst][k] rows of length ldk_g      (B operand of y = Z Rp)
@@ -357,6 +402,41 @@ cudaError_t launch_reduce_parts(float* dst, const float* part, int64_t n, int64_
     const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
     KernelTimer kt(K_GEMM, s);
     k_reduce_parts<<<blocks, 256, 0, s>>>(dst, part, n, stride, splits);
+    count_launch();
+    return cudaGetLastError();
+}
+
+void PackQueue::add(const Direction& dir, int transposed, int n_major, const float* R, void* hi, void* lo) {
+    if (p->uvu || n >= kMaxPackJobs) { overflow = overflow || (!p->uvu && n >= kMaxPackJobs); return; }
+    j[n++] = PackJob{dir.d_paths, n_major ? dir.d_nk_off : dir.d_kn_off, n_major ? dir.d_nk_ld : dir.d_kn_ld, dir.d_path_group,
+                     (int)dir.paths.size(), transposed, n_major, R, hi, lo};
+}
+cudaError_t PackQueue::flush(cudaStream_t s) {
+    if (overflow) return cudaErrorInvalidValue;
+    if (n == 0) return cudaSuccess;
+    PackJobsArg J{};
+    int max_paths = 0;
+    for (int i = 0; i < n; ++i) { J.j[i] = j[i]; max_paths = std::max(max_paths, j[i].n_paths); }
+    J.K = p->K; J.N_w = p->N_w;
+    dim3 grid(32, (unsigned)max_paths, (unsigned)n);
+    n = 0;
+    if (max_paths == 0) return cudaSuccess;
+    KernelTimer kt(K_PACK, s);
+    k_pack_R_jobs<<<grid, 256, 0, s>>>(J);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split_jobs(const SplitJob* jobs, int n, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    if (n > kMaxSplitJobs) return cudaErrorInvalidValue;
+    SplitJobs J{};
+    int64_t tmax = 0;
+    for (int i = 0; i < n; ++i) { J.j[i] = jobs[i]; tmax = std::max(tmax, jobs[i].rows * jobs[i].cols); }
+    if (tmax <= 0) return cudaSuccess;
+    dim3 grid((unsigned)std::min<int64_t>((tmax + 255) / 256, 148 * 8), (unsigned)n);
+    KernelTimer kt(K_PACK, s);
+    k_split_jobs<<<grid, 256, 0, s>>>(J);
     count_launch();
     return cudaGetLastError();
 }

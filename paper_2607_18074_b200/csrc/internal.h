@@ -426,6 +426,28 @@ SOBEK_FUSED_DECL(fused_launch_k16_dual);
 
 // --- gemm_tc.cu ---------------------------------------------------------------------
 int64_t round8(int64_t v);
+// the packings of R (or of its direction vR) into GEMM operand layouts that one call needs, queued and run as one launch
+struct PackJob {
+    const DPath* paths; const int64_t* grp_off; const int32_t* grp_ld; const int32_t* path_group;
+    int n_paths, transposed, n_major;
+    const float* R; void* hi; void* lo;
+};
+constexpr int kMaxPackJobs = 6;
+struct PackQueue {
+    const sobek_plan* p;
+    PackJob j[kMaxPackJobs];
+    int n = 0;
+    bool overflow = false;
+    explicit PackQueue(const sobek_plan* plan) : p(plan) {}
+    // n_major = 1: [c_dst][k] rows (B operand of y = Z Rp); 0: [k][c_dst] rows (B operand of Zbar = gy Rp^T); no-op in
+    // the channelwise mode, which has no operand copies
+    void add(const Direction& dir, int transposed, int n_major, const float* R, void* hi, void* lo);
+    cudaError_t flush(cudaStream_t s);
+};
+// several fp32 -> (bf16 hi, lo) conversions with mapped source rows in one launch (see launch_split)
+struct SplitJob { const float* src; int64_t s_outer, s_inner; int s_d; int64_t rows; int cols; int64_t ld; void* hi; void* lo; };
+constexpr int kMaxSplitJobs = 8;
+cudaError_t launch_split_jobs(const SplitJob* jobs, int n, cudaStream_t s);
 cudaError_t launch_split(const float* src, int64_t s_outer, int64_t s_inner, int s_d, int64_t rows, int cols,
                          int64_t ld, void* hi, void* lo, cudaStream_t s);
 cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int transposed, int n_major,
