@@ -20,6 +20,8 @@
 // kernel always reaches its TMEM release and returns.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -538,6 +540,12 @@ cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s) {
     if (gb.n == 0) return cudaSuccess;
     TcBatch& B = *reinterpret_cast<TcBatch*>(gb.storage);
     B.n = gb.n;
+    // longest contraction first: the CTAs that run longest start first, the short ones fill the tail
+    std::stable_sort(B.p, B.p + gb.n, [](const TcProblem& x, const TcProblem& y) {
+        return (x.g.Kd + x.g.splits - 1) / x.g.splits > (y.g.Kd + y.g.splits - 1) / y.g.splits;
+    });
+    B.tile0[0] = 0;
+    for (int i = 0; i < gb.n; ++i) B.tile0[i + 1] = B.tile0[i] + B.p[i].gx * B.p[i].gy * (uint32_t)B.p[i].g.splits;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
