@@ -116,15 +116,34 @@ def geo_bwd(orc, row_ptr, col, rvec, x, R, gy, r_c: float, basis: int = BESSEL, 
     return gx, g_rvec.numpy(), gR
 
 
-def geo_dbwd(orc, row_ptr, col, rvec, x, R, gy, vx, v_rvec, vR, r_c: float, basis: int = BESSEL, p: int = 6, act=None):
-    """(ggy, hx, hR): derivatives of  <vx, gx> + <v_rvec, g_rvec> + <vR, gR>  (the adjoints of geo_bwd) with respect to
-    gy, x and R -- what a loss on the forces needs for its parameter and feature gradients.  Since
+def geo_dbwd(orc, row_ptr, col, rvec, x, R, gy, vx, v_rvec, vR, r_c: float, basis: int = BESSEL, p: int = 6, act=None,
+             with_h_rvec: bool = False):
+    """(ggy, hx, hR): derivatives of  Phi = <vx, gx> + <v_rvec, g_rvec> + <vR, gR>  (the adjoints of geo_bwd) with respect
+    to gy, x and R -- what a loss on the forces needs for its parameter and feature gradients.  Since
     <v_rvec, g_rvec> = <J_Y v_rvec, gY> + <J_phi v_rvec, gphi>, this is the double backward of the convolution with the
     directions vY = J_Y v_rvec and vphi = J_phi v_rvec (Jacobian-vector products of the definitions above, by
-    torch.autograd).  The derivative with respect to rvec itself (second derivatives of both bases) is not provided."""
+    torch.autograd).
+
+    with_h_rvec: also h_rvec = dPhi / d rvec, returned as a fourth array.  Phi depends on the edge vector of an edge
+    through Y_e, phi_e (inside gx, gR, gY, gphi: the convolution's own second-order edge adjoints hY, hphi, pulled back
+    through the Jacobians) and through the Jacobians in g_rvec = J_Y^T gY + J_phi^T gphi themselves (second derivatives
+    of both bases, contracted with the first-order adjoints gY, gphi and the direction):
+        h_rvec_e = J_Y^T hY_e + J_phi^T hphi_e + d/dr [ <J_Y(r) v_e, gY_e> + <J_phi(r) v_e, gphi_e> ]  (gY, gphi held fixed)."""
     t = torch.as_tensor(np.asarray(rvec, dtype=np.float64))
     v = torch.as_tensor(np.asarray(v_rvec, dtype=np.float64))
-    Y, vY = torch.autograd.functional.jvp(lambda r: real_sh(r, orc.l_max), t, v)
-    phi, vphi = torch.autograd.functional.jvp(lambda r: radial(torch.linalg.norm(r, dim=-1), orc.K, r_c, basis, p), t, v)
-    ggy, hx, _, _, hR = orc.dbwd(row_ptr, col, x, Y.numpy(), phi.numpy(), R, gy, vx, vY.numpy(), vphi.numpy(), vR, act=act)
-    return ggy, hx, hR
+    sh = lambda r: real_sh(r, orc.l_max)
+    rad = lambda r: radial(torch.linalg.norm(r, dim=-1), orc.K, r_c, basis, p)
+    Y, vY = torch.autograd.functional.jvp(sh, t, v)
+    phi, vphi = torch.autograd.functional.jvp(rad, t, v)
+    ggy, hx, hY, hphi, hR = orc.dbwd(row_ptr, col, x, Y.numpy(), phi.numpy(), R, gy, vx, vY.numpy(), vphi.numpy(), vR, act=act)
+    if not with_h_rvec:
+        return ggy, hx, hR
+    _, gY, gphi, _ = orc.bwd(row_ptr, col, x, Y.numpy(), phi.numpy(), R, gy, act=act)
+    tt = t.clone().requires_grad_(True)
+    # first part: the pull-back of hY, hphi; second part: the derivative of the Jacobians along v, with gY, gphi fixed
+    first = (sh(tt) * torch.as_tensor(hY)).sum() + (rad(tt) * torch.as_tensor(hphi)).sum()
+    _, Yv = torch.autograd.functional.jvp(sh, tt, v, create_graph=True)
+    _, phiv = torch.autograd.functional.jvp(rad, tt, v, create_graph=True)
+    second = (Yv * torch.as_tensor(gY)).sum() + (phiv * torch.as_tensor(gphi)).sum()
+    (h_rvec,) = torch.autograd.grad(first + second, tt)
+    return ggy, hx, hR, h_rvec.numpy()

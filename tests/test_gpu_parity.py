@@ -461,12 +461,14 @@ def test_scratch_budget():
     assert rel_err(got[2][ed], ref[2][ed]) <= BWD_TOL and rel_err(got[3][ed], ref[3][ed]) <= BWD_TOL
 
 
-def test_cuda_graph_capture(cases):
+@pytest.mark.parametrize("name", ["cfg2_N200", "uvu_32x4_K16"])
+def test_cuda_graph_capture(cases, name):
     """A call neither allocates nor synchronises, and its side streams fork from and join the caller's
-    stream with events, so the three orders can be captured into one CUDA graph and replayed."""
+    stream with events, so the three orders can be captured into one CUDA graph and replayed (fully connected mode;
+    channelwise mode with its direct kernels)."""
     import torch
     import paper_2607_18074_b200 as sb
-    c = get(cases, "cfg2_N200")
+    c = get(cases, name) if name in CASES else Case(uvu_cases()[name])
     i = c.plan.info
     eager = [c.fwd()] + c.bwd() + c.dbwd()
     new = lambda *s: torch.full(s, float("nan"), dtype=torch.float32, device="cuda:0")

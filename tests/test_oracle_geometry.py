@@ -201,3 +201,32 @@ def test_force_loss_double_backward_by_central_differences():
     g2 = geometry.geo_dbwd(o, d.row_ptr, d.col, rv, d.x, d.R, d.gy, d.vx, np.zeros_like(rv), d.vR, w.r_c)
     ref = o.dbwd(d.row_ptr, d.col, d.x, d.Y, d.phi, d.R, d.gy, d.vx, np.zeros_like(d.vY), np.zeros_like(d.vphi), d.vR)
     assert np.allclose(g2[0], ref[0], atol=1e-11) and np.allclose(g2[1], ref[1], atol=1e-11) and np.allclose(g2[2], ref[4], atol=1e-11)
+
+
+def test_second_order_edge_vector_adjoint_by_central_differences():
+    """h_rvec of geo_dbwd (with_h_rvec) against central differences of  Phi = <vx, gx> + <v_r, g_r> + <vR, gR>  with
+    respect to entries of the edge vectors, Phi evaluated with geo_bwd; both radial bases."""
+    for basis, seed in ((geometry.BESSEL, 5), (geometry.GAUSSIAN, 6)):
+        o, w, d = _tiny(seed=seed)
+        rv = geometry.edge_vectors(d.col, d.recv, d.pos)
+        rng = np.random.default_rng(13)
+        v_r = rng.standard_normal(rv.shape)
+        out = geometry.geo_dbwd(o, d.row_ptr, d.col, rv, d.x, d.R, d.gy, d.vx, v_r, d.vR, w.r_c, basis, with_h_rvec=True)
+        assert len(out) == 4
+        h_r = out[3]
+        # the first three outputs do not depend on the flag
+        for a, b in zip(out[:3], geometry.geo_dbwd(o, d.row_ptr, d.col, rv, d.x, d.R, d.gy, d.vx, v_r, d.vR, w.r_c, basis)):
+            assert np.allclose(a, b, rtol=1e-12, atol=1e-12 * np.abs(b).max())
+
+        def Phi(r):
+            gx, g_r, gR = geometry.geo_bwd(o, d.row_ptr, d.col, r, d.x, d.R, d.gy, w.r_c, basis)
+            return (d.vx * gx).sum() + (v_r * g_r).sum() + (d.vR * gR).sum()
+
+        scale = np.abs(h_r).max()
+        assert scale > 1e-6
+        h = 1e-5
+        for _ in range(8):
+            e, k = int(rng.integers(rv.shape[0])), int(rng.integers(3))
+            dp = np.zeros_like(rv); dp[e, k] = h
+            fd = (Phi(rv + dp) - Phi(rv - dp)) / (2 * h)
+            assert abs(fd - h_r[e, k]) < 2e-6 * scale + 1e-9
