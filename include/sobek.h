@@ -270,7 +270,15 @@ int sobek_conv_dbwd(const sobek_plan* plan, const sobek_graph* g,
  *                          hR = d<v,b>/dR (Eqs. streamed_directional_terms .. streamed_operand_second_adjoints with
  *                          the directions vY = J_Y v_rvec, vphi = J_phi v_rvec, which the dual stream passes compute
  *                          from rvec and v_rvec themselves).  Any of the cotangents and of the outputs may be NULL.  The
- *                          derivative with respect to rvec itself (second derivatives of both bases) is not provided.
+ *                          derivative with respect to rvec itself is what sobek_conv_geo_dbwd_full adds.
+ * sobek_conv_geo_dbwd_full the same three outputs plus h_rvec [E][3] = d<v,b>/d rvec (second derivatives of both
+ *                          bases): h_rvec_e = J_Y^T hY_e + J_phi^T hphi_e + d/dr [<J_Y(r) v_e, gY_e> + <J_phi(r) v_e,
+ *                          gphi_e>] with the first- and second-order edge adjoints of the convolution.  NOT streaming
+ *                          in the edge inputs: Y, phi, their directions and the four edge adjoints are materialised in
+ *                          the workspace (8 arrays of E x dim_sh or E x K floats) around stored-input calls of
+ *                          sobek_conv_bwd and sobek_conv_dbwd, so every plan those accept is accepted (l_max <= 4,
+ *                          K <= 32; else UNSUPPORTED).  Workspace: sobek_geo_dbwd_full_workspace_bytes(plan, N, E).
+ *                          Any of vx, v_rvec, vR and of the four outputs may be NULL.
  * sobek_position_gradient  gpos[n] = sum_{e: sender(e) = n} g_rvec[e] - sum_{e: receiver(e) = n} g_rvec[e], the
  *                          adjoint of sobek_edge_vectors (forces are its negative); each node sums its own edges in
  *                          a fixed order (needs src_ptr and src_perm).  Only enqueues.
@@ -288,6 +296,11 @@ int sobek_conv_geo_dbwd(const sobek_plan* plan, const sobek_graph* g, const floa
                         int envelope_p, const float* x, const float* R, const float* gy, const float* vx,
                         const float* v_rvec, const float* vR, float* ggy, float* hx, float* hR, void* ws,
                         size_t ws_bytes, void* stream);
+size_t sobek_geo_dbwd_full_workspace_bytes(const sobek_plan* plan, int64_t N, int64_t E);
+int sobek_conv_geo_dbwd_full(const sobek_plan* plan, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                             int envelope_p, const float* x, const float* R, const float* gy, const float* vx,
+                             const float* v_rvec, const float* vR, float* ggy, float* hx, float* hR, float* h_rvec,
+                             void* ws, size_t ws_bytes, void* stream);
 int sobek_position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, void* stream);
 
 /*

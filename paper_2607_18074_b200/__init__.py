@@ -39,6 +39,7 @@ EXPORTS = [
     "sobek_timing_collect", "sobek_static_scratch_bytes", "sobek_conv_fwd_static", "sobek_selftest_wait_timeout",
     "sobek_conv_fwd_retain", "sobek_conv_bwd_retained", "sobek_static_last_status", "sobek_measure_fp32_peak",
     "sobek_edge_vectors", "sobek_conv_geo_fwd", "sobek_conv_geo_bwd", "sobek_conv_geo_dbwd", "sobek_position_gradient",
+    "sobek_geo_dbwd_full_workspace_bytes", "sobek_conv_geo_dbwd_full",
 ]
 BASIS_BESSEL, BASIS_GAUSSIAN = 0, 1
 
@@ -104,6 +105,9 @@ def lib():
         L.sobek_conv_geo_fwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 4 + [c_size_t, c_void_p]
         L.sobek_conv_geo_bwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 7 + [c_size_t, c_void_p]
         L.sobek_conv_geo_dbwd.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 10 + [c_size_t, c_void_p]
+        L.sobek_conv_geo_dbwd_full.argtypes = [c_void_p, POINTER(Graph), c_void_p, c_int, c_float, c_int] + [c_void_p] * 11 + [c_size_t, c_void_p]
+        L.sobek_geo_dbwd_full_workspace_bytes.argtypes = [c_void_p, c_int64, c_int64]
+        L.sobek_geo_dbwd_full_workspace_bytes.restype = c_size_t
         L.sobek_selftest_wait_timeout.argtypes = [c_void_p, c_uint, c_void_p]
         L.sobek_last_device_status.argtypes = [c_void_p, c_void_p]
         L.sobek_static_scratch_bytes.restype = c_size_t
@@ -317,6 +321,18 @@ def conv_geo_dbwd(plan, graph, rvec, basis, r_cut, envelope_p, x, R, gy, vx, v_r
     _check(lib().sobek_conv_geo_dbwd(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
                                      _ptr(x), _ptr(R), _ptr(gy), _ptr(vx), _ptr(v_rvec), _ptr(vR), _ptr(ggy), _ptr(hx),
                                      _ptr(hR), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "sobek_conv_geo_dbwd")
+
+
+def geo_dbwd_full_workspace_bytes(plan, N: int, E: int) -> int:
+    return int(lib().sobek_geo_dbwd_full_workspace_bytes(plan.handle, int(N), int(E)))
+
+
+def conv_geo_dbwd_full(plan, graph, rvec, basis, r_cut, envelope_p, x, R, gy, vx, v_rvec, vR, ggy, hx, hR, h_rvec, ws):
+    """sobek_conv_geo_dbwd_full: the outputs of conv_geo_dbwd plus h_rvec [E, 3]; ws of geo_dbwd_full_workspace_bytes."""
+    _check(lib().sobek_conv_geo_dbwd_full(plan.handle, byref(graph), _ptr(rvec), int(basis), float(r_cut), int(envelope_p),
+                                          _ptr(x), _ptr(R), _ptr(gy), _ptr(vx), _ptr(v_rvec), _ptr(vR), _ptr(ggy),
+                                          _ptr(hx), _ptr(hR), _ptr(h_rvec), _ptr(ws), ws.numel() * ws.element_size(),
+                                          _stream()), "sobek_conv_geo_dbwd_full")
 
 
 def conv_fwd_retain(plan, graph, x, Y, phi, R, y, ws) -> int:

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libsobek.so")
 SOURCES = ["plan.cu", "graph.cu", "kernels.cu", "edge_stream.cu", "edge_stream_k8.cu", "edge_stream_k8d.cu",
-           "edge_stream_k16.cu", "edge_stream_k16d.cu", "stream_tc.cu", "edge_pass.cu", "edge_pass_tc.cu", "fused.cu", "fused_k8.cu", "fused_k8d.cu", "fused_k16.cu", "fused_k16d.cu", "gemm_tc.cu", "node_uvu.cu", "uvu_direct.cu", "api.cu", "static_scratch.cu"]
+           "edge_stream_k16.cu", "edge_stream_k16d.cu", "stream_tc.cu", "edge_pass.cu", "edge_pass_tc.cu", "fused.cu", "fused_k8.cu", "fused_k8d.cu", "fused_k16.cu", "fused_k16d.cu", "gemm_tc.cu", "node_uvu.cu", "uvu_direct.cu", "geometry_second.cu", "api.cu", "static_scratch.cu"]
 FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
          "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -728,6 +728,57 @@ extern "C" int sobek_conv_geo_dbwd(const sobek_plan* p, const sobek_graph* g, co
                           ws_bytes, stream, &geo);
 }
 
+// the eight edge arrays of sobek_conv_geo_dbwd_full behind the workspace of the stored-input calls
+namespace {
+struct GeoFullWs { size_t core; float *Y, *vY, *gY, *hY, *phi, *vphi, *gphi, *hphi; size_t bytes; };
+GeoFullWs geo_full_carve(const sobek_plan* p, int64_t N, int64_t E, void* ws) {
+    GeoFullWs w{};
+    w.core = (std::max(sobek_workspace_bytes(p, N, E, 1), sobek_workspace_bytes(p, N, E, 2)) + 255) & ~size_t(255);
+    size_t off = w.core;
+    auto take = [&](size_t n) { float* q = ws ? reinterpret_cast<float*>((char*)ws + off) : nullptr; off += (n * 4 + 255) & ~size_t(255); return q; };
+    const size_t ny = (size_t)E * p->dim_sh, nk = (size_t)E * p->K;
+    w.Y = take(ny); w.vY = take(ny); w.gY = take(ny); w.hY = take(ny);
+    w.phi = take(nk); w.vphi = take(nk); w.gphi = take(nk); w.hphi = take(nk);
+    w.bytes = off;
+    return w;
+}
+}  // namespace
+
+extern "C" size_t sobek_geo_dbwd_full_workspace_bytes(const sobek_plan* p, int64_t N, int64_t E) {
+    if (!p || N < 0 || E < 0) return 0;
+    return geo_full_carve(p, N, E, nullptr).bytes;
+}
+
+extern "C" int sobek_conv_geo_dbwd_full(const sobek_plan* p, const sobek_graph* g, const float* rvec, int basis, float r_cut,
+                                        int envelope_p, const float* x, const float* R, const float* gy, const float* vx,
+                                        const float* v_rvec, const float* vR, float* ggy, float* hx, float* hR,
+                                        float* h_rvec, void* ws, size_t ws_bytes, void* stream) {
+    if (!p || !g) return SOBEK_ERR_INVALID_ARG;
+    if (g->E > 0 && !rvec) return SOBEK_ERR_INVALID_ARG;
+    if (basis != SOBEK_BASIS_BESSEL && basis != SOBEK_BASIS_GAUSSIAN) return SOBEK_ERR_INVALID_ARG;
+    if (!(r_cut > 0.f) || (basis == SOBEK_BASIS_BESSEL && envelope_p < 1)) return SOBEK_ERR_INVALID_ARG;
+    if (!geo_second_supported(p->l_max, p->K)) return SOBEK_ERR_UNSUPPORTED;
+    if (!aligned16(rvec, v_rvec, h_rvec)) return SOBEK_ERR_INVALID_ARG;
+    if (!ws || ((uintptr_t)ws & 255)) return SOBEK_ERR_WORKSPACE;
+    const GeoFullWs w = geo_full_carve(p, g->N, g->E, ws);
+    if (ws_bytes < w.bytes) return SOBEK_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    CK(launch_geo_edge_inputs(rvec, v_rvec, g->E, p->l_max, p->K, r_cut, basis, envelope_p, w.Y, w.phi, w.vY, w.vphi, s));
+    int rc;
+    if (h_rvec) {       // the first-order edge adjoints, which the derivative of the Jacobians is contracted with
+        if ((rc = sobek_conv_bwd(p, g, x, w.Y, w.phi, R, gy, nullptr, w.gY, w.gphi, nullptr, ws, w.core, stream))) return rc;
+    }
+    const float* vYp = v_rvec ? w.vY : nullptr;
+    const float* vpp = v_rvec ? w.vphi : nullptr;
+    if ((rc = sobek_conv_dbwd(p, g, x, w.Y, w.phi, R, gy, vx, vYp, vpp, vR, ggy, hx, h_rvec ? w.hY : nullptr,
+                              h_rvec ? w.hphi : nullptr, hR, ws, w.core, stream)))
+        return rc;
+    if (h_rvec)
+        CK(launch_geo_second_adjoint(rvec, v_rvec, g->E, p->l_max, p->K, r_cut, basis, envelope_p, w.gY, w.gphi, w.hY, w.hphi,
+                                     h_rvec, s));
+    return SOBEK_OK;
+}
+
 extern "C" int sobek_conv_fwd_retain(const sobek_plan* p, const sobek_graph* g, const float* x, const float* Y,
                                      const float* phi, const float* R, float* y, void* ws, size_t ws_bytes,
                                      void* stream, int* retained) {

@@ -477,6 +477,13 @@ cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s)
 constexpr int kMaxSplits = 8;                                  // split-K pieces of the weight-adjoint GEMM
 constexpr size_t kPartBudgetBytes = size_t(64) << 20;          // bound on its partial-result buffer
 
+// --- geometry_second.cu: second-order geometry by hyper-dual evaluation of the bases --------------------
+bool geo_second_supported(int l_max, int K);
+cudaError_t launch_geo_edge_inputs(const float* rvec, const float* vrvec, int64_t E, int l_max, int K, float r_c, int basis, int p,
+                                   float* Y, float* phi, float* vY, float* vphi, cudaStream_t s);
+cudaError_t launch_geo_second_adjoint(const float* rvec, const float* vrvec, int64_t E, int l_max, int K, float r_c, int basis,
+                                      int p, const float* gY, const float* gphi, const float* hY, const float* hphi,
+                                      float* h_rvec, cudaStream_t s);
 // --- uvu_direct.cu ------------------------------------------------------------------------
 void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out);
 // transposed = 0: y[N, C_y] from src = x on the receiver view; 1: gx[N, C_x] from src = gy on the sender view

@@ -152,6 +152,48 @@ def test_force_loss_double_backward(name):
     assert part[0] is None and part[2] is None and np.array_equal(part[1], full[1])
 
 
+@pytest.mark.parametrize("name", ["cfg2_N200", "cfg5_N60", "tc_K6_dense", "gauss_K12"])
+def test_second_order_edge_vector_adjoint(name):
+    """sobek_conv_geo_dbwd_full: ggy, hx, hR as the streaming double backward, and h_rvec = d<v, b>/d rvec (second
+    derivatives of the spherical harmonics and the radial basis) against the oracle; single directions; NULL outputs."""
+    import torch
+    c = GeoCase(CASES[name])
+    d, i = c.d, c.plan.info
+    v_r = np.random.default_rng(19).standard_normal((c.E, 3))
+    v_rt = torch.from_numpy(v_r.astype(np.float32)).to("cuda:0")
+    v_r = v_rt.cpu().numpy().astype(np.float64)
+    ws = torch.empty(c.sb.geo_dbwd_full_workspace_bytes(c.plan, c.N, c.E), dtype=torch.uint8, device="cuda:0")
+
+    def run(dirs=(True, True, True), outs=(True, True, True, True)):
+        res = [c._new(c.N, i.C_y), c._new(c.N, i.C_x), c._new(i.K, i.N_w), c._new(c.E, 3)]
+        o = [t if on else None for t, on in zip(res, outs)]
+        v = [t if on else None for t, on in zip((c.vx, v_rt, c.vR), dirs)]
+        c.sb.conv_geo_dbwd_full(c.plan, c.graph, c.rvec, c.basis, c.w.r_c, 6, c.x, c.R, c.gy, *v, *o, ws)
+        assert c.sb.last_device_status(ws) == 0
+        return [None if t is None else t.cpu().numpy() for t in o]
+
+    def ref(dirs=(True, True, True)):
+        z = lambda a, on: a if on else np.zeros_like(a)
+        return geometry.geo_dbwd(c.oracle, d.row_ptr, d.col, c.o_rvec, d.x, d.R, d.gy, z(d.vx, dirs[0]), z(v_r, dirs[1]),
+                                 z(d.vR, dirs[2]), c.w.r_c, c.basis, with_h_rvec=True)
+
+    got, want = run(), ref()
+    for a, b, nm in zip(got, want, ("ggy", "hx", "hR", "h_rvec")):
+        assert np.isfinite(a).all() and np.abs(b).max() > 1e-3 and rel_err(a, b) <= BWD_TOL, nm
+    for dirs in [(False, True, False), (True, False, True)]:
+        got, want = run(dirs), ref(dirs)
+        for a, b, nm in zip(got, want, ("ggy", "hx", "hR", "h_rvec")):
+            assert (rel_err(a, b) <= BWD_TOL if np.abs(b).max() > 0 else np.all(a == 0)), (dirs, nm)
+    full = run()
+    part = run(outs=(False, False, False, True))
+    assert part[0] is None and part[1] is None and part[2] is None and np.array_equal(part[3], full[3])
+    # the streaming entry point computes the same three outputs
+    three = [c._new(c.N, i.C_y), c._new(c.N, i.C_x), c._new(i.K, i.N_w)]
+    c.sb.conv_geo_dbwd(c.plan, c.graph, c.rvec, c.basis, c.w.r_c, 6, c.x, c.R, c.gy, c.vx, v_rt, c.vR, *three, c.ws(2))
+    for a, t in zip(full[:3], three):
+        assert rel_err(a, t.cpu().numpy().astype(np.float64)) <= BWD_TOL
+
+
 def test_partial_outputs_and_argument_errors():
     c = GeoCase(CASES["cfg3_N120"])
     full = c.geo_bwd()

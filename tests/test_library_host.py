@@ -123,6 +123,9 @@ def test_argument_errors_are_status_codes():
     assert L.sobek_conv_geo_fwd(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, None, None, None, None, 0, None) == -1   # no rvec
     assert L.sobek_conv_geo_bwd(plan.handle, ctypes.byref(g1), None, 5, 1.0, 6, None, None, None, None, None, None, None, 0, None) == -1
     assert L.sobek_conv_geo_dbwd(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, *([None] * 10), 0, None) == -1
+    assert L.sobek_conv_geo_dbwd_full(None, ctypes.byref(g1), None, 0, 1.0, 6, *([None] * 11), 0, None) == -1
+    assert L.sobek_conv_geo_dbwd_full(plan.handle, ctypes.byref(g1), None, 0, 1.0, 6, *([None] * 11), 0, None) == -1    # no rvec
+    assert L.sobek_geo_dbwd_full_workspace_bytes(None, 4, 8) == 0
 
 
 def test_uvu_plan_weight_counts_match_the_paper():
