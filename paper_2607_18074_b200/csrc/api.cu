@@ -198,7 +198,7 @@ cudaError_t mix_tc(const sobek_plan* p, const Direction& dir, int64_t n0, int64_
                                     nn * G.d_dst, G.c_dst, G.D, accumulate, 0, status, s, 1, 0, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    return gemm_tc_flush(gb, s);
+    return gemm_tc_flush(gb, s, p);
 }
 
 // Zbar_g = gy_g * Rp_g^T       (Eq. receiver_adjoint)
@@ -223,7 +223,7 @@ cudaError_t state_adjoint_tc(const sobek_plan* p, const Direction& dir, int64_t 
                             p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    return gemm_tc_flush(gb, s);
+    return gemm_tc_flush(gb, s, p);
 }
 
 // gRp_g += Z_g^T * gy_g        (Eq. receiver_adjoint).  The contraction runs over every (node, component)
@@ -244,7 +244,7 @@ cudaError_t weight_grad_tc(const sobek_plan* p, const Direction& dir, int64_t nn
                                     sp, KN, nullptr, nullptr, p->gemm_passes);
         if (e != cudaSuccess) return e;
     }
-    cudaError_t e = gemm_tc_flush(gb, s0);
+    cudaError_t e = gemm_tc_flush(gb, s0, p);
     if (e != cudaSuccess) return e;
     // the pieces of every group, summed in a fixed order: one launch over the groups' column ranges
     ReduceRange rr[kMaxReduceRanges];

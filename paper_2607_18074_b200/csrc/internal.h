@@ -463,7 +463,8 @@ cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t
                         int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                         int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits,
                         int64_t split_stride, void* Chi, void* Clo, int passes);
-cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s);
+// p: the plan whose side streams carry the products when they are launched one by one (NULL: all on s)
+cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s, const sobek_plan* p);
 cudaError_t launch_gemm_tc(const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
                            int64_t ldb, float* C, int64_t c_outer, int64_t c_inner, int c_d, int64_t M, int64_t N,
                            int64_t Kd, int accumulate, int mn_major, int* status, cudaStream_t s, int splits = 1,
