@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <new>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -56,7 +57,7 @@ struct TcArgs {
 // One launch runs up to TC_MAX_BATCH independent products (the output groups of one node-side step): the CTAs
 // tile0[b] .. tile0[b+1]-1 belong to product b and number its (m tile, n tile, split) triples.
 constexpr int TC_MAX_BATCH = 5;
-constexpr unsigned kBatchTileLimit = 592;      // two CTAs on each of 148 SMs, twice over
+constexpr unsigned kSmallQueueTiles = 592;     // two CTAs on each of 148 SMs, twice over
 struct alignas(64) TcProblem {
     CUtensorMap tmAh, tmAl, tmBh, tmBl;
     TcArgs g;
@@ -490,11 +491,8 @@ cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t
     if (M <= 0 || N <= 0 || Kd <= 0) return cudaSuccess;
     if (M >= (int64_t(1) << 32)) return cudaErrorInvalidValue;   // the epilogue maps rows with 32-bit divisions
     TcBatch& B = *reinterpret_cast<TcBatch*>(gb.storage);
-    if (gb.n == TC_MAX_BATCH) {
-        cudaError_t e = gemm_tc_flush(gb, s, nullptr);
-        if (e != cudaSuccess) return e;
-    }
-    TcProblem& pr = B.p[gb.n];
+    TcProblem fresh;
+    TcProblem& pr = fresh;
     TcArgs& g = pr.g;
     g = TcArgs{};
     g.C = C; g.Ch = (__nv_bfloat16*)Chi; g.Cl = (__nv_bfloat16*)Clo; g.c_outer = c_outer; g.c_inner = c_inner; g.c_d = c_d; g.accumulate = accumulate; g.passes = passes == 1 ? 1 : 3;
@@ -529,58 +527,86 @@ cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t
     pr.gx = (uint32_t)((M + BM - 1) / BM);
     pr.gy = (uint32_t)((N + BN - 1) / BN);
     const uint64_t tiles = (uint64_t)pr.gx * pr.gy * (uint64_t)g.splits;
+    const size_t sh = (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16;
+    if (gb.n > 0 && (gb.n == TC_MAX_BATCH || tiles + B.tile0[gb.n] >= (uint64_t(1) << 31))) {
+        cudaError_t e = gemm_tc_flush(gb, s, nullptr);
+        if (e != cudaSuccess) return e;
+    }
+    if (tiles >= (uint64_t(1) << 31)) return cudaErrorInvalidValue;
     if (gb.n == 0) B.tile0[0] = 0;
-    if (tiles + B.tile0[gb.n] >= (uint64_t(1) << 31)) return cudaErrorInvalidValue;
+    B.p[gb.n] = fresh;
     B.tile0[gb.n + 1] = B.tile0[gb.n] + (uint32_t)tiles;
-    gb.sh = std::max(gb.sh, (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16);
+    gb.sh = std::max(gb.sh, sh);
+    gb.sh_of[gb.n] = sh;
     ++gb.n;
     return cudaSuccess;
 }
 
+namespace {
+// one launch over the products q[0..n) of B (indices into B.p), in that order
+void launch_sub(const TcBatch& B, const int* q, int n, size_t sh, cudaStream_t s) {
+    TcBatch sub;
+    sub.n = n;
+    sub.tile0[0] = 0;
+    for (int i = 0; i < n; ++i) {
+        sub.p[i] = B.p[q[i]];
+        sub.tile0[i + 1] = sub.tile0[i] + sub.p[i].gx * sub.p[i].gy * (uint32_t)sub.p[i].g.splits;
+    }
+    KernelTimer kt(K_GEMM, s);
+    k_gemm_tc<<<sub.tile0[n], TC_THREADS, sh, s>>>(sub);
+    count_launch();
+}
+}  // namespace
+
+// One launch has one shared-memory size, the largest of its products, so a product that fits three CTAs on an SM runs
+// one per SM beside a product that needs the whole SM (measured on the 64-channel profile, whose l = 0 block has 128
+// channels: 30,872 single-k-block tiles took 1.57 ms in one launch with the 197 KB of the widest product against
+// 0.75 ms in three launches).  Hence: a queue of at most kSmallQueueTiles tiles cannot fill the GPU anyway and runs as
+// one launch (what counts there is the number of launches); a larger queue runs one launch per class of products with
+// the same number of CTAs per SM, the classes side by side on the plan's side streams where a plan is given.
 cudaError_t gemm_tc_flush(GemmBatch& gb, cudaStream_t s, const sobek_plan* p) {
     if (gb.n == 0) return cudaSuccess;
     TcBatch& B = *reinterpret_cast<TcBatch*>(gb.storage);
-    B.n = gb.n;
-    // longest contraction first: the CTAs that run longest start first, the short ones fill the tail
-    std::stable_sort(B.p, B.p + gb.n, [](const TcProblem& x, const TcProblem& y) {
-        return (x.g.Kd + x.g.splits - 1) / x.g.splits > (y.g.Kd + y.g.splits - 1) / y.g.splits;
-    });
-    B.tile0[0] = 0;
-    for (int i = 0; i < gb.n; ++i) B.tile0[i + 1] = B.tile0[i] + B.p[i].gx * B.p[i].gy * (uint32_t)B.p[i].g.splits;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    const unsigned grid = B.tile0[gb.n];
-    if (gb.n > 1 && grid > kBatchTileLimit) {
-        // Products that fill the GPU on their own run faster one launch each (measured: a queue of 30,872 single-k-block
-        // tiles took 1.57 ms in one launch against 0.75 ms in three); only the small ones gain from sharing a launch.
-        auto launch_one = [&](int i, cudaStream_t si) {
-            TcBatch one;
-            one.p[0] = B.p[i];
-            one.n = 1;
-            one.tile0[0] = 0;
-            one.tile0[1] = B.tile0[i + 1] - B.tile0[i];
-            const TcArgs& g = one.p[0].g;
-            const size_t sh = (size_t)g.ring_bytes + 1024 + 8 * (2 * g.stages + 1) + 16;
-            KernelTimer kt(K_GEMM, si);
-            k_gemm_tc<<<one.tile0[1], TC_THREADS, sh, si>>>(one);
-            count_launch();
-        };
-        if (p) {        // on the plan's side streams: the launches overlap each other's tails
-            Fork fork(p, s);
-            for (int i = 0; i < gb.n; ++i) launch_one(i, fork.pick());
-            const cudaError_t e = fork.join();
-            if (e != cudaSuccess) return e;
-        } else {
-            for (int i = 0; i < gb.n; ++i) launch_one(i, s);
-        }
+    // longest contraction first: the CTAs that run longest start first, the short ones fill the tail
+    int order[TC_MAX_BATCH];
+    for (int i = 0; i < gb.n; ++i) order[i] = i;
+    auto len = [&](int i) { return (B.p[i].g.Kd + B.p[i].g.splits - 1) / B.p[i].g.splits; };
+    std::stable_sort(order, order + gb.n, [&](int x, int y) { return len(x) > len(y); });
+    auto per_sm = [](size_t bytes) { return (int)std::min<size_t>(8, (size_t)(227 * 1024) / std::max<size_t>(bytes, 1)); };
+    bool one_class = true;
+    for (int i = 1; i < gb.n; ++i) one_class = one_class && per_sm(gb.sh_of[i]) == per_sm(gb.sh_of[0]);
+    if (one_class || B.tile0[gb.n] <= kSmallQueueTiles) {
+        launch_sub(B, order, gb.n, gb.sh, s);
     } else {
-        KernelTimer kt(K_GEMM, s);
-        k_gemm_tc<<<grid, TC_THREADS, gb.sh, s>>>(B);
-        count_launch();
+        bool done[TC_MAX_BATCH] = {};
+        int n_class = 0;
+        cudaError_t err = cudaSuccess;
+        {
+            // (a Fork only where there is a plan to take side streams from)
+            Fork* fork = nullptr;
+            alignas(Fork) unsigned char fork_mem[sizeof(Fork)];
+            if (p) fork = new (fork_mem) Fork(p, s);
+            for (int a = 0; a < gb.n; ++a) {
+                const int ia = order[a];
+                if (done[ia]) continue;
+                int q[TC_MAX_BATCH], nq = 0;
+                size_t sh = 0;
+                for (int b = a; b < gb.n; ++b) {
+                    const int ib = order[b];
+                    if (!done[ib] && per_sm(gb.sh_of[ib]) == per_sm(gb.sh_of[ia])) { q[nq++] = ib; done[ib] = true; sh = std::max(sh, gb.sh_of[ib]); }
+                }
+                launch_sub(B, q, nq, sh, fork ? fork->pick() : s);
+                ++n_class;
+            }
+            if (fork) { err = fork->join(); fork->~Fork(); }
+        }
+        if (err != cudaSuccess) return err;
     }
     gb.n = 0; gb.sh = 0;
     return cudaGetLastError();

@@ -456,7 +456,8 @@ cudaError_t launch_pack_R_bf16(const sobek_plan* p, const Direction& dir, int tr
 // tensor-map type
 struct GemmBatch {
     alignas(64) unsigned char storage[4096];
-    size_t sh = 0;      // dynamic shared memory the queued products need
+    size_t sh = 0;      // dynamic shared memory the queued products need (the largest)
+    size_t sh_of[8] = {};   // and each of them
     int n = 0;
 };
 cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t lda, const void* Bhi, const void* Blo,
