@@ -501,7 +501,7 @@ cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t
     int BN;
     const int num_kb = (int)((Kd + BK - 1) / BK);
     if (mn_major) BN = N <= 64 ? 64 : (N <= 128 ? 128 : 256);     // whole 64-wide boxes
-    else BN = (int)std::min<int64_t>(num_kb == 1 ? 128 : 256, (N + 15) / 16 * 16);   // a single k-block is all epilogue: narrower tiles, more CTAs
+    else BN = (int)std::min<int64_t>(num_kb <= 2 ? 128 : 256, (N + 15) / 16 * 16);   // one or two k-blocks are all epilogue: narrower tiles, more CTAs
     g.BN = BN;
     const size_t stage = 2 * (size_t)BM * BK * 2 + 2 * (size_t)BN * BK * 2;
     // two (or more) CTAs per SM where the ring fits twice (more loads and epilogues in flight per SM), else one
@@ -509,6 +509,9 @@ cudaError_t gemm_tc_add(GemmBatch& gb, const void* Ahi, const void* Alo, int64_t
     int stages = (int)std::min<size_t>(4, (108 * 1024) / stage);
     if (stages < 2) stages = (int)std::min<size_t>(4, (200 * 1024) / stage);
     stages = std::max(1, std::min(stages, (num_kb + g.splits - 1) / g.splits));
+    // one or two k-blocks per tile: the tile is all epilogue, and three CTAs per SM with a single stage each overlap
+    // their epilogues better than one CTA with a stage per k-block
+    if ((num_kb + g.splits - 1) / g.splits <= 2 && stage <= 72 * 1024) stages = 1;
     g.stages = stages;
     const size_t park = (size_t)4 * 32 * (BN + 4) * sizeof(float);       // epilogue staging of the four drain warps
     g.ring_bytes = (int32_t)((std::max(park, (size_t)stages * stage) + 1023) & ~size_t(1023));
