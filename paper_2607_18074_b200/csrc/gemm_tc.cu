@@ -562,8 +562,8 @@ void launch_sub(const TcBatch& B, const int* q, int n, size_t sh, cudaStream_t s
 }  // namespace
 
 // One launch has one shared-memory size, the largest of its products, so a product that fits three CTAs on an SM runs
-// one per SM beside a product that needs the whole SM (measured on the 64-channel profile, whose l = 0 block has 128
-// channels: 30,872 single-k-block tiles took 1.57 ms in one launch with the 197 KB of the widest product against
+// one per SM beside a product that needs the whole SM (measured on the profile 128x0e + 64x1o + 64x2e:
+// 30,872 single-k-block tiles took 1.57 ms in one launch with the 197 KB of the widest product against
 // 0.75 ms in three launches).  Hence: a queue of at most kSmallQueueTiles tiles cannot fill the GPU anyway and runs as
 // one launch (what counts there is the number of launches); a larger queue runs one launch per class of products with
 // the same number of CTAs per SM, the classes side by side on the plan's side streams where a plan is given.
