@@ -75,7 +75,7 @@ k_gemm_tc(const __grid_constant__ TcBatch B) {
     int bi = 0;
     while (bi + 1 < B.n && blockIdx.x >= B.tile0[bi + 1]) ++bi;
     const TcProblem& pr = B.p[bi];
-    const TcArgs& g = pr.g;
+    const TcArgs g = pr.g;        // by value: read once (the product is picked by a run-time index into the parameter)
     const CUtensorMap& tmAh = pr.tmAh;
     const CUtensorMap& tmAl = pr.tmAl;
     const CUtensorMap& tmBh = pr.tmBh;
