@@ -77,7 +77,7 @@ def test_state_widths():
 
 def test_workspace_does_not_grow_with_edges():
     w = synth.config("cfg4")
-    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, state_budget_mib=2048)      # (the default depends on the device)
     for order in (0, 1, 2):
         a = sb.workspace_bytes(plan, 3125, 10**5, order)
         assert a > 0
@@ -92,7 +92,7 @@ def test_workspace_does_not_grow_with_edges():
         assert sb.workspace_bytes(plan, 10**6, 10**8, order) - 10**6 * per_node < 4300 * 2**20
     # the widest benchmark contract: bounded by the state budget (or 512 nodes) plus the feature copies, whatever the edge count
     w = synth.config("cfg5")
-    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K)
+    plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, state_budget_mib=2048)
     a = sb.workspace_bytes(plan, 50000, 2 * 10**6, 2)
     assert a == sb.workspace_bytes(plan, 50000, 4 * 10**8, 2)
     assert a - 50000 * 4 * (2 * plan.info.C_x + plan.info.C_y) < 5400 * 2**20
