@@ -44,6 +44,7 @@ NCU_TRAFFIC_BYTES_PER_EDGE = {
     ("cfg5", "edge_stream_state"): (813.0e6 + 2087.1e6) / 90891.0,     # k_stream_tc, two launches
     ("cfg5", "edge_pass"): (255.4e6 + 13.4e6) / 90891.0,                # k_edge_tc, three launches
 }
+STATE_BUDGET_MIB = None         # --state-budget-mib: the plan's scratch budget (None = the library's default, 2048)
 STREAM_CALLS_PER_STEP = 7      # edge-stream passes over all edges per step: 1 fwd + 2 bwd + 4 dbwd
 
 
@@ -229,7 +230,7 @@ class Run:
 
     def __init__(self, sb, torch, dev, w, seed):
         self.sb, self.torch, self.dev, self.w = sb, torch, dev, w
-        self.plan = plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode)
+        self.plan = plan = sb.Plan(w.irreps_in, w.irreps_out, w.l_max, w.K, mode=w.mode, state_budget_mib=STATE_BUDGET_MIB)
         w.seed = seed
         self.d = d = synth.make_inputs(w, synth.plan_col_std(plan))
         self.info = i = plan.info
@@ -329,10 +330,14 @@ def main():
     ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="skip the table of the other configurations")
+    ap.add_argument("--state-budget-mib", type=int, default=0,
+                    help="scratch budget of the plan in MiB (0 = the library default, 2048); a throughput knob")
     ap.add_argument("--nodes", type=int, default=0,
                     help="run the workload's profile on a graph scaled to this many nodes (same density and degree): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    global STATE_BUDGET_MIB
+    STATE_BUDGET_MIB = args.state_budget_mib if args.state_budget_mib > 0 else None
     if args.impl == "reference":
         run_reference(args)
         return
@@ -567,6 +572,7 @@ def main():
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": w.name, "mode": w.mode, "N": N, "E": E, "K": i.K, "N_w": int(i.N_w), "C_x": i.C_x, "C_y": i.C_y,
+                   "state_budget_mib": STATE_BUDGET_MIB or 2048,
                    "l_max": i.l_max, "replicas": world, "l2": f"flushed before every order ({L2_FLUSH_BYTES >> 20} MiB write)",
                    "timing": "every step is one sample (CUDA events per order); ms_per_step and the per-order times are medians"},
         "ms_per_step_mean": step_ms_mean, "timed_ms_total": float(per.sum()),
