@@ -190,7 +190,8 @@ int sobek_graph_receivers(int64_t N, int64_t E, const int64_t* row_ptr, const in
  * re-laid-out copies of R, the bounded receiver/sender state of one node chunk (at most 2 GiB,
  * whatever the graph), a status word and, for the tensor-core edge kernels, bf16 (hi, lo)
  * copies of the node features they gather from (4 bytes per feature of x, and of gy / vx for
- * orders 1 / 2).  It depends on the plan and on N only -- never on E.
+ * orders 1 / 2) and the processing order of the nodes of every chunk (16 bytes per node and graph view).
+ * It depends on the plan and on N only -- never on E.
  * The pointer passed as `ws` must be 256-byte aligned.
  */
 size_t sobek_workspace_bytes(const sobek_plan* plan, int64_t N, int64_t E, int order);

@@ -29,11 +29,15 @@ struct Workspace {
     // bf16 (hi, lo) copies of x, gy and vx, [N][C] each: the gathered operand of the tensor-core stream
     uint16_t *xsh, *xsl, *gsh, *gsl, *vsh, *vsl;
     uint16_t *zqh, *zql;      // bf16 (hi, lo) adjoint state of one chunk (input of the tensor-core edge pass)
+    int4 *oseg_r, *oseg_s;    // processing order of the nodes of every chunk, receiver / sender view (launch_chunk_order)
     // mul_ir plans: ir_mul copies of the node feature arrays of a call (inputs x, gy, vx; outputs on C_y, on C_x)
     float *lx, *lgy, *lvx, *ly, *lgx;
     int64_t chunk;
     size_t bytes;
 };
+
+constexpr int64_t kOrderMinChunk = 4 * 148;   // nodes per chunk from which the processing order is balanced
+constexpr int kOrderPeriod = 148;             // persistent CTAs of the edge kernels (one per SM)
 
 Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
     Workspace w{};
@@ -97,6 +101,11 @@ Workspace carve(const sobek_plan* p, int64_t N, int order, void* ws) {
         if (p->fwd.tc[0].ok || (order >= 2 && p->fwd.tc[1].ok) || (order >= 1 && w.zqh)) { w.xsh = (uint16_t*)take(nx); w.xsl = (uint16_t*)take(nx); }
         if (order >= 1 && (p->tr.tc[0].ok || (order >= 2 && p->tr.tc[1].ok))) { w.gsh = (uint16_t*)take(ny); w.gsl = (uint16_t*)take(ny); }
         if (order >= 2 && (p->fwd.tc[1].ok || (w.zqh && p->fwd.etc[1].ok))) { w.vsh = (uint16_t*)take(nx); w.vsl = (uint16_t*)take(nx); }
+        // load balance of the persistent edge kernels: only where a CTA takes several nodes of a chunk
+        if (w.chunk >= kOrderMinChunk && N >= kOrderMinChunk) {
+            w.oseg_r = (int4*)take((size_t)N * sizeof(int4));
+            if (order >= 1) w.oseg_s = (int4*)take((size_t)N * sizeof(int4));
+        }
     }
     if (p->mul_ir) {
         const size_t nx = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_x * 4, ny = (size_t)std::max<int64_t>(N, 0) * (size_t)p->C_y * 4;
@@ -360,6 +369,7 @@ int conv_fwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
     CK(pack_R(p, p->fwd, 0, 1, R, w.fNKh, w.fNKl, s));
     SplitSrc xs{};
     if (geo) xs = *geo;
+    if (w.oseg_r) { CK(launch_chunk_order(rv, w.chunk, kOrderPeriod, w.oseg_r, w.status, s)); xs.oseg = w.oseg_r; }
     if (w.xsh) { CK(split_features(x, g->N, p->C_x, w.xsh, w.xsl, s)); xs.h = w.xsh; xs.l = w.xsl; }
     for (int64_t n0 = 0; n0 < g->N; n0 += w.chunk) {
         const int64_t nn = std::min(w.chunk, g->N - n0);
@@ -404,6 +414,11 @@ int conv_bwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, con
         CK(launch_uvu_direct_wgrad(p, rv, x, Y, phi, gy, w.part, w.splits, &n_parts, w.status, s));
         CK(launch_reduce_parts(gR, w.part, KN, KN, n_parts, s));
         gR = nullptr;
+    }
+    if (w.oseg_r && (gR || gphi || gY)) { CK(launch_chunk_order(rv, w.chunk, kOrderPeriod, w.oseg_r, w.status, s)); xs.oseg = w.oseg_r; }
+    if (w.oseg_s && gx && !gx_direct && !w.fused_t) {
+        CK(launch_chunk_order(sender_view(g), w.chunk, kOrderPeriod, w.oseg_s, w.status, s));
+        gs.oseg = w.oseg_s;
     }
     FeatureSplits fs;
     if (w.xsh && (gR || ((gphi || gY) && tc_edge))) { fs.add(x, g->N, p->C_x, w.xsh, w.xsl); xs.h = w.xsh; xs.l = w.xsl; }
@@ -501,6 +516,11 @@ int conv_dbwd_core(const sobek_plan* p, const sobek_graph* g, const float* x, co
     SplitSrc xs{}, gs{};
     if (geo) { xs = *geo; gs = *geo; }
     const bool tc_edge_plain = w.zqh != nullptr, tc_edge_dual = tc_edge_plain && p->fwd.etc[1].ok && (!vx || w.vsh);
+    if (w.oseg_r && (ggy || hR || hphi || hY)) { CK(launch_chunk_order(rv, w.chunk, kOrderPeriod, w.oseg_r, w.status, s)); xs.oseg = w.oseg_r; }
+    if (w.oseg_s && hx && !w.fused_t) {
+        CK(launch_chunk_order(sender_view(g), w.chunk, kOrderPeriod, w.oseg_s, w.status, s));
+        gs.oseg = w.oseg_s;
+    }
     FeatureSplits fs;
     if (w.xsh && (ggy || hR || ((hphi || hY) && tc_edge_plain))) {
         fs.add(x, g->N, p->C_x, w.xsh, w.xsl); xs.h = w.xsh; xs.l = w.xsl;

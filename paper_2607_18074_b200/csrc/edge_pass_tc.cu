@@ -56,6 +56,7 @@ struct EtArgs {
     const int64_t* row_ptr;
     const int32_t* col;
     int64_t node0, n_nodes;
+    const int4* oseg;           // the chunk's nodes in processing order {local node, segment begin, end} or NULL
     int64_t N, E;               // sizes of the graph: every gathered id and segment bound is checked against them
     const __nv_bfloat16* sh;
     const __nv_bfloat16* sl;
@@ -134,6 +135,13 @@ __host__ __device__ inline int raw_floats(int KP, bool dual, int dsh, int tb) {
 }
 
 // GEO: the geometry mode (edge inputs recomputed from edge vectors, adjoint of the edge vectors out); plain pass only
+// segment of the node at position v of the chunk's processing order; returns the node's local index
+__device__ __forceinline__ int64_t et_bounds(const EtArgs& a, int64_t v, int* status, int64_t& s0, int64_t& s1) {
+    if (a.oseg) { const int4 q = __ldg(a.oseg + v); s0 = q.y; s1 = q.z; return q.x; }
+    seg_bounds(a.row_ptr, a.node0 + v, a.E, status, s0, s1);
+    return v;
+}
+
 template <int KP, bool DUAL, int NCW, int NLW, bool GEO, int MINB>
 __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const EtArgs a) {
     constexpr int TT = (NCW + NLW + 1) * 32;
@@ -236,9 +244,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
         // =========================== loader warps ===========================
         const int lt = (warp - NCW) * 32 + lane;
         uint32_t it = 0, zi = 0;
-        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+        for (int64_t v = blockIdx.x; v < a.n_nodes; v += gridDim.x) {
             int64_t seg0, seg1;
-            seg_bounds(a.row_ptr, a.node0 + nl, a.E, a.status, seg0, seg1);
+            const int64_t nl = et_bounds(a, v, a.status, seg0, seg1);
             if (!any_op) seg1 = seg0;
             if (seg1 <= seg0) continue;
             // ---- Zbar slabs, unit by unit (each once the previous receiver's MMAs of that unit have read theirs);
@@ -355,9 +363,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
         // =========================== geometry warp ===========================
         // walks the same receivers and batches as the loaders; lane <-> (edge, share of the radial indices and components)
         uint32_t it = 0;
-        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+        for (int64_t v = blockIdx.x; v < a.n_nodes; v += gridDim.x) {
             int64_t seg0, seg1;
-            seg_bounds(a.row_ptr, a.node0 + nl, a.E, nullptr, seg0, seg1);
+            et_bounds(a, v, nullptr, seg0, seg1);
             if (!any_op) seg1 = seg0;
             for (int64_t b0 = seg0; b0 < seg1; b0 += tb, ++it) {
                 const int nb = (int)min((int64_t)tb, seg1 - b0);
@@ -390,9 +398,9 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
         if (lane == 0) {
             uint32_t it = 0, zi = 0, ai = 0;
             const uint32_t sZ_u = smem_u32(sZ);
-            for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+            for (int64_t v = blockIdx.x; v < a.n_nodes; v += gridDim.x) {
                 int64_t seg0, seg1;
-                seg_bounds(a.row_ptr, a.node0 + nl, a.E, nullptr, seg0, seg1);
+                et_bounds(a, v, nullptr, seg0, seg1);
                 if (!any_op) seg1 = seg0;
                 if (seg1 <= seg0) continue;
                 for (int64_t b0 = seg0; b0 < seg1; b0 += tb)
@@ -443,10 +451,10 @@ __global__ void __launch_bounds__((NCW + NLW + 1) * 32, MINB) k_edge_tc(const Et
         const int GW = KP + a.dsh;                   // row pitch of sGeo
         // bounds of the next receiver, requested one receiver ahead
         int64_t nx0 = 0, nx1 = 0;
-        if ((int64_t)blockIdx.x < a.n_nodes) seg_bounds(a.row_ptr, a.node0 + blockIdx.x, a.E, nullptr, nx0, nx1);
-        for (int64_t nl = blockIdx.x; nl < a.n_nodes; nl += gridDim.x) {
+        if ((int64_t)blockIdx.x < a.n_nodes) et_bounds(a, blockIdx.x, nullptr, nx0, nx1);
+        for (int64_t v = blockIdx.x; v < a.n_nodes; v += gridDim.x) {
             const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
-            if (nl + gridDim.x < a.n_nodes) seg_bounds(a.row_ptr, a.node0 + nl + gridDim.x, a.E, nullptr, nx0, nx1);
+            if (v + gridDim.x < a.n_nodes) et_bounds(a, v + gridDim.x, nullptr, nx0, nx1);
             {
                 for (int64_t b0 = seg0; b0 < seg1; b0 += tb) {
                     const int nb = (int)min((int64_t)tb, seg1 - b0);     // edges of the batch
@@ -854,6 +862,7 @@ cudaError_t launch_edge_pass_tc(const sobek_plan* p, const Direction& dir, const
     a.zqh = (const __nv_bfloat16*)zqh; a.zql = (const __nv_bfloat16*)zql;
     a.gphi = gphi; a.gY = gY;
     a.rvec = ss.rvec; a.g_rvec = ss.g_rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p;
+    a.oseg = ss.oseg ? ss.oseg + node0 : nullptr;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src;
     a.status = status;
     const bool k8 = p->K <= 8;

@@ -2,6 +2,7 @@
 // sender-sorted view (src_ptr, src_perm).  Integer work only; the result is unique
 // (edges of one sender appear in increasing edge id), so it does not depend on the order
 // in which threads run even though the placement step uses integer atomics.
+#include "guard.cuh"
 #include "internal.h"
 
 namespace sobek {
@@ -246,6 +247,66 @@ int position_gradient(const sobek_graph* g, const float* g_rvec, float* gpos, cu
     k_position_gradient<<<grid, 128, 0, s>>>(g->N, g->E, g->row_ptr, g->src_ptr, g->src_perm, g_rvec, gpos);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? SOBEK_OK : SOBEK_ERR_CUDA;
+}
+
+// ---- processing order of the nodes of a chunk (load balance of the persistent edge kernels) -------------------------
+namespace {
+constexpr int ORD_BINS = 2048;
+__global__ void __launch_bounds__(1024) k_chunk_order(const int64_t* __restrict__ ptr, int64_t N, int64_t E, int64_t chunk,
+                                                      int period, int4* __restrict__ oseg, int* status) {
+    __shared__ int hist[ORD_BINS];
+    __shared__ int wsum[32];
+    const int64_t n0 = (int64_t)blockIdx.x * chunk;
+    const int64_t nn = min(chunk, N - n0);
+    for (int i = threadIdx.x; i < ORD_BINS; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    // bucket = ORD_BINS - 1 - min(length, ORD_BINS - 1): longest segments first
+    for (int64_t i = threadIdx.x; i < nn; i += blockDim.x) {
+        int64_t s0, s1;
+        seg_bounds(ptr, n0 + i, E, status, s0, s1);
+        atomicAdd(&hist[ORD_BINS - 1 - (int)min(s1 - s0, (int64_t)(ORD_BINS - 1))], 1);
+    }
+    __syncthreads();
+    // exclusive scan of the histogram: two bins per thread, warp scans, then the warp totals
+    {
+        const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+        const int a0 = hist[2 * t], a1 = hist[2 * t + 1];
+        int v = a0 + a1;
+        for (int d = 1; d < 32; d <<= 1) { const int u = __shfl_up_sync(0xffffffffu, v, d); if (lane >= d) v += u; }
+        if (lane == 31) wsum[w] = v;
+        __syncthreads();
+        if (w == 0) {
+            int x = wsum[lane];
+            for (int d = 1; d < 32; d <<= 1) { const int u = __shfl_up_sync(0xffffffffu, x, d); if (lane >= d) x += u; }
+            wsum[lane] = x;
+        }
+        __syncthreads();
+        const int base = (w > 0 ? wsum[w - 1] : 0) + v - (a0 + a1);
+        hist[2 * t] = base;
+        hist[2 * t + 1] = base + a0;
+    }
+    __syncthreads();
+    const int64_t full = (nn / period) * period;       // entries in whole rounds
+    for (int64_t i = threadIdx.x; i < nn; i += blockDim.x) {
+        int64_t s0, s1;
+        seg_bounds(ptr, n0 + i, E, nullptr, s0, s1);
+        const int64_t r = atomicAdd(&hist[ORD_BINS - 1 - (int)min(s1 - s0, (int64_t)(ORD_BINS - 1))], 1);
+        int64_t v = r;
+        if (r < full) {                                  // every second whole round runs backwards
+            const int64_t round = r / period, k = r - round * period;
+            if (round & 1) v = round * period + (period - 1 - k);
+        }
+        oseg[n0 + v] = make_int4((int)i, (int)s0, (int)s1, 0);
+    }
+}
+}  // namespace
+
+cudaError_t launch_chunk_order(const EdgeView& ev, int64_t chunk, int period, int4* oseg, int* status, cudaStream_t s) {
+    if (ev.N <= 0 || chunk <= 0 || !oseg) return cudaSuccess;
+    const int64_t n_chunks = (ev.N + chunk - 1) / chunk;
+    k_chunk_order<<<(unsigned)n_chunks, 1024, 0, s>>>(ev.ptr, ev.N, ev.E, chunk, period, oseg, status);
+    count_launch();
+    return cudaGetLastError();
 }
 
 }  // namespace sobek

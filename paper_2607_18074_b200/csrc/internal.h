@@ -355,6 +355,9 @@ struct SplitSrc {
     int geo_basis = 0, geo_p = 6;
     float* g_rvec = nullptr;
     const float* vrvec = nullptr;     // double backward: direction on the edge vectors (dual stream passes only)
+    // load balance of the tensor-core edge kernels: [N] entries {local node, segment begin, segment end, 0}, the nodes of
+    // every chunk in the order its persistent CTAs take them (launch_chunk_order); NULL: index order
+    const int4* oseg = nullptr;
 };
 cudaError_t launch_stream(const sobek_plan* p, const Direction& dir, const EdgeView& ev, int64_t node0,
                           int64_t n_nodes, const float* src, const float* vsrc, const SplitSrc& ss, const float* Y,
@@ -486,6 +489,9 @@ cudaError_t launch_geo_edge_inputs(const float* rvec, const float* vrvec, int64_
 cudaError_t launch_geo_second_adjoint(const float* rvec, const float* vrvec, int64_t E, int l_max, int K, float r_c, int basis,
                                       int p, const float* gY, const float* gphi, const float* hY, const float* hphi,
                                       float* h_rvec, cudaStream_t s);
+// For every chunk of `chunk` nodes of the view: its nodes sorted by segment length, longest first, dealt in rounds of
+// `period` that alternate direction, so that CTAs taking the entries round-robin get equal shares of the edges.
+cudaError_t launch_chunk_order(const EdgeView& ev, int64_t chunk, int period, int4* oseg, int* status, cudaStream_t s);
 // --- uvu_direct.cu ------------------------------------------------------------------------
 void build_uvu_direct(sobek_plan* p, const sobek_irrep* in, int n_in, const sobek_irrep* out, int n_out);
 // transposed = 0: y[N, C_y] from src = x on the receiver view; 1: gx[N, C_x] from src = gy on the sender view

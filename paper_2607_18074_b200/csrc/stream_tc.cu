@@ -80,6 +80,7 @@ struct TcArgs {
     const CompS* comps;
     EdgeView ev;
     int64_t node0, n_nodes;
+    const int4* oseg;           // the chunk's nodes in processing order {local node, segment begin, end} or NULL
     const __nv_bfloat16* sh;    // bf16 hi / lo copies of the source features [N][C_src]
     const __nv_bfloat16* sl;
     const __nv_bfloat16* vsh;   // DUAL: the same for the source direction; NULL without it
@@ -276,6 +277,12 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
         __device__ void init(int64_t item, int64_t n) { nl = item % n; set = (int)(item / n); }
         __device__ void step(int64_t by, int64_t n) { nl += by; while (nl >= n) { nl -= n; ++set; } }
     };
+    // segment of the node at position v of the chunk's processing order; returns the node's local index
+    auto item_bounds = [&](int64_t v, int* status, int64_t& s0, int64_t& s1) -> int64_t {
+        if (a.oseg) { const int4 q = __ldg(a.oseg + v); s0 = q.y; s1 = q.z; return q.x; }
+        seg_bounds(a.ev.ptr, a.node0 + v, a.ev.E, status, s0, s1);
+        return v;
+    };
 
     if (warp >= W_LOAD && warp < W_LOAD + NLW) {
         // =========================== loader warps ===========================
@@ -287,7 +294,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
         ItemPos lp; lp.init(p_item, a.n_nodes);
         auto prefetch_item = [&]() {
             if (p_item < total) {
-                seg_bounds(a.ev.ptr, a.node0 + lp.nl, a.ev.E, a.status, p_seg0, p_seg1);
+                item_bounds(lp.nl, a.status, p_seg0, p_seg1);
                 if (!any_op) p_seg1 = p_seg0;
             }
         };
@@ -441,7 +448,7 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             ItemPos lp; lp.init(p_item, a.n_nodes);
             auto prefetch_item = [&]() {
                 if (p_item < total) {
-                    seg_bounds(a.ev.ptr, a.node0 + lp.nl, a.ev.E, nullptr, p_seg0, p_seg1);
+                    item_bounds(lp.nl, nullptr, p_seg0, p_seg1);
                     if (!any_op) p_seg1 = p_seg0;
                 }
             };
@@ -512,14 +519,14 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
             int st = 0; uint32_t round = 0;
             int64_t nx0 = 0, nx1 = 0;
             ItemPos mp; mp.init(blockIdx.x, a.n_nodes);      // position of the item whose bounds are in flight
-            if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
+            if ((int64_t)blockIdx.x < total) item_bounds(mp.nl, nullptr, nx0, nx1);
             const uint64_t bcap16 = (uint64_t)(a.b_cap >> 4);
             for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
                 const TSet S = sSet[mp.set];
                 const int64_t seg0 = nx0, seg1 = any_op ? nx1 : nx0;
                 mp.step(gridDim.x, a.n_nodes);
                 if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
-                    seg_bounds(a.ev.ptr, a.node0 + mp.nl, a.ev.E, nullptr, nx0, nx1);
+                    item_bounds(mp.nl, nullptr, nx0, nx1);
                 if (seg1 <= seg0) continue;
                 const uint32_t buf = a.nbuf == 2 ? (mi & 1) : 0u, gen = a.nbuf == 2 ? (mi >> 1) : mi;    // buffer and its use count
                 if (mi >= (uint32_t)a.nbuf) mbar_wait(bar_accfree + 8 * buf, (gen & 1) ^ 1, a.status);
@@ -571,13 +578,14 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
         uint32_t mi = 0;
         int64_t dx0 = 0, dx1 = 0;
         ItemPos dp; dp.init(blockIdx.x, a.n_nodes);
-        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + dp.nl, a.ev.E, nullptr, dx0, dx1);
+        int64_t dnl = 0;                 // local index of the node whose bounds are in flight
+        if ((int64_t)blockIdx.x < total) dnl = item_bounds(dp.nl, nullptr, dx0, dx1);
         for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
-            const int64_t nl = dp.nl;
+            const int64_t nl = dnl;
             const TSet S = sSet[dp.set];
             const int64_t seg0 = dx0, seg1 = any_op ? dx1 : dx0;
             dp.step(gridDim.x, a.n_nodes);
-            if (item + gridDim.x < total) seg_bounds(a.ev.ptr, a.node0 + dp.nl, a.ev.E, nullptr, dx0, dx1);
+            if (item + gridDim.x < total) dnl = item_bounds(dp.nl, nullptr, dx0, dx1);
             const bool wrote = seg1 > seg0;      // a node without edges has a state of zeros
             const uint32_t buf = a.nbuf == 2 ? (mi & 1) : 0u, gen = a.nbuf == 2 ? (mi >> 1) : mi;
             if (wrote) {
@@ -658,14 +666,14 @@ __global__ void __launch_bounds__(TT, 1) k_stream_tc(const TcArgs a) {
         int cur_set = -1;
         int64_t cx0 = 0, cx1 = 0;
         ItemPos cp_; cp_.init(blockIdx.x, a.n_nodes);        // position of the item whose bounds are in flight
-        if ((int64_t)blockIdx.x < total) seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
+        if ((int64_t)blockIdx.x < total) item_bounds(cp_.nl, nullptr, cx0, cx1);
         for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
             const int set = cp_.set;
             const TSet S = sSet[set];
             const int64_t seg0 = cx0, seg1 = any_op ? cx1 : cx0;
             cp_.step(gridDim.x, a.n_nodes);
             if (item + gridDim.x < total)       // the next item's bounds, requested one item ahead
-                seg_bounds(a.ev.ptr, a.node0 + cp_.nl, a.ev.E, nullptr, cx0, cx1);
+                item_bounds(cp_.nl, nullptr, cx0, cx1);
             if (set != cur_set && seg1 > seg0) {     // entry and sparse-term tables of the set
                 builder_sync();
                 for (int i = tid; i < S.nent; i += NBW * 32) sEnt[i] = a.ents[S.ent_begin + i];
@@ -1000,6 +1008,7 @@ cudaError_t launch_stream_tc(const sobek_plan* p, const Direction& dir, const Ed
     a.vsh = (const __nv_bfloat16*)ss.vh; a.vsl = (const __nv_bfloat16*)ss.vl;
     a.Y = Y; a.vY = vY; a.phi = phi; a.vphi = vphi;
     a.rvec = ss.rvec; a.geo_rc = ss.geo_rc; a.geo_basis = ss.geo_basis; a.geo_p = ss.geo_p; a.geo_inline = 0;
+    a.oseg = ss.oseg ? ss.oseg + node0 : nullptr;
     a.vrvec = dual ? ss.vrvec : nullptr;
     a.zh = (__nv_bfloat16*)zh; a.zl = (__nv_bfloat16*)zl;
     a.K = p->K; a.dsh = p->dim_sh; a.C_src = dir.C_src; a.nsets = (int)T.sets.size();

@@ -87,6 +87,7 @@ def test_workspace_does_not_grow_with_edges():
         # copy of the node features that the tensor-core stream gathers from (4 bytes per feature)
         C_x, C_y = plan.info.C_x, plan.info.C_y
         per_node = 4 * (C_x + (C_y if order >= 1 else 0) + (C_x if order >= 2 else 0))
+        per_node += 16 * (1 if order == 0 else 2)      # and the chunks' processing order of each view (one int4 per node)
         grow = sb.workspace_bytes(plan, 3 * 10**6, 10**8, order) - sb.workspace_bytes(plan, 10**6, 10**8, order)
         assert abs(grow - 2 * 10**6 * per_node) < 4096
         assert sb.workspace_bytes(plan, 10**6, 10**8, order) - 10**6 * per_node < 4300 * 2**20
