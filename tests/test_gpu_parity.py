@@ -436,6 +436,20 @@ def test_scaling_axes_sampled(name):
         del FULL[name]
 
 
+def test_balanced_processing_order():
+    """From 592 nodes per chunk on, the tensor-core edge kernels take the nodes of a chunk longest neighbourhood first
+    in alternating rounds (a per-chunk counting sort of the degrees) instead of by index: every output of every order
+    against the oracle on a graph large enough for that, with hubs, isolated nodes and several chunks."""
+    w = synth.scaled(synth.config("cfg2"), 1500)
+    c = Case(w, state_budget_mib=32)             # about 35 KB of state per node: two chunks of 750 to 1,100 nodes
+    assert rel_err(c.fwd(), c.o_fwd()) <= FWD_TOL
+    for got, ref, nm in zip(c.bwd(), c.o_bwd(), ("gx", "gY", "gphi", "gR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+    for got, ref, nm in zip(c.dbwd(), c.o_dbwd(), ("ggy", "hx", "hY", "hphi", "hR")):
+        assert rel_err(got, ref) <= BWD_TOL, nm
+    assert np.array_equal(c.fwd(), c.fwd())
+
+
 def test_scratch_budget():
     """The scratch budget (section "Runtime scratch-budget policy") only changes the chunking: with the
     paper's 128 MiB the workspace shrinks and every output still matches the oracle."""
