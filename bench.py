@@ -41,8 +41,8 @@ DTYPE = "f32 storage; products as split bf16 x3 (hi*hi + lo*hi + hi*lo) with f32
 # the state of the chunk written once (0.92 MB per node as bf16 hi + lo, i.e. 23 KB per edge at 40 edges per node)
 # plus the gathered sender rows.
 NCU_TRAFFIC_BYTES_PER_EDGE = {
-    ("cfg5", "edge_stream_state"): (813.0e6 + 2087.1e6) / 90891.0,     # k_stream_tc, two launches
-    ("cfg5", "edge_pass"): (255.4e6 + 13.4e6) / 90891.0,                # k_edge_tc, three launches
+    ("cfg5", "edge_stream_state"): (719.4e6 + 2082.7e6) / 90891.0,     # k_stream_tc, two launches
+    ("cfg5", "edge_pass"): (359.0e6 + 15.3e6) / 90891.0,                # k_edge_tc, three launches
 }
 STATE_BUDGET_MIB = None         # --state-budget-mib: the plan's scratch budget (None = the library's default, 2048)
 STREAM_CALLS_PER_STEP = 7      # edge-stream passes over all edges per step: 1 fwd + 2 bwd + 4 dbwd
