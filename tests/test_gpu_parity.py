@@ -21,6 +21,7 @@ def small_cases():
     c["cfg3_N120"] = synth.scaled(synth.config("cfg3"), 120)
     c["cfg4_N150"] = synth.scaled(synth.config("cfg4"), 150)
     c["cfg5_N60"] = synth.scaled(synth.config("cfg5"), 60)
+    c["cfg2_N700"] = synth.scaled(synth.config("cfg2"), 700)      # a chunk of 592 nodes or more: balanced processing order
     # ragged multiplicities, odd K, mixed parities (odd-sum paths), a block with no path
     c["ragged"] = synth.Workload("ragged", P("5x0e+3x1o+2x1e+33x2e"), P("7x0e+1x0o+35x1o+2x2e+3x3o+2x4e"),
                                  3, 3, 40, 4.0, 1.9, "gaussian", seed=3)
@@ -190,7 +191,7 @@ def test_errors_on_device_calls(cases):
     assert ei.value.code == -5
 
 
-@pytest.mark.parametrize("name,fp32_pipe", [("cfg1", False), ("cfg1", True), ("tc_K6_dense", False)])
+@pytest.mark.parametrize("name,fp32_pipe", [("cfg1", False), ("cfg1", True), ("tc_K6_dense", False), ("cfg2_N700", False)])
 def test_stale_graph_arrays_are_reported_not_followed(name, fp32_pipe):
     """The graph arrays are the caller's: an entry that is out of range when a kernel reads it (a freed or
     overwritten buffer) must end in SOBEK_ERR_GRAPH in the status word with finite outputs, never in an
